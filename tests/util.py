@@ -1,0 +1,32 @@
+"""Helpers shared by the tests: flat tensor list <-> the oracle's parameter containers."""
+import numpy as np
+
+from paper_2608_18469_b200 import synth
+
+
+def structure(spec, flat):
+    """Flat list (tensor-index order) -> {"input": {...}, "blocks": [{...}]} in float64."""
+    out = {"input": {}, "blocks": [dict() for _ in spec["blocks"]]}
+    for (b, name, _shape, _tr), v in zip(synth.tensor_list(spec), flat):
+        (out["input"] if b < 0 else out["blocks"][b])[name] = np.asarray(v, np.float64)
+    return out
+
+
+def flatten_blocks(spec, per_block):
+    """List of per-block dicts -> flat list over the trainable tensors, tensor-index order."""
+    return [per_block[b][name] for (b, name, _s, tr) in synth.tensor_list(spec) if tr]
+
+
+def trainable_index(spec):
+    return [i for i, (_b, _n, _s, tr) in enumerate(synth.tensor_list(spec)) if tr]
+
+
+def tiny_specs():
+    """One tiny instance per block kind (a few rows, a few columns), chain or parallel."""
+    s = {}
+    s["mlp_relu"] = synth.mlp_spec(4, 6, 2, 3, "relu", "f32")
+    s["mlp_gelu"] = synth.mlp_spec(4, 6, 3, 3, "gelu", "f32")
+    s["lm"] = synth.lm_spec(2, 4, 2, 6, 3, 2, 5, dtype="f32")
+    s["ctr"] = synth.ctr_spec(batch=3, n_dense=2, n_sparse=3, table_rows=7, emb_dim=4,
+                              tower=(6, 5, 4), n_cross=2, dtype="f32")
+    return s
