@@ -1,0 +1,220 @@
+/*
+ * erase.h -- C ABI of the ERASE training-step library for NVIDIA B200 (sm_100a).
+ *
+ * The library runs one training step of a network cut into B detached blocks, each trained by
+ * its own local loss (paper Section 2.1, Eq. 1):
+ *
+ *     z_0 = x,   z_b = f_b( sg[z_{b-1}] ; theta_b ),   l_b = loss( head_b(z_b), target )
+ *
+ * sg[] is the stop-gradient: identity going forward, zero Jacobian going backward, so the
+ * gradient of theta_b depends on block b alone and is ready as soon as block b's forward and
+ * local loss have run.  The step can be enqueued in two orders that give bit-identical results:
+ *
+ *   serial (n_streams = 1)  F_1 .. F_B, B_B .. B_1, optimizer  on one stream -- the conventional
+ *                           forward-then-backward order of Section 2.2, Eq. 2 (all lambda_i = 1,
+ *                           no L_main);
+ *   ERASE  (n_streams >= 2) F_b on the main stream; a per-block event releases B_b onto side
+ *                           stream (b-1) mod (n_streams-1) as soon as F_b and l_b are enqueued, so
+ *                           B_b overlaps F_{b+1} (Section 2.2); the optimizer waits on every
+ *                           block's backward event.
+ *
+ * Every pointer in this interface is a HOST pointer unless its comment says DEVICE.  Device
+ * pointers must belong to the CUDA device that was current when erase_create() ran.  No call
+ * throws or aborts; every failure is reported through the returned status, and a message can be
+ * read with erase_last_error().  All calls on one model must come from one host thread at a time.
+ */
+#ifndef ERASE_H_
+#define ERASE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define ERASE_API __attribute__((visibility("default")))
+#else
+#define ERASE_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct erase_model erase_model; /* opaque; owned by the library */
+
+typedef enum {
+  ERASE_OK = 0,
+  ERASE_EINVAL = 1,       /* bad argument or spec; nothing was launched                     */
+  ERASE_ENOMEM = 2,       /* device or host allocation failed, or the caller's arena is small */
+  ERASE_ECUDA = 3,        /* a CUDA call failed; text in erase_last_error()                  */
+  ERASE_ESTATE = 4,       /* call not valid in this state (e.g. step before parameters set)  */
+  ERASE_ETIMEOUT = 5,     /* a bounded device-side wait expired; the step's results are void */
+  ERASE_EUNSUPPORTED = 6  /* valid request that this build does not implement                */
+} erase_status;
+
+typedef enum { ERASE_F32 = 0, ERASE_BF16 = 1 } erase_dtype;      /* operand/activation precision;
+                                                   accumulation, gradients, optimizer are fp32 */
+typedef enum { ERASE_IN_DENSE = 0, ERASE_IN_TOKENS = 1, ERASE_IN_CTR = 2 } erase_input_kind;
+typedef enum { ERASE_BLK_MLP = 0,         /* Linear act Linear ... (no activation after the last) */
+               ERASE_BLK_TOWER = 1,       /* Linear act after every Linear                        */
+               ERASE_BLK_TRANSFORMER = 2, /* pre-LN causal transformer block, dims = {d, d_ff}    */
+               ERASE_BLK_CROSS = 3,       /* n_cross DCN-v2 layers x_{l+1} = x0 * (W x_l + b) + x_l */
+               ERASE_BLK_DOT = 4          /* dense projection, pairwise dots, then a tower        */
+} erase_block_kind;
+typedef enum { ERASE_ACT_NONE = 0, ERASE_ACT_RELU = 1, ERASE_ACT_GELU = 2 } erase_act;
+typedef enum { ERASE_HEAD_BCE = 0,        /* Linear(d->1) + mean binary cross-entropy with logits */
+               ERASE_HEAD_SOFTMAX_CE = 1  /* Linear(d->head_out) + mean softmax cross-entropy     */
+} erase_head_kind;
+typedef enum { ERASE_OPT_SGD = 0, ERASE_OPT_ADAM = 1, ERASE_OPT_ADAMW = 2 } erase_opt_kind;
+typedef enum { ERASE_TOPO_CHAIN = 0,      /* block b reads sg[z_{b-1}] (Eq. 1)                    */
+               ERASE_TOPO_PARALLEL = 1    /* every block reads sg[z_0]                            */
+} erase_topology;
+
+#define ERASE_MAX_DIMS 8
+
+/* One detached block f_b together with its local head (Section 2.1). */
+typedef struct {
+  int32_t kind;                 /* erase_block_kind                                              */
+  int32_t n_dims;               /* entries used in dims                                          */
+  int32_t dims[ERASE_MAX_DIMS]; /* MLP/TOWER: layer widths d0..dL; TRANSFORMER: {d_model, d_ff};
+                                   CROSS: {width}; DOT: {padded feature count, tower widths...}   */
+  int32_t act;                  /* erase_act between (MLP) / after (TOWER, DOT) the Linears;
+                                   TRANSFORMER always uses exact-erf GELU, CROSS none             */
+  int32_t n_heads;              /* TRANSFORMER: attention heads; head width must be 64 or a
+                                   divisor of d_model with d_model/n_heads <= 128                */
+  int32_t n_cross;              /* CROSS: number of cross layers                                 */
+  int32_t head;                 /* erase_head_kind                                               */
+  int32_t head_out;             /* 1 for BCE; vocabulary size for softmax cross-entropy          */
+} erase_block_spec;
+
+/* The whole model.  Trainable tensors are Linear weights W [out, in] row-major, biases, and
+ * LayerNorm gain/shift; the input tables (token/position embeddings, CTR tables) sit under
+ * sg[z_0] and are frozen. */
+typedef struct {
+  int32_t dtype;      /* erase_dtype                                                             */
+  int32_t input;      /* erase_input_kind                                                        */
+  int32_t topo;       /* erase_topology                                                          */
+  int32_t batch;      /* samples per step (sequences for TOKENS)                                 */
+  int32_t width;      /* DENSE: input width; TOKENS: d_model; CTR: packed width of x0            */
+  int32_t seq;        /* TOKENS: sequence length T (targets are the inputs shifted by one)       */
+  int32_t vocab;      /* TOKENS: vocabulary size                                                 */
+  int32_t n_dense;    /* CTR: dense features per sample                                          */
+  int32_t n_sparse;   /* CTR: sparse features (= embedding tables), one id each                  */
+  int32_t table_rows; /* CTR: rows per table                                                     */
+  int32_t emb_dim;    /* CTR: embedding width                                                    */
+  int32_t n_blocks;
+  const erase_block_spec* blocks; /* n_blocks entries; copied by erase_create                    */
+  int32_t opt;        /* erase_opt_kind                                                          */
+  float lr, beta1, beta2, eps, weight_decay; /* Adam: m,v with bias correction, update
+                         lr*mhat/(sqrt(vhat)+eps); AdamW first shrinks theta by (1 - lr*wd)      */
+  void* arena;        /* DEVICE, optional: caller-owned memory the model lives in (256-byte
+                         aligned); NULL = the library allocates with cudaMalloc                  */
+  size_t arena_bytes; /* size of arena; at least erase_arena_bytes(spec)                         */
+} erase_model_spec;
+
+/* One batch, all DEVICE pointers, owned by the caller and kept alive and unmodified until the
+ * step has been synchronised (erase_sync / erase_losses).
+ *   DENSE : x [batch, width] row-major in the model dtype (float or bfloat16 bits); y [batch] float
+ *   TOKENS: ids [batch, seq+1] int32 in [0, vocab); inputs are ids[:, :seq], targets ids[:, 1:]
+ *   CTR   : x = dense features [batch, n_dense] float; ids [batch, n_sparse] int32 in
+ *           [0, table_rows); y [batch] float.  x0 = [table_t[ids[n,t]] for t | dense | zero pad]. */
+typedef struct {
+  const void* x;
+  const int32_t* ids;
+  const float* y;
+} erase_batch;
+
+/* erase_step_ex flags */
+#define ERASE_GRAPH 1u   /* replay the whole step (either schedule) as one CUDA graph, captured on
+                            first use per (batch pointers, n_streams, flags); Section 1.1/2.2      */
+#define ERASE_NO_OPT 2u  /* stop after the backward passes: gradients only, parameters untouched   */
+
+/* Device bytes erase_create needs for this spec when given an arena; 0 if the spec is invalid. */
+ERASE_API size_t erase_arena_bytes(const erase_model_spec* spec);
+
+/* Builds the model on the current CUDA device: validates the spec, lays out parameters,
+ * gradients, optimizer state, per-block activation stashes and scratch, creates streams and
+ * events.  Parameters start undefined: set every tensor with erase_set_params before stepping.
+ * On failure *out is untouched.  Errors: EINVAL (spec), ENOMEM, ECUDA. */
+ERASE_API erase_status erase_create(const erase_model_spec* spec, erase_model** out);
+
+/* Waits for outstanding work, frees everything the library allocated.  NULL is allowed. */
+ERASE_API void erase_destroy(erase_model* m);
+
+/* Tensor table.  Order: frozen input tables first (tok_emb, pos_emb | table0..), then block by
+ * block: MLP/TOWER W0,b0,W1,b1,..; TRANSFORMER ln1_g,ln1_b,Wqkv,bqkv,Wproj,bproj,ln2_g,ln2_b,
+ * W1,b1,W2,b2; CROSS Wc0,bc0,..; DOT Wd,bd,W0,b0,..; each block ends with its head Wh,bh. */
+ERASE_API int32_t erase_num_tensors(const erase_model* m);
+/* block = -1 for frozen input tables; name receives a NUL-terminated string (<= 31 chars);
+ * shape has rank entries (<= 2).  Errors: EINVAL (index, NULL). */
+ERASE_API erase_status erase_tensor_info(const erase_model* m, int32_t idx, int32_t* block, char name[32],
+                               int32_t* rank, int64_t shape[4], int32_t* trainable);
+
+/* Parameters travel as fp32 host arrays of exactly n = product(shape) elements.
+ * set: copies into the fp32 master (and refreshes the bf16 operand copy); synchronous.
+ * params/grads: wait for the last enqueued step, then copy out.  grads are those of the last
+ * step (d l_b / d theta_b, fp32).  Errors: EINVAL (index, size, NULL, frozen tensor for grads). */
+ERASE_API erase_status erase_set_params(erase_model* m, int32_t idx, const float* src, size_t n);
+ERASE_API erase_status erase_params(erase_model* m, int32_t idx, float* dst, size_t n);
+ERASE_API erase_status erase_grads(erase_model* m, int32_t idx, float* dst, size_t n);
+
+/* Adam moments of one trainable tensor and the global step counter t (number of optimizer
+ * steps taken).  Any of mom1/mom2/t may be NULL.  With SGD the moments read as zeros. */
+ERASE_API erase_status erase_opt_state(erase_model* m, int32_t idx, float* mom1, float* mom2, size_t n, int64_t* t);
+ERASE_API erase_status erase_set_opt_state(erase_model* m, int32_t idx, const float* mom1, const float* mom2,
+                                 size_t n, int64_t t);
+
+/* Enqueues one training step on the model's streams and returns without waiting.
+ * n_streams = 1: serial schedule; n_streams >= 2: ERASE with n_streams-1 side streams (values
+ * above n_blocks+1 are clamped).  erase_step(m,b,n) == erase_step_ex(m,b,n,0).
+ * Errors: EINVAL (NULL, missing batch pointer, n_streams < 1), ESTATE (a tensor was never set),
+ * ECUDA. */
+ERASE_API erase_status erase_step(erase_model* m, const erase_batch* batch, int32_t n_streams);
+ERASE_API erase_status erase_step_ex(erase_model* m, const erase_batch* batch, int32_t n_streams, uint32_t flags);
+
+/* Waits for the last step and copies the local losses l_1..l_B (n_blocks floats) to dst. */
+ERASE_API erase_status erase_losses(erase_model* m, float* dst, int32_t n_blocks);
+
+/* Waits until everything enqueued on the model has finished. */
+ERASE_API erase_status erase_sync(erase_model* m);
+
+/* The CUDA stream (cudaStream_t) that steps start and end on; valid until erase_destroy.  A
+ * caller may record its own events on it to time steps. */
+ERASE_API void* erase_main_stream(erase_model* m);
+
+/* Kernels launched by this library on behalf of the model since it was created. */
+ERASE_API int64_t erase_launch_count(const erase_model* m);
+
+/* Device-side begin/end times of the last step's phases, in milliseconds relative to the step's
+ * start, from CUDA events: out[2*b], out[2*b+1] = start and end of F_b for b < n_blocks, then
+ * the same for B_b, then for the optimizer: 2*(2*n_blocks+1) floats.  Only recorded for steps
+ * run without ERASE_GRAPH.  Waits for the step.  Errors: EINVAL, ESTATE (no such step). */
+ERASE_API erase_status erase_timeline(erase_model* m, float* out, int32_t n);
+
+/* One record per operation of a profiled step. */
+typedef struct {
+  char name[32];    /* kernel class: gemm_fwd, gemm_dgrad, gemm_wgrad, softmax_ce, opt_update, ...   */
+  int32_t block;    /* block index, -1 for input staging and the optimizer                         */
+  int32_t phase;    /* 0 input staging, 1 forward F_b, 2 backward B_b, 3 optimizer                  */
+  int32_t launches; /* kernels this operation launches                                             */
+  float ms;         /* device time between CUDA events recorded around the operation               */
+  double flops;     /* algorithmic floating-point operations (2*M*N*K for a GEMM)                  */
+  double bytes;     /* algorithmic bytes: every operand read once, every result written once       */
+} erase_op_record;
+
+/* Runs one complete step in the serial order on the main stream with a pair of CUDA events around
+ * every operation, waits for it, and writes one record per operation to out (at most cap; *n
+ * receives the number of operations the step has).  It is a real step: parameters are updated.
+ * Used to attribute time to kernels (the roofline of the dominant kernel); the event pairs
+ * serialise nothing but add launch gaps, so whole-step time is NOT measured here.
+ * Errors: as erase_step, and EINVAL for NULL out/n. */
+ERASE_API erase_status erase_profile_step(erase_model* m, const erase_batch* batch, erase_op_record* out,
+                                          int32_t cap, int32_t* n);
+
+/* Text of the last error on this model ("" if none); NULL model gives the text of the last
+ * failed erase_create on this thread. */
+ERASE_API const char* erase_last_error(const erase_model* m);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ERASE_H_ */

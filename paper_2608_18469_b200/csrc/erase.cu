@@ -1,0 +1,1085 @@
+// Host side of the ERASE step library: model layout, the per-block operation lists, the two
+// schedules (serial, and early backward on side streams released by per-block events), whole-step
+// CUDA-graph replay, and the C ABI declared in include/erase.h.
+#include "../../include/erase.h"
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <functional>
+#include <map>
+#include <string>
+#include <tuple>
+#include <vector>
+
+#include "gemm_tc.cuh"
+#include "kernels.cuh"
+
+using namespace erase;
+
+namespace {
+
+thread_local std::string g_create_error;
+
+struct Op {
+  std::function<cudaError_t(cudaStream_t)> fn;
+  int launches;
+  const char* name = "op";  // kernel class, for the per-operation profile
+  double flops = 0;         // algorithmic floating-point operations of one run
+  double bytes = 0;         // algorithmic bytes (each operand read once, each result written once)
+};
+typedef std::vector<Op> OpList;
+
+struct Tensor {
+  int block;
+  std::string name;
+  int rank;
+  int64_t shape[2];
+  bool trainable;
+  size_t n;    // elements
+  size_t off;  // element offset inside the frozen or the trainable arena
+  bool set;
+};
+
+struct GraphKey {
+  const void* x;
+  const void* ids;
+  const void* y;
+  int n_streams;
+  unsigned flags;
+  bool operator<(const GraphKey& o) const {
+    return std::tie(x, ids, y, n_streams, flags) < std::tie(o.x, o.ids, o.y, o.n_streams, o.flags);
+  }
+};
+
+}  // namespace
+
+struct erase_model {
+  erase_model_spec spec;
+  std::vector<erase_block_spec> blocks;
+  bool bf16 = false;
+  bool dry = false;  // sizing pass: no device memory is touched
+  int rows = 0;      // samples, or tokens = batch*seq
+  int B = 0;
+  size_t esz = 4;    // bytes per activation element
+
+  std::vector<Tensor> tensors;
+  size_t frozen_n = 0, train_n = 0;
+  float* frozen = nullptr;
+  float* theta = nullptr;
+  float* grad = nullptr;
+  float* mom1 = nullptr;
+  float* mom2 = nullptr;
+  void* shadow = nullptr;  // bf16 copy of theta (operands of the bf16 GEMMs)
+  double* tick = nullptr;  // {t, 1-beta1^t, 1-beta2^t}
+  float* losses = nullptr;
+
+  // device memory
+  char* arena = nullptr;
+  size_t arena_bytes = 0, arena_used = 0;
+  std::vector<void*> owned;
+
+  cudaStream_t main = nullptr;
+  std::vector<cudaStream_t> side;
+  std::vector<cudaEvent_t> ev_f, ev_b;
+  cudaEvent_t ev_opt = nullptr;
+  std::vector<cudaEvent_t> ev_time;  // 2*(2B+1) timing events + 1 step start
+  std::vector<cudaEvent_t> ev_prof;  // pairs around every operation of a profiled step
+  bool timeline_valid = false;
+
+  OpList stage, opt;
+  std::vector<OpList> fwd, bwd;
+  erase_batch cur = {nullptr, nullptr, nullptr};
+  std::map<GraphKey, cudaGraphExec_t> graphs;
+
+  int64_t launches = 0;
+  bool stepped = false;
+  std::string err;
+  erase_status fail(erase_status st, const std::string& msg) {
+    err = msg;
+    return st;
+  }
+};
+
+namespace {
+
+#define CK(call)                                                                     \
+  do {                                                                               \
+    cudaError_t e_ = (call);                                                         \
+    if (e_ != cudaSuccess)                                                           \
+      return m->fail(ERASE_ECUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); \
+  } while (0)
+
+size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Host<->device copies are ordered on the model's main stream (a non-blocking stream does not
+// synchronise with the legacy default stream that a plain cudaMemcpy uses) and waited for.
+cudaError_t copy_sync(erase_model* m, void* dst, const void* src, size_t bytes, cudaMemcpyKind kind) {
+  cudaError_t e = cudaMemcpyAsync(dst, src, bytes, kind, m->main);
+  if (e != cudaSuccess) return e;
+  return cudaStreamSynchronize(m->main);
+}
+
+// ---- device memory: bump allocation from the caller's arena, else cudaMalloc ---------------
+void* dev_alloc(erase_model* m, size_t bytes, bool* ok) {
+  bytes = round_up(bytes ? bytes : 1, 256);
+  if (m->dry) {
+    m->arena_used += bytes;
+    return (void*)(uintptr_t)(4096 + m->arena_used);  // never dereferenced
+  }
+  if (m->arena) {
+    if (m->arena_used + bytes > m->arena_bytes) { *ok = false; return nullptr; }
+    void* p = m->arena + m->arena_used;
+    m->arena_used += bytes;
+    if (cudaMemset(p, 0, bytes) != cudaSuccess) *ok = false;
+    return p;
+  }
+  void* p = nullptr;
+  if (cudaMalloc(&p, bytes) != cudaSuccess) { *ok = false; cudaGetLastError(); return nullptr; }
+  m->owned.push_back(p);
+  if (cudaMemset(p, 0, bytes) != cudaSuccess) *ok = false;
+  return p;
+}
+
+// ---- spec validation ------------------------------------------------------------------------
+bool validate(const erase_model_spec* s, std::string* why) {
+  auto bad = [&](const char* w) { *why = w; return false; };
+  if (!s) return bad("spec is NULL");
+  if (s->dtype != ERASE_F32 && s->dtype != ERASE_BF16) return bad("dtype");
+  if (s->input < 0 || s->input > ERASE_IN_CTR) return bad("input kind");
+  if (s->topo != ERASE_TOPO_CHAIN && s->topo != ERASE_TOPO_PARALLEL) return bad("topology");
+  if (s->batch < 1 || s->width < 1) return bad("batch/width must be positive");
+  if (s->n_blocks < 1 || s->n_blocks > 4096 || !s->blocks) return bad("n_blocks/blocks");
+  if (s->opt < 0 || s->opt > ERASE_OPT_ADAMW) return bad("optimizer kind");
+  if (!(s->lr >= 0.f)) return bad("lr");
+  if (s->opt != ERASE_OPT_SGD && (!(s->beta1 >= 0.f && s->beta1 < 1.f) || !(s->beta2 >= 0.f && s->beta2 < 1.f) || !(s->eps > 0.f)))
+    return bad("Adam constants");
+  if (s->input == ERASE_IN_TOKENS && (s->seq < 1 || s->vocab < 1)) return bad("seq/vocab");
+  if ((long long)s->batch * (s->input == ERASE_IN_TOKENS ? s->seq : 1) > (1LL << 30)) return bad("too many rows");
+  if (s->input == ERASE_IN_CTR) {
+    if (s->n_dense < 0 || s->n_sparse < 1 || s->table_rows < 1 || s->emb_dim < 1) return bad("CTR sizes");
+    if (s->width < s->n_sparse * s->emb_dim + s->n_dense) return bad("CTR width too small for x0");
+  }
+  if (s->arena && ((uintptr_t)s->arena & 255)) return bad("arena must be 256-byte aligned");
+  int prev = s->width;
+  for (int b = 0; b < s->n_blocks; b++) {
+    const erase_block_spec& k = s->blocks[b];
+    int in = s->topo == ERASE_TOPO_PARALLEL ? s->width : prev;
+    if (k.n_dims < 1 || k.n_dims > ERASE_MAX_DIMS) return bad("block n_dims");
+    for (int i = 0; i < k.n_dims; i++)
+      if (k.dims[i] < 1) return bad("block dims must be positive");
+    if (k.act < 0 || k.act > ERASE_ACT_GELU) return bad("block act");
+    if (k.head == ERASE_HEAD_BCE) {
+      if (k.head_out != 1) return bad("BCE head_out must be 1");
+      if (s->input == ERASE_IN_TOKENS) return bad("BCE head needs labels (dense or CTR input)");
+    } else if (k.head == ERASE_HEAD_SOFTMAX_CE) {
+      if (s->input != ERASE_IN_TOKENS) return bad("softmax-CE head needs token input");
+      if (k.head_out != s->vocab) return bad("softmax-CE head_out must equal vocab");
+    } else return bad("head kind");
+    int out = 0;
+    switch (k.kind) {
+      case ERASE_BLK_MLP:
+      case ERASE_BLK_TOWER:
+        if (k.n_dims < 2) return bad("MLP/TOWER need at least two dims");
+        if (k.dims[0] != in) return bad("block input width does not match its producer");
+        out = k.dims[k.n_dims - 1];
+        break;
+      case ERASE_BLK_TRANSFORMER:
+        if (s->input != ERASE_IN_TOKENS) return bad("transformer block needs token input");
+        if (k.n_dims != 2 || k.dims[0] != in) return bad("transformer dims = {d_model, d_ff}");
+        if (k.n_heads < 1 || k.dims[0] % k.n_heads || k.dims[0] / k.n_heads > 128) return bad("n_heads");
+        out = k.dims[0];
+        break;
+      case ERASE_BLK_CROSS:
+        if (k.n_dims != 1 || k.dims[0] != in || k.n_cross < 0 || k.n_cross > 64) return bad("cross dims/n_cross");
+        out = in;
+        break;
+      case ERASE_BLK_DOT: {
+        if (s->input != ERASE_IN_CTR || s->topo != ERASE_TOPO_PARALLEL) return bad("dot block needs CTR input, parallel topology");
+        if (k.n_dims < 2) return bad("dot block needs a tower");
+        int nv = s->n_sparse + 1;
+        if (k.dims[0] < nv * (nv - 1) / 2 + s->emb_dim) return bad("dot feature width too small");
+        if (s->width - s->n_sparse * s->emb_dim < 1) return bad("dot block needs dense columns");
+        out = k.dims[k.n_dims - 1];
+        break;
+      }
+      default:
+        return bad("block kind");
+    }
+    prev = out;
+  }
+  return true;
+}
+
+// ---- tensor table ---------------------------------------------------------------------------
+void add_tensor(erase_model* m, int block, const std::string& name, int64_t d0, int64_t d1, bool trainable) {
+  Tensor t;
+  t.block = block;
+  t.name = name;
+  t.rank = d1 > 0 ? 2 : 1;
+  t.shape[0] = d0;
+  t.shape[1] = d1 > 0 ? d1 : 0;
+  t.trainable = trainable;
+  t.n = (size_t)d0 * (size_t)(d1 > 0 ? d1 : 1);
+  size_t& top = trainable ? m->train_n : m->frozen_n;
+  t.off = top;
+  top += round_up(t.n, 64);
+  t.set = false;
+  m->tensors.push_back(t);
+}
+
+void build_tensor_table(erase_model* m) {
+  const erase_model_spec& s = m->spec;
+  if (s.input == ERASE_IN_TOKENS) {
+    add_tensor(m, -1, "tok_emb", s.vocab, s.width, false);
+    add_tensor(m, -1, "pos_emb", s.seq, s.width, false);
+  } else if (s.input == ERASE_IN_CTR) {
+    for (int t = 0; t < s.n_sparse; t++) add_tensor(m, -1, "table" + std::to_string(t), s.table_rows, s.emb_dim, false);
+  }
+  for (int b = 0; b < m->B; b++) {
+    const erase_block_spec& k = m->blocks[b];
+    int out = 0;
+    auto linears = [&](int first) {
+      for (int i = first; i + 1 < k.n_dims; i++) {
+        add_tensor(m, b, "W" + std::to_string(i - first), k.dims[i + 1], k.dims[i], true);
+        add_tensor(m, b, "b" + std::to_string(i - first), k.dims[i + 1], 0, true);
+      }
+      out = k.dims[k.n_dims - 1];
+    };
+    switch (k.kind) {
+      case ERASE_BLK_MLP:
+      case ERASE_BLK_TOWER:
+        linears(0);
+        break;
+      case ERASE_BLK_TRANSFORMER: {
+        int d = k.dims[0], ff = k.dims[1];
+        add_tensor(m, b, "ln1_g", d, 0, true);
+        add_tensor(m, b, "ln1_b", d, 0, true);
+        add_tensor(m, b, "Wqkv", 3 * d, d, true);
+        add_tensor(m, b, "bqkv", 3 * d, 0, true);
+        add_tensor(m, b, "Wproj", d, d, true);
+        add_tensor(m, b, "bproj", d, 0, true);
+        add_tensor(m, b, "ln2_g", d, 0, true);
+        add_tensor(m, b, "ln2_b", d, 0, true);
+        add_tensor(m, b, "W1", ff, d, true);
+        add_tensor(m, b, "b1", ff, 0, true);
+        add_tensor(m, b, "W2", d, ff, true);
+        add_tensor(m, b, "b2", d, 0, true);
+        out = d;
+        break;
+      }
+      case ERASE_BLK_CROSS:
+        for (int i = 0; i < k.n_cross; i++) {
+          add_tensor(m, b, "Wc" + std::to_string(i), k.dims[0], k.dims[0], true);
+          add_tensor(m, b, "bc" + std::to_string(i), k.dims[0], 0, true);
+        }
+        out = k.dims[0];
+        break;
+      case ERASE_BLK_DOT:
+        add_tensor(m, b, "Wd", m->spec.emb_dim, m->spec.width - m->spec.n_sparse * m->spec.emb_dim, true);
+        add_tensor(m, b, "bd", m->spec.emb_dim, 0, true);
+        linears(0);
+        break;
+    }
+    add_tensor(m, b, "Wh", k.head_out, out, true);
+    add_tensor(m, b, "bh", k.head_out, 0, true);
+  }
+}
+
+// ---- plan builder ---------------------------------------------------------------------------
+struct Builder {
+  erase_model* m;
+  bool ok = true;
+  int cursor = 0;  // next tensor index of the block being built
+
+  void* act_buf(size_t elems) { return dev_alloc(m, elems * m->esz, &ok); }
+  float* f32_buf(size_t elems) { return (float*)dev_alloc(m, elems * sizeof(float), &ok); }
+
+  const Tensor& T(int idx) const { return m->tensors[idx]; }
+  const void* Wop(int idx) const {  // GEMM operand copy of a weight matrix
+    return m->bf16 ? (const void*)((const __nv_bfloat16*)m->shadow + T(idx).off) : (const void*)(m->theta + T(idx).off);
+  }
+  const float* Wf(int idx) const { return m->theta + T(idx).off; }
+  float* G(int idx) const { return m->grad + T(idx).off; }
+
+  static void note(OpList& ops, const char* name, double flops = 0, double bytes = 0) {
+    ops.back().name = name;
+    ops.back().flops = flops;
+    ops.back().bytes = bytes;
+  }
+  const char* gemm_tag = "gemm";
+
+  void gemm(OpList& ops, GemmArgs g) {
+    bool bf = m->bf16;
+    size_t before = ops.size();
+    gemm_inner(ops, g);
+    double fl = 2.0 * g.M * g.N * g.K;
+    double by = ((double)g.M * g.K + (double)g.N * g.K) * m->esz + (double)g.M * g.N * (g.c_f32 ? 4 : m->esz);
+    (void)bf;
+    if (ops.size() > before) note(ops, gemm_tag, fl, by);
+  }
+  void gemm_inner(OpList& ops, GemmArgs g) {
+    bool bf = m->bf16;
+    TcPlan plan;
+    if (bf && !m->dry && tc_gemm_plan(g, &plan)) {
+      ops.push_back({[g, plan](cudaStream_t s) { return tc_gemm_launch(g, plan, s); }, plan.launches});
+      return;
+    }
+    if (g.splits > 1) {
+      g.ws = f32_buf((size_t)g.splits * g.M * g.N);
+      float* out = (float*)g.C;
+      long long ldo = g.ldc;
+      ops.push_back({[g, bf, out, ldo](cudaStream_t s) {
+                       cudaError_t e = gemm_simt(g, bf, s);
+                       if (e != cudaSuccess) return e;
+                       return splitk_reduce(g.ws, g.splits, (long long)g.M * g.N, g.N, out, ldo, s);
+                     }, 2});
+    } else {
+      ops.push_back({[g, bf](cudaStream_t s) { return gemm_simt(g, bf, s); }, 1});
+    }
+  }
+
+  // Y[M,N] = epi(X[M,K] W[N,K]^T)
+  void lin_fwd(OpList& ops, const void* X, long long ldx, int widx, int bidx, void* Y, int M, int N, int K, Epilogue e) {
+    GemmArgs g;
+    g.M = M; g.N = N; g.K = K;
+    g.A = X; g.sa_m = ldx; g.sa_k = 1;
+    g.B = Wop(widx); g.sb_n = K; g.sb_k = 1;
+    g.C = Y; g.ldc = N;
+    e.bias = bidx >= 0 ? Wf(bidx) : nullptr;
+    if (e.ld_aux == 0) e.ld_aux = N;
+    g.epi = e;
+    gemm_tag = "gemm_fwd";
+    gemm(ops, g);
+  }
+  // dX[M,K] = epi(dY[M,N] W[N,K])
+  void lin_dgrad(OpList& ops, const void* dY, int widx, void* dX, int M, int N, int K, Epilogue e) {
+    GemmArgs g;
+    g.M = M; g.N = K; g.K = N;
+    g.A = dY; g.sa_m = N; g.sa_k = 1;
+    g.B = Wop(widx); g.sb_n = 1; g.sb_k = K;
+    g.C = dX; g.ldc = K;
+    if (e.ld_aux == 0) e.ld_aux = K;
+    g.epi = e;
+    gemm_tag = "gemm_dgrad";
+    gemm(ops, g);
+  }
+  // dW[N,K] = dY[M,N]^T X[M,K]  (fp32, deterministic split over M), db[N] = column sums of dY
+  void lin_wgrad(OpList& ops, const void* dY, const void* X, long long ldx, int widx, int bidx, int M, int N, int K) {
+    GemmArgs g;
+    g.M = N; g.N = K; g.K = M;
+    g.A = dY; g.sa_m = 1; g.sa_k = N;
+    g.B = X; g.sb_n = 1; g.sb_k = ldx;
+    g.C = G(widx); g.ldc = K; g.c_f32 = 1;
+    long long tiles = (long long)((N + 63) / 64) * ((K + 63) / 64);
+    int splits = (int)((296 + tiles - 1) / tiles);
+    int maxs = M / 64 > 0 ? M / 64 : 1;
+    if (splits > maxs) splits = maxs;
+    if (splits > 64) splits = 64;
+    g.splits = splits < 1 ? 1 : splits;
+    gemm_tag = "gemm_wgrad";
+    gemm(ops, g);
+    if (bidx >= 0) bias_grad(ops, dY, N, M, N, bidx);
+  }
+  void bias_grad(OpList& ops, const void* dY, long long ld, int M, int N, int bidx) {
+    int chunks = colsum_chunks(M, N);
+    float* ws = chunks > 1 ? f32_buf((size_t)chunks * N) : nullptr;
+    float* out = G(bidx);
+    bool bf = m->bf16;
+    ops.push_back({[=](cudaStream_t s) { return colsum(dY, bf, ld, M, N, nullptr, ws, chunks, out, s); }, chunks > 1 ? 2 : 1});
+    note(ops, "colsum", (double)M * N, (double)M * N * m->esz);
+  }
+
+  // ---- heads: forward computes the local loss and the loss gradient, backward the head's own
+  // gradients and dz (times act'(src) when the block ends in an activation) ------------------
+  void head(int b, const erase_block_spec& k, const void* z, int d, int wh, int bh, OpList& f, OpList& bw, void* dz,
+            int dact, const void* dact_src) {
+    erase_model* mm = m;
+    bool bf = m->bf16;
+    int rows = m->rows;
+    float* rowloss = f32_buf(rows);
+    float* loss_out = m->losses + b;
+    float inv = 1.f / (float)rows;
+    if (k.head == ERASE_HEAD_BCE) {
+      float* ds = f32_buf(rows);
+      const float* w = Wf(wh);
+      const float* bb = Wf(bh);
+      f.push_back({[=](cudaStream_t s) { return bce_head_fwd(z, d, w, bb, mm->cur.y, rowloss, ds, rows, d, inv, bf, s); }, 1});
+      note(f, "bce_head_fwd", 2.0 * rows * d, (double)rows * d * m->esz);
+      f.push_back({[=](cudaStream_t s) { return reduce_sum(rowloss, rows, inv, loss_out, s); }, 1});
+      note(f, "loss_reduce", rows, 4.0 * rows);
+      bw.push_back({[=](cudaStream_t s) { return bce_head_dz(ds, w, dz, dact, dact_src, rows, d, bf, s); }, 1});
+      note(bw, "bce_head_dz", (double)rows * d, (double)rows * d * m->esz);
+      {
+        int chunks = colsum_chunks(rows, d);
+        float* ws = chunks > 1 ? f32_buf((size_t)chunks * d) : nullptr;
+        float* out = G(wh);
+        bw.push_back({[=](cudaStream_t s) { return colsum(z, bf, d, rows, d, ds, ws, chunks, out, s); }, chunks > 1 ? 2 : 1});
+        note(bw, "colsum", 2.0 * rows * d, (double)rows * d * m->esz);
+      }
+      {
+        int chunks = colsum_chunks(rows, 1);
+        float* ws = chunks > 1 ? f32_buf((size_t)chunks) : nullptr;
+        float* out = G(bh);
+        bw.push_back({[=](cudaStream_t s) { return colsum(ds, false, 1, rows, 1, nullptr, ws, chunks, out, s); }, chunks > 1 ? 2 : 1});
+        note(bw, "colsum", rows, 4.0 * rows);
+      }
+    } else {
+      int V = k.head_out, T_ = m->spec.seq;
+      void* logits = act_buf((size_t)rows * V);
+      lin_fwd(f, z, d, wh, bh, logits, rows, V, d, Epilogue());
+      f.push_back({[=](cudaStream_t s) { return softmax_ce_inplace(logits, mm->cur.ids, T_, rowloss, rows, V, inv, bf, s); }, 1});
+      note(f, "softmax_ce", 4.0 * rows * V, 2.0 * rows * V * m->esz);
+      f.push_back({[=](cudaStream_t s) { return reduce_sum(rowloss, rows, inv, loss_out, s); }, 1});
+      note(f, "loss_reduce", rows, 4.0 * rows);
+      lin_wgrad(bw, logits, z, d, wh, bh, rows, V, d);
+      lin_dgrad(bw, logits, wh, dz, rows, V, d, Epilogue());
+      if (dact != ACT_NONE) {
+        long long n = (long long)rows * d;
+        bw.push_back({[=](cudaStream_t s) { return ew_dact(dz, dact_src, dact, n, bf, s); }, 1});
+        note(bw, "ew_dact", (double)n, 3.0 * n * m->esz);
+      }
+    }
+  }
+
+  // ---- Linear stack (MLP / TOWER / tower of the DOT block) ---------------------------------
+  // returns the output buffer; fills last-activation info for the head backward
+  struct Stack {
+    std::vector<const void*> in;   // input of layer i
+    std::vector<const void*> src;  // activation-derivative source of layer i (pre-act for GELU, output for ReLU)
+    std::vector<int> act;          // activation after layer i
+    void* out = nullptr;
+  };
+  Stack stack_fwd(OpList& f, const erase_block_spec& k, const void* zin, long long ldin, bool act_last, int first_tensor) {
+    Stack st;
+    int L = k.n_dims - 1;
+    const void* h = zin;
+    long long ldh = ldin;
+    for (int i = 0; i < L; i++) {
+      int K = k.dims[i], N = k.dims[i + 1];
+      bool use = act_last || i < L - 1;
+      int a = use ? k.act : ACT_NONE;
+      void* y = act_buf((size_t)m->rows * N);
+      Epilogue e;
+      e.act = a;
+      const void* src = y;
+      if (a == ACT_GELU) {
+        void* u = act_buf((size_t)m->rows * N);
+        e.pre_out = u;
+        src = u;
+      }
+      lin_fwd(f, h, ldh, first_tensor + 2 * i, first_tensor + 2 * i + 1, y, m->rows, N, K, e);
+      st.in.push_back(h);
+      st.src.push_back(src);
+      st.act.push_back(a);
+      h = y;
+      ldh = N;
+      st.out = y;
+    }
+    return st;
+  }
+  // d = gradient w.r.t. the stack output already multiplied by the last activation's derivative.
+  // Returns the gradient w.r.t. the stack input when need_dx.
+  void* stack_bwd(OpList& bw, const erase_block_spec& k, const Stack& st, long long ldin, void* d, int first_tensor, bool need_dx) {
+    int L = k.n_dims - 1;
+    for (int i = L - 1; i >= 0; i--) {
+      int K = k.dims[i], N = k.dims[i + 1];
+      lin_wgrad(bw, d, st.in[i], i == 0 ? ldin : K, first_tensor + 2 * i, first_tensor + 2 * i + 1, m->rows, N, K);
+      if (i > 0 || need_dx) {
+        void* dx = act_buf((size_t)m->rows * K);
+        Epilogue e;
+        if (i > 0 && st.act[i - 1] != ACT_NONE) {
+          e.dact = st.act[i - 1];
+          e.dact_src = st.src[i - 1];
+        }
+        lin_dgrad(bw, d, first_tensor + 2 * i, dx, m->rows, N, K, e);
+        d = dx;
+      }
+    }
+    return d;
+  }
+
+  // ---- blocks ----------------------------------------------------------------------------------
+  // Each returns z_b (output buffer).  `first` is the tensor index of the block's first tensor.
+  void* block_mlp(int b, const erase_block_spec& k, const void* zin, int first, OpList& f, OpList& bw) {
+    bool tower = k.kind == ERASE_BLK_TOWER;
+    int L = k.n_dims - 1;
+    Stack st = stack_fwd(f, k, zin, k.dims[0], tower, first);
+    int dout = k.dims[L];
+    void* dz = act_buf((size_t)m->rows * dout);
+    head(b, k, st.out, dout, first + 2 * L, first + 2 * L + 1, f, bw, dz, st.act[L - 1], st.src[L - 1]);
+    stack_bwd(bw, k, st, k.dims[0], dz, first, false);
+    return st.out;
+  }
+
+  void* block_transformer(int b, const erase_block_spec& k, const void* z, int first, OpList& f, OpList& bw) {
+    const int d = k.dims[0], ff = k.dims[1], H = k.n_heads, dh = d / H;
+    const int rows = m->rows, batch = m->spec.batch, T_ = m->spec.seq;
+    const bool bf = m->bf16;
+    enum { LN1G = 0, LN1B, WQKV, BQKV, WPROJ, BPROJ, LN2G, LN2B, W1, B1, W2, B2, WH, BH };
+    auto t = [&](int i) { return first + i; };
+    // forward
+    void* a = act_buf((size_t)rows * d);
+    float* mean1 = f32_buf(rows); float* rstd1 = f32_buf(rows);
+    void* qkv = act_buf((size_t)rows * 3 * d);
+    void* o = act_buf((size_t)rows * d);
+    float* lse = f32_buf((size_t)batch * H * T_);
+    void* h = act_buf((size_t)rows * d);
+    void* mm2 = act_buf((size_t)rows * d);
+    float* mean2 = f32_buf(rows); float* rstd2 = f32_buf(rows);
+    void* u = act_buf((size_t)rows * ff);
+    void* g = act_buf((size_t)rows * ff);
+    void* zout = act_buf((size_t)rows * d);
+    {
+      const float* g1 = Wf(t(LN1G)); const float* b1 = Wf(t(LN1B));
+      f.push_back({[=](cudaStream_t s) { return layernorm_fwd(z, g1, b1, a, mean1, rstd1, rows, d, bf, s); }, 1});
+      note(f, "layernorm_fwd", 8.0 * rows * d, 2.0 * rows * d * m->esz);
+      lin_fwd(f, a, d, t(WQKV), t(BQKV), qkv, rows, 3 * d, d, Epilogue());
+      f.push_back({[=](cudaStream_t s) { return attention_fwd(qkv, o, lse, batch, T_, H, dh, bf, s); }, 1});
+      note(f, "attention_fwd", 4.0 * batch * H * ((double)T_ * (T_ + 1) / 2) * dh, 4.0 * rows * d * m->esz);
+      Epilogue e1; e1.res = z;
+      lin_fwd(f, o, d, t(WPROJ), t(BPROJ), h, rows, d, d, e1);
+      const float* g2 = Wf(t(LN2G)); const float* b2 = Wf(t(LN2B));
+      f.push_back({[=](cudaStream_t s) { return layernorm_fwd(h, g2, b2, mm2, mean2, rstd2, rows, d, bf, s); }, 1});
+      note(f, "layernorm_fwd", 8.0 * rows * d, 2.0 * rows * d * m->esz);
+      Epilogue e2; e2.act = ACT_GELU; e2.pre_out = u;
+      lin_fwd(f, mm2, d, t(W1), t(B1), g, rows, ff, d, e2);
+      Epilogue e3; e3.res = h;
+      lin_fwd(f, g, ff, t(W2), t(B2), zout, rows, d, ff, e3);
+    }
+    // head + backward
+    void* dz = act_buf((size_t)rows * d);
+    head(b, k, zout, d, t(WH), t(BH), f, bw, dz, ACT_NONE, nullptr);
+    void* du = act_buf((size_t)rows * ff);
+    void* dm = act_buf((size_t)rows * d);
+    void* dhb = act_buf((size_t)rows * d);
+    void* dO = act_buf((size_t)rows * d);
+    void* dqkv = act_buf((size_t)rows * 3 * d);
+    float* delta = f32_buf((size_t)batch * H * T_);
+    void* da = act_buf((size_t)rows * d);
+    {
+      lin_wgrad(bw, dz, g, ff, t(W2), t(B2), rows, d, ff);
+      Epilogue e; e.dact = ACT_GELU; e.dact_src = u;
+      lin_dgrad(bw, dz, t(W2), du, rows, d, ff, e);
+      lin_wgrad(bw, du, mm2, d, t(W1), t(B1), rows, ff, d);
+      lin_dgrad(bw, du, t(W1), dm, rows, ff, d, Epilogue());
+      ln_bwd(bw, dm, h, mean2, rstd2, t(LN2G), t(LN2B), dz, dhb, d);
+      lin_wgrad(bw, dhb, o, d, t(WPROJ), t(BPROJ), rows, d, d);
+      lin_dgrad(bw, dhb, t(WPROJ), dO, rows, d, d, Epilogue());
+      bw.push_back({[=](cudaStream_t s) { return attention_bwd(qkv, o, dO, lse, delta, dqkv, batch, T_, H, dh, bf, s); }, 3});
+      note(bw, "attention_bwd", 8.0 * batch * H * ((double)T_ * (T_ + 1) / 2) * dh, 8.0 * rows * d * m->esz);
+      lin_wgrad(bw, dqkv, a, d, t(WQKV), t(BQKV), rows, 3 * d, d);
+      lin_dgrad(bw, dqkv, t(WQKV), da, rows, 3 * d, d, Epilogue());
+      // LN1: only its gain/shift gradients; dx would flow into the detached z_{b-1}
+      ln_bwd(bw, da, z, mean1, rstd1, t(LN1G), t(LN1B), nullptr, nullptr, d);
+    }
+    return zout;
+  }
+  // dx = LNbwd(dy) + add (skipped when dx == nullptr); gain/shift gradients always
+  void ln_bwd(OpList& bw, const void* dy, const void* x, const float* mean, const float* rstd, int gidx, int bidx,
+              const void* add, void* dx, int d) {
+    int rows = m->rows;
+    bool bf = m->bf16;
+    const float* gain = Wf(gidx);
+    if (dx) bw.push_back({[=](cudaStream_t s) { return layernorm_bwd_dx(dy, x, gain, mean, rstd, add, dx, rows, d, bf, s); }, 1});
+    if (dx) note(bw, "layernorm_bwd", 12.0 * rows * d, 4.0 * rows * d * m->esz);
+    int chunks = colsum_chunks(rows, d);
+    float* ws = chunks > 1 ? f32_buf((size_t)2 * chunks * d) : nullptr;
+    float* dg = G(gidx); float* db = G(bidx);
+    bw.push_back({[=](cudaStream_t s) { return layernorm_param_grad(dy, x, mean, rstd, ws, chunks, dg, db, rows, d, bf, s); }, chunks > 1 ? 3 : 1});
+    note(bw, "layernorm_param_grad", 4.0 * rows * d, 2.0 * rows * d * m->esz);
+  }
+
+  void* block_cross(int b, const erase_block_spec& k, const void* x0, int first, OpList& f, OpList& bw) {
+    const int w = k.dims[0], L = k.n_cross, rows = m->rows;
+    const bool bf = m->bf16;
+    std::vector<const void*> xs;
+    const void* xl = x0;
+    for (int l = 0; l < L; l++) {
+      void* y = act_buf((size_t)rows * w);
+      Epilogue e; e.mul = x0; e.res = xl;
+      lin_fwd(f, xl, w, first + 2 * l, first + 2 * l + 1, y, rows, w, w, e);
+      xs.push_back(xl);
+      xl = y;
+    }
+    void* dz = act_buf((size_t)rows * w);
+    head(b, k, xl, w, first + 2 * L, first + 2 * L + 1, f, bw, dz, ACT_NONE, nullptr);
+    void* d = dz;
+    for (int l = L - 1; l >= 0; l--) {
+      void* tt = act_buf((size_t)rows * w);
+      long long n = (long long)rows * w;
+      const void* dc = d;
+      bw.push_back({[=](cudaStream_t s) { return ew_mul(dc, x0, tt, n, bf, s); }, 1});
+      note(bw, "ew_mul", (double)n, 3.0 * n * m->esz);
+      lin_wgrad(bw, tt, xs[l], w, first + 2 * l, first + 2 * l + 1, rows, w, w);
+      if (l > 0) {
+        void* dn = act_buf((size_t)rows * w);
+        Epilogue e; e.res = d;
+        lin_dgrad(bw, tt, first + 2 * l, dn, rows, w, w, e);
+        d = dn;
+      }
+    }
+    return const_cast<void*>(xl);
+  }
+
+  void* block_dot(int b, const erase_block_spec& k, const void* x0, int first, OpList& f, OpList& bw) {
+    const erase_model_spec& s = m->spec;
+    const int rows = m->rows, e_ = s.emb_dim, ns = s.n_sparse, w0 = s.width;
+    const int dp = w0 - ns * e_;  // padded dense columns
+    const int fw = k.dims[0];
+    const bool bf = m->bf16;
+    const char* dense_cols = (const char*)x0 + (size_t)ns * e_ * m->esz;
+    void* proj = act_buf((size_t)rows * e_);
+    lin_fwd(f, dense_cols, w0, first, first + 1, proj, rows, e_, dp, Epilogue());
+    void* feats = act_buf((size_t)rows * fw);
+    f.push_back({[=](cudaStream_t st) { return dot_fwd(proj, x0, w0, feats, rows, ns, e_, fw, bf, st); }, 1});
+    note(f, "dot_fwd", (double)rows * (ns + 1) * ns * e_, (double)rows * (w0 + fw) * m->esz);
+    int L = k.n_dims - 1;
+    Stack st = stack_fwd(f, k, feats, fw, true, first + 2);
+    int dout = k.dims[L];
+    void* dz = act_buf((size_t)rows * dout);
+    head(b, k, st.out, dout, first + 2 + 2 * L, first + 2 + 2 * L + 1, f, bw, dz, st.act[L - 1], st.src[L - 1]);
+    void* dfeat = stack_bwd(bw, k, st, fw, dz, first + 2, true);
+    void* dproj = act_buf((size_t)rows * e_);
+    bw.push_back({[=](cudaStream_t s2) { return dot_bwd(dfeat, x0, w0, dproj, rows, ns, e_, fw, bf, s2); }, 1});
+    note(bw, "dot_bwd", 2.0 * rows * ns * e_, (double)rows * (w0 + fw) * m->esz);
+    lin_wgrad(bw, dproj, dense_cols, w0, first, first + 1, rows, e_, dp);
+    return st.out;
+  }
+
+  bool build() {
+    erase_model* mm = m;
+    const erase_model_spec& s = m->spec;
+    const bool bf = m->bf16;
+    // arenas
+    m->frozen = m->frozen_n ? f32_buf(m->frozen_n) : nullptr;
+    m->theta = f32_buf(m->train_n);
+    m->grad = f32_buf(m->train_n);
+    if (s.opt != ERASE_OPT_SGD) { m->mom1 = f32_buf(m->train_n); m->mom2 = f32_buf(m->train_n); }
+    if (bf) m->shadow = dev_alloc(m, m->train_n * 2, &ok);
+    m->tick = (double*)dev_alloc(m, 3 * sizeof(double), &ok);
+    m->losses = f32_buf(m->B);
+    // z_0
+    // z_0: dense batches are copied into a model-owned buffer (so every block reads memory whose
+    // address is fixed at build time); token and CTR batches are gathered from the frozen tables.
+    const void* z0 = nullptr;
+    {
+      void* buf = act_buf((size_t)m->rows * s.width);
+      z0 = buf;
+      if (s.input == ERASE_IN_DENSE) {
+        size_t bytes = (size_t)m->rows * s.width * m->esz;
+        m->stage.push_back({[=](cudaStream_t st) { return cudaMemcpyAsync(buf, mm->cur.x, bytes, cudaMemcpyDeviceToDevice, st); }, 0});
+        note(m->stage, "copy_input", 0, 2.0 * bytes);
+      } else if (s.input == ERASE_IN_TOKENS) {
+        const float* tok = m->frozen + m->tensors[0].off;
+        const float* pos = m->frozen + m->tensors[1].off;
+        int batch = s.batch, T_ = s.seq, d = s.width;
+        m->stage.push_back({[=](cudaStream_t st) { return gather_tokens(tok, pos, mm->cur.ids, buf, batch, T_, d, bf, st); }, 1});
+        note(m->stage, "gather_tokens", (double)m->rows * d, (double)m->rows * d * (4 + m->esz));
+      } else {
+        const float* tables = m->frozen;
+        long long stride = s.n_sparse > 1 ? (long long)(m->tensors[1].off - m->tensors[0].off) : 0;
+        int batch = s.batch, ns = s.n_sparse, e_ = s.emb_dim, nd = s.n_dense, w0 = s.width;
+        m->stage.push_back({[=](cudaStream_t st) {
+                              return gather_ctr(tables, stride, mm->cur.ids, (const float*)mm->cur.x, buf, batch, ns, e_, nd, w0, bf, st);
+                            }, 1});
+        note(m->stage, "gather_ctr", 0, (double)m->rows * w0 * (4 + m->esz));
+      }
+    }
+    int first = 0;
+    while (first < (int)m->tensors.size() && m->tensors[first].block < 0) first++;
+    m->fwd.resize(m->B);
+    m->bwd.resize(m->B);
+    const void* z = z0;
+    for (int b = 0; b < m->B; b++) {
+      const erase_block_spec& k = m->blocks[b];
+      const void* zin = s.topo == ERASE_TOPO_PARALLEL ? z0 : z;
+      void* zout = nullptr;
+      switch (k.kind) {
+        case ERASE_BLK_MLP:
+        case ERASE_BLK_TOWER: zout = block_mlp(b, k, zin, first, m->fwd[b], m->bwd[b]); break;
+        case ERASE_BLK_TRANSFORMER: zout = block_transformer(b, k, zin, first, m->fwd[b], m->bwd[b]); break;
+        case ERASE_BLK_CROSS: zout = block_cross(b, k, zin, first, m->fwd[b], m->bwd[b]); break;
+        case ERASE_BLK_DOT: zout = block_dot(b, k, zin, first, m->fwd[b], m->bwd[b]); break;
+      }
+      z = zout;
+      while (first < (int)m->tensors.size() && m->tensors[first].block == b) first++;
+    }
+    // optimizer: one sweep over the flat parameter arena
+    {
+      float* th = m->theta; float* gr = m->grad; float* m1 = m->mom1; float* m2 = m->mom2;
+      void* sh = m->shadow; double* tick = m->tick;
+      long long n = (long long)m->train_n;
+      int kind = s.opt;
+      float lr = s.lr, b1 = s.beta1, b2 = s.beta2, eps = s.eps, wd = s.weight_decay;
+      m->opt.push_back({[=](cudaStream_t st) { return opt_tick(tick, b1, b2, st); }, 1});
+      note(m->opt, "opt_tick");
+      m->opt.push_back({[=](cudaStream_t st) { return opt_update(th, gr, m1, m2, sh, n, kind, lr, b1, b2, eps, wd, tick, st); }, 1});
+      note(m->opt, "opt_update", 10.0 * n, (double)n * (kind == ERASE_OPT_SGD ? 12 : 28) + (sh ? 2.0 * n : 0));
+    }
+    return ok;
+  }
+};
+
+erase_status init_model(erase_model* m, const erase_model_spec* spec, bool dry) {
+  m->spec = *spec;
+  m->blocks.assign(spec->blocks, spec->blocks + spec->n_blocks);
+  m->spec.blocks = m->blocks.data();
+  m->B = spec->n_blocks;
+  m->bf16 = spec->dtype == ERASE_BF16;
+  m->esz = m->bf16 ? 2 : 4;
+  m->rows = spec->batch * (spec->input == ERASE_IN_TOKENS ? spec->seq : 1);
+  m->dry = dry;
+  if (!dry && spec->arena) {
+    m->arena = (char*)spec->arena;
+    m->arena_bytes = spec->arena_bytes;
+  }
+  build_tensor_table(m);
+  Builder bld;
+  bld.m = m;
+  if (!bld.build()) return m->fail(ERASE_ENOMEM, m->arena ? "arena too small" : "device allocation failed");
+  return ERASE_OK;
+}
+
+int tensor_check(erase_model* m, int32_t idx, size_t n) {
+  return m && idx >= 0 && idx < (int)m->tensors.size() && m->tensors[idx].n == n;
+}
+
+cudaError_t run_ops(erase_model* m, OpList& ops, cudaStream_t s) {
+  for (Op& op : ops) {
+    cudaError_t e = op.fn(s);
+    if (e != cudaSuccess) return e;
+    m->launches += op.launches;
+  }
+  return cudaSuccess;
+}
+
+// Enqueue one step.  `timed` adds the per-phase timing events (never while capturing).
+erase_status enqueue_step(erase_model* m, int n_streams, unsigned flags, bool timed) {
+  const int B = m->B;
+  const bool do_opt = !(flags & ERASE_NO_OPT);
+  auto tev = [&](int i) { return m->ev_time[i]; };
+  if (timed) CK(cudaEventRecord(tev(2 * (2 * B + 1)), m->main));
+  CK(run_ops(m, m->stage, m->main));
+  if (n_streams <= 1) {
+    for (int b = 0; b < B; b++) {
+      if (timed) CK(cudaEventRecord(tev(2 * b), m->main));
+      CK(run_ops(m, m->fwd[b], m->main));
+      if (timed) CK(cudaEventRecord(tev(2 * b + 1), m->main));
+    }
+    for (int b = B - 1; b >= 0; b--) {
+      if (timed) CK(cudaEventRecord(tev(2 * (B + b)), m->main));
+      CK(run_ops(m, m->bwd[b], m->main));
+      if (timed) CK(cudaEventRecord(tev(2 * (B + b) + 1), m->main));
+    }
+  } else {
+    const int ns = n_streams - 1;
+    for (int b = 0; b < B; b++) {
+      if (timed) CK(cudaEventRecord(tev(2 * b), m->main));
+      CK(run_ops(m, m->fwd[b], m->main));
+      if (timed) CK(cudaEventRecord(tev(2 * b + 1), m->main));
+      CK(cudaEventRecord(m->ev_f[b], m->main));          // F_b and l_b are enqueued: release B_b
+      cudaStream_t sd = m->side[b % ns];
+      CK(cudaStreamWaitEvent(sd, m->ev_f[b], 0));
+      if (timed) CK(cudaEventRecord(tev(2 * (B + b)), sd));
+      CK(run_ops(m, m->bwd[b], sd));
+      if (timed) CK(cudaEventRecord(tev(2 * (B + b) + 1), sd));
+      CK(cudaEventRecord(m->ev_b[b], sd));
+    }
+    for (int b = 0; b < B; b++) CK(cudaStreamWaitEvent(m->main, m->ev_b[b], 0));  // join
+  }
+  if (timed) CK(cudaEventRecord(tev(4 * B), m->main));
+  if (do_opt) CK(run_ops(m, m->opt, m->main));
+  if (timed) CK(cudaEventRecord(tev(4 * B + 1), m->main));
+  return ERASE_OK;
+}
+
+}  // namespace
+
+// =================================================================================================
+// C ABI
+// =================================================================================================
+extern "C" {
+
+size_t erase_arena_bytes(const erase_model_spec* spec) {
+  std::string why;
+  if (!validate(spec, &why)) return 0;
+  erase_model tmp;
+  if (init_model(&tmp, spec, true) != ERASE_OK) return 0;
+  return tmp.arena_used + 4096;
+}
+
+erase_status erase_create(const erase_model_spec* spec, erase_model** out) {
+  if (!out) { g_create_error = "out is NULL"; return ERASE_EINVAL; }
+  std::string why;
+  if (!validate(spec, &why)) { g_create_error = "invalid spec: " + why; return ERASE_EINVAL; }
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) {
+    cudaGetLastError();
+    g_create_error = "no CUDA device";
+    return ERASE_ECUDA;
+  }
+  erase_model* m = new (std::nothrow) erase_model();
+  if (!m) { g_create_error = "host allocation failed"; return ERASE_ENOMEM; }
+  erase_status st = init_model(m, spec, false);
+  auto bail = [&](erase_status s, const std::string& msg) {
+    g_create_error = msg;
+    erase_destroy(m);
+    return s;
+  };
+  if (st != ERASE_OK) return bail(st, m->err);
+  if (cudaStreamCreateWithFlags(&m->main, cudaStreamNonBlocking) != cudaSuccess) return bail(ERASE_ECUDA, "stream creation failed");
+  m->side.resize(m->B);
+  for (int i = 0; i < m->B; i++)
+    if (cudaStreamCreateWithFlags(&m->side[i], cudaStreamNonBlocking) != cudaSuccess) { m->side.resize(i); return bail(ERASE_ECUDA, "stream creation failed"); }
+  auto mk = [&](cudaEvent_t* e, unsigned fl) { return cudaEventCreateWithFlags(e, fl) == cudaSuccess; };
+  m->ev_f.assign(m->B, nullptr);
+  m->ev_b.assign(m->B, nullptr);
+  for (int i = 0; i < m->B; i++)
+    if (!mk(&m->ev_f[i], cudaEventDisableTiming) || !mk(&m->ev_b[i], cudaEventDisableTiming)) return bail(ERASE_ECUDA, "event creation failed");
+  if (!mk(&m->ev_opt, cudaEventDisableTiming)) return bail(ERASE_ECUDA, "event creation failed");
+  m->ev_time.assign(2 * (2 * m->B + 1) + 1, nullptr);
+  for (auto& e : m->ev_time)
+    if (!mk(&e, cudaEventDefault)) return bail(ERASE_ECUDA, "event creation failed");
+  if (cudaDeviceSynchronize() != cudaSuccess) return bail(ERASE_ECUDA, "device error after model set-up");
+  *out = m;
+  return ERASE_OK;
+}
+
+void erase_destroy(erase_model* m) {
+  if (!m) return;
+  if (m->main) cudaStreamSynchronize(m->main);
+  for (auto s : m->side) if (s) cudaStreamSynchronize(s);
+  for (auto& kv : m->graphs) cudaGraphExecDestroy(kv.second);
+  for (auto e : m->ev_f) if (e) cudaEventDestroy(e);
+  for (auto e : m->ev_b) if (e) cudaEventDestroy(e);
+  for (auto e : m->ev_time) if (e) cudaEventDestroy(e);
+  for (auto e : m->ev_prof) if (e) cudaEventDestroy(e);
+  if (m->ev_opt) cudaEventDestroy(m->ev_opt);
+  for (auto s : m->side) if (s) cudaStreamDestroy(s);
+  if (m->main) cudaStreamDestroy(m->main);
+  for (void* p : m->owned) cudaFree(p);
+  cudaGetLastError();
+  delete m;
+}
+
+int32_t erase_num_tensors(const erase_model* m) { return m ? (int32_t)m->tensors.size() : 0; }
+
+erase_status erase_tensor_info(const erase_model* m, int32_t idx, int32_t* block, char name[32], int32_t* rank,
+                               int64_t shape[4], int32_t* trainable) {
+  if (!m || idx < 0 || idx >= (int)m->tensors.size()) return ERASE_EINVAL;
+  const Tensor& t = m->tensors[idx];
+  if (block) *block = t.block;
+  if (name) { std::strncpy(name, t.name.c_str(), 31); name[31] = 0; }
+  if (rank) *rank = t.rank;
+  if (shape) { shape[0] = t.shape[0]; shape[1] = t.rank > 1 ? t.shape[1] : 0; shape[2] = shape[3] = 0; }
+  if (trainable) *trainable = t.trainable ? 1 : 0;
+  return ERASE_OK;
+}
+
+erase_status erase_sync(erase_model* m) {
+  if (!m) return ERASE_EINVAL;
+  CK(cudaStreamSynchronize(m->main));
+  for (auto s : m->side) CK(cudaStreamSynchronize(s));
+  return ERASE_OK;
+}
+
+erase_status erase_set_params(erase_model* m, int32_t idx, const float* src, size_t n) {
+  if (!m) return ERASE_EINVAL;
+  if (!src || !tensor_check(m, idx, n)) return m->fail(ERASE_EINVAL, "erase_set_params: bad index, size or pointer");
+  erase_status st = erase_sync(m);
+  if (st != ERASE_OK) return st;
+  Tensor& t = m->tensors[idx];
+  float* dst = (t.trainable ? m->theta : m->frozen) + t.off;
+  CK(copy_sync(m, dst, src, n * sizeof(float), cudaMemcpyHostToDevice));
+  if (t.trainable && m->shadow) {
+    CK(to_bf16(dst, (__nv_bfloat16*)m->shadow + t.off, (long long)n, m->main));
+    m->launches++;
+    CK(cudaStreamSynchronize(m->main));
+  }
+  t.set = true;
+  return ERASE_OK;
+}
+
+static erase_status copy_out(erase_model* m, int32_t idx, float* dst, size_t n, const float* base_train, const float* base_frozen, const char* who) {
+  if (!m) return ERASE_EINVAL;
+  if (!dst || !tensor_check(m, idx, n)) return m->fail(ERASE_EINVAL, std::string(who) + ": bad index, size or pointer");
+  const Tensor& t = m->tensors[idx];
+  const float* base = t.trainable ? base_train : base_frozen;
+  if (!base) return m->fail(ERASE_EINVAL, std::string(who) + ": tensor has no such data");
+  erase_status st = erase_sync(m);
+  if (st != ERASE_OK) return st;
+  CK(copy_sync(m, dst, base + t.off, n * sizeof(float), cudaMemcpyDeviceToHost));
+  return ERASE_OK;
+}
+
+erase_status erase_params(erase_model* m, int32_t idx, float* dst, size_t n) {
+  return copy_out(m, idx, dst, n, m ? m->theta : nullptr, m ? m->frozen : nullptr, "erase_params");
+}
+erase_status erase_grads(erase_model* m, int32_t idx, float* dst, size_t n) {
+  return copy_out(m, idx, dst, n, m ? m->grad : nullptr, nullptr, "erase_grads");
+}
+
+erase_status erase_opt_state(erase_model* m, int32_t idx, float* mom1, float* mom2, size_t n, int64_t* t) {
+  if (!m) return ERASE_EINVAL;
+  if (!tensor_check(m, idx, n) || !m->tensors[idx].trainable) return m->fail(ERASE_EINVAL, "erase_opt_state: bad index or size");
+  erase_status st = erase_sync(m);
+  if (st != ERASE_OK) return st;
+  const Tensor& tt = m->tensors[idx];
+  if (mom1) { if (m->mom1) CK(copy_sync(m, mom1, m->mom1 + tt.off, n * 4, cudaMemcpyDeviceToHost)); else std::memset(mom1, 0, n * 4); }
+  if (mom2) { if (m->mom2) CK(copy_sync(m, mom2, m->mom2 + tt.off, n * 4, cudaMemcpyDeviceToHost)); else std::memset(mom2, 0, n * 4); }
+  if (t) {
+    double tk[3];
+    CK(copy_sync(m, tk, m->tick, sizeof(tk), cudaMemcpyDeviceToHost));
+    *t = (int64_t)tk[0];
+  }
+  return ERASE_OK;
+}
+
+erase_status erase_set_opt_state(erase_model* m, int32_t idx, const float* mom1, const float* mom2, size_t n, int64_t t) {
+  if (!m) return ERASE_EINVAL;
+  if (!tensor_check(m, idx, n) || !m->tensors[idx].trainable || t < 0) return m->fail(ERASE_EINVAL, "erase_set_opt_state: bad index, size or t");
+  erase_status st = erase_sync(m);
+  if (st != ERASE_OK) return st;
+  const Tensor& tt = m->tensors[idx];
+  if (mom1 && m->mom1) CK(copy_sync(m, m->mom1 + tt.off, mom1, n * 4, cudaMemcpyHostToDevice));
+  if (mom2 && m->mom2) CK(copy_sync(m, m->mom2 + tt.off, mom2, n * 4, cudaMemcpyHostToDevice));
+  double tk[3] = {(double)t, 1.0 - std::pow((double)m->spec.beta1, (double)t), 1.0 - std::pow((double)m->spec.beta2, (double)t)};
+  CK(copy_sync(m, m->tick, tk, sizeof(tk), cudaMemcpyHostToDevice));
+  return ERASE_OK;
+}
+
+static erase_status check_step_args(erase_model* m, const erase_batch* batch);
+
+erase_status erase_step_ex(erase_model* m, const erase_batch* batch, int32_t n_streams, uint32_t flags) {
+  if (!m) return ERASE_EINVAL;
+  if (n_streams < 1) return m->fail(ERASE_EINVAL, "erase_step: n_streams must be >= 1");
+  if (flags & ~(ERASE_GRAPH | ERASE_NO_OPT)) return m->fail(ERASE_EINVAL, "erase_step: unknown flag");
+  erase_status cst = check_step_args(m, batch);
+  if (cst != ERASE_OK) return cst;
+  if (n_streams > m->B + 1) n_streams = m->B + 1;
+  m->cur = *batch;
+  if (flags & ERASE_GRAPH) {
+    GraphKey key{batch->x, batch->ids, batch->y, n_streams, flags};
+    auto it = m->graphs.find(key);
+    if (it == m->graphs.end()) {
+      int64_t before = m->launches;
+      CK(cudaStreamBeginCapture(m->main, cudaStreamCaptureModeThreadLocal));
+      erase_status st = enqueue_step(m, n_streams, flags, false);
+      cudaGraph_t graph = nullptr;
+      cudaError_t e = cudaStreamEndCapture(m->main, &graph);
+      m->launches = before;
+      if (st != ERASE_OK) { if (graph) cudaGraphDestroy(graph); cudaGetLastError(); return st; }
+      if (e != cudaSuccess) return m->fail(ERASE_ECUDA, std::string("graph capture: ") + cudaGetErrorString(e));
+      cudaGraphExec_t exec = nullptr;
+      e = cudaGraphInstantiate(&exec, graph, 0);
+      cudaGraphDestroy(graph);
+      if (e != cudaSuccess) return m->fail(ERASE_ECUDA, std::string("graph instantiate: ") + cudaGetErrorString(e));
+      it = m->graphs.emplace(key, exec).first;
+    }
+    CK(cudaGraphLaunch(it->second, m->main));
+    int64_t per = 0;
+    for (auto& op : m->stage) per += op.launches;
+    for (int b = 0; b < m->B; b++) {
+      for (auto& op : m->fwd[b]) per += op.launches;
+      for (auto& op : m->bwd[b]) per += op.launches;
+    }
+    if (!(flags & ERASE_NO_OPT)) for (auto& op : m->opt) per += op.launches;
+    m->launches += per;
+    m->timeline_valid = false;
+  } else {
+    erase_status st = enqueue_step(m, n_streams, flags, true);
+    if (st != ERASE_OK) return st;
+    m->timeline_valid = true;
+  }
+  m->stepped = true;
+  return ERASE_OK;
+}
+
+static erase_status check_step_args(erase_model* m, const erase_batch* batch) {
+  if (!batch) return m->fail(ERASE_EINVAL, "erase_step: batch is NULL");
+  const erase_model_spec& s = m->spec;
+  bool need_x = s.input != ERASE_IN_TOKENS, need_ids = s.input != ERASE_IN_DENSE, need_y = s.input != ERASE_IN_TOKENS;
+  if ((need_x && !batch->x) || (need_ids && !batch->ids) || (need_y && !batch->y))
+    return m->fail(ERASE_EINVAL, "erase_step: a batch pointer this input kind needs is NULL");
+  for (const Tensor& t : m->tensors)
+    if (!t.set) return m->fail(ERASE_ESTATE, "erase_step: tensor '" + t.name + "' was never set");
+  return ERASE_OK;
+}
+
+erase_status erase_profile_step(erase_model* m, const erase_batch* batch, erase_op_record* out, int32_t cap, int32_t* n) {
+  if (!m) return ERASE_EINVAL;
+  if (!out || !n || cap < 0) return m->fail(ERASE_EINVAL, "erase_profile_step: out or n is NULL");
+  erase_status st = check_step_args(m, batch);
+  if (st != ERASE_OK) return st;
+  m->cur = *batch;
+  struct Ref { Op* op; int block, phase; };
+  std::vector<Ref> refs;
+  for (auto& op : m->stage) refs.push_back({&op, -1, 0});
+  for (int b = 0; b < m->B; b++) for (auto& op : m->fwd[b]) refs.push_back({&op, b, 1});
+  for (int b = m->B - 1; b >= 0; b--) for (auto& op : m->bwd[b]) refs.push_back({&op, b, 2});
+  for (auto& op : m->opt) refs.push_back({&op, -1, 3});
+  while (m->ev_prof.size() < 2 * refs.size()) {
+    cudaEvent_t e;
+    CK(cudaEventCreate(&e));
+    m->ev_prof.push_back(e);
+  }
+  for (size_t i = 0; i < refs.size(); i++) {
+    CK(cudaEventRecord(m->ev_prof[2 * i], m->main));
+    CK(refs[i].op->fn(m->main));
+    m->launches += refs[i].op->launches;
+    CK(cudaEventRecord(m->ev_prof[2 * i + 1], m->main));
+  }
+  CK(cudaStreamSynchronize(m->main));
+  m->stepped = true;
+  m->timeline_valid = false;
+  *n = (int32_t)refs.size();
+  for (size_t i = 0; i < refs.size() && (int32_t)i < cap; i++) {
+    erase_op_record& r = out[i];
+    std::memset(&r, 0, sizeof(r));
+    std::strncpy(r.name, refs[i].op->name, 31);
+    r.block = refs[i].block;
+    r.phase = refs[i].phase;
+    r.launches = refs[i].op->launches;
+    r.flops = refs[i].op->flops;
+    r.bytes = refs[i].op->bytes;
+    CK(cudaEventElapsedTime(&r.ms, m->ev_prof[2 * i], m->ev_prof[2 * i + 1]));
+  }
+  return ERASE_OK;
+}
+
+erase_status erase_step(erase_model* m, const erase_batch* batch, int32_t n_streams) {
+  return erase_step_ex(m, batch, n_streams, 0);
+}
+
+erase_status erase_losses(erase_model* m, float* dst, int32_t n_blocks) {
+  if (!m) return ERASE_EINVAL;
+  if (!dst || n_blocks != m->B) return m->fail(ERASE_EINVAL, "erase_losses: dst is NULL or n_blocks differs from the model's");
+  if (!m->stepped) return m->fail(ERASE_ESTATE, "erase_losses: no step has run");
+  erase_status st = erase_sync(m);
+  if (st != ERASE_OK) return st;
+  CK(copy_sync(m, dst, m->losses, m->B * sizeof(float), cudaMemcpyDeviceToHost));
+  return ERASE_OK;
+}
+
+void* erase_main_stream(erase_model* m) { return m ? (void*)m->main : nullptr; }
+
+int64_t erase_launch_count(const erase_model* m) { return m ? m->launches : 0; }
+
+erase_status erase_timeline(erase_model* m, float* out, int32_t n) {
+  if (!m) return ERASE_EINVAL;
+  const int need = 2 * (2 * m->B + 1);
+  if (!out || n != need) return m->fail(ERASE_EINVAL, "erase_timeline: out is NULL or n != 2*(2*n_blocks+1)");
+  if (!m->timeline_valid) return m->fail(ERASE_ESTATE, "erase_timeline: the last step recorded no timeline");
+  erase_status st = erase_sync(m);
+  if (st != ERASE_OK) return st;
+  for (int i = 0; i < need; i++) CK(cudaEventElapsedTime(&out[i], m->ev_time[need], m->ev_time[i]));
+  return ERASE_OK;
+}
+
+const char* erase_last_error(const erase_model* m) { return m ? m->err.c_str() : g_create_error.c_str(); }
+
+}  // extern "C"

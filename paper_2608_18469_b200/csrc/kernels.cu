@@ -1,0 +1,925 @@
+// Hand-written CUDA kernels (plain SIMT) of the ERASE step library: the general GEMM used for
+// fp32 models and for shapes the tensor-core path does not take, and every non-GEMM operation
+// of the step (LayerNorm, causal attention, losses, gathers, dot interaction, optimizer).
+// Reductions are fixed-partition / fixed-order: no floating-point atomics anywhere.
+#include "kernels.cuh"
+
+#include <cuda_bf16.h>
+#include <math.h>
+
+namespace erase {
+
+typedef __nv_bfloat16 bf16_t;
+
+template <typename T> __device__ __forceinline__ float ldf(const T* p);
+template <> __device__ __forceinline__ float ldf<float>(const float* p) { return *p; }
+template <> __device__ __forceinline__ float ldf<bf16_t>(const bf16_t* p) { return __bfloat162float(*p); }
+template <typename T> __device__ __forceinline__ void stf(T* p, float v);
+template <> __device__ __forceinline__ void stf<float>(float* p, float v) { *p = v; }
+template <> __device__ __forceinline__ void stf<bf16_t>(bf16_t* p, float v) { *p = __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float act_apply(int act, float v) {
+  if (act == ACT_RELU) return v > 0.f ? v : 0.f;
+  if (act == ACT_GELU) return v * 0.5f * (1.f + erff(v * 0.70710678118654752f));
+  return v;
+}
+// derivative of the activation; GELU takes the pre-activation, ReLU accepts either the
+// pre-activation or the output (same sign test; 0 at exactly 0).
+__device__ __forceinline__ float act_deriv(int act, float u) {
+  if (act == ACT_RELU) return u > 0.f ? 1.f : 0.f;
+  if (act == ACT_GELU) {
+    float cdf = 0.5f * (1.f + erff(u * 0.70710678118654752f));
+    float pdf = 0.39894228040143268f * expf(-0.5f * u * u);
+    return cdf + u * pdf;
+  }
+  return 1.f;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+static inline unsigned cdiv(long long a, long long b) { return (unsigned)((a + b - 1) / b); }
+
+// ------------------------------------------------------------------------------------------
+// general GEMM, 64x64x16 tiles, 256 threads, 4x4 outputs per thread, fp32 FMA
+// ------------------------------------------------------------------------------------------
+template <typename T, bool AK, bool BK>
+__global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
+  __shared__ __align__(16) float As[16][68];
+  __shared__ __align__(16) float Bs[16][68];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64, split = blockIdx.z;
+  const int kchunk = (((g.K + g.splits - 1) / g.splits) + 15) / 16 * 16;
+  const int kbeg = split * kchunk;
+  const int kend = min(g.K, kbeg + kchunk);
+  const T* A = (const T*)g.A;
+  const T* B = (const T*)g.B;
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; i++)
+#pragma unroll
+    for (int j = 0; j < 4; j++) acc[i][j] = 0.f;
+
+  for (int k0 = kbeg; k0 < kend; k0 += 16) {
+#pragma unroll
+    for (int it = 0; it < 4; it++) {
+      int i = tid + it * 256;
+      int mm, kk;
+      if (AK) { kk = i & 15; mm = i >> 4; } else { mm = i & 63; kk = i >> 6; }
+      int gm = m0 + mm, gk = k0 + kk;
+      float v = 0.f;
+      if (gm < g.M && gk < kend) v = ldf(A + (long long)gm * g.sa_m + (long long)gk * g.sa_k);
+      As[kk][mm] = v;
+      int nn;
+      if (BK) { kk = i & 15; nn = i >> 4; } else { nn = i & 63; kk = i >> 6; }
+      int gn = n0 + nn;
+      gk = k0 + kk;
+      v = 0.f;
+      if (gn < g.N && gk < kend) v = ldf(B + (long long)gn * g.sb_n + (long long)gk * g.sb_k);
+      Bs[kk][nn] = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < 16; kk++) {
+      float4 a4 = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+      float4 b4 = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+      float a[4] = {a4.x, a4.y, a4.z, a4.w};
+      float b[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+      for (int i = 0; i < 4; i++)
+#pragma unroll
+        for (int j = 0; j < 4; j++) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+
+  const Epilogue& e = g.epi;
+#pragma unroll
+  for (int i = 0; i < 4; i++) {
+    int m = m0 + ty * 4 + i;
+    if (m >= g.M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+      int n = n0 + tx * 4 + j;
+      if (n >= g.N) continue;
+      float v = acc[i][j];
+      if (g.splits > 1) {
+        g.ws[(long long)split * g.M * g.N + (long long)m * g.N + n] = v;
+        continue;
+      }
+      v *= e.alpha;
+      if (e.bias) v += e.bias[n];
+      long long ia = (long long)m * e.ld_aux + n;
+      if (e.pre_out) stf((T*)e.pre_out + ia, v);
+      v = act_apply(e.act, v);
+      if (e.mul) v *= ldf((const T*)e.mul + ia);
+      if (e.res) v += ldf((const T*)e.res + ia);
+      if (e.dact != ACT_NONE) v *= act_deriv(e.dact, ldf((const T*)e.dact_src + ia));
+      long long ic = (long long)m * g.ldc + n;
+      if (g.c_f32) ((float*)g.C)[ic] = v; else stf((T*)g.C + ic, v);
+    }
+  }
+}
+
+template <typename T>
+static cudaError_t gemm_simt_t(const GemmArgs& g, cudaStream_t s) {
+  dim3 grid(cdiv(g.N, 64), cdiv(g.M, 64), g.splits);
+  bool ak = g.sa_k == 1, bk = g.sb_k == 1;
+  if (ak && bk) gemm_simt_kernel<T, true, true><<<grid, 256, 0, s>>>(g);
+  else if (ak && !bk) gemm_simt_kernel<T, true, false><<<grid, 256, 0, s>>>(g);
+  else if (!ak && bk) gemm_simt_kernel<T, false, true><<<grid, 256, 0, s>>>(g);
+  else gemm_simt_kernel<T, false, false><<<grid, 256, 0, s>>>(g);
+  return cudaGetLastError();
+}
+
+cudaError_t gemm_simt(const GemmArgs& g, bool bf16, cudaStream_t s) {
+  if (g.M <= 0 || g.N <= 0) return cudaSuccess;
+  return bf16 ? gemm_simt_t<bf16_t>(g, s) : gemm_simt_t<float>(g, s);
+}
+
+__global__ void splitk_reduce_kernel(const float* __restrict__ ws, int splits, long long mn, int N,
+                                     float* __restrict__ out, long long ldo) {
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= mn) return;
+  float a = 0.f;
+  for (int s = 0; s < splits; s++) a += ws[(long long)s * mn + i];
+  out[(i / N) * ldo + (i % N)] = a;
+}
+
+cudaError_t splitk_reduce(const float* ws, int splits, long long mn, int N, float* out, long long ldo,
+                          cudaStream_t s) {
+  if (mn <= 0) return cudaSuccess;
+  splitk_reduce_kernel<<<cdiv(mn, 256), 256, 0, s>>>(ws, splits, mn, N, out, ldo);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// column sums (bias gradients, head weight gradient of the BCE head)
+// ------------------------------------------------------------------------------------------
+int colsum_chunks(int rows, int cols) {
+  int strips = (cols + 31) / 32;
+  int want = (296 + strips - 1) / strips;
+  int maxc = rows / 64;
+  if (maxc < 1) maxc = 1;
+  if (want > maxc) want = maxc;
+  if (want < 1) want = 1;
+  return want;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) colsum_kernel(const T* __restrict__ X, long long ldx, int rows,
+                                                     int cols, const float* __restrict__ scale,
+                                                     float* __restrict__ dst, int chunks) {
+  __shared__ float sm[8][33];
+  int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
+  int c = blockIdx.x * 32 + cx;
+  int per = (rows + chunks - 1) / chunks;
+  int rb = blockIdx.y * per, re = min(rows, rb + per);
+  float a = 0.f;
+  if (c < cols)
+    for (int r = rb + ry; r < re; r += 8) {
+      float v = ldf(X + (long long)r * ldx + c);
+      if (scale) v *= scale[r];
+      a += v;
+    }
+  sm[ry][cx] = a;
+  __syncthreads();
+  if (ry == 0 && c < cols) {
+    float t = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; i++) t += sm[i][cx];
+    dst[(long long)blockIdx.y * cols + c] = t;
+  }
+}
+
+cudaError_t colsum(const void* X, bool x_bf16, long long ldx, int rows, int cols, const float* scale,
+                   float* ws, int chunks, float* out, cudaStream_t s) {
+  dim3 grid(cdiv(cols, 32), chunks);
+  float* dst = chunks == 1 ? out : ws;
+  if (x_bf16) colsum_kernel<bf16_t><<<grid, 256, 0, s>>>((const bf16_t*)X, ldx, rows, cols, scale, dst, chunks);
+  else colsum_kernel<float><<<grid, 256, 0, s>>>((const float*)X, ldx, rows, cols, scale, dst, chunks);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess || chunks == 1) return e;
+  return splitk_reduce(ws, chunks, cols, cols, out, cols, s);
+}
+
+// ------------------------------------------------------------------------------------------
+// LayerNorm
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) layernorm_fwd_kernel(const T* __restrict__ x, const float* __restrict__ gain,
+                                                            const float* __restrict__ shift, T* __restrict__ y,
+                                                            float* __restrict__ mean, float* __restrict__ rstd,
+                                                            int rows, int d) {
+  int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  const T* xr = x + (long long)row * d;
+  float s = 0.f;
+  for (int c = lane; c < d; c += 32) s += ldf(xr + c);
+  float mu = warp_sum(s) / d;
+  float q = 0.f;
+  for (int c = lane; c < d; c += 32) { float t = ldf(xr + c) - mu; q += t * t; }
+  float r = rsqrtf(warp_sum(q) / d + 1e-5f);
+  for (int c = lane; c < d; c += 32)
+    stf(y + (long long)row * d + c, (ldf(xr + c) - mu) * r * gain[c] + shift[c]);
+  if (lane == 0) { mean[row] = mu; rstd[row] = r; }
+}
+
+cudaError_t layernorm_fwd(const void* x, const float* gain, const float* shift, void* y, float* mean,
+                          float* rstd, int rows, int d, bool bf16, cudaStream_t s) {
+  if (bf16) layernorm_fwd_kernel<bf16_t><<<cdiv(rows, 8), 256, 0, s>>>((const bf16_t*)x, gain, shift, (bf16_t*)y, mean, rstd, rows, d);
+  else layernorm_fwd_kernel<float><<<cdiv(rows, 8), 256, 0, s>>>((const float*)x, gain, shift, (float*)y, mean, rstd, rows, d);
+  return cudaGetLastError();
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) layernorm_bwd_dx_kernel(const T* __restrict__ dy, const T* __restrict__ x,
+                                                               const float* __restrict__ gain,
+                                                               const float* __restrict__ mean,
+                                                               const float* __restrict__ rstd, const T* add,
+                                                               T* dx, int rows, int d) {
+  int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  long long o = (long long)row * d;
+  float mu = mean[row], r = rstd[row];
+  float s1 = 0.f, s2 = 0.f;
+  for (int c = lane; c < d; c += 32) {
+    float g = ldf(dy + o + c) * gain[c];
+    float xh = (ldf(x + o + c) - mu) * r;
+    s1 += g;
+    s2 += g * xh;
+  }
+  s1 = warp_sum(s1) / d;
+  s2 = warp_sum(s2) / d;
+  for (int c = lane; c < d; c += 32) {
+    float g = ldf(dy + o + c) * gain[c];
+    float xh = (ldf(x + o + c) - mu) * r;
+    float v = r * (g - s1 - xh * s2);
+    if (add) v += ldf(add + o + c);
+    stf(dx + o + c, v);
+  }
+}
+
+cudaError_t layernorm_bwd_dx(const void* dy, const void* x, const float* gain, const float* mean,
+                             const float* rstd, const void* add, void* dx, int rows, int d, bool bf16,
+                             cudaStream_t s) {
+  if (bf16) layernorm_bwd_dx_kernel<bf16_t><<<cdiv(rows, 8), 256, 0, s>>>((const bf16_t*)dy, (const bf16_t*)x, gain, mean, rstd, (const bf16_t*)add, (bf16_t*)dx, rows, d);
+  else layernorm_bwd_dx_kernel<float><<<cdiv(rows, 8), 256, 0, s>>>((const float*)dy, (const float*)x, gain, mean, rstd, (const float*)add, (float*)dx, rows, d);
+  return cudaGetLastError();
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) layernorm_param_grad_kernel(const T* __restrict__ dy, const T* __restrict__ x,
+                                                                   const float* __restrict__ mean,
+                                                                   const float* __restrict__ rstd,
+                                                                   float* __restrict__ dst_g, float* __restrict__ dst_b,
+                                                                   int rows, int d, int chunks) {
+  __shared__ float sg[8][33], sb[8][33];
+  int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
+  int c = blockIdx.x * 32 + cx;
+  int per = (rows + chunks - 1) / chunks;
+  int rb = blockIdx.y * per, re = min(rows, rb + per);
+  float ag = 0.f, ab = 0.f;
+  if (c < d)
+    for (int r = rb + ry; r < re; r += 8) {
+      float g = ldf(dy + (long long)r * d + c);
+      float xh = (ldf(x + (long long)r * d + c) - mean[r]) * rstd[r];
+      ag += g * xh;
+      ab += g;
+    }
+  sg[ry][cx] = ag;
+  sb[ry][cx] = ab;
+  __syncthreads();
+  if (ry == 0 && c < d) {
+    float tg = 0.f, tb = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; i++) { tg += sg[i][cx]; tb += sb[i][cx]; }
+    dst_g[(long long)blockIdx.y * d + c] = tg;
+    dst_b[(long long)blockIdx.y * d + c] = tb;
+  }
+}
+
+cudaError_t layernorm_param_grad(const void* dy, const void* x, const float* mean, const float* rstd,
+                                 float* ws, int chunks, float* dgain, float* dshift, int rows, int d,
+                                 bool bf16, cudaStream_t s) {
+  dim3 grid(cdiv(d, 32), chunks);
+  float* pg = chunks == 1 ? dgain : ws;
+  float* pb = chunks == 1 ? dshift : ws + (long long)chunks * d;
+  if (bf16) layernorm_param_grad_kernel<bf16_t><<<grid, 256, 0, s>>>((const bf16_t*)dy, (const bf16_t*)x, mean, rstd, pg, pb, rows, d, chunks);
+  else layernorm_param_grad_kernel<float><<<grid, 256, 0, s>>>((const float*)dy, (const float*)x, mean, rstd, pg, pb, rows, d, chunks);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess || chunks == 1) return e;
+  e = splitk_reduce(pg, chunks, d, d, dgain, d, s);
+  if (e != cudaSuccess) return e;
+  return splitk_reduce(pb, chunks, d, d, dshift, d, s);
+}
+
+// ------------------------------------------------------------------------------------------
+// causal attention, flash-style (no T x T matrix in memory), fp32 SIMT
+// tiles of 32 queries x 32 keys; a warp owns 4 rows; lanes run over the 32 keys of a tile for
+// the scores and over head columns (lane, lane+32, ..) for the accumulators.
+// ------------------------------------------------------------------------------------------
+#define ATT_MAXC 4  // head width <= 128
+
+template <typename T>
+__device__ __forceinline__ void att_load_tile(float* dst, int ldk, const T* src, long long ld, int r0,
+                                              int T_, int dh) {
+  for (int i = threadIdx.x; i < 32 * dh; i += 256) {
+    int r = i / dh, c = i - r * dh;
+    int t = r0 + r;
+    dst[r * ldk + c] = t < T_ ? ldf(src + (long long)t * ld + c) : 0.f;
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) attn_fwd_kernel(const T* __restrict__ qkv, T* __restrict__ o,
+                                                       float* __restrict__ lse, int T_, int H, int dh,
+                                                       float scale) {
+  extern __shared__ float sm[];
+  const int ldk = dh + 1;
+  float* Qs = sm;
+  float* Ks = Qs + 32 * ldk;
+  float* Vs = Ks + 32 * ldk;
+  const int q0 = blockIdx.x * 32, h = blockIdx.y, b = blockIdx.z;
+  const int d = H * dh;
+  const long long ld = 3LL * d;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const T* base = qkv + (long long)b * T_ * ld + h * dh;
+  att_load_tile(Qs, ldk, base, ld, q0, T_, dh);
+  float mrow[4], lrow[4], acc[4][ATT_MAXC];
+#pragma unroll
+  for (int r = 0; r < 4; r++) {
+    mrow[r] = -INFINITY;
+    lrow[r] = 0.f;
+#pragma unroll
+    for (int cc = 0; cc < ATT_MAXC; cc++) acc[r][cc] = 0.f;
+  }
+  for (int j0 = 0; j0 <= q0; j0 += 32) {
+    __syncthreads();
+    att_load_tile(Ks, ldk, base + d, ld, j0, T_, dh);
+    att_load_tile(Vs, ldk, base + 2 * d, ld, j0, T_, dh);
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < 4; r++) {
+      const int il = warp * 4 + r, i = q0 + il;
+      if (i >= T_) continue;
+      const int j = j0 + lane;
+      float sc = 0.f;
+      for (int c = 0; c < dh; c++) sc = fmaf(Qs[il * ldk + c], Ks[lane * ldk + c], sc);
+      sc *= scale;
+      const bool valid = j <= i;
+      if (!valid) sc = -INFINITY;
+      float mnew = fmaxf(mrow[r], warp_max(sc));
+      float p = valid ? expf(sc - mnew) : 0.f;
+      float corr = expf(mrow[r] - mnew);
+      lrow[r] = lrow[r] * corr + warp_sum(p);
+      mrow[r] = mnew;
+#pragma unroll
+      for (int cc = 0; cc < ATT_MAXC; cc++) acc[r][cc] *= corr;
+      for (int jj = 0; jj < 32; jj++) {
+        float pj = __shfl_sync(0xffffffffu, p, jj);
+#pragma unroll
+        for (int cc = 0; cc < ATT_MAXC; cc++) {
+          int c = lane + 32 * cc;
+          if (c < dh) acc[r][cc] = fmaf(pj, Vs[jj * ldk + c], acc[r][cc]);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < 4; r++) {
+    const int i = q0 + warp * 4 + r;
+    if (i >= T_) continue;
+    float inv = 1.f / lrow[r];
+#pragma unroll
+    for (int cc = 0; cc < ATT_MAXC; cc++) {
+      int c = lane + 32 * cc;
+      if (c < dh) stf(o + ((long long)b * T_ + i) * d + h * dh + c, acc[r][cc] * inv);
+    }
+    if (lane == 0) lse[((long long)b * H + h) * T_ + i] = mrow[r] + logf(lrow[r]);
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) attn_delta_kernel(const T* __restrict__ o, const T* __restrict__ dout,
+                                                         float* __restrict__ delta, int rows, int T_, int H,
+                                                         int dh) {
+  // one warp per (row, head)
+  long long w = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  int lane = threadIdx.x & 31;
+  if (w >= (long long)rows * H) return;
+  int n = (int)(w / H), h = (int)(w % H);
+  long long off = (long long)n * H * dh + h * dh;
+  float s = 0.f;
+  for (int c = lane; c < dh; c += 32) s += ldf(o + off + c) * ldf(dout + off + c);
+  s = warp_sum(s);
+  if (lane == 0) {
+    int b = n / T_, t = n % T_;
+    delta[((long long)b * H + h) * T_ + t] = s;
+  }
+}
+
+// dK, dV for a tile of 32 keys: loop over the query tiles at or after it.
+template <typename T>
+__global__ void __launch_bounds__(256) attn_bwd_kv_kernel(const T* __restrict__ qkv, const T* __restrict__ dout,
+                                                          const float* __restrict__ lse,
+                                                          const float* __restrict__ delta, T* __restrict__ dqkv,
+                                                          int T_, int H, int dh, float scale) {
+  extern __shared__ float sm[];
+  const int ldk = dh + 1;
+  float* Ks = sm;
+  float* Vs = Ks + 32 * ldk;
+  float* Qs = Vs + 32 * ldk;
+  float* Ds = Qs + 32 * ldk;
+  float* Ls = Ds + 32 * ldk;  // [32] lse
+  float* Es = Ls + 32;        // [32] delta
+  const int k0 = blockIdx.x * 32, h = blockIdx.y, b = blockIdx.z;
+  const int d = H * dh;
+  const long long ld = 3LL * d;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const T* base = qkv + (long long)b * T_ * ld + h * dh;
+  const T* dob = dout + (long long)b * T_ * d + h * dh;
+  att_load_tile(Ks, ldk, base + d, ld, k0, T_, dh);
+  att_load_tile(Vs, ldk, base + 2 * d, ld, k0, T_, dh);
+  float dk[4][ATT_MAXC], dv[4][ATT_MAXC];
+#pragma unroll
+  for (int r = 0; r < 4; r++)
+#pragma unroll
+    for (int cc = 0; cc < ATT_MAXC; cc++) dk[r][cc] = dv[r][cc] = 0.f;
+  for (int i0 = k0; i0 < T_; i0 += 32) {
+    __syncthreads();
+    att_load_tile(Qs, ldk, base, ld, i0, T_, dh);
+    att_load_tile(Ds, ldk, dob, (long long)d, i0, T_, dh);
+    if (threadIdx.x < 32) {
+      int i = i0 + threadIdx.x;
+      Ls[threadIdx.x] = i < T_ ? lse[((long long)b * H + h) * T_ + i] : 0.f;
+      Es[threadIdx.x] = i < T_ ? delta[((long long)b * H + h) * T_ + i] : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < 4; r++) {
+      const int jl = warp * 4 + r, j = k0 + jl;
+      if (j >= T_) continue;
+      const int i = i0 + lane;
+      float sc = 0.f, dp = 0.f;
+      for (int c = 0; c < dh; c++) {
+        sc = fmaf(Qs[lane * ldk + c], Ks[jl * ldk + c], sc);
+        dp = fmaf(Ds[lane * ldk + c], Vs[jl * ldk + c], dp);
+      }
+      const bool valid = i < T_ && j <= i;
+      float p = valid ? expf(sc * scale - Ls[lane]) : 0.f;
+      float ds = p * (dp - Es[lane]);
+      for (int ii = 0; ii < 32; ii++) {
+        float pi = __shfl_sync(0xffffffffu, p, ii);
+        float di = __shfl_sync(0xffffffffu, ds, ii);
+#pragma unroll
+        for (int cc = 0; cc < ATT_MAXC; cc++) {
+          int c = lane + 32 * cc;
+          if (c < dh) {
+            dv[r][cc] = fmaf(pi, Ds[ii * ldk + c], dv[r][cc]);
+            dk[r][cc] = fmaf(di, Qs[ii * ldk + c], dk[r][cc]);
+          }
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < 4; r++) {
+    const int j = k0 + warp * 4 + r;
+    if (j >= T_) continue;
+    T* row = dqkv + ((long long)b * T_ + j) * ld + h * dh;
+#pragma unroll
+    for (int cc = 0; cc < ATT_MAXC; cc++) {
+      int c = lane + 32 * cc;
+      if (c < dh) {
+        stf(row + d + c, dk[r][cc] * scale);
+        stf(row + 2 * d + c, dv[r][cc]);
+      }
+    }
+  }
+}
+
+// dQ for a tile of 32 queries: loop over the key tiles at or before it.
+template <typename T>
+__global__ void __launch_bounds__(256) attn_bwd_q_kernel(const T* __restrict__ qkv, const T* __restrict__ dout,
+                                                         const float* __restrict__ lse,
+                                                         const float* __restrict__ delta, T* __restrict__ dqkv,
+                                                         int T_, int H, int dh, float scale) {
+  extern __shared__ float sm[];
+  const int ldk = dh + 1;
+  float* Qs = sm;
+  float* Ds = Qs + 32 * ldk;
+  float* Ks = Ds + 32 * ldk;
+  float* Vs = Ks + 32 * ldk;
+  const int q0 = blockIdx.x * 32, h = blockIdx.y, b = blockIdx.z;
+  const int d = H * dh;
+  const long long ld = 3LL * d;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const T* base = qkv + (long long)b * T_ * ld + h * dh;
+  const T* dob = dout + (long long)b * T_ * d + h * dh;
+  att_load_tile(Qs, ldk, base, ld, q0, T_, dh);
+  att_load_tile(Ds, ldk, dob, (long long)d, q0, T_, dh);
+  float dq[4][ATT_MAXC], lrow[4], erow[4];
+#pragma unroll
+  for (int r = 0; r < 4; r++) {
+    int i = q0 + warp * 4 + r;
+    lrow[r] = i < T_ ? lse[((long long)b * H + h) * T_ + i] : 0.f;
+    erow[r] = i < T_ ? delta[((long long)b * H + h) * T_ + i] : 0.f;
+#pragma unroll
+    for (int cc = 0; cc < ATT_MAXC; cc++) dq[r][cc] = 0.f;
+  }
+  for (int j0 = 0; j0 <= q0; j0 += 32) {
+    __syncthreads();
+    att_load_tile(Ks, ldk, base + d, ld, j0, T_, dh);
+    att_load_tile(Vs, ldk, base + 2 * d, ld, j0, T_, dh);
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < 4; r++) {
+      const int il = warp * 4 + r, i = q0 + il;
+      if (i >= T_) continue;
+      const int j = j0 + lane;
+      float sc = 0.f, dp = 0.f;
+      for (int c = 0; c < dh; c++) {
+        sc = fmaf(Qs[il * ldk + c], Ks[lane * ldk + c], sc);
+        dp = fmaf(Ds[il * ldk + c], Vs[lane * ldk + c], dp);
+      }
+      float p = j <= i ? expf(sc * scale - lrow[r]) : 0.f;
+      float ds = p * (dp - erow[r]);
+      for (int jj = 0; jj < 32; jj++) {
+        float dj = __shfl_sync(0xffffffffu, ds, jj);
+#pragma unroll
+        for (int cc = 0; cc < ATT_MAXC; cc++) {
+          int c = lane + 32 * cc;
+          if (c < dh) dq[r][cc] = fmaf(dj, Ks[jj * ldk + c], dq[r][cc]);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < 4; r++) {
+    const int i = q0 + warp * 4 + r;
+    if (i >= T_) continue;
+    T* row = dqkv + ((long long)b * T_ + i) * ld + h * dh;
+#pragma unroll
+    for (int cc = 0; cc < ATT_MAXC; cc++) {
+      int c = lane + 32 * cc;
+      if (c < dh) stf(row + c, dq[r][cc] * scale);
+    }
+  }
+}
+
+template <typename K>
+static cudaError_t set_smem(K kernel, size_t bytes) {
+  if (bytes <= 48 * 1024) return cudaSuccess;
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+template <typename T>
+static cudaError_t attention_fwd_t(const T* qkv, T* o, float* lse, int batch, int T_, int heads, int dh,
+                                   cudaStream_t s) {
+  size_t smem = (size_t)3 * 32 * (dh + 1) * sizeof(float);
+  cudaError_t e = set_smem(attn_fwd_kernel<T>, smem);
+  if (e != cudaSuccess) return e;
+  dim3 grid(cdiv(T_, 32), heads, batch);
+  attn_fwd_kernel<T><<<grid, 256, smem, s>>>(qkv, o, lse, T_, heads, dh, 1.f / sqrtf((float)dh));
+  return cudaGetLastError();
+}
+
+cudaError_t attention_fwd(const void* qkv, void* o, float* lse, int batch, int T_, int heads, int dh,
+                          bool bf16, cudaStream_t s) {
+  if (dh > 32 * ATT_MAXC) return cudaErrorInvalidValue;
+  return bf16 ? attention_fwd_t<bf16_t>((const bf16_t*)qkv, (bf16_t*)o, lse, batch, T_, heads, dh, s)
+              : attention_fwd_t<float>((const float*)qkv, (float*)o, lse, batch, T_, heads, dh, s);
+}
+
+template <typename T>
+static cudaError_t attention_bwd_t(const T* qkv, const T* o, const T* dout, const float* lse, float* delta,
+                                   T* dqkv, int batch, int T_, int heads, int dh, cudaStream_t s) {
+  int rows = batch * T_;
+  attn_delta_kernel<T><<<cdiv((long long)rows * heads, 8), 256, 0, s>>>(o, dout, delta, rows, T_, heads, dh);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  size_t smem = ((size_t)4 * 32 * (dh + 1) + 64) * sizeof(float);
+  if ((e = set_smem(attn_bwd_kv_kernel<T>, smem)) != cudaSuccess) return e;
+  if ((e = set_smem(attn_bwd_q_kernel<T>, smem)) != cudaSuccess) return e;
+  dim3 grid(cdiv(T_, 32), heads, batch);
+  float scale = 1.f / sqrtf((float)dh);
+  attn_bwd_kv_kernel<T><<<grid, 256, smem, s>>>(qkv, dout, lse, delta, dqkv, T_, heads, dh, scale);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  attn_bwd_q_kernel<T><<<grid, 256, smem, s>>>(qkv, dout, lse, delta, dqkv, T_, heads, dh, scale);
+  return cudaGetLastError();
+}
+
+cudaError_t attention_bwd(const void* qkv, const void* o, const void* dout, const float* lse, float* delta,
+                          void* dqkv, int batch, int T_, int heads, int dh, bool bf16, cudaStream_t s) {
+  if (dh > 32 * ATT_MAXC) return cudaErrorInvalidValue;
+  return bf16 ? attention_bwd_t<bf16_t>((const bf16_t*)qkv, (const bf16_t*)o, (const bf16_t*)dout, lse, delta, (bf16_t*)dqkv, batch, T_, heads, dh, s)
+              : attention_bwd_t<float>((const float*)qkv, (const float*)o, (const float*)dout, lse, delta, (float*)dqkv, batch, T_, heads, dh, s);
+}
+
+// ------------------------------------------------------------------------------------------
+// losses
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ float block_reduce_256(float v, float* sm, bool is_max) {
+  int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  v = is_max ? warp_max(v) : warp_sum(v);
+  __syncthreads();
+  if (lane == 0) sm[warp] = v;
+  __syncthreads();
+  float r = sm[0];
+#pragma unroll
+  for (int i = 1; i < 8; i++) r = is_max ? fmaxf(r, sm[i]) : r + sm[i];
+  return r;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) softmax_ce_kernel(T* __restrict__ logits, const int32_t* __restrict__ ids,
+                                                         int T_, float* __restrict__ rowloss, int V,
+                                                         float inv_rows) {
+  __shared__ float sm[8];
+  const int row = blockIdx.x;
+  T* p = logits + (long long)row * V;
+  const int tgt = ids[(long long)(row / T_) * (T_ + 1) + (row % T_) + 1];
+  const float lt = ldf(p + tgt);
+  float mx = -INFINITY;
+  for (int v = threadIdx.x; v < V; v += 256) mx = fmaxf(mx, ldf(p + v));
+  mx = block_reduce_256(mx, sm, true);
+  float se = 0.f;
+  for (int v = threadIdx.x; v < V; v += 256) se += expf(ldf(p + v) - mx);
+  se = block_reduce_256(se, sm, false);
+  const float lse = mx + logf(se);
+  __syncthreads();  // lt was read by every thread before any store below
+  for (int v = threadIdx.x; v < V; v += 256) {
+    float g = expf(ldf(p + v) - lse) - (v == tgt ? 1.f : 0.f);
+    stf(p + v, g * inv_rows);
+  }
+  if (threadIdx.x == 0) rowloss[row] = lse - lt;
+}
+
+cudaError_t softmax_ce_inplace(void* logits, const int32_t* ids, int T_, float* rowloss, int rows, int V,
+                               float inv_rows, bool bf16, cudaStream_t s) {
+  if (bf16) softmax_ce_kernel<bf16_t><<<rows, 256, 0, s>>>((bf16_t*)logits, ids, T_, rowloss, V, inv_rows);
+  else softmax_ce_kernel<float><<<rows, 256, 0, s>>>((float*)logits, ids, T_, rowloss, V, inv_rows);
+  return cudaGetLastError();
+}
+
+__global__ void __launch_bounds__(1024) reduce_sum_kernel(const float* __restrict__ v, int n, float scale,
+                                                          float* __restrict__ out) {
+  __shared__ float sm[1024];
+  float a = 0.f;
+  for (int i = threadIdx.x; i < n; i += 1024) a += v[i];
+  sm[threadIdx.x] = a;
+  __syncthreads();
+  for (int o = 512; o > 0; o >>= 1) {
+    if (threadIdx.x < o) sm[threadIdx.x] += sm[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) out[0] = sm[0] * scale;
+}
+
+cudaError_t reduce_sum(const float* v, int n, float scale, float* out, cudaStream_t s) {
+  reduce_sum_kernel<<<1, 1024, 0, s>>>(v, n, scale, out);
+  return cudaGetLastError();
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) bce_head_fwd_kernel(const T* __restrict__ z, long long ldz,
+                                                           const float* __restrict__ w, const float* __restrict__ b,
+                                                           const float* __restrict__ y, float* __restrict__ rowloss,
+                                                           float* __restrict__ ds, int rows, int d, float inv_rows) {
+  int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  float s = 0.f;
+  for (int c = lane; c < d; c += 32) s = fmaf(ldf(z + (long long)row * ldz + c), w[c], s);
+  s = warp_sum(s) + b[0];
+  if (lane == 0) {
+    float yy = y[row];
+    float e = expf(-fabsf(s));
+    rowloss[row] = fmaxf(s, 0.f) - s * yy + log1pf(e);
+    float sig = s >= 0.f ? 1.f / (1.f + e) : e / (1.f + e);
+    ds[row] = (sig - yy) * inv_rows;
+  }
+}
+
+cudaError_t bce_head_fwd(const void* z, long long ldz, const float* w, const float* b, const float* y,
+                         float* rowloss, float* ds, int rows, int d, float inv_rows, bool bf16,
+                         cudaStream_t s) {
+  if (bf16) bce_head_fwd_kernel<bf16_t><<<cdiv(rows, 8), 256, 0, s>>>((const bf16_t*)z, ldz, w, b, y, rowloss, ds, rows, d, inv_rows);
+  else bce_head_fwd_kernel<float><<<cdiv(rows, 8), 256, 0, s>>>((const float*)z, ldz, w, b, y, rowloss, ds, rows, d, inv_rows);
+  return cudaGetLastError();
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) bce_head_dz_kernel(const float* __restrict__ ds, const float* __restrict__ w,
+                                                          T* __restrict__ dz, int dact, const T* __restrict__ src,
+                                                          long long n, int d) {
+  long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (i >= n) return;
+  float v = ds[i / d] * w[i % d];
+  if (dact != ACT_NONE) v *= act_deriv(dact, ldf(src + i));
+  stf(dz + i, v);
+}
+
+cudaError_t bce_head_dz(const float* ds, const float* w, void* dz, int dact, const void* src, int rows,
+                        int d, bool bf16, cudaStream_t s) {
+  long long n = (long long)rows * d;
+  if (bf16) bce_head_dz_kernel<bf16_t><<<cdiv(n, 256), 256, 0, s>>>(ds, w, (bf16_t*)dz, dact, (const bf16_t*)src, n, d);
+  else bce_head_dz_kernel<float><<<cdiv(n, 256), 256, 0, s>>>(ds, w, (float*)dz, dact, (const float*)src, n, d);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// elementwise
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void ew_mul_kernel(const T* a, const T* b, T* out, long long n) {
+  long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (i < n) stf(out + i, ldf(a + i) * ldf(b + i));
+}
+cudaError_t ew_mul(const void* a, const void* b, void* out, long long n, bool bf16, cudaStream_t s) {
+  if (bf16) ew_mul_kernel<bf16_t><<<cdiv(n, 256), 256, 0, s>>>((const bf16_t*)a, (const bf16_t*)b, (bf16_t*)out, n);
+  else ew_mul_kernel<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)a, (const float*)b, (float*)out, n);
+  return cudaGetLastError();
+}
+template <typename T>
+__global__ void ew_dact_kernel(T* d, const T* src, int act, long long n) {
+  long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (i < n) stf(d + i, ldf(d + i) * act_deriv(act, ldf(src + i)));
+}
+cudaError_t ew_dact(void* d, const void* src, int act, long long n, bool bf16, cudaStream_t s) {
+  if (bf16) ew_dact_kernel<bf16_t><<<cdiv(n, 256), 256, 0, s>>>((bf16_t*)d, (const bf16_t*)src, act, n);
+  else ew_dact_kernel<float><<<cdiv(n, 256), 256, 0, s>>>((float*)d, (const float*)src, act, n);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// input staging (z_0)
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void gather_tokens_kernel(const float* __restrict__ tok, const float* __restrict__ pos,
+                                     const int32_t* __restrict__ ids, T* __restrict__ z0, int T_, int d,
+                                     long long n) {
+  long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (i >= n) return;
+  int c = (int)(i % d);
+  long long row = i / d;
+  int t = (int)(row % T_);
+  long long b = row / T_;
+  int id = ids[b * (T_ + 1) + t];
+  stf(z0 + i, tok[(long long)id * d + c] + pos[(long long)t * d + c]);
+}
+cudaError_t gather_tokens(const float* tok, const float* pos, const int32_t* ids, void* z0, int batch,
+                          int T_, int d, bool bf16, cudaStream_t s) {
+  long long n = (long long)batch * T_ * d;
+  if (bf16) gather_tokens_kernel<bf16_t><<<cdiv(n, 256), 256, 0, s>>>(tok, pos, ids, (bf16_t*)z0, T_, d, n);
+  else gather_tokens_kernel<float><<<cdiv(n, 256), 256, 0, s>>>(tok, pos, ids, (float*)z0, T_, d, n);
+  return cudaGetLastError();
+}
+
+template <typename T>
+__global__ void gather_ctr_kernel(const float* __restrict__ tables, long long table_stride,
+                                  const int32_t* __restrict__ ids, const float* __restrict__ dense,
+                                  T* __restrict__ x0, int ns, int e, int nd, int width, long long n) {
+  long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (i >= n) return;
+  int c = (int)(i % width);
+  long long row = i / width;
+  float v = 0.f;
+  if (c < ns * e) {
+    int t = c / e, cc = c - t * e;
+    int id = ids[row * ns + t];
+    v = tables[(long long)t * table_stride + (long long)id * e + cc];
+  } else if (c < ns * e + nd) {
+    v = dense[row * nd + (c - ns * e)];
+  }
+  stf(x0 + i, v);
+}
+cudaError_t gather_ctr(const float* tables, long long table_stride, const int32_t* ids, const float* dense,
+                       void* x0, int batch, int ns, int e, int nd, int width, bool bf16, cudaStream_t s) {
+  long long n = (long long)batch * width;
+  if (bf16) gather_ctr_kernel<bf16_t><<<cdiv(n, 256), 256, 0, s>>>(tables, table_stride, ids, dense, (bf16_t*)x0, ns, e, nd, width, n);
+  else gather_ctr_kernel<float><<<cdiv(n, 256), 256, 0, s>>>(tables, table_stride, ids, dense, (float*)x0, ns, e, nd, width, n);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// dot interaction: one CTA of 128 threads per sample
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(128) dot_fwd_kernel(const T* __restrict__ proj, const T* __restrict__ x0,
+                                                      long long ldx0, T* __restrict__ feats, int ns, int e, int fw) {
+  extern __shared__ float sm[];  // [(ns+1)][e+1]
+  const int n = blockIdx.x, nv = ns + 1, lde = e + 1;
+  for (int i = threadIdx.x; i < nv * e; i += 128) {
+    int j = i / e, c = i - j * e;
+    sm[j * lde + c] = j == 0 ? ldf(proj + (long long)n * e + c) : ldf(x0 + (long long)n * ldx0 + (j - 1) * e + c);
+  }
+  __syncthreads();
+  const int npair = nv * (nv - 1) / 2;
+  T* f = feats + (long long)n * fw;
+  for (int p = threadIdx.x; p < fw; p += 128) {
+    float v = 0.f;
+    if (p < npair) {
+      // invert p = i(i-1)/2 + j, 0 <= j < i
+      int i = (int)((1.f + sqrtf(1.f + 8.f * p)) * 0.5f);
+      while (i * (i - 1) / 2 > p) i--;
+      while ((i + 1) * i / 2 <= p) i++;
+      int j = p - i * (i - 1) / 2;
+      for (int c = 0; c < e; c++) v = fmaf(sm[i * lde + c], sm[j * lde + c], v);
+    } else if (p < npair + e) {
+      v = sm[p - npair];
+    }
+    stf(f + p, v);
+  }
+}
+cudaError_t dot_fwd(const void* proj, const void* x0, long long ldx0, void* feats, int batch, int ns, int e,
+                    int fw, bool bf16, cudaStream_t s) {
+  size_t smem = (size_t)(ns + 1) * (e + 1) * sizeof(float);
+  if (bf16) dot_fwd_kernel<bf16_t><<<batch, 128, smem, s>>>((const bf16_t*)proj, (const bf16_t*)x0, ldx0, (bf16_t*)feats, ns, e, fw);
+  else dot_fwd_kernel<float><<<batch, 128, smem, s>>>((const float*)proj, (const float*)x0, ldx0, (float*)feats, ns, e, fw);
+  return cudaGetLastError();
+}
+
+template <typename T>
+__global__ void __launch_bounds__(128) dot_bwd_kernel(const T* __restrict__ dfeat, const T* __restrict__ x0,
+                                                      long long ldx0, T* __restrict__ dproj, int ns, int e, int fw) {
+  const int n = blockIdx.x, nv = ns + 1;
+  const int npair = nv * (nv - 1) / 2;
+  const T* df = dfeat + (long long)n * fw;
+  for (int c = threadIdx.x; c < e; c += 128) {
+    float v = ldf(df + npair + c);
+    for (int j = 1; j < nv; j++)
+      v = fmaf(ldf(df + j * (j - 1) / 2), ldf(x0 + (long long)n * ldx0 + (j - 1) * e + c), v);
+    stf(dproj + (long long)n * e + c, v);
+  }
+}
+cudaError_t dot_bwd(const void* dfeat, const void* x0, long long ldx0, void* dproj, int batch, int ns, int e,
+                    int fw, bool bf16, cudaStream_t s) {
+  if (bf16) dot_bwd_kernel<bf16_t><<<batch, 128, 0, s>>>((const bf16_t*)dfeat, (const bf16_t*)x0, ldx0, (bf16_t*)dproj, ns, e, fw);
+  else dot_bwd_kernel<float><<<batch, 128, 0, s>>>((const float*)dfeat, (const float*)x0, ldx0, (float*)dproj, ns, e, fw);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// optimizer
+// ------------------------------------------------------------------------------------------
+__global__ void opt_tick_kernel(double* tick, double b1, double b2) {
+  double t = tick[0] + 1.0;
+  tick[0] = t;
+  tick[1] = 1.0 - pow(b1, t);
+  tick[2] = 1.0 - pow(b2, t);
+}
+cudaError_t opt_tick(double* tick, float beta1, float beta2, cudaStream_t s) {
+  opt_tick_kernel<<<1, 1, 0, s>>>(tick, (double)beta1, (double)beta2);
+  return cudaGetLastError();
+}
+
+__global__ void __launch_bounds__(256) opt_update_kernel(float* __restrict__ theta, const float* __restrict__ grad,
+                                                         float* __restrict__ m, float* __restrict__ v,
+                                                         bf16_t* __restrict__ shadow, long long n, int kind, float lr,
+                                                         float b1, float b2, float eps, float wd,
+                                                         const double* __restrict__ tick) {
+  long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (i >= n) return;
+  float th = theta[i], g = grad[i];
+  if (kind == 0) {
+    th -= lr * g;
+  } else {
+    float bc1 = (float)tick[1], bc2 = (float)tick[2];
+    if (kind == 2) th *= (1.f - lr * wd);
+    float mm = b1 * m[i] + (1.f - b1) * g;
+    float vv = b2 * v[i] + (1.f - b2) * g * g;
+    m[i] = mm;
+    v[i] = vv;
+    th -= lr * (mm / bc1) / (sqrtf(vv / bc2) + eps);
+  }
+  theta[i] = th;
+  if (shadow) shadow[i] = __float2bfloat16_rn(th);
+}
+cudaError_t opt_update(float* theta, const float* grad, float* m, float* v, void* shadow, long long n, int kind,
+                       float lr, float beta1, float beta2, float eps, float wd, const double* tick,
+                       cudaStream_t s) {
+  if (n <= 0) return cudaSuccess;
+  opt_update_kernel<<<cdiv(n, 256), 256, 0, s>>>(theta, grad, m, v, (bf16_t*)shadow, n, kind, lr, beta1, beta2, eps, wd, tick);
+  return cudaGetLastError();
+}
+
+__global__ void to_bf16_kernel(const float* __restrict__ src, bf16_t* __restrict__ dst, long long n) {
+  long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (i < n) dst[i] = __float2bfloat16_rn(src[i]);
+}
+cudaError_t to_bf16(const float* src, void* dst, long long n, cudaStream_t s) {
+  if (n <= 0) return cudaSuccess;
+  to_bf16_kernel<<<cdiv(n, 256), 256, 0, s>>>(src, (bf16_t*)dst, n);
+  return cudaGetLastError();
+}
+
+}  // namespace erase

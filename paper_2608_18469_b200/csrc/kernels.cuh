@@ -1,0 +1,128 @@
+// Launchers of the hand-written CUDA kernels behind the ERASE step library (host-callable).
+// Every launcher only enqueues on the given stream and returns the launch's cudaError_t.
+// "T" below is the model's activation type: float (ERASE_F32) or __nv_bfloat16 (ERASE_BF16),
+// selected at run time by `bf16`.  All reductions use a fixed partition and a fixed combine
+// order, so results do not depend on which stream or in which order kernels were enqueued.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace erase {
+
+enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU = 2 };
+
+// Epilogue of C = A * B^T.  With v = alpha * acc (+ bias[n]):
+//   pre_out != 0 : pre_out[m,n] = v                    (pre-activation kept for the backward)
+//   v = act(v)
+//   mul    != 0 : v *= mul[m,n]                        (DCN-v2 cross: x0 (.) (W x + b))
+//   res    != 0 : v += res[m,n]                        (residual / cross skip path)
+//   dact   != 0 : v *= act'(dact_src[m,n])             (dgrad through an activation; GELU reads
+//                                                       the pre-activation, ReLU the output)
+// mul/res/dact_src/pre_out are T matrices with the row stride ld_aux.
+struct Epilogue {
+  const float* bias = nullptr;
+  int act = ACT_NONE;
+  void* pre_out = nullptr;
+  const void* mul = nullptr;
+  const void* res = nullptr;
+  int dact = ACT_NONE;
+  const void* dact_src = nullptr;
+  long long ld_aux = 0;
+  float alpha = 1.f;
+};
+
+// C[M,N] = epilogue( sum_k A(m,k) * B(n,k) ).  A(m,k) = A[m*sa_m + k*sa_k], B likewise, so one
+// routine serves the forward (X W^T), the dgrad (dY W: B strided over k) and the wgrad
+// (dY^T X: both strided over k).  c_f32: C is float whatever T is (weight gradients).
+// splits > 1: deterministic split-K; partial s is written to ws + s*M*N (float, row stride N)
+// and summed in order s = 0..splits-1 by splitk_reduce; the epilogue must then be empty.
+struct GemmArgs {
+  int M = 0, N = 0, K = 0;
+  const void* A = nullptr; long long sa_m = 0, sa_k = 0;
+  const void* B = nullptr; long long sb_n = 0, sb_k = 0;
+  void* C = nullptr; long long ldc = 0;
+  int c_f32 = 0;
+  int splits = 1;
+  float* ws = nullptr;
+  Epilogue epi;
+};
+
+cudaError_t gemm_simt(const GemmArgs& g, bool bf16, cudaStream_t s);
+cudaError_t splitk_reduce(const float* ws, int splits, long long mn, int N, float* out, long long ldo,
+                          cudaStream_t s);
+
+// out[c] = sum_r scale[r] * X[r, c]  (scale may be null); X is [rows, cols] with row stride ldx.
+// Two-stage with a fixed row partition into `chunks`; ws holds chunks*cols floats.
+int colsum_chunks(int rows, int cols);
+cudaError_t colsum(const void* X, bool x_bf16, long long ldx, int rows, int cols, const float* scale,
+                   float* ws, int chunks, float* out, cudaStream_t s);
+
+// LayerNorm over the last dimension (eps 1e-5, biased variance); saves mean and 1/std per row.
+cudaError_t layernorm_fwd(const void* x, const float* gain, const float* shift, void* y, float* mean,
+                          float* rstd, int rows, int d, bool bf16, cudaStream_t s);
+// dx = rstd*(g - mean(g) - xhat*mean(g*xhat)) + add, g = dy*gain  (add may be null)
+cudaError_t layernorm_bwd_dx(const void* dy, const void* x, const float* gain, const float* mean,
+                             const float* rstd, const void* add, void* dx, int rows, int d, bool bf16,
+                             cudaStream_t s);
+// dgain[c] = sum_r dy*xhat, dshift[c] = sum_r dy; ws holds 2*chunks*d floats.
+cudaError_t layernorm_param_grad(const void* dy, const void* x, const float* mean, const float* rstd,
+                                 float* ws, int chunks, float* dgain, float* dshift, int rows, int d,
+                                 bool bf16, cudaStream_t s);
+
+// Causal self-attention over qkv [batch*T, 3*d] = [Q | K | V], heads are contiguous dh-wide
+// column slices; scale 1/sqrt(dh); o [batch*T, d]; lse [batch*heads*T] (natural log).
+cudaError_t attention_fwd(const void* qkv, void* o, float* lse, int batch, int T, int heads, int dh,
+                          bool bf16, cudaStream_t s);
+// dqkv [batch*T, 3*d] from do, with delta [batch*heads*T] as scratch.
+cudaError_t attention_bwd(const void* qkv, const void* o, const void* dout, const float* lse,
+                          float* delta, void* dqkv, int batch, int T, int heads, int dh, bool bf16,
+                          cudaStream_t s);
+
+// Softmax cross-entropy over logits [rows, V] (row stride V), in place:
+// logits <- (softmax - onehot(target)) * inv_rows; rowloss[r] = logsumexp - logit[target].
+// target of row r = ids[(r / T) * (T + 1) + (r % T) + 1].
+cudaError_t softmax_ce_inplace(void* logits, const int32_t* ids, int T, float* rowloss, int rows, int V,
+                               float inv_rows, bool bf16, cudaStream_t s);
+// out[0] = (sum of v[0..n)) * scale, fixed-order tree in one CTA.
+cudaError_t reduce_sum(const float* v, int n, float scale, float* out, cudaStream_t s);
+
+// BCE head: s = z[r,:].w + b; rowloss = softplus(s) - y*s; ds[r] = (sigmoid(s) - y) * inv_rows
+cudaError_t bce_head_fwd(const void* z, long long ldz, const float* w, const float* b, const float* y,
+                         float* rowloss, float* ds, int rows, int d, float inv_rows, bool bf16,
+                         cudaStream_t s);
+// dz[r,c] = ds[r] * w[c]  (times act'(src[r,c]) when dact != ACT_NONE)
+cudaError_t bce_head_dz(const float* ds, const float* w, void* dz, int dact, const void* src, int rows,
+                        int d, bool bf16, cudaStream_t s);
+
+// out = a (.) b, all [n] of T
+cudaError_t ew_mul(const void* a, const void* b, void* out, long long n, bool bf16, cudaStream_t s);
+// d <- d * act'(src)
+cudaError_t ew_dact(void* d, const void* src, int act, long long n, bool bf16, cudaStream_t s);
+
+// z0[b*T+t, :] = tok[ids[b*(T+1)+t], :] + pos[t, :]
+cudaError_t gather_tokens(const float* tok, const float* pos, const int32_t* ids, void* z0, int batch,
+                          int T, int d, bool bf16, cudaStream_t s);
+// x0[n, t*e + c] = tables[t*table_stride + ids[n*ns+t]*e + c]; x0[n, ns*e + j] = dense[n, j]; pad 0
+cudaError_t gather_ctr(const float* tables, long long table_stride, const int32_t* ids,
+                       const float* dense, void* x0, int batch, int ns, int e, int nd, int width,
+                       bool bf16, cudaStream_t s);
+
+// Dot interaction.  vectors of sample n: v_0 = proj[n, 0:e], v_j = x0[n, (j-1)e : je], j = 1..ns.
+// feats[n, i(i-1)/2 + j] = v_i . v_j (i > j), then proj[n,:], then zeros up to width fw.
+cudaError_t dot_fwd(const void* proj, const void* x0, long long ldx0, void* feats, int batch, int ns,
+                    int e, int fw, bool bf16, cudaStream_t s);
+// dproj[n,:] = dfeat[n, npair : npair+e] + sum_{j>=1} dfeat[n, j(j-1)/2] * v_j
+cudaError_t dot_bwd(const void* dfeat, const void* x0, long long ldx0, void* dproj, int batch, int ns,
+                    int e, int fw, bool bf16, cudaStream_t s);
+
+// Optimizer over a flat range.  kind 0 SGD, 1 Adam, 2 AdamW.  tick[0] = step count t (as float
+// bits of an int64 are avoided: tick is {t, 1-beta1^t, 1-beta2^t} kept on the device so that a
+// replayed CUDA graph advances it).  shadow (bf16 copy of theta) may be null.
+cudaError_t opt_tick(double* tick, float beta1, float beta2, cudaStream_t s);
+cudaError_t opt_update(float* theta, const float* grad, float* m, float* v, void* shadow, long long n,
+                       int kind, float lr, float beta1, float beta2, float eps, float wd,
+                       const double* tick, cudaStream_t s);
+// shadow[i] = bf16(theta[i])
+cudaError_t to_bf16(const float* src, void* dst, long long n, cudaStream_t s);
+
+}  // namespace erase

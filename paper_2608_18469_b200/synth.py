@@ -155,16 +155,35 @@ def tensor_list(spec):
     return out
 
 
+def _followed_by_activation(blk, name):
+    """True if this Linear weight feeds an activation (sets the init gain)."""
+    k = blk["kind"]
+    if not (name.startswith("W") and name[1:].isdigit()):
+        return False
+    i = int(name[1:])
+    if k == "mlp":
+        return blk["act"] != "none" and i < len(blk["dims"]) - 2
+    if k in ("tower", "dot"):
+        return blk["act"] != "none"
+    if k == "transformer":
+        return name == "W1"
+    return False
+
+
 def init_params(spec, seed=0, zero_heads=False):
     """Initial fp32 values, drawn in tensor-index order.
 
-    Linear W, b ~ U(-1/sqrt(in), 1/sqrt(in)); LayerNorm gain 1, shift 0;
-    CTR tables N(0, (1/8)^2); token embedding N(0, 1); position embedding N(0, 0.1^2).
+    Linear W ~ U(-a, a) with a = sqrt(3 g / in): g = 2 when the Linear feeds a ReLU/GELU, else 1,
+    so that the second moment of the activations is roughly kept from layer to layer (with the
+    smaller 1/sqrt(in) bound an 8-deep stack without residuals or norms collapses every sample
+    onto the same bias-driven vector, and the gradients become differences of nearly equal sums);
+    Linear b ~ U(-1/sqrt(in), 1/sqrt(in)); LayerNorm gain 1, shift 0; CTR tables N(0, (1/8)^2);
+    token embedding N(0, 1); position embedding N(0, 0.1^2).
     Returns a list of float32 arrays aligned with ``tensor_list(spec)``.
     """
     rng = np.random.Generator(np.random.PCG64(seed))
     vals = []
-    bound = None
+    fan_in = None
     for (b, name, shape, _tr) in tensor_list(spec):
         if name == "tok_emb":
             v = rng.standard_normal(shape)
@@ -177,11 +196,14 @@ def init_params(spec, seed=0, zero_heads=False):
         elif name.endswith("_b") and name.startswith("ln"):
             v = np.zeros(shape)
         elif len(shape) == 2:                       # Linear weight [out, in]
-            bound = 1.0 / math.sqrt(shape[1])
+            fan_in = shape[1]
+            gain = 2.0 if _followed_by_activation(spec["blocks"][b], name) else 1.0
+            bound = math.sqrt(3.0 * gain / fan_in)
             v = rng.uniform(-bound, bound, shape)
             if zero_heads and name == "Wh":
                 v = np.zeros(shape)
-        else:                                       # Linear bias, same bound as its weight
+        else:                                       # Linear bias
+            bound = 1.0 / math.sqrt(fan_in)
             v = rng.uniform(-bound, bound, shape)
             if zero_heads and name == "bh":
                 v = np.zeros(shape)

@@ -1,0 +1,126 @@
+"""GPU-side test helpers: stage synthetic batches on the device (torch owns the memory) and
+compare the CUDA library with the oracle.  Imported only by tests marked gpu."""
+import numpy as np
+import torch
+
+from oracle import erase_oracle as orc
+from paper_2608_18469_b200 import binding, synth
+from tests import util
+
+TOL = {"f32": 1e-4, "bf16": 2e-2}     # relative L2 per tensor against the fp64 oracle
+
+
+class DevBatch:
+    """Device copies of one batch; keeps the torch tensors alive."""
+
+    def __init__(self, spec, batch):
+        dev = "cuda"
+        self.x = self.ids = self.y = None
+        self.t = {}
+        if spec["input"] == "dense":
+            x = torch.from_numpy(batch["x"])
+            self.t["x"] = (x.to(torch.bfloat16) if spec["dtype"] == "bf16" else x).to(dev).contiguous()
+            self.t["y"] = torch.from_numpy(batch["y"]).to(dev)
+        elif spec["input"] == "tokens":
+            self.t["ids"] = torch.from_numpy(batch["ids"]).to(dev)
+        else:
+            self.t["x"] = torch.from_numpy(batch["dense"]).to(dev)
+            self.t["ids"] = torch.from_numpy(batch["ids"]).to(dev)
+            self.t["y"] = torch.from_numpy(batch["y"]).to(dev)
+        torch.cuda.synchronize()
+        for k, v in self.t.items():
+            setattr(self, k, v.data_ptr())
+
+    def args(self):
+        return dict(x=self.x, ids=self.ids, y=self.y)
+
+
+def new_model(spec, flat):
+    m = binding.Model(spec)
+    names = [(b, n, tuple(s), tr) for (b, n, s, tr) in synth.tensor_list(spec)]
+    assert m.num_tensors() == len(names)
+    for i, want in enumerate(names):
+        assert m.tensor_info(i) == want, (i, m.tensor_info(i), want)
+    m.set_all(flat)
+    return m
+
+
+def compare_teacher_forced(spec, steps, seed=0, n_streams=2, flags=0, report=None):
+    """Each step: library and oracle start from the same fp32 parameters and optimizer state;
+    losses and every gradient tensor must agree within TOL; the parameters after the
+    optimizer must match the update rule applied in fp64 to the library's own gradients."""
+    tol = TOL[spec["dtype"]]
+    flat = synth.init_params(spec, seed)
+    tl = synth.tensor_list(spec)
+    tidx = util.trainable_index(spec)
+    m = new_model(spec, flat)
+    params = util.structure(spec, flat)
+    state = orc.new_opt_state(params)
+    worst = {}
+    try:
+        for it in range(steps):
+            batch = synth.make_batch(spec, seed, index=it)
+            db = DevBatch(spec, batch)
+            # teacher forcing: library <- oracle state (rounded to fp32, oracle continues from the same)
+            if it > 0:
+                for i in tidx:
+                    b, name, _s, _t = tl[i]
+                    p32 = params["blocks"][b][name].astype(np.float32)
+                    params["blocks"][b][name] = p32.astype(np.float64)
+                    m32 = state["m"][b][name].astype(np.float32)
+                    v32 = state["v"][b][name].astype(np.float32)
+                    state["m"][b][name], state["v"][b][name] = m32.astype(np.float64), v32.astype(np.float64)
+                    m.set_params(i, p32)
+                    m.set_opt_state(i, m32, v32, state["t"])
+            m.step(n_streams=n_streams, flags=flags, **db.args())
+            got_l = m.losses()
+            want_l, want_g, new_params, new_state = orc.step(spec, params, state, batch)
+            for b in range(len(want_l)):
+                err = abs(got_l[b] - want_l[b]) / max(abs(want_l[b]), 1e-12)
+                worst[f"loss{b}"] = max(worst.get(f"loss{b}", 0), err)
+                if report is None:
+                    assert err <= tol, (it, "loss", b, got_l[b], want_l[b])
+            for i in tidx:
+                b, name, _s, _t = tl[i]
+                g = m.grads(i)
+                err = synth.rel_l2(g, want_g[b][name])
+                key = f"grad b{b} {name}"
+                worst[key] = max(worst.get(key, 0), err)
+                if report is None:
+                    assert err <= tol, (it, key, err)
+                # optimizer alone: update rule in fp64 on the library's gradient
+                th, _, _ = orc.optimizer_update(spec["opt"], params["blocks"][b][name], g.astype(np.float64),
+                                                state["m"][b][name], state["v"][b][name], state["t"] + 1)
+                perr = synth.rel_l2(m.params(i), th)
+                key = f"param b{b} {name}"
+                worst[key] = max(worst.get(key, 0), perr)
+                if report is None:
+                    assert perr <= 2e-6, (it, key, perr)
+            params, state = new_params, new_state
+    finally:
+        m.close()
+    if report is not None:
+        report.update(worst)
+    return worst
+
+
+def run_steps(spec, flat, batches, n_streams, flags=0):
+    """Free-running steps; returns per-step losses and the final raw state for bit comparison."""
+    m = new_model(spec, flat)
+    try:
+        losses = []
+        for db in batches:
+            m.step(n_streams=n_streams, flags=flags, **db.args())
+            losses.append(m.losses().copy())
+        tidx = util.trainable_index(spec)
+        final = {"losses": np.array(losses)}
+        for i in tidx:
+            final[f"p{i}"] = m.params(i)
+            final[f"g{i}"] = m.grads(i)
+            mm, vv, t = m.opt_state(i)
+            final[f"m{i}"], final[f"v{i}"] = mm, vv
+        final["t"] = np.array([t])
+        final["launches"] = m.launch_count()
+        return final
+    finally:
+        m.close()

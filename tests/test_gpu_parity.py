@@ -1,0 +1,112 @@
+"""Parity of the CUDA library (through the C ABI) with the CPU oracle, and bit-identity of the
+ERASE schedule with the serial one.  All inputs are seeded and synthetic."""
+import numpy as np
+import pytest
+
+from paper_2608_18469_b200 import synth
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+
+def _gu():
+    from tests import gpu_util
+    return gpu_util
+
+
+@pytest.mark.parametrize("name", list(util.tiny_specs()))
+def test_tiny_fp32_every_block_kind(name):
+    _gu().compare_teacher_forced(util.tiny_specs()[name], steps=3, seed=1)
+
+
+def _midsize():
+    s = {}
+    # several 64-wide tiles with ragged tails in every dimension
+    s["mlp_f32_ragged"] = synth.mlp_spec(70, 150, 3, 200, "gelu", "f32",
+                                         opt={"kind": "adam", "lr": 1e-3, "wd": 0.0, "beta1": 0.9,
+                                              "beta2": 0.999, "eps": 1e-8})
+    s["tower_f32"] = {**synth.mlp_spec(48, 96, 2, 130, "relu", "f32")}
+    for blk in s["tower_f32"]["blocks"]:
+        blk["kind"] = "tower"
+    s["lm_f32"] = synth.lm_spec(2, 96, 3, 160, 70, 3, 301, dtype="f32")       # dh 32, T ragged
+    s["lm_f32_dh64"] = synth.lm_spec(2, 128, 2, 256, 48, 2, 200, dtype="f32")
+    s["ctr_f32"] = synth.ctr_spec(batch=150, n_dense=13, n_sparse=5, table_rows=50, emb_dim=8,
+                                  tower=(72, 40, 24), n_cross=3, dtype="f32")
+    return s
+
+
+@pytest.mark.parametrize("name", list(_midsize()))
+def test_midsize_fp32(name):
+    _gu().compare_teacher_forced(_midsize()[name], steps=2, seed=2)
+
+
+def test_config1_fp32_ten_steps_and_free_running_losses():
+    from oracle import erase_oracle as orc
+    gu = _gu()
+    spec = synth.config("C1")
+    gu.compare_teacher_forced(spec, steps=10, seed=0)
+    # free running: ten steps from seed 0, losses against the oracle's own trajectory
+    flat = synth.init_params(spec, 0)
+    batches = [synth.make_batch(spec, 0, index=i) for i in range(10)]
+    got = gu.run_steps(spec, flat, [gu.DevBatch(spec, b) for b in batches], n_streams=3)
+    params = util.structure(spec, flat)
+    state = orc.new_opt_state(params)
+    for i, b in enumerate(batches):
+        want, _, params, state = orc.step(spec, params, state, b)
+        assert np.allclose(got["losses"][i], want, rtol=1e-4, atol=0)
+
+
+def _bf16_cases():
+    s = {}
+    s["c5_w128_b512"] = synth.config("C5", w=128, batch=512)
+    s["c5_w512_b512"] = synth.config("C5", w=512, batch=512)
+    s["mlp_bf16_ragged"] = synth.mlp_spec(200, 328, 2, 300, "gelu", "bf16")
+    s["lm_bf16_small"] = synth.lm_spec(2, 128, 2, 512, 128, 4, 1000)
+    s["ctr_bf16_small"] = synth.ctr_spec(batch=512, table_rows=1000, tower=(256, 128, 64))
+    return s
+
+
+@pytest.mark.parametrize("name", list(_bf16_cases()))
+def test_bf16_small(name):
+    _gu().compare_teacher_forced(_bf16_cases()[name], steps=2, seed=3)
+
+
+def test_config2_small_lm_bf16_full_size():
+    _gu().compare_teacher_forced(synth.config("C2"), steps=3, seed=0)
+
+
+def test_config3_ctr_bf16_full_size():
+    _gu().compare_teacher_forced(synth.config("C3"), steps=2, seed=0)
+
+
+def test_config4_reduced_two_blocks():
+    spec = synth.lm_spec(2, 768, 12, 3072, 128, 8, 32768)
+    _gu().compare_teacher_forced(spec, steps=1, seed=0)
+
+
+# ------------------------------------------------------------------ schedules: bit identity
+
+def _bits_equal(a, b):
+    for k in a:
+        if k == "launches":
+            continue
+        assert a[k].tobytes() == b[k].tobytes(), k
+
+
+@pytest.mark.parametrize("name", ["C1", "lm", "ctr", "c5"])
+def test_erase_schedule_is_bit_identical_to_serial(name):
+    gu = _gu()
+    spec = {"C1": synth.config("C1"),
+            "lm": synth.lm_spec(3, 128, 2, 256, 64, 4, 512),
+            "ctr": synth.ctr_spec(batch=256, table_rows=500, tower=(128, 64, 32)),
+            "c5": synth.config("C5", w=128, batch=512)}[name]
+    flat = synth.init_params(spec, 5)
+    batches = [gu.DevBatch(spec, synth.make_batch(spec, 5, index=i)) for i in range(4)]
+    serial = gu.run_steps(spec, flat, batches, n_streams=1)
+    nb = len(spec["blocks"])
+    for ns in sorted({2, 3, nb + 1}):
+        _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=ns))
+    from paper_2608_18469_b200 import binding
+    _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=1, flags=binding.GRAPH))
+    _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=nb + 1, flags=binding.GRAPH))
+    assert serial["launches"] > 0

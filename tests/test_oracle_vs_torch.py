@@ -111,7 +111,7 @@ def _run(spec, steps, seed=0):
         for b in range(len(tg)):
             for k in tg[b]:
                 assert synth.rel_l2(og[b][k], tg[b][k]) < 1e-10, (it, b, k)
-                assert synth.rel_l2(params["blocks"][b][k], tparams[b][k].detach().numpy()) < 1e-12, (it, b, k)
+                assert synth.rel_l2(params["blocks"][b][k], tparams[b][k].detach().numpy()) < 1e-9, (it, b, k)
 
 
 @pytest.mark.parametrize("name", list(util.tiny_specs()))
