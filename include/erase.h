@@ -190,6 +190,22 @@ ERASE_API int64_t erase_launch_count(const erase_model* m);
  * run without ERASE_GRAPH.  Waits for the step.  Errors: EINVAL, ESTATE (no such step). */
 ERASE_API erase_status erase_timeline(erase_model* m, float* out, int32_t n);
 
+/* The GEMM the block linears are made of, on its own (paper Section 1: the "small GEMMs" of proxy
+ * models are where the accelerator's capacity goes unused).  C[M,N] = sum_k A(m,k) B(n,k) with
+ * A(m,k) = A[m*sa_m + k*sa_k] and B(n,k) = B[n*sb_n + k*sb_k] (element strides; one stride of
+ * each operand must be 1), so the same call covers X W^T (forward), dY W (dgrad, B strided over
+ * k) and dY^T X (wgrad, both strided over k).  A, B, C are DEVICE pointers; dtype selects float
+ * or bfloat16 operands; C is float when c_f32 != 0, else the operand type, row stride ldc.
+ * splits > 1 runs a deterministic split-K (fixed partition, partial sums added in order).
+ * engine: 0 = SIMT kernel, 1 = tcgen05 tensor-core kernel (bf16 only; EUNSUPPORTED when the
+ * shape or alignment does not qualify: K >= 64, N >= 16, 16-byte aligned bases, leading strides
+ * multiples of 8).  The call allocates its split-K workspace, runs on `stream` (a cudaStream_t,
+ * may be NULL for the default stream), waits for completion and frees the workspace.
+ * Errors: EINVAL, ENOMEM, EUNSUPPORTED, ECUDA, ETIMEOUT (a bounded device wait expired). */
+ERASE_API erase_status erase_gemm(int32_t dtype, int32_t M, int32_t N, int32_t K, const void* A, int64_t sa_m,
+                                  int64_t sa_k, const void* B, int64_t sb_n, int64_t sb_k, void* C, int64_t ldc,
+                                  int32_t c_f32, int32_t splits, int32_t engine, void* stream);
+
 /* One record per operation of a profiled step. */
 typedef struct {
   char name[32];    /* kernel class: gemm_fwd, gemm_dgrad, gemm_wgrad, softmax_ce, opt_update, ...   */

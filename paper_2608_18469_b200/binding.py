@@ -80,6 +80,9 @@ EXPORTS = {
     "erase_main_stream": (C.c_void_p, [C.c_void_p]),
     "erase_launch_count": (C.c_int64, [C.c_void_p]),
     "erase_timeline": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32]),
+    "erase_gemm": (C.c_int, [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int64, C.c_int64,
+                             C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_int64, C.c_int32, C.c_int32,
+                             C.c_int32, C.c_void_p]),
     "erase_profile_step": (C.c_int, [C.c_void_p, C.POINTER(Batch), C.POINTER(OpRecord), C.c_int32,
                                      C.POINTER(C.c_int32)]),
     "erase_last_error": (C.c_char_p, [C.c_void_p]),
@@ -232,6 +235,14 @@ class Model:
         out = np.empty(n, np.float32)
         self._ck(lib().erase_timeline(self.h, _fptr(out), n))
         return out.reshape(-1, 2)
+
+
+def gemm(dtype, M, N, K, A, sa_m, sa_k, B, sb_n, sb_k, Cptr, ldc, c_f32=False, splits=1, engine=0, stream=None):
+    """erase_gemm on device pointers (ints); raises EraseError on failure."""
+    st = lib().erase_gemm(_DTYPE[dtype], M, N, K, A, sa_m, sa_k, B, sb_n, sb_k, Cptr, ldc, int(c_f32), splits,
+                          engine, stream)
+    if st != OK:
+        raise EraseError(st, lib().erase_last_error(None).decode())
 
 
 def arena_bytes(spec):

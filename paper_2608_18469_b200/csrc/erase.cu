@@ -75,6 +75,7 @@ struct erase_model {
   float* mom2 = nullptr;
   void* shadow = nullptr;  // bf16 copy of theta (operands of the bf16 GEMMs)
   double* tick = nullptr;  // {t, 1-beta1^t, 1-beta2^t}
+  int* status = nullptr;   // device word: non-zero once a bounded device-side wait has expired
   float* losses = nullptr;
 
   // device memory
@@ -313,25 +314,32 @@ struct Builder {
   const char* gemm_tag = "gemm";
 
   void gemm(OpList& ops, GemmArgs g) {
-    bool bf = m->bf16;
     size_t before = ops.size();
     gemm_inner(ops, g);
     double fl = 2.0 * g.M * g.N * g.K;
     double by = ((double)g.M * g.K + (double)g.N * g.K) * m->esz + (double)g.M * g.N * (g.c_f32 ? 4 : m->esz);
-    (void)bf;
     if (ops.size() > before) note(ops, gemm_tag, fl, by);
   }
   void gemm_inner(OpList& ops, GemmArgs g) {
-    bool bf = m->bf16;
+    const bool bf = m->bf16;
+    const bool tc_ok = bf && tc_gemm_supported(g);
+    float* out = (float*)g.C;
+    const long long ldo = g.ldc;
+    if (g.splits > 1) g.ws = f32_buf((size_t)g.splits * g.M * g.N);
     TcPlan plan;
-    if (bf && !m->dry && tc_gemm_plan(g, &plan)) {
-      ops.push_back({[g, plan](cudaStream_t s) { return tc_gemm_launch(g, plan, s); }, plan.launches});
+    const bool use_tc = tc_ok && !m->dry && tc_gemm_plan(g, m->status, &plan);
+    if (use_tc) {
+      if (g.splits > 1)
+        ops.push_back({[g, plan, out, ldo](cudaStream_t s) {
+                         cudaError_t e = tc_gemm_launch(g, plan, s);
+                         if (e != cudaSuccess) return e;
+                         return splitk_reduce(g.ws, g.splits, (long long)g.M * g.N, g.N, out, ldo, s);
+                       }, 2});
+      else
+        ops.push_back({[g, plan](cudaStream_t s) { return tc_gemm_launch(g, plan, s); }, 1});
       return;
     }
     if (g.splits > 1) {
-      g.ws = f32_buf((size_t)g.splits * g.M * g.N);
-      float* out = (float*)g.C;
-      long long ldo = g.ldc;
       ops.push_back({[g, bf, out, ldo](cudaStream_t s) {
                        cudaError_t e = gemm_simt(g, bf, s);
                        if (e != cudaSuccess) return e;
@@ -661,6 +669,7 @@ struct Builder {
     if (s.opt != ERASE_OPT_SGD) { m->mom1 = f32_buf(m->train_n); m->mom2 = f32_buf(m->train_n); }
     if (bf) m->shadow = dev_alloc(m, m->train_n * 2, &ok);
     m->tick = (double*)dev_alloc(m, 3 * sizeof(double), &ok);
+    m->status = (int*)dev_alloc(m, sizeof(int), &ok);
     m->losses = f32_buf(m->B);
     // z_0
     // z_0: dense batches are copied into a model-owned buffer (so every block reads memory whose
@@ -884,6 +893,15 @@ erase_status erase_sync(erase_model* m) {
   if (!m) return ERASE_EINVAL;
   CK(cudaStreamSynchronize(m->main));
   for (auto s : m->side) CK(cudaStreamSynchronize(s));
+  if (m->status) {
+    int st = 0;
+    CK(copy_sync(m, &st, m->status, sizeof(int), cudaMemcpyDeviceToHost));
+    if (st != 0) {
+      int zero = 0;
+      CK(copy_sync(m, m->status, &zero, sizeof(int), cudaMemcpyHostToDevice));
+      return m->fail(ERASE_ETIMEOUT, "a bounded device-side wait expired (code " + std::to_string(st) + "); results of the step are void");
+    }
+  }
   return ERASE_OK;
 }
 
@@ -1077,6 +1095,65 @@ erase_status erase_timeline(erase_model* m, float* out, int32_t n) {
   erase_status st = erase_sync(m);
   if (st != ERASE_OK) return st;
   for (int i = 0; i < need; i++) CK(cudaEventElapsedTime(&out[i], m->ev_time[need], m->ev_time[i]));
+  return ERASE_OK;
+}
+
+erase_status erase_gemm(int32_t dtype, int32_t M, int32_t N, int32_t K, const void* A, int64_t sa_m, int64_t sa_k,
+                        const void* B, int64_t sb_n, int64_t sb_k, void* C, int64_t ldc, int32_t c_f32, int32_t splits,
+                        int32_t engine, void* stream) {
+  if ((dtype != ERASE_F32 && dtype != ERASE_BF16) || M < 1 || N < 1 || K < 1 || !A || !B || !C || splits < 1 ||
+      splits > 1024 || (engine != 0 && engine != 1) || ldc < N || (sa_m != 1 && sa_k != 1) || (sb_n != 1 && sb_k != 1)) {
+    g_create_error = "erase_gemm: bad argument";
+    return ERASE_EINVAL;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  GemmArgs g;
+  g.M = M; g.N = N; g.K = K;
+  g.A = A; g.sa_m = sa_m; g.sa_k = sa_k;
+  g.B = B; g.sb_n = sb_n; g.sb_k = sb_k;
+  g.C = C; g.ldc = ldc; g.c_f32 = (c_f32 || dtype == ERASE_F32) ? 1 : 0;
+  g.splits = splits;
+  g.epi.ld_aux = N;
+  const bool bf = dtype == ERASE_BF16;
+  if (engine == 1 && (!bf || !tc_gemm_supported(g))) {
+    g_create_error = "erase_gemm: the tensor-core kernel does not take this shape/alignment/dtype";
+    return ERASE_EUNSUPPORTED;
+  }
+  if (splits > 1 && !g.c_f32) {
+    g_create_error = "erase_gemm: split-K needs a float result (c_f32)";
+    return ERASE_EINVAL;
+  }
+  float* ws = nullptr;
+  int* status = nullptr;
+  auto cleanup = [&]() { if (ws) cudaFree(ws); if (status) cudaFree(status); cudaGetLastError(); };
+  auto cuda_fail = [&](cudaError_t e, const char* what) {
+    g_create_error = std::string("erase_gemm: ") + what + ": " + cudaGetErrorString(e);
+    cleanup();
+    return ERASE_ECUDA;
+  };
+  if (splits > 1 && cudaMalloc(&ws, (size_t)splits * M * N * sizeof(float)) != cudaSuccess) { cleanup(); g_create_error = "erase_gemm: workspace allocation failed"; return ERASE_ENOMEM; }
+  if (cudaMalloc(&status, sizeof(int)) != cudaSuccess) { cleanup(); g_create_error = "erase_gemm: allocation failed"; return ERASE_ENOMEM; }
+  cudaError_t e = cudaMemsetAsync(status, 0, sizeof(int), st);
+  if (e != cudaSuccess) return cuda_fail(e, "memset");
+  g.ws = ws;
+  if (engine == 1) {
+    TcPlan plan;
+    if (!tc_gemm_plan(g, status, &plan)) { cleanup(); g_create_error = "erase_gemm: TMA descriptor encoding failed"; return ERASE_EUNSUPPORTED; }
+    e = tc_gemm_launch(g, plan, st);
+  } else {
+    e = gemm_simt(g, bf, st);
+  }
+  if (e != cudaSuccess) return cuda_fail(e, "launch");
+  if (splits > 1) {
+    e = splitk_reduce(ws, splits, (long long)M * N, N, (float*)C, ldc, st);
+    if (e != cudaSuccess) return cuda_fail(e, "reduce launch");
+  }
+  int hst = 0;
+  e = cudaMemcpyAsync(&hst, status, sizeof(int), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return cuda_fail(e, "execution");
+  cleanup();
+  if (hst != 0) { g_create_error = "erase_gemm: a bounded device-side wait expired (code " + std::to_string(hst) + ")"; return ERASE_ETIMEOUT; }
   return ERASE_OK;
 }
 

@@ -1,8 +1,465 @@
+// tcgen05 / TMEM / TMA GEMM for sm_100a.  See gemm_tc.cuh for the contract.
+//
+// CTA = one 128 x BN output tile (one split of K when split-K is on), 192 threads:
+//   warp 0      TMA producer: one elected thread fills a ring of STAGES shared-memory stages,
+//               each holding a 128 x 64 slab of A and a BN x 64 slab of B (bf16, 128-byte swizzle)
+//   warp 1      allocates TMEM, then one elected thread issues tcgen05.mma (M=128, N=BN, K=16),
+//               four per stage, and commits each stage back to the producer through an mbarrier
+//   warps 2..5  epilogue: wait for the accumulator, read their TMEM lane quarter with
+//               tcgen05.ld, apply the fused epilogue, store to global memory
+// Every mbarrier wait is bounded by a clock limit; on expiry the kernel records a status word,
+// skips the rest of its work, still frees its TMEM and returns.
 #include "gemm_tc.cuh"
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <string.h>
 
 namespace erase {
 
-bool tc_gemm_plan(const GemmArgs&, TcPlan*) { return false; }
-cudaError_t tc_gemm_launch(const GemmArgs&, const TcPlan&, cudaStream_t) { return cudaErrorNotSupported; }
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;          // bf16 elements = 128 bytes = one swizzle row
+constexpr int UMMA_K = 16;
+constexpr int STAGES = 4;
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;  // ~2 s at 2 GHz
+
+struct TcArgs {
+  int M, N, K;
+  void* C;
+  long long ldc;
+  int c_f32;
+  int splits;
+  float* ws;
+  Epilogue epi;
+  int* status;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if the limit expired (status word is set by the caller).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > WAIT_LIMIT_CYCLES) return false;
+  }
+  return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// 32 lanes x 32 consecutive fp32 columns: thread i of the warp receives lane (base + i).
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1.
+//   bits  0..13  start address >> 4        bits 16..29  leading byte offset >> 4
+//   bits 32..45  stride byte offset >> 4   bits 46..47  version (1)      bits 61..63  swizzle (2 = 128B)
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+  return (uint64_t)((addr & 0x3FFFF) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+
+__device__ __forceinline__ float bf2f(uint32_t bits16) { return __uint_as_float(bits16 << 16); }
+
+__device__ __forceinline__ float act_apply_d(int act, float v) {
+  if (act == ACT_RELU) return v > 0.f ? v : 0.f;
+  if (act == ACT_GELU) return v * 0.5f * (1.f + erff(v * 0.70710678118654752f));
+  return v;
+}
+__device__ __forceinline__ float act_deriv_d(int act, float u) {
+  if (act == ACT_RELU) return u > 0.f ? 1.f : 0.f;
+  if (act == ACT_GELU) {
+    float cdf = 0.5f * (1.f + erff(u * 0.70710678118654752f));
+    float pdf = 0.39894228040143268f * expf(-0.5f * u * u);
+    return cdf + u * pdf;
+  }
+  return 1.f;
+}
+
+// 8 consecutive bf16 -> floats (16-byte load when aligned and fully inside, else scalar with bound)
+__device__ __forceinline__ void load8_bf16(const __nv_bfloat16* p, int valid, bool vec, float* out) {
+  if (vec) {
+    uint4 q = *reinterpret_cast<const uint4*>(p);
+    out[0] = bf2f(q.x & 0xffffu); out[1] = bf2f(q.x >> 16);
+    out[2] = bf2f(q.y & 0xffffu); out[3] = bf2f(q.y >> 16);
+    out[4] = bf2f(q.z & 0xffffu); out[5] = bf2f(q.z >> 16);
+    out[6] = bf2f(q.w & 0xffffu); out[7] = bf2f(q.w >> 16);
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; j++) out[j] = j < valid ? __bfloat162float(p[j]) : 0.f;
+  }
+}
+__device__ __forceinline__ uint32_t pack2(float a, float b) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+__device__ __forceinline__ void store8_bf16(__nv_bfloat16* p, int valid, bool vec, const float* v) {
+  if (vec) {
+    uint4 q;
+    q.x = pack2(v[0], v[1]); q.y = pack2(v[2], v[3]); q.z = pack2(v[4], v[5]); q.w = pack2(v[6], v[7]);
+    *reinterpret_cast<uint4*>(p) = q;
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; j++)
+      if (j < valid) p[j] = __float2bfloat16_rn(v[j]);
+  }
+}
+
+template <int BN, bool A_MN, bool B_MN>
+__global__ void __launch_bounds__(192, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TcArgs p) {
+  extern __shared__ uint8_t smem_raw[];
+  constexpr uint32_t A_BYTES = BM * BK * 2;
+  constexpr uint32_t B_BYTES = BN * BK * 2;
+  constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bar_base = smem_base + STAGES * STAGE_BYTES;  // full[S], empty[S], accum, then tmem slot
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  const uint32_t accum_bar = bar_base + 8u * (2 * STAGES);
+  const uint32_t tmem_slot = bar_base + 8u * (2 * STAGES + 1);
+  uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
+  volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE_BYTES + 8u * (2 * STAGES + 1));
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN, split = blockIdx.z;
+  const int kchunk = (((p.K + p.splits - 1) / p.splits) + BK - 1) / BK * BK;
+  const int kbeg = split * kchunk;
+  const int kend = min(p.K, kbeg + kchunk);
+  const int num_kb = kend > kbeg ? (kend - kbeg + BK - 1) / BK : 0;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; s++) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    mbar_init(accum_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"((uint32_t)BN) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot_ptr;
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------
+    if (lane == 0) {
+      for (int kb = 0; kb < num_kb; kb++) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        if (!mbar_wait(empty_bar(s), ph ^ 1)) { atomicExch(p.status, 1); break; }
+        mbar_expect_tx(full_bar(s), STAGE_BYTES);
+        const uint32_t a_dst = smem_base + s * STAGE_BYTES;
+        const uint32_t b_dst = a_dst + A_BYTES;
+        const int k0 = kbeg + kb * BK;
+        if (!A_MN) {
+          tma_load_2d(a_dst, &map_a, k0, m0, full_bar(s));
+        } else {
+#pragma unroll
+          for (int a = 0; a < BM / 64; a++) tma_load_2d(a_dst + a * (BK * 128), &map_a, m0 + a * 64, k0, full_bar(s));
+        }
+        if (!B_MN) {
+          tma_load_2d(b_dst, &map_b, k0, n0, full_bar(s));
+        } else {
+#pragma unroll
+          for (int a = 0; a < BN / 64; a++) tma_load_2d(b_dst + a * (BK * 128), &map_b, n0 + a * 64, k0, full_bar(s));
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer ------------------------------
+    if (lane == 0) {
+      // instruction descriptor: fp32 accumulate, bf16 x bf16, majors, N>>3 at bit 17, M>>4 at bit 24
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16) |
+                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      bool ok = true;
+      for (int kb = 0; kb < num_kb && ok; kb++) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        if (!mbar_wait(full_bar(s), ph)) { atomicExch(p.status, 2); ok = false; break; }
+        tc_fence_after();
+        const uint32_t a_src = smem_base + s * STAGE_BYTES;
+        const uint32_t b_src = a_src + A_BYTES;
+#pragma unroll
+        for (int k = 0; k < BK / UMMA_K; k++) {
+          // K-major: rows of 128 bytes, 8-row groups 1024 bytes apart; a K step of 16 elements is
+          //          32 bytes inside the swizzled row.
+          // MN-major: 64-element (128-byte) runs along M/N, one per K index; 8 K rows form a
+          //          1024-byte group (stride offset), the next 64 M/N elements sit BK*128 bytes
+          //          further (leading offset); a K step of 16 is 16 rows = 2048 bytes.
+          const uint64_t ad = A_MN ? smem_desc(a_src + k * (UMMA_K * 128), BK * 128, 1024)
+                                   : smem_desc(a_src + k * (UMMA_K * 2), 16, 1024);
+          const uint64_t bd = B_MN ? smem_desc(b_src + k * (UMMA_K * 128), BK * 128, 1024)
+                                   : smem_desc(b_src + k * (UMMA_K * 2), 16, 1024);
+          tc_mma(tmem_base, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+        }
+        tc_commit(empty_bar(s));  // stage may be refilled once these MMAs have read it
+      }
+      tc_commit(accum_bar);       // accumulator complete (also fires when the loop bailed out)
+    }
+  } else {
+    // ------------------------------ epilogue ------------------------------
+    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    const int row = m0 + q * 32 + lane;
+    bool ok = mbar_wait(accum_bar, 0);
+    if (!ok) atomicExch(p.status, 3);
+    ok = __all_sync(0xffffffffu, ok);
+    tc_fence_after();
+    if (ok) {
+      const Epilogue& e = p.epi;
+      const bool row_ok = row < p.M;
+      const bool plain_store = p.splits > 1;
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        if (n0 + c0 >= p.N) break;  // warp-uniform
+        uint32_t r[32];
+        if (num_kb > 0) {
+          tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+        } else {  // an empty K range (a trailing split): the partial sum is zero
+#pragma unroll
+          for (int j = 0; j < 32; j++) r[j] = 0u;
+        }
+        if (!row_ok) continue;
+#pragma unroll
+        for (int g8 = 0; g8 < 4; g8++) {
+          const int n = n0 + c0 + g8 * 8;
+          const int valid = min(8, p.N - n);
+          if (valid <= 0) break;
+          float v[8];
+#pragma unroll
+          for (int j = 0; j < 8; j++) v[j] = __uint_as_float(r[g8 * 8 + j]);
+          if (plain_store) {
+            float* dst = p.ws + (long long)split * p.M * p.N + (long long)row * p.N + n;
+            const bool vec = valid == 8 && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0);
+            if (vec) {
+              reinterpret_cast<float4*>(dst)[0] = make_float4(v[0], v[1], v[2], v[3]);
+              reinterpret_cast<float4*>(dst)[1] = make_float4(v[4], v[5], v[6], v[7]);
+            } else {
+              for (int j = 0; j < valid; j++) dst[j] = v[j];
+            }
+            continue;
+          }
+          const long long ia = (long long)row * e.ld_aux + n;
+          const bool avec = valid == 8 && (e.ld_aux % 8 == 0);
+          float t[8];
+#pragma unroll
+          for (int j = 0; j < 8; j++) v[j] *= e.alpha;
+          if (e.bias) {
+#pragma unroll
+            for (int j = 0; j < 8; j++) if (j < valid) v[j] += __ldg(e.bias + n + j);
+          }
+          if (e.pre_out) {
+            __nv_bfloat16* po = (__nv_bfloat16*)e.pre_out + ia;
+            store8_bf16(po, valid, avec && ((reinterpret_cast<uintptr_t>(po) & 15) == 0), v);
+          }
+          if (e.act != ACT_NONE) {
+#pragma unroll
+            for (int j = 0; j < 8; j++) v[j] = act_apply_d(e.act, v[j]);
+          }
+          if (e.mul) {
+            const __nv_bfloat16* pm = (const __nv_bfloat16*)e.mul + ia;
+            load8_bf16(pm, valid, avec && ((reinterpret_cast<uintptr_t>(pm) & 15) == 0), t);
+#pragma unroll
+            for (int j = 0; j < 8; j++) v[j] *= t[j];
+          }
+          if (e.res) {
+            const __nv_bfloat16* pr = (const __nv_bfloat16*)e.res + ia;
+            load8_bf16(pr, valid, avec && ((reinterpret_cast<uintptr_t>(pr) & 15) == 0), t);
+#pragma unroll
+            for (int j = 0; j < 8; j++) v[j] += t[j];
+          }
+          if (e.dact != ACT_NONE) {
+            const __nv_bfloat16* pd = (const __nv_bfloat16*)e.dact_src + ia;
+            load8_bf16(pd, valid, avec && ((reinterpret_cast<uintptr_t>(pd) & 15) == 0), t);
+#pragma unroll
+            for (int j = 0; j < 8; j++) v[j] *= act_deriv_d(e.dact, t[j]);
+          }
+          const long long ic = (long long)row * p.ldc + n;
+          if (p.c_f32) {
+            float* dst = (float*)p.C + ic;
+            const bool vec = valid == 8 && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0);
+            if (vec) {
+              reinterpret_cast<float4*>(dst)[0] = make_float4(v[0], v[1], v[2], v[3]);
+              reinterpret_cast<float4*>(dst)[1] = make_float4(v[4], v[5], v[6], v[7]);
+            } else {
+              for (int j = 0; j < valid; j++) dst[j] = v[j];
+            }
+          } else {
+            __nv_bfloat16* dst = (__nv_bfloat16*)p.C + ic;
+            store8_bf16(dst, valid, valid == 8 && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0), v);
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)BN) : "memory");
+  }
+}
+
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn encode_fn() {
+  static EncodeFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = (EncodeFn)p;
+    else
+      cudaGetLastError();
+  }
+  return fn;
+}
+
+// 2-D bf16 tensor map: `inner` contiguous elements per row, `outer` rows `ld` elements apart;
+// box = 64 x box_outer, 128-byte swizzle, out-of-bounds elements read as zero.
+bool encode_2d(void* out, const void* base, long long inner, long long outer, long long ld, int box_outer) {
+  EncodeFn fn = encode_fn();
+  if (!fn) return false;
+  CUtensorMap tmp;
+  cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {64u, (cuuint32_t)box_outer};
+  cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = fn(&tmp, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r == CUDA_SUCCESS) memcpy(out, &tmp, sizeof(tmp));
+  return r == CUDA_SUCCESS;
+}
+
+template <int BN, bool A_MN, bool B_MN>
+cudaError_t launch_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s) {
+  constexpr size_t smem = (size_t)STAGES * (BM * BK * 2 + BN * BK * 2) + 8 * (2 * STAGES + 2) + 1024;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<BN, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  TcArgs p;
+  p.M = g.M; p.N = g.N; p.K = g.K;
+  p.C = g.C; p.ldc = g.ldc; p.c_f32 = g.c_f32;
+  p.splits = g.splits; p.ws = g.ws; p.epi = g.epi; p.status = plan.status;
+  dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, g.splits);
+  CUtensorMap ma, mb;
+  static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
+  memcpy(&ma, plan.map_a, sizeof(ma));
+  memcpy(&mb, plan.map_b, sizeof(mb));
+  tc_gemm_kernel<BN, A_MN, B_MN><<<grid, 192, smem, s>>>(ma, mb, p);
+  return cudaGetLastError();
+}
+
+template <int BN>
+cudaError_t launch_bn(const GemmArgs& g, const TcPlan& plan, cudaStream_t s) {
+  if (!plan.a_mn && !plan.b_mn) return launch_t<BN, false, false>(g, plan, s);
+  if (!plan.a_mn && plan.b_mn) return launch_t<BN, false, true>(g, plan, s);
+  if (plan.a_mn && !plan.b_mn) return launch_t<BN, true, false>(g, plan, s);
+  return launch_t<BN, true, true>(g, plan, s);
+}
+
+}  // namespace
+
+bool tc_gemm_supported(const GemmArgs& g) {
+  if (g.K < 64 || g.N < 16 || g.M < 1) return false;
+  auto operand_ok = [](const void* p, long long s_mn, long long s_k) {
+    if (reinterpret_cast<uintptr_t>(p) & 15) return false;
+    if (s_k == 1) return s_mn % 8 == 0 && s_mn > 0;
+    if (s_mn == 1) return s_k % 8 == 0 && s_k > 0;
+    return false;
+  };
+  if (!operand_ok(g.A, g.sa_m, g.sa_k) || !operand_ok(g.B, g.sb_n, g.sb_k)) return false;
+  // a [1 x K] operand is ambiguous (both strides may be 1): leave such GEMVs to the SIMT kernel
+  if ((g.sa_m == 1 && g.sa_k == 1) || (g.sb_n == 1 && g.sb_k == 1)) return false;
+  return true;
+}
+
+bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan) {
+  if (!tc_gemm_supported(g)) return false;
+  plan->a_mn = g.sa_k != 1;
+  plan->b_mn = g.sb_k != 1;
+  plan->bn = g.N <= 64 ? 64 : 128;
+  plan->status = status;
+  plan->launches = 1;
+  bool ok;
+  if (!plan->a_mn) ok = encode_2d(plan->map_a, g.A, g.K, g.M, g.sa_m, BM);
+  else ok = encode_2d(plan->map_a, g.A, g.M, g.K, g.sa_k, BK);
+  if (!ok) return false;
+  if (!plan->b_mn) ok = encode_2d(plan->map_b, g.B, g.K, g.N, g.sb_n, plan->bn);
+  else ok = encode_2d(plan->map_b, g.B, g.N, g.K, g.sb_k, BK);
+  return ok;
+}
+
+cudaError_t tc_gemm_launch(const GemmArgs& g, const TcPlan& plan, cudaStream_t s) {
+  return plan.bn == 64 ? launch_bn<64>(g, plan, s) : launch_bn<128>(g, plan, s);
+}
 
 }  // namespace erase

@@ -1,4 +1,9 @@
-// Tensor-core GEMM path (tcgen05 + TMEM accumulators, operands staged by TMA) for bf16 models.
+// Tensor-core GEMM path for bf16 models on sm_100a: operands staged in shared memory by TMA
+// (cp.async.bulk.tensor, 128-byte swizzle), tcgen05.mma issued by one thread with the fp32
+// accumulator in tensor memory (TMEM), epilogue warps reading it back with tcgen05.ld and
+// applying the fused epilogue (bias, activation, residual, DCN-v2 cross, activation derivative).
+// One kernel serves the forward (both operands K-major), the dgrad (B MN-major) and the wgrad
+// (both MN-major), so no operand is ever transposed in memory.
 #pragma once
 #include <cuda_runtime.h>
 
@@ -7,12 +12,21 @@
 namespace erase {
 
 struct TcPlan {
-  int launches = 0;
+  unsigned char map_a[128];  // CUtensorMap of A (copied into an aligned object at launch)
+  unsigned char map_b[128];  // CUtensorMap of B
+  int bn = 128;       // tile width (N)
+  int a_mn = 0;       // A is contiguous along M (not along K)
+  int b_mn = 0;
+  int launches = 1;
+  int* status = nullptr;  // device word set non-zero when a bounded wait expired
 };
 
-// Decides whether the tensor-core kernel takes this GEMM (bf16 operands, aligned strides) and,
-// if so, prepares everything the launch needs.  Returns false to leave it to the SIMT kernel.
-bool tc_gemm_plan(const GemmArgs& g, TcPlan* plan);
+// True if the tensor-core kernel can take this GEMM: bf16 operands, 16-byte aligned bases,
+// leading strides that are multiples of 8 elements, K >= 64 and N >= 16.
+bool tc_gemm_supported(const GemmArgs& g);
+// Encodes the TMA descriptors.  g.ws must already point at splits*M*N floats when g.splits > 1.
+// Returns false (and leaves the GEMM to the SIMT kernel) if a descriptor cannot be encoded.
+bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan);
 cudaError_t tc_gemm_launch(const GemmArgs& g, const TcPlan& plan, cudaStream_t s);
 
 }  // namespace erase

@@ -8,6 +8,11 @@ from paper_2608_18469_b200 import binding, synth
 from tests import util
 
 TOL = {"f32": 1e-4, "bf16": 2e-2}     # relative L2 per tensor against the fp64 oracle
+# Optimizer alone (fp64 update rule applied to the library's own gradient vs the fp32 kernel).
+# A tensor that starts at zero (LayerNorm shift) consists of the update only, so its relative
+# error is that of a handful of fp32 operations (m, v, two bias corrections, sqrt, divide):
+# a few 1e-7 each, 2e-6 observed; any formula mistake shows up at 1e-3 or more.
+OPT_TOL = 1e-5
 
 
 class DevBatch:
@@ -95,7 +100,7 @@ def compare_teacher_forced(spec, steps, seed=0, n_streams=2, flags=0, report=Non
                 key = f"param b{b} {name}"
                 worst[key] = max(worst.get(key, 0), perr)
                 if report is None:
-                    assert perr <= 2e-6, (it, key, perr)
+                    assert perr <= OPT_TOL, (it, key, perr)
             params, state = new_params, new_state
     finally:
         m.close()
