@@ -289,7 +289,7 @@ def run_gpu(args, spec, cfg_name):
         cpu = {"value": val, "unit": unit_name(spec), "cores": oracle_threads(), "kind": "oracle",
                "sample": f"1 full oracle step of the workload's batch ({units} units) after 1 warm-up step; {ms:.0f} ms"}
 
-    del main, stage, dev
+    del main, stage, dev, host
     torch.cuda.synchronize()
     model.close()
     if rank != 0:

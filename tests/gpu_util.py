@@ -79,7 +79,18 @@ def compare_teacher_forced(spec, steps, seed=0, n_streams=2, flags=0, report=Non
                     m.set_opt_state(i, m32, v32, state["t"])
             m.step(n_streams=n_streams, flags=flags, **db.args())
             got_l = m.losses()
-            want_l, want_g, new_params, new_state = orc.step(spec, params, state, batch)
+            # oracle: forward/backward at the operand values, optimizer on the fp32 masters
+            want_l, want_g = orc.forward_backward(spec, util.operand_params(spec, params), batch)
+            new_params = {"input": params["input"], "blocks": []}
+            new_state = {"t": state["t"] + 1, "m": [], "v": []}
+            for b, p in enumerate(params["blocks"]):
+                np_, nm, nv = {}, {}, {}
+                for k in p:
+                    np_[k], nm[k], nv[k] = orc.optimizer_update(spec["opt"], p[k], want_g[b][k], state["m"][b][k],
+                                                                state["v"][b][k], state["t"] + 1)
+                new_params["blocks"].append(np_)
+                new_state["m"].append(nm)
+                new_state["v"].append(nv)
             for b in range(len(want_l)):
                 err = abs(got_l[b] - want_l[b]) / max(abs(want_l[b]), 1e-12)
                 worst[f"loss{b}"] = max(worst.get(f"loss{b}", 0), err)

@@ -30,3 +30,26 @@ def tiny_specs():
     s["ctr"] = synth.ctr_spec(batch=3, n_dense=2, n_sparse=3, table_rows=7, emb_dim=4,
                               tower=(6, 5, 4), n_cross=2, dtype="f32")
     return s
+
+
+def operand_params(spec, params):
+    """The parameter values the bf16 path actually multiplies with.
+
+    A bf16 model keeps fp32 master parameters and feeds its GEMMs bf16 roundings of the weight
+    matrices (refreshed by the optimizer).  Those roundings are the operands ("bf16 operands,
+    fp32 accumulation"), so parity evaluates the oracle at the same operand values; gradients are
+    then applied to the fp32 masters.  Biases, LayerNorm parameters and the 1-wide BCE head vector
+    are consumed in fp32 and stay unrounded.  fp32 models are returned unchanged.
+    """
+    if spec["dtype"] != "bf16":
+        return params
+    out = {"input": params["input"], "blocks": []}
+    for blk, p in zip(spec["blocks"], params["blocks"]):
+        q = {}
+        for k, v in p.items():
+            if v.ndim == 2 and not (k == "Wh" and blk["head"] == "bce"):
+                q[k] = synth.bf16_round(v.astype(np.float32)).astype(np.float64)
+            else:
+                q[k] = v
+        out["blocks"].append(q)
+    return out
