@@ -181,117 +181,130 @@ def run_gpu(args, spec, cfg_name):
 
     model = binding.Model(spec)
     model.set_all(synth.init_params(spec, 0))
-    main = torch.cuda.ExternalStream(model.main_stream())
 
-    # pool of batches resident in HBM, and their pinned host copies for the end-to-end leg
-    host, dev = [], []
-    for i in range(POOL):
-        b = synth.make_batch(spec, 0, index=i)
-        h = {}
-        if spec["input"] == "dense":
-            x = torch.from_numpy(b["x"])
-            h["x"] = x.to(torch.bfloat16) if spec["dtype"] == "bf16" else x
-            h["y"] = torch.from_numpy(b["y"])
-        elif spec["input"] == "tokens":
-            h["ids"] = torch.from_numpy(b["ids"])
+    def measure():
+        """Everything that owns torch tensors, events or streams lives in this scope, so that it
+        is released before the model (and its CUDA streams) is destroyed."""
+        main = torch.cuda.ExternalStream(model.main_stream())
+
+        # pool of batches resident in HBM, and their pinned host copies for the end-to-end leg
+        host, dev = [], []
+        for i in range(POOL):
+            b = synth.make_batch(spec, 0, index=i)
+            h = {}
+            if spec["input"] == "dense":
+                x = torch.from_numpy(b["x"])
+                h["x"] = x.to(torch.bfloat16) if spec["dtype"] == "bf16" else x
+                h["y"] = torch.from_numpy(b["y"])
+            elif spec["input"] == "tokens":
+                h["ids"] = torch.from_numpy(b["ids"])
+            else:
+                h["x"], h["ids"], h["y"] = (torch.from_numpy(b[k]) for k in ("dense", "ids", "y"))
+            h = {k: v.contiguous().pin_memory() for k, v in h.items()}
+            host.append(h)
+            dev.append({k: v.cuda() for k, v in h.items()})
+        torch.cuda.synchronize()
+
+        def ptrs(d):
+            return {k: d[k].data_ptr() if k in d else None for k in ("x", "ids", "y")}
+
+        def timed(ns, fl, steps, warmup):
+            """K steps on resident inputs, per-step CUDA events on the launching stream."""
+            for i in range(warmup):
+                model.step(n_streams=ns, flags=fl, **ptrs(dev[i % POOL]))
+            model.sync()
+            evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+            l0 = model.launch_count()
+            barrier()
+            evs[0].record(main)
+            for i in range(steps):
+                model.step(n_streams=ns, flags=fl, **ptrs(dev[(warmup + i) % POOL]))
+                evs[i + 1].record(main)
+            model.sync()
+            barrier()
+            total_ms = evs[0].elapsed_time(evs[-1])
+            per = np.array([evs[i].elapsed_time(evs[i + 1]) for i in range(steps)])
+            return max_over_ranks(total_ms), per, model.launch_count() - l0
+
+        sampler = ClockSampler(local)
+        # serial first (context), then the ERASE schedule under the clock sampler
+        ser_ms, ser_per, _ = timed(1, flags, args.steps, args.warmup)
+        sampler.start()
+        era_ms, era_per, launches = timed(n_streams, flags, args.steps, args.warmup)
+        clocks = sampler.stop()
+
+        # end to end through the C ABI: pinned host batch -> device copy, step, losses back to host
+        stage = {k: torch.empty_like(v) for k, v in dev[0].items()}
+        h2d = sum(v.numel() * v.element_size() for v in stage.values())
+        d2h = nb * 4
+
+        def e2e_step(i):
+            with torch.cuda.stream(main):
+                for k in stage:
+                    stage[k].copy_(host[i % POOL][k], non_blocking=True)
+            model.step(n_streams=n_streams, flags=flags, **ptrs(stage))
+            return model.losses()
+
+        for i in range(args.warmup):
+            e2e_step(i)
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(args.steps):
+            e2e_step(args.warmup + i)
+        model.sync()
+        barrier()
+        e2e_ms = max_over_ranks(1e3 * (time.perf_counter() - t0))
+
+        # per-kernel attribution: profiled serial steps (events around every operation)
+        agg = {}
+        nprof = 3
+        for i in range(nprof + 1):
+            recs = model.profile_step(**ptrs(dev[i % POOL]))
+            if i == 0:
+                continue    # warm-up of the profiling path
+            for r in recs:
+                a = agg.setdefault(r["name"], {"ms": 0.0, "flops": 0.0, "bytes": 0.0, "runs": 0, "launches": 0})
+                a["ms"] += r["ms"]; a["flops"] += r["flops"]; a["bytes"] += r["bytes"]
+                a["runs"] += 1; a["launches"] += r["launches"]
+        top = max(agg, key=lambda k: agg[k]["ms"])
+        peaks = measured_peaks()
+        t = agg[top]
+        if top.startswith("gemm") or top.startswith("attention"):
+            ach = t["flops"] / (t["ms"] * 1e-3) / 1e12
+            roof = {"kernel": top, "bound": "tensor", "achieved": ach, "peak": peaks["tflops"], "unit": "TFLOP/s",
+                    "frac": ach / peaks["tflops"]}
         else:
-            h["x"], h["ids"], h["y"] = (torch.from_numpy(b[k]) for k in ("dense", "ids", "y"))
-        h = {k: v.contiguous().pin_memory() for k, v in h.items()}
-        host.append(h)
-        dev.append({k: v.cuda() for k, v in h.items()})
-    torch.cuda.synchronize()
+            ach = t["bytes"] / (t["ms"] * 1e-3) / 1e9
+            roof = {"kernel": top, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": ach / peaks["hbm_gbs"]}
+        roof["peak_source"] = peaks["source"] + (" (sustained bf16 GEMM)" if roof["bound"] == "tensor" else " (copy)")
+        roof["avg_launch_ms"] = t["ms"] / max(t["launches"], 1)
+        tr = None
+        tp = os.path.join(ROOT, "profiles", "traffic.json")
+        if os.path.exists(tp):
+            tr = json.load(open(tp)).get(cfg_name, {}).get(top)
+        roof["traffic"] = tr
+        roof["kernel_share"] = {k: round(v["ms"] / sum(x["ms"] for x in agg.values()), 4)
+                                for k, v in sorted(agg.items(), key=lambda kv: -kv[1]["ms"])[:8]}
 
-    def ptrs(d):
-        return {k: d[k].data_ptr() if k in d else None for k in ("x", "ids", "y")}
+        cpu = None
+        if rank == 0 and world == 1 and not args.no_cpu_baseline:
+            val, ms = time_oracle(spec, 1, 1)
+            cpu = {"value": val, "unit": unit_name(spec), "cores": oracle_threads(), "kind": "oracle",
+                   "sample": f"1 full oracle step of the workload's batch ({units} units) after 1 warm-up step; {ms:.0f} ms"}
 
-    def timed(ns, fl, steps, warmup):
-        """K steps on resident inputs, per-step CUDA events on the launching stream."""
-        for i in range(warmup):
-            model.step(n_streams=ns, flags=fl, **ptrs(dev[i % POOL]))
-        model.sync()
-        evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
-        l0 = model.launch_count()
-        barrier()
-        evs[0].record(main)
-        for i in range(steps):
-            model.step(n_streams=ns, flags=fl, **ptrs(dev[(warmup + i) % POOL]))
-            evs[i + 1].record(main)
-        model.sync()
-        barrier()
-        total_ms = evs[0].elapsed_time(evs[-1])
-        per = np.array([evs[i].elapsed_time(evs[i + 1]) for i in range(steps)])
-        return max_over_ranks(total_ms), per, model.launch_count() - l0
 
-    sampler = ClockSampler(local)
-    # serial first (context), then the ERASE schedule under the clock sampler
-    ser_ms, ser_per, _ = timed(1, flags, args.steps, args.warmup)
-    sampler.start()
-    era_ms, era_per, launches = timed(n_streams, flags, args.steps, args.warmup)
-    clocks = sampler.stop()
+        return dict(ser_ms=ser_ms, ser_per=ser_per, era_ms=era_ms, era_per=era_per, launches=launches,
+                    clocks=clocks, e2e_ms=e2e_ms, h2d=h2d, d2h=d2h, roof=roof, cpu=cpu)
 
-    # end to end through the C ABI: pinned host batch -> device copy, step, losses back to host
-    stage = {k: torch.empty_like(v) for k, v in dev[0].items()}
-    h2d = sum(v.numel() * v.element_size() for v in stage.values())
-    d2h = nb * 4
-
-    def e2e_step(i):
-        with torch.cuda.stream(main):
-            for k in stage:
-                stage[k].copy_(host[i % POOL][k], non_blocking=True)
-        model.step(n_streams=n_streams, flags=flags, **ptrs(stage))
-        return model.losses()
-
-    for i in range(args.warmup):
-        e2e_step(i)
-    barrier()
-    t0 = time.perf_counter()
-    for i in range(args.steps):
-        e2e_step(args.warmup + i)
-    model.sync()
-    barrier()
-    e2e_ms = max_over_ranks(1e3 * (time.perf_counter() - t0))
-
-    # per-kernel attribution: profiled serial steps (events around every operation)
-    agg = {}
-    nprof = 3
-    for i in range(nprof + 1):
-        recs = model.profile_step(**ptrs(dev[i % POOL]))
-        if i == 0:
-            continue    # warm-up of the profiling path
-        for r in recs:
-            a = agg.setdefault(r["name"], {"ms": 0.0, "flops": 0.0, "bytes": 0.0, "runs": 0, "launches": 0})
-            a["ms"] += r["ms"]; a["flops"] += r["flops"]; a["bytes"] += r["bytes"]
-            a["runs"] += 1; a["launches"] += r["launches"]
-    top = max(agg, key=lambda k: agg[k]["ms"])
+    import gc
     peaks = measured_peaks()
-    t = agg[top]
-    if top.startswith("gemm") or top.startswith("attention"):
-        ach = t["flops"] / (t["ms"] * 1e-3) / 1e12
-        roof = {"kernel": top, "bound": "tensor", "achieved": ach, "peak": peaks["tflops"], "unit": "TFLOP/s",
-                "frac": ach / peaks["tflops"]}
-    else:
-        ach = t["bytes"] / (t["ms"] * 1e-3) / 1e9
-        roof = {"kernel": top, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": ach / peaks["hbm_gbs"]}
-    roof["peak_source"] = peaks["source"] + (" (sustained bf16 GEMM)" if roof["bound"] == "tensor" else " (copy)")
-    roof["avg_launch_ms"] = t["ms"] / max(t["launches"], 1)
-    tr = None
-    tp = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tp):
-        tr = json.load(open(tp)).get(cfg_name, {}).get(top)
-    roof["traffic"] = tr
-    roof["kernel_share"] = {k: round(v["ms"] / sum(x["ms"] for x in agg.values()), 4)
-                            for k, v in sorted(agg.items(), key=lambda kv: -kv[1]["ms"])[:8]}
-
-    cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        val, ms = time_oracle(spec, 1, 1)
-        cpu = {"value": val, "unit": unit_name(spec), "cores": oracle_threads(), "kind": "oracle",
-               "sample": f"1 full oracle step of the workload's batch ({units} units) after 1 warm-up step; {ms:.0f} ms"}
-
-    del main, stage, dev, host
+    r = measure()
+    gc.collect()
     torch.cuda.synchronize()
     model.close()
+    ser_ms, ser_per, era_ms, era_per, launches = r["ser_ms"], r["ser_per"], r["era_ms"], r["era_per"], r["launches"]
+    clocks, e2e_ms, h2d, d2h, roof, cpu = r["clocks"], r["e2e_ms"], r["h2d"], r["d2h"], r["roof"], r["cpu"]
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()

@@ -376,7 +376,8 @@ struct Builder {
     gemm(ops, g);
   }
   // dW[N,K] = dY[M,N]^T X[M,K]  (fp32, deterministic split over M), db[N] = column sums of dY
-  void lin_wgrad(OpList& ops, const void* dY, const void* X, long long ldx, int widx, int bidx, int M, int N, int K) {
+  void lin_wgrad(OpList& ops, const void* dY, const void* X, long long ldx, int widx, int bidx, int M, int N, int K,
+                 bool skip_bias = false) {
     GemmArgs g;
     g.M = N; g.N = K; g.K = M;
     g.A = dY; g.sa_m = 1; g.sa_k = N;
@@ -390,7 +391,7 @@ struct Builder {
     g.splits = splits < 1 ? 1 : splits;
     gemm_tag = "gemm_wgrad";
     gemm(ops, g);
-    if (bidx >= 0) bias_grad(ops, dY, N, M, N, bidx);
+    if (bidx >= 0 && !skip_bias) bias_grad(ops, dY, N, M, N, bidx);
   }
   void bias_grad(OpList& ops, const void* dY, long long ld, int M, int N, int bidx) {
     int chunks = colsum_chunks(M, N);
@@ -403,8 +404,12 @@ struct Builder {
 
   // ---- heads: forward computes the local loss and the loss gradient, backward the head's own
   // gradients and dz (times act'(src) when the block ends in an activation) ------------------
-  void head(int b, const erase_block_spec& k, const void* z, int d, int wh, int bh, OpList& f, OpList& bw, void* dz,
-            int dact, const void* dact_src) {
+  // last_bias >= 0 (BCE head only): also emit the gradient of the bias of the Linear that produced z,
+  // db[c] = w[c] * sum_r ds[r] * act'(src[r,c]), from the fp32 loss gradient rather than from the
+  // bf16-rounded dz (the sum over r cancels heavily when the labels are balanced).  Returns true
+  // if it did, so that the caller skips the ordinary column sum for that bias.
+  bool head(int b, const erase_block_spec& k, const void* z, int d, int wh, int bh, OpList& f, OpList& bw, void* dz,
+            int dact, const void* dact_src, int last_bias = -1) {
     erase_model* mm = m;
     bool bf = m->bf16;
     int rows = m->rows;
@@ -435,6 +440,16 @@ struct Builder {
         bw.push_back({[=](cudaStream_t s) { return colsum(ds, false, 1, rows, 1, nullptr, ws, chunks, out, s); }, chunks > 1 ? 2 : 1});
         note(bw, "colsum", rows, 4.0 * rows);
       }
+      if (last_bias >= 0) {
+        int chunks = colsum_chunks(rows, d);
+        float* ws = chunks > 1 ? f32_buf((size_t)chunks * d) : nullptr;
+        float* out = G(last_bias);
+        const void* src = dact != ACT_NONE ? dact_src : nullptr;
+        bw.push_back({[=](cudaStream_t s) { return colsum(src, bf, d, rows, d, ds, ws, chunks, out, s, dact, w); }, chunks > 1 ? 2 : 1});
+        note(bw, "colsum", 2.0 * rows * d, src ? (double)rows * d * m->esz : 4.0 * rows);
+        return true;
+      }
+      return false;
     } else {
       int V = k.head_out, T_ = m->spec.seq;
       void* logits = act_buf((size_t)rows * V);
@@ -450,6 +465,7 @@ struct Builder {
         bw.push_back({[=](cudaStream_t s) { return ew_dact(dz, dact_src, dact, n, bf, s); }, 1});
         note(bw, "ew_dact", (double)n, 3.0 * n * m->esz);
       }
+      return false;
     }
   }
 
@@ -491,11 +507,13 @@ struct Builder {
   }
   // d = gradient w.r.t. the stack output already multiplied by the last activation's derivative.
   // Returns the gradient w.r.t. the stack input when need_dx.
-  void* stack_bwd(OpList& bw, const erase_block_spec& k, const Stack& st, long long ldin, void* d, int first_tensor, bool need_dx) {
+  void* stack_bwd(OpList& bw, const erase_block_spec& k, const Stack& st, long long ldin, void* d, int first_tensor, bool need_dx,
+                  bool last_bias_done) {
     int L = k.n_dims - 1;
     for (int i = L - 1; i >= 0; i--) {
       int K = k.dims[i], N = k.dims[i + 1];
-      lin_wgrad(bw, d, st.in[i], i == 0 ? ldin : K, first_tensor + 2 * i, first_tensor + 2 * i + 1, m->rows, N, K);
+      lin_wgrad(bw, d, st.in[i], i == 0 ? ldin : K, first_tensor + 2 * i, first_tensor + 2 * i + 1, m->rows, N, K,
+                last_bias_done && i == L - 1);
       if (i > 0 || need_dx) {
         void* dx = act_buf((size_t)m->rows * K);
         Epilogue e;
@@ -518,8 +536,9 @@ struct Builder {
     Stack st = stack_fwd(f, k, zin, k.dims[0], tower, first);
     int dout = k.dims[L];
     void* dz = act_buf((size_t)m->rows * dout);
-    head(b, k, st.out, dout, first + 2 * L, first + 2 * L + 1, f, bw, dz, st.act[L - 1], st.src[L - 1]);
-    stack_bwd(bw, k, st, k.dims[0], dz, first, false);
+    bool lb = head(b, k, st.out, dout, first + 2 * L, first + 2 * L + 1, f, bw, dz, st.act[L - 1], st.src[L - 1],
+                   first + 2 * (L - 1) + 1);
+    stack_bwd(bw, k, st, k.dims[0], dz, first, false, lb);
     return st.out;
   }
 
@@ -649,8 +668,9 @@ struct Builder {
     Stack st = stack_fwd(f, k, feats, fw, true, first + 2);
     int dout = k.dims[L];
     void* dz = act_buf((size_t)rows * dout);
-    head(b, k, st.out, dout, first + 2 + 2 * L, first + 2 + 2 * L + 1, f, bw, dz, st.act[L - 1], st.src[L - 1]);
-    void* dfeat = stack_bwd(bw, k, st, fw, dz, first + 2, true);
+    bool lb = head(b, k, st.out, dout, first + 2 + 2 * L, first + 2 + 2 * L + 1, f, bw, dz, st.act[L - 1], st.src[L - 1],
+                   first + 2 + 2 * (L - 1) + 1);
+    void* dfeat = stack_bwd(bw, k, st, fw, dz, first + 2, true, lb);
     void* dproj = act_buf((size_t)rows * e_);
     bw.push_back({[=](cudaStream_t s2) { return dot_bwd(dfeat, x0, w0, dproj, rows, ns, e_, fw, bf, s2); }, 1});
     note(bw, "dot_bwd", 2.0 * rows * ns * e_, (double)rows * (w0 + fw) * m->esz);

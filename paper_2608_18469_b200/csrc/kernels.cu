@@ -177,7 +177,8 @@ int colsum_chunks(int rows, int cols) {
 template <typename T>
 __global__ void __launch_bounds__(256) colsum_kernel(const T* __restrict__ X, long long ldx, int rows,
                                                      int cols, const float* __restrict__ scale,
-                                                     float* __restrict__ dst, int chunks) {
+                                                     float* __restrict__ dst, int chunks, int dact,
+                                                     const float* __restrict__ colscale) {
   __shared__ float sm[8][33];
   int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
   int c = blockIdx.x * 32 + cx;
@@ -186,7 +187,8 @@ __global__ void __launch_bounds__(256) colsum_kernel(const T* __restrict__ X, lo
   float a = 0.f;
   if (c < cols)
     for (int r = rb + ry; r < re; r += 8) {
-      float v = ldf(X + (long long)r * ldx + c);
+      float v = X ? ldf(X + (long long)r * ldx + c) : 1.f;
+      if (dact != ACT_NONE) v = act_deriv(dact, v);
       if (scale) v *= scale[r];
       a += v;
     }
@@ -196,16 +198,17 @@ __global__ void __launch_bounds__(256) colsum_kernel(const T* __restrict__ X, lo
     float t = 0.f;
 #pragma unroll
     for (int i = 0; i < 8; i++) t += sm[i][cx];
+    if (colscale) t *= colscale[c];
     dst[(long long)blockIdx.y * cols + c] = t;
   }
 }
 
 cudaError_t colsum(const void* X, bool x_bf16, long long ldx, int rows, int cols, const float* scale,
-                   float* ws, int chunks, float* out, cudaStream_t s) {
+                   float* ws, int chunks, float* out, cudaStream_t s, int dact, const float* colscale) {
   dim3 grid(cdiv(cols, 32), chunks);
   float* dst = chunks == 1 ? out : ws;
-  if (x_bf16) colsum_kernel<bf16_t><<<grid, 256, 0, s>>>((const bf16_t*)X, ldx, rows, cols, scale, dst, chunks);
-  else colsum_kernel<float><<<grid, 256, 0, s>>>((const float*)X, ldx, rows, cols, scale, dst, chunks);
+  if (x_bf16) colsum_kernel<bf16_t><<<grid, 256, 0, s>>>((const bf16_t*)X, ldx, rows, cols, scale, dst, chunks, dact, colscale);
+  else colsum_kernel<float><<<grid, 256, 0, s>>>((const float*)X, ldx, rows, cols, scale, dst, chunks, dact, colscale);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess || chunks == 1) return e;
   return splitk_reduce(ws, chunks, cols, cols, out, cols, s);

@@ -51,11 +51,14 @@ cudaError_t gemm_simt(const GemmArgs& g, bool bf16, cudaStream_t s);
 cudaError_t splitk_reduce(const float* ws, int splits, long long mn, int N, float* out, long long ldo,
                           cudaStream_t s);
 
-// out[c] = sum_r scale[r] * X[r, c]  (scale may be null); X is [rows, cols] with row stride ldx.
-// Two-stage with a fixed row partition into `chunks`; ws holds chunks*cols floats.
+// out[c] = colscale[c] * sum_r scale[r] * f(X[r, c]); X is [rows, cols] with row stride ldx,
+// f = identity or the derivative of activation `dact` evaluated at X; scale and colscale may be
+// null (read as 1) and so may X (read as 1).  Two-stage with a fixed row partition into `chunks`;
+// ws holds chunks*cols floats.
 int colsum_chunks(int rows, int cols);
 cudaError_t colsum(const void* X, bool x_bf16, long long ldx, int rows, int cols, const float* scale,
-                   float* ws, int chunks, float* out, cudaStream_t s);
+                   float* ws, int chunks, float* out, cudaStream_t s, int dact = ACT_NONE,
+                   const float* colscale = nullptr);
 
 // LayerNorm over the last dimension (eps 1e-5, biased variance); saves mean and 1/std per row.
 cudaError_t layernorm_fwd(const void* x, const float* gain, const float* shift, void* y, float* mean,

@@ -43,7 +43,10 @@ def operand_params(spec, params):
     """
     if spec["dtype"] != "bf16":
         return params
-    out = {"input": params["input"], "blocks": []}
+    inp = params["input"]
+    if spec["input"] == "ctr":      # x0 is stored in bf16: the frozen table rows are operands too
+        inp = {k: synth.bf16_round(v.astype(np.float32)).astype(np.float64) for k, v in inp.items()}
+    out = {"input": inp, "blocks": []}
     for blk, p in zip(spec["blocks"], params["blocks"]):
         q = {}
         for k, v in p.items():
@@ -53,3 +56,10 @@ def operand_params(spec, params):
                 q[k] = v
         out["blocks"].append(q)
     return out
+
+
+def operand_batch(spec, batch):
+    """The batch as the bf16 path sees it: CTR dense features are packed into the bf16 x0."""
+    if spec["dtype"] == "bf16" and spec["input"] == "ctr":
+        return dict(batch, dense=synth.bf16_round(batch["dense"]))
+    return batch
