@@ -206,6 +206,32 @@ ERASE_API erase_status erase_gemm(int32_t dtype, int32_t M, int32_t N, int32_t K
                                   int64_t sa_k, const void* B, int64_t sb_n, int64_t sb_k, void* C, int64_t ldc,
                                   int32_t c_f32, int32_t splits, int32_t engine, void* stream);
 
+/* erase_gemm for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this is a deployment convenience of the library, not part of the method.)
+ *
+ * Who needs it: code running inside a process whose device memory is entirely managed by
+ * someone else's pool, code on a latency budget that cannot afford the device-wide
+ * synchronisation a cudaMalloc/cudaFree may imply, and code called at moments when allocation is
+ * forbidden.  Same arguments, semantics and results as erase_gemm, but the split-K workspace and
+ * the status word live in one fixed array inside the library's device image
+ * (ERASE_STATIC_WS_FLOATS floats, 8 MiB, plus 256 bytes; every GPU that loads the library holds
+ * it until the process exits).  The call performs no cudaMalloc, cudaFree or other allocating
+ * call, here or in any library.
+ *   - splits*M*N must not exceed ERASE_STATIC_WS_FLOATS (only when splits > 1); larger
+ *     requests are refused with EINVAL and a message naming the limit.  Nothing is launched.
+ *   - The first call on each device looks up the array's device address (once per device, with
+ *     that device current).  Make that first call outside any CUDA stream capture.
+ *   - All calls on a device share the array and it keeps the last call's contents; the call
+ *     clears what must start at zero itself.  Two calls whose GPU work overlaps in time (different
+ *     streams or threads) race on it: issue them one after the other.
+ * The text of this entry point's last error on the calling thread: erase_gemm_static_error(). */
+#define ERASE_STATIC_WS_FLOATS (2u * 1024u * 1024u)
+ERASE_API erase_status erase_gemm_static(int32_t dtype, int32_t M, int32_t N, int32_t K, const void* A,
+                                         int64_t sa_m, int64_t sa_k, const void* B, int64_t sb_n, int64_t sb_k,
+                                         void* C, int64_t ldc, int32_t c_f32, int32_t splits, int32_t engine,
+                                         void* stream);
+ERASE_API const char* erase_gemm_static_error(void);
+
 /* One record per operation of a profiled step. */
 typedef struct {
   char name[32];    /* kernel class: gemm_fwd, gemm_dgrad, gemm_wgrad, softmax_ce, opt_update, ...   */

@@ -83,6 +83,10 @@ EXPORTS = {
     "erase_gemm": (C.c_int, [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int64, C.c_int64,
                              C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_int64, C.c_int32, C.c_int32,
                              C.c_int32, C.c_void_p]),
+    "erase_gemm_static": (C.c_int, [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int64, C.c_int64,
+                                    C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_int64, C.c_int32, C.c_int32,
+                                    C.c_int32, C.c_void_p]),
+    "erase_gemm_static_error": (C.c_char_p, []),
     "erase_profile_step": (C.c_int, [C.c_void_p, C.POINTER(Batch), C.POINTER(OpRecord), C.c_int32,
                                      C.POINTER(C.c_int32)]),
     "erase_last_error": (C.c_char_p, [C.c_void_p]),
@@ -243,6 +247,18 @@ def gemm(dtype, M, N, K, A, sa_m, sa_k, B, sb_n, sb_k, Cptr, ldc, c_f32=False, s
                           engine, stream)
     if st != OK:
         raise EraseError(st, lib().erase_last_error(None).decode())
+
+
+STATIC_WS_FLOATS = 2 * 1024 * 1024
+
+
+def gemm_static(dtype, M, N, K, A, sa_m, sa_k, B, sb_n, sb_k, Cptr, ldc, c_f32=False, splits=1, engine=0,
+                stream=None):
+    """erase_gemm_static (no device allocation) on device pointers; raises EraseError on failure."""
+    st = lib().erase_gemm_static(_DTYPE[dtype], M, N, K, A, sa_m, sa_k, B, sb_n, sb_k, Cptr, ldc, int(c_f32),
+                                 splits, engine, stream)
+    if st != OK:
+        raise EraseError(st, lib().erase_gemm_static_error().decode())
 
 
 def arena_bytes(spec):
