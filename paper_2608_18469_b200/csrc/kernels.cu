@@ -599,6 +599,7 @@ static cudaError_t attention_fwd_t(const T* qkv, T* o, float* lse, int batch, in
 cudaError_t attention_fwd(const void* qkv, void* o, float* lse, int batch, int T_, int heads, int dh,
                           bool bf16, cudaStream_t s) {
   if (dh > 32 * ATT_MAXC) return cudaErrorInvalidValue;
+  if (bf16 && attention_mma_supported(dh, heads * dh)) return attention_fwd_mma(qkv, o, lse, batch, T_, heads, s);
   return bf16 ? attention_fwd_t<bf16_t>((const bf16_t*)qkv, (bf16_t*)o, lse, batch, T_, heads, dh, s)
               : attention_fwd_t<float>((const float*)qkv, (float*)o, lse, batch, T_, heads, dh, s);
 }
@@ -624,6 +625,7 @@ static cudaError_t attention_bwd_t(const T* qkv, const T* o, const T* dout, cons
 cudaError_t attention_bwd(const void* qkv, const void* o, const void* dout, const float* lse, float* delta,
                           void* dqkv, int batch, int T_, int heads, int dh, bool bf16, cudaStream_t s) {
   if (dh > 32 * ATT_MAXC) return cudaErrorInvalidValue;
+  if (bf16 && attention_mma_supported(dh, heads * dh)) return attention_bwd_mma(qkv, o, dout, lse, delta, dqkv, batch, T_, heads, s);
   return bf16 ? attention_bwd_t<bf16_t>((const bf16_t*)qkv, (const bf16_t*)o, (const bf16_t*)dout, lse, delta, (bf16_t*)dqkv, batch, T_, heads, dh, s)
               : attention_bwd_t<float>((const float*)qkv, (const float*)o, (const float*)dout, lse, delta, (float*)dqkv, batch, T_, heads, dh, s);
 }

@@ -81,6 +81,12 @@ cudaError_t attention_bwd(const void* qkv, const void* o, const void* dout, cons
                           float* delta, void* dqkv, int batch, int T, int heads, int dh, bool bf16,
                           cudaStream_t s);
 
+// Tensor-core versions (mma.sync m16n8k16) for bf16 with 64-wide heads; same contracts.
+bool attention_mma_supported(int dh, int d);
+cudaError_t attention_fwd_mma(const void* qkv, void* o, float* lse, int batch, int T, int heads, cudaStream_t s);
+cudaError_t attention_bwd_mma(const void* qkv, const void* o, const void* dout, const float* lse, float* delta,
+                              void* dqkv, int batch, int T, int heads, cudaStream_t s);
+
 // Softmax cross-entropy over logits [rows, V] (row stride V), in place:
 // logits <- (softmax - onehot(target)) * inv_rows; rowloss[r] = logsumexp - logit[target].
 // target of row r = ids[(r / T) * (T + 1) + (r % T) + 1].

@@ -62,6 +62,9 @@ def _bf16_cases():
     s["c5_w512_b512"] = synth.config("C5", w=512, batch=512)
     s["mlp_bf16_ragged"] = synth.mlp_spec(200, 328, 2, 300, "gelu", "bf16")
     s["lm_bf16_small"] = synth.lm_spec(2, 128, 2, 512, 128, 4, 1000)
+    s["lm_bf16_ragged_T"] = synth.lm_spec(2, 192, 3, 384, 100, 3, 777)     # T not a multiple of the 64-tile
+    s["lm_bf16_T320"] = synth.lm_spec(1, 64, 1, 128, 320, 2, 300)            # five key tiles per head
+    s["lm_bf16_dh32"] = synth.lm_spec(1, 128, 4, 256, 96, 2, 300)            # head width 32: SIMT attention
     s["ctr_bf16_small"] = synth.ctr_spec(batch=512, table_rows=1000, tower=(256, 128, 64))
     return s
 
