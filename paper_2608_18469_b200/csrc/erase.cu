@@ -8,6 +8,7 @@
 
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <functional>
 #include <map>
@@ -1156,9 +1157,19 @@ erase_status erase_gemm(int32_t dtype, int32_t M, int32_t N, int32_t K, const vo
   cudaError_t e = cudaMemsetAsync(status, 0, sizeof(int), st);
   if (e != cudaSuccess) return cuda_fail(e, "memset");
   g.ws = ws;
+  long long* dbg = nullptr;
   if (engine == 1) {
     TcPlan plan;
     if (!tc_gemm_plan(g, status, &plan)) { cleanup(); g_create_error = "erase_gemm: TMA descriptor encoding failed"; return ERASE_EUNSUPPORTED; }
+    if (getenv("ERASE_TC_TIMELINE")) {   // development aid: print CTA 0's clock stamps for its first tile
+      if (cudaMalloc(&dbg, 16 * sizeof(long long)) == cudaSuccess) {
+        long long h[16] = {0};
+        h[15] = atoll(getenv("ERASE_TC_TIMELINE"));   // bit 0: skip the stores, bit 1: skip the TMEM loads
+        cudaMemcpyAsync(dbg, h, sizeof(h), cudaMemcpyHostToDevice, st);
+        cudaStreamSynchronize(st);
+      }
+      plan.dbg = dbg;
+    }
     e = tc_gemm_launch(g, plan, st);
   } else {
     e = gemm_simt(g, bf, st);
@@ -1172,6 +1183,16 @@ erase_status erase_gemm(int32_t dtype, int32_t M, int32_t N, int32_t K, const vo
   e = cudaMemcpyAsync(&hst, status, sizeof(int), cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) return cuda_fail(e, "execution");
+  if (dbg) {
+    long long h[16];
+    if (cudaMemcpy(h, dbg, sizeof(h), cudaMemcpyDeviceToHost) == cudaSuccess)
+      fprintf(stderr, "tc timeline (cycles from CTA start): setup %lld | first TMA issued %lld | 4th TMA issued %lld | first stage landed %lld | 4th stage landed %lld | "
+              "tile MMAs issued %lld | epilogue starts %lld | epilogue done %lld | CTA end %lld\n",
+              h[1] - h[0], h[2] - h[0], h[8] - h[0], h[3] - h[0], h[9] - h[0], h[4] - h[0], h[5] - h[0], h[6] - h[0], h[7] - h[0]);
+    fprintf(stderr, "   epilogue detail: staged %lld | store issued %lld | loop done %lld | fenced %lld | arrived %lld\n",
+            h[10] - h[0], h[11] - h[0], h[12] - h[0], h[13] - h[0], h[6] - h[0]);
+    cudaFree(dbg);
+  }
   cleanup();
   if (hst != 0) { g_create_error = "erase_gemm: a bounded device-side wait expired (code " + std::to_string(hst) + ")"; return ERASE_ETIMEOUT; }
   return ERASE_OK;

@@ -1,12 +1,16 @@
 // tcgen05 / TMEM / TMA GEMM for sm_100a.  See gemm_tc.cuh for the contract.
 //
-// CTA = one 128 x BN output tile (one split of K when split-K is on), 192 threads:
+// Persistent kernel: one CTA per SM walks over 128 x BN output tiles (one split of K each when
+// split-K is on); 320 threads:
 //   warp 0      TMA producer: one elected thread fills a ring of STAGES shared-memory stages,
 //               each holding a 128 x 64 slab of A and a BN x 64 slab of B (bf16, 128-byte swizzle)
-//   warp 1      allocates TMEM, then one elected thread issues tcgen05.mma (M=128, N=BN, K=16),
-//               four per stage, and commits each stage back to the producer through an mbarrier
-//   warps 2..5  epilogue: wait for the accumulator, read their TMEM lane quarter with
-//               tcgen05.ld, apply the fused epilogue, store to global memory
+//   warp 1      allocates TMEM (two accumulators), then one elected thread issues tcgen05.mma
+//               (M=128, N=BN, K=16), four per stage, commits each stage back to the producer and
+//               each finished accumulator to the epilogue through mbarriers
+//   warps 2..9  epilogue: wait for an accumulator, read their TMEM lane quarter with tcgen05.ld
+//               (two warps per quarter, half of the columns each), apply the fused epilogue,
+//               store to global memory, hand the accumulator back; this overlaps the next
+//               tile's main loop
 // Every mbarrier wait is bounded by a clock limit; on expiry the kernel records a status word,
 // skips the rest of its work, still frees its TMEM and returns.
 #include "gemm_tc.cuh"
@@ -24,6 +28,9 @@ constexpr int BM = 128;
 constexpr int BK = 64;          // bf16 elements = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
 constexpr int STAGES = 4;
+constexpr int EPI_WARPS = 8;                       // two per TMEM lane quarter, each takes half the columns
+constexpr int TC_THREADS = 32 * (2 + EPI_WARPS);
+constexpr uint32_t EPI_STAGE_BYTES = 4096;             // 32 rows x 128 bytes per epilogue warp
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;  // ~2 s at 2 GHz
 
 struct TcArgs {
@@ -35,6 +42,10 @@ struct TcArgs {
   float* ws;
   Epilogue epi;
   int* status;
+  long long* dbg;  // optional: clock64 stamps of CTA 0's first tile (development aid), else null
+  int tma_c;       // C (or the split-K partials) leaves through shared memory + TMA store
+  int tma_p;       // so does the pre-activation copy
+  int plain;       // the epilogue is the identity (no alpha, bias, activation or auxiliary operand)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -114,12 +125,13 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
 
 __device__ __forceinline__ float bf2f(uint32_t bits16) { return __uint_as_float(bits16 << 16); }
 
-__device__ __forceinline__ float act_apply_d(int act, float v) {
+// out of line: keeps the erff/expf expansions out of the unrolled epilogue (instruction-cache footprint)
+__device__ __noinline__ float act_apply_d(int act, float v) {
   if (act == ACT_RELU) return v > 0.f ? v : 0.f;
   if (act == ACT_GELU) return v * 0.5f * (1.f + erff(v * 0.70710678118654752f));
   return v;
 }
-__device__ __forceinline__ float act_deriv_d(int act, float u) {
+__device__ __noinline__ float act_deriv_d(int act, float u) {
   if (act == ACT_RELU) return u > 0.f ? 1.f : 0.f;
   if (act == ACT_GELU) {
     float cdf = 0.5f * (1.f + erff(u * 0.70710678118654752f));
@@ -158,71 +170,190 @@ __device__ __forceinline__ void store8_bf16(__nv_bfloat16* p, int valid, bool ve
   }
 }
 
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+// Fused epilogue on 8 accumulator values of one output row (columns n..n+7), in place.
+// stop_at_pre: return alpha*acc + bias (the pre-activation) and nothing else.
+// The pre-activation copy is written here directly unless it leaves through TMA (p.tma_p).
+struct F8 { float v[8]; };
+
+// The epilogue body runs once per tile in each warp, so its instruction-cache footprint matters
+// more than its instruction count: the activation functions are calls, the column loop is rolled.
+__device__ __forceinline__ F8 epilogue_values8(const TcArgs& p, F8 in, int row, int n, bool stop_at_pre, const float* bias8) {
+  float* v = in.v;
+  const Epilogue& e = p.epi;
+  const int valid = min(8, p.N - n);
+  const long long ia = (long long)row * e.ld_aux + n;
+  const bool avec = valid == 8 && (e.ld_aux % 8 == 0);
+  float t[8];
+  if (e.alpha != 1.f) {
+#pragma unroll
+    for (int j = 0; j < 8; j++) v[j] *= e.alpha;
+  }
+  if (e.bias) {   // this warp's slice of the bias was copied to shared memory while the tile was being multiplied
+    const float4 b0 = *reinterpret_cast<const float4*>(bias8);
+    const float4 b1 = *reinterpret_cast<const float4*>(bias8 + 4);
+    v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w;
+    v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+  }
+  if (stop_at_pre) return in;
+  if (e.pre_out && !p.tma_p) {
+    __nv_bfloat16* po = (__nv_bfloat16*)e.pre_out + ia;
+    store8_bf16(po, valid, avec && ((reinterpret_cast<uintptr_t>(po) & 15) == 0), v);
+  }
+  if (e.act != ACT_NONE) {
+#pragma unroll
+    for (int j = 0; j < 8; j++) v[j] = act_apply_d(e.act, v[j]);
+  }
+  if (e.mul) {
+    const __nv_bfloat16* pm = (const __nv_bfloat16*)e.mul + ia;
+    load8_bf16(pm, valid, avec && ((reinterpret_cast<uintptr_t>(pm) & 15) == 0), t);
+#pragma unroll
+    for (int j = 0; j < 8; j++) v[j] *= t[j];
+  }
+  if (e.res) {
+    const __nv_bfloat16* pr = (const __nv_bfloat16*)e.res + ia;
+    load8_bf16(pr, valid, avec && ((reinterpret_cast<uintptr_t>(pr) & 15) == 0), t);
+#pragma unroll
+    for (int j = 0; j < 8; j++) v[j] += t[j];
+  }
+  if (e.dact != ACT_NONE) {
+    const __nv_bfloat16* pd = (const __nv_bfloat16*)e.dact_src + ia;
+    load8_bf16(pd, valid, avec && ((reinterpret_cast<uintptr_t>(pd) & 15) == 0), t);
+#pragma unroll
+    for (int j = 0; j < 8; j++) v[j] *= act_deriv_d(e.dact, t[j]);
+  }
+  return in;
+}
+
+// Direct global store of 8 finished values (used when the output cannot go through TMA).
+__device__ __forceinline__ void direct_store8(const TcArgs& p, F8 in, int row, int n, int split) {
+  const float* v = in.v;
+  const int valid = min(8, p.N - n);
+  if (p.splits > 1 || p.c_f32) {
+    float* dst = p.splits > 1 ? p.ws + (long long)split * p.M * p.N + (long long)row * p.N + n
+                              : (float*)p.C + (long long)row * p.ldc + n;
+    if (valid == 8 && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
+      reinterpret_cast<float4*>(dst)[0] = make_float4(v[0], v[1], v[2], v[3]);
+      reinterpret_cast<float4*>(dst)[1] = make_float4(v[4], v[5], v[6], v[7]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; j++) if (j < valid) dst[j] = v[j];
+    }
+  } else {
+    __nv_bfloat16* dst = (__nv_bfloat16*)p.C + (long long)row * p.ldc + n;
+    store8_bf16(dst, valid, valid == 8 && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0), v);
+  }
+}
+
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(x), "r"(y), "r"(src) : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
+               ::"l"(map), "r"(x), "r"(y), "r"(z), "r"(src) : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+
+// Persistent kernel: CTA c works on tiles c, c + gridDim.x, ... (m fastest, then n, then split).
 template <int BN, bool A_MN, bool B_MN>
-__global__ void __launch_bounds__(192, 1)
-tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TcArgs p) {
+__global__ void __launch_bounds__(TC_THREADS, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_p,
+               const __grid_constant__ TcArgs p) {
   extern __shared__ uint8_t smem_raw[];
   constexpr uint32_t A_BYTES = BM * BK * 2;
   constexpr uint32_t B_BYTES = BN * BK * 2;
   constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr uint32_t TMEM_COLS = 2 * BN;            // two accumulators: epilogue(i) overlaps mainloop(i+1)
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bar_base = smem_base + STAGES * STAGE_BYTES;  // full[S], empty[S], accum, then tmem slot
+  const uint32_t epi_base = smem_base + STAGES * STAGE_BYTES;          // EPI_WARPS x 4 KB output staging
+  const uint32_t bias_base = epi_base + EPI_WARPS * EPI_STAGE_BYTES;    // EPI_WARPS x 64 floats of bias
+  const uint32_t bar_base = bias_base + EPI_WARPS * 256;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
-  const uint32_t accum_bar = bar_base + 8u * (2 * STAGES);
-  const uint32_t tmem_slot = bar_base + 8u * (2 * STAGES + 1);
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
   uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
-  volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE_BYTES + 8u * (2 * STAGES + 1));
+  volatile uint32_t* tmem_slot_ptr =
+      reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * (EPI_STAGE_BYTES + 256) + 8u * (2 * STAGES + 4));
+  const uint32_t tmem_slot = bar_base + 8u * (2 * STAGES + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN, split = blockIdx.z;
+  const bool dbg = p.dbg != nullptr && blockIdx.x == 0;
+  if (dbg && threadIdx.x == 0) p.dbg[0] = clock64();
+  const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
+  const int total = tiles_m * tiles_n * p.splits;
   const int kchunk = (((p.K + p.splits - 1) / p.splits) + BK - 1) / BK * BK;
-  const int kbeg = split * kchunk;
-  const int kend = min(p.K, kbeg + kchunk);
-  const int num_kb = kend > kbeg ? (kend - kbeg + BK - 1) / BK : 0;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; s++) {
       mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
     }
-    mbar_init(accum_bar, 1);
+    for (int a = 0; a < 2; a++) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), EPI_WARPS);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"((uint32_t)BN) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_ptr;
+  if (dbg && threadIdx.x == 0) p.dbg[1] = clock64();
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
-      for (int kb = 0; kb < num_kb; kb++) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (kb / STAGES) & 1;
-        if (!mbar_wait(empty_bar(s), ph ^ 1)) { atomicExch(p.status, 1); break; }
-        mbar_expect_tx(full_bar(s), STAGE_BYTES);
-        const uint32_t a_dst = smem_base + s * STAGE_BYTES;
-        const uint32_t b_dst = a_dst + A_BYTES;
-        const int k0 = kbeg + kb * BK;
-        if (!A_MN) {
-          tma_load_2d(a_dst, &map_a, k0, m0, full_bar(s));
-        } else {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+      uint32_t it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
+        const int m0 = (t % tiles_m) * BM, n0 = ((t / tiles_m) % tiles_n) * BN, split = t / (tiles_m * tiles_n);
+        const int kbeg = split * kchunk, kend = min(p.K, kbeg + kchunk);
+        const int num_kb = kend > kbeg ? (kend - kbeg + BK - 1) / BK : 0;
+        for (int kb = 0; kb < num_kb; kb++, it++) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!mbar_wait(empty_bar(s), ph ^ 1)) { atomicExch(p.status, 1); ok = false; break; }
+          mbar_expect_tx(full_bar(s), STAGE_BYTES);
+          const uint32_t a_dst = smem_base + s * STAGE_BYTES;
+          const uint32_t b_dst = a_dst + A_BYTES;
+          const int k0 = kbeg + kb * BK;
+          if (!A_MN) {
+            tma_load_2d(a_dst, &map_a, k0, m0, full_bar(s));
+          } else {
 #pragma unroll
-          for (int a = 0; a < BM / 64; a++) tma_load_2d(a_dst + a * (BK * 128), &map_a, m0 + a * 64, k0, full_bar(s));
-        }
-        if (!B_MN) {
-          tma_load_2d(b_dst, &map_b, k0, n0, full_bar(s));
-        } else {
+            for (int a = 0; a < BM / 64; a++) tma_load_2d(a_dst + a * (BK * 128), &map_a, m0 + a * 64, k0, full_bar(s));
+          }
+          if (!B_MN) {
+            tma_load_2d(b_dst, &map_b, k0, n0, full_bar(s));
+          } else {
 #pragma unroll
-          for (int a = 0; a < BN / 64; a++) tma_load_2d(b_dst + a * (BK * 128), &map_b, n0 + a * 64, k0, full_bar(s));
+            for (int a = 0; a < BN / 64; a++) tma_load_2d(b_dst + a * (BK * 128), &map_b, n0 + a * 64, k0, full_bar(s));
+          }
+          if (dbg && it == 0) p.dbg[2] = clock64();
+          if (dbg && it == 3) p.dbg[8] = clock64();
         }
+      }
+      if (!ok) {  // give copies already in flight time to land before the CTA's shared memory is released
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) {}
       }
     }
   } else if (warp == 1) {
@@ -231,132 +362,160 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       // instruction descriptor: fp32 accumulate, bf16 x bf16, majors, N>>3 at bit 17, M>>4 at bit 24
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16) |
                              ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      uint32_t it = 0, lt = 0;
       bool ok = true;
-      for (int kb = 0; kb < num_kb && ok; kb++) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (kb / STAGES) & 1;
-        if (!mbar_wait(full_bar(s), ph)) { atomicExch(p.status, 2); ok = false; break; }
+      for (int t = blockIdx.x; t < total && ok; t += gridDim.x, lt++) {
+        const int split = t / (tiles_m * tiles_n);
+        const int kbeg = split * kchunk, kend = min(p.K, kbeg + kchunk);
+        const int num_kb = kend > kbeg ? (kend - kbeg + BK - 1) / BK : 0;
+        const uint32_t ab = lt & 1, aph = (lt >> 1) & 1;
+        if (!mbar_wait(tempty_bar(ab), aph ^ 1)) { atomicExch(p.status, 4); ok = false; break; }
         tc_fence_after();
-        const uint32_t a_src = smem_base + s * STAGE_BYTES;
-        const uint32_t b_src = a_src + A_BYTES;
+        const uint32_t tmem_d = tmem_base + ab * BN;
+        for (int kb = 0; kb < num_kb; kb++, it++) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!mbar_wait(full_bar(s), ph)) { atomicExch(p.status, 2); ok = false; break; }
+          tc_fence_after();
+          if (dbg && it == 0) p.dbg[3] = clock64();
+          if (dbg && it == 3) p.dbg[9] = clock64();
+          const uint32_t a_src = smem_base + s * STAGE_BYTES;
+          const uint32_t b_src = a_src + A_BYTES;
 #pragma unroll
-        for (int k = 0; k < BK / UMMA_K; k++) {
-          // K-major: rows of 128 bytes, 8-row groups 1024 bytes apart; a K step of 16 elements is
-          //          32 bytes inside the swizzled row.
-          // MN-major: 64-element (128-byte) runs along M/N, one per K index; 8 K rows form a
-          //          1024-byte group (stride offset), the next 64 M/N elements sit BK*128 bytes
-          //          further (leading offset); a K step of 16 is 16 rows = 2048 bytes.
-          const uint64_t ad = A_MN ? smem_desc(a_src + k * (UMMA_K * 128), BK * 128, 1024)
-                                   : smem_desc(a_src + k * (UMMA_K * 2), 16, 1024);
-          const uint64_t bd = B_MN ? smem_desc(b_src + k * (UMMA_K * 128), BK * 128, 1024)
-                                   : smem_desc(b_src + k * (UMMA_K * 2), 16, 1024);
-          tc_mma(tmem_base, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < BK / UMMA_K; k++) {
+            // K-major: rows of 128 bytes, 8-row groups 1024 bytes apart; a K step of 16 elements is
+            //          32 bytes inside the swizzled row.
+            // MN-major: 64-element (128-byte) runs along M/N, one per K index; 8 K rows form a
+            //          1024-byte group (stride offset), the next 64 M/N elements sit BK*128 bytes
+            //          further (leading offset); a K step of 16 is 16 rows = 2048 bytes.
+            const uint64_t ad = A_MN ? smem_desc(a_src + k * (UMMA_K * 128), BK * 128, 1024)
+                                     : smem_desc(a_src + k * (UMMA_K * 2), 16, 1024);
+            const uint64_t bd = B_MN ? smem_desc(b_src + k * (UMMA_K * 128), BK * 128, 1024)
+                                     : smem_desc(b_src + k * (UMMA_K * 2), 16, 1024);
+            tc_mma(tmem_d, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          }
+          tc_commit(empty_bar(s));  // stage may be refilled once these MMAs have read it
         }
-        tc_commit(empty_bar(s));  // stage may be refilled once these MMAs have read it
+        tc_commit(tfull_bar(ab));   // accumulator ab complete (also fires when the loop bailed out)
+        if (dbg && lt == 0) p.dbg[4] = clock64();
       }
-      tc_commit(accum_bar);       // accumulator complete (also fires when the loop bailed out)
     }
   } else {
     // ------------------------------ epilogue ------------------------------
-    const int q = warp & 3;  // TMEM lane quarter this warp may read
-    const int row = m0 + q * 32 + lane;
-    bool ok = mbar_wait(accum_bar, 0);
-    if (!ok) atomicExch(p.status, 3);
-    ok = __all_sync(0xffffffffu, ok);
-    tc_fence_after();
-    if (ok) {
-      const Epilogue& e = p.epi;
-      const bool row_ok = row < p.M;
-      const bool plain_store = p.splits > 1;
-      for (int c0 = 0; c0 < BN; c0 += 32) {
-        if (n0 + c0 >= p.N) break;  // warp-uniform
-        uint32_t r[32];
-        if (num_kb > 0) {
-          tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
-        } else {  // an empty K range (a trailing split): the partial sum is zero
-#pragma unroll
-          for (int j = 0; j < 32; j++) r[j] = 0u;
+    // A warp owns 32 rows (its TMEM lane quarter) x 64 columns of the tile, as two 32-column
+    // chunks.  Finished values go to a 4 KB staging buffer in shared memory (one 128-byte row
+    // per lane, 16-byte pieces XOR-swizzled with the row so that writes are conflict-free and
+    // match the tensor map's 128-byte swizzle) and leave with one TMA store per 128-byte-wide
+    // box, which also clips the M and N tails.  Outputs that cannot be described to TMA
+    // (unaligned leading dimension) are stored directly.
+    const int ew = warp - 2;
+    const int q = warp & 3;                       // TMEM lane quarter this warp may read
+    const int cbeg = (ew / 4) * 64;               // first tile column of this warp
+    const bool active = cbeg < BN;                // BN = 64: only one warp per quarter has columns
+    const uint32_t stage = epi_base + ew * EPI_STAGE_BYTES;
+    const uint32_t my_row = stage + lane * 128;
+    float* bias_s = reinterpret_cast<float*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * EPI_STAGE_BYTES + ew * 256);
+    const bool out_f32 = p.splits > 1 || p.c_f32;
+    bool store_pending = false;                   // lane 0: a TMA store may still be reading the staging buffer
+    uint32_t lt = 0;
+    for (int t = blockIdx.x; t < total; t += gridDim.x, lt++) {
+      const int m0 = (t % tiles_m) * BM, n0 = ((t / tiles_m) % tiles_n) * BN, split = t / (tiles_m * tiles_n);
+      const int kbeg = split * kchunk, kend = min(p.K, kbeg + kchunk);
+      const bool empty_k = kend <= kbeg;          // a trailing split with no K range: partial sum is zero
+      const uint32_t ab = lt & 1, aph = (lt >> 1) & 1;
+      if (p.epi.bias && active) {   // fetch this warp's 64 bias values now; the latency hides behind the MMAs
+        __syncwarp();
+        for (int j = lane; j < 64; j += 32) {
+          const int n = n0 + cbeg + j;
+          bias_s[j] = n < p.N ? __ldg(p.epi.bias + n) : 0.f;
         }
-        if (!row_ok) continue;
-#pragma unroll
-        for (int g8 = 0; g8 < 4; g8++) {
-          const int n = n0 + c0 + g8 * 8;
-          const int valid = min(8, p.N - n);
-          if (valid <= 0) break;
-          float v[8];
-#pragma unroll
-          for (int j = 0; j < 8; j++) v[j] = __uint_as_float(r[g8 * 8 + j]);
-          if (plain_store) {
-            float* dst = p.ws + (long long)split * p.M * p.N + (long long)row * p.N + n;
-            const bool vec = valid == 8 && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0);
-            if (vec) {
-              reinterpret_cast<float4*>(dst)[0] = make_float4(v[0], v[1], v[2], v[3]);
-              reinterpret_cast<float4*>(dst)[1] = make_float4(v[4], v[5], v[6], v[7]);
+        __syncwarp();
+      }
+      bool ok = mbar_wait(tfull_bar(ab), aph);
+      if (!ok) atomicExch(p.status, 3);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      if (dbg && lt == 0 && threadIdx.x == 64) p.dbg[5] = clock64();
+      const int row = m0 + q * 32 + lane;
+      const bool row_ok = row < p.M;
+      const long long dflags = p.dbg ? p.dbg[15] : 0;
+      const int npass = (p.epi.pre_out && p.tma_p) ? 2 : 1;   // pass 0 of 2 writes the pre-activation copy
+      if (active && n0 + cbeg < p.N) {
+        for (int pass = 0; pass < npass; pass++) {
+          const bool pre_pass = npass == 2 && pass == 0;
+          const bool via_tma = pre_pass ? true : (p.tma_c != 0);
+          const bool f32 = !pre_pass && out_f32;
+#pragma unroll 1
+          for (int cc = 0; cc < 64; cc += 32) {
+            const int c0 = cbeg + cc;
+            if (n0 + c0 >= p.N) break;  // warp-uniform
+            uint32_t r[32];
+            if (!empty_k && !(dflags & 2)) {
+              tc_ld32(tmem_base + ab * BN + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
             } else {
-              for (int j = 0; j < valid; j++) dst[j] = v[j];
+#pragma unroll
+              for (int j = 0; j < 32; j++) r[j] = 0u;
             }
-            continue;
-          }
-          const long long ia = (long long)row * e.ld_aux + n;
-          const bool avec = valid == 8 && (e.ld_aux % 8 == 0);
-          float t[8];
-#pragma unroll
-          for (int j = 0; j < 8; j++) v[j] *= e.alpha;
-          if (e.bias) {
-#pragma unroll
-            for (int j = 0; j < 8; j++) if (j < valid) v[j] += __ldg(e.bias + n + j);
-          }
-          if (e.pre_out) {
-            __nv_bfloat16* po = (__nv_bfloat16*)e.pre_out + ia;
-            store8_bf16(po, valid, avec && ((reinterpret_cast<uintptr_t>(po) & 15) == 0), v);
-          }
-          if (e.act != ACT_NONE) {
-#pragma unroll
-            for (int j = 0; j < 8; j++) v[j] = act_apply_d(e.act, v[j]);
-          }
-          if (e.mul) {
-            const __nv_bfloat16* pm = (const __nv_bfloat16*)e.mul + ia;
-            load8_bf16(pm, valid, avec && ((reinterpret_cast<uintptr_t>(pm) & 15) == 0), t);
-#pragma unroll
-            for (int j = 0; j < 8; j++) v[j] *= t[j];
-          }
-          if (e.res) {
-            const __nv_bfloat16* pr = (const __nv_bfloat16*)e.res + ia;
-            load8_bf16(pr, valid, avec && ((reinterpret_cast<uintptr_t>(pr) & 15) == 0), t);
-#pragma unroll
-            for (int j = 0; j < 8; j++) v[j] += t[j];
-          }
-          if (e.dact != ACT_NONE) {
-            const __nv_bfloat16* pd = (const __nv_bfloat16*)e.dact_src + ia;
-            load8_bf16(pd, valid, avec && ((reinterpret_cast<uintptr_t>(pd) & 15) == 0), t);
-#pragma unroll
-            for (int j = 0; j < 8; j++) v[j] *= act_deriv_d(e.dact, t[j]);
-          }
-          const long long ic = (long long)row * p.ldc + n;
-          if (p.c_f32) {
-            float* dst = (float*)p.C + ic;
-            const bool vec = valid == 8 && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0);
-            if (vec) {
-              reinterpret_cast<float4*>(dst)[0] = make_float4(v[0], v[1], v[2], v[3]);
-              reinterpret_cast<float4*>(dst)[1] = make_float4(v[4], v[5], v[6], v[7]);
-            } else {
-              for (int j = 0; j < valid; j++) dst[j] = v[j];
+            if (via_tma && (f32 || cc == 0)) {       // the staging buffer is about to be overwritten
+              if (lane == 0 && store_pending) { tma_store_wait_read(); store_pending = false; }
+              __syncwarp();
             }
-          } else {
-            __nv_bfloat16* dst = (__nv_bfloat16*)p.C + ic;
-            store8_bf16(dst, valid, valid == 8 && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0), v);
+#pragma unroll
+            for (int g8 = 0; g8 < 4; g8++) {
+              const int n = n0 + c0 + g8 * 8;
+              F8 f;
+#pragma unroll
+              for (int j = 0; j < 8; j++) f.v[j] = __uint_as_float(r[g8 * 8 + j]);
+              if (row_ok && n < p.N && p.splits == 1 && !p.plain) f = epilogue_values8(p, f, row, n, pre_pass, bias_s + cc + g8 * 8);
+              const float* v = f.v;
+              if (!via_tma) {
+                if (row_ok && n < p.N && !(dflags & 1)) direct_store8(p, f, row, n, split);
+              } else if (f32) {                      // 32 floats per row: pieces 2*g8 and 2*g8+1 of the 128-byte row
+                const uint32_t s0 = my_row + (((2 * g8) ^ (lane & 7)) << 4), s1 = my_row + (((2 * g8 + 1) ^ (lane & 7)) << 4);
+                st_shared_v4(s0, __float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]));
+                st_shared_v4(s1, __float_as_uint(v[4]), __float_as_uint(v[5]), __float_as_uint(v[6]), __float_as_uint(v[7]));
+              } else {                               // 64 bf16 per row: piece cc/8 + g8
+                const uint32_t s0 = my_row + ((((cc >> 3) + g8) ^ (lane & 7)) << 4);
+                st_shared_v4(s0, pack2(v[0], v[1]), pack2(v[2], v[3]), pack2(v[4], v[5]), pack2(v[6], v[7]));
+              }
+            }
+            const bool last_chunk = cc == 32 || n0 + c0 + 32 >= p.N;
+            if (via_tma && (f32 || last_chunk)) {
+              asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+              __syncwarp();
+              if (dbg && lt == 0 && threadIdx.x == 64 && p.dbg[10] == 0) p.dbg[10] = clock64();
+              if (lane == 0 && !(dflags & 1)) {
+                const int x = f32 ? n0 + c0 : n0 + cbeg, y = m0 + q * 32;
+                if (pre_pass) tma_store_2d(&map_p, stage, x, y);
+                else if (p.splits > 1) tma_store_3d(&map_c, stage, x, y, split);
+                else tma_store_2d(&map_c, stage, x, y);
+                tma_store_commit();
+                store_pending = true;
+                if (dbg && lt == 0 && threadIdx.x == 64 && p.dbg[11] == 0) p.dbg[11] = clock64();
+              }
+            }
           }
         }
       }
+      // all TMEM reads of this warp are complete (tcgen05.wait::ld): hand the accumulator back
+      if (dbg && lt == 0 && threadIdx.x == 64) p.dbg[12] = clock64();
+      tc_fence_before();
+      __syncwarp();
+      if (dbg && lt == 0 && threadIdx.x == 64) p.dbg[13] = clock64();
+      if (lane == 0) mbar_arrive(tempty_bar(ab));
+      if (dbg && lt == 0 && threadIdx.x == 64) p.dbg[6] = clock64();
     }
+    if (lane == 0 && store_pending) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // stores complete before exit
   }
 
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)BN) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
+  if (dbg && threadIdx.x == 0) p.dbg[7] = clock64();
 }
 
 typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -379,26 +538,36 @@ EncodeFn encode_fn() {
   return fn;
 }
 
-// 2-D bf16 tensor map: `inner` contiguous elements per row, `outer` rows `ld` elements apart;
-// box = 64 x box_outer, 128-byte swizzle, out-of-bounds elements read as zero.
-bool encode_2d(void* out, const void* base, long long inner, long long outer, long long ld, int box_outer) {
+// Tensor map of a row-major bf16 or fp32 matrix (rank 2) or stack of matrices (rank 3):
+// dims[0] contiguous elements per row, rows stride_bytes[0] apart, 128-byte swizzle; the box's
+// inner extent is 128 bytes.  Out-of-bounds elements read as zero and are not written.
+bool encode_map(void* out, const void* base, bool f32, int rank, const cuuint64_t* dims, const cuuint64_t* stride_bytes,
+                const cuuint32_t* box) {
   EncodeFn fn = encode_fn();
   if (!fn) return false;
+  for (int i = 0; i + 1 < rank; i++)
+    if (stride_bytes[i] % 16) return false;
+  if (reinterpret_cast<uintptr_t>(base) & 15) return false;
   CUtensorMap tmp;
-  cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
-  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-  cuuint32_t box[2] = {64u, (cuuint32_t)box_outer};
-  cuuint32_t estr[2] = {1u, 1u};
-  CUresult r = fn(&tmp, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  cuuint32_t estr[3] = {1u, 1u, 1u};
+  CUresult r = fn(&tmp, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank,
+                  const_cast<void*>(base), dims, stride_bytes, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r == CUDA_SUCCESS) memcpy(out, &tmp, sizeof(tmp));
   return r == CUDA_SUCCESS;
 }
 
+// operand map: `inner` contiguous bf16 elements per row, `outer` rows `ld` elements apart; box 64 x box_outer
+bool encode_2d(void* out, const void* base, long long inner, long long outer, long long ld, int box_outer) {
+  cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {64u, (cuuint32_t)box_outer};
+  return encode_map(out, base, false, 2, dims, strides, box);
+}
+
 template <int BN, bool A_MN, bool B_MN>
 cudaError_t launch_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s) {
-  constexpr size_t smem = (size_t)STAGES * (BM * BK * 2 + BN * BK * 2) + 8 * (2 * STAGES + 2) + 1024;
+  constexpr size_t smem = (size_t)STAGES * (BM * BK * 2 + BN * BK * 2) + EPI_WARPS * (EPI_STAGE_BYTES + 256) + 8 * (2 * STAGES + 6) + 1024;
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<BN, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -408,13 +577,26 @@ cudaError_t launch_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s) {
   TcArgs p;
   p.M = g.M; p.N = g.N; p.K = g.K;
   p.C = g.C; p.ldc = g.ldc; p.c_f32 = g.c_f32;
-  p.splits = g.splits; p.ws = g.ws; p.epi = g.epi; p.status = plan.status;
-  dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, g.splits);
-  CUtensorMap ma, mb;
+  p.splits = g.splits; p.ws = g.ws; p.epi = g.epi; p.status = plan.status; p.dbg = plan.dbg;
+  static int num_sms = 0;
+  if (num_sms == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms < 1) num_sms = 148;
+  }
+  const long long total = (long long)((g.N + BN - 1) / BN) * ((g.M + BM - 1) / BM) * g.splits;
+  dim3 grid((unsigned)(total < num_sms ? total : num_sms));
+  CUtensorMap ma, mb, mc, mp;
   static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
   memcpy(&ma, plan.map_a, sizeof(ma));
   memcpy(&mb, plan.map_b, sizeof(mb));
-  tc_gemm_kernel<BN, A_MN, B_MN><<<grid, 192, smem, s>>>(ma, mb, p);
+  memcpy(&mc, plan.map_c, sizeof(mc));
+  memcpy(&mp, plan.map_p, sizeof(mp));
+  p.tma_c = plan.tma_c;
+  p.tma_p = plan.tma_p;
+  const Epilogue& e = g.epi;
+  p.plain = (e.alpha == 1.f && !e.bias && e.act == ACT_NONE && !e.pre_out && !e.mul && !e.res && e.dact == ACT_NONE) ? 1 : 0;
+  tc_gemm_kernel<BN, A_MN, B_MN><<<grid, TC_THREADS, smem, s>>>(ma, mb, mc, mp, p);
   return cudaGetLastError();
 }
 
@@ -455,7 +637,34 @@ bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan) {
   if (!ok) return false;
   if (!plan->b_mn) ok = encode_2d(plan->map_b, g.B, g.K, g.N, g.sb_n, plan->bn);
   else ok = encode_2d(plan->map_b, g.B, g.N, g.K, g.sb_k, BK);
-  return ok;
+  if (!ok) return false;
+  // outputs through TMA stores where their layout allows it (else the kernel stores directly)
+  memset(plan->map_c, 0, sizeof(plan->map_c));
+  memset(plan->map_p, 0, sizeof(plan->map_p));
+  plan->tma_c = plan->tma_p = 0;
+  if (g.splits > 1) {
+    cuuint64_t dims[3] = {(cuuint64_t)g.N, (cuuint64_t)g.M, (cuuint64_t)g.splits};
+    cuuint64_t str[2] = {(cuuint64_t)g.N * 4, (cuuint64_t)g.M * g.N * 4};
+    cuuint32_t box[3] = {32u, 32u, 1u};
+    plan->tma_c = g.ws && encode_map(plan->map_c, g.ws, true, 3, dims, str, box) ? 1 : 0;
+  } else if (g.c_f32) {
+    cuuint64_t dims[2] = {(cuuint64_t)g.N, (cuuint64_t)g.M};
+    cuuint64_t str[1] = {(cuuint64_t)g.ldc * 4};
+    cuuint32_t box[2] = {32u, 32u};
+    plan->tma_c = encode_map(plan->map_c, g.C, true, 2, dims, str, box) ? 1 : 0;
+  } else {
+    cuuint64_t dims[2] = {(cuuint64_t)g.N, (cuuint64_t)g.M};
+    cuuint64_t str[1] = {(cuuint64_t)g.ldc * 2};
+    cuuint32_t box[2] = {64u, 32u};
+    plan->tma_c = encode_map(plan->map_c, g.C, false, 2, dims, str, box) ? 1 : 0;
+  }
+  if (g.splits == 1 && g.epi.pre_out) {
+    cuuint64_t dims[2] = {(cuuint64_t)g.N, (cuuint64_t)g.M};
+    cuuint64_t str[1] = {(cuuint64_t)g.epi.ld_aux * 2};
+    cuuint32_t box[2] = {64u, 32u};
+    plan->tma_p = encode_map(plan->map_p, g.epi.pre_out, false, 2, dims, str, box) ? 1 : 0;
+  }
+  return true;
 }
 
 cudaError_t tc_gemm_launch(const GemmArgs& g, const TcPlan& plan, cudaStream_t s) {

@@ -14,11 +14,15 @@ namespace erase {
 struct TcPlan {
   unsigned char map_a[128];  // CUtensorMap of A (copied into an aligned object at launch)
   unsigned char map_b[128];  // CUtensorMap of B
+  unsigned char map_c[128];  // CUtensorMap of the output (or of the split-K partials), if tma_c
+  unsigned char map_p[128];  // CUtensorMap of the pre-activation copy, if tma_p
+  int tma_c = 0, tma_p = 0;
   int bn = 128;       // tile width (N)
   int a_mn = 0;       // A is contiguous along M (not along K)
   int b_mn = 0;
   int launches = 1;
   int* status = nullptr;  // device word set non-zero when a bounded wait expired
+  long long* dbg = nullptr;  // optional device buffer (16 slots) for clock64 stamps of CTA 0, development aid
 };
 
 // True if the tensor-core kernel can take this GEMM: bf16 operands, 16-byte aligned bases,
