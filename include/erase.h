@@ -127,6 +127,13 @@ typedef struct {
 #define ERASE_GRAPH 1u   /* replay the whole step (either schedule) as one CUDA graph, captured on
                             first use per (batch pointers, n_streams, flags); Section 1.1/2.2      */
 #define ERASE_NO_OPT 2u  /* stop after the backward passes: gradients only, parameters untouched   */
+#define ERASE_EARLY_HEAD 4u /* ERASE schedules only: release the side stream right after the block
+                            BODY's forward and run the local head, its loss and the backward there.
+                            The next block's forward needs z_b but not l_b, so the head leaves the
+                            main stream's critical path (Section 2.1: the gradient is ready once
+                            forward and local loss are done -- nothing else waits for the loss).
+                            Same kernels, same bits.  Without the flag the head and loss run on the
+                            main stream before the release, as the paper schedules them.          */
 
 /* Device bytes erase_create needs for this spec when given an arena; 0 if the spec is invalid. */
 ERASE_API size_t erase_arena_bytes(const erase_model_spec* spec);

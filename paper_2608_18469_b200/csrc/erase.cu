@@ -93,10 +93,11 @@ struct erase_model {
   bool timeline_valid = false;
 
   OpList stage, opt;
-  std::vector<OpList> fwd, bwd;
+  std::vector<OpList> fwd, hfwd, bwd;  // per block: body forward, local head + loss, backward
   erase_batch cur = {nullptr, nullptr, nullptr};
   std::map<GraphKey, cudaGraphExec_t> graphs;
 
+  int sm_budget = 0;   // CTA cap for persistent GEMMs enqueued next (0 = all SMs); set per stream by the scheduler
   int64_t launches = 0;
   bool stepped = false;
   std::string err;
@@ -299,6 +300,7 @@ struct Builder {
 
   void* act_buf(size_t elems) { return dev_alloc(m, elems * m->esz, &ok); }
   float* f32_buf(size_t elems) { return (float*)dev_alloc(m, elems * sizeof(float), &ok); }
+  int* tickets(int cols) { return (int*)dev_alloc(m, (size_t)((cols + 63) / 64) * sizeof(int), &ok); }  // zero-initialised
 
   const Tensor& T(int idx) const { return m->tensors[idx]; }
   const void* Wop(int idx) const {  // GEMM operand copy of a weight matrix
@@ -331,13 +333,13 @@ struct Builder {
     const bool use_tc = tc_ok && !m->dry && tc_gemm_plan(g, m->status, &plan);
     if (use_tc) {
       if (g.splits > 1)
-        ops.push_back({[g, plan, out, ldo](cudaStream_t s) {
-                         cudaError_t e = tc_gemm_launch(g, plan, s);
+        ops.push_back({[g, plan, out, ldo, mm = m](cudaStream_t s) {
+                         cudaError_t e = tc_gemm_launch(g, plan, s, mm->sm_budget);
                          if (e != cudaSuccess) return e;
                          return splitk_reduce(g.ws, g.splits, (long long)g.M * g.N, g.N, out, ldo, s);
                        }, 2});
       else
-        ops.push_back({[g, plan](cudaStream_t s) { return tc_gemm_launch(g, plan, s); }, 1});
+        ops.push_back({[g, plan, mm = m](cudaStream_t s) { return tc_gemm_launch(g, plan, s, mm->sm_budget); }, 1});
       return;
     }
     if (g.splits > 1) {
@@ -399,7 +401,8 @@ struct Builder {
     float* ws = chunks > 1 ? f32_buf((size_t)chunks * N) : nullptr;
     float* out = G(bidx);
     bool bf = m->bf16;
-    ops.push_back({[=](cudaStream_t s) { return colsum(dY, bf, ld, M, N, nullptr, ws, chunks, out, s); }, chunks > 1 ? 2 : 1});
+    int* tk = tickets(N);
+    ops.push_back({[=](cudaStream_t s) { return colsum(dY, bf, ld, M, N, nullptr, ws, chunks, tk, out, s); }, 1});
     note(ops, "colsum", (double)M * N, (double)M * N * m->esz);
   }
 
@@ -409,9 +412,10 @@ struct Builder {
   // db[c] = w[c] * sum_r ds[r] * act'(src[r,c]), from the fp32 loss gradient rather than from the
   // bf16-rounded dz (the sum over r cancels heavily when the labels are balanced).  Returns true
   // if it did, so that the caller skips the ordinary column sum for that bias.
-  bool head(int b, const erase_block_spec& k, const void* z, int d, int wh, int bh, OpList& f, OpList& bw, void* dz,
+  bool head(int b, const erase_block_spec& k, const void* z, int d, int wh, int bh, OpList& /*body forward*/, OpList& bw, void* dz,
             int dact, const void* dact_src, int last_bias = -1) {
     erase_model* mm = m;
+    OpList& f = m->hfwd[b];   // the head and its loss form their own list: only the backward consumes them
     bool bf = m->bf16;
     int rows = m->rows;
     float* rowloss = f32_buf(rows);
@@ -431,14 +435,16 @@ struct Builder {
         int chunks = colsum_chunks(rows, d);
         float* ws = chunks > 1 ? f32_buf((size_t)chunks * d) : nullptr;
         float* out = G(wh);
-        bw.push_back({[=](cudaStream_t s) { return colsum(z, bf, d, rows, d, ds, ws, chunks, out, s); }, chunks > 1 ? 2 : 1});
+        int* tk = tickets(d);
+        bw.push_back({[=](cudaStream_t s) { return colsum(z, bf, d, rows, d, ds, ws, chunks, tk, out, s); }, 1});
         note(bw, "colsum", 2.0 * rows * d, (double)rows * d * m->esz);
       }
       {
         int chunks = colsum_chunks(rows, 1);
         float* ws = chunks > 1 ? f32_buf((size_t)chunks) : nullptr;
         float* out = G(bh);
-        bw.push_back({[=](cudaStream_t s) { return colsum(ds, false, 1, rows, 1, nullptr, ws, chunks, out, s); }, chunks > 1 ? 2 : 1});
+        int* tk = tickets(1);
+        bw.push_back({[=](cudaStream_t s) { return colsum(ds, false, 1, rows, 1, nullptr, ws, chunks, tk, out, s); }, 1});
         note(bw, "colsum", rows, 4.0 * rows);
       }
       if (last_bias >= 0) {
@@ -446,7 +452,8 @@ struct Builder {
         float* ws = chunks > 1 ? f32_buf((size_t)chunks * d) : nullptr;
         float* out = G(last_bias);
         const void* src = dact != ACT_NONE ? dact_src : nullptr;
-        bw.push_back({[=](cudaStream_t s) { return colsum(src, bf, d, rows, d, ds, ws, chunks, out, s, dact, w); }, chunks > 1 ? 2 : 1});
+        int* tk = tickets(d);
+        bw.push_back({[=](cudaStream_t s) { return colsum(src, bf, d, rows, d, ds, ws, chunks, tk, out, s, dact, w); }, 1});
         note(bw, "colsum", 2.0 * rows * d, src ? (double)rows * d * m->esz : 4.0 * rows);
         return true;
       }
@@ -617,7 +624,8 @@ struct Builder {
     int chunks = colsum_chunks(rows, d);
     float* ws = chunks > 1 ? f32_buf((size_t)2 * chunks * d) : nullptr;
     float* dg = G(gidx); float* db = G(bidx);
-    bw.push_back({[=](cudaStream_t s) { return layernorm_param_grad(dy, x, mean, rstd, ws, chunks, dg, db, rows, d, bf, s); }, chunks > 1 ? 3 : 1});
+    int* tk = tickets(d);
+    bw.push_back({[=](cudaStream_t s) { return layernorm_param_grad(dy, x, mean, rstd, ws, chunks, tk, dg, db, rows, d, bf, s); }, 1});
     note(bw, "layernorm_param_grad", 4.0 * rows * d, 2.0 * rows * d * m->esz);
   }
 
@@ -722,6 +730,7 @@ struct Builder {
     int first = 0;
     while (first < (int)m->tensors.size() && m->tensors[first].block < 0) first++;
     m->fwd.resize(m->B);
+    m->hfwd.resize(m->B);
     m->bwd.resize(m->B);
     const void* z = z0;
     for (int b = 0; b < m->B; b++) {
@@ -794,10 +803,12 @@ erase_status enqueue_step(erase_model* m, int n_streams, unsigned flags, bool ti
   auto tev = [&](int i) { return m->ev_time[i]; };
   if (timed) CK(cudaEventRecord(tev(2 * (2 * B + 1)), m->main));
   CK(run_ops(m, m->stage, m->main));
+  const bool early_head = (flags & ERASE_EARLY_HEAD) != 0;
   if (n_streams <= 1) {
     for (int b = 0; b < B; b++) {
       if (timed) CK(cudaEventRecord(tev(2 * b), m->main));
       CK(run_ops(m, m->fwd[b], m->main));
+      CK(run_ops(m, m->hfwd[b], m->main));
       if (timed) CK(cudaEventRecord(tev(2 * b + 1), m->main));
     }
     for (int b = B - 1; b >= 0; b--) {
@@ -807,19 +818,29 @@ erase_status enqueue_step(erase_model* m, int n_streams, unsigned flags, bool ti
     }
   } else {
     const int ns = n_streams - 1;
+    // SM budget: persistent GEMMs of the main stream and of the side streams each leave SMs free
+    // for the other, so that B_b really runs beside F_{b+1} instead of queueing behind it.
+    static const int env_main = getenv("ERASE_SM_MAIN") ? atoi(getenv("ERASE_SM_MAIN")) : 0;
+    static const int env_side = getenv("ERASE_SM_SIDE") ? atoi(getenv("ERASE_SM_SIDE")) : 0;
+    const int budget_main = env_main, budget_side = env_side;
     for (int b = 0; b < B; b++) {
+      m->sm_budget = budget_main;
       if (timed) CK(cudaEventRecord(tev(2 * b), m->main));
       CK(run_ops(m, m->fwd[b], m->main));
+      if (!early_head) CK(run_ops(m, m->hfwd[b], m->main));
       if (timed) CK(cudaEventRecord(tev(2 * b + 1), m->main));
-      CK(cudaEventRecord(m->ev_f[b], m->main));          // F_b and l_b are enqueued: release B_b
+      CK(cudaEventRecord(m->ev_f[b], m->main));          // F_b (and l_b) are enqueued: release B_b
       cudaStream_t sd = m->side[b % ns];
       CK(cudaStreamWaitEvent(sd, m->ev_f[b], 0));
       if (timed) CK(cudaEventRecord(tev(2 * (B + b)), sd));
+      m->sm_budget = budget_side;
+      if (early_head) CK(run_ops(m, m->hfwd[b], sd));    // z_b's only other consumer is F_{b+1}, which does not wait
       CK(run_ops(m, m->bwd[b], sd));
       if (timed) CK(cudaEventRecord(tev(2 * (B + b) + 1), sd));
       CK(cudaEventRecord(m->ev_b[b], sd));
     }
     for (int b = 0; b < B; b++) CK(cudaStreamWaitEvent(m->main, m->ev_b[b], 0));  // join
+    m->sm_budget = 0;
   }
   if (timed) CK(cudaEventRecord(tev(4 * B), m->main));
   if (do_opt) CK(run_ops(m, m->opt, m->main));
@@ -996,7 +1017,7 @@ static erase_status check_step_args(erase_model* m, const erase_batch* batch);
 erase_status erase_step_ex(erase_model* m, const erase_batch* batch, int32_t n_streams, uint32_t flags) {
   if (!m) return ERASE_EINVAL;
   if (n_streams < 1) return m->fail(ERASE_EINVAL, "erase_step: n_streams must be >= 1");
-  if (flags & ~(ERASE_GRAPH | ERASE_NO_OPT)) return m->fail(ERASE_EINVAL, "erase_step: unknown flag");
+  if (flags & ~(ERASE_GRAPH | ERASE_NO_OPT | ERASE_EARLY_HEAD)) return m->fail(ERASE_EINVAL, "erase_step: unknown flag");
   erase_status cst = check_step_args(m, batch);
   if (cst != ERASE_OK) return cst;
   if (n_streams > m->B + 1) n_streams = m->B + 1;
@@ -1024,6 +1045,7 @@ erase_status erase_step_ex(erase_model* m, const erase_batch* batch, int32_t n_s
     for (auto& op : m->stage) per += op.launches;
     for (int b = 0; b < m->B; b++) {
       for (auto& op : m->fwd[b]) per += op.launches;
+      for (auto& op : m->hfwd[b]) per += op.launches;
       for (auto& op : m->bwd[b]) per += op.launches;
     }
     if (!(flags & ERASE_NO_OPT)) for (auto& op : m->opt) per += op.launches;
@@ -1058,7 +1080,10 @@ erase_status erase_profile_step(erase_model* m, const erase_batch* batch, erase_
   struct Ref { Op* op; int block, phase; };
   std::vector<Ref> refs;
   for (auto& op : m->stage) refs.push_back({&op, -1, 0});
-  for (int b = 0; b < m->B; b++) for (auto& op : m->fwd[b]) refs.push_back({&op, b, 1});
+  for (int b = 0; b < m->B; b++) {
+    for (auto& op : m->fwd[b]) refs.push_back({&op, b, 1});
+    for (auto& op : m->hfwd[b]) refs.push_back({&op, b, 1});
+  }
   for (int b = m->B - 1; b >= 0; b--) for (auto& op : m->bwd[b]) refs.push_back({&op, b, 2});
   for (auto& op : m->opt) refs.push_back({&op, -1, 3});
   while (m->ev_prof.size() < 2 * refs.size()) {

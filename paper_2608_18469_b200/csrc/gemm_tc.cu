@@ -566,7 +566,7 @@ bool encode_2d(void* out, const void* base, long long inner, long long outer, lo
 }
 
 template <int BN, bool A_MN, bool B_MN>
-cudaError_t launch_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s) {
+cudaError_t launch_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas) {
   constexpr size_t smem = (size_t)STAGES * (BM * BK * 2 + BN * BK * 2) + EPI_WARPS * (EPI_STAGE_BYTES + 256) + 8 * (2 * STAGES + 6) + 1024;
   static bool attr_set = false;
   if (!attr_set) {
@@ -585,7 +585,8 @@ cudaError_t launch_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s) {
     if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms < 1) num_sms = 148;
   }
   const long long total = (long long)((g.N + BN - 1) / BN) * ((g.M + BM - 1) / BM) * g.splits;
-  dim3 grid((unsigned)(total < num_sms ? total : num_sms));
+  long long cap = (max_ctas > 0 && max_ctas < num_sms) ? max_ctas : num_sms;
+  dim3 grid((unsigned)(total < cap ? total : cap));
   CUtensorMap ma, mb, mc, mp;
   static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
   memcpy(&ma, plan.map_a, sizeof(ma));
@@ -601,11 +602,11 @@ cudaError_t launch_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s) {
 }
 
 template <int BN>
-cudaError_t launch_bn(const GemmArgs& g, const TcPlan& plan, cudaStream_t s) {
-  if (!plan.a_mn && !plan.b_mn) return launch_t<BN, false, false>(g, plan, s);
-  if (!plan.a_mn && plan.b_mn) return launch_t<BN, false, true>(g, plan, s);
-  if (plan.a_mn && !plan.b_mn) return launch_t<BN, true, false>(g, plan, s);
-  return launch_t<BN, true, true>(g, plan, s);
+cudaError_t launch_bn(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas) {
+  if (!plan.a_mn && !plan.b_mn) return launch_t<BN, false, false>(g, plan, s, max_ctas);
+  if (!plan.a_mn && plan.b_mn) return launch_t<BN, false, true>(g, plan, s, max_ctas);
+  if (plan.a_mn && !plan.b_mn) return launch_t<BN, true, false>(g, plan, s, max_ctas);
+  return launch_t<BN, true, true>(g, plan, s, max_ctas);
 }
 
 }  // namespace
@@ -667,8 +668,8 @@ bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan) {
   return true;
 }
 
-cudaError_t tc_gemm_launch(const GemmArgs& g, const TcPlan& plan, cudaStream_t s) {
-  return plan.bn == 64 ? launch_bn<64>(g, plan, s) : launch_bn<128>(g, plan, s);
+cudaError_t tc_gemm_launch(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas) {
+  return plan.bn == 64 ? launch_bn<64>(g, plan, s, max_ctas) : launch_bn<128>(g, plan, s, max_ctas);
 }
 
 }  // namespace erase

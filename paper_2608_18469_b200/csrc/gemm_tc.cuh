@@ -31,6 +31,8 @@ bool tc_gemm_supported(const GemmArgs& g);
 // Encodes the TMA descriptors.  g.ws must already point at splits*M*N floats when g.splits > 1.
 // Returns false (and leaves the GEMM to the SIMT kernel) if a descriptor cannot be encoded.
 bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan);
-cudaError_t tc_gemm_launch(const GemmArgs& g, const TcPlan& plan, cudaStream_t s);
+// max_ctas > 0 caps the persistent grid (an SM budget: lets kernels of other streams run beside it);
+// the tile-to-CTA assignment does not enter the arithmetic, so results do not depend on it.
+cudaError_t tc_gemm_launch(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas = 0);
 
 }  // namespace erase

@@ -163,10 +163,14 @@ cudaError_t splitk_reduce(const float* ws, int splits, long long mn, int N, floa
 
 // ------------------------------------------------------------------------------------------
 // column sums (bias gradients, head weight gradient of the BCE head)
+// A CTA sums a strip of 64 columns over one chunk of the rows (a thread owns two adjacent
+// columns: one 4-byte load per bf16 pair, 128 bytes per warp and row); the chunk partials go to
+// ws and the last CTA of a strip to finish (atomic ticket) adds them in chunk order, so the
+// result does not depend on which CTA that is.  The ticket counter is left at zero again.
 // ------------------------------------------------------------------------------------------
 int colsum_chunks(int rows, int cols) {
-  int strips = (cols + 31) / 32;
-  int want = (296 + strips - 1) / strips;
+  int strips = (cols + 127) / 128;   // at least as many strips as either element type uses
+  int want = (592 + strips - 1) / strips;
   int maxc = rows / 64;
   if (maxc < 1) maxc = 1;
   if (want > maxc) want = maxc;
@@ -174,44 +178,149 @@ int colsum_chunks(int rows, int cols) {
   return want;
 }
 
+template <typename T> __device__ __forceinline__ float2 ld2(const T* p, bool vec);
+template <> __device__ __forceinline__ float2 ld2<float>(const float* p, bool vec) {
+  if (vec) return *reinterpret_cast<const float2*>(p);
+  return make_float2(p[0], p[1]);
+}
+template <> __device__ __forceinline__ float2 ld2<bf16_t>(const bf16_t* p, bool vec) {
+  if (vec) return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(p));
+  return make_float2(__bfloat162float(p[0]), __bfloat162float(p[1]));
+}
+
+// Shared tail of the two-stage reductions: returns true in the CTA that arrives last on `ticket`.
+__device__ __forceinline__ bool last_cta(int* ticket, int expected) {
+  __shared__ int s_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int t = atomicAdd(ticket, 1);
+    s_last = (t == expected - 1);
+    if (s_last) *ticket = 0;
+  }
+  __syncthreads();
+  if (s_last) __threadfence();
+  return s_last != 0;
+}
+
+template <typename T> struct VecOf;
+template <> struct VecOf<float> { static constexpr int N = 4; };
+template <> struct VecOf<bf16_t> { static constexpr int N = 8; };
+
+// 16 bytes = VecOf<T>::N consecutive elements -> floats
+template <typename T> __device__ __forceinline__ void ld_vec(const T* p, float* out);
+template <> __device__ __forceinline__ void ld_vec<float>(const float* p, float* out) {
+  const float4 q = *reinterpret_cast<const float4*>(p);
+  out[0] = q.x; out[1] = q.y; out[2] = q.z; out[3] = q.w;
+}
+template <> __device__ __forceinline__ void ld_vec<bf16_t>(const bf16_t* p, float* out) {
+  const uint4 q = *reinterpret_cast<const uint4*>(p);
+  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+  for (int j = 0; j < 4; j++) {
+    out[2 * j] = __uint_as_float(w[j] << 16);
+    out[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+  }
+}
+
+// A CTA sums a strip of 32*VEC columns over one chunk of rows: a thread owns VEC adjacent
+// columns (one 16-byte load per row) and every 8th row, four rows in flight.
 template <typename T>
 __global__ void __launch_bounds__(256) colsum_kernel(const T* __restrict__ X, long long ldx, int rows,
                                                      int cols, const float* __restrict__ scale,
-                                                     float* __restrict__ dst, int chunks, int dact,
-                                                     const float* __restrict__ colscale) {
-  __shared__ float sm[8][33];
-  int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
-  int c = blockIdx.x * 32 + cx;
-  int per = (rows + chunks - 1) / chunks;
-  int rb = blockIdx.y * per, re = min(rows, rb + per);
-  float a = 0.f;
-  if (c < cols)
-    for (int r = rb + ry; r < re; r += 8) {
-      float v = X ? ldf(X + (long long)r * ldx + c) : 1.f;
-      if (dact != ACT_NONE) v = act_deriv(dact, v);
-      if (scale) v *= scale[r];
-      a += v;
-    }
-  sm[ry][cx] = a;
-  __syncthreads();
-  if (ry == 0 && c < cols) {
-    float t = 0.f;
+                                                     float* __restrict__ ws, float* __restrict__ out, int chunks,
+                                                     int dact, const float* __restrict__ colscale, int* tickets) {
+  constexpr int VEC = VecOf<T>::N;
+  constexpr int SW = 32 * VEC;  // strip width
+  __shared__ float sm[8][SW];
+  const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
+  const int c = blockIdx.x * SW + cx * VEC;
+  const int per = (rows + chunks - 1) / chunks;
+  const int rb = blockIdx.y * per, re = min(rows, rb + per);
+  const bool vec = X && (c + VEC <= cols) && (ldx % VEC == 0) && ((reinterpret_cast<uintptr_t>(X) & 15) == 0);
+  float a[VEC];
 #pragma unroll
-    for (int i = 0; i < 8; i++) t += sm[i][cx];
-    if (colscale) t *= colscale[c];
-    dst[(long long)blockIdx.y * cols + c] = t;
+  for (int j = 0; j < VEC; j++) a[j] = 0.f;
+  if (c < cols) {
+    if (vec) {
+      int r = rb + ry;
+      for (; r + 24 < re; r += 32) {
+        float v[4][VEC];
+#pragma unroll
+        for (int u = 0; u < 4; u++) ld_vec<T>(X + (long long)(r + 8 * u) * ldx + c, v[u]);
+#pragma unroll
+        for (int u = 0; u < 4; u++) {
+          const float sc = scale ? scale[r + 8 * u] : 1.f;
+#pragma unroll
+          for (int j = 0; j < VEC; j++) {
+            float t = v[u][j];
+            if (dact != ACT_NONE) t = act_deriv(dact, t);
+            a[j] = fmaf(t, sc, a[j]);
+          }
+        }
+      }
+      for (; r < re; r += 8) {
+        float v[VEC];
+        ld_vec<T>(X + (long long)r * ldx + c, v);
+        const float sc = scale ? scale[r] : 1.f;
+#pragma unroll
+        for (int j = 0; j < VEC; j++) {
+          float t = v[j];
+          if (dact != ACT_NONE) t = act_deriv(dact, t);
+          a[j] = fmaf(t, sc, a[j]);
+        }
+      }
+    } else {
+      for (int r = rb + ry; r < re; r += 8) {
+        const float sc = scale ? scale[r] : 1.f;
+#pragma unroll
+        for (int j = 0; j < VEC; j++) {
+          if (c + j < cols) {
+            float t = X ? ldf(X + (long long)r * ldx + c + j) : 1.f;
+            if (dact != ACT_NONE) t = act_deriv(dact, t);
+            a[j] = fmaf(t, sc, a[j]);
+          }
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < VEC; j++) sm[ry][cx * VEC + j] = a[j];
+  __syncthreads();
+  float* dst = chunks == 1 ? out : ws + (long long)blockIdx.y * cols;
+  for (int i = threadIdx.x; i < SW; i += 256) {
+    const int cc = blockIdx.x * SW + i;
+    if (cc < cols) {
+      float t = 0.f;
+#pragma unroll
+      for (int k = 0; k < 8; k++) t += sm[k][i];
+      if (chunks == 1 && colscale) t *= colscale[cc];
+      dst[cc] = t;
+    }
+  }
+  if (chunks == 1) return;
+  if (!last_cta(tickets + blockIdx.x, chunks)) return;
+  for (int i = threadIdx.x; i < SW; i += 256) {
+    const int cc = blockIdx.x * SW + i;
+    if (cc < cols) {
+      float t = 0.f;
+      for (int k = 0; k < chunks; k++) t += ws[(long long)k * cols + cc];
+      if (colscale) t *= colscale[cc];
+      out[cc] = t;
+    }
   }
 }
 
 cudaError_t colsum(const void* X, bool x_bf16, long long ldx, int rows, int cols, const float* scale,
-                   float* ws, int chunks, float* out, cudaStream_t s, int dact, const float* colscale) {
-  dim3 grid(cdiv(cols, 32), chunks);
-  float* dst = chunks == 1 ? out : ws;
-  if (x_bf16) colsum_kernel<bf16_t><<<grid, 256, 0, s>>>((const bf16_t*)X, ldx, rows, cols, scale, dst, chunks, dact, colscale);
-  else colsum_kernel<float><<<grid, 256, 0, s>>>((const float*)X, ldx, rows, cols, scale, dst, chunks, dact, colscale);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess || chunks == 1) return e;
-  return splitk_reduce(ws, chunks, cols, cols, out, cols, s);
+                   float* ws, int chunks, int* tickets, float* out, cudaStream_t s, int dact, const float* colscale) {
+  if (x_bf16) {
+    dim3 grid(cdiv(cols, 256), chunks);
+    colsum_kernel<bf16_t><<<grid, 256, 0, s>>>((const bf16_t*)X, ldx, rows, cols, scale, ws, out, chunks, dact, colscale, tickets);
+  } else {
+    dim3 grid(cdiv(cols, 128), chunks);
+    colsum_kernel<float><<<grid, 256, 0, s>>>((const float*)X, ldx, rows, cols, scale, ws, out, chunks, dact, colscale, tickets);
+  }
+  return cudaGetLastError();
 }
 
 // ------------------------------------------------------------------------------------------
@@ -283,46 +392,64 @@ template <typename T>
 __global__ void __launch_bounds__(256) layernorm_param_grad_kernel(const T* __restrict__ dy, const T* __restrict__ x,
                                                                    const float* __restrict__ mean,
                                                                    const float* __restrict__ rstd,
-                                                                   float* __restrict__ dst_g, float* __restrict__ dst_b,
-                                                                   int rows, int d, int chunks) {
-  __shared__ float sg[8][33], sb[8][33];
-  int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
-  int c = blockIdx.x * 32 + cx;
-  int per = (rows + chunks - 1) / chunks;
-  int rb = blockIdx.y * per, re = min(rows, rb + per);
-  float ag = 0.f, ab = 0.f;
-  if (c < d)
+                                                                   float* __restrict__ ws, float* __restrict__ dgain,
+                                                                   float* __restrict__ dshift, int rows, int d, int chunks,
+                                                                   int* tickets) {
+  __shared__ float sg[8][64], sb[8][64];
+  const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
+  const int c = blockIdx.x * 64 + cx * 2;
+  const int per = (rows + chunks - 1) / chunks;
+  const int rb = blockIdx.y * per, re = min(rows, rb + per);
+  const bool two = c + 1 < d;
+  const bool vec = two && (d % 2 == 0);
+  float g0 = 0.f, g1 = 0.f, b0 = 0.f, b1 = 0.f;
+  if (c < d) {
     for (int r = rb + ry; r < re; r += 8) {
-      float g = ldf(dy + (long long)r * d + c);
-      float xh = (ldf(x + (long long)r * d + c) - mean[r]) * rstd[r];
-      ag += g * xh;
-      ab += g;
+      float2 gy, xv;
+      if (two) { gy = ld2<T>(dy + (long long)r * d + c, vec); xv = ld2<T>(x + (long long)r * d + c, vec); }
+      else { gy = make_float2(ldf(dy + (long long)r * d + c), 0.f); xv = make_float2(ldf(x + (long long)r * d + c), 0.f); }
+      const float mu = mean[r], rs = rstd[r];
+      g0 = fmaf(gy.x, (xv.x - mu) * rs, g0);
+      g1 = fmaf(gy.y, (xv.y - mu) * rs, g1);
+      b0 += gy.x;
+      b1 += gy.y;
     }
-  sg[ry][cx] = ag;
-  sb[ry][cx] = ab;
+  }
+  sg[ry][cx * 2] = g0; sg[ry][cx * 2 + 1] = g1;
+  sb[ry][cx * 2] = b0; sb[ry][cx * 2 + 1] = b1;
   __syncthreads();
-  if (ry == 0 && c < d) {
-    float tg = 0.f, tb = 0.f;
+  float* pg = chunks == 1 ? dgain : ws + (long long)blockIdx.y * d;
+  float* pb = chunks == 1 ? dshift : ws + (long long)(chunks + blockIdx.y) * d;
+  if (threadIdx.x < 64) {
+    const int cc = blockIdx.x * 64 + threadIdx.x;
+    if (cc < d) {
+      float tg = 0.f, tb = 0.f;
 #pragma unroll
-    for (int i = 0; i < 8; i++) { tg += sg[i][cx]; tb += sb[i][cx]; }
-    dst_g[(long long)blockIdx.y * d + c] = tg;
-    dst_b[(long long)blockIdx.y * d + c] = tb;
+      for (int i = 0; i < 8; i++) { tg += sg[i][threadIdx.x]; tb += sb[i][threadIdx.x]; }
+      pg[cc] = tg;
+      pb[cc] = tb;
+    }
+  }
+  if (chunks == 1) return;
+  if (!last_cta(tickets + blockIdx.x, chunks)) return;
+  if (threadIdx.x < 64) {
+    const int cc = blockIdx.x * 64 + threadIdx.x;
+    if (cc < d) {
+      float tg = 0.f, tb = 0.f;
+      for (int k = 0; k < chunks; k++) { tg += ws[(long long)k * d + cc]; tb += ws[(long long)(chunks + k) * d + cc]; }
+      dgain[cc] = tg;
+      dshift[cc] = tb;
+    }
   }
 }
 
 cudaError_t layernorm_param_grad(const void* dy, const void* x, const float* mean, const float* rstd,
-                                 float* ws, int chunks, float* dgain, float* dshift, int rows, int d,
+                                 float* ws, int chunks, int* tickets, float* dgain, float* dshift, int rows, int d,
                                  bool bf16, cudaStream_t s) {
-  dim3 grid(cdiv(d, 32), chunks);
-  float* pg = chunks == 1 ? dgain : ws;
-  float* pb = chunks == 1 ? dshift : ws + (long long)chunks * d;
-  if (bf16) layernorm_param_grad_kernel<bf16_t><<<grid, 256, 0, s>>>((const bf16_t*)dy, (const bf16_t*)x, mean, rstd, pg, pb, rows, d, chunks);
-  else layernorm_param_grad_kernel<float><<<grid, 256, 0, s>>>((const float*)dy, (const float*)x, mean, rstd, pg, pb, rows, d, chunks);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess || chunks == 1) return e;
-  e = splitk_reduce(pg, chunks, d, d, dgain, d, s);
-  if (e != cudaSuccess) return e;
-  return splitk_reduce(pb, chunks, d, d, dshift, d, s);
+  dim3 grid(cdiv(d, 64), chunks);
+  if (bf16) layernorm_param_grad_kernel<bf16_t><<<grid, 256, 0, s>>>((const bf16_t*)dy, (const bf16_t*)x, mean, rstd, ws, dgain, dshift, rows, d, chunks, tickets);
+  else layernorm_param_grad_kernel<float><<<grid, 256, 0, s>>>((const float*)dy, (const float*)x, mean, rstd, ws, dgain, dshift, rows, d, chunks, tickets);
+  return cudaGetLastError();
 }
 
 // ------------------------------------------------------------------------------------------
@@ -669,8 +796,87 @@ __global__ void __launch_bounds__(256) softmax_ce_kernel(T* __restrict__ logits,
   if (threadIdx.x == 0) rowloss[row] = lse - lt;
 }
 
+// bf16 rows kept in registers: one 16-byte load and one 16-byte store per 8 logits, nothing re-read.
+// A thread owns vectors tid, tid+THREADS, ...; VPT of them (V <= THREADS*8*VPT, V % 8 == 0).
+template <int THREADS, int VPT>
+__global__ void __launch_bounds__(THREADS) softmax_ce_reg_kernel(bf16_t* __restrict__ logits,
+                                                                  const int32_t* __restrict__ ids, int T_,
+                                                                  float* __restrict__ rowloss, int V, float inv_rows) {
+  __shared__ float sm[THREADS / 32];
+  const int row = blockIdx.x, nvec = V >> 3;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint4* p = reinterpret_cast<uint4*>(logits + (long long)row * V);
+  const int tgt = ids[(long long)(row / T_) * (T_ + 1) + (row % T_) + 1];
+  const float L2E = 1.4426950408889634f;
+  float x[VPT][8];
+  float mx = -INFINITY, lt = 0.f;
+#pragma unroll
+  for (int k = 0; k < VPT; k++) {
+    const int i = threadIdx.x + k * THREADS;
+    if (i < nvec) {
+      const uint4 q = p[i];
+      const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+      for (int j = 0; j < 4; j++) {
+        x[k][2 * j] = __uint_as_float(w[j] << 16);
+        x[k][2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+      }
+#pragma unroll
+      for (int j = 0; j < 8; j++) {
+        mx = fmaxf(mx, x[k][j]);
+        if (i * 8 + j == tgt) lt = x[k][j];
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; j++) x[k][j] = -INFINITY;
+    }
+  }
+  auto block_reduce = [&](float v, bool is_max) {
+    v = is_max ? warp_max(v) : warp_sum(v);
+    __syncthreads();
+    if (lane == 0) sm[warp] = v;
+    __syncthreads();
+    float r = sm[0];
+    for (int i = 1; i < THREADS / 32; i++) r = is_max ? fmaxf(r, sm[i]) : r + sm[i];
+    return r;
+  };
+  mx = block_reduce(mx, true);
+  float se = 0.f;
+#pragma unroll
+  for (int k = 0; k < VPT; k++)
+#pragma unroll
+    for (int j = 0; j < 8; j++) se += exp2f((x[k][j] - mx) * L2E);
+  se = block_reduce(se, false);
+  const float lse = mx + logf(se);
+#pragma unroll
+  for (int k = 0; k < VPT; k++) {
+    const int i = threadIdx.x + k * THREADS;
+    if (i < nvec) {
+      float g[8];
+#pragma unroll
+      for (int j = 0; j < 8; j++) g[j] = (exp2f((x[k][j] - lse) * L2E) - (i * 8 + j == tgt ? 1.f : 0.f)) * inv_rows;
+      uint4 q;
+      __nv_bfloat162 h;
+      h = __floats2bfloat162_rn(g[0], g[1]); q.x = *reinterpret_cast<uint32_t*>(&h);
+      h = __floats2bfloat162_rn(g[2], g[3]); q.y = *reinterpret_cast<uint32_t*>(&h);
+      h = __floats2bfloat162_rn(g[4], g[5]); q.z = *reinterpret_cast<uint32_t*>(&h);
+      h = __floats2bfloat162_rn(g[6], g[7]); q.w = *reinterpret_cast<uint32_t*>(&h);
+      p[i] = q;
+    }
+  }
+  if ((tgt >> 3) % THREADS == threadIdx.x) rowloss[row] = lse - lt;   // the thread that holds the target logit
+}
+
 cudaError_t softmax_ce_inplace(void* logits, const int32_t* ids, int T_, float* rowloss, int rows, int V,
                                float inv_rows, bool bf16, cudaStream_t s) {
+  if (bf16 && V % 8 == 0 && (reinterpret_cast<uintptr_t>(logits) & 15) == 0) {
+    const int nvec = V / 8;
+    bf16_t* lg = (bf16_t*)logits;
+    if (nvec <= 256 * 2) { softmax_ce_reg_kernel<256, 2><<<rows, 256, 0, s>>>(lg, ids, T_, rowloss, V, inv_rows); return cudaGetLastError(); }
+    if (nvec <= 256 * 4) { softmax_ce_reg_kernel<256, 4><<<rows, 256, 0, s>>>(lg, ids, T_, rowloss, V, inv_rows); return cudaGetLastError(); }
+    if (nvec <= 1024 * 2) { softmax_ce_reg_kernel<1024, 2><<<rows, 1024, 0, s>>>(lg, ids, T_, rowloss, V, inv_rows); return cudaGetLastError(); }
+    if (nvec <= 1024 * 4) { softmax_ce_reg_kernel<1024, 4><<<rows, 1024, 0, s>>>(lg, ids, T_, rowloss, V, inv_rows); return cudaGetLastError(); }
+  }
   if (bf16) softmax_ce_kernel<bf16_t><<<rows, 256, 0, s>>>((bf16_t*)logits, ids, T_, rowloss, V, inv_rows);
   else softmax_ce_kernel<float><<<rows, 256, 0, s>>>((float*)logits, ids, T_, rowloss, V, inv_rows);
   return cudaGetLastError();

@@ -53,11 +53,12 @@ cudaError_t splitk_reduce(const float* ws, int splits, long long mn, int N, floa
 
 // out[c] = colscale[c] * sum_r scale[r] * f(X[r, c]); X is [rows, cols] with row stride ldx,
 // f = identity or the derivative of activation `dact` evaluated at X; scale and colscale may be
-// null (read as 1) and so may X (read as 1).  Two-stage with a fixed row partition into `chunks`;
-// ws holds chunks*cols floats.
+// null (read as 1) and so may X (read as 1).  Two-stage with a fixed row partition into `chunks`
+// in ONE launch: ws holds chunks*cols floats, tickets ceil(cols/64) zero-initialised ints (left
+// at zero); the CTA that finishes a column strip last adds the partials in chunk order.
 int colsum_chunks(int rows, int cols);
 cudaError_t colsum(const void* X, bool x_bf16, long long ldx, int rows, int cols, const float* scale,
-                   float* ws, int chunks, float* out, cudaStream_t s, int dact = ACT_NONE,
+                   float* ws, int chunks, int* tickets, float* out, cudaStream_t s, int dact = ACT_NONE,
                    const float* colscale = nullptr);
 
 // LayerNorm over the last dimension (eps 1e-5, biased variance); saves mean and 1/std per row.
@@ -67,9 +68,9 @@ cudaError_t layernorm_fwd(const void* x, const float* gain, const float* shift, 
 cudaError_t layernorm_bwd_dx(const void* dy, const void* x, const float* gain, const float* mean,
                              const float* rstd, const void* add, void* dx, int rows, int d, bool bf16,
                              cudaStream_t s);
-// dgain[c] = sum_r dy*xhat, dshift[c] = sum_r dy; ws holds 2*chunks*d floats.
+// dgain[c] = sum_r dy*xhat, dshift[c] = sum_r dy; ws holds 2*chunks*d floats, tickets as for colsum.
 cudaError_t layernorm_param_grad(const void* dy, const void* x, const float* mean, const float* rstd,
-                                 float* ws, int chunks, float* dgain, float* dshift, int rows, int d,
+                                 float* ws, int chunks, int* tickets, float* dgain, float* dshift, int rows, int d,
                                  bool bf16, cudaStream_t s);
 
 // Causal self-attention over qkv [batch*T, 3*d] = [Q | K | V], heads are contiguous dh-wide

@@ -112,4 +112,6 @@ def test_erase_schedule_is_bit_identical_to_serial(name):
     from paper_2608_18469_b200 import binding
     _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=1, flags=binding.GRAPH))
     _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=nb + 1, flags=binding.GRAPH))
+    _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=nb + 1, flags=binding.EARLY_HEAD))
+    _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=2, flags=binding.GRAPH | binding.EARLY_HEAD))
     assert serial["launches"] > 0
