@@ -45,7 +45,7 @@ struct TcArgs {
   long long* dbg;  // optional: clock64 stamps of CTA 0's first tile (development aid), else null
   int tma_c;       // C (or the split-K partials) leaves through shared memory + TMA store
   int tma_p;       // so does the pre-activation copy
-  int plain;       // the epilogue is the identity (no alpha, bias, activation or auxiliary operand)
+  int plain;       // 1: the epilogue is the identity; 2: bias add only; 0: general
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -263,7 +263,10 @@ __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 
 // Persistent kernel: CTA c works on tiles c, c + gridDim.x, ... (m fastest, then n, then split).
-template <int BN, bool A_MN, bool B_MN>
+// GENERAL = false compiles the epilogue down to "identity or bias add" (forward Linears without
+// activation, every dgrad/wgrad without auxiliary operand): a much smaller loop body, which is what
+// bounds the epilogue (instruction fetch), so those GEMMs get their own instantiation.
+template <int BN, bool A_MN, bool B_MN, bool GENERAL>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_p,
@@ -440,7 +443,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const int row = m0 + q * 32 + lane;
       const bool row_ok = row < p.M;
       const long long dflags = p.dbg ? p.dbg[15] : 0;
-      const int npass = (p.epi.pre_out && p.tma_p) ? 2 : 1;   // pass 0 of 2 writes the pre-activation copy
+      const int npass = (GENERAL && p.epi.pre_out && p.tma_p) ? 2 : 1;   // pass 0 of 2 writes the pre-activation copy
       if (active && n0 + cbeg < p.N) {
         for (int pass = 0; pass < npass; pass++) {
           const bool pre_pass = npass == 2 && pass == 0;
@@ -467,7 +470,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               F8 f;
 #pragma unroll
               for (int j = 0; j < 8; j++) f.v[j] = __uint_as_float(r[g8 * 8 + j]);
-              if (row_ok && n < p.N && p.splits == 1 && !p.plain) f = epilogue_values8(p, f, row, n, pre_pass, bias_s + cc + g8 * 8);
+              if (p.plain == 2) {          // bias only: the common forward case, kept free of the general path
+                const float4 b0 = *reinterpret_cast<const float4*>(bias_s + cc + g8 * 8);
+                const float4 b1 = *reinterpret_cast<const float4*>(bias_s + cc + g8 * 8 + 4);
+                f.v[0] += b0.x; f.v[1] += b0.y; f.v[2] += b0.z; f.v[3] += b0.w;
+                f.v[4] += b1.x; f.v[5] += b1.y; f.v[6] += b1.z; f.v[7] += b1.w;
+              } else if (GENERAL && row_ok && n < p.N && p.splits == 1 && !p.plain) {
+                f = epilogue_values8(p, f, row, n, pre_pass, bias_s + cc + g8 * 8);
+              }
               const float* v = f.v;
               if (!via_tma) {
                 if (row_ok && n < p.N && !(dflags & 1)) direct_store8(p, f, row, n, split);
@@ -565,12 +575,12 @@ bool encode_2d(void* out, const void* base, long long inner, long long outer, lo
   return encode_map(out, base, false, 2, dims, strides, box);
 }
 
-template <int BN, bool A_MN, bool B_MN>
+template <int BN, bool A_MN, bool B_MN, bool GENERAL>
 cudaError_t launch_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas) {
   constexpr size_t smem = (size_t)STAGES * (BM * BK * 2 + BN * BK * 2) + EPI_WARPS * (EPI_STAGE_BYTES + 256) + 8 * (2 * STAGES + 6) + 1024;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<BN, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<BN, A_MN, B_MN, GENERAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -596,17 +606,23 @@ cudaError_t launch_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int 
   p.tma_c = plan.tma_c;
   p.tma_p = plan.tma_p;
   const Epilogue& e = g.epi;
-  p.plain = (e.alpha == 1.f && !e.bias && e.act == ACT_NONE && !e.pre_out && !e.mul && !e.res && e.dact == ACT_NONE) ? 1 : 0;
-  tc_gemm_kernel<BN, A_MN, B_MN><<<grid, TC_THREADS, smem, s>>>(ma, mb, mc, mp, p);
+  const bool no_aux = e.alpha == 1.f && e.act == ACT_NONE && !e.pre_out && !e.mul && !e.res && e.dact == ACT_NONE;
+  p.plain = no_aux ? (e.bias ? (g.splits == 1 ? 2 : 1) : 1) : 0;   // 1: identity, 2: bias only, 0: general
+  tc_gemm_kernel<BN, A_MN, B_MN, GENERAL><<<grid, TC_THREADS, smem, s>>>(ma, mb, mc, mp, p);
   return cudaGetLastError();
 }
 
-template <int BN>
+static bool epilogue_is_simple(const GemmArgs& g) {
+  const Epilogue& e = g.epi;
+  return g.splits > 1 || (e.alpha == 1.f && e.act == ACT_NONE && !e.pre_out && !e.mul && !e.res && e.dact == ACT_NONE);
+}
+
+template <int BN, bool GENERAL>
 cudaError_t launch_bn(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas) {
-  if (!plan.a_mn && !plan.b_mn) return launch_t<BN, false, false>(g, plan, s, max_ctas);
-  if (!plan.a_mn && plan.b_mn) return launch_t<BN, false, true>(g, plan, s, max_ctas);
-  if (plan.a_mn && !plan.b_mn) return launch_t<BN, true, false>(g, plan, s, max_ctas);
-  return launch_t<BN, true, true>(g, plan, s, max_ctas);
+  if (!plan.a_mn && !plan.b_mn) return launch_t<BN, false, false, GENERAL>(g, plan, s, max_ctas);
+  if (!plan.a_mn && plan.b_mn) return launch_t<BN, false, true, GENERAL>(g, plan, s, max_ctas);
+  if (plan.a_mn && !plan.b_mn) return launch_t<BN, true, false, GENERAL>(g, plan, s, max_ctas);
+  return launch_t<BN, true, true, GENERAL>(g, plan, s, max_ctas);
 }
 
 }  // namespace
@@ -669,7 +685,8 @@ bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan) {
 }
 
 cudaError_t tc_gemm_launch(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas) {
-  return plan.bn == 64 ? launch_bn<64>(g, plan, s, max_ctas) : launch_bn<128>(g, plan, s, max_ctas);
+  if (epilogue_is_simple(g)) return plan.bn == 64 ? launch_bn<64, false>(g, plan, s, max_ctas) : launch_bn<128, false>(g, plan, s, max_ctas);
+  return plan.bn == 64 ? launch_bn<64, true>(g, plan, s, max_ctas) : launch_bn<128, true>(g, plan, s, max_ctas);
 }
 
 }  // namespace erase
