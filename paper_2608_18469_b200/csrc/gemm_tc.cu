@@ -18,6 +18,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
+#include <stdlib.h>
 #include <string.h>
 
 namespace erase {
@@ -27,7 +28,8 @@ namespace {
 constexpr int BM = 128;
 constexpr int BK = 64;          // bf16 elements = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
-constexpr int STAGES = 4;
+__host__ __device__ constexpr int stages_for(int bn) { return bn == 256 ? 3 : 4; }   // 3 x 48 KB or 4 x 32 KB (or 24 KB)
+constexpr uint32_t EPI_BIAS_BYTES = 512;              // up to 128 bias floats per epilogue warp
 constexpr int EPI_WARPS = 8;                       // two per TMEM lane quarter, each takes half the columns
 constexpr int TC_THREADS = 32 * (2 + EPI_WARPS);
 constexpr uint32_t EPI_STAGE_BYTES = 4096;             // 32 rows x 128 bytes per epilogue warp
@@ -262,7 +264,22 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t sr
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 
-// Persistent kernel: CTA c works on tiles c, c + gridDim.x, ... (m fastest, then n, then split).
+// Tile order: splits outermost; inside a split, bands of 8 column tiles, and inside a band m
+// outer / n inner.  The ~148 tiles in flight at any time then cover about 18 row tiles x 8
+// column tiles, so each operand slab fetched from HBM is reused out of L2 by its neighbours.
+__device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int& mt, int& nt, int& split) {
+  const int per_split = tiles_m * tiles_n;
+  split = t / per_split;
+  const int r = t - split * per_split;
+  const int band = r / (8 * tiles_m);
+  const int n_first = band * 8;
+  const int width = min(8, tiles_n - n_first);
+  const int rr = r - band * 8 * tiles_m;
+  mt = rr / width;
+  nt = n_first + rr - mt * width;
+}
+
+// Persistent kernel: CTA c works on tiles c, c + gridDim.x, ... in the order of tile_coords.
 // GENERAL = false compiles the epilogue down to "identity or bias add" (forward Linears without
 // activation, every dgrad/wgrad without auxiliary operand): a much smaller loop body, which is what
 // bounds the epilogue (instruction fetch), so those GEMMs get their own instantiation.
@@ -276,23 +293,31 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   constexpr uint32_t B_BYTES = BN * BK * 2;
   constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
   constexpr uint32_t TMEM_COLS = 2 * BN;            // two accumulators: epilogue(i) overlaps mainloop(i+1)
+  constexpr int STAGES = stages_for(BN);
+  constexpr int CPW = BN >= 128 ? BN / 2 : 64;      // tile columns per epilogue warp (two warps per lane quarter)
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t epi_base = smem_base + STAGES * STAGE_BYTES;          // EPI_WARPS x 4 KB output staging
-  const uint32_t bias_base = epi_base + EPI_WARPS * EPI_STAGE_BYTES;    // EPI_WARPS x 64 floats of bias
-  const uint32_t bar_base = bias_base + EPI_WARPS * 256;
+  const uint32_t bias_base = epi_base + EPI_WARPS * EPI_STAGE_BYTES;    // EPI_WARPS x CPW floats of bias
+  const uint32_t bar_base = bias_base + EPI_WARPS * EPI_BIAS_BYTES;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
   uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
   volatile uint32_t* tmem_slot_ptr =
-      reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * (EPI_STAGE_BYTES + 256) + 8u * (2 * STAGES + 4));
+      reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * (EPI_STAGE_BYTES + EPI_BIAS_BYTES) + 8u * (2 * STAGES + 4));
   const uint32_t tmem_slot = bar_base + 8u * (2 * STAGES + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const bool dbg = p.dbg != nullptr && blockIdx.x == 0;
   if (dbg && threadIdx.x == 0) p.dbg[0] = clock64();
+  if (threadIdx.x == 32) {   // descriptor fetches overlap the barrier and TMEM set-up
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+    if (p.tma_c) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_c) : "memory");
+    if (p.tma_p) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_p) : "memory");
+  }
   const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
   const int total = tiles_m * tiles_n * p.splits;
   const int kchunk = (((p.K + p.splits - 1) / p.splits) + BK - 1) / BK * BK;
@@ -322,12 +347,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
       uint32_t it = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
-        const int m0 = (t % tiles_m) * BM, n0 = ((t / tiles_m) % tiles_n) * BN, split = t / (tiles_m * tiles_n);
+        int mt, nt, split;
+        tile_coords(t, tiles_m, tiles_n, mt, nt, split);
+        const int m0 = mt * BM, n0 = nt * BN;
         const int kbeg = split * kchunk, kend = min(p.K, kbeg + kchunk);
         const int num_kb = kend > kbeg ? (kend - kbeg + BK - 1) / BK : 0;
         for (int kb = 0; kb < num_kb; kb++, it++) {
@@ -413,22 +438,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // (unaligned leading dimension) are stored directly.
     const int ew = warp - 2;
     const int q = warp & 3;                       // TMEM lane quarter this warp may read
-    const int cbeg = (ew / 4) * 64;               // first tile column of this warp
+    const int cbeg = (ew / 4) * CPW;              // first tile column of this warp
     const bool active = cbeg < BN;                // BN = 64: only one warp per quarter has columns
     const uint32_t stage = epi_base + ew * EPI_STAGE_BYTES;
     const uint32_t my_row = stage + lane * 128;
-    float* bias_s = reinterpret_cast<float*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * EPI_STAGE_BYTES + ew * 256);
+    float* bias_s = reinterpret_cast<float*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * EPI_STAGE_BYTES + ew * EPI_BIAS_BYTES);
     const bool out_f32 = p.splits > 1 || p.c_f32;
     bool store_pending = false;                   // lane 0: a TMA store may still be reading the staging buffer
     uint32_t lt = 0;
     for (int t = blockIdx.x; t < total; t += gridDim.x, lt++) {
-      const int m0 = (t % tiles_m) * BM, n0 = ((t / tiles_m) % tiles_n) * BN, split = t / (tiles_m * tiles_n);
+      int mt, nt, split;
+      tile_coords(t, tiles_m, tiles_n, mt, nt, split);
+      const int m0 = mt * BM, n0 = nt * BN;
       const int kbeg = split * kchunk, kend = min(p.K, kbeg + kchunk);
       const bool empty_k = kend <= kbeg;          // a trailing split with no K range: partial sum is zero
       const uint32_t ab = lt & 1, aph = (lt >> 1) & 1;
-      if (p.epi.bias && active) {   // fetch this warp's 64 bias values now; the latency hides behind the MMAs
+      if (p.epi.bias && active) {   // fetch this warp's bias slice now; the latency hides behind the MMAs
         __syncwarp();
-        for (int j = lane; j < 64; j += 32) {
+        for (int j = lane; j < CPW; j += 32) {
           const int n = n0 + cbeg + j;
           bias_s[j] = n < p.N ? __ldg(p.epi.bias + n) : 0.f;
         }
@@ -450,7 +477,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const bool via_tma = pre_pass ? true : (p.tma_c != 0);
           const bool f32 = !pre_pass && out_f32;
 #pragma unroll 1
-          for (int cc = 0; cc < 64; cc += 32) {
+          for (int cc = 0; cc < CPW; cc += 32) {
             const int c0 = cbeg + cc;
             if (n0 + c0 >= p.N) break;  // warp-uniform
             uint32_t r[32];
@@ -460,7 +487,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
               for (int j = 0; j < 32; j++) r[j] = 0u;
             }
-            if (via_tma && (f32 || cc == 0)) {       // the staging buffer is about to be overwritten
+            if (via_tma && (f32 || (cc & 63) == 0)) { // the staging buffer is about to be overwritten
               if (lane == 0 && store_pending) { tma_store_wait_read(); store_pending = false; }
               __syncwarp();
             }
@@ -485,18 +512,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const uint32_t s0 = my_row + (((2 * g8) ^ (lane & 7)) << 4), s1 = my_row + (((2 * g8 + 1) ^ (lane & 7)) << 4);
                 st_shared_v4(s0, __float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]));
                 st_shared_v4(s1, __float_as_uint(v[4]), __float_as_uint(v[5]), __float_as_uint(v[6]), __float_as_uint(v[7]));
-              } else {                               // 64 bf16 per row: piece cc/8 + g8
-                const uint32_t s0 = my_row + ((((cc >> 3) + g8) ^ (lane & 7)) << 4);
+              } else {                               // 64 bf16 per row: piece (cc mod 64)/8 + g8
+                const uint32_t s0 = my_row + (((((cc & 63) >> 3) + g8) ^ (lane & 7)) << 4);
                 st_shared_v4(s0, pack2(v[0], v[1]), pack2(v[2], v[3]), pack2(v[4], v[5]), pack2(v[6], v[7]));
               }
             }
-            const bool last_chunk = cc == 32 || n0 + c0 + 32 >= p.N;
+            const bool last_chunk = (cc & 63) == 32 || n0 + c0 + 32 >= p.N;
             if (via_tma && (f32 || last_chunk)) {
               asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
               __syncwarp();
               if (dbg && lt == 0 && threadIdx.x == 64 && p.dbg[10] == 0) p.dbg[10] = clock64();
               if (lane == 0 && !(dflags & 1)) {
-                const int x = f32 ? n0 + c0 : n0 + cbeg, y = m0 + q * 32;
+                const int x = f32 ? n0 + c0 : n0 + cbeg + (cc & ~63), y = m0 + q * 32;
                 if (pre_pass) tma_store_2d(&map_p, stage, x, y);
                 else if (p.splits > 1) tma_store_3d(&map_c, stage, x, y, split);
                 else tma_store_2d(&map_c, stage, x, y);
@@ -577,7 +604,8 @@ bool encode_2d(void* out, const void* base, long long inner, long long outer, lo
 
 template <int BN, bool A_MN, bool B_MN, bool GENERAL>
 cudaError_t launch_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas) {
-  constexpr size_t smem = (size_t)STAGES * (BM * BK * 2 + BN * BK * 2) + EPI_WARPS * (EPI_STAGE_BYTES + 256) + 8 * (2 * STAGES + 6) + 1024;
+  constexpr int STAGES = stages_for(BN);
+  constexpr size_t smem = (size_t)STAGES * (BM * BK * 2 + BN * BK * 2) + EPI_WARPS * (EPI_STAGE_BYTES + EPI_BIAS_BYTES) + 8 * (2 * STAGES + 6) + 1024;
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<BN, A_MN, B_MN, GENERAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -645,7 +673,10 @@ bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan) {
   if (!tc_gemm_supported(g)) return false;
   plan->a_mn = g.sa_k != 1;
   plan->b_mn = g.sb_k != 1;
-  plan->bn = g.N <= 64 ? 64 : 128;
+  // tile width: 256 halves the A-operand traffic per FLOP, taken when it still leaves every SM a tile
+  const long long tiles256 = (long long)((g.M + BM - 1) / BM) * ((g.N + 255) / 256) * g.splits;
+  plan->bn = g.N <= 64 ? 64 : (g.N >= 256 && tiles256 >= 148 ? 256 : 128);
+  if (getenv("ERASE_TC_BN")) { int f = atoi(getenv("ERASE_TC_BN")); if ((f == 64 || f == 128 || f == 256) && f <= (g.N + 63) / 64 * 64) plan->bn = f; }
   plan->status = status;
   plan->launches = 1;
   bool ok;
@@ -685,8 +716,12 @@ bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan) {
 }
 
 cudaError_t tc_gemm_launch(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas) {
-  if (epilogue_is_simple(g)) return plan.bn == 64 ? launch_bn<64, false>(g, plan, s, max_ctas) : launch_bn<128, false>(g, plan, s, max_ctas);
-  return plan.bn == 64 ? launch_bn<64, true>(g, plan, s, max_ctas) : launch_bn<128, true>(g, plan, s, max_ctas);
+  const bool simple = epilogue_is_simple(g);
+  switch (plan.bn) {
+    case 64: return simple ? launch_bn<64, false>(g, plan, s, max_ctas) : launch_bn<64, true>(g, plan, s, max_ctas);
+    case 256: return simple ? launch_bn<256, false>(g, plan, s, max_ctas) : launch_bn<256, true>(g, plan, s, max_ctas);
+    default: return simple ? launch_bn<128, false>(g, plan, s, max_ctas) : launch_bn<128, true>(g, plan, s, max_ctas);
+  }
 }
 
 }  // namespace erase
