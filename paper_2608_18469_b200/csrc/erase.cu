@@ -330,7 +330,9 @@ struct Builder {
     const long long ldo = g.ldc;
     if (g.splits > 1) g.ws = f32_buf((size_t)g.splits * g.M * g.N);
     TcPlan plan;
+    int* sched = tc_ok ? (int*)dev_alloc(m, 2 * sizeof(int), &ok) : nullptr;   // dynamic tile scheduler words (zeroed)
     const bool use_tc = tc_ok && !m->dry && tc_gemm_plan(g, m->status, &plan);
+    plan.sched = sched;
     if (use_tc) {
       if (g.splits > 1)
         ops.push_back({[g, plan, out, ldo, mm = m](cudaStream_t s) {
@@ -1178,14 +1180,15 @@ erase_status erase_gemm(int32_t dtype, int32_t M, int32_t N, int32_t K, const vo
     return ERASE_ECUDA;
   };
   if (splits > 1 && cudaMalloc(&ws, (size_t)splits * M * N * sizeof(float)) != cudaSuccess) { cleanup(); g_create_error = "erase_gemm: workspace allocation failed"; return ERASE_ENOMEM; }
-  if (cudaMalloc(&status, sizeof(int)) != cudaSuccess) { cleanup(); g_create_error = "erase_gemm: allocation failed"; return ERASE_ENOMEM; }
-  cudaError_t e = cudaMemsetAsync(status, 0, sizeof(int), st);
+  if (cudaMalloc(&status, 4 * sizeof(int)) != cudaSuccess) { cleanup(); g_create_error = "erase_gemm: allocation failed"; return ERASE_ENOMEM; }
+  cudaError_t e = cudaMemsetAsync(status, 0, 4 * sizeof(int), st);   // status word + two scheduler words
   if (e != cudaSuccess) return cuda_fail(e, "memset");
   g.ws = ws;
   long long* dbg = nullptr;
   if (engine == 1) {
     TcPlan plan;
     if (!tc_gemm_plan(g, status, &plan)) { cleanup(); g_create_error = "erase_gemm: TMA descriptor encoding failed"; return ERASE_EUNSUPPORTED; }
+    plan.sched = status + 1;
     if (getenv("ERASE_TC_TIMELINE")) {   // development aid: print CTA 0's clock stamps for its first tile
       if (cudaMalloc(&dbg, 16 * sizeof(long long)) == cudaSuccess) {
         long long h[16] = {0};

@@ -19,7 +19,7 @@ using namespace erase;
 namespace {
 
 // Scratch shared by every call on a device: [0, ERASE_STATIC_WS_FLOATS) split-K partial sums,
-// then one status word.  Held by every device that loads the library until the process exits.
+// then one status word and two tile-scheduler words.  Held by every device that loads the library until the process exits.
 constexpr size_t kWsFloats = ERASE_STATIC_WS_FLOATS;
 static __device__ __align__(256) float g_static_scratch[kWsFloats + 64];
 
@@ -84,11 +84,12 @@ ERASE_API erase_status erase_gemm_static(int32_t dtype, int32_t M, int32_t N, in
 
   // The array keeps the previous call's contents.  The partial sums need no clearing (every
   // element that is read was written by this call); the status word must start at zero.
-  e = cudaMemsetAsync(status, 0, sizeof(int), st);
+  e = cudaMemsetAsync(status, 0, 4 * sizeof(int), st);   // status word and the two tile-scheduler words after it
   if (e != cudaSuccess) return fail(ERASE_ECUDA, std::string("status clear: ") + cudaGetErrorString(e));
   if (engine == 1) {
     TcPlan plan;
     if (!tc_gemm_plan(g, status, &plan)) return fail(ERASE_EUNSUPPORTED, "TMA descriptor encoding failed");
+    plan.sched = status + 1;
     e = tc_gemm_launch(g, plan, st);
   } else {
     e = gemm_simt(g, bf, st);

@@ -48,6 +48,7 @@ struct TcArgs {
   int tma_c;       // C (or the split-K partials) leaves through shared memory + TMA store
   int tma_p;       // so does the pre-activation copy
   int plain;       // 1: the epilogue is the identity; 2: bias add only; 0: general
+  int* sched;      // {next tile counter, finished CTAs}, zero between launches; null = static round-robin
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -304,9 +305,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+  // tile queue: the producer publishes the tiles this CTA works on (dynamic scheduling) to the MMA
+  // and epilogue warps through a 4-entry ring
+  auto tq_full = [&](int i) { return bar_base + 8u * (2 * STAGES + 6 + i); };
+  auto tq_empty = [&](int i) { return bar_base + 8u * (2 * STAGES + 10 + i); };
   uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
   volatile uint32_t* tmem_slot_ptr =
       reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * (EPI_STAGE_BYTES + EPI_BIAS_BYTES) + 8u * (2 * STAGES + 4));
+  volatile int* tile_ring =
+      reinterpret_cast<volatile int*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * (EPI_STAGE_BYTES + EPI_BIAS_BYTES) + 8u * (2 * STAGES + 14));
   const uint32_t tmem_slot = bar_base + 8u * (2 * STAGES + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -331,6 +338,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       mbar_init(tfull_bar(a), 1);
       mbar_init(tempty_bar(a), EPI_WARPS);
     }
+    for (int i = 0; i < 4; i++) {
+      mbar_init(tq_full(i), 1);
+      mbar_init(tq_empty(i), 1 + EPI_WARPS);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -347,9 +358,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
-      uint32_t it = 0;
+      uint32_t it = 0, slot = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
+      int t = (int)blockIdx.x < total ? (int)blockIdx.x : -1;
+      while (ok) {
+        // publish the tile (or the end marker -1) to the other roles
+        if (!mbar_wait(tq_empty(slot & 3), ((slot >> 2) & 1) ^ 1)) { atomicExch(p.status, 5); ok = false; break; }
+        tile_ring[slot & 3] = t;
+        mbar_arrive(tq_full(slot & 3));
+        slot++;
+        if (t < 0) break;
+        // claim the next tile now: the atomic's latency hides behind this tile's loads
+        int next = p.sched ? (int)gridDim.x + atomicAdd(p.sched, 1) : t + (int)gridDim.x;
         int mt, nt, split;
         tile_coords(t, tiles_m, tiles_n, mt, nt, split);
         const int m0 = mt * BM, n0 = nt * BN;
@@ -378,6 +398,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (dbg && it == 0) p.dbg[2] = clock64();
           if (dbg && it == 3) p.dbg[8] = clock64();
         }
+        t = next < total ? next : -1;
       }
       if (!ok) {  // give copies already in flight time to land before the CTA's shared memory is released
         const long long t0 = clock64();
@@ -392,7 +413,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                              ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
       uint32_t it = 0, lt = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < total && ok; t += gridDim.x, lt++) {
+      for (;; lt++) {
+        if (!mbar_wait(tq_full(lt & 3), (lt >> 2) & 1)) { atomicExch(p.status, 6); break; }
+        const int t = tile_ring[lt & 3];
+        mbar_arrive(tq_empty(lt & 3));
+        if (t < 0 || !ok) break;
         const int split = t / (tiles_m * tiles_n);
         const int kbeg = split * kchunk, kend = min(p.K, kbeg + kchunk);
         const int num_kb = kend > kbeg ? (kend - kbeg + BK - 1) / BK : 0;
@@ -446,7 +471,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const bool out_f32 = p.splits > 1 || p.c_f32;
     bool store_pending = false;                   // lane 0: a TMA store may still be reading the staging buffer
     uint32_t lt = 0;
-    for (int t = blockIdx.x; t < total; t += gridDim.x, lt++) {
+    for (;; lt++) {
+      int t = -1;
+      if (lane == 0) {
+        if (mbar_wait(tq_full(lt & 3), (lt >> 2) & 1)) {
+          t = tile_ring[lt & 3];
+          mbar_arrive(tq_empty(lt & 3));
+        } else {
+          atomicExch(p.status, 7);
+        }
+      }
+      t = __shfl_sync(0xffffffffu, t, 0);
+      if (t < 0) break;
       int mt, nt, split;
       tile_coords(t, tiles_m, tiles_n, mt, nt, split);
       const int m0 = mt * BM, n0 = nt * BN;
@@ -552,6 +588,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
+  if (p.sched && threadIdx.x == 0) {   // the CTA that finishes last leaves the scheduler words at zero
+    __threadfence();
+    if (atomicAdd(p.sched + 1, 1) == (int)gridDim.x - 1) {
+      p.sched[0] = 0;
+      p.sched[1] = 0;
+      __threadfence();
+    }
+  }
   if (dbg && threadIdx.x == 0) p.dbg[7] = clock64();
 }
 
@@ -605,7 +649,7 @@ bool encode_2d(void* out, const void* base, long long inner, long long outer, lo
 template <int BN, bool A_MN, bool B_MN, bool GENERAL>
 cudaError_t launch_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas) {
   constexpr int STAGES = stages_for(BN);
-  constexpr size_t smem = (size_t)STAGES * (BM * BK * 2 + BN * BK * 2) + EPI_WARPS * (EPI_STAGE_BYTES + EPI_BIAS_BYTES) + 8 * (2 * STAGES + 6) + 1024;
+  constexpr size_t smem = (size_t)STAGES * (BM * BK * 2 + BN * BK * 2) + EPI_WARPS * (EPI_STAGE_BYTES + EPI_BIAS_BYTES) + 8 * (2 * STAGES + 16) + 1024;
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<BN, A_MN, B_MN, GENERAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -615,7 +659,7 @@ cudaError_t launch_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int 
   TcArgs p;
   p.M = g.M; p.N = g.N; p.K = g.K;
   p.C = g.C; p.ldc = g.ldc; p.c_f32 = g.c_f32;
-  p.splits = g.splits; p.ws = g.ws; p.epi = g.epi; p.status = plan.status; p.dbg = plan.dbg;
+  p.splits = g.splits; p.ws = g.ws; p.epi = g.epi; p.status = plan.status; p.dbg = plan.dbg; p.sched = plan.sched;
   static int num_sms = 0;
   if (num_sms == 0) {
     int dev = 0;
@@ -636,6 +680,7 @@ cudaError_t launch_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int 
   const Epilogue& e = g.epi;
   const bool no_aux = e.alpha == 1.f && e.act == ACT_NONE && !e.pre_out && !e.mul && !e.res && e.dact == ACT_NONE;
   p.plain = no_aux ? (e.bias ? (g.splits == 1 ? 2 : 1) : 1) : 0;   // 1: identity, 2: bias only, 0: general
+  if (total <= (long long)grid.x) p.sched = nullptr;   // one tile per CTA: nothing to balance
   tc_gemm_kernel<BN, A_MN, B_MN, GENERAL><<<grid, TC_THREADS, smem, s>>>(ma, mb, mc, mp, p);
   return cudaGetLastError();
 }

@@ -22,6 +22,7 @@ struct TcPlan {
   int b_mn = 0;
   int launches = 1;
   int* status = nullptr;  // device word set non-zero when a bounded wait expired
+  int* sched = nullptr;   // two zero-initialised device ints for dynamic tile scheduling (null: static order)
   long long* dbg = nullptr;  // optional device buffer (16 slots) for clock64 stamps of CTA 0, development aid
 };
 
