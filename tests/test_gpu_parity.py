@@ -78,6 +78,17 @@ def test_config2_small_lm_bf16_full_size():
     _gu().compare_teacher_forced(synth.config("C2"), steps=3, seed=0)
 
 
+def test_config2_in_the_benchmark_launch_configuration():
+    from paper_2608_18469_b200 import binding
+    spec = synth.config("C2")
+    _gu().compare_teacher_forced(spec, steps=2, seed=1, n_streams=len(spec["blocks"]) + 1,
+                                 flags=binding.GRAPH | binding.EARLY_HEAD)
+
+
+def test_config5_mid_point_w1024_b4096():
+    _gu().compare_teacher_forced(synth.config("C5", w=1024, batch=4096), steps=1, seed=0)
+
+
 def test_config3_ctr_bf16_full_size():
     _gu().compare_teacher_forced(synth.config("C3"), steps=2, seed=0)
 
