@@ -27,6 +27,11 @@ from paper_2608_18469_b200 import synth  # noqa: E402
 
 POOL = 8   # distinct pre-staged batches, cycled
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from ncu captures of the largest member
+# of each kernel class at C2 (the local head's GEMMs; profiles/tc_gemm_c2_head_fwd_dgrad_wgrad.md).
+# They sit below the algorithmic bytes where a 64 MiB operand or result is still L2-resident.
+NCU_DRAM_BYTES = {"C2": {"gemm_fwd": 16.1e6, "gemm_dgrad": 72.9e6, "gemm_wgrad": 73.5e6}}
+
 
 def unit_name(spec):
     return "tokens/s" if spec["input"] == "tokens" else "samples/s"
@@ -153,26 +158,17 @@ def run_gpu(args, spec, cfg_name):
     import torch
     from paper_2608_18469_b200 import binding
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    from paper_2608_18469_b200.replicas import Replicas
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    rep = Replicas(backend="nccl", device="cuda")
+    rank, world, dist = rep.rank, rep.world, rep.dist
 
     def barrier():
-        if dist is not None:
-            dist.barrier()
+        rep.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(v):
-        if dist is None:
-            return v
-        t = torch.tensor([v], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    max_over_ranks = rep.max_over_ranks
 
     nb = len(spec["blocks"])
     n_streams = args.n_streams if args.n_streams > 0 else nb + 1
@@ -281,11 +277,9 @@ def run_gpu(args, spec, cfg_name):
                     "frac": ach / peaks["hbm_gbs"]}
         roof["peak_source"] = peaks["source"] + (" (sustained bf16 GEMM)" if roof["bound"] == "tensor" else " (copy)")
         roof["avg_launch_ms"] = t["ms"] / max(t["launches"], 1)
-        tr = None
-        tp = os.path.join(ROOT, "profiles", "traffic.json")
-        if os.path.exists(tp):
-            tr = json.load(open(tp)).get(cfg_name, {}).get(top)
+        tr = NCU_DRAM_BYTES.get(cfg_name, {}).get(top)
         roof["traffic"] = tr
+        roof["traffic_note"] = "ncu DRAM bytes of the class's largest GEMM (local head), one launch" if tr else None
         roof["kernel_share"] = {k: round(v["ms"] / sum(x["ms"] for x in agg.values()), 4)
                                 for k, v in sorted(agg.items(), key=lambda kv: -kv[1]["ms"])[:8]}
 
@@ -309,7 +303,7 @@ def run_gpu(args, spec, cfg_name):
     clocks, e2e_ms, h2d, d2h, roof, cpu = r["clocks"], r["e2e_ms"], r["h2d"], r["d2h"], r["roof"], r["cpu"]
     if rank != 0:
         if dist is not None:
-            dist.destroy_process_group()
+            rep.close()
         return
     flops = synth.step_flops(spec)
     value = world * units * args.steps / (era_ms * 1e-3)
@@ -346,7 +340,7 @@ def run_gpu(args, spec, cfg_name):
     }
     print(json.dumps(line), flush=True)
     if dist is not None:
-        dist.destroy_process_group()
+        rep.close()
 
 
 def main():
