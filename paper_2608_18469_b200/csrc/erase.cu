@@ -355,6 +355,20 @@ struct Builder {
     }
   }
 
+  // GELU is NOT fused into the GEMM epilogues: its erf/exp chain on the few epilogue warps made
+  // those GEMMs 2-3x slower than the GEMM plus a separate, fully occupied elementwise pass
+  // (which moves 4-6 bytes per element at HBM speed).  ReLU (a compare) stays fused.
+  void act_op(OpList& ops, const void* u, void* y, int act, long long n) {
+    bool bf = m->bf16;
+    ops.push_back({[=](cudaStream_t s) { return ew_act(u, y, act, n, bf, s); }, 1});
+    note(ops, "ew_act", 10.0 * n, 2.0 * n * m->esz);
+  }
+  void dact_op(OpList& ops, void* d, const void* src, int act, long long n) {
+    bool bf = m->bf16;
+    ops.push_back({[=](cudaStream_t s) { return ew_dact(d, src, act, n, bf, s); }, 1});
+    note(ops, "ew_dact", 10.0 * n, 3.0 * n * m->esz);
+  }
+
   // Y[M,N] = epi(X[M,K] W[N,K]^T)
   void lin_fwd(OpList& ops, const void* X, long long ldx, int widx, int bidx, void* Y, int M, int N, int K, Epilogue e) {
     GemmArgs g;
@@ -498,14 +512,16 @@ struct Builder {
       int a = use ? k.act : ACT_NONE;
       void* y = act_buf((size_t)m->rows * N);
       Epilogue e;
-      e.act = a;
       const void* src = y;
       if (a == ACT_GELU) {
         void* u = act_buf((size_t)m->rows * N);
-        e.pre_out = u;
+        lin_fwd(f, h, ldh, first_tensor + 2 * i, first_tensor + 2 * i + 1, u, m->rows, N, K, e);
+        act_op(f, u, y, a, (long long)m->rows * N);
         src = u;
+      } else {
+        e.act = a;
+        lin_fwd(f, h, ldh, first_tensor + 2 * i, first_tensor + 2 * i + 1, y, m->rows, N, K, e);
       }
-      lin_fwd(f, h, ldh, first_tensor + 2 * i, first_tensor + 2 * i + 1, y, m->rows, N, K, e);
       st.in.push_back(h);
       st.src.push_back(src);
       st.act.push_back(a);
@@ -527,11 +543,13 @@ struct Builder {
       if (i > 0 || need_dx) {
         void* dx = act_buf((size_t)m->rows * K);
         Epilogue e;
-        if (i > 0 && st.act[i - 1] != ACT_NONE) {
-          e.dact = st.act[i - 1];
+        const int da = i > 0 ? st.act[i - 1] : ACT_NONE;
+        if (da == ACT_RELU) {
+          e.dact = da;
           e.dact_src = st.src[i - 1];
         }
         lin_dgrad(bw, d, first_tensor + 2 * i, dx, m->rows, N, K, e);
+        if (da == ACT_GELU) dact_op(bw, dx, st.src[i - 1], da, (long long)m->rows * K);
         d = dx;
       }
     }
@@ -582,8 +600,8 @@ struct Builder {
       const float* g2 = Wf(t(LN2G)); const float* b2 = Wf(t(LN2B));
       f.push_back({[=](cudaStream_t s) { return layernorm_fwd(h, g2, b2, mm2, mean2, rstd2, rows, d, bf, s); }, 1});
       note(f, "layernorm_fwd", 8.0 * rows * d, 2.0 * rows * d * m->esz);
-      Epilogue e2; e2.act = ACT_GELU; e2.pre_out = u;
-      lin_fwd(f, mm2, d, t(W1), t(B1), g, rows, ff, d, e2);
+      lin_fwd(f, mm2, d, t(W1), t(B1), u, rows, ff, d, Epilogue());
+      act_op(f, u, g, ACT_GELU, (long long)rows * ff);
       Epilogue e3; e3.res = h;
       lin_fwd(f, g, ff, t(W2), t(B2), zout, rows, d, ff, e3);
     }
@@ -599,8 +617,8 @@ struct Builder {
     void* da = act_buf((size_t)rows * d);
     {
       lin_wgrad(bw, dz, g, ff, t(W2), t(B2), rows, d, ff);
-      Epilogue e; e.dact = ACT_GELU; e.dact_src = u;
-      lin_dgrad(bw, dz, t(W2), du, rows, d, ff, e);
+      lin_dgrad(bw, dz, t(W2), du, rows, d, ff, Epilogue());
+      dact_op(bw, du, u, ACT_GELU, (long long)rows * ff);
       lin_wgrad(bw, du, mm2, d, t(W1), t(B1), rows, ff, d);
       lin_dgrad(bw, du, t(W1), dm, rows, ff, d, Epilogue());
       ln_bwd(bw, dm, h, mean2, rstd2, t(LN2G), t(LN2B), dz, dhb, d);

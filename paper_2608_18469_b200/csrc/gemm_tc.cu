@@ -32,7 +32,7 @@ __host__ __device__ constexpr int stages_for(int bn) { return bn == 256 ? 3 : 4;
 constexpr uint32_t EPI_BIAS_BYTES = 512;              // up to 128 bias floats per epilogue warp
 constexpr int EPI_WARPS = 8;                       // two per TMEM lane quarter, each takes half the columns
 constexpr int TC_THREADS = 32 * (2 + EPI_WARPS);
-constexpr uint32_t EPI_STAGE_BYTES = 4096;             // 32 rows x 128 bytes per epilogue warp
+constexpr uint32_t EPI_STAGE_BYTES = 8192;             // two buffers of 32 rows x 128 bytes per epilogue warp
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;  // ~2 s at 2 GHz
 
 struct TcArgs {
@@ -128,18 +128,37 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
 
 __device__ __forceinline__ float bf2f(uint32_t bits16) { return __uint_as_float(bits16 << 16); }
 
-// out of line: keeps the erff/expf expansions out of the unrolled epilogue (instruction-cache footprint)
-__device__ __noinline__ float act_apply_d(int act, float v) {
+// Phi(u) and phi(u) of the standard normal for the exact-erf GELU, with erf from the
+// Abramowitz-Stegun 7.1.26 rational form (|error| <= 1.5e-7, far below bf16 resolution): one
+// reciprocal, one exp2 and a 5-term polynomial, shared by the value and the derivative.  Short
+// enough to stay inline in the epilogue (erff's expansion was not).
+__device__ __forceinline__ void normal_cdf_pdf(float u, float& cdf, float& pdf) {
+  const float x = fabsf(u) * 0.70710678118654752f;
+  const float t = __frcp_rn(fmaf(0.3275911f, x, 1.f));
+  const float e = exp2f(-1.4426950408889634f * x * x);          // exp(-u^2/2)
+  float poly = fmaf(1.061405429f, t, -1.453152027f);
+  poly = fmaf(poly, t, 1.421413741f);
+  poly = fmaf(poly, t, -0.284496736f);
+  poly = fmaf(poly, t, 0.254829592f);
+  const float half_erfc = 0.5f * poly * t * e;                   // 0.5*(1 - erf(x)), x >= 0
+  cdf = u >= 0.f ? 1.f - half_erfc : half_erfc;
+  pdf = 0.39894228040143268f * e;
+}
+__device__ __forceinline__ float act_apply_d(int act, float v) {
   if (act == ACT_RELU) return v > 0.f ? v : 0.f;
-  if (act == ACT_GELU) return v * 0.5f * (1.f + erff(v * 0.70710678118654752f));
+  if (act == ACT_GELU) {
+    float cdf, pdf;
+    normal_cdf_pdf(v, cdf, pdf);
+    return v * cdf;
+  }
   return v;
 }
-__device__ __noinline__ float act_deriv_d(int act, float u) {
+__device__ __forceinline__ float act_deriv_d(int act, float u) {
   if (act == ACT_RELU) return u > 0.f ? 1.f : 0.f;
   if (act == ACT_GELU) {
-    float cdf = 0.5f * (1.f + erff(u * 0.70710678118654752f));
-    float pdf = 0.39894228040143268f * expf(-0.5f * u * u);
-    return cdf + u * pdf;
+    float cdf, pdf;
+    normal_cdf_pdf(u, cdf, pdf);
+    return fmaf(u, pdf, cdf);
   }
   return 1.f;
 }
@@ -263,7 +282,8 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t sr
                ::"l"(map), "r"(x), "r"(y), "r"(z), "r"(src) : "memory");
 }
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// all but the most recent store of this thread have finished reading their shared-memory source
+__device__ __forceinline__ void tma_store_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 
 // Tile order: splits outermost; inside a split, bands of 8 column tiles, and inside a band m
 // outer / n inner.  The ~148 tiles in flight at any time then cover about 18 row tiles x 8
@@ -465,11 +485,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int q = warp & 3;                       // TMEM lane quarter this warp may read
     const int cbeg = (ew / 4) * CPW;              // first tile column of this warp
     const bool active = cbeg < BN;                // BN = 64: only one warp per quarter has columns
-    const uint32_t stage = epi_base + ew * EPI_STAGE_BYTES;
-    const uint32_t my_row = stage + lane * 128;
+    const uint32_t stage0 = epi_base + ew * EPI_STAGE_BYTES;   // two 4 KB buffers, used alternately
+    uint32_t sbuf = 0;
     float* bias_s = reinterpret_cast<float*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * EPI_STAGE_BYTES + ew * EPI_BIAS_BYTES);
     const bool out_f32 = p.splits > 1 || p.c_f32;
-    bool store_pending = false;                   // lane 0: a TMA store may still be reading the staging buffer
+    bool store_pending = false;                   // lane 0: TMA stores may still be reading the staging buffers
     uint32_t lt = 0;
     for (;; lt++) {
       int t = -1;
@@ -523,10 +543,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
               for (int j = 0; j < 32; j++) r[j] = 0u;
             }
-            if (via_tma && (f32 || (cc & 63) == 0)) { // the staging buffer is about to be overwritten
-              if (lane == 0 && store_pending) { tma_store_wait_read(); store_pending = false; }
+            if (via_tma && (f32 || (cc & 63) == 0)) { // next staging buffer: its previous store (two stores ago) must have read it
+              sbuf ^= 1;
+              if (lane == 0 && store_pending) tma_store_wait_read1();
               __syncwarp();
             }
+            const uint32_t stage = stage0 + sbuf * 4096;
+            const uint32_t my_row = stage + lane * 128;
 #pragma unroll
             for (int g8 = 0; g8 < 4; g8++) {
               const int n = n0 + c0 + g8 * 8;

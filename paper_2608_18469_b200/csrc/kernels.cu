@@ -845,16 +845,20 @@ __global__ void __launch_bounds__(THREADS) softmax_ce_reg_kernel(bf16_t* __restr
 #pragma unroll
   for (int k = 0; k < VPT; k++)
 #pragma unroll
-    for (int j = 0; j < 8; j++) se += exp2f((x[k][j] - mx) * L2E);
+    for (int j = 0; j < 8; j++) {
+      x[k][j] = exp2f((x[k][j] - mx) * L2E);     // keep exp(x - max): the probabilities are this over the sum
+      se += x[k][j];
+    }
   se = block_reduce(se, false);
   const float lse = mx + logf(se);
+  const float inv_se = 1.f / se;
 #pragma unroll
   for (int k = 0; k < VPT; k++) {
     const int i = threadIdx.x + k * THREADS;
     if (i < nvec) {
       float g[8];
 #pragma unroll
-      for (int j = 0; j < 8; j++) g[j] = (exp2f((x[k][j] - lse) * L2E) - (i * 8 + j == tgt ? 1.f : 0.f)) * inv_rows;
+      for (int j = 0; j < 8; j++) g[j] = (x[k][j] * inv_se - (i * 8 + j == tgt ? 1.f : 0.f)) * inv_rows;
       uint4 q;
       __nv_bfloat162 h;
       h = __floats2bfloat162_rn(g[0], g[1]); q.x = *reinterpret_cast<uint32_t*>(&h);
@@ -950,25 +954,60 @@ cudaError_t bce_head_dz(const float* ds, const float* w, void* dz, int dact, con
 // ------------------------------------------------------------------------------------------
 // elementwise
 // ------------------------------------------------------------------------------------------
+// One 16-byte vector per thread and step (8 bf16 or 4 floats); the element tail is scalar.
+// mode 0: out = a * b      mode 1: out = act(a)      mode 2: out = a * act'(b)
 template <typename T>
-__global__ void ew_mul_kernel(const T* a, const T* b, T* out, long long n) {
-  long long i = (long long)blockIdx.x * 256 + threadIdx.x;
-  if (i < n) stf(out + i, ldf(a + i) * ldf(b + i));
+__global__ void __launch_bounds__(256) ew_kernel(const T* a, const T* __restrict__ b, T* out,   // a may alias out
+                                                 long long n, int mode, int act) {
+  constexpr int VEC = VecOf<T>::N;
+  const long long nvec = n / VEC;
+  const long long stride = (long long)gridDim.x * 256;
+  for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < nvec; i += stride) {
+    float x[VEC], y[VEC];
+    ld_vec<T>(a + i * VEC, x);
+    if (mode != 1) ld_vec<T>(b + i * VEC, y);
+#pragma unroll
+    for (int j = 0; j < VEC; j++)
+      x[j] = mode == 0 ? x[j] * y[j] : (mode == 1 ? act_apply(act, x[j]) : x[j] * act_deriv(act, y[j]));
+    if (VEC == 8) {
+      uint4 q;
+      __nv_bfloat162 h;
+      h = __floats2bfloat162_rn(x[0], x[1]); q.x = *reinterpret_cast<uint32_t*>(&h);
+      h = __floats2bfloat162_rn(x[2], x[3]); q.y = *reinterpret_cast<uint32_t*>(&h);
+      h = __floats2bfloat162_rn(x[4 % VEC], x[5 % VEC]); q.z = *reinterpret_cast<uint32_t*>(&h);
+      h = __floats2bfloat162_rn(x[6 % VEC], x[7 % VEC]); q.w = *reinterpret_cast<uint32_t*>(&h);
+      *reinterpret_cast<uint4*>(out + i * VEC) = q;
+    } else {
+      *reinterpret_cast<float4*>(out + i * VEC) = make_float4(x[0], x[1], x[2], x[3]);
+    }
+  }
+  if (blockIdx.x == 0)
+    for (long long i = nvec * VEC + threadIdx.x; i < n; i += 256) {
+      const float xa = ldf(a + i);
+      stf(out + i, mode == 0 ? xa * ldf(b + i) : (mode == 1 ? act_apply(act, xa) : xa * act_deriv(act, ldf(b + i))));
+    }
+}
+
+static cudaError_t ew_launch(const void* a, const void* b, void* out, long long n, int mode, int act, bool bf16, cudaStream_t s) {
+  if (n <= 0) return cudaSuccess;
+  const bool aligned = ((reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b) | reinterpret_cast<uintptr_t>(out)) & 15) == 0;
+  if (!aligned) return cudaErrorMisalignedAddress;   // every buffer of the library is 256-byte aligned
+  const long long nvec = n / (bf16 ? 8 : 4);
+  long long blocks = (nvec + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  if (bf16) ew_kernel<bf16_t><<<(unsigned)blocks, 256, 0, s>>>((const bf16_t*)a, (const bf16_t*)b, (bf16_t*)out, n, mode, act);
+  else ew_kernel<float><<<(unsigned)blocks, 256, 0, s>>>((const float*)a, (const float*)b, (float*)out, n, mode, act);
+  return cudaGetLastError();
 }
 cudaError_t ew_mul(const void* a, const void* b, void* out, long long n, bool bf16, cudaStream_t s) {
-  if (bf16) ew_mul_kernel<bf16_t><<<cdiv(n, 256), 256, 0, s>>>((const bf16_t*)a, (const bf16_t*)b, (bf16_t*)out, n);
-  else ew_mul_kernel<float><<<cdiv(n, 256), 256, 0, s>>>((const float*)a, (const float*)b, (float*)out, n);
-  return cudaGetLastError();
+  return ew_launch(a, b, out, n, 0, ACT_NONE, bf16, s);
 }
-template <typename T>
-__global__ void ew_dact_kernel(T* d, const T* src, int act, long long n) {
-  long long i = (long long)blockIdx.x * 256 + threadIdx.x;
-  if (i < n) stf(d + i, ldf(d + i) * act_deriv(act, ldf(src + i)));
+cudaError_t ew_act(const void* u, void* out, int act, long long n, bool bf16, cudaStream_t s) {
+  return ew_launch(u, nullptr, out, n, 1, act, bf16, s);
 }
 cudaError_t ew_dact(void* d, const void* src, int act, long long n, bool bf16, cudaStream_t s) {
-  if (bf16) ew_dact_kernel<bf16_t><<<cdiv(n, 256), 256, 0, s>>>((bf16_t*)d, (const bf16_t*)src, act, n);
-  else ew_dact_kernel<float><<<cdiv(n, 256), 256, 0, s>>>((float*)d, (const float*)src, act, n);
-  return cudaGetLastError();
+  return ew_launch(d, src, d, n, 2, act, bf16, s);
 }
 
 // ------------------------------------------------------------------------------------------

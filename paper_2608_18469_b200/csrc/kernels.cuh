@@ -106,6 +106,8 @@ cudaError_t bce_head_dz(const float* ds, const float* w, void* dz, int dact, con
 
 // out = a (.) b, all [n] of T
 cudaError_t ew_mul(const void* a, const void* b, void* out, long long n, bool bf16, cudaStream_t s);
+// out = act(u)
+cudaError_t ew_act(const void* u, void* out, int act, long long n, bool bf16, cudaStream_t s);
 // d <- d * act'(src)
 cudaError_t ew_dact(void* d, const void* src, int act, long long n, bool bf16, cudaStream_t s);
 
