@@ -173,7 +173,7 @@ def run_gpu(args, spec, cfg_name):
     nb = len(spec["blocks"])
     n_streams = args.n_streams if args.n_streams > 0 else nb + 1
     flags = 0 if args.no_graph else binding.GRAPH
-    eflags = flags | (0 if args.loss_on_main else binding.EARLY_HEAD)
+    eflags = flags | (0 if args.loss_on_main else (binding.EARLY_HEAD | binding.BLOCK_OPT))
     units = units_per_step(spec)
 
     model = binding.Model(spec)
@@ -316,7 +316,7 @@ def run_gpu(args, spec, cfg_name):
         "ms_per_step": era_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": spec["dtype"], "data": "synthetic",
         "config": {"workload": workload_name(cfg_name, spec), "n_streams": n_streams,
-                   "schedule": "ERASE, local head+loss+backward released onto side streams after the block body"
+                   "schedule": "ERASE, local head+loss+backward+optimizer of each block released onto side streams after the block body"
                                if not args.loss_on_main else "ERASE, backward released after forward and local loss",
                    "cuda_graph": not args.no_graph, "batch_pool": POOL,
                    "l2": f"no flush: the step's working set ({arena_mb:.0f} MiB of stashes, logits, parameters) exceeds the 126 MB L2",

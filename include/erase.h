@@ -135,6 +135,12 @@ typedef struct {
                             Same kernels, same bits.  Without the flag the head and loss run on the
                             main stream before the release, as the paper schedules them.          */
 
+#define ERASE_BLOCK_OPT 8u /* ERASE schedules only: update theta_b on block b's side stream right after
+                            B_b instead of in one sweep after every backward has finished.  theta_b is
+                            read by F_b and B_b alone (Section 2.1: the gradient of block b is final
+                            once B_b ends), so the optimizer's serial tail disappears under the other
+                            blocks' work.  Same update kernel on the same values: same bits.          */
+
 /* Device bytes erase_create needs for this spec when given an arena; 0 if the spec is invalid. */
 ERASE_API size_t erase_arena_bytes(const erase_model_spec* spec);
 

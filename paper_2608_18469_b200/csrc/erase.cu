@@ -93,9 +93,11 @@ struct erase_model {
   bool timeline_valid = false;
 
   OpList stage, opt;
+  OpList opt_tick_op;            // advances the Adam step counter (per-block optimizer mode)
+  std::vector<OpList> opt_blk;   // the optimizer restricted to block b's slice of the parameter arena
   std::vector<OpList> fwd, hfwd, bwd;  // per block: body forward, local head + loss, backward
   erase_batch cur = {nullptr, nullptr, nullptr};
-  std::map<GraphKey, cudaGraphExec_t> graphs;
+  std::map<GraphKey, std::pair<cudaGraphExec_t, int64_t>> graphs;   // executable graph and the kernels it launches
 
   int sm_budget = 0;   // CTA cap for persistent GEMMs enqueued next (0 = all SMs); set per stream by the scheduler
   int64_t launches = 0;
@@ -778,6 +780,26 @@ struct Builder {
       note(m->opt, "opt_tick");
       m->opt.push_back({[=](cudaStream_t st) { return opt_update(th, gr, m1, m2, sh, n, kind, lr, b1, b2, eps, wd, tick, st); }, 1});
       note(m->opt, "opt_update", 10.0 * n, (double)n * (kind == ERASE_OPT_SGD ? 12 : 28) + (sh ? 2.0 * n : 0));
+      // per-block variant: the same update on block b's contiguous slice, runnable as soon as B_b is done
+      m->opt_tick_op.push_back({[=](cudaStream_t st) { return opt_tick(tick, b1, b2, st); }, 1});
+      note(m->opt_tick_op, "opt_tick");
+      m->opt_blk.resize(m->B);
+      for (int b = 0; b < m->B; b++) {
+        size_t lo = (size_t)-1, hi = 0;
+        for (const Tensor& t : m->tensors)
+          if (t.trainable && t.block == b) {
+            if (t.off < lo) lo = t.off;
+            size_t end = t.off + round_up(t.n, 64);
+            if (end > hi) hi = end;
+          }
+        if (hi <= lo) continue;
+        long long nb = (long long)(hi - lo);
+        float* thb = th + lo; float* grb = gr + lo;
+        float* m1b = m1 ? m1 + lo : nullptr; float* m2b = m2 ? m2 + lo : nullptr;
+        void* shb = sh ? (void*)((__nv_bfloat16*)sh + lo) : nullptr;
+        m->opt_blk[b].push_back({[=](cudaStream_t st) { return opt_update(thb, grb, m1b, m2b, shb, nb, kind, lr, b1, b2, eps, wd, tick, st); }, 1});
+        note(m->opt_blk[b], "opt_update", 10.0 * nb, (double)nb * (kind == ERASE_OPT_SGD ? 12 : 28) + (sh ? 2.0 * nb : 0));
+      }
     }
     return ok;
   }
@@ -824,6 +846,9 @@ erase_status enqueue_step(erase_model* m, int n_streams, unsigned flags, bool ti
   if (timed) CK(cudaEventRecord(tev(2 * (2 * B + 1)), m->main));
   CK(run_ops(m, m->stage, m->main));
   const bool early_head = (flags & ERASE_EARLY_HEAD) != 0;
+  // per-block optimizer: theta_b is read by F_b and B_b only, so it can be updated right behind B_b
+  const bool block_opt = do_opt && n_streams > 1 && (flags & ERASE_BLOCK_OPT) != 0;
+  if (block_opt) CK(run_ops(m, m->opt_tick_op, m->main));
   if (n_streams <= 1) {
     for (int b = 0; b < B; b++) {
       if (timed) CK(cudaEventRecord(tev(2 * b), m->main));
@@ -857,13 +882,14 @@ erase_status enqueue_step(erase_model* m, int n_streams, unsigned flags, bool ti
       if (early_head) CK(run_ops(m, m->hfwd[b], sd));    // z_b's only other consumer is F_{b+1}, which does not wait
       CK(run_ops(m, m->bwd[b], sd));
       if (timed) CK(cudaEventRecord(tev(2 * (B + b) + 1), sd));
+      if (block_opt) CK(run_ops(m, m->opt_blk[b], sd));
       CK(cudaEventRecord(m->ev_b[b], sd));
     }
     for (int b = 0; b < B; b++) CK(cudaStreamWaitEvent(m->main, m->ev_b[b], 0));  // join
     m->sm_budget = 0;
   }
   if (timed) CK(cudaEventRecord(tev(4 * B), m->main));
-  if (do_opt) CK(run_ops(m, m->opt, m->main));
+  if (do_opt && !block_opt) CK(run_ops(m, m->opt, m->main));
   if (timed) CK(cudaEventRecord(tev(4 * B + 1), m->main));
   return ERASE_OK;
 }
@@ -924,7 +950,7 @@ void erase_destroy(erase_model* m) {
   if (!m) return;
   if (m->main) cudaStreamSynchronize(m->main);
   for (auto s : m->side) if (s) cudaStreamSynchronize(s);
-  for (auto& kv : m->graphs) cudaGraphExecDestroy(kv.second);
+  for (auto& kv : m->graphs) cudaGraphExecDestroy(kv.second.first);
   for (auto e : m->ev_f) if (e) cudaEventDestroy(e);
   for (auto e : m->ev_b) if (e) cudaEventDestroy(e);
   for (auto e : m->ev_time) if (e) cudaEventDestroy(e);
@@ -1037,7 +1063,7 @@ static erase_status check_step_args(erase_model* m, const erase_batch* batch);
 erase_status erase_step_ex(erase_model* m, const erase_batch* batch, int32_t n_streams, uint32_t flags) {
   if (!m) return ERASE_EINVAL;
   if (n_streams < 1) return m->fail(ERASE_EINVAL, "erase_step: n_streams must be >= 1");
-  if (flags & ~(ERASE_GRAPH | ERASE_NO_OPT | ERASE_EARLY_HEAD)) return m->fail(ERASE_EINVAL, "erase_step: unknown flag");
+  if (flags & ~(ERASE_GRAPH | ERASE_NO_OPT | ERASE_EARLY_HEAD | ERASE_BLOCK_OPT)) return m->fail(ERASE_EINVAL, "erase_step: unknown flag");
   erase_status cst = check_step_args(m, batch);
   if (cst != ERASE_OK) return cst;
   if (n_streams > m->B + 1) n_streams = m->B + 1;
@@ -1051,6 +1077,7 @@ erase_status erase_step_ex(erase_model* m, const erase_batch* batch, int32_t n_s
       erase_status st = enqueue_step(m, n_streams, flags, false);
       cudaGraph_t graph = nullptr;
       cudaError_t e = cudaStreamEndCapture(m->main, &graph);
+      const int64_t captured = m->launches - before;
       m->launches = before;
       if (st != ERASE_OK) { if (graph) cudaGraphDestroy(graph); cudaGetLastError(); return st; }
       if (e != cudaSuccess) return m->fail(ERASE_ECUDA, std::string("graph capture: ") + cudaGetErrorString(e));
@@ -1058,18 +1085,10 @@ erase_status erase_step_ex(erase_model* m, const erase_batch* batch, int32_t n_s
       e = cudaGraphInstantiate(&exec, graph, 0);
       cudaGraphDestroy(graph);
       if (e != cudaSuccess) return m->fail(ERASE_ECUDA, std::string("graph instantiate: ") + cudaGetErrorString(e));
-      it = m->graphs.emplace(key, exec).first;
+      it = m->graphs.emplace(key, std::make_pair(exec, captured)).first;
     }
-    CK(cudaGraphLaunch(it->second, m->main));
-    int64_t per = 0;
-    for (auto& op : m->stage) per += op.launches;
-    for (int b = 0; b < m->B; b++) {
-      for (auto& op : m->fwd[b]) per += op.launches;
-      for (auto& op : m->hfwd[b]) per += op.launches;
-      for (auto& op : m->bwd[b]) per += op.launches;
-    }
-    if (!(flags & ERASE_NO_OPT)) for (auto& op : m->opt) per += op.launches;
-    m->launches += per;
+    CK(cudaGraphLaunch(it->second.first, m->main));
+    m->launches += it->second.second;
     m->timeline_valid = false;
   } else {
     erase_status st = enqueue_step(m, n_streams, flags, true);

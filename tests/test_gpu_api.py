@@ -144,7 +144,7 @@ def test_full_size_lm_configs_schedules_agree_and_losses_start_near_ln_vocab():
         flat = synth.init_params(spec, 0)
         batches = [gu.DevBatch(spec, synth.make_batch(spec, 0, index=i)) for i in range(steps)]
         serial = gu.run_steps(spec, flat, batches, n_streams=1)
-        bench_cfg = gu.run_steps(spec, flat, batches, n_streams=nb + 1, flags=binding.GRAPH | binding.EARLY_HEAD)
+        bench_cfg = gu.run_steps(spec, flat, batches, n_streams=nb + 1, flags=binding.GRAPH | binding.EARLY_HEAD | binding.BLOCK_OPT)
         for k in serial:
             if k != "launches":
                 assert serial[k].tobytes() == bench_cfg[k].tobytes(), (name, k)

@@ -82,7 +82,7 @@ def test_config2_in_the_benchmark_launch_configuration():
     from paper_2608_18469_b200 import binding
     spec = synth.config("C2")
     _gu().compare_teacher_forced(spec, steps=2, seed=1, n_streams=len(spec["blocks"]) + 1,
-                                 flags=binding.GRAPH | binding.EARLY_HEAD)
+                                 flags=binding.GRAPH | binding.EARLY_HEAD | binding.BLOCK_OPT)
 
 
 def test_config5_mid_point_w1024_b4096():
@@ -125,4 +125,7 @@ def test_erase_schedule_is_bit_identical_to_serial(name):
     _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=nb + 1, flags=binding.GRAPH))
     _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=nb + 1, flags=binding.EARLY_HEAD))
     _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=2, flags=binding.GRAPH | binding.EARLY_HEAD))
+    _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=nb + 1, flags=binding.BLOCK_OPT))
+    _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=nb + 1,
+                                     flags=binding.GRAPH | binding.EARLY_HEAD | binding.BLOCK_OPT))
     assert serial["launches"] > 0
