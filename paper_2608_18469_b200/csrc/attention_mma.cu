@@ -50,6 +50,20 @@ __device__ __forceinline__ void load_tile(bf16_t* dst, const bf16_t* src, long l
   }
 }
 
+// The same tile, fetched with cp.async (16 bytes per request, zero-filled past rows_valid) so that
+// the next tile streams in while the current one is being multiplied.  rows_valid >= 1.
+__device__ __forceinline__ void load_tile_async(bf16_t* dst, const bf16_t* src, long long ld, int rows_valid) {
+  for (int i = threadIdx.x; i < TS * (DH / 8); i += 128) {
+    const int r = i >> 3, c = (i & 7) * 8;
+    const int rs = r < rows_valid ? r : rows_valid - 1;
+    const uint32_t bytes = r < rows_valid ? 16u : 0u;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(s_u32(dst + r * LDS + c)),
+                 "l"(src + (long long)rs * ld + c), "r"(bytes) : "memory");
+  }
+}
+__device__ __forceinline__ void async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 // A fragments (16 rows x 64 k) of a row-major tile, rows row0..row0+15: a[kk][0..3]
 __device__ __forceinline__ void load_a_frags(const bf16_t* tile, int row0, uint32_t a[4][4]) {
   const int lane = threadIdx.x & 31;
@@ -113,18 +127,19 @@ __device__ __forceinline__ void zero_acc(float a[8][4]) {
 __global__ void __launch_bounds__(128) attn_fwd_mma(const bf16_t* __restrict__ qkv, bf16_t* __restrict__ o,
                                                     float* __restrict__ lse, int T, int H, float scale) {
   __shared__ __align__(16) bf16_t Qs[TS * LDS];
-  __shared__ __align__(16) bf16_t Ks[TS * LDS];
-  __shared__ __align__(16) bf16_t Vs[TS * LDS];
-  const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  __shared__ __align__(16) bf16_t KVs[2][2][TS * LDS];   // [buffer][K|V]: the next key tile loads while this one is used
+  const int qt = gridDim.x - 1 - blockIdx.x;             // heaviest (longest key loop) query tiles first
+  const int h = blockIdx.y, b = blockIdx.z;
   const int d = H * DH;
   const long long ld = 3LL * d;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t4 = lane & 3;
   const int q0 = qt * TS;
   const bf16_t* base = qkv + (long long)b * T * ld + h * DH;
-  load_tile(Qs, base + (long long)q0 * ld, ld, T - q0);
-  __syncthreads();
+  load_tile_async(Qs, base + (long long)q0 * ld, ld, T - q0);
+  load_tile_async(KVs[0][0], base + d, ld, T);
+  load_tile_async(KVs[0][1], base + 2 * d, ld, T);
+  async_commit();
   uint32_t qa[4][4];
-  load_a_frags(Qs, warp * 16, qa);
   float oacc[8][4];
   zero_acc(oacc);
   float mrow[2] = {-INFINITY, -INFINITY}, lrow[2] = {0.f, 0.f};
@@ -132,10 +147,18 @@ __global__ void __launch_bounds__(128) attn_fwd_mma(const bf16_t* __restrict__ q
   const int row_a = q0 + warp * 16 + g, row_b = row_a + 8;
   for (int jt = 0; jt <= qt; jt++) {
     const int j0 = jt * TS;
+    if (jt < qt) {
+      load_tile_async(KVs[(jt + 1) & 1][0], base + d + (long long)(j0 + TS) * ld, ld, T - j0 - TS);
+      load_tile_async(KVs[(jt + 1) & 1][1], base + 2 * d + (long long)(j0 + TS) * ld, ld, T - j0 - TS);
+      async_commit();
+      async_wait<1>();
+    } else {
+      async_wait<0>();
+    }
     __syncthreads();
-    load_tile(Ks, base + d + (long long)j0 * ld, ld, T - j0);
-    load_tile(Vs, base + 2 * d + (long long)j0 * ld, ld, T - j0);
-    __syncthreads();
+    if (jt == 0) load_a_frags(Qs, warp * 16, qa);
+    const bf16_t* Ks = KVs[jt & 1][0];
+    const bf16_t* Vs = KVs[jt & 1][1];
     float s[8][4];
     zero_acc(s);
     mma_a_xt(s, qa, Ks);
@@ -173,6 +196,7 @@ __global__ void __launch_bounds__(128) attn_fwd_mma(const bf16_t* __restrict__ q
       }
     }
     mma_p_x(oacc, s, Vs);
+    __syncthreads();   // every warp is done with this buffer before the load two tiles ahead reuses it
   }
 #pragma unroll
   for (int r = 0; r < 2; r++) {
@@ -200,9 +224,8 @@ __global__ void __launch_bounds__(128) attn_bwd_kv_mma(const bf16_t* __restrict_
                                                        const float* __restrict__ lse, const float* __restrict__ delta,
                                                        bf16_t* __restrict__ dqkv, int T, int H, float scale) {
   __shared__ __align__(16) bf16_t Xs[TS * LDS];   // K then V of this key tile (to build fragments), later unused
-  __shared__ __align__(16) bf16_t Qs[TS * LDS];
-  __shared__ __align__(16) bf16_t Ds[TS * LDS];   // dO
-  __shared__ float Ls[TS], Es[TS];
+  __shared__ __align__(16) bf16_t QDs[2][2][TS * LDS];   // [buffer][Q|dO]: the next query tile loads while this one is used
+  __shared__ float LEs[2][2][TS];                        // [buffer][lse*log2e | delta]
   const int kt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int d = H * DH;
   const long long ld = 3LL * d;
@@ -224,17 +247,32 @@ __global__ void __launch_bounds__(128) attn_bwd_kv_mma(const bf16_t* __restrict_
   const float sc2 = scale * 1.4426950408889634f;
   const int key_a = k0 + warp * 16 + g, key_b = key_a + 8;
   const int n_qt = (T + TS - 1) / TS;
-  for (int it = kt; it < n_qt; it++) {
+  auto fetch = [&](int it, int buf) {   // query tile `it` -> buffer `buf` (asynchronous)
     const int i0 = it * TS;
-    __syncthreads();
-    load_tile(Qs, base + (long long)i0 * ld, ld, T - i0);
-    load_tile(Ds, dob + (long long)i0 * d, d, T - i0);
+    load_tile_async(QDs[buf][0], base + (long long)i0 * ld, ld, T - i0);
+    load_tile_async(QDs[buf][1], dob + (long long)i0 * d, d, T - i0);
+    async_commit();
     if (threadIdx.x < TS) {
       const int i = i0 + threadIdx.x;
-      Ls[threadIdx.x] = i < T ? lse[((long long)b * H + h) * T + i] * 1.4426950408889634f : 0.f;
-      Es[threadIdx.x] = i < T ? delta[((long long)b * H + h) * T + i] : 0.f;
+      LEs[buf][0][threadIdx.x] = i < T ? lse[((long long)b * H + h) * T + i] * 1.4426950408889634f : 0.f;
+      LEs[buf][1][threadIdx.x] = i < T ? delta[((long long)b * H + h) * T + i] : 0.f;
+    }
+  };
+  fetch(kt, 0);
+  for (int it = kt; it < n_qt; it++) {
+    const int i0 = it * TS;
+    const int buf = (it - kt) & 1;
+    if (it + 1 < n_qt) {
+      fetch(it + 1, buf ^ 1);
+      async_wait<1>();
+    } else {
+      async_wait<0>();
     }
     __syncthreads();
+    const bf16_t* Qs = QDs[buf][0];
+    const bf16_t* Ds = QDs[buf][1];
+    const float* Ls = LEs[buf][0];
+    const float* Es = LEs[buf][1];
     float st[8][4], dp[8][4];
     zero_acc(st);
     zero_acc(dp);
@@ -255,6 +293,7 @@ __global__ void __launch_bounds__(128) attn_bwd_kv_mma(const bf16_t* __restrict_
     }
     mma_p_x(dv, st, Ds);    // dV += P^T dO
     mma_p_x(dk, dp, Qs);    // dK += dS^T Q
+    __syncthreads();        // this buffer is refilled two tiles ahead
   }
 #pragma unroll
   for (int r = 0; r < 2; r++) {
@@ -276,9 +315,9 @@ __global__ void __launch_bounds__(128) attn_bwd_q_mma(const bf16_t* __restrict__
                                                       const float* __restrict__ lse, const float* __restrict__ delta,
                                                       bf16_t* __restrict__ dqkv, int T, int H, float scale) {
   __shared__ __align__(16) bf16_t Xs[TS * LDS];   // Q then dO of this query tile (fragments only)
-  __shared__ __align__(16) bf16_t Ks[TS * LDS];
-  __shared__ __align__(16) bf16_t Vs[TS * LDS];
-  const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  __shared__ __align__(16) bf16_t KVs[2][2][TS * LDS];   // [buffer][K|V]
+  const int qt = gridDim.x - 1 - blockIdx.x;             // heaviest query tiles first
+  const int h = blockIdx.y, b = blockIdx.z;
   const int d = H * DH;
   const long long ld = 3LL * d;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t4 = lane & 3;
@@ -304,12 +343,22 @@ __global__ void __launch_bounds__(128) attn_bwd_q_mma(const bf16_t* __restrict__
   float dq[8][4];
   zero_acc(dq);
   const float sc2 = scale * 1.4426950408889634f;
+  load_tile_async(KVs[0][0], base + d, ld, T);
+  load_tile_async(KVs[0][1], base + 2 * d, ld, T);
+  async_commit();
   for (int jt = 0; jt <= qt; jt++) {
     const int j0 = jt * TS;
+    if (jt < qt) {
+      load_tile_async(KVs[(jt + 1) & 1][0], base + d + (long long)(j0 + TS) * ld, ld, T - j0 - TS);
+      load_tile_async(KVs[(jt + 1) & 1][1], base + 2 * d + (long long)(j0 + TS) * ld, ld, T - j0 - TS);
+      async_commit();
+      async_wait<1>();
+    } else {
+      async_wait<0>();
+    }
     __syncthreads();
-    load_tile(Ks, base + d + (long long)j0 * ld, ld, T - j0);
-    load_tile(Vs, base + 2 * d + (long long)j0 * ld, ld, T - j0);
-    __syncthreads();
+    const bf16_t* Ks = KVs[jt & 1][0];
+    const bf16_t* Vs = KVs[jt & 1][1];
     float s[8][4], dp[8][4];
     zero_acc(s);
     zero_acc(dp);
@@ -326,6 +375,7 @@ __global__ void __launch_bounds__(128) attn_bwd_q_mma(const bf16_t* __restrict__
       }
     }
     mma_p_x(dq, dp, Ks);    // dQ += dS K
+    __syncthreads();        // this buffer is refilled two tiles ahead
   }
 #pragma unroll
   for (int r = 0; r < 2; r++) {
