@@ -871,6 +871,84 @@ __global__ void __launch_bounds__(THREADS) softmax_ce_reg_kernel(bf16_t* __restr
   if ((tgt >> 3) % THREADS == threadIdx.x) rowloss[row] = lse - lt;   // the thread that holds the target logit
 }
 
+// Long rows (vocabularies beyond 16 Ki): the row is kept PACKED (bf16 pairs) in registers so
+// that two 512-thread CTAs fit on an SM and their load / reduce / store phases overlap; the
+// exponentials of the first pass overwrite the logits in place (as bf16) and the second pass only
+// scales them, so each element costs one exp.
+template <int THREADS, int VPT>
+__global__ void __launch_bounds__(THREADS, 2) softmax_ce_packed_kernel(bf16_t* __restrict__ logits,
+                                                                       const int32_t* __restrict__ ids, int T_,
+                                                                       float* __restrict__ rowloss, int V,
+                                                                       float inv_rows) {
+  __shared__ float sm[THREADS / 32];
+  const int row = blockIdx.x, nvec = V >> 3;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint4* p = reinterpret_cast<uint4*>(logits + (long long)row * V);
+  const int tgt = ids[(long long)(row / T_) * (T_ + 1) + (row % T_) + 1];
+  const float L2E = 1.4426950408889634f;
+  uint32_t w[VPT][4];
+  float mx = -INFINITY, lt = 0.f;
+#pragma unroll
+  for (int k = 0; k < VPT; k++) {
+    const int i = threadIdx.x + k * THREADS;
+    if (i < nvec) {
+      const uint4 q = p[i];
+      w[k][0] = q.x; w[k][1] = q.y; w[k][2] = q.z; w[k][3] = q.w;
+#pragma unroll
+      for (int j = 0; j < 4; j++) {
+        const float lo = __uint_as_float(w[k][j] << 16), hi = __uint_as_float(w[k][j] & 0xffff0000u);
+        mx = fmaxf(mx, fmaxf(lo, hi));
+        if (i * 8 + 2 * j == tgt) lt = lo;
+        if (i * 8 + 2 * j + 1 == tgt) lt = hi;
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; j++) w[k][j] = 0xff80ff80u;   // two bf16 -inf
+    }
+  }
+  auto block_reduce = [&](float v, bool is_max) {
+    v = is_max ? warp_max(v) : warp_sum(v);
+    __syncthreads();
+    if (lane == 0) sm[warp] = v;
+    __syncthreads();
+    float r = sm[0];
+    for (int i = 1; i < THREADS / 32; i++) r = is_max ? fmaxf(r, sm[i]) : r + sm[i];
+    return r;
+  };
+  mx = block_reduce(mx, true);
+  float se = 0.f;
+#pragma unroll
+  for (int k = 0; k < VPT; k++)
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+      const float lo = exp2f((__uint_as_float(w[k][j] << 16) - mx) * L2E);
+      const float hi = exp2f((__uint_as_float(w[k][j] & 0xffff0000u) - mx) * L2E);
+      se += lo + hi;                                       // the sum uses the unrounded exponentials
+      __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+      w[k][j] = *reinterpret_cast<uint32_t*>(&h);
+    }
+  se = block_reduce(se, false);
+  const float lse = mx + logf(se);
+  const float scale = inv_rows / se;
+#pragma unroll
+  for (int k = 0; k < VPT; k++) {
+    const int i = threadIdx.x + k * THREADS;
+    if (i < nvec) {
+      uint32_t o[4];
+#pragma unroll
+      for (int j = 0; j < 4; j++) {
+        float lo = __uint_as_float(w[k][j] << 16) * scale, hi = __uint_as_float(w[k][j] & 0xffff0000u) * scale;
+        if (i * 8 + 2 * j == tgt) lo -= inv_rows;
+        if (i * 8 + 2 * j + 1 == tgt) hi -= inv_rows;
+        __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+        o[j] = *reinterpret_cast<uint32_t*>(&h);
+      }
+      p[i] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+  }
+  if ((tgt >> 3) % THREADS == threadIdx.x) rowloss[row] = lse - lt;
+}
+
 cudaError_t softmax_ce_inplace(void* logits, const int32_t* ids, int T_, float* rowloss, int rows, int V,
                                float inv_rows, bool bf16, cudaStream_t s) {
   if (bf16 && V % 8 == 0 && (reinterpret_cast<uintptr_t>(logits) & 15) == 0) {
@@ -878,8 +956,9 @@ cudaError_t softmax_ce_inplace(void* logits, const int32_t* ids, int T_, float* 
     bf16_t* lg = (bf16_t*)logits;
     if (nvec <= 256 * 2) { softmax_ce_reg_kernel<256, 2><<<rows, 256, 0, s>>>(lg, ids, T_, rowloss, V, inv_rows); return cudaGetLastError(); }
     if (nvec <= 256 * 4) { softmax_ce_reg_kernel<256, 4><<<rows, 256, 0, s>>>(lg, ids, T_, rowloss, V, inv_rows); return cudaGetLastError(); }
-    if (nvec <= 1024 * 2) { softmax_ce_reg_kernel<1024, 2><<<rows, 1024, 0, s>>>(lg, ids, T_, rowloss, V, inv_rows); return cudaGetLastError(); }
-    if (nvec <= 1024 * 4) { softmax_ce_reg_kernel<1024, 4><<<rows, 1024, 0, s>>>(lg, ids, T_, rowloss, V, inv_rows); return cudaGetLastError(); }
+    if (nvec <= 512 * 4) { softmax_ce_packed_kernel<512, 4><<<rows, 512, 0, s>>>(lg, ids, T_, rowloss, V, inv_rows); return cudaGetLastError(); }
+    if (nvec <= 512 * 8) { softmax_ce_packed_kernel<512, 8><<<rows, 512, 0, s>>>(lg, ids, T_, rowloss, V, inv_rows); return cudaGetLastError(); }
+    if (nvec <= 512 * 16) { softmax_ce_packed_kernel<512, 16><<<rows, 512, 0, s>>>(lg, ids, T_, rowloss, V, inv_rows); return cudaGetLastError(); }
   }
   if (bf16) softmax_ce_kernel<bf16_t><<<rows, 256, 0, s>>>((bf16_t*)logits, ids, T_, rowloss, V, inv_rows);
   else softmax_ce_kernel<float><<<rows, 256, 0, s>>>((float*)logits, ids, T_, rowloss, V, inv_rows);
