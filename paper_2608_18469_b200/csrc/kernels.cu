@@ -188,6 +188,20 @@ template <> __device__ __forceinline__ float2 ld2<bf16_t>(const bf16_t* p, bool 
   return make_float2(__bfloat162float(p[0]), __bfloat162float(p[1]));
 }
 
+// sum_{k < chunks} p[k*stride] added in the order k = 0, 1, ..; eight loads are issued before the
+// first add so that the final pass costs one memory latency per eight partials, not per partial.
+__device__ __forceinline__ float ordered_sum(const float* p, long long stride, int chunks) {
+  float t = 0.f;
+  for (int k0 = 0; k0 < chunks; k0 += 8) {
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; u++) v[u] = k0 + u < chunks ? __ldcg(p + (long long)(k0 + u) * stride) : 0.f;
+#pragma unroll
+    for (int u = 0; u < 8; u++) if (k0 + u < chunks) t += v[u];
+  }
+  return t;
+}
+
 // Shared tail of the two-stage reductions: returns true in the CTA that arrives last on `ticket`.
 __device__ __forceinline__ bool last_cta(int* ticket, int expected) {
   __shared__ int s_last;
@@ -303,8 +317,7 @@ __global__ void __launch_bounds__(256) colsum_kernel(const T* __restrict__ X, lo
   for (int i = threadIdx.x; i < SW; i += 256) {
     const int cc = blockIdx.x * SW + i;
     if (cc < cols) {
-      float t = 0.f;
-      for (int k = 0; k < chunks; k++) t += ws[(long long)k * cols + cc];
+      float t = ordered_sum(ws + cc, cols, chunks);
       if (colscale) t *= colscale[cc];
       out[cc] = t;
     }
@@ -388,6 +401,8 @@ cudaError_t layernorm_bwd_dx(const void* dy, const void* x, const float* gain, c
   return cudaGetLastError();
 }
 
+// dgain / dshift partial sums: a CTA takes a strip of 32*VEC columns and one chunk of rows, a thread
+// VEC adjacent columns (16-byte loads of dy and x) and every 8th row, four rows in flight.
 template <typename T>
 __global__ void __launch_bounds__(256) layernorm_param_grad_kernel(const T* __restrict__ dy, const T* __restrict__ x,
                                                                    const float* __restrict__ mean,
@@ -395,50 +410,83 @@ __global__ void __launch_bounds__(256) layernorm_param_grad_kernel(const T* __re
                                                                    float* __restrict__ ws, float* __restrict__ dgain,
                                                                    float* __restrict__ dshift, int rows, int d, int chunks,
                                                                    int* tickets) {
-  __shared__ float sg[8][64], sb[8][64];
+  constexpr int VEC = VecOf<T>::N;
+  constexpr int SW = 32 * VEC;
+  __shared__ float sg[8][SW], sb[8][SW];
   const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
-  const int c = blockIdx.x * 64 + cx * 2;
+  const int c = blockIdx.x * SW + cx * VEC;
   const int per = (rows + chunks - 1) / chunks;
   const int rb = blockIdx.y * per, re = min(rows, rb + per);
-  const bool two = c + 1 < d;
-  const bool vec = two && (d % 2 == 0);
-  float g0 = 0.f, g1 = 0.f, b0 = 0.f, b1 = 0.f;
+  const bool vec = (c + VEC <= d) && (d % VEC == 0);
+  float ag[VEC], ab[VEC];
+#pragma unroll
+  for (int j = 0; j < VEC; j++) ag[j] = ab[j] = 0.f;
   if (c < d) {
-    for (int r = rb + ry; r < re; r += 8) {
-      float2 gy, xv;
-      if (two) { gy = ld2<T>(dy + (long long)r * d + c, vec); xv = ld2<T>(x + (long long)r * d + c, vec); }
-      else { gy = make_float2(ldf(dy + (long long)r * d + c), 0.f); xv = make_float2(ldf(x + (long long)r * d + c), 0.f); }
-      const float mu = mean[r], rs = rstd[r];
-      g0 = fmaf(gy.x, (xv.x - mu) * rs, g0);
-      g1 = fmaf(gy.y, (xv.y - mu) * rs, g1);
-      b0 += gy.x;
-      b1 += gy.y;
+    if (vec) {
+      int r = rb + ry;
+      for (; r + 24 < re; r += 32) {
+        float gy[4][VEC], xv[4][VEC], mu[4], rs[4];
+#pragma unroll
+        for (int u = 0; u < 4; u++) {
+          ld_vec<T>(dy + (long long)(r + 8 * u) * d + c, gy[u]);
+          ld_vec<T>(x + (long long)(r + 8 * u) * d + c, xv[u]);
+          mu[u] = mean[r + 8 * u];
+          rs[u] = rstd[r + 8 * u];
+        }
+#pragma unroll
+        for (int u = 0; u < 4; u++)
+#pragma unroll
+          for (int j = 0; j < VEC; j++) {
+            ag[j] = fmaf(gy[u][j], (xv[u][j] - mu[u]) * rs[u], ag[j]);
+            ab[j] += gy[u][j];
+          }
+      }
+      for (; r < re; r += 8) {
+        float gy[VEC], xv[VEC];
+        ld_vec<T>(dy + (long long)r * d + c, gy);
+        ld_vec<T>(x + (long long)r * d + c, xv);
+        const float mu = mean[r], rs = rstd[r];
+#pragma unroll
+        for (int j = 0; j < VEC; j++) {
+          ag[j] = fmaf(gy[j], (xv[j] - mu) * rs, ag[j]);
+          ab[j] += gy[j];
+        }
+      }
+    } else {
+      for (int r = rb + ry; r < re; r += 8) {
+        const float mu = mean[r], rs = rstd[r];
+#pragma unroll
+        for (int j = 0; j < VEC; j++)
+          if (c + j < d) {
+            const float g = ldf(dy + (long long)r * d + c + j);
+            ag[j] = fmaf(g, (ldf(x + (long long)r * d + c + j) - mu) * rs, ag[j]);
+            ab[j] += g;
+          }
+      }
     }
   }
-  sg[ry][cx * 2] = g0; sg[ry][cx * 2 + 1] = g1;
-  sb[ry][cx * 2] = b0; sb[ry][cx * 2 + 1] = b1;
+#pragma unroll
+  for (int j = 0; j < VEC; j++) { sg[ry][cx * VEC + j] = ag[j]; sb[ry][cx * VEC + j] = ab[j]; }
   __syncthreads();
   float* pg = chunks == 1 ? dgain : ws + (long long)blockIdx.y * d;
   float* pb = chunks == 1 ? dshift : ws + (long long)(chunks + blockIdx.y) * d;
-  if (threadIdx.x < 64) {
-    const int cc = blockIdx.x * 64 + threadIdx.x;
+  for (int i = threadIdx.x; i < SW; i += 256) {
+    const int cc = blockIdx.x * SW + i;
     if (cc < d) {
       float tg = 0.f, tb = 0.f;
 #pragma unroll
-      for (int i = 0; i < 8; i++) { tg += sg[i][threadIdx.x]; tb += sb[i][threadIdx.x]; }
+      for (int k = 0; k < 8; k++) { tg += sg[k][i]; tb += sb[k][i]; }
       pg[cc] = tg;
       pb[cc] = tb;
     }
   }
   if (chunks == 1) return;
   if (!last_cta(tickets + blockIdx.x, chunks)) return;
-  if (threadIdx.x < 64) {
-    const int cc = blockIdx.x * 64 + threadIdx.x;
+  for (int i = threadIdx.x; i < SW; i += 256) {
+    const int cc = blockIdx.x * SW + i;
     if (cc < d) {
-      float tg = 0.f, tb = 0.f;
-      for (int k = 0; k < chunks; k++) { tg += ws[(long long)k * d + cc]; tb += ws[(long long)(chunks + k) * d + cc]; }
-      dgain[cc] = tg;
-      dshift[cc] = tb;
+      dgain[cc] = ordered_sum(ws + cc, d, chunks);
+      dshift[cc] = ordered_sum(ws + (long long)chunks * d + cc, d, chunks);
     }
   }
 }
@@ -446,7 +494,7 @@ __global__ void __launch_bounds__(256) layernorm_param_grad_kernel(const T* __re
 cudaError_t layernorm_param_grad(const void* dy, const void* x, const float* mean, const float* rstd,
                                  float* ws, int chunks, int* tickets, float* dgain, float* dshift, int rows, int d,
                                  bool bf16, cudaStream_t s) {
-  dim3 grid(cdiv(d, 64), chunks);
+  dim3 grid(cdiv(d, bf16 ? 256 : 128), chunks);
   if (bf16) layernorm_param_grad_kernel<bf16_t><<<grid, 256, 0, s>>>((const bf16_t*)dy, (const bf16_t*)x, mean, rstd, ws, dgain, dshift, rows, d, chunks, tickets);
   else layernorm_param_grad_kernel<float><<<grid, 256, 0, s>>>((const float*)dy, (const float*)x, mean, rstd, ws, dgain, dshift, rows, d, chunks, tickets);
   return cudaGetLastError();
