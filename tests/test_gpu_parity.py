@@ -98,6 +98,23 @@ def test_config4_reduced_two_blocks():
     _gu().compare_teacher_forced(spec, steps=1, seed=0)
 
 
+def _edge_cases():
+    s = {}
+    s["mlp_bf16_batch1"] = synth.mlp_spec(64, 128, 2, 1, "gelu", "bf16")                 # a single row
+    s["mlp_bf16_odd_width"] = synth.mlp_spec(50, 77, 2, 33, "relu", "bf16")             # strides not multiples of 8: SIMT GEMMs
+    s["lm_bf16_seq1"] = synth.lm_spec(1, 64, 1, 128, 1, 3, 40)                           # one position per sequence
+    s["lm_bf16_vocab_odd"] = synth.lm_spec(1, 64, 1, 128, 20, 2, 203)                    # vocabulary not a multiple of 8
+    s["lm_bf16_T65"] = synth.lm_spec(1, 64, 1, 128, 65, 2, 96)                           # one row past a 64-tile
+    s["ctr_bf16_batch3"] = synth.ctr_spec(batch=3, table_rows=9, tower=(64, 32, 16))     # fewer rows than any tile
+    s["mlp_f32_batch1"] = synth.mlp_spec(8, 8, 1, 1, "relu", "f32")
+    return s
+
+
+@pytest.mark.parametrize("name", list(_edge_cases()))
+def test_edge_shapes(name):
+    _gu().compare_teacher_forced(_edge_cases()[name], steps=2, seed=4)
+
+
 # ------------------------------------------------------------------ schedules: bit identity
 
 def _bits_equal(a, b):
