@@ -357,7 +357,10 @@ def main():
     ap.add_argument("--loss-on-main", action="store_true", help="paper's placement of the local loss")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "ours":
+        # at least 3 warm-up steps; with graph replay at least one per pooled batch, so that every
+        # (batch pointers, schedule) graph is captured and instantiated before the timed region
+        args.warmup = max(args.warmup, 3 if args.no_graph else POOL)
     spec = synth.config(args.config, w=args.w, batch=args.batch)
     if args.impl == "reference":
         run_reference(args, spec, args.config)
