@@ -174,6 +174,8 @@ def run_gpu(args, spec, cfg_name):
     n_streams = args.n_streams if args.n_streams > 0 else nb + 1
     flags = 0 if args.no_graph else binding.GRAPH
     eflags = flags | (0 if args.loss_on_main else (binding.EARLY_HEAD | binding.BLOCK_OPT))
+    if args.split_bwd:
+        eflags |= binding.SPLIT_BWD
     units = units_per_step(spec)
 
     model = binding.Model(spec)
@@ -356,6 +358,7 @@ def main():
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--loss-on-main", action="store_true", help="paper's placement of the local loss")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--split-bwd", action="store_true", help="parameter-gradient work of each B_b on a second stream")
     args = ap.parse_args()
     if args.impl == "ours":
         # at least 3 warm-up steps; with graph replay at least one per pooled batch, so that every

@@ -141,6 +141,16 @@ typedef struct {
                             once B_b ends), so the optimizer's serial tail disappears under the other
                             blocks' work.  Same update kernel on the same values: same bits.          */
 
+#define ERASE_SPLIT_BWD 16u /* ERASE schedules only: inside B_b, the operations that only produce a
+                            parameter gradient (weight-gradient GEMMs and their reductions, bias column
+                            sums, LayerNorm gain/shift gradients) run on a second stream per block,
+                            each released by an event behind the gradient-chain operation whose output
+                            it reads; the chain (dgrads, attention, LayerNorm dx) stays on the block's
+                            side stream and the two join before the block's optimizer.  Nothing in B_b
+                            reads a parameter gradient, and every backward buffer is written once per
+                            step, so this is the overlap of Section 2.2 applied one level down.  Same
+                            kernels on the same values: same bits.                                    */
+
 /* Device bytes erase_create needs for this spec when given an arena; 0 if the spec is invalid. */
 ERASE_API size_t erase_arena_bytes(const erase_model_spec* spec);
 

@@ -31,6 +31,7 @@ struct Op {
   const char* name = "op";  // kernel class, for the per-operation profile
   double flops = 0;         // algorithmic floating-point operations of one run
   double bytes = 0;         // algorithmic bytes (each operand read once, each result written once)
+  bool leaf = false;        // backward op that only produces parameter gradients: nothing in B_b reads its output
 };
 typedef std::vector<Op> OpList;
 
@@ -87,6 +88,8 @@ struct erase_model {
   cudaStream_t main = nullptr;
   std::vector<cudaStream_t> side;
   std::vector<cudaEvent_t> ev_f, ev_b;
+  std::vector<cudaStream_t> leaf;                 // second side stream per block (ERASE_SPLIT_BWD)
+  std::vector<std::vector<cudaEvent_t>> ev_leaf;  // per block: one event per chain->leaf hand-over, plus the join
   cudaEvent_t ev_opt = nullptr;
   std::vector<cudaEvent_t> ev_time;  // 2*(2B+1) timing events + 1 step start
   std::vector<cudaEvent_t> ev_prof;  // pairs around every operation of a profiled step
@@ -411,8 +414,10 @@ struct Builder {
     if (splits > 64) splits = 64;
     g.splits = splits < 1 ? 1 : splits;
     gemm_tag = "gemm_wgrad";
+    const size_t before = ops.size();
     gemm(ops, g);
     if (bidx >= 0 && !skip_bias) bias_grad(ops, dY, N, M, N, bidx);
+    for (size_t i = before; i < ops.size(); i++) ops[i].leaf = true;
   }
   void bias_grad(OpList& ops, const void* dY, long long ld, int M, int N, int bidx) {
     int chunks = colsum_chunks(M, N);
@@ -456,6 +461,7 @@ struct Builder {
         int* tk = tickets(d);
         bw.push_back({[=](cudaStream_t s) { return colsum(z, bf, d, rows, d, ds, ws, chunks, tk, out, s); }, 1});
         note(bw, "colsum", 2.0 * rows * d, (double)rows * d * m->esz);
+        bw.back().leaf = true;
       }
       {
         int chunks = colsum_chunks(rows, 1);
@@ -464,6 +470,7 @@ struct Builder {
         int* tk = tickets(1);
         bw.push_back({[=](cudaStream_t s) { return colsum(ds, false, 1, rows, 1, nullptr, ws, chunks, tk, out, s); }, 1});
         note(bw, "colsum", rows, 4.0 * rows);
+        bw.back().leaf = true;
       }
       if (last_bias >= 0) {
         int chunks = colsum_chunks(rows, d);
@@ -473,6 +480,7 @@ struct Builder {
         int* tk = tickets(d);
         bw.push_back({[=](cudaStream_t s) { return colsum(src, bf, d, rows, d, ds, ws, chunks, tk, out, s, dact, w); }, 1});
         note(bw, "colsum", 2.0 * rows * d, src ? (double)rows * d * m->esz : 4.0 * rows);
+        bw.back().leaf = true;
         return true;
       }
       return false;
@@ -649,6 +657,7 @@ struct Builder {
     int* tk = tickets(d);
     bw.push_back({[=](cudaStream_t s) { return layernorm_param_grad(dy, x, mean, rstd, ws, chunks, tk, dg, db, rows, d, bf, s); }, 1});
     note(bw, "layernorm_param_grad", 4.0 * rows * d, 2.0 * rows * d * m->esz);
+    bw.back().leaf = true;
   }
 
   void* block_cross(int b, const erase_block_spec& k, const void* x0, int first, OpList& f, OpList& bw) {
@@ -848,6 +857,7 @@ erase_status enqueue_step(erase_model* m, int n_streams, unsigned flags, bool ti
   const bool early_head = (flags & ERASE_EARLY_HEAD) != 0;
   // per-block optimizer: theta_b is read by F_b and B_b only, so it can be updated right behind B_b
   const bool block_opt = do_opt && n_streams > 1 && (flags & ERASE_BLOCK_OPT) != 0;
+  const bool split_bwd = n_streams > 1 && (flags & ERASE_SPLIT_BWD) != 0;
   if (block_opt) CK(run_ops(m, m->opt_tick_op, m->main));
   if (n_streams <= 1) {
     for (int b = 0; b < B; b++) {
@@ -880,7 +890,35 @@ erase_status enqueue_step(erase_model* m, int n_streams, unsigned flags, bool ti
       if (timed) CK(cudaEventRecord(tev(2 * (B + b)), sd));
       m->sm_budget = budget_side;
       if (early_head) CK(run_ops(m, m->hfwd[b], sd));    // z_b's only other consumer is F_{b+1}, which does not wait
-      CK(run_ops(m, m->bwd[b], sd));
+      if (!split_bwd) {
+        CK(run_ops(m, m->bwd[b], sd));
+      } else {
+        // The gradient chain (dgrads, attention, LayerNorm dx, ...) stays on sd; every operation
+        // that only produces a parameter gradient goes to a second stream behind the chain op
+        // whose output it reads.  Every backward buffer is written once per step, so a leaf never
+        // races with a later chain op; the two streams join before the block's optimizer.
+        cudaStream_t lf = m->leaf[b % ns];
+        size_t ne = 0;
+        bool handed = false;   // has lf already been made to wait for everything enqueued on sd so far?
+        for (Op& op : m->bwd[b]) {
+          if (op.leaf) {
+            if (!handed) {
+              cudaEvent_t e = m->ev_leaf[b][ne++];
+              CK(cudaEventRecord(e, sd));
+              CK(cudaStreamWaitEvent(lf, e, 0));
+              handed = true;
+            }
+            CK(op.fn(lf));
+          } else {
+            CK(op.fn(sd));
+            handed = false;
+          }
+          m->launches += op.launches;
+        }
+        cudaEvent_t e = m->ev_leaf[b][ne++];
+        CK(cudaEventRecord(e, lf));
+        CK(cudaStreamWaitEvent(sd, e, 0));
+      }
       if (timed) CK(cudaEventRecord(tev(2 * (B + b) + 1), sd));
       if (block_opt) CK(run_ops(m, m->opt_blk[b], sd));
       CK(cudaEventRecord(m->ev_b[b], sd));
@@ -932,7 +970,19 @@ erase_status erase_create(const erase_model_spec* spec, erase_model** out) {
   m->side.resize(m->B);
   for (int i = 0; i < m->B; i++)
     if (cudaStreamCreateWithFlags(&m->side[i], cudaStreamNonBlocking) != cudaSuccess) { m->side.resize(i); return bail(ERASE_ECUDA, "stream creation failed"); }
+  m->leaf.resize(m->B);
+  for (int i = 0; i < m->B; i++)
+    if (cudaStreamCreateWithFlags(&m->leaf[i], cudaStreamNonBlocking) != cudaSuccess) { m->leaf.resize(i); return bail(ERASE_ECUDA, "stream creation failed"); }
   auto mk = [&](cudaEvent_t* e, unsigned fl) { return cudaEventCreateWithFlags(e, fl) == cudaSuccess; };
+  m->ev_leaf.resize(m->B);
+  for (int b = 0; b < m->B; b++) {
+    size_t n = 1;   // the join
+    bool prev_leaf = false;
+    for (const Op& op : m->bwd[b]) { if (op.leaf && !prev_leaf) n++; prev_leaf = op.leaf; }
+    m->ev_leaf[b].assign(n, nullptr);
+    for (auto& e : m->ev_leaf[b])
+      if (!mk(&e, cudaEventDisableTiming)) return bail(ERASE_ECUDA, "event creation failed");
+  }
   m->ev_f.assign(m->B, nullptr);
   m->ev_b.assign(m->B, nullptr);
   for (int i = 0; i < m->B; i++)
@@ -950,13 +1000,16 @@ void erase_destroy(erase_model* m) {
   if (!m) return;
   if (m->main) cudaStreamSynchronize(m->main);
   for (auto s : m->side) if (s) cudaStreamSynchronize(s);
+  for (auto s : m->leaf) if (s) cudaStreamSynchronize(s);
   for (auto& kv : m->graphs) cudaGraphExecDestroy(kv.second.first);
   for (auto e : m->ev_f) if (e) cudaEventDestroy(e);
   for (auto e : m->ev_b) if (e) cudaEventDestroy(e);
   for (auto e : m->ev_time) if (e) cudaEventDestroy(e);
   for (auto e : m->ev_prof) if (e) cudaEventDestroy(e);
   if (m->ev_opt) cudaEventDestroy(m->ev_opt);
+  for (auto& v : m->ev_leaf) for (auto e : v) if (e) cudaEventDestroy(e);
   for (auto s : m->side) if (s) cudaStreamDestroy(s);
+  for (auto s : m->leaf) if (s) cudaStreamDestroy(s);
   if (m->main) cudaStreamDestroy(m->main);
   for (void* p : m->owned) cudaFree(p);
   cudaGetLastError();
@@ -1063,7 +1116,7 @@ static erase_status check_step_args(erase_model* m, const erase_batch* batch);
 erase_status erase_step_ex(erase_model* m, const erase_batch* batch, int32_t n_streams, uint32_t flags) {
   if (!m) return ERASE_EINVAL;
   if (n_streams < 1) return m->fail(ERASE_EINVAL, "erase_step: n_streams must be >= 1");
-  if (flags & ~(ERASE_GRAPH | ERASE_NO_OPT | ERASE_EARLY_HEAD | ERASE_BLOCK_OPT)) return m->fail(ERASE_EINVAL, "erase_step: unknown flag");
+  if (flags & ~(ERASE_GRAPH | ERASE_NO_OPT | ERASE_EARLY_HEAD | ERASE_BLOCK_OPT | ERASE_SPLIT_BWD)) return m->fail(ERASE_EINVAL, "erase_step: unknown flag");
   erase_status cst = check_step_args(m, batch);
   if (cst != ERASE_OK) return cst;
   if (n_streams > m->B + 1) n_streams = m->B + 1;

@@ -145,4 +145,9 @@ def test_erase_schedule_is_bit_identical_to_serial(name):
     _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=nb + 1, flags=binding.BLOCK_OPT))
     _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=nb + 1,
                                      flags=binding.GRAPH | binding.EARLY_HEAD | binding.BLOCK_OPT))
+    _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=nb + 1, flags=binding.SPLIT_BWD))
+    _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=2,
+                                     flags=binding.GRAPH | binding.EARLY_HEAD | binding.BLOCK_OPT | binding.SPLIT_BWD))
+    _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=nb + 1,
+                                     flags=binding.GRAPH | binding.EARLY_HEAD | binding.BLOCK_OPT | binding.SPLIT_BWD))
     assert serial["launches"] > 0
