@@ -1309,6 +1309,7 @@ erase_status erase_gemm(int32_t dtype, int32_t M, int32_t N, int32_t K, const vo
               h[1] - h[0], h[2] - h[0], h[8] - h[0], h[3] - h[0], h[9] - h[0], h[4] - h[0], h[5] - h[0], h[6] - h[0], h[7] - h[0]);
     fprintf(stderr, "   epilogue detail: staged %lld | store issued %lld | loop done %lld | fenced %lld | arrived %lld\n",
             h[10] - h[0], h[11] - h[0], h[12] - h[0], h[13] - h[0], h[6] - h[0]);
+    if (getenv("ERASE_TC_PAIR")) fprintf(stderr, "   pair kernel: TMEM base of the leader %lld, of the peer %lld\n", h[8], h[9]);
     cudaFree(dbg);
   }
   cleanup();

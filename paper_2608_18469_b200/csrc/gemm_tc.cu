@@ -46,7 +46,6 @@ struct TcArgs {
   int* status;
   long long* dbg;  // optional: clock64 stamps of CTA 0's first tile (development aid), else null
   int tma_c;       // C (or the split-K partials) leaves through shared memory + TMA store
-  int tma_p;       // so does the pre-activation copy
   int plain;       // 1: the epilogue is the identity; 2: bias add only; 0: general
   int* sched;      // {next tile counter, finished CTAs}, zero between launches; null = static round-robin
 };
@@ -128,52 +127,29 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
 
 __device__ __forceinline__ float bf2f(uint32_t bits16) { return __uint_as_float(bits16 << 16); }
 
-// Phi(u) and phi(u) of the standard normal for the exact-erf GELU, with erf from the
-// Abramowitz-Stegun 7.1.26 rational form (|error| <= 1.5e-7, far below bf16 resolution): one
-// reciprocal, one exp2 and a 5-term polynomial, shared by the value and the derivative.  Short
-// enough to stay inline in the epilogue (erff's expansion was not).
-__device__ __forceinline__ void normal_cdf_pdf(float u, float& cdf, float& pdf) {
-  const float x = fabsf(u) * 0.70710678118654752f;
-  const float t = __frcp_rn(fmaf(0.3275911f, x, 1.f));
-  const float e = exp2f(-1.4426950408889634f * x * x);          // exp(-u^2/2)
-  float poly = fmaf(1.061405429f, t, -1.453152027f);
-  poly = fmaf(poly, t, 1.421413741f);
-  poly = fmaf(poly, t, -0.284496736f);
-  poly = fmaf(poly, t, 0.254829592f);
-  const float half_erfc = 0.5f * poly * t * e;                   // 0.5*(1 - erf(x)), x >= 0
-  cdf = u >= 0.f ? 1.f - half_erfc : half_erfc;
-  pdf = 0.39894228040143268f * e;
-}
-__device__ __forceinline__ float act_apply_d(int act, float v) {
-  if (act == ACT_RELU) return v > 0.f ? v : 0.f;
-  if (act == ACT_GELU) {
-    float cdf, pdf;
-    normal_cdf_pdf(v, cdf, pdf);
-    return v * cdf;
-  }
-  return v;
-}
-__device__ __forceinline__ float act_deriv_d(int act, float u) {
-  if (act == ACT_RELU) return u > 0.f ? 1.f : 0.f;
-  if (act == ACT_GELU) {
-    float cdf, pdf;
-    normal_cdf_pdf(u, cdf, pdf);
-    return fmaf(u, pdf, cdf);
-  }
-  return 1.f;
+// Only ReLU is fused (a compare).  GELU's erf chain on the few epilogue warps, and the instruction
+// footprint of its inlined copies, made a fused GEMM slower than the GEMM plus a separate
+// elementwise pass, so GEMMs that ask for it (or for a pre-activation copy) use the SIMT kernel.
+
+// 8 bf16 held in a 16-byte register quad -> floats
+__device__ __forceinline__ void unpack8_bf16(uint4 q, float* out) {
+  out[0] = __uint_as_float(q.x << 16); out[1] = __uint_as_float(q.x & 0xffff0000u);
+  out[2] = __uint_as_float(q.y << 16); out[3] = __uint_as_float(q.y & 0xffff0000u);
+  out[4] = __uint_as_float(q.z << 16); out[5] = __uint_as_float(q.z & 0xffff0000u);
+  out[6] = __uint_as_float(q.w << 16); out[7] = __uint_as_float(q.w & 0xffff0000u);
 }
 
-// 8 consecutive bf16 -> floats (16-byte load when aligned and fully inside, else scalar with bound)
-__device__ __forceinline__ void load8_bf16(const __nv_bfloat16* p, int valid, bool vec, float* out) {
-  if (vec) {
-    uint4 q = *reinterpret_cast<const uint4*>(p);
-    out[0] = bf2f(q.x & 0xffffu); out[1] = bf2f(q.x >> 16);
-    out[2] = bf2f(q.y & 0xffffu); out[3] = bf2f(q.y >> 16);
-    out[4] = bf2f(q.z & 0xffffu); out[5] = bf2f(q.z >> 16);
-    out[6] = bf2f(q.w & 0xffffu); out[7] = bf2f(q.w >> 16);
-  } else {
+// The epilogue's auxiliary operands (residual; multiplier or activation-derivative source) of one
+// output row x 32 columns, as raw bf16.  A warp's 32 lanes read 32 different rows, so each of
+// these loads is a full memory round trip: they are issued one chunk ahead -- the first chunk
+// before the warp starts waiting for its accumulator -- and consumed from registers.
+struct Aux32 { uint4 a[4], b[4]; };
+__device__ __forceinline__ void aux_issue(const __nv_bfloat16* pa, const __nv_bfloat16* pb, bool row_ok, int n, int N, Aux32& r) {
 #pragma unroll
-    for (int j = 0; j < 8; j++) out[j] = j < valid ? __bfloat162float(p[j]) : 0.f;
+  for (int g = 0; g < 4; g++) {
+    const bool ok = row_ok && n + 8 * g < N;   // N is a multiple of 8 whenever an auxiliary operand is present
+    r.a[g] = (pa && ok) ? *reinterpret_cast<const uint4*>(pa + n + 8 * g) : make_uint4(0u, 0u, 0u, 0u);
+    r.b[g] = (pb && ok) ? *reinterpret_cast<const uint4*>(pb + n + 8 * g) : make_uint4(0u, 0u, 0u, 0u);
   }
 }
 __device__ __forceinline__ uint32_t pack2(float a, float b) {
@@ -196,19 +172,14 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
-// Fused epilogue on 8 accumulator values of one output row (columns n..n+7), in place.
-// stop_at_pre: return alpha*acc + bias (the pre-activation) and nothing else.
-// The pre-activation copy is written here directly unless it leaves through TMA (p.tma_p).
+// Fused epilogue on 8 accumulator values of one output row (columns n..n+7), in place:
+//   v = alpha*acc + bias; v = relu(v); v *= mul; v += res; v *= relu'(dact_src)
+// aux_a: 8 residual values, aux_b: 8 multiplier or derivative-source values (raw bf16).
 struct F8 { float v[8]; };
 
-// The epilogue body runs once per tile in each warp, so its instruction-cache footprint matters
-// more than its instruction count: the activation functions are calls, the column loop is rolled.
-__device__ __forceinline__ F8 epilogue_values8(const TcArgs& p, F8 in, int row, int n, bool stop_at_pre, const float* bias8) {
+__device__ __forceinline__ F8 epilogue_values8(const TcArgs& p, F8 in, const float* bias8, uint4 aux_a, uint4 aux_b) {
   float* v = in.v;
   const Epilogue& e = p.epi;
-  const int valid = min(8, p.N - n);
-  const long long ia = (long long)row * e.ld_aux + n;
-  const bool avec = valid == 8 && (e.ld_aux % 8 == 0);
   float t[8];
   if (e.alpha != 1.f) {
 #pragma unroll
@@ -220,32 +191,24 @@ __device__ __forceinline__ F8 epilogue_values8(const TcArgs& p, F8 in, int row, 
     v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w;
     v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
   }
-  if (stop_at_pre) return in;
-  if (e.pre_out && !p.tma_p) {
-    __nv_bfloat16* po = (__nv_bfloat16*)e.pre_out + ia;
-    store8_bf16(po, valid, avec && ((reinterpret_cast<uintptr_t>(po) & 15) == 0), v);
-  }
-  if (e.act != ACT_NONE) {
+  if (e.act == ACT_RELU) {
 #pragma unroll
-    for (int j = 0; j < 8; j++) v[j] = act_apply_d(e.act, v[j]);
+    for (int j = 0; j < 8; j++) v[j] = fmaxf(v[j], 0.f);
   }
-  if (e.mul) {
-    const __nv_bfloat16* pm = (const __nv_bfloat16*)e.mul + ia;
-    load8_bf16(pm, valid, avec && ((reinterpret_cast<uintptr_t>(pm) & 15) == 0), t);
+  if (e.mul) {          // aux_b holds the multiplier (never together with a derivative source)
+    unpack8_bf16(aux_b, t);
 #pragma unroll
     for (int j = 0; j < 8; j++) v[j] *= t[j];
   }
   if (e.res) {
-    const __nv_bfloat16* pr = (const __nv_bfloat16*)e.res + ia;
-    load8_bf16(pr, valid, avec && ((reinterpret_cast<uintptr_t>(pr) & 15) == 0), t);
+    unpack8_bf16(aux_a, t);
 #pragma unroll
     for (int j = 0; j < 8; j++) v[j] += t[j];
   }
-  if (e.dact != ACT_NONE) {
-    const __nv_bfloat16* pd = (const __nv_bfloat16*)e.dact_src + ia;
-    load8_bf16(pd, valid, avec && ((reinterpret_cast<uintptr_t>(pd) & 15) == 0), t);
+  if (e.dact == ACT_RELU) {
+    unpack8_bf16(aux_b, t);
 #pragma unroll
-    for (int j = 0; j < 8; j++) v[j] *= act_deriv_d(e.dact, t[j]);
+    for (int j = 0; j < 8; j++) v[j] = t[j] > 0.f ? v[j] : 0.f;
   }
   return in;
 }
@@ -307,7 +270,7 @@ __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int
 template <int BN, bool A_MN, bool B_MN, bool GENERAL>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_p,
+               const __grid_constant__ CUtensorMap map_c,
                const __grid_constant__ TcArgs p) {
   extern __shared__ uint8_t smem_raw[];
   constexpr uint32_t A_BYTES = BM * BK * 2;
@@ -343,7 +306,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
     if (p.tma_c) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_c) : "memory");
-    if (p.tma_p) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_p) : "memory");
   }
   const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
   const int total = tiles_m * tiles_n * p.splits;
@@ -517,25 +479,41 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         __syncwarp();
       }
+      const int row = m0 + q * 32 + lane;
+      const bool row_ok = row < p.M;
+      // auxiliary operands of this thread's row (raw bf16), fetched one 32-column chunk ahead
+      const __nv_bfloat16* aux_pa = nullptr;
+      const __nv_bfloat16* aux_pb = nullptr;
+      Aux32 aux_cur, aux_nxt;
+      if (GENERAL && !p.plain && p.splits == 1) {
+        const long long ro = (long long)row * p.epi.ld_aux;
+        if (p.epi.res) aux_pa = (const __nv_bfloat16*)p.epi.res + ro;
+        const void* bsrc = p.epi.mul ? p.epi.mul : (p.epi.dact != ACT_NONE ? p.epi.dact_src : nullptr);
+        if (bsrc) aux_pb = (const __nv_bfloat16*)bsrc + ro;
+        if (active && n0 + cbeg < p.N && (aux_pa || aux_pb)) {   // in flight while the MMAs still run
+          aux_issue(aux_pa, aux_pb, row_ok, n0 + cbeg, p.N, aux_nxt);
+        }
+      }
+      const bool use_aux = GENERAL && (aux_pa || aux_pb);
       bool ok = mbar_wait(tfull_bar(ab), aph);
       if (!ok) atomicExch(p.status, 3);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
       if (dbg && lt == 0 && threadIdx.x == 64) p.dbg[5] = clock64();
-      const int row = m0 + q * 32 + lane;
-      const bool row_ok = row < p.M;
       const long long dflags = p.dbg ? p.dbg[15] : 0;
-      const int npass = (GENERAL && p.epi.pre_out && p.tma_p) ? 2 : 1;   // pass 0 of 2 writes the pre-activation copy
       if (active && n0 + cbeg < p.N) {
-        for (int pass = 0; pass < npass; pass++) {
-          const bool pre_pass = npass == 2 && pass == 0;
-          const bool via_tma = pre_pass ? true : (p.tma_c != 0);
-          const bool f32 = !pre_pass && out_f32;
+        {
+          const bool via_tma = p.tma_c != 0;
+          const bool f32 = out_f32;
 #pragma unroll 1
           for (int cc = 0; cc < CPW; cc += 32) {
             const int c0 = cbeg + cc;
             if (n0 + c0 >= p.N) break;  // warp-uniform
+            if (GENERAL && use_aux) {
+              aux_cur = aux_nxt;
+              if (cc + 32 < CPW && n0 + c0 + 32 < p.N) aux_issue(aux_pa, aux_pb, row_ok, n0 + c0 + 32, p.N, aux_nxt);
+            }
             uint32_t r[32];
             if (!empty_k && !(dflags & 2)) {
               tc_ld32(tmem_base + ab * BN + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
@@ -562,7 +540,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 f.v[0] += b0.x; f.v[1] += b0.y; f.v[2] += b0.z; f.v[3] += b0.w;
                 f.v[4] += b1.x; f.v[5] += b1.y; f.v[6] += b1.z; f.v[7] += b1.w;
               } else if (GENERAL && row_ok && n < p.N && p.splits == 1 && !p.plain) {
-                f = epilogue_values8(p, f, row, n, pre_pass, bias_s + cc + g8 * 8);
+                f = epilogue_values8(p, f, bias_s + cc + g8 * 8, aux_cur.a[g8], aux_cur.b[g8]);
               }
               const float* v = f.v;
               if (!via_tma) {
@@ -583,8 +561,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               if (dbg && lt == 0 && threadIdx.x == 64 && p.dbg[10] == 0) p.dbg[10] = clock64();
               if (lane == 0 && !(dflags & 1)) {
                 const int x = f32 ? n0 + c0 : n0 + cbeg + (cc & ~63), y = m0 + q * 32;
-                if (pre_pass) tma_store_2d(&map_p, stage, x, y);
-                else if (p.splits > 1) tma_store_3d(&map_c, stage, x, y, split);
+                if (p.splits > 1) tma_store_3d(&map_c, stage, x, y, split);
                 else tma_store_2d(&map_c, stage, x, y);
                 tma_store_commit();
                 store_pending = true;
@@ -620,6 +597,307 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
   }
   if (dbg && threadIdx.x == 0) p.dbg[7] = clock64();
+}
+
+// =================================================================================================
+// CTA-pair kernel (tcgen05 cta_group::2): two CTAs of a cluster, on neighbouring SMs, share one
+// 256 x 256 output tile.  Each CTA stages its own 128 rows of A and HALF of the B slab (128 of the
+// 256 columns) per K block; the pair's tensor cores read both halves, so every SM moves 32 KB per
+// K block through shared memory and L2 instead of the 48 KB of the single-CTA 128 x 256 tile --
+// which is what bounds the large GEMMs.  The leader CTA (cluster rank 0) issues the MMAs
+// (M = 256, N = 256, K = 16) for both; the accumulator rows 0..127 land in the leader's TMEM,
+// rows 128..255 in the peer's, and each CTA's epilogue warps drain their own.
+//   full[s]    leader only: TMA bytes of BOTH CTAs' stage s have landed (both CTAs' copies signal it)
+//   empty[s]   per CTA: the MMAs that read stage s are done (one commit, delivered to both CTAs)
+//   tfull[a]   per CTA: accumulator a is complete (delivered to both CTAs)
+//   tempty[a]  leader only: both CTAs' epilogue warps have drained accumulator a (the peer's warps
+//              arrive on it through the cluster's shared-memory window)
+// Tiles are assigned round-robin to clusters, in the order of tile_coords.  Only the identity /
+// bias-only epilogue with TMA-stored output is implemented; other GEMMs use tc_gemm_kernel.
+constexpr int PAIR_BN = 256;
+constexpr int PAIR_STAGES = 4;
+constexpr uint32_t PAIR_STAGE_BYTES = 2u * BM * BK * 2u;   // 128 x 64 of A + 128 x 64 of B, bf16
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {   // same offset in CTA `rank` of the cluster
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// copy into this CTA's shared memory; the byte count is credited to `bar`, which may be the peer's
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {   // arrives on `bar` in both CTAs of the pair
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask) : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+template <bool A_MN, bool B_MN>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
+tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                    const __grid_constant__ CUtensorMap map_c, const __grid_constant__ TcArgs p, const uint32_t tmem_cols) {
+  extern __shared__ uint8_t smem_raw[];
+  constexpr int BN = PAIR_BN;
+  constexpr int STAGES = PAIR_STAGES;
+  constexpr uint32_t A_BYTES = BM * BK * 2;
+  constexpr uint32_t STAGE_BYTES = PAIR_STAGE_BYTES;
+  constexpr int CPW = BN / 2;
+
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t epi_base = smem_base + STAGES * STAGE_BYTES;
+  const uint32_t bias_base = epi_base + EPI_WARPS * EPI_STAGE_BYTES;
+  const uint32_t bar_base = bias_base + EPI_WARPS * EPI_BIAS_BYTES;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+  uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
+  volatile uint32_t* tmem_slot_ptr =
+      reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * (EPI_STAGE_BYTES + EPI_BIAS_BYTES) + 8u * (2 * STAGES + 4));
+  const uint32_t tmem_slot = bar_base + 8u * (2 * STAGES + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+  const int naccum = tmem_cols >= 2u * BN ? 2 : 1;      // accumulators in TMEM (two: epilogue overlaps the next main loop)
+  if (threadIdx.x == 32) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_c) : "memory");
+  }
+  const int tiles_m = (p.M + 2 * BM - 1) / (2 * BM), tiles_n = (p.N + BN - 1) / BN;
+  const int total = tiles_m * tiles_n * p.splits;
+  const int kchunk = (((p.K + p.splits - 1) / p.splits) + BK - 1) / BK * BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; s++) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; a++) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), 2 * EPI_WARPS);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {   // one warp of EACH CTA of the pair takes part in the allocation
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();      // the peer's barriers exist before anything is sent to them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot_ptr;
+  if (p.dbg && threadIdx.x == 0 && cluster_id == 0) p.dbg[8 + rank] = (long long)tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer (both CTAs) ------------------------------
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int t = cluster_id; t < total && ok; t += n_clusters) {
+        int mt, nt, split;
+        tile_coords(t, tiles_m, tiles_n, mt, nt, split);
+        const int m0 = mt * 2 * BM + (int)rank * BM;        // this CTA's 128 rows of A
+        const int nb0 = nt * BN + (int)rank * (BN / 2);     // this CTA's 128 columns of B
+        const int kbeg = split * kchunk, kend = min(p.K, kbeg + kchunk);
+        const int num_kb = kend > kbeg ? (kend - kbeg + BK - 1) / BK : 0;
+        for (int kb = 0; kb < num_kb; kb++, it++) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!mbar_wait(empty_bar(s), ph ^ 1)) { atomicExch(p.status, 1); ok = false; break; }
+          if (leader) mbar_expect_tx(full_bar(s), 2 * STAGE_BYTES);   // this CTA's bytes and the peer's
+          const uint32_t lfull = map_to_cta(full_bar(s), 0);
+          const uint32_t a_dst = smem_base + s * STAGE_BYTES;
+          const uint32_t b_dst = a_dst + A_BYTES;
+          const int k0 = kbeg + kb * BK;
+          if (!A_MN) {
+            tma_load_2d_pair(a_dst, &map_a, k0, m0, lfull);
+          } else {
+#pragma unroll
+            for (int a = 0; a < BM / 64; a++) tma_load_2d_pair(a_dst + a * (BK * 128), &map_a, m0 + a * 64, k0, lfull);
+          }
+          if (!B_MN) {
+            tma_load_2d_pair(b_dst, &map_b, k0, nb0, lfull);
+          } else {
+#pragma unroll
+            for (int a = 0; a < BN / 128; a++) tma_load_2d_pair(b_dst + a * (BK * 128), &map_b, nb0 + a * 64, k0, lfull);
+          }
+        }
+      }
+      if (!ok) {  // give copies already in flight time to land before the CTA's shared memory is released
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) {}
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer (leader CTA only) ------------------------------
+    if (lane == 0 && leader) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16) |
+                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+      uint32_t it = 0, lt = 0;
+      bool ok = true;
+      for (int t = cluster_id; t < total && ok; t += n_clusters, lt++) {
+        const int split = t / (tiles_m * tiles_n);
+        const int kbeg = split * kchunk, kend = min(p.K, kbeg + kchunk);
+        const int num_kb = kend > kbeg ? (kend - kbeg + BK - 1) / BK : 0;
+        const uint32_t ab = naccum == 2 ? (lt & 1) : 0u, aph = naccum == 2 ? ((lt >> 1) & 1) : (lt & 1);
+        if (!mbar_wait(tempty_bar(ab), aph ^ 1)) { atomicExch(p.status, 4); ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + ab * BN;
+        for (int kb = 0; kb < num_kb; kb++, it++) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!mbar_wait(full_bar(s), ph)) { atomicExch(p.status, 2); ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_src = smem_base + s * STAGE_BYTES;
+          const uint32_t b_src = a_src + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; k++) {
+            // the same descriptors address this CTA's and the peer's shared memory (identical layout)
+            const uint64_t ad = A_MN ? smem_desc(a_src + k * (UMMA_K * 128), BK * 128, 1024)
+                                     : smem_desc(a_src + k * (UMMA_K * 2), 16, 1024);
+            const uint64_t bd = B_MN ? smem_desc(b_src + k * (UMMA_K * 128), BK * 128, 1024)
+                                     : smem_desc(b_src + k * (UMMA_K * 2), 16, 1024);
+            tc_mma_pair(tmem_d, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          }
+          tc_commit_pair(empty_bar(s));
+        }
+        tc_commit_pair(tfull_bar(ab));
+      }
+    }
+  } else {
+    // ------------------------------ epilogue (both CTAs, own 128 rows) ------------------------------
+    const int ew = warp - 2;
+    const int q = warp & 3;
+    const int cbeg = (ew / 4) * CPW;
+    const uint32_t stage0 = epi_base + ew * EPI_STAGE_BYTES;
+    uint32_t sbuf = 0;
+    float* bias_s = reinterpret_cast<float*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * EPI_STAGE_BYTES + ew * EPI_BIAS_BYTES);
+    const bool f32 = p.splits > 1 || p.c_f32;
+    const uint32_t ltempty0 = map_to_cta(tempty_bar(0), 0), ltempty1 = map_to_cta(tempty_bar(1), 0);
+    bool store_pending = false;
+    uint32_t lt = 0;
+    for (int t = cluster_id; t < total; t += n_clusters, lt++) {
+      int mt, nt, split;
+      tile_coords(t, tiles_m, tiles_n, mt, nt, split);
+      const int m0 = mt * 2 * BM + (int)rank * BM, n0 = nt * BN;
+      const int kbeg = split * kchunk, kend = min(p.K, kbeg + kchunk);
+      const bool empty_k = kend <= kbeg;
+      const uint32_t ab = naccum == 2 ? (lt & 1) : 0u, aph = naccum == 2 ? ((lt >> 1) & 1) : (lt & 1);
+      if (p.plain == 2) {
+        __syncwarp();
+        for (int j = lane; j < CPW; j += 32) {
+          const int n = n0 + cbeg + j;
+          bias_s[j] = n < p.N ? __ldg(p.epi.bias + n) : 0.f;
+        }
+        __syncwarp();
+      }
+      bool ok = mbar_wait(tfull_bar(ab), aph);
+      if (!ok) atomicExch(p.status, 3);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const bool rows_in = m0 + q * 32 < p.M;      // warp-uniform: any of this warp's 32 rows inside the matrix
+      if (n0 + cbeg < p.N) {
+#pragma unroll 1
+        for (int cc = 0; cc < CPW; cc += 32) {
+          const int c0 = cbeg + cc;
+          if (n0 + c0 >= p.N) break;  // warp-uniform
+          uint32_t r[32];
+          if (!empty_k) {
+            tc_ld32(tmem_base + ab * BN + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; j++) r[j] = 0u;
+          }
+          if (f32 || (cc & 63) == 0) {
+            sbuf ^= 1;
+            if (lane == 0 && store_pending) tma_store_wait_read1();
+            __syncwarp();
+          }
+          const uint32_t stage = stage0 + sbuf * 4096;
+          const uint32_t my_row = stage + lane * 128;
+#pragma unroll
+          for (int g8 = 0; g8 < 4; g8++) {
+            float v[8];
+#pragma unroll
+            for (int j = 0; j < 8; j++) v[j] = __uint_as_float(r[g8 * 8 + j]);
+            if (p.plain == 2) {
+              const float4 b0 = *reinterpret_cast<const float4*>(bias_s + cc + g8 * 8);
+              const float4 b1 = *reinterpret_cast<const float4*>(bias_s + cc + g8 * 8 + 4);
+              v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w;
+              v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+            }
+            if (f32) {
+              const uint32_t s0 = my_row + (((2 * g8) ^ (lane & 7)) << 4), s1 = my_row + (((2 * g8 + 1) ^ (lane & 7)) << 4);
+              st_shared_v4(s0, __float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]));
+              st_shared_v4(s1, __float_as_uint(v[4]), __float_as_uint(v[5]), __float_as_uint(v[6]), __float_as_uint(v[7]));
+            } else {
+              const uint32_t s0 = my_row + (((((cc & 63) >> 3) + g8) ^ (lane & 7)) << 4);
+              st_shared_v4(s0, pack2(v[0], v[1]), pack2(v[2], v[3]), pack2(v[4], v[5]), pack2(v[6], v[7]));
+            }
+          }
+          const bool last_chunk = (cc & 63) == 32 || n0 + c0 + 32 >= p.N;
+          if (f32 || last_chunk) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0 && rows_in) {
+              const int x = f32 ? n0 + c0 : n0 + cbeg + (cc & ~63), y = m0 + q * 32;
+              if (p.splits > 1) tma_store_3d(&map_c, stage, x, y, split);
+              else tma_store_2d(&map_c, stage, x, y);
+              tma_store_commit();
+              store_pending = true;
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {   // accumulator drained: tell the leader's MMA thread
+        if (leader) mbar_arrive(tempty_bar(ab));
+        else mbar_arrive_cluster(ab ? ltempty1 : ltempty0);
+      }
+    }
+    if (lane == 0 && store_pending) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  }
+
+  // Neither CTA may leave (or free its TMEM) while the other can still read its shared memory,
+  // write its TMEM or signal its barriers.
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+  }
 }
 
 typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -692,19 +970,49 @@ cudaError_t launch_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int 
   const long long total = (long long)((g.N + BN - 1) / BN) * ((g.M + BM - 1) / BM) * g.splits;
   long long cap = (max_ctas > 0 && max_ctas < num_sms) ? max_ctas : num_sms;
   dim3 grid((unsigned)(total < cap ? total : cap));
-  CUtensorMap ma, mb, mc, mp;
+  CUtensorMap ma, mb, mc;
   static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
   memcpy(&ma, plan.map_a, sizeof(ma));
   memcpy(&mb, plan.map_b, sizeof(mb));
   memcpy(&mc, plan.map_c, sizeof(mc));
-  memcpy(&mp, plan.map_p, sizeof(mp));
   p.tma_c = plan.tma_c;
-  p.tma_p = plan.tma_p;
   const Epilogue& e = g.epi;
   const bool no_aux = e.alpha == 1.f && e.act == ACT_NONE && !e.pre_out && !e.mul && !e.res && e.dact == ACT_NONE;
   p.plain = no_aux ? (e.bias ? (g.splits == 1 ? 2 : 1) : 1) : 0;   // 1: identity, 2: bias only, 0: general
   if (total <= (long long)grid.x) p.sched = nullptr;   // one tile per CTA: nothing to balance
-  tc_gemm_kernel<BN, A_MN, B_MN, GENERAL><<<grid, TC_THREADS, smem, s>>>(ma, mb, mc, mp, p);
+  tc_gemm_kernel<BN, A_MN, B_MN, GENERAL><<<grid, TC_THREADS, smem, s>>>(ma, mb, mc, p);
+  return cudaGetLastError();
+}
+
+template <bool A_MN, bool B_MN>
+cudaError_t launch_pair_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas) {
+  constexpr size_t smem = (size_t)PAIR_STAGES * PAIR_STAGE_BYTES + EPI_WARPS * (EPI_STAGE_BYTES + EPI_BIAS_BYTES) + 8 * (2 * PAIR_STAGES + 16) + 1024;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(tc_gemm_pair_kernel<A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  TcArgs p;
+  p.M = g.M; p.N = g.N; p.K = g.K;
+  p.C = g.C; p.ldc = g.ldc; p.c_f32 = g.c_f32;
+  p.splits = g.splits; p.ws = g.ws; p.epi = g.epi; p.status = plan.status; p.dbg = plan.dbg; p.sched = nullptr;
+  p.tma_c = 1;
+  p.plain = (g.epi.bias && g.splits == 1) ? 2 : 1;
+  static int num_sms = 0;
+  if (num_sms == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms < 2) num_sms = 148;
+  }
+  const long long total = (long long)((g.N + PAIR_BN - 1) / PAIR_BN) * ((g.M + 2 * BM - 1) / (2 * BM)) * g.splits;
+  long long cap = ((max_ctas > 1 && max_ctas < num_sms) ? max_ctas : num_sms) / 2;
+  dim3 grid(2u * (unsigned)(total < cap ? total : cap));
+  CUtensorMap ma, mb, mc;
+  memcpy(&ma, plan.map_a, sizeof(ma));
+  memcpy(&mb, plan.b_mn ? plan.map_b : plan.map_b_half, sizeof(mb));
+  memcpy(&mc, plan.map_c, sizeof(mc));
+  tc_gemm_pair_kernel<A_MN, B_MN><<<grid, TC_THREADS, smem, s>>>(ma, mb, mc, p, (uint32_t)plan.pair_tmem_cols);
   return cudaGetLastError();
 }
 
@@ -734,6 +1042,18 @@ bool tc_gemm_supported(const GemmArgs& g) {
   if (!operand_ok(g.A, g.sa_m, g.sa_k) || !operand_ok(g.B, g.sb_n, g.sb_k)) return false;
   // a [1 x K] operand is ambiguous (both strides may be 1): leave such GEMVs to the SIMT kernel
   if ((g.sa_m == 1 && g.sa_k == 1) || (g.sb_n == 1 && g.sb_k == 1)) return false;
+  // the fused epilogue reads its auxiliary operands as aligned 16-byte pieces of 8 columns, and keeps
+  // one register set for "multiplier or activation-derivative source"
+  const Epilogue& e = g.epi;
+  if (g.splits == 1 && (e.pre_out || e.act == ACT_GELU || e.dact == ACT_GELU)) return false;   // SIMT kernel
+  if (g.splits == 1 && (e.mul || e.res || e.dact != ACT_NONE)) {
+    if (e.mul && e.dact != ACT_NONE) return false;
+    const long long ld = e.ld_aux ? e.ld_aux : g.N;
+    if (ld % 8 != 0 || g.N % 8 != 0) return false;
+    const void* aux[3] = {e.mul, e.res, e.dact != ACT_NONE ? e.dact_src : nullptr};
+    for (const void* a : aux)
+      if (a && (reinterpret_cast<uintptr_t>(a) & 15)) return false;
+  }
   return true;
 }
 
@@ -756,8 +1076,7 @@ bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan) {
   if (!ok) return false;
   // outputs through TMA stores where their layout allows it (else the kernel stores directly)
   memset(plan->map_c, 0, sizeof(plan->map_c));
-  memset(plan->map_p, 0, sizeof(plan->map_p));
-  plan->tma_c = plan->tma_p = 0;
+  plan->tma_c = 0;
   if (g.splits > 1) {
     cuuint64_t dims[3] = {(cuuint64_t)g.N, (cuuint64_t)g.M, (cuuint64_t)g.splits};
     cuuint64_t str[2] = {(cuuint64_t)g.N * 4, (cuuint64_t)g.M * g.N * 4};
@@ -774,17 +1093,30 @@ bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan) {
     cuuint32_t box[2] = {64u, 32u};
     plan->tma_c = encode_map(plan->map_c, g.C, false, 2, dims, str, box) ? 1 : 0;
   }
-  if (g.splits == 1 && g.epi.pre_out) {
-    cuuint64_t dims[2] = {(cuuint64_t)g.N, (cuuint64_t)g.M};
-    cuuint64_t str[1] = {(cuuint64_t)g.epi.ld_aux * 2};
-    cuuint32_t box[2] = {64u, 32u};
-    plan->tma_p = encode_map(plan->map_p, g.epi.pre_out, false, 2, dims, str, box) ? 1 : 0;
+  // CTA-pair kernel (256 x 256 tiles over two SMs): identity / bias-only epilogue, TMA-stored output
+  plan->pair = 0;
+  {
+    static const int env_pair = getenv("ERASE_TC_PAIR") ? atoi(getenv("ERASE_TC_PAIR")) : 1;
+    static const int env_cols = getenv("ERASE_TC_PAIR_COLS") ? atoi(getenv("ERASE_TC_PAIR_COLS")) : 512;
+    plan->pair_tmem_cols = env_cols == 256 ? 256 : 512;
+    const bool simple = epilogue_is_simple(g);
+    if (env_pair && simple && plan->tma_c && plan->bn == 256 && g.M >= 256) {
+      bool okp = true;
+      if (!plan->b_mn) okp = encode_2d(plan->map_b_half, g.B, g.K, g.N, g.sb_n, PAIR_BN / 2);
+      plan->pair = okp ? 1 : 0;
+    }
   }
   return true;
 }
 
 cudaError_t tc_gemm_launch(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas) {
   const bool simple = epilogue_is_simple(g);
+  if (plan.pair) {
+    if (!plan.a_mn && !plan.b_mn) return launch_pair_t<false, false>(g, plan, s, max_ctas);
+    if (!plan.a_mn && plan.b_mn) return launch_pair_t<false, true>(g, plan, s, max_ctas);
+    if (plan.a_mn && !plan.b_mn) return launch_pair_t<true, false>(g, plan, s, max_ctas);
+    return launch_pair_t<true, true>(g, plan, s, max_ctas);
+  }
   switch (plan.bn) {
     case 64: return simple ? launch_bn<64, false>(g, plan, s, max_ctas) : launch_bn<64, true>(g, plan, s, max_ctas);
     case 256: return simple ? launch_bn<256, false>(g, plan, s, max_ctas) : launch_bn<256, true>(g, plan, s, max_ctas);

@@ -15,8 +15,10 @@ struct TcPlan {
   unsigned char map_a[128];  // CUtensorMap of A (copied into an aligned object at launch)
   unsigned char map_b[128];  // CUtensorMap of B
   unsigned char map_c[128];  // CUtensorMap of the output (or of the split-K partials), if tma_c
-  unsigned char map_p[128];  // CUtensorMap of the pre-activation copy, if tma_p
-  int tma_c = 0, tma_p = 0;
+  unsigned char map_b_half[128];  // CTA-pair kernel, K-major B: box of 128 rows (each CTA stages half of the 256 columns)
+  int tma_c = 0;
+  int pair = 0;       // run the CTA-pair kernel (tcgen05 cta_group::2, 256 x 256 tiles)
+  int pair_tmem_cols = 512;
   int bn = 128;       // tile width (N)
   int a_mn = 0;       // A is contiguous along M (not along K)
   int b_mn = 0;
