@@ -331,8 +331,9 @@ struct Builder {
   void gemm_inner(OpList& ops, GemmArgs g) {
     const bool bf = m->bf16;
     const bool tc_ok = bf && tc_gemm_supported(g);
-    float* out = (float*)g.C;
+    void* out = g.C;
     const long long ldo = g.ldc;
+    const bool out_bf = bf && !g.c_f32;   // split-K partials are summed in fp32 and rounded once
     if (g.splits > 1) g.ws = f32_buf((size_t)g.splits * g.M * g.N);
     TcPlan plan;
     int* sched = tc_ok ? (int*)dev_alloc(m, 2 * sizeof(int), &ok) : nullptr;   // dynamic tile scheduler words (zeroed)
@@ -340,20 +341,20 @@ struct Builder {
     plan.sched = sched;
     if (use_tc) {
       if (g.splits > 1)
-        ops.push_back({[g, plan, out, ldo, mm = m](cudaStream_t s) {
+        ops.push_back({[g, plan, out, ldo, out_bf, mm = m](cudaStream_t s) {
                          cudaError_t e = tc_gemm_launch(g, plan, s, mm->sm_budget);
                          if (e != cudaSuccess) return e;
-                         return splitk_reduce(g.ws, g.splits, (long long)g.M * g.N, g.N, out, ldo, s);
+                         return splitk_reduce(g.ws, g.splits, (long long)g.M * g.N, g.N, out, ldo, s, out_bf);
                        }, 2});
       else
         ops.push_back({[g, plan, mm = m](cudaStream_t s) { return tc_gemm_launch(g, plan, s, mm->sm_budget); }, 1});
       return;
     }
     if (g.splits > 1) {
-      ops.push_back({[g, bf, out, ldo](cudaStream_t s) {
+      ops.push_back({[g, bf, out, ldo, out_bf](cudaStream_t s) {
                        cudaError_t e = gemm_simt(g, bf, s);
                        if (e != cudaSuccess) return e;
-                       return splitk_reduce(g.ws, g.splits, (long long)g.M * g.N, g.N, out, ldo, s);
+                       return splitk_reduce(g.ws, g.splits, (long long)g.M * g.N, g.N, out, ldo, s, out_bf);
                      }, 2});
     } else {
       ops.push_back({[g, bf](cudaStream_t s) { return gemm_simt(g, bf, s); }, 1});
@@ -396,6 +397,17 @@ struct Builder {
     g.C = dX; g.ldc = K;
     if (e.ld_aux == 0) e.ld_aux = K;
     g.epi = e;
+    // A narrow dX (few output tiles) with a long contraction leaves most SMs idle and each busy one
+    // bound by what a single SM can pull from L2: split the contraction over CTA pairs instead
+    // (fp32 partials, summed in a fixed order and rounded once).
+    const bool plain = !e.bias && e.act == ACT_NONE && !e.mul && !e.res && e.dact == ACT_NONE && !e.pre_out && e.alpha == 1.f;
+    if (m->bf16 && plain && M >= 256 && K >= 256 && N >= 2048) {
+      const long long pair_tiles = (long long)((M + 255) / 256) * ((K + 255) / 256);
+      int splits = (int)(74 / pair_tiles);
+      if (splits > N / 1024) splits = N / 1024;
+      if (splits > 8) splits = 8;
+      if (splits > 1) g.splits = splits;
+    }
     gemm_tag = "gemm_dgrad";
     gemm(ops, g);
   }

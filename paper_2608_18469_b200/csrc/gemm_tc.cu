@@ -1064,6 +1064,11 @@ bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan) {
   // tile width: 256 halves the A-operand traffic per FLOP, taken when it still leaves every SM a tile
   const long long tiles256 = (long long)((g.M + BM - 1) / BM) * ((g.N + 255) / 256) * g.splits;
   plan->bn = g.N <= 64 ? 64 : (g.N >= 256 && tiles256 >= 148 ? 256 : 128);
+  // CTA-pair kernel (256 x 256 tiles over two SMs) when its tiles keep most of the 74 pairs busy
+  static const int env_pair = getenv("ERASE_TC_PAIR") ? atoi(getenv("ERASE_TC_PAIR")) : 1;
+  const long long pair_tiles = (long long)((g.M + 2 * BM - 1) / (2 * BM)) * ((g.N + PAIR_BN - 1) / PAIR_BN) * g.splits;
+  const bool want_pair = env_pair && epilogue_is_simple(g) && g.M >= 256 && g.N > 128 && pair_tiles >= 56;
+  if (want_pair) plan->bn = 256;
   if (getenv("ERASE_TC_BN")) { int f = atoi(getenv("ERASE_TC_BN")); if ((f == 64 || f == 128 || f == 256) && f <= (g.N + 63) / 64 * 64) plan->bn = f; }
   plan->status = status;
   plan->launches = 1;
@@ -1096,11 +1101,9 @@ bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan) {
   // CTA-pair kernel (256 x 256 tiles over two SMs): identity / bias-only epilogue, TMA-stored output
   plan->pair = 0;
   {
-    static const int env_pair = getenv("ERASE_TC_PAIR") ? atoi(getenv("ERASE_TC_PAIR")) : 1;
     static const int env_cols = getenv("ERASE_TC_PAIR_COLS") ? atoi(getenv("ERASE_TC_PAIR_COLS")) : 512;
     plan->pair_tmem_cols = env_cols == 256 ? 256 : 512;
-    const bool simple = epilogue_is_simple(g);
-    if (env_pair && simple && plan->tma_c && plan->bn == 256 && g.M >= 256) {
+    if (want_pair && plan->tma_c && plan->bn == 256) {
       bool okp = true;
       if (!plan->b_mn) okp = encode_2d(plan->map_b_half, g.B, g.K, g.N, g.sb_n, PAIR_BN / 2);
       plan->pair = okp ? 1 : 0;

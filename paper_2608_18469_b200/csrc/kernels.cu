@@ -145,19 +145,58 @@ cudaError_t gemm_simt(const GemmArgs& g, bool bf16, cudaStream_t s) {
   return bf16 ? gemm_simt_t<bf16_t>(g, s) : gemm_simt_t<float>(g, s);
 }
 
+template <bool BF16_OUT>
 __global__ void splitk_reduce_kernel(const float* __restrict__ ws, int splits, long long mn, int N,
-                                     float* __restrict__ out, long long ldo) {
+                                     void* __restrict__ out, long long ldo) {
   long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= mn) return;
   float a = 0.f;
   for (int s = 0; s < splits; s++) a += ws[(long long)s * mn + i];
-  out[(i / N) * ldo + (i % N)] = a;
+  const long long o = (i / N) * ldo + (i % N);
+  if (BF16_OUT) ((bf16_t*)out)[o] = __float2bfloat16_rn(a);
+  else ((float*)out)[o] = a;
 }
 
-cudaError_t splitk_reduce(const float* ws, int splits, long long mn, int N, float* out, long long ldo,
-                          cudaStream_t s) {
+// four adjacent columns per thread (N, ldo multiples of 4); the partials of up to four splits are in flight at once
+template <bool BF16_OUT>
+__global__ void splitk_reduce_v4_kernel(const float4* __restrict__ ws, int splits, long long mn4, int N4,
+                                        void* __restrict__ out, long long ldo) {
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= mn4) return;
+  float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s0 = 0; s0 < splits; s0 += 4) {
+    float4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; u++) v[u] = s0 + u < splits ? __ldcs(ws + (long long)(s0 + u) * mn4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int u = 0; u < 4; u++)
+      if (s0 + u < splits) { a.x += v[u].x; a.y += v[u].y; a.z += v[u].z; a.w += v[u].w; }
+  }
+  const long long o = (i / N4) * ldo + (i % N4) * 4;
+  if (BF16_OUT) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(a.x, a.y), hi = __floats2bfloat162_rn(a.z, a.w);
+    uint2 q;
+    q.x = *reinterpret_cast<uint32_t*>(&lo);
+    q.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>((bf16_t*)out + o) = q;
+  } else {
+    *reinterpret_cast<float4*>((float*)out + o) = a;
+  }
+}
+
+cudaError_t splitk_reduce(const float* ws, int splits, long long mn, int N, void* out, long long ldo,
+                          cudaStream_t s, bool out_bf16) {
   if (mn <= 0) return cudaSuccess;
-  splitk_reduce_kernel<<<cdiv(mn, 256), 256, 0, s>>>(ws, splits, mn, N, out, ldo);
+  const bool vec = N % 4 == 0 && ldo % 4 == 0 && (reinterpret_cast<uintptr_t>(ws) & 15) == 0 &&
+                   (reinterpret_cast<uintptr_t>(out) & 15) == 0;
+  if (vec) {
+    const long long mn4 = mn / 4;
+    if (out_bf16) splitk_reduce_v4_kernel<true><<<cdiv(mn4, 256), 256, 0, s>>>((const float4*)ws, splits, mn4, N / 4, out, ldo);
+    else splitk_reduce_v4_kernel<false><<<cdiv(mn4, 256), 256, 0, s>>>((const float4*)ws, splits, mn4, N / 4, out, ldo);
+  } else {
+    if (out_bf16) splitk_reduce_kernel<true><<<cdiv(mn, 256), 256, 0, s>>>(ws, splits, mn, N, out, ldo);
+    else splitk_reduce_kernel<false><<<cdiv(mn, 256), 256, 0, s>>>(ws, splits, mn, N, out, ldo);
+  }
   return cudaGetLastError();
 }
 

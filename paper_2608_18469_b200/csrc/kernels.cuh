@@ -48,8 +48,9 @@ struct GemmArgs {
 };
 
 cudaError_t gemm_simt(const GemmArgs& g, bool bf16, cudaStream_t s);
-cudaError_t splitk_reduce(const float* ws, int splits, long long mn, int N, float* out, long long ldo,
-                          cudaStream_t s);
+// out: float, or bfloat16 when out_bf16 (the sum is rounded once, after the last partial)
+cudaError_t splitk_reduce(const float* ws, int splits, long long mn, int N, void* out, long long ldo,
+                          cudaStream_t s, bool out_bf16 = false);
 
 // out[c] = colscale[c] * sum_r scale[r] * f(X[r, c]); X is [rows, cols] with row stride ldx,
 // f = identity or the derivative of activation `dact` evaluated at X; scale and colscale may be
