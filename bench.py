@@ -174,7 +174,10 @@ def run_gpu(args, spec, cfg_name):
     n_streams = args.n_streams if args.n_streams > 0 else nb + 1
     flags = 0 if args.no_graph else binding.GRAPH
     eflags = flags | (0 if args.loss_on_main else (binding.EARLY_HEAD | binding.BLOCK_OPT))
-    if args.split_bwd:
+    # chains of blocks: the parameter-gradient work of each B_b goes to a second stream per block
+    # (measured faster on C1, C2, C4, C5; not on C3, whose blocks already all run side by side)
+    split_bwd = not args.loss_on_main and not args.no_split_bwd and spec["topo"] == "chain"
+    if split_bwd:
         eflags |= binding.SPLIT_BWD
     units = units_per_step(spec)
 
@@ -318,7 +321,8 @@ def run_gpu(args, spec, cfg_name):
         "ms_per_step": era_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": spec["dtype"], "data": "synthetic",
         "config": {"workload": workload_name(cfg_name, spec), "n_streams": n_streams,
-                   "schedule": "ERASE, local head+loss+backward+optimizer of each block released onto side streams after the block body"
+                   "schedule": ("ERASE, local head+loss+backward+optimizer of each block released onto side streams after the block body"
+                                + (", parameter-gradient work of each backward on a second stream per block" if split_bwd else ""))
                                if not args.loss_on_main else "ERASE, backward released after forward and local loss",
                    "cuda_graph": not args.no_graph, "batch_pool": POOL,
                    "l2": f"no flush: the step's working set ({arena_mb:.0f} MiB of stashes, logits, parameters) exceeds the 126 MB L2",
@@ -358,7 +362,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--loss-on-main", action="store_true", help="paper's placement of the local loss")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--split-bwd", action="store_true", help="parameter-gradient work of each B_b on a second stream")
+    ap.add_argument("--no-split-bwd", action="store_true",
+                    help="keep the parameter-gradient work of each B_b on the block's own side stream")
     args = ap.parse_args()
     if args.impl == "ours":
         # at least 3 warm-up steps; with graph replay at least one per pooled batch, so that every

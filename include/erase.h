@@ -151,6 +151,12 @@ typedef struct {
                             step, so this is the overlap of Section 2.2 applied one level down.  Same
                             kernels on the same values: same bits.                                    */
 
+#define ERASE_STAMPS 32u  /* record the phase timeline of this step with device clock stamps (a one-thread
+                            kernel per phase boundary) instead of CUDA events, which cannot be captured:
+                            with ERASE_GRAPH the stamps are part of the graph, and erase_timeline then
+                            shows how the phases of a REPLAYED step overlap.  A measuring aid: it adds
+                            2*(2*n_blocks+1)+1 tiny kernels to the step.                               */
+
 /* Device bytes erase_create needs for this spec when given an arena; 0 if the spec is invalid. */
 ERASE_API size_t erase_arena_bytes(const erase_model_spec* spec);
 
@@ -209,8 +215,10 @@ ERASE_API int64_t erase_launch_count(const erase_model* m);
 
 /* Device-side begin/end times of the last step's phases, in milliseconds relative to the step's
  * start, from CUDA events: out[2*b], out[2*b+1] = start and end of F_b for b < n_blocks, then
- * the same for B_b, then for the optimizer: 2*(2*n_blocks+1) floats.  Only recorded for steps
- * run without ERASE_GRAPH.  Waits for the step.  Errors: EINVAL, ESTATE (no such step). */
+ * the same for B_b, then for the optimizer: 2*(2*n_blocks+1) floats.  Recorded for steps run
+ * without ERASE_GRAPH (CUDA events) and for steps run with ERASE_STAMPS (device clock stamps,
+ * graph replay included).  With ERASE_BLOCK_OPT the optimizer entries bracket the join only.
+ * Waits for the step.  Errors: EINVAL, ESTATE (no such step). */
 ERASE_API erase_status erase_timeline(erase_model* m, float* out, int32_t n);
 
 /* The GEMM the block linears are made of, on its own (paper Section 1: the "small GEMMs" of proxy

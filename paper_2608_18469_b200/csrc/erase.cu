@@ -88,6 +88,8 @@ struct erase_model {
   cudaStream_t main = nullptr;
   std::vector<cudaStream_t> side;
   std::vector<cudaEvent_t> ev_f, ev_b;
+  unsigned long long* stamps = nullptr;            // device clock stamps of the phase boundaries (ERASE_STAMPS)
+  bool timeline_stamps = false;
   std::vector<cudaStream_t> leaf;                 // second side stream per block (ERASE_SPLIT_BWD)
   std::vector<std::vector<cudaEvent_t>> ev_leaf;  // per block: one event per chain->leaf hand-over, plus the join
   cudaEvent_t ev_opt = nullptr;
@@ -424,6 +426,13 @@ struct Builder {
     int maxs = M / 64 > 0 ? M / 64 : 1;
     if (splits > maxs) splits = maxs;
     if (splits > 64) splits = 64;
+    // wide enough for 256 x 256 tiles over CTA pairs: split so that one wave of the 74 pairs is nearly full
+    if (m->bf16 && N >= 256 && K > 128) {
+      const long long pt = (long long)((N + 255) / 256) * ((K + 255) / 256);
+      const int s_lo = (int)(74 / pt);
+      static const int pair_min = getenv("ERASE_WGRAD_PAIR_MIN") ? atoi(getenv("ERASE_WGRAD_PAIR_MIN")) : 66;
+      if (s_lo >= 1 && pt * s_lo >= pair_min && s_lo <= M / 512 && s_lo <= 16) splits = s_lo;
+    }
     g.splits = splits < 1 ? 1 : splits;
     gemm_tag = "gemm_wgrad";
     const size_t before = ops.size();
@@ -743,6 +752,7 @@ struct Builder {
     m->tick = (double*)dev_alloc(m, 3 * sizeof(double), &ok);
     m->status = (int*)dev_alloc(m, sizeof(int), &ok);
     m->losses = f32_buf(m->B);
+    m->stamps = (unsigned long long*)dev_alloc(m, (size_t)(2 * (2 * m->B + 1) + 1) * sizeof(unsigned long long), &ok);
     // z_0
     // z_0: dense batches are copied into a model-owned buffer (so every block reads memory whose
     // address is fixed at build time); token and CTR batches are gathered from the frozen tables.
@@ -859,12 +869,17 @@ cudaError_t run_ops(erase_model* m, OpList& ops, cudaStream_t s) {
   return cudaSuccess;
 }
 
-// Enqueue one step.  `timed` adds the per-phase timing events (never while capturing).
-erase_status enqueue_step(erase_model* m, int n_streams, unsigned flags, bool timed) {
+// timed: 0 no timeline, 1 CUDA events (never while capturing), 2 device clock stamps written by
+// one-thread kernels (these can be captured, so the timeline of a graph replay can be read).
+erase_status enqueue_step(erase_model* m, int n_streams, unsigned flags, int timed) {
   const int B = m->B;
   const bool do_opt = !(flags & ERASE_NO_OPT);
-  auto tev = [&](int i) { return m->ev_time[i]; };
-  if (timed) CK(cudaEventRecord(tev(2 * (2 * B + 1)), m->main));
+  auto mark = [&](int i, cudaStream_t st) -> cudaError_t {
+    if (timed == 1) return cudaEventRecord(m->ev_time[i], st);
+    if (timed == 2) { m->launches += 1; return stamp_time(m->stamps + i, st); }
+    return cudaSuccess;
+  };
+  CK(mark(2 * (2 * B + 1), m->main));
   CK(run_ops(m, m->stage, m->main));
   const bool early_head = (flags & ERASE_EARLY_HEAD) != 0;
   // per-block optimizer: theta_b is read by F_b and B_b only, so it can be updated right behind B_b
@@ -873,15 +888,15 @@ erase_status enqueue_step(erase_model* m, int n_streams, unsigned flags, bool ti
   if (block_opt) CK(run_ops(m, m->opt_tick_op, m->main));
   if (n_streams <= 1) {
     for (int b = 0; b < B; b++) {
-      if (timed) CK(cudaEventRecord(tev(2 * b), m->main));
+      CK(mark(2 * b, m->main));
       CK(run_ops(m, m->fwd[b], m->main));
       CK(run_ops(m, m->hfwd[b], m->main));
-      if (timed) CK(cudaEventRecord(tev(2 * b + 1), m->main));
+      CK(mark(2 * b + 1, m->main));
     }
     for (int b = B - 1; b >= 0; b--) {
-      if (timed) CK(cudaEventRecord(tev(2 * (B + b)), m->main));
+      CK(mark(2 * (B + b), m->main));
       CK(run_ops(m, m->bwd[b], m->main));
-      if (timed) CK(cudaEventRecord(tev(2 * (B + b) + 1), m->main));
+      CK(mark(2 * (B + b) + 1, m->main));
     }
   } else {
     const int ns = n_streams - 1;
@@ -892,14 +907,14 @@ erase_status enqueue_step(erase_model* m, int n_streams, unsigned flags, bool ti
     const int budget_main = env_main, budget_side = env_side;
     for (int b = 0; b < B; b++) {
       m->sm_budget = budget_main;
-      if (timed) CK(cudaEventRecord(tev(2 * b), m->main));
+      CK(mark(2 * b, m->main));
       CK(run_ops(m, m->fwd[b], m->main));
       if (!early_head) CK(run_ops(m, m->hfwd[b], m->main));
-      if (timed) CK(cudaEventRecord(tev(2 * b + 1), m->main));
+      CK(mark(2 * b + 1, m->main));
       CK(cudaEventRecord(m->ev_f[b], m->main));          // F_b (and l_b) are enqueued: release B_b
       cudaStream_t sd = m->side[b % ns];
       CK(cudaStreamWaitEvent(sd, m->ev_f[b], 0));
-      if (timed) CK(cudaEventRecord(tev(2 * (B + b)), sd));
+      CK(mark(2 * (B + b), sd));
       m->sm_budget = budget_side;
       if (early_head) CK(run_ops(m, m->hfwd[b], sd));    // z_b's only other consumer is F_{b+1}, which does not wait
       if (!split_bwd) {
@@ -931,16 +946,16 @@ erase_status enqueue_step(erase_model* m, int n_streams, unsigned flags, bool ti
         CK(cudaEventRecord(e, lf));
         CK(cudaStreamWaitEvent(sd, e, 0));
       }
-      if (timed) CK(cudaEventRecord(tev(2 * (B + b) + 1), sd));
+      CK(mark(2 * (B + b) + 1, sd));
       if (block_opt) CK(run_ops(m, m->opt_blk[b], sd));
       CK(cudaEventRecord(m->ev_b[b], sd));
     }
     for (int b = 0; b < B; b++) CK(cudaStreamWaitEvent(m->main, m->ev_b[b], 0));  // join
     m->sm_budget = 0;
   }
-  if (timed) CK(cudaEventRecord(tev(4 * B), m->main));
+  CK(mark(4 * B, m->main));
   if (do_opt && !block_opt) CK(run_ops(m, m->opt, m->main));
-  if (timed) CK(cudaEventRecord(tev(4 * B + 1), m->main));
+  CK(mark(4 * B + 1, m->main));
   return ERASE_OK;
 }
 
@@ -1128,7 +1143,8 @@ static erase_status check_step_args(erase_model* m, const erase_batch* batch);
 erase_status erase_step_ex(erase_model* m, const erase_batch* batch, int32_t n_streams, uint32_t flags) {
   if (!m) return ERASE_EINVAL;
   if (n_streams < 1) return m->fail(ERASE_EINVAL, "erase_step: n_streams must be >= 1");
-  if (flags & ~(ERASE_GRAPH | ERASE_NO_OPT | ERASE_EARLY_HEAD | ERASE_BLOCK_OPT | ERASE_SPLIT_BWD)) return m->fail(ERASE_EINVAL, "erase_step: unknown flag");
+  if (flags & ~(ERASE_GRAPH | ERASE_NO_OPT | ERASE_EARLY_HEAD | ERASE_BLOCK_OPT | ERASE_SPLIT_BWD | ERASE_STAMPS)) return m->fail(ERASE_EINVAL, "erase_step: unknown flag");
+  const int stamp_mode = (flags & ERASE_STAMPS) ? 2 : 0;
   erase_status cst = check_step_args(m, batch);
   if (cst != ERASE_OK) return cst;
   if (n_streams > m->B + 1) n_streams = m->B + 1;
@@ -1139,7 +1155,7 @@ erase_status erase_step_ex(erase_model* m, const erase_batch* batch, int32_t n_s
     if (it == m->graphs.end()) {
       int64_t before = m->launches;
       CK(cudaStreamBeginCapture(m->main, cudaStreamCaptureModeThreadLocal));
-      erase_status st = enqueue_step(m, n_streams, flags, false);
+      erase_status st = enqueue_step(m, n_streams, flags, stamp_mode);
       cudaGraph_t graph = nullptr;
       cudaError_t e = cudaStreamEndCapture(m->main, &graph);
       const int64_t captured = m->launches - before;
@@ -1154,11 +1170,13 @@ erase_status erase_step_ex(erase_model* m, const erase_batch* batch, int32_t n_s
     }
     CK(cudaGraphLaunch(it->second.first, m->main));
     m->launches += it->second.second;
-    m->timeline_valid = false;
+    m->timeline_valid = stamp_mode != 0;
+    m->timeline_stamps = true;
   } else {
-    erase_status st = enqueue_step(m, n_streams, flags, true);
+    erase_status st = enqueue_step(m, n_streams, flags, stamp_mode ? 2 : 1);
     if (st != ERASE_OK) return st;
     m->timeline_valid = true;
+    m->timeline_stamps = stamp_mode != 0;
   }
   m->stepped = true;
   return ERASE_OK;
@@ -1244,6 +1262,12 @@ erase_status erase_timeline(erase_model* m, float* out, int32_t n) {
   if (!m->timeline_valid) return m->fail(ERASE_ESTATE, "erase_timeline: the last step recorded no timeline");
   erase_status st = erase_sync(m);
   if (st != ERASE_OK) return st;
+  if (m->timeline_stamps) {
+    std::vector<unsigned long long> h(need + 1);
+    CK(copy_sync(m, h.data(), m->stamps, h.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+    for (int i = 0; i < need; i++) out[i] = (float)((double)((long long)h[i] - (long long)h[need]) * 1e-6);   // ns -> ms
+    return ERASE_OK;
+  }
   for (int i = 0; i < need; i++) CK(cudaEventElapsedTime(&out[i], m->ev_time[need], m->ev_time[i]));
   return ERASE_OK;
 }

@@ -612,8 +612,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 //   tfull[a]   per CTA: accumulator a is complete (delivered to both CTAs)
 //   tempty[a]  leader only: both CTAs' epilogue warps have drained accumulator a (the peer's warps
 //              arrive on it through the cluster's shared-memory window)
-// Tiles are assigned round-robin to clusters, in the order of tile_coords.  Only the identity /
-// bias-only epilogue with TMA-stored output is implemented; other GEMMs use tc_gemm_kernel.
+// Tiles are assigned round-robin to clusters, in the order of tile_coords.  The output must be
+// describable to TMA (it leaves through staged TMA stores); GENERAL as in tc_gemm_kernel.
 constexpr int PAIR_BN = 256;
 constexpr int PAIR_STAGES = 4;
 constexpr uint32_t PAIR_STAGE_BYTES = 2u * BM * BK * 2u;   // 128 x 64 of A + 128 x 64 of B, bf16
@@ -656,7 +656,7 @@ __device__ __forceinline__ void tc_mma_pair(uint32_t tmem_d, uint64_t adesc, uin
       : "memory");
 }
 
-template <bool A_MN, bool B_MN>
+template <bool A_MN, bool B_MN, bool GENERAL>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     const __grid_constant__ CUtensorMap map_c, const __grid_constant__ TcArgs p, const uint32_t tmem_cols) {
@@ -812,7 +812,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       const int kbeg = split * kchunk, kend = min(p.K, kbeg + kchunk);
       const bool empty_k = kend <= kbeg;
       const uint32_t ab = naccum == 2 ? (lt & 1) : 0u, aph = naccum == 2 ? ((lt >> 1) & 1) : (lt & 1);
-      if (p.plain == 2) {
+      if (p.epi.bias && p.splits == 1) {
         __syncwarp();
         for (int j = lane; j < CPW; j += 32) {
           const int n = n0 + cbeg + j;
@@ -820,6 +820,20 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         }
         __syncwarp();
       }
+      const int row = m0 + q * 32 + lane;
+      const bool row_ok = row < p.M;
+      // auxiliary operands of this thread's row (raw bf16), fetched one 32-column chunk ahead
+      const __nv_bfloat16* aux_pa = nullptr;
+      const __nv_bfloat16* aux_pb = nullptr;
+      Aux32 aux_cur, aux_nxt;
+      if (GENERAL && !p.plain && p.splits == 1) {
+        const long long ro = (long long)row * p.epi.ld_aux;
+        if (p.epi.res) aux_pa = (const __nv_bfloat16*)p.epi.res + ro;
+        const void* bsrc = p.epi.mul ? p.epi.mul : (p.epi.dact != ACT_NONE ? p.epi.dact_src : nullptr);
+        if (bsrc) aux_pb = (const __nv_bfloat16*)bsrc + ro;
+        if (n0 + cbeg < p.N && (aux_pa || aux_pb)) aux_issue(aux_pa, aux_pb, row_ok, n0 + cbeg, p.N, aux_nxt);
+      }
+      const bool use_aux = GENERAL && (aux_pa || aux_pb);
       bool ok = mbar_wait(tfull_bar(ab), aph);
       if (!ok) atomicExch(p.status, 3);
       ok = __all_sync(0xffffffffu, ok);
@@ -831,6 +845,10 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         for (int cc = 0; cc < CPW; cc += 32) {
           const int c0 = cbeg + cc;
           if (n0 + c0 >= p.N) break;  // warp-uniform
+          if (GENERAL && use_aux) {
+            aux_cur = aux_nxt;
+            if (cc + 32 < CPW && n0 + c0 + 32 < p.N) aux_issue(aux_pa, aux_pb, row_ok, n0 + c0 + 32, p.N, aux_nxt);
+          }
           uint32_t r[32];
           if (!empty_k) {
             tc_ld32(tmem_base + ab * BN + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
@@ -847,7 +865,8 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           const uint32_t my_row = stage + lane * 128;
 #pragma unroll
           for (int g8 = 0; g8 < 4; g8++) {
-            float v[8];
+            F8 f;
+            float* v = f.v;
 #pragma unroll
             for (int j = 0; j < 8; j++) v[j] = __uint_as_float(r[g8 * 8 + j]);
             if (p.plain == 2) {
@@ -855,6 +874,8 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
               const float4 b1 = *reinterpret_cast<const float4*>(bias_s + cc + g8 * 8 + 4);
               v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w;
               v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+            } else if (GENERAL && !p.plain && p.splits == 1 && row_ok && n0 + c0 + g8 * 8 < p.N) {
+              f = epilogue_values8(p, f, bias_s + cc + g8 * 8, aux_cur.a[g8], aux_cur.b[g8]);
             }
             if (f32) {
               const uint32_t s0 = my_row + (((2 * g8) ^ (lane & 7)) << 4), s1 = my_row + (((2 * g8 + 1) ^ (lane & 7)) << 4);
@@ -984,12 +1005,12 @@ cudaError_t launch_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int 
   return cudaGetLastError();
 }
 
-template <bool A_MN, bool B_MN>
+template <bool A_MN, bool B_MN, bool GENERAL>
 cudaError_t launch_pair_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas) {
   constexpr size_t smem = (size_t)PAIR_STAGES * PAIR_STAGE_BYTES + EPI_WARPS * (EPI_STAGE_BYTES + EPI_BIAS_BYTES) + 8 * (2 * PAIR_STAGES + 16) + 1024;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(tc_gemm_pair_kernel<A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(tc_gemm_pair_kernel<A_MN, B_MN, GENERAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -998,7 +1019,9 @@ cudaError_t launch_pair_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s,
   p.C = g.C; p.ldc = g.ldc; p.c_f32 = g.c_f32;
   p.splits = g.splits; p.ws = g.ws; p.epi = g.epi; p.status = plan.status; p.dbg = plan.dbg; p.sched = nullptr;
   p.tma_c = 1;
-  p.plain = (g.epi.bias && g.splits == 1) ? 2 : 1;
+  const Epilogue& e = g.epi;
+  const bool no_aux = e.alpha == 1.f && e.act == ACT_NONE && !e.pre_out && !e.mul && !e.res && e.dact == ACT_NONE;
+  p.plain = no_aux ? (e.bias ? (g.splits == 1 ? 2 : 1) : 1) : 0;   // 1: identity, 2: bias only, 0: general
   static int num_sms = 0;
   if (num_sms == 0) {
     int dev = 0;
@@ -1012,7 +1035,7 @@ cudaError_t launch_pair_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s,
   memcpy(&ma, plan.map_a, sizeof(ma));
   memcpy(&mb, plan.b_mn ? plan.map_b : plan.map_b_half, sizeof(mb));
   memcpy(&mc, plan.map_c, sizeof(mc));
-  tc_gemm_pair_kernel<A_MN, B_MN><<<grid, TC_THREADS, smem, s>>>(ma, mb, mc, p, (uint32_t)plan.pair_tmem_cols);
+  tc_gemm_pair_kernel<A_MN, B_MN, GENERAL><<<grid, TC_THREADS, smem, s>>>(ma, mb, mc, p, (uint32_t)plan.pair_tmem_cols);
   return cudaGetLastError();
 }
 
@@ -1067,7 +1090,7 @@ bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan) {
   // CTA-pair kernel (256 x 256 tiles over two SMs) when its tiles keep most of the 74 pairs busy
   static const int env_pair = getenv("ERASE_TC_PAIR") ? atoi(getenv("ERASE_TC_PAIR")) : 1;
   const long long pair_tiles = (long long)((g.M + 2 * BM - 1) / (2 * BM)) * ((g.N + PAIR_BN - 1) / PAIR_BN) * g.splits;
-  const bool want_pair = env_pair && epilogue_is_simple(g) && g.M >= 256 && g.N > 128 && pair_tiles >= 56;
+  const bool want_pair = env_pair && (epilogue_is_simple(g) || !plan->a_mn) && g.M >= 256 && g.N > 128 && pair_tiles >= 56;
   if (want_pair) plan->bn = 256;
   if (getenv("ERASE_TC_BN")) { int f = atoi(getenv("ERASE_TC_BN")); if ((f == 64 || f == 128 || f == 256) && f <= (g.N + 63) / 64 * 64) plan->bn = f; }
   plan->status = status;
@@ -1115,10 +1138,15 @@ bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan) {
 cudaError_t tc_gemm_launch(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas) {
   const bool simple = epilogue_is_simple(g);
   if (plan.pair) {
-    if (!plan.a_mn && !plan.b_mn) return launch_pair_t<false, false>(g, plan, s, max_ctas);
-    if (!plan.a_mn && plan.b_mn) return launch_pair_t<false, true>(g, plan, s, max_ctas);
-    if (plan.a_mn && !plan.b_mn) return launch_pair_t<true, false>(g, plan, s, max_ctas);
-    return launch_pair_t<true, true>(g, plan, s, max_ctas);
+    if (simple) {
+      if (!plan.a_mn && !plan.b_mn) return launch_pair_t<false, false, false>(g, plan, s, max_ctas);
+      if (!plan.a_mn && plan.b_mn) return launch_pair_t<false, true, false>(g, plan, s, max_ctas);
+      if (plan.a_mn && !plan.b_mn) return launch_pair_t<true, false, false>(g, plan, s, max_ctas);
+      return launch_pair_t<true, true, false>(g, plan, s, max_ctas);
+    }
+    // fused epilogues occur on forward (both operands K-major) and dgrad (B MN-major) GEMMs only
+    if (!plan.a_mn && !plan.b_mn) return launch_pair_t<false, false, true>(g, plan, s, max_ctas);
+    if (!plan.a_mn && plan.b_mn) return launch_pair_t<false, true, true>(g, plan, s, max_ctas);
   }
   switch (plan.bn) {
     case 64: return simple ? launch_bn<64, false>(g, plan, s, max_ctas) : launch_bn<64, true>(g, plan, s, max_ctas);

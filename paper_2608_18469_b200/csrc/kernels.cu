@@ -145,6 +145,17 @@ cudaError_t gemm_simt(const GemmArgs& g, bool bf16, cudaStream_t s) {
   return bf16 ? gemm_simt_t<bf16_t>(g, s) : gemm_simt_t<float>(g, s);
 }
 
+// one thread writes the GPU's nanosecond clock: a phase boundary that can be captured into a graph
+__global__ void stamp_kernel(unsigned long long* slot) {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  *slot = t;
+}
+cudaError_t stamp_time(unsigned long long* slot, cudaStream_t s) {
+  stamp_kernel<<<1, 1, 0, s>>>(slot);
+  return cudaGetLastError();
+}
+
 template <bool BF16_OUT>
 __global__ void splitk_reduce_kernel(const float* __restrict__ ws, int splits, long long mn, int N,
                                      void* __restrict__ out, long long ldo) {
@@ -1128,10 +1139,7 @@ __global__ void __launch_bounds__(256) ew_kernel(const T* a, const T* __restrict
   constexpr int VEC = VecOf<T>::N;
   const long long nvec = n / VEC;
   const long long stride = (long long)gridDim.x * 256;
-  for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < nvec; i += stride) {
-    float x[VEC], y[VEC];
-    ld_vec<T>(a + i * VEC, x);
-    if (mode != 1) ld_vec<T>(b + i * VEC, y);
+  auto finish = [&](long long i, float* x, const float* y) {
 #pragma unroll
     for (int j = 0; j < VEC; j++)
       x[j] = mode == 0 ? x[j] * y[j] : (mode == 1 ? act_apply(act, x[j]) : x[j] * act_deriv(act, y[j]));
@@ -1146,6 +1154,22 @@ __global__ void __launch_bounds__(256) ew_kernel(const T* a, const T* __restrict
     } else {
       *reinterpret_cast<float4*>(out + i * VEC) = make_float4(x[0], x[1], x[2], x[3]);
     }
+  };
+  // two vectors per thread and step: both loads (four with a second operand) are in flight together
+  long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+  for (; i + stride < nvec; i += 2 * stride) {
+    float x0[VEC], y0[VEC], x1[VEC], y1[VEC];
+    ld_vec<T>(a + i * VEC, x0);
+    ld_vec<T>(a + (i + stride) * VEC, x1);
+    if (mode != 1) { ld_vec<T>(b + i * VEC, y0); ld_vec<T>(b + (i + stride) * VEC, y1); }
+    finish(i, x0, y0);
+    finish(i + stride, x1, y1);
+  }
+  if (i < nvec) {
+    float x[VEC], y[VEC];
+    ld_vec<T>(a + i * VEC, x);
+    if (mode != 1) ld_vec<T>(b + i * VEC, y);
+    finish(i, x, y);
   }
   if (blockIdx.x == 0)
     for (long long i = nvec * VEC + threadIdx.x; i < n; i += 256) {
@@ -1298,33 +1322,67 @@ cudaError_t opt_tick(double* tick, float beta1, float beta2, cudaStream_t s) {
   return cudaGetLastError();
 }
 
+// One element of SGD / Adam / AdamW; every path below applies exactly this arithmetic.
+__device__ __forceinline__ void opt_element(float& th, float g, float& mm, float& vv, int kind, float lr, float b1, float b2,
+                                            float eps, float wd, float bc1, float bc2) {
+  if (kind == 0) {
+    th -= lr * g;
+  } else {
+    if (kind == 2) th *= (1.f - lr * wd);
+    mm = b1 * mm + (1.f - b1) * g;
+    vv = b2 * vv + (1.f - b2) * g * g;
+    th -= lr * (mm / bc1) / (sqrtf(vv / bc2) + eps);
+  }
+}
+
+// Four consecutive parameters per thread (16-byte accesses; the arenas are 256-byte aligned and a
+// block's slice starts on a multiple of 64 elements); the last, partial quad is done element-wise.
 __global__ void __launch_bounds__(256) opt_update_kernel(float* __restrict__ theta, const float* __restrict__ grad,
                                                          float* __restrict__ m, float* __restrict__ v,
                                                          bf16_t* __restrict__ shadow, long long n, int kind, float lr,
                                                          float b1, float b2, float eps, float wd,
-                                                         const double* __restrict__ tick) {
-  long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+                                                         const double* __restrict__ tick, int vec) {
+  const long long q = (long long)blockIdx.x * 256 + threadIdx.x;
+  const long long i = q * 4;
   if (i >= n) return;
-  float th = theta[i], g = grad[i];
-  if (kind == 0) {
-    th -= lr * g;
-  } else {
-    float bc1 = (float)tick[1], bc2 = (float)tick[2];
-    if (kind == 2) th *= (1.f - lr * wd);
-    float mm = b1 * m[i] + (1.f - b1) * g;
-    float vv = b2 * v[i] + (1.f - b2) * g * g;
-    m[i] = mm;
-    v[i] = vv;
-    th -= lr * (mm / bc1) / (sqrtf(vv / bc2) + eps);
+  float bc1 = 1.f, bc2 = 1.f;
+  if (kind != 0) { bc1 = (float)tick[1]; bc2 = (float)tick[2]; }
+  if (vec && i + 4 <= n) {
+    float4 th = reinterpret_cast<float4*>(theta)[q];
+    const float4 g = reinterpret_cast<const float4*>(grad)[q];
+    float4 mm = make_float4(0.f, 0.f, 0.f, 0.f), vv = mm;
+    if (kind != 0) { mm = reinterpret_cast<float4*>(m)[q]; vv = reinterpret_cast<float4*>(v)[q]; }
+    opt_element(th.x, g.x, mm.x, vv.x, kind, lr, b1, b2, eps, wd, bc1, bc2);
+    opt_element(th.y, g.y, mm.y, vv.y, kind, lr, b1, b2, eps, wd, bc1, bc2);
+    opt_element(th.z, g.z, mm.z, vv.z, kind, lr, b1, b2, eps, wd, bc1, bc2);
+    opt_element(th.w, g.w, mm.w, vv.w, kind, lr, b1, b2, eps, wd, bc1, bc2);
+    if (kind != 0) { reinterpret_cast<float4*>(m)[q] = mm; reinterpret_cast<float4*>(v)[q] = vv; }
+    reinterpret_cast<float4*>(theta)[q] = th;
+    if (shadow) {
+      __nv_bfloat162 lo = __floats2bfloat162_rn(th.x, th.y), hi = __floats2bfloat162_rn(th.z, th.w);
+      uint2 w;
+      w.x = *reinterpret_cast<uint32_t*>(&lo);
+      w.y = *reinterpret_cast<uint32_t*>(&hi);
+      reinterpret_cast<uint2*>(shadow)[q] = w;
+    }
+    return;
   }
-  theta[i] = th;
-  if (shadow) shadow[i] = __float2bfloat16_rn(th);
+  for (long long k = i; k < n && k < i + 4; k++) {
+    float th = theta[k], mm = 0.f, vv = 0.f;
+    if (kind != 0) { mm = m[k]; vv = v[k]; }
+    opt_element(th, grad[k], mm, vv, kind, lr, b1, b2, eps, wd, bc1, bc2);
+    if (kind != 0) { m[k] = mm; v[k] = vv; }
+    theta[k] = th;
+    if (shadow) shadow[k] = __float2bfloat16_rn(th);
+  }
 }
 cudaError_t opt_update(float* theta, const float* grad, float* m, float* v, void* shadow, long long n, int kind,
                        float lr, float beta1, float beta2, float eps, float wd, const double* tick,
                        cudaStream_t s) {
   if (n <= 0) return cudaSuccess;
-  opt_update_kernel<<<cdiv(n, 256), 256, 0, s>>>(theta, grad, m, v, (bf16_t*)shadow, n, kind, lr, beta1, beta2, eps, wd, tick);
+  auto al = [](const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; };
+  const int vec = al(theta, 16) && al(grad, 16) && (!m || al(m, 16)) && (!v || al(v, 16)) && (!shadow || al(shadow, 8));
+  opt_update_kernel<<<cdiv((n + 3) / 4, 256), 256, 0, s>>>(theta, grad, m, v, (bf16_t*)shadow, n, kind, lr, beta1, beta2, eps, wd, tick, vec);
   return cudaGetLastError();
 }
 

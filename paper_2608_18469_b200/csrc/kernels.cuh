@@ -48,6 +48,8 @@ struct GemmArgs {
 };
 
 cudaError_t gemm_simt(const GemmArgs& g, bool bf16, cudaStream_t s);
+// writes the device's nanosecond clock to *slot when the stream reaches this point
+cudaError_t stamp_time(unsigned long long* slot, cudaStream_t s);
 // out: float, or bfloat16 when out_bf16 (the sum is rounded once, after the last partial)
 cudaError_t splitk_reduce(const float* ws, int splits, long long mn, int N, void* out, long long ldo,
                           cudaStream_t s, bool out_bf16 = false);
