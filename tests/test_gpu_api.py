@@ -125,6 +125,18 @@ def test_timeline_profile_and_launch_count():
     with pytest.raises(binding.EraseError) as e:
         m.timeline()                                      # graph replay records no timeline
     assert e.value.status == binding.ESTATE
+    # device clock stamps are part of the captured graph: the timeline of a REPLAYED step
+    stamps = 2 * (2 * nb + 1) + 1
+    for rep in range(2):
+        l1 = m.launch_count()
+        m.step(n_streams=nb + 1, flags=binding.GRAPH | binding.STAMPS | binding.EARLY_HEAD | binding.BLOCK_OPT, **db.args())
+        assert m.launch_count() - l1 == per_step + stamps + (nb - 1)   # one optimizer launch per block instead of one
+        tg = m.timeline()
+        assert tg.shape == (2 * nb + 1, 2) and (tg[:, 1] >= tg[:, 0]).all() and tg.min() >= 0 and tg.max() < 1e3
+        for b in range(nb):
+            assert tg[nb + b, 0] >= tg[b, 1] - 1e-3           # B_b starts after F_b's body
+            if b + 1 < nb:
+                assert tg[b + 1, 0] >= tg[b, 1] - 1e-3        # F_{b+1} follows F_b on the main stream
     recs = m.profile_step(**db.args())
     assert sum(r["launches"] for r in recs) == per_step
     assert {r["name"] for r in recs} >= {"gemm_fwd", "gemm_dgrad", "gemm_wgrad", "softmax_ce", "opt_update"}
@@ -144,7 +156,8 @@ def test_full_size_lm_configs_schedules_agree_and_losses_start_near_ln_vocab():
         flat = synth.init_params(spec, 0)
         batches = [gu.DevBatch(spec, synth.make_batch(spec, 0, index=i)) for i in range(steps)]
         serial = gu.run_steps(spec, flat, batches, n_streams=1)
-        bench_cfg = gu.run_steps(spec, flat, batches, n_streams=nb + 1, flags=binding.GRAPH | binding.EARLY_HEAD | binding.BLOCK_OPT)
+        bench_cfg = gu.run_steps(spec, flat, batches, n_streams=nb + 1,
+                                 flags=binding.GRAPH | binding.EARLY_HEAD | binding.BLOCK_OPT | binding.SPLIT_BWD)
         for k in serial:
             if k != "launches":
                 assert serial[k].tobytes() == bench_cfg[k].tobytes(), (name, k)

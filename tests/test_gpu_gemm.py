@@ -48,6 +48,27 @@ def test_tensor_core_gemm_bf16(shape, layout):
     assert _run("bf16", M, N, K, a_mn, b_mn, engine=1, c_f32=True) < 2e-5
 
 
+# Shapes that the CTA-pair kernel takes (256 x 256 tiles over two SMs, at least 56 of them): full
+# tiles, ragged M / N / K tails, a single K block, a peer CTA whose rows lie wholly outside M.
+PAIR_SHAPES = [(2048, 2048, 192), (3896, 1032, 200), (4096, 8192, 64), (14400 + 8, 264, 136)]
+
+
+@pytest.mark.parametrize("layout", list(LAYOUTS))
+@pytest.mark.parametrize("shape", PAIR_SHAPES)
+def test_cta_pair_gemm_bf16(shape, layout):
+    M, N, K = shape
+    a_mn, b_mn = LAYOUTS[layout]
+    assert _run("bf16", M, N, K, a_mn, b_mn, engine=1) < 4e-3
+    assert _run("bf16", M, N, K, a_mn, b_mn, engine=1, c_f32=True) < 2e-5
+
+
+@pytest.mark.parametrize("layout", list(LAYOUTS))
+def test_cta_pair_split_k(layout):
+    a_mn, b_mn = LAYOUTS[layout]
+    assert _run("bf16", 2048, 512, 4096 + 72, a_mn, b_mn, engine=1, splits=7, c_f32=True) < 2e-5
+    assert _run("bf16", 4096, 256, 200, a_mn, b_mn, engine=1, splits=4, c_f32=True) < 2e-5   # trailing empty split
+
+
 @pytest.mark.parametrize("layout", list(LAYOUTS))
 def test_tensor_core_split_k_matches_and_is_deterministic(layout):
     a_mn, b_mn = LAYOUTS[layout]

@@ -82,7 +82,7 @@ def test_config2_in_the_benchmark_launch_configuration():
     from paper_2608_18469_b200 import binding
     spec = synth.config("C2")
     _gu().compare_teacher_forced(spec, steps=2, seed=1, n_streams=len(spec["blocks"]) + 1,
-                                 flags=binding.GRAPH | binding.EARLY_HEAD | binding.BLOCK_OPT)
+                                 flags=binding.GRAPH | binding.EARLY_HEAD | binding.BLOCK_OPT | binding.SPLIT_BWD)
 
 
 def test_config5_mid_point_w1024_b4096():
