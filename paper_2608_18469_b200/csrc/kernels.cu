@@ -1139,7 +1139,10 @@ __global__ void __launch_bounds__(256) ew_kernel(const T* a, const T* __restrict
   constexpr int VEC = VecOf<T>::N;
   const long long nvec = n / VEC;
   const long long stride = (long long)gridDim.x * 256;
-  auto finish = [&](long long i, float* x, const float* y) {
+  for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < nvec; i += stride) {
+    float x[VEC], y[VEC];
+    ld_vec<T>(a + i * VEC, x);
+    if (mode != 1) ld_vec<T>(b + i * VEC, y);
 #pragma unroll
     for (int j = 0; j < VEC; j++)
       x[j] = mode == 0 ? x[j] * y[j] : (mode == 1 ? act_apply(act, x[j]) : x[j] * act_deriv(act, y[j]));
@@ -1154,22 +1157,6 @@ __global__ void __launch_bounds__(256) ew_kernel(const T* a, const T* __restrict
     } else {
       *reinterpret_cast<float4*>(out + i * VEC) = make_float4(x[0], x[1], x[2], x[3]);
     }
-  };
-  // two vectors per thread and step: both loads (four with a second operand) are in flight together
-  long long i = (long long)blockIdx.x * 256 + threadIdx.x;
-  for (; i + stride < nvec; i += 2 * stride) {
-    float x0[VEC], y0[VEC], x1[VEC], y1[VEC];
-    ld_vec<T>(a + i * VEC, x0);
-    ld_vec<T>(a + (i + stride) * VEC, x1);
-    if (mode != 1) { ld_vec<T>(b + i * VEC, y0); ld_vec<T>(b + (i + stride) * VEC, y1); }
-    finish(i, x0, y0);
-    finish(i + stride, x1, y1);
-  }
-  if (i < nvec) {
-    float x[VEC], y[VEC];
-    ld_vec<T>(a + i * VEC, x);
-    if (mode != 1) ld_vec<T>(b + i * VEC, y);
-    finish(i, x, y);
   }
   if (blockIdx.x == 0)
     for (long long i = nvec * VEC + threadIdx.x; i < n; i += 256) {
