@@ -289,18 +289,21 @@ template <> __device__ __forceinline__ void ld_vec<bf16_t>(const bf16_t* p, floa
 
 // A CTA sums a strip of 32*VEC columns over one chunk of rows: a thread owns VEC adjacent
 // columns (one 16-byte load per row) and every 8th row, four rows in flight.
+// bx = column strip, by = row chunk of this CTA (the grid of the plain kernel, or what the batched
+// kernel derived from its job table).
 template <typename T>
-__global__ void __launch_bounds__(256) colsum_kernel(const T* __restrict__ X, long long ldx, int rows,
-                                                     int cols, const float* __restrict__ scale,
-                                                     float* __restrict__ ws, float* __restrict__ out, int chunks,
-                                                     int dact, const float* __restrict__ colscale, int* tickets) {
+__device__ __forceinline__ void colsum_body(const T* __restrict__ X, long long ldx, int rows,
+                                            int cols, const float* __restrict__ scale,
+                                            float* __restrict__ ws, float* __restrict__ out, int chunks,
+                                            int dact, const float* __restrict__ colscale, int* tickets, int bx, int by,
+                                            float* smem) {   // 8 * 32*VEC floats
   constexpr int VEC = VecOf<T>::N;
   constexpr int SW = 32 * VEC;  // strip width
-  __shared__ float sm[8][SW];
+  float (*sm)[SW] = reinterpret_cast<float (*)[SW]>(smem);
   const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
-  const int c = blockIdx.x * SW + cx * VEC;
+  const int c = bx * SW + cx * VEC;
   const int per = (rows + chunks - 1) / chunks;
-  const int rb = blockIdx.y * per, re = min(rows, rb + per);
+  const int rb = by * per, re = min(rows, rb + per);
   const bool vec = X && (c + VEC <= cols) && (ldx % VEC == 0) && ((reinterpret_cast<uintptr_t>(X) & 15) == 0);
   float a[VEC];
 #pragma unroll
@@ -351,9 +354,9 @@ __global__ void __launch_bounds__(256) colsum_kernel(const T* __restrict__ X, lo
 #pragma unroll
   for (int j = 0; j < VEC; j++) sm[ry][cx * VEC + j] = a[j];
   __syncthreads();
-  float* dst = chunks == 1 ? out : ws + (long long)blockIdx.y * cols;
+  float* dst = chunks == 1 ? out : ws + (long long)by * cols;
   for (int i = threadIdx.x; i < SW; i += 256) {
-    const int cc = blockIdx.x * SW + i;
+    const int cc = bx * SW + i;
     if (cc < cols) {
       float t = 0.f;
 #pragma unroll
@@ -363,15 +366,24 @@ __global__ void __launch_bounds__(256) colsum_kernel(const T* __restrict__ X, lo
     }
   }
   if (chunks == 1) return;
-  if (!last_cta(tickets + blockIdx.x, chunks)) return;
+  if (!last_cta(tickets + bx, chunks)) return;
   for (int i = threadIdx.x; i < SW; i += 256) {
-    const int cc = blockIdx.x * SW + i;
+    const int cc = bx * SW + i;
     if (cc < cols) {
       float t = ordered_sum(ws + cc, cols, chunks);
       if (colscale) t *= colscale[cc];
       out[cc] = t;
     }
   }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) colsum_kernel(const T* __restrict__ X, long long ldx, int rows,
+                                                     int cols, const float* __restrict__ scale,
+                                                     float* __restrict__ ws, float* __restrict__ out, int chunks,
+                                                     int dact, const float* __restrict__ colscale, int* tickets) {
+  __shared__ float smem[8 * 32 * VecOf<T>::N];
+  colsum_body<T>(X, ldx, rows, cols, scale, ws, out, chunks, dact, colscale, tickets, blockIdx.x, blockIdx.y, smem);
 }
 
 cudaError_t colsum(const void* X, bool x_bf16, long long ldx, int rows, int cols, const float* scale,
@@ -454,19 +466,20 @@ cudaError_t layernorm_bwd_dx(const void* dy, const void* x, const float* gain, c
 // dgain / dshift partial sums: a CTA takes a strip of 32*VEC columns and one chunk of rows, a thread
 // VEC adjacent columns (16-byte loads of dy and x) and every 8th row, four rows in flight.
 template <typename T>
-__global__ void __launch_bounds__(256) layernorm_param_grad_kernel(const T* __restrict__ dy, const T* __restrict__ x,
-                                                                   const float* __restrict__ mean,
-                                                                   const float* __restrict__ rstd,
-                                                                   float* __restrict__ ws, float* __restrict__ dgain,
-                                                                   float* __restrict__ dshift, int rows, int d, int chunks,
-                                                                   int* tickets) {
+__device__ __forceinline__ void layernorm_param_grad_body(const T* __restrict__ dy, const T* __restrict__ x,
+                                                          const float* __restrict__ mean,
+                                                          const float* __restrict__ rstd,
+                                                          float* __restrict__ ws, float* __restrict__ dgain,
+                                                          float* __restrict__ dshift, int rows, int d, int chunks,
+                                                          int* tickets, int bx, int by, float* smem) {   // 16 * 32*VEC floats
   constexpr int VEC = VecOf<T>::N;
   constexpr int SW = 32 * VEC;
-  __shared__ float sg[8][SW], sb[8][SW];
+  float (*sg)[SW] = reinterpret_cast<float (*)[SW]>(smem);
+  float (*sb)[SW] = reinterpret_cast<float (*)[SW]>(smem + 8 * SW);
   const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
-  const int c = blockIdx.x * SW + cx * VEC;
+  const int c = bx * SW + cx * VEC;
   const int per = (rows + chunks - 1) / chunks;
-  const int rb = blockIdx.y * per, re = min(rows, rb + per);
+  const int rb = by * per, re = min(rows, rb + per);
   const bool vec = (c + VEC <= d) && (d % VEC == 0);
   float ag[VEC], ab[VEC];
 #pragma unroll
@@ -518,10 +531,10 @@ __global__ void __launch_bounds__(256) layernorm_param_grad_kernel(const T* __re
 #pragma unroll
   for (int j = 0; j < VEC; j++) { sg[ry][cx * VEC + j] = ag[j]; sb[ry][cx * VEC + j] = ab[j]; }
   __syncthreads();
-  float* pg = chunks == 1 ? dgain : ws + (long long)blockIdx.y * d;
-  float* pb = chunks == 1 ? dshift : ws + (long long)(chunks + blockIdx.y) * d;
+  float* pg = chunks == 1 ? dgain : ws + (long long)by * d;
+  float* pb = chunks == 1 ? dshift : ws + (long long)(chunks + by) * d;
   for (int i = threadIdx.x; i < SW; i += 256) {
-    const int cc = blockIdx.x * SW + i;
+    const int cc = bx * SW + i;
     if (cc < d) {
       float tg = 0.f, tb = 0.f;
 #pragma unroll
@@ -531,14 +544,57 @@ __global__ void __launch_bounds__(256) layernorm_param_grad_kernel(const T* __re
     }
   }
   if (chunks == 1) return;
-  if (!last_cta(tickets + blockIdx.x, chunks)) return;
+  if (!last_cta(tickets + bx, chunks)) return;
   for (int i = threadIdx.x; i < SW; i += 256) {
-    const int cc = blockIdx.x * SW + i;
+    const int cc = bx * SW + i;
     if (cc < d) {
       dgain[cc] = ordered_sum(ws + cc, d, chunks);
       dshift[cc] = ordered_sum(ws + (long long)chunks * d + cc, d, chunks);
     }
   }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) layernorm_param_grad_kernel(const T* __restrict__ dy, const T* __restrict__ x,
+                                                                   const float* __restrict__ mean,
+                                                                   const float* __restrict__ rstd,
+                                                                   float* __restrict__ ws, float* __restrict__ dgain,
+                                                                   float* __restrict__ dshift, int rows, int d, int chunks,
+                                                                   int* tickets) {
+  __shared__ float smem[16 * 32 * VecOf<T>::N];
+  layernorm_param_grad_body<T>(dy, x, mean, rstd, ws, dgain, dshift, rows, d, chunks, tickets, blockIdx.x, blockIdx.y, smem);
+}
+
+// Several column reductions in ONE launch: the bias gradients and LayerNorm gain/shift gradients of
+// a block are each a few MB of input, so separate launches spend most of their time ramping up and
+// waiting for their last CTA.  A CTA looks its job up in a table (at most a few entries) and then
+// runs exactly the code of the single-job kernels on the same partition: same bits.
+__global__ void __launch_bounds__(256, 4) reduce_batch_kernel(const ReduceJob* __restrict__ jobs, int njobs) {
+  __shared__ float smem[16 * 256];   // the largest need: gain and shift partials of a 256-column bf16 strip
+  int j = 0;
+  while (j + 1 < njobs && (int)blockIdx.x >= jobs[j + 1].cta_begin) j++;
+  const ReduceJob job = jobs[j];
+  const int local = (int)blockIdx.x - job.cta_begin;
+  const int bx = local % job.strips, by = local / job.strips;
+  if (job.kind == 0) {
+    if (job.x_f32)
+      colsum_body<float>((const float*)job.X, job.ldx, job.rows, job.cols, job.a, job.ws, job.out0, job.chunks, job.dact, job.b, job.tickets, bx, by, smem);
+    else
+      colsum_body<bf16_t>((const bf16_t*)job.X, job.ldx, job.rows, job.cols, job.a, job.ws, job.out0, job.chunks, job.dact, job.b, job.tickets, bx, by, smem);
+  } else {
+    if (job.x_f32)
+      layernorm_param_grad_body<float>((const float*)job.X, (const float*)job.X2, job.a, job.b, job.ws, job.out0, job.out1, job.rows, job.cols, job.chunks, job.tickets, bx, by, smem);
+    else
+      layernorm_param_grad_body<bf16_t>((const bf16_t*)job.X, (const bf16_t*)job.X2, job.a, job.b, job.ws, job.out0, job.out1, job.rows, job.cols, job.chunks, job.tickets, bx, by, smem);
+  }
+}
+
+int reduce_job_strips(const ReduceJob& j) { return (int)cdiv(j.cols, j.x_f32 ? 128 : 256); }
+
+cudaError_t reduce_batch(const ReduceJob* jobs_dev, int njobs, int total_ctas, cudaStream_t s) {
+  if (njobs <= 0 || total_ctas <= 0) return cudaSuccess;
+  reduce_batch_kernel<<<total_ctas, 256, 0, s>>>(jobs_dev, njobs);
+  return cudaGetLastError();
 }
 
 cudaError_t layernorm_param_grad(const void* dy, const void* x, const float* mean, const float* rstd,

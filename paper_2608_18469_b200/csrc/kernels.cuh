@@ -64,6 +64,28 @@ cudaError_t colsum(const void* X, bool x_bf16, long long ldx, int rows, int cols
                    float* ws, int chunks, int* tickets, float* out, cudaStream_t s, int dact = ACT_NONE,
                    const float* colscale = nullptr);
 
+// One entry of reduce_batch's job table (device memory).  kind 0: colsum with X, ldx, a = scale,
+// b = colscale, dact, out0; kind 1: layernorm_param_grad with X = dy, X2 = x, a = mean, b = rstd,
+// cols = d, out0 = dgain, out1 = dshift.  x_f32: X (and X2) hold floats, else bfloat16.  The job's
+// CTAs are cta_begin .. cta_begin + strips*chunks - 1 of the launch (strip fastest).
+struct ReduceJob {
+  int kind = 0, x_f32 = 0, dact = ACT_NONE;
+  int rows = 0, cols = 0, chunks = 1, strips = 1, cta_begin = 0;
+  long long ldx = 0;
+  const void* X = nullptr;
+  const void* X2 = nullptr;
+  const float* a = nullptr;
+  const float* b = nullptr;
+  float* ws = nullptr;
+  float* out0 = nullptr;
+  float* out1 = nullptr;
+  int* tickets = nullptr;
+};
+int reduce_job_strips(const ReduceJob& j);
+// All jobs of the table in one launch of total_ctas CTAs; each job computes what colsum /
+// layernorm_param_grad would with the same arguments.
+cudaError_t reduce_batch(const ReduceJob* jobs_dev, int njobs, int total_ctas, cudaStream_t s);
+
 // LayerNorm over the last dimension (eps 1e-5, biased variance); saves mean and 1/std per row.
 cudaError_t layernorm_fwd(const void* x, const float* gain, const float* shift, void* y, float* mean,
                           float* rstd, int rows, int d, bool bf16, cudaStream_t s);
