@@ -464,6 +464,15 @@ struct Builder {
     g.A = dY; g.sa_m = 1; g.sa_k = N;
     g.B = X; g.sb_n = 1; g.sb_k = ldx;
     g.C = G(widx); g.ldc = K; g.c_f32 = 1;
+    if (groupable(g)) {   // a small weight gradient: runs with the block's other small ones in one launch
+      group.push_back(g);
+      if (bidx >= 0 && !skip_bias) {
+        if (bias_now || (double)M * N * m->esz > 16.0e6) { bias_grad(ops, dY, N, M, N, bidx); ops.back().leaf = true; }
+        else colsum_job(ops, dY, m->bf16, N, M, N, nullptr, G(bidx), ACT_NONE, nullptr, (double)M * N, (double)M * N * m->esz);
+      }
+      if ((int)group.size() == 4) flush_group(ops);
+      return;
+    }
     long long tiles = (long long)((N + 63) / 64) * ((K + 63) / 64);
     int splits = (int)((296 + tiles - 1) / tiles);
     int maxs = M / 64 > 0 ? M / 64 : 1;
@@ -487,6 +496,71 @@ struct Builder {
     }
     for (size_t i = before; i < ops.size(); i++) ops[i].leaf = true;
   }
+  // ---- small weight gradients of a block, grouped into one launch --------------------------------
+  std::vector<GemmArgs> group;
+  int group_mode = getenv("ERASE_WGRAD_GROUP") ? atoi(getenv("ERASE_WGRAD_GROUP")) : 1;
+  bool groupable(const GemmArgs& g) const {
+    if (!group_mode || !m->bf16 || !tc_gemm_supported(g)) return false;
+    const long long tiles = (long long)((g.M + 127) / 128) * ((g.N + 127) / 128);
+    return tiles <= 32 && g.K >= 512 && g.N % 4 == 0 && g.ldc % 4 == 0 && (reinterpret_cast<uintptr_t>(g.C) & 15) == 0;
+  }
+  void flush_group(OpList& ops) {
+    const int n = (int)group.size();
+    if (n == 0) return;
+    long long tiles = 0;
+    int kmin = 1 << 30;
+    for (const GemmArgs& g : group) {
+      tiles += (long long)((g.M + 127) / 128) * ((g.N + 127) / 128);
+      kmin = std::min(kmin, g.K);
+    }
+    // CTAs of the launch: a full wave (148) is fastest alone (C2 serial 1.41 ms against 1.51 ms
+    // ungrouped) but its persistent CTAs then hold every SM while the other streams' kernels wait
+    // (C2 ERASE 1.120 ms against 1.088 ms); about 64 keeps most of the serial gain (1.44 ms) at no
+    // cost under ERASE (1.087 ms; C3 1.196 ms against 1.285 ms ungrouped at any setting).
+    static const int group_ctas = getenv("ERASE_GROUP_CTAS") ? atoi(getenv("ERASE_GROUP_CTAS")) : 64;
+    int splits = (int)(group_ctas / tiles);
+    splits = std::max(1, std::min(std::min(splits, kmin / 128), 16));
+    double flops = 0, bytes = 0;
+    std::vector<ReduceJob> rj;
+    int total = 0;
+    for (GemmArgs& g : group) {
+      g.splits = splits;
+      g.ws = f32_buf((size_t)splits * g.M * g.N);
+      ReduceJob j;
+      j.kind = 2; j.x_f32 = 1; j.rows = splits; j.cols = g.N; j.chunks = 1; j.ldx = g.ldc; j.mn = (long long)g.M * g.N;
+      j.X = g.ws; j.out0 = (float*)g.C;
+      j.strips = reduce_job_strips(j);
+      j.cta_begin = total;
+      total += j.strips;
+      rj.push_back(j);
+      flops += 2.0 * g.M * g.N * g.K;
+      bytes += ((double)g.M * g.K + (double)g.N * g.K) * m->esz + 4.0 * g.M * g.N;
+    }
+    ReduceJob* dev = (ReduceJob*)dev_alloc(m, sizeof(ReduceJob) * rj.size(), &ok);
+    if (ok && dev && !m->dry && cudaMemcpy(dev, rj.data(), sizeof(ReduceJob) * rj.size(), cudaMemcpyHostToDevice) != cudaSuccess) ok = false;
+    TcGroupPlan plan;
+    const bool planned = !m->dry && tc_wgrad_group_plan(group.data(), n, m->status, &plan);
+    std::vector<GemmArgs> gs = group;
+    erase_model* mm = m;
+    if (planned)
+      ops.push_back({[plan, dev, n, total, mm](cudaStream_t s) {
+                       cudaError_t e = tc_wgrad_group_launch(plan, s, mm->sm_budget);
+                       if (e != cudaSuccess) return e;
+                       return reduce_batch(dev, n, total, s);
+                     }, 2});
+    else   // descriptors could not be encoded (never expected): the same partials from the SIMT kernel
+      ops.push_back({[gs, dev, n, total](cudaStream_t s) {
+                       for (const GemmArgs& g : gs) {
+                         cudaError_t e = gemm_simt(g, true, s);
+                         if (e != cudaSuccess) return e;
+                       }
+                       return reduce_batch(dev, n, total, s);
+                     }, n + 1});
+    note(ops, "gemm_wgrad", flops, bytes);
+    ops.back().leaf = true;
+    group.clear();
+  }
+
   void bias_grad(OpList& ops, const void* dY, long long ld, int M, int N, int bidx) {
     int chunks = colsum_chunks(M, N);
     float* ws = chunks > 1 ? f32_buf((size_t)chunks * N) : nullptr;
@@ -681,6 +755,7 @@ struct Builder {
       lin_wgrad(bw, du, mm2, d, t(W1), t(B1), rows, ff, d);
       lin_dgrad(bw, du, t(W1), dm, rows, ff, d, Epilogue());
       ln_bwd(bw, dm, h, mean2, rstd2, t(LN2G), t(LN2B), dz, dhb, d);
+      flush_group(bw);  // dW2 and dW1 in one launch; dWproj and dWqkv at the end of B_b
       mid_flush(bw);   // (off by default) b2, b1, LN2 half-way; the rest (bproj, bqkv, LN1) at the end of B_b
       lin_wgrad(bw, dhb, o, d, t(WPROJ), t(BPROJ), rows, d, d);
       lin_dgrad(bw, dhb, t(WPROJ), dO, rows, d, d, Epilogue());
@@ -826,6 +901,7 @@ struct Builder {
         case ERASE_BLK_CROSS: zout = block_cross(b, k, zin, first, m->fwd[b], m->bwd[b]); break;
         case ERASE_BLK_DOT: zout = block_dot(b, k, zin, first, m->fwd[b], m->bwd[b]); break;
       }
+      flush_group(m->bwd[b]);
       flush_jobs(m->bwd[b]);
       z = zout;
       while (first < (int)m->tensors.size() && m->tensors[first].block == b) first++;

@@ -921,6 +921,221 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   }
 }
 
+// =================================================================================================
+// Grouped weight-gradient kernel: up to four small wgrad GEMMs (dW_i = dY_i^T X_i, both operands
+// MN-major, fp32 split-K partials) in ONE launch.  A block's weight gradients are each a few
+// 128 x 128 tiles; launched one by one they pay launch, prologue, pipeline fill and drain four
+// times with most SMs idle.  Here a tile index runs over all problems (problem, split, m, n), one
+// CTA per SM takes tiles round-robin, and the roles are those of tc_gemm_kernel (BN = 128,
+// identity epilogue, partials TMA-stored through each problem's 3-D map).
+constexpr int GROUP_MAX = 4;
+struct GroupProblem {
+  int M, N, K, splits, kchunk, tiles_m, tiles_n, tile_begin;
+};
+struct GroupArgs {
+  int nprob, total;
+  int* status;
+  GroupProblem prob[GROUP_MAX];
+};
+struct GroupMaps {
+  CUtensorMap a[GROUP_MAX], b[GROUP_MAX], c[GROUP_MAX];
+};
+
+__device__ __forceinline__ void group_tile(const GroupArgs& g, int t, int& pi, int& mt, int& nt, int& split) {
+  pi = 0;
+  while (pi + 1 < g.nprob && t >= g.prob[pi + 1].tile_begin) pi++;
+  const GroupProblem& q = g.prob[pi];
+  const int local = t - q.tile_begin, per = q.tiles_m * q.tiles_n;
+  split = local / per;
+  const int r = local - split * per;
+  mt = r / q.tiles_n;
+  nt = r - mt * q.tiles_n;
+}
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+tc_wgrad_group_kernel(const __grid_constant__ GroupMaps maps, const __grid_constant__ GroupArgs g) {
+  extern __shared__ uint8_t smem_raw[];
+  constexpr int BN = 128;
+  constexpr uint32_t A_BYTES = BM * BK * 2;
+  constexpr uint32_t B_BYTES = BN * BK * 2;
+  constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr uint32_t TMEM_COLS = 2 * BN;
+  constexpr int STAGES = 4;
+  constexpr int CPW = BN / 2;
+
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t epi_base = smem_base + STAGES * STAGE_BYTES;
+  const uint32_t bar_base = epi_base + EPI_WARPS * EPI_STAGE_BYTES;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+  uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
+  volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(gen_base + (bar_base - smem_base) + 8u * (2 * STAGES + 4));
+  const uint32_t tmem_slot = bar_base + 8u * (2 * STAGES + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 32) {
+    for (int i = 0; i < g.nprob; i++) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.a[i]) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.b[i]) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.c[i]) : "memory");
+    }
+  }
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; s++) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; a++) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), EPI_WARPS);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot_ptr;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < g.total && ok; t += gridDim.x) {
+        int pi, mt, nt, split;
+        group_tile(g, t, pi, mt, nt, split);
+        const GroupProblem& q = g.prob[pi];
+        const int m0 = mt * BM, n0 = nt * BN;
+        const int kbeg = split * q.kchunk, kend = min(q.K, kbeg + q.kchunk);
+        const int num_kb = kend > kbeg ? (kend - kbeg + BK - 1) / BK : 0;
+        for (int kb = 0; kb < num_kb; kb++, it++) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!mbar_wait(empty_bar(s), ph ^ 1)) { atomicExch(g.status, 1); ok = false; break; }
+          mbar_expect_tx(full_bar(s), STAGE_BYTES);
+          const uint32_t a_dst = smem_base + s * STAGE_BYTES;
+          const uint32_t b_dst = a_dst + A_BYTES;
+          const int k0 = kbeg + kb * BK;
+#pragma unroll
+          for (int a = 0; a < BM / 64; a++) tma_load_2d(a_dst + a * (BK * 128), &maps.a[pi], m0 + a * 64, k0, full_bar(s));
+#pragma unroll
+          for (int a = 0; a < BN / 64; a++) tma_load_2d(b_dst + a * (BK * 128), &maps.b[pi], n0 + a * 64, k0, full_bar(s));
+        }
+      }
+      if (!ok) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) {}
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) |
+                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      uint32_t it = 0, lt = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < g.total && ok; t += gridDim.x, lt++) {
+        int pi, mt, nt, split;
+        group_tile(g, t, pi, mt, nt, split);
+        const GroupProblem& q = g.prob[pi];
+        const int kbeg = split * q.kchunk, kend = min(q.K, kbeg + q.kchunk);
+        const int num_kb = kend > kbeg ? (kend - kbeg + BK - 1) / BK : 0;
+        const uint32_t ab = lt & 1, aph = (lt >> 1) & 1;
+        if (!mbar_wait(tempty_bar(ab), aph ^ 1)) { atomicExch(g.status, 4); ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + ab * BN;
+        for (int kb = 0; kb < num_kb; kb++, it++) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!mbar_wait(full_bar(s), ph)) { atomicExch(g.status, 2); ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_src = smem_base + s * STAGE_BYTES;
+          const uint32_t b_src = a_src + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; k++) {
+            const uint64_t ad = smem_desc(a_src + k * (UMMA_K * 128), BK * 128, 1024);
+            const uint64_t bd = smem_desc(b_src + k * (UMMA_K * 128), BK * 128, 1024);
+            tc_mma(tmem_d, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          }
+          tc_commit(empty_bar(s));
+        }
+        tc_commit(tfull_bar(ab));
+      }
+    }
+  } else {
+    const int ew = warp - 2;
+    const int q4 = warp & 3;
+    const int cbeg = (ew / 4) * CPW;
+    const uint32_t stage0 = epi_base + ew * EPI_STAGE_BYTES;
+    uint32_t sbuf = 0;
+    bool store_pending = false;
+    uint32_t lt = 0;
+    for (int t = blockIdx.x; t < g.total; t += gridDim.x, lt++) {
+      int pi, mt, nt, split;
+      group_tile(g, t, pi, mt, nt, split);
+      const GroupProblem& q = g.prob[pi];
+      const int m0 = mt * BM, n0 = nt * BN;
+      const int kbeg = split * q.kchunk, kend = min(q.K, kbeg + q.kchunk);
+      const bool empty_k = kend <= kbeg;
+      const uint32_t ab = lt & 1, aph = (lt >> 1) & 1;
+      bool ok = mbar_wait(tfull_bar(ab), aph);
+      if (!ok) atomicExch(g.status, 3);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const bool rows_in = m0 + q4 * 32 < q.M;
+      if (n0 + cbeg < q.N) {
+#pragma unroll 1
+        for (int cc = 0; cc < CPW; cc += 32) {
+          const int c0 = cbeg + cc;
+          if (n0 + c0 >= q.N) break;
+          uint32_t r[32];
+          if (!empty_k) {
+            tc_ld32(tmem_base + ab * BN + ((uint32_t)(q4 * 32) << 16) + (uint32_t)c0, r);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; j++) r[j] = 0u;
+          }
+          sbuf ^= 1;
+          if (lane == 0 && store_pending) tma_store_wait_read1();
+          __syncwarp();
+          const uint32_t stage = stage0 + sbuf * 4096;
+          const uint32_t my_row = stage + lane * 128;
+#pragma unroll
+          for (int g8 = 0; g8 < 4; g8++) {
+            const uint32_t s0 = my_row + (((2 * g8) ^ (lane & 7)) << 4), s1 = my_row + (((2 * g8 + 1) ^ (lane & 7)) << 4);
+            st_shared_v4(s0, r[g8 * 8 + 0], r[g8 * 8 + 1], r[g8 * 8 + 2], r[g8 * 8 + 3]);
+            st_shared_v4(s1, r[g8 * 8 + 4], r[g8 * 8 + 5], r[g8 * 8 + 6], r[g8 * 8 + 7]);
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (lane == 0 && rows_in) {
+            tma_store_3d(&maps.c[pi], stage, n0 + c0, m0 + q4 * 32, split);
+            tma_store_commit();
+            store_pending = true;
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(ab));
+    }
+    if (lane == 0 && store_pending) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
 typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -1053,6 +1268,62 @@ cudaError_t launch_bn(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int
 }
 
 }  // namespace
+
+bool tc_wgrad_group_plan(const GemmArgs* gs, int n, int* status, TcGroupPlan* plan) {
+  if (n < 1 || n > GROUP_MAX) return false;
+  plan->n = n;
+  plan->status = status;
+  int total = 0;
+  for (int i = 0; i < n; i++) {
+    const GemmArgs& g = gs[i];
+    if (!tc_gemm_supported(g) || g.sa_k == 1 || g.sb_k == 1 || g.splits < 1 || !g.ws) return false;   // both operands MN-major
+    plan->M[i] = g.M; plan->N[i] = g.N; plan->K[i] = g.K; plan->splits[i] = g.splits;
+    plan->kchunk[i] = (((g.K + g.splits - 1) / g.splits) + BK - 1) / BK * BK;
+    plan->tiles_m[i] = (g.M + BM - 1) / BM;
+    plan->tiles_n[i] = (g.N + 127) / 128;
+    plan->tile_begin[i] = total;
+    total += plan->tiles_m[i] * plan->tiles_n[i] * g.splits;
+    if (!encode_2d(plan->map_a[i], g.A, g.M, g.K, g.sa_k, BK)) return false;
+    if (!encode_2d(plan->map_b[i], g.B, g.N, g.K, g.sb_k, BK)) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)g.N, (cuuint64_t)g.M, (cuuint64_t)g.splits};
+    cuuint64_t str[2] = {(cuuint64_t)g.N * 4, (cuuint64_t)g.M * g.N * 4};
+    cuuint32_t box[3] = {32u, 32u, 1u};
+    if (!encode_map(plan->map_c[i], g.ws, true, 3, dims, str, box)) return false;
+  }
+  plan->total = total;
+  return true;
+}
+
+cudaError_t tc_wgrad_group_launch(const TcGroupPlan& plan, cudaStream_t s, int max_ctas) {
+  constexpr size_t smem = (size_t)4 * (BM * BK * 2 + 128 * BK * 2) + EPI_WARPS * EPI_STAGE_BYTES + 8 * (2 * 4 + 16) + 1024;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(tc_wgrad_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  GroupMaps maps;
+  GroupArgs g;
+  memset(&g, 0, sizeof(g));
+  g.nprob = plan.n; g.total = plan.total; g.status = plan.status;
+  for (int i = 0; i < plan.n; i++) {
+    memcpy(&maps.a[i], plan.map_a[i], 128);
+    memcpy(&maps.b[i], plan.map_b[i], 128);
+    memcpy(&maps.c[i], plan.map_c[i], 128);
+    g.prob[i] = GroupProblem{plan.M[i], plan.N[i], plan.K[i], plan.splits[i], plan.kchunk[i], plan.tiles_m[i], plan.tiles_n[i], plan.tile_begin[i]};
+  }
+  for (int i = plan.n; i < GROUP_MAX; i++) { maps.a[i] = maps.a[0]; maps.b[i] = maps.b[0]; maps.c[i] = maps.c[0]; }
+  static int num_sms = 0;
+  if (num_sms == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms < 1) num_sms = 148;
+  }
+  int cap = (max_ctas > 0 && max_ctas < num_sms) ? max_ctas : num_sms;
+  dim3 grid((unsigned)(plan.total < cap ? plan.total : cap));
+  tc_wgrad_group_kernel<<<grid, TC_THREADS, smem, s>>>(maps, g);
+  return cudaGetLastError();
+}
 
 bool tc_gemm_supported(const GemmArgs& g) {
   if (g.K < 64 || g.N < 16 || g.M < 1) return false;

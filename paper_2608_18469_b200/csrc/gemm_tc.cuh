@@ -38,4 +38,15 @@ bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan);
 // the tile-to-CTA assignment does not enter the arithmetic, so results do not depend on it.
 cudaError_t tc_gemm_launch(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas = 0);
 
+// Up to four weight-gradient GEMMs (both operands MN-major, g.splits >= 1, g.ws set: fp32 partials)
+// in one launch; each problem's partials still need splitk_reduce.
+struct TcGroupPlan {
+  int n = 0, total = 0;
+  int M[4], N[4], K[4], splits[4], kchunk[4], tiles_m[4], tiles_n[4], tile_begin[4];
+  unsigned char map_a[4][128], map_b[4][128], map_c[4][128];
+  int* status = nullptr;
+};
+bool tc_wgrad_group_plan(const GemmArgs* gs, int n, int* status, TcGroupPlan* plan);
+cudaError_t tc_wgrad_group_launch(const TcGroupPlan& plan, cudaStream_t s, int max_ctas = 0);
+
 }  // namespace erase

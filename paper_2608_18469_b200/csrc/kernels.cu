@@ -170,9 +170,8 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ ws, int splits, l
 
 // four adjacent columns per thread (N, ldo multiples of 4); the partials of up to four splits are in flight at once
 template <bool BF16_OUT>
-__global__ void splitk_reduce_v4_kernel(const float4* __restrict__ ws, int splits, long long mn4, int N4,
-                                        void* __restrict__ out, long long ldo) {
-  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+__device__ __forceinline__ void splitk_reduce_v4_body(const float4* __restrict__ ws, int splits, long long mn4, int N4,
+                                                      void* __restrict__ out, long long ldo, long long i) {
   if (i >= mn4) return;
   float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
   for (int s0 = 0; s0 < splits; s0 += 4) {
@@ -193,6 +192,11 @@ __global__ void splitk_reduce_v4_kernel(const float4* __restrict__ ws, int split
   } else {
     *reinterpret_cast<float4*>((float*)out + o) = a;
   }
+}
+template <bool BF16_OUT>
+__global__ void splitk_reduce_v4_kernel(const float4* __restrict__ ws, int splits, long long mn4, int N4,
+                                        void* __restrict__ out, long long ldo) {
+  splitk_reduce_v4_body<BF16_OUT>(ws, splits, mn4, N4, out, ldo, (long long)blockIdx.x * blockDim.x + threadIdx.x);
 }
 
 cudaError_t splitk_reduce(const float* ws, int splits, long long mn, int N, void* out, long long ldo,
@@ -576,6 +580,11 @@ __global__ void __launch_bounds__(256, 4) reduce_batch_kernel(const ReduceJob* _
   const ReduceJob job = jobs[j];
   const int local = (int)blockIdx.x - job.cta_begin;
   const int bx = local % job.strips, by = local / job.strips;
+  if (job.kind == 2) {   // split-K partials -> fp32 result, 1024 outputs per CTA
+    splitk_reduce_v4_body<false>((const float4*)job.X, job.rows, job.mn / 4, job.cols / 4, job.out0, job.ldx,
+                                 (long long)local * 256 + threadIdx.x);
+    return;
+  }
   if (job.kind == 0) {
     if (job.x_f32)
       colsum_body<float>((const float*)job.X, job.ldx, job.rows, job.cols, job.a, job.ws, job.out0, job.chunks, job.dact, job.b, job.tickets, bx, by, smem);
@@ -589,7 +598,10 @@ __global__ void __launch_bounds__(256, 4) reduce_batch_kernel(const ReduceJob* _
   }
 }
 
-int reduce_job_strips(const ReduceJob& j) { return (int)cdiv(j.cols, j.x_f32 ? 128 : 256); }
+int reduce_job_strips(const ReduceJob& j) {
+  if (j.kind == 2) return (int)cdiv(j.mn / 4, 256);
+  return (int)cdiv(j.cols, j.x_f32 ? 128 : 256);
+}
 
 cudaError_t reduce_batch(const ReduceJob* jobs_dev, int njobs, int total_ctas, cudaStream_t s) {
   if (njobs <= 0 || total_ctas <= 0) return cudaSuccess;

@@ -66,12 +66,14 @@ cudaError_t colsum(const void* X, bool x_bf16, long long ldx, int rows, int cols
 
 // One entry of reduce_batch's job table (device memory).  kind 0: colsum with X, ldx, a = scale,
 // b = colscale, dact, out0; kind 1: layernorm_param_grad with X = dy, X2 = x, a = mean, b = rstd,
-// cols = d, out0 = dgain, out1 = dshift.  x_f32: X (and X2) hold floats, else bfloat16.  The job's
-// CTAs are cta_begin .. cta_begin + strips*chunks - 1 of the launch (strip fastest).
+// cols = d, out0 = dgain, out1 = dshift; kind 2: splitk_reduce to a float result with X = ws,
+// rows = splits, mn, cols = N, ldx = ldo (mn, N, ldo multiples of 4, 16-byte aligned), chunks = 1.
+// x_f32: X (and X2) hold floats, else bfloat16.  The job's CTAs are
+// cta_begin .. cta_begin + strips*chunks - 1 of the launch (strip fastest).
 struct ReduceJob {
   int kind = 0, x_f32 = 0, dact = ACT_NONE;
   int rows = 0, cols = 0, chunks = 1, strips = 1, cta_begin = 0;
-  long long ldx = 0;
+  long long ldx = 0, mn = 0;
   const void* X = nullptr;
   const void* X2 = nullptr;
   const float* a = nullptr;
