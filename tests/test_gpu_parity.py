@@ -66,6 +66,9 @@ def _bf16_cases():
     s["lm_bf16_T320"] = synth.lm_spec(1, 64, 1, 128, 320, 2, 300)            # five key tiles per head
     s["lm_bf16_dh32"] = synth.lm_spec(1, 128, 4, 256, 96, 2, 300)            # head width 32: SIMT attention
     s["ctr_bf16_small"] = synth.ctr_spec(batch=512, table_rows=1000, tower=(256, 128, 64))
+    # enough rows (>= 512) for the grouped weight-gradient kernel, with ragged M / N / K tails in every problem
+    s["lm_bf16_grouped_ragged"] = synth.lm_spec(2, 192, 3, 328, 100, 6, 777)
+    s["mlp_bf16_grouped_ragged"] = synth.mlp_spec(200, 328, 2, 600, "relu", "bf16")
     return s
 
 
