@@ -346,16 +346,27 @@ struct Builder {
                   int dact, const float* colscale, double flops, double bytes) {
     ReduceJob j;
     j.kind = 0; j.x_f32 = x_bf16 ? 0 : 1; j.dact = dact;
-    j.rows = rows; j.cols = cols; j.chunks = colsum_chunks(rows, cols); j.ldx = ldx;
+    j.rows = rows; j.cols = cols; j.ldx = ldx;      // chunks and workspace are set when the batch is flushed
     j.X = X; j.a = scale; j.b = colscale;
-    j.ws = j.chunks > 1 ? f32_buf((size_t)j.chunks * cols) : nullptr;
     j.out0 = out; j.tickets = tickets(cols);
     add_job(ops, j, flops, bytes);
   }
   void flush_jobs(OpList& bw) {
     if (jobs.empty()) return;
+    // Row partition: the launch as a whole gets about two CTAs per SM, shared out over the jobs'
+    // column strips, so that a CTA has a few hundred rows to stream instead of 64.
+    int all_strips = 0;
+    for (const ReduceJob& j : jobs) all_strips += j.strips;
+    static const int batch_ctas = getenv("ERASE_REDUCE_CTAS") ? atoi(getenv("ERASE_REDUCE_CTAS")) : 296;
     int total = 0;
-    for (ReduceJob& j : jobs) { j.cta_begin = total; total += j.strips * j.chunks; }
+    for (ReduceJob& j : jobs) {
+      int chunks = std::max(1, batch_ctas / std::max(1, all_strips));
+      chunks = std::min(chunks, std::max(1, j.rows / 64));
+      j.chunks = chunks;
+      j.ws = chunks > 1 ? f32_buf((size_t)(j.kind == 1 ? 2 : 1) * chunks * j.cols) : nullptr;
+      j.cta_begin = total;
+      total += j.strips * j.chunks;
+    }
     const int n = (int)jobs.size();
     ReduceJob* dev = (ReduceJob*)dev_alloc(m, sizeof(ReduceJob) * jobs.size(), &ok);
     if (ok && dev && !m->dry && cudaMemcpy(dev, jobs.data(), sizeof(ReduceJob) * jobs.size(), cudaMemcpyHostToDevice) != cudaSuccess) ok = false;
@@ -778,9 +789,8 @@ struct Builder {
     if (dx) note(bw, "layernorm_bwd", 12.0 * rows * d, 4.0 * rows * d * m->esz);
     ReduceJob j;
     j.kind = 1; j.x_f32 = bf ? 0 : 1;
-    j.rows = rows; j.cols = d; j.chunks = colsum_chunks(rows, d); j.ldx = d;
+    j.rows = rows; j.cols = d; j.ldx = d;
     j.X = dy; j.X2 = x; j.a = mean; j.b = rstd;
-    j.ws = j.chunks > 1 ? f32_buf((size_t)2 * j.chunks * d) : nullptr;
     j.out0 = G(gidx); j.out1 = G(bidx); j.tickets = tickets(d);
     add_job(bw, j, 4.0 * rows * d, 2.0 * rows * d * m->esz);
   }
