@@ -4,6 +4,8 @@
 // Reductions are fixed-partition / fixed-order: no floating-point atomics anywhere.
 #include "kernels.cuh"
 
+#include <stdlib.h>
+
 #include <cuda_bf16.h>
 #include <math.h>
 
@@ -1113,6 +1115,158 @@ __global__ void __launch_bounds__(THREADS, 2) softmax_ce_packed_kernel(bf16_t* _
     }
   }
   if ((tgt >> 3) % THREADS == threadIdx.x) rowloss[row] = lse - lt;
+}
+
+// Persistent variant that also produces the head's bias gradient.  A CTA walks over rows
+// blockIdx.x, blockIdx.x + gridDim.x, ...; the next row streams into a shared-memory buffer
+// (cp.async) while the current one, held packed in registers, goes through max / exp-sum / scale,
+// so the memory system stays busy through the reductions; every thread adds the gradients it
+// writes (unrounded, fp32) to column sums it alone owns in shared memory, and the CTA leaves one
+// row of partial sums per CTA: colpart[gridDim.x][V].  Their ordered sum over the CTAs is the bias
+// gradient -- without reading the rows x V gradient matrix a second time.
+// Dynamic shared memory: V*2 bytes (row buffer) + V*4 bytes (column sums).
+template <int THREADS, int VPT>
+__global__ void __launch_bounds__(THREADS) softmax_ce_fused_kernel(bf16_t* __restrict__ logits,
+                                                                    const int32_t* __restrict__ ids, int T_,
+                                                                    float* __restrict__ rowloss, float* __restrict__ colpart,
+                                                                    int rows, int V, float inv_rows) {
+  extern __shared__ __align__(16) uint8_t dyn[];
+  __shared__ float sm[THREADS / 32];
+  uint4* buf = reinterpret_cast<uint4*>(dyn);
+  float* acc = reinterpret_cast<float*>(dyn + (size_t)V * 2);
+  const int nvec = V >> 3;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const float L2E = 1.4426950408889634f;
+  for (int i = threadIdx.x; i < V; i += THREADS) acc[i] = 0.f;
+  auto fetch = [&](int row) {
+    const uint4* src = reinterpret_cast<const uint4*>(logits + (long long)row * V);
+#pragma unroll
+    for (int k = 0; k < VPT; k++) {
+      const int i = threadIdx.x + k * THREADS;
+      if (i < nvec)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(buf + i)), "l"(src + i) : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  auto block_reduce = [&](float v, bool is_max) {
+    v = is_max ? warp_max(v) : warp_sum(v);
+    __syncthreads();
+    if (lane == 0) sm[warp] = v;
+    __syncthreads();
+    float r = sm[0];
+    for (int i = 1; i < THREADS / 32; i++) r = is_max ? fmaxf(r, sm[i]) : r + sm[i];
+    return r;
+  };
+  int row = blockIdx.x;
+  if (row < rows) fetch(row);
+  for (; row < rows; row += gridDim.x) {
+    uint4* p = reinterpret_cast<uint4*>(logits + (long long)row * V);
+    const int tgt = ids[(long long)(row / T_) * (T_ + 1) + (row % T_) + 1];
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+    uint32_t w[VPT][4];
+    float mx = -INFINITY, lt = 0.f;
+#pragma unroll
+    for (int k = 0; k < VPT; k++) {
+      const int i = threadIdx.x + k * THREADS;
+      if (i < nvec) {
+        const uint4 q = buf[i];
+        w[k][0] = q.x; w[k][1] = q.y; w[k][2] = q.z; w[k][3] = q.w;
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+          const float lo = __uint_as_float(w[k][j] << 16), hi = __uint_as_float(w[k][j] & 0xffff0000u);
+          mx = fmaxf(mx, fmaxf(lo, hi));
+          if (i * 8 + 2 * j == tgt) lt = lo;
+          if (i * 8 + 2 * j + 1 == tgt) lt = hi;
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 4; j++) w[k][j] = 0xff80ff80u;   // two bf16 -inf
+      }
+    }
+    mx = block_reduce(mx, true);                 // its first barrier also says: every thread has read buf
+    if (row + (int)gridDim.x < rows) fetch(row + gridDim.x);
+    float se = 0.f;
+#pragma unroll
+    for (int k = 0; k < VPT; k++)
+#pragma unroll
+      for (int j = 0; j < 4; j++) {
+        const float lo = exp2f((__uint_as_float(w[k][j] << 16) - mx) * L2E);
+        const float hi = exp2f((__uint_as_float(w[k][j] & 0xffff0000u) - mx) * L2E);
+        se += lo + hi;                                       // the sum uses the unrounded exponentials
+        __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+        w[k][j] = *reinterpret_cast<uint32_t*>(&h);
+      }
+    se = block_reduce(se, false);
+    const float lse = mx + logf(se);
+    const float scale = inv_rows / se;
+#pragma unroll
+    for (int k = 0; k < VPT; k++) {
+      const int i = threadIdx.x + k * THREADS;
+      if (i < nvec) {
+        uint32_t o[4];
+        float g[8];
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+          float lo = __uint_as_float(w[k][j] << 16) * scale, hi = __uint_as_float(w[k][j] & 0xffff0000u) * scale;
+          if (i * 8 + 2 * j == tgt) lo -= inv_rows;
+          if (i * 8 + 2 * j + 1 == tgt) hi -= inv_rows;
+          g[2 * j] = lo; g[2 * j + 1] = hi;
+          __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+          o[j] = *reinterpret_cast<uint32_t*>(&h);
+        }
+        p[i] = make_uint4(o[0], o[1], o[2], o[3]);
+        float4* a4 = reinterpret_cast<float4*>(acc + i * 8);   // columns i*8 .. i*8+7 belong to this thread alone
+        float4 a0 = a4[0], a1 = a4[1];
+        a0.x += g[0]; a0.y += g[1]; a0.z += g[2]; a0.w += g[3];
+        a1.x += g[4]; a1.y += g[5]; a1.z += g[6]; a1.w += g[7];
+        a4[0] = a0; a4[1] = a1;
+      }
+    }
+    if ((tgt >> 3) % THREADS == threadIdx.x) rowloss[row] = lse - lt;
+  }
+  // this CTA's column sums (zeros if it had no row)
+  float4* dst = reinterpret_cast<float4*>(colpart + (long long)blockIdx.x * V);
+#pragma unroll
+  for (int k = 0; k < VPT; k++) {
+    const int i = threadIdx.x + k * THREADS;
+    if (i < nvec) {
+      const float4* a4 = reinterpret_cast<const float4*>(acc + i * 8);
+      dst[2 * i] = a4[0];
+      dst[2 * i + 1] = a4[1];
+    }
+  }
+}
+
+int softmax_ce_fused_ctas(int rows) { return rows < 296 ? rows : 296; }
+
+bool softmax_ce_fused_supported(int V, bool bf16, const void* logits) {
+  return bf16 && V % 8 == 0 && V / 8 <= 512 * 16 && (size_t)V * 6 <= 200 * 1024 && (reinterpret_cast<uintptr_t>(logits) & 15) == 0;
+}
+
+template <int THREADS, int VPT>
+static cudaError_t softmax_ce_fused_launch(bf16_t* lg, const int32_t* ids, int T_, float* rowloss, float* colpart, int rows, int V,
+                                           float inv_rows, cudaStream_t s) {
+  const size_t smem = (size_t)V * 6;
+  static size_t attr = 0;
+  if (smem > 40 * 1024 && smem > attr) {   // dynamic + static shared memory beyond the 48 KB default
+    cudaError_t e = cudaFuncSetAttribute(softmax_ce_fused_kernel<THREADS, VPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr = smem;
+  }
+  softmax_ce_fused_kernel<THREADS, VPT><<<softmax_ce_fused_ctas(rows), THREADS, smem, s>>>(lg, ids, T_, rowloss, colpart, rows, V, inv_rows);
+  return cudaGetLastError();
+}
+
+cudaError_t softmax_ce_fused(void* logits, const int32_t* ids, int T_, float* rowloss, float* colpart, int rows, int V,
+                             float inv_rows, cudaStream_t s) {
+  const int nvec = V / 8;
+  bf16_t* lg = (bf16_t*)logits;
+  if (nvec <= 256 * 2) return softmax_ce_fused_launch<256, 2>(lg, ids, T_, rowloss, colpart, rows, V, inv_rows, s);
+  if (nvec <= 256 * 4) return softmax_ce_fused_launch<256, 4>(lg, ids, T_, rowloss, colpart, rows, V, inv_rows, s);
+  if (nvec <= 512 * 4) return softmax_ce_fused_launch<512, 4>(lg, ids, T_, rowloss, colpart, rows, V, inv_rows, s);
+  if (nvec <= 512 * 8) return softmax_ce_fused_launch<512, 8>(lg, ids, T_, rowloss, colpart, rows, V, inv_rows, s);
+  return softmax_ce_fused_launch<512, 16>(lg, ids, T_, rowloss, colpart, rows, V, inv_rows, s);
 }
 
 cudaError_t softmax_ce_inplace(void* logits, const int32_t* ids, int T_, float* rowloss, int rows, int V,

@@ -118,6 +118,14 @@ cudaError_t attention_bwd_mma(const void* qkv, const void* o, const void* dout, 
 // Softmax cross-entropy over logits [rows, V] (row stride V), in place:
 // logits <- (softmax - onehot(target)) * inv_rows; rowloss[r] = logsumexp - logit[target].
 // target of row r = ids[(r / T) * (T + 1) + (r % T) + 1].
+// The same in-place softmax-CE (bf16 logits, V % 8 == 0, V <= 32768) as a persistent kernel of
+// softmax_ce_fused_ctas(rows) CTAs that also leaves per-CTA column sums of the gradient it writes
+// (fp32, before the bf16 rounding) in colpart[ctas][V]: summed over the CTAs they are the gradient
+// of the head's bias.
+int softmax_ce_fused_ctas(int rows);
+bool softmax_ce_fused_supported(int V, bool bf16, const void* logits);
+cudaError_t softmax_ce_fused(void* logits, const int32_t* ids, int T, float* rowloss, float* colpart, int rows, int V,
+                             float inv_rows, cudaStream_t s);
 cudaError_t softmax_ce_inplace(void* logits, const int32_t* ids, int T, float* rowloss, int rows, int V,
                                float inv_rows, bool bf16, cudaStream_t s);
 // out[0] = (sum of v[0..n)) * scale, fixed-order tree in one CTA.

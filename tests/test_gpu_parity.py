@@ -77,6 +77,21 @@ def test_bf16_small(name):
     _gu().compare_teacher_forced(_bf16_cases()[name], steps=2, seed=3)
 
 
+@pytest.mark.parametrize("name", ["lm_bf16_small", "lm_bf16_ragged_T", "lm_bf16_grouped_ragged"])
+def test_bf16_small_with_the_fused_loss_and_bias_gradient_kernel(name, monkeypatch):
+    """The persistent softmax-CE kernel that also produces the head's bias gradient is chosen by
+    size (gradient matrices far beyond L2); here it is forced onto small cases, including
+    vocabularies whose vector count is not a multiple of the CTA width and fewer rows than CTAs."""
+    monkeypatch.setenv("ERASE_CE_FUSED", "2")
+    _gu().compare_teacher_forced(_bf16_cases()[name], steps=2, seed=3)
+
+
+def test_large_vocabulary_head_uses_the_fused_loss_kernel_by_size():
+    # 4224 rows x 32000 logits = 270 MB of bf16 gradients: beyond the size threshold; 4000 vectors per row
+    spec = synth.lm_spec(1, 64, 1, 128, 528, 8, 32000)
+    _gu().compare_teacher_forced(spec, steps=1, seed=4)
+
+
 def test_config2_small_lm_bf16_full_size():
     _gu().compare_teacher_forced(synth.config("C2"), steps=3, seed=0)
 
