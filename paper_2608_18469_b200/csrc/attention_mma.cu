@@ -234,13 +234,6 @@ __global__ void __launch_bounds__(128) attn_bwd_kv_mma(const bf16_t* __restrict_
   const bf16_t* base = qkv + (long long)b * T * ld + h * DH;
   const bf16_t* dob = dout + (long long)b * T * d + h * DH;
   uint32_t ka[4][4], va[4][4];
-  load_tile(Xs, base + d + (long long)k0 * ld, ld, T - k0);
-  __syncthreads();
-  load_a_frags(Xs, warp * 16, ka);
-  __syncthreads();
-  load_tile(Xs, base + 2 * d + (long long)k0 * ld, ld, T - k0);
-  __syncthreads();
-  load_a_frags(Xs, warp * 16, va);
   float dk[8][4], dv[8][4];
   zero_acc(dk);
   zero_acc(dv);
@@ -258,7 +251,17 @@ __global__ void __launch_bounds__(128) attn_bwd_kv_mma(const bf16_t* __restrict_
       LEs[buf][1][threadIdx.x] = i < T ? delta[((long long)b * H + h) * T + i] : 0.f;
     }
   };
+  // One memory round trip for the whole prologue: this key tile's K and V (K into Xs, V into the
+  // second query buffer, which the loop only refills after the fragments have been read) and the
+  // first query tile are all requested before anything is waited for.
+  load_tile_async(Xs, base + d + (long long)k0 * ld, ld, T - k0);
+  load_tile_async(QDs[1][0], base + 2 * d + (long long)k0 * ld, ld, T - k0);
   fetch(kt, 0);
+  async_wait<0>();
+  __syncthreads();
+  load_a_frags(Xs, warp * 16, ka);
+  load_a_frags(QDs[1][0], warp * 16, va);
+  __syncthreads();
   for (int it = kt; it < n_qt; it++) {
     const int i0 = it * TS;
     const int buf = (it - kt) & 1;
@@ -325,13 +328,18 @@ __global__ void __launch_bounds__(128) attn_bwd_q_mma(const bf16_t* __restrict__
   const bf16_t* base = qkv + (long long)b * T * ld + h * DH;
   const bf16_t* dob = dout + (long long)b * T * d + h * DH;
   uint32_t qa[4][4], da[4][4];
-  load_tile(Xs, base + (long long)q0 * ld, ld, T - q0);
+  // One memory round trip for the prologue: Q into Xs, dO into the second key buffer (refilled by
+  // the loop only after the fragments have been read), the first key tile into the first buffer.
+  load_tile_async(Xs, base + (long long)q0 * ld, ld, T - q0);
+  load_tile_async(KVs[1][0], dob + (long long)q0 * d, d, T - q0);
+  load_tile_async(KVs[0][0], base + d, ld, T);
+  load_tile_async(KVs[0][1], base + 2 * d, ld, T);
+  async_commit();
+  async_wait<0>();
   __syncthreads();
   load_a_frags(Xs, warp * 16, qa);
+  load_a_frags(KVs[1][0], warp * 16, da);
   __syncthreads();
-  load_tile(Xs, dob + (long long)q0 * d, d, T - q0);
-  __syncthreads();
-  load_a_frags(Xs, warp * 16, da);
   const int row_a = q0 + warp * 16 + g, row_b = row_a + 8;
   float lrow[2], erow[2];
 #pragma unroll
@@ -343,9 +351,6 @@ __global__ void __launch_bounds__(128) attn_bwd_q_mma(const bf16_t* __restrict__
   float dq[8][4];
   zero_acc(dq);
   const float sc2 = scale * 1.4426950408889634f;
-  load_tile_async(KVs[0][0], base + d, ld, T);
-  load_tile_async(KVs[0][1], base + 2 * d, ld, T);
-  async_commit();
   for (int jt = 0; jt <= qt; jt++) {
     const int j0 = jt * TS;
     if (jt < qt) {
