@@ -114,6 +114,46 @@ __device__ __forceinline__ void mma_p_x(float out[8][4], const float p[8][4], co
   }
 }
 
+// Half-tile versions for the dK/dV kernel, which works on 32 of the 64 query columns at a time so
+// that its score and dP accumulators take 32 registers instead of 64 (three CTAs per SM, not two).
+// acc[nt] (nt = 0..3: columns 32*half + 8*nt ..) += A(16 x 64) * X^T, X rows 32*half .. 32*half+31
+__device__ __forceinline__ void mma_a_xt_half(float acc[4][4], const uint32_t a[4][4], const bf16_t* x, int half) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int kk = 0; kk < 4; kk++) {
+#pragma unroll
+    for (int np = 0; np < 2; np++) {
+      const int r = (2 * half + np) * 16 + (lane & 7) + (lane >> 4) * 8;
+      const int c = kk * 16 + ((lane >> 3) & 1) * 8;
+      uint32_t b0, b1, b2, b3;
+      ldsm_x4(s_u32(x + r * LDS + c), b0, b1, b2, b3);
+      mma16816(acc[2 * np], a[kk], b0, b1);
+      mma16816(acc[2 * np + 1], a[kk], b2, b3);
+    }
+  }
+}
+// out (16 x 64) += P(16 x 32: contraction rows 32*half .. 32*half+31 of X, from accumulators p) * X
+__device__ __forceinline__ void mma_p_x_half(float out[8][4], const float p[4][4], const bf16_t* x, int half) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int kk = 0; kk < 2; kk++) {
+    uint32_t a[4];
+    a[0] = pack_bf16(p[2 * kk][0], p[2 * kk][1]);
+    a[1] = pack_bf16(p[2 * kk][2], p[2 * kk][3]);
+    a[2] = pack_bf16(p[2 * kk + 1][0], p[2 * kk + 1][1]);
+    a[3] = pack_bf16(p[2 * kk + 1][2], p[2 * kk + 1][3]);
+#pragma unroll
+    for (int np = 0; np < 4; np++) {
+      const int r = (2 * half + kk) * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+      const int c = np * 16 + (lane >> 4) * 8;
+      uint32_t b0, b1, b2, b3;
+      ldsm_x4_t(s_u32(x + r * LDS + c), b0, b1, b2, b3);
+      mma16816(out[2 * np], a, b0, b1);
+      mma16816(out[2 * np + 1], a, b2, b3);
+    }
+  }
+}
+
 __device__ __forceinline__ void zero_acc(float a[8][4]) {
 #pragma unroll
   for (int i = 0; i < 8; i++)
@@ -276,26 +316,31 @@ __global__ void __launch_bounds__(128) attn_bwd_kv_mma(const bf16_t* __restrict_
     const bf16_t* Ds = QDs[buf][1];
     const float* Ls = LEs[buf][0];
     const float* Es = LEs[buf][1];
-    float st[8][4], dp[8][4];
-    zero_acc(st);
-    zero_acc(dp);
-    mma_a_xt(st, ka, Qs);   // S^T = K Q^T
-    mma_a_xt(dp, va, Ds);   // dP^T = V dO^T
+#pragma unroll 1
+    for (int half = 0; half < 2; half++) {   // 32 query columns at a time
+      float st[4][4], dp[4][4];
 #pragma unroll
-    for (int nt = 0; nt < 8; nt++) {
+      for (int nt = 0; nt < 4; nt++)
 #pragma unroll
-      for (int e = 0; e < 4; e++) {
-        const int cl = nt * 8 + t4 * 2 + (e & 1);
-        const int qi = i0 + cl;
-        const int key = (e < 2) ? key_a : key_b;
-        const bool valid = qi < T && key <= qi;
-        const float p = valid ? exp2f(st[nt][e] * sc2 - Ls[cl]) : 0.f;
-        st[nt][e] = p;
-        dp[nt][e] = p * (dp[nt][e] - Es[cl]);
+        for (int e = 0; e < 4; e++) st[nt][e] = dp[nt][e] = 0.f;
+      mma_a_xt_half(st, ka, Qs, half);   // S^T = K Q^T
+      mma_a_xt_half(dp, va, Ds, half);   // dP^T = V dO^T
+#pragma unroll
+      for (int nt = 0; nt < 4; nt++) {
+#pragma unroll
+        for (int e = 0; e < 4; e++) {
+          const int cl = half * 32 + nt * 8 + t4 * 2 + (e & 1);
+          const int qi = i0 + cl;
+          const int key = (e < 2) ? key_a : key_b;
+          const bool valid = qi < T && key <= qi;
+          const float p = valid ? exp2f(st[nt][e] * sc2 - Ls[cl]) : 0.f;
+          st[nt][e] = p;
+          dp[nt][e] = p * (dp[nt][e] - Es[cl]);
+        }
       }
+      mma_p_x_half(dv, st, Ds, half);    // dV += P^T dO
+      mma_p_x_half(dk, dp, Qs, half);    // dK += dS^T Q
     }
-    mma_p_x(dv, st, Ds);    // dV += P^T dO
-    mma_p_x(dk, dp, Qs);    // dK += dS^T Q
     __syncthreads();        // this buffer is refilled two tiles ahead
   }
 #pragma unroll
@@ -364,22 +409,27 @@ __global__ void __launch_bounds__(128) attn_bwd_q_mma(const bf16_t* __restrict__
     __syncthreads();
     const bf16_t* Ks = KVs[jt & 1][0];
     const bf16_t* Vs = KVs[jt & 1][1];
-    float s[8][4], dp[8][4];
-    zero_acc(s);
-    zero_acc(dp);
-    mma_a_xt(s, qa, Ks);    // S = Q K^T
-    mma_a_xt(dp, da, Vs);   // dP = dO V^T
+#pragma unroll 1
+    for (int half = 0; half < 2; half++) {   // 32 key columns at a time: half the score / dP registers
+      float s[4][4], dp[4][4];
 #pragma unroll
-    for (int nt = 0; nt < 8; nt++) {
+      for (int nt = 0; nt < 4; nt++)
 #pragma unroll
-      for (int e = 0; e < 4; e++) {
-        const int col = j0 + nt * 8 + t4 * 2 + (e & 1);
-        const int row = (e < 2) ? row_a : row_b;
-        const float p = col <= row ? exp2f(s[nt][e] * sc2 - lrow[e >> 1]) : 0.f;
-        dp[nt][e] = p * (dp[nt][e] - erow[e >> 1]);
+        for (int e = 0; e < 4; e++) s[nt][e] = dp[nt][e] = 0.f;
+      mma_a_xt_half(s, qa, Ks, half);    // S = Q K^T
+      mma_a_xt_half(dp, da, Vs, half);   // dP = dO V^T
+#pragma unroll
+      for (int nt = 0; nt < 4; nt++) {
+#pragma unroll
+        for (int e = 0; e < 4; e++) {
+          const int col = j0 + half * 32 + nt * 8 + t4 * 2 + (e & 1);
+          const int row = (e < 2) ? row_a : row_b;
+          const float p = col <= row ? exp2f(s[nt][e] * sc2 - lrow[e >> 1]) : 0.f;
+          dp[nt][e] = p * (dp[nt][e] - erow[e >> 1]);
+        }
       }
+      mma_p_x_half(dq, dp, Ks, half);    // dQ += dS K
     }
-    mma_p_x(dq, dp, Ks);    // dQ += dS K
     __syncthreads();        // this buffer is refilled two tiles ahead
   }
 #pragma unroll
