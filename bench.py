@@ -179,6 +179,10 @@ def run_gpu(args, spec, cfg_name):
     split_bwd = not args.loss_on_main and not args.no_split_bwd and spec["topo"] == "chain"
     if split_bwd:
         eflags |= binding.SPLIT_BWD
+    # blocks that all read z_0 (C3): their forwards run side by side as well
+    par_fwd = not args.loss_on_main and not args.no_par_fwd and spec["topo"] == "parallel"
+    if par_fwd:
+        eflags |= binding.PAR_FWD
     units = units_per_step(spec)
 
     model = binding.Model(spec)
@@ -322,7 +326,8 @@ def run_gpu(args, spec, cfg_name):
         "scaling": "weak", "vs_baseline": None, "dtype": spec["dtype"], "data": "synthetic",
         "config": {"workload": workload_name(cfg_name, spec), "n_streams": n_streams,
                    "schedule": ("ERASE, local head+loss+backward+optimizer of each block released onto side streams after the block body"
-                                + (", parameter-gradient work of each backward on a second stream per block" if split_bwd else ""))
+                                + (", parameter-gradient work of each backward on a second stream per block" if split_bwd else "")
+                                + (", every block's forward on its own side stream too (parallel topology)" if par_fwd else ""))
                                if not args.loss_on_main else "ERASE, backward released after forward and local loss",
                    "cuda_graph": not args.no_graph, "batch_pool": POOL,
                    "l2": f"no flush: the step's working set ({arena_mb:.0f} MiB of stashes, logits, parameters) exceeds the 126 MB L2",
@@ -362,6 +367,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--loss-on-main", action="store_true", help="paper's placement of the local loss")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-par-fwd", action="store_true",
+                    help="parallel topology: keep the blocks' forwards on the main stream, one after the other")
     ap.add_argument("--no-split-bwd", action="store_true",
                     help="keep the parameter-gradient work of each B_b on the block's own side stream")
     args = ap.parse_args()

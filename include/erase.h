@@ -157,6 +157,13 @@ typedef struct {
                             shows how the phases of a REPLAYED step overlap.  A measuring aid: it adds
                             2*(2*n_blocks+1)+1 tiny kernels to the step.                               */
 
+#define ERASE_PAR_FWD 64u /* ERASE schedules on the PARALLEL topology only (every block reads z_0; ignored
+                            on chains): the blocks' forwards do not depend on one another either, so
+                            block b's whole chain F_b, l_b, B_b (and, with ERASE_BLOCK_OPT, its
+                            optimizer) runs on its side stream, released by one event behind the input
+                            staging: up to n_streams-1 blocks train side by side.  Wider than the
+                            paper's overlap of B_b with F_{b+1} (Section 2.2); same kernels, same bits. */
+
 /* Device bytes erase_create needs for this spec when given an arena; 0 if the spec is invalid. */
 ERASE_API size_t erase_arena_bytes(const erase_model_spec* spec);
 

@@ -1035,15 +1035,24 @@ erase_status enqueue_step(erase_model* m, int n_streams, unsigned flags, int tim
     static const int env_main = getenv("ERASE_SM_MAIN") ? atoi(getenv("ERASE_SM_MAIN")) : 0;
     static const int env_side = getenv("ERASE_SM_SIDE") ? atoi(getenv("ERASE_SM_SIDE")) : 0;
     const int budget_main = env_main, budget_side = env_side;
+    // Parallel topology (every block reads z_0): the forwards are independent of one another too, so
+    // with ERASE_PAR_FWD block b's whole chain F_b, l_b, B_b (and its optimizer) runs on its side
+    // stream, released by ONE event behind the input staging.
+    const bool par_fwd = (flags & ERASE_PAR_FWD) != 0 && m->spec.topo == ERASE_TOPO_PARALLEL;
+    if (par_fwd) CK(cudaEventRecord(m->ev_opt, m->main));
     for (int b = 0; b < B; b++) {
-      m->sm_budget = budget_main;
-      CK(mark(2 * b, m->main));
-      CK(run_ops(m, m->fwd[b], m->main));
-      if (!early_head) CK(run_ops(m, m->hfwd[b], m->main));
-      CK(mark(2 * b + 1, m->main));
-      CK(cudaEventRecord(m->ev_f[b], m->main));          // F_b (and l_b) are enqueued: release B_b
       cudaStream_t sd = m->side[b % ns];
-      CK(cudaStreamWaitEvent(sd, m->ev_f[b], 0));
+      cudaStream_t fs = par_fwd ? sd : m->main;          // the stream F_b runs on
+      if (par_fwd) CK(cudaStreamWaitEvent(sd, m->ev_opt, 0));
+      m->sm_budget = budget_main;
+      CK(mark(2 * b, fs));
+      CK(run_ops(m, m->fwd[b], fs));
+      if (!early_head) CK(run_ops(m, m->hfwd[b], fs));
+      CK(mark(2 * b + 1, fs));
+      if (!par_fwd) {
+        CK(cudaEventRecord(m->ev_f[b], m->main));          // F_b (and l_b) are enqueued: release B_b
+        CK(cudaStreamWaitEvent(sd, m->ev_f[b], 0));
+      }
       CK(mark(2 * (B + b), sd));
       m->sm_budget = budget_side;
       if (early_head) CK(run_ops(m, m->hfwd[b], sd));    // z_b's only other consumer is F_{b+1}, which does not wait
@@ -1273,7 +1282,7 @@ static erase_status check_step_args(erase_model* m, const erase_batch* batch);
 erase_status erase_step_ex(erase_model* m, const erase_batch* batch, int32_t n_streams, uint32_t flags) {
   if (!m) return ERASE_EINVAL;
   if (n_streams < 1) return m->fail(ERASE_EINVAL, "erase_step: n_streams must be >= 1");
-  if (flags & ~(ERASE_GRAPH | ERASE_NO_OPT | ERASE_EARLY_HEAD | ERASE_BLOCK_OPT | ERASE_SPLIT_BWD | ERASE_STAMPS)) return m->fail(ERASE_EINVAL, "erase_step: unknown flag");
+  if (flags & ~(ERASE_GRAPH | ERASE_NO_OPT | ERASE_EARLY_HEAD | ERASE_BLOCK_OPT | ERASE_SPLIT_BWD | ERASE_STAMPS | ERASE_PAR_FWD)) return m->fail(ERASE_EINVAL, "erase_step: unknown flag");
   const int stamp_mode = (flags & ERASE_STAMPS) ? 2 : 0;
   erase_status cst = check_step_args(m, batch);
   if (cst != ERASE_OK) return cst;

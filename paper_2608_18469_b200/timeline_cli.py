@@ -50,7 +50,11 @@ def main():
                          ("graph replay, ERASE, loss on the main stream", nb + 1, G),
                          ("graph replay, ERASE, head+loss+backward+optimizer on side streams", nb + 1, G | E),
                          ("graph replay, ERASE, as above with the parameter-gradient work on a second stream per block",
-                          nb + 1, G | E | binding.SPLIT_BWD)):
+                          nb + 1, G | E | binding.SPLIT_BWD),
+                         ("graph replay, ERASE, every block's forward on its side stream too (parallel topology only)",
+                          nb + 1, G | E | binding.PAR_FWD)):
+        if fl & binding.PAR_FWD and spec["topo"] != "parallel":
+            continue
         tl = None
         for _ in range(a.reps):          # the last repetition is reported (warm caches, warm clocks)
             m.step(n_streams=ns, flags=fl, **args)

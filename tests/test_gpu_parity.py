@@ -168,4 +168,10 @@ def test_erase_schedule_is_bit_identical_to_serial(name):
                                      flags=binding.GRAPH | binding.EARLY_HEAD | binding.BLOCK_OPT | binding.SPLIT_BWD))
     _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=nb + 1,
                                      flags=binding.GRAPH | binding.EARLY_HEAD | binding.BLOCK_OPT | binding.SPLIT_BWD))
+    # parallel topology: every block's forward on its side stream too (ignored on chains)
+    P = binding.PAR_FWD
+    _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=nb + 1, flags=P))
+    _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=3, flags=P | binding.EARLY_HEAD | binding.SPLIT_BWD))
+    _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=nb + 1,
+                                     flags=binding.GRAPH | binding.EARLY_HEAD | binding.BLOCK_OPT | P))
     assert serial["launches"] > 0
