@@ -62,7 +62,11 @@ typedef enum { ERASE_BLK_MLP = 0,         /* Linear act Linear ... (no activatio
 } erase_block_kind;
 typedef enum { ERASE_ACT_NONE = 0, ERASE_ACT_RELU = 1, ERASE_ACT_GELU = 2 } erase_act;
 typedef enum { ERASE_HEAD_BCE = 0,        /* Linear(d->1) + mean binary cross-entropy with logits */
-               ERASE_HEAD_SOFTMAX_CE = 1  /* Linear(d->head_out) + mean softmax cross-entropy     */
+               ERASE_HEAD_SOFTMAX_CE = 1, /* Linear(d->head_out) + mean softmax cross-entropy     */
+               ERASE_HEAD_GOODNESS = 2    /* Section 2.1: binary cross-entropy on the goodness score
+                                             G = sum_j z_j^2; logit G + bh (bh: trainable scalar, minus
+                                             the threshold), labels y (1 = positive); no head weights;
+                                             head_out = 1; dense or CTR input                     */
 } erase_head_kind;
 typedef enum { ERASE_OPT_SGD = 0, ERASE_OPT_ADAM = 1, ERASE_OPT_ADAMW = 2 } erase_opt_kind;
 typedef enum { ERASE_TOPO_CHAIN = 0,      /* block b reads sg[z_{b-1}] (Eq. 1)                    */
@@ -178,7 +182,8 @@ ERASE_API void erase_destroy(erase_model* m);
 
 /* Tensor table.  Order: frozen input tables first (tok_emb, pos_emb | table0..), then block by
  * block: MLP/TOWER W0,b0,W1,b1,..; TRANSFORMER ln1_g,ln1_b,Wqkv,bqkv,Wproj,bproj,ln2_g,ln2_b,
- * W1,b1,W2,b2; CROSS Wc0,bc0,..; DOT Wd,bd,W0,b0,..; each block ends with its head Wh,bh. */
+ * W1,b1,W2,b2; CROSS Wc0,bc0,..; DOT Wd,bd,W0,b0,..; each block ends with its head Wh,bh (the
+ * goodness head: bh only). */
 ERASE_API int32_t erase_num_tensors(const erase_model* m);
 /* block = -1 for frozen input tables; name receives a NUL-terminated string (<= 31 chars);
  * shape has rank entries (<= 2).  Errors: EINVAL (index, NULL). */

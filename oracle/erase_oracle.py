@@ -312,8 +312,19 @@ def block_backward(spec, blk, p, zin, cache, dz, grads):
         raise ValueError(k)
 
 
+def goodness_head(p, z, target):
+    """Section 2.1: binary cross-entropy applied to the goodness score G_b = sum_j z_bj^2.
+    The logit is s_n = G_n + bh (bh: trainable scalar, minus the threshold); labels 1 = positive.
+    dG/dz = 2 z, so dz = 2 ds z; the threshold's gradient is sum_n ds_n."""
+    s = np.sum(z * z, axis=1) + p["bh"][0]
+    loss, ds = bce_with_logits(s, target)
+    return loss, 2.0 * ds[:, None] * z, {"bh": np.array([ds.sum()])}
+
+
 def head_loss(blk, p, z, target):
     """Local head applied to z_b and its loss.  Returns loss, dz, {Wh, bh grads}."""
+    if blk["head"] == "goodness":
+        return goodness_head(p, z, target)
     s = linear_fwd(z, p["Wh"], p["bh"])
     if blk["head"] == "bce":
         loss, ds = bce_with_logits(s[:, 0], target)
@@ -358,6 +369,9 @@ def forward_only(spec, params, batch):
         p = {k: np.asarray(v, F) for k, v in p64.items()}
         zin = z0 if spec["topo"] == "parallel" else z
         z, _ = block_forward(spec, blk, p, zin)
+        if blk["head"] == "goodness":
+            out.append(float(goodness_head(p, z, target)[0]))
+            continue
         s = linear_fwd(z, p["Wh"], p["bh"])
         if blk["head"] == "bce":
             out.append(float(bce_with_logits(s[:, 0], target)[0]))

@@ -23,7 +23,7 @@ _DTYPE = {"f32": 0, "bf16": 1}
 _INPUT = {"dense": 0, "tokens": 1, "ctr": 2}
 _KIND = {"mlp": 0, "tower": 1, "transformer": 2, "cross": 3, "dot": 4}
 _ACT = {"none": 0, "relu": 1, "gelu": 2}
-_HEAD = {"bce": 0, "ce": 1}
+_HEAD = {"bce": 0, "ce": 1, "goodness": 2}
 _OPT = {"sgd": 0, "adam": 1, "adamw": 2}
 _TOPO = {"chain": 0, "parallel": 1}
 

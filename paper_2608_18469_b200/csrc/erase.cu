@@ -188,6 +188,9 @@ bool validate(const erase_model_spec* s, std::string* why) {
     } else if (k.head == ERASE_HEAD_SOFTMAX_CE) {
       if (s->input != ERASE_IN_TOKENS) return bad("softmax-CE head needs token input");
       if (k.head_out != s->vocab) return bad("softmax-CE head_out must equal vocab");
+    } else if (k.head == ERASE_HEAD_GOODNESS) {
+      if (k.head_out != 1) return bad("goodness head_out must be 1");
+      if (s->input == ERASE_IN_TOKENS) return bad("goodness head needs labels (dense or CTR input)");
     } else return bad("head kind");
     int out = 0;
     switch (k.kind) {
@@ -294,7 +297,7 @@ void build_tensor_table(erase_model* m) {
         linears(0);
         break;
     }
-    add_tensor(m, b, "Wh", k.head_out, out, true);
+    if (k.head != ERASE_HEAD_GOODNESS) add_tensor(m, b, "Wh", k.head_out, out, true);   // the goodness head has only its threshold
     add_tensor(m, b, "bh", k.head_out, 0, true);
   }
 }
@@ -598,6 +601,22 @@ struct Builder {
     float* rowloss = f32_buf(rows);
     float* loss_out = m->losses + b;
     float inv = 1.f / (float)rows;
+    if (k.head == ERASE_HEAD_GOODNESS) {
+      // Section 2.1: BCE on the goodness score G = sum_j z_j^2 with the logit G + bh.  The head has
+      // no weight tensor, so its threshold sits where Wh would (index wh).
+      const int bh_idx = wh;
+      float* ds = f32_buf(rows);
+      const float* bb = Wf(bh_idx);
+      f.push_back({[=](cudaStream_t s) { return goodness_head_fwd(z, d, bb, mm->cur.y, rowloss, ds, rows, d, inv, bf, s); }, 1});
+      note(f, "goodness_head_fwd", 2.0 * rows * d, (double)rows * d * m->esz);
+      f.push_back({[=](cudaStream_t s) { return reduce_sum(rowloss, rows, inv, loss_out, s); }, 1});
+      note(f, "loss_reduce", rows, 4.0 * rows);
+      bw.push_back({[=](cudaStream_t s) { return goodness_head_dz(ds, z, dz, dact, dact_src, rows, d, bf, s); }, 1});
+      note(bw, "goodness_head_dz", 2.0 * rows * d, 2.0 * rows * d * m->esz);
+      colsum_job(bw, ds, false, 1, rows, 1, nullptr, G(bh_idx), ACT_NONE, nullptr, rows, 4.0 * rows);
+      head_flush(bw);
+      return false;
+    }
     if (k.head == ERASE_HEAD_BCE) {
       float* ds = f32_buf(rows);
       const float* w = Wf(wh);

@@ -1350,6 +1350,55 @@ cudaError_t bce_head_dz(const float* ds, const float* w, void* dz, int dact, con
   return cudaGetLastError();
 }
 
+// Goodness head (binary cross-entropy on G = sum_j z_j^2 with the logit G + b): one warp per row,
+// the same outputs as the BCE head (row losses, ds = (sigmoid(s) - y)/rows).
+template <typename T>
+__global__ void __launch_bounds__(256) goodness_head_fwd_kernel(const T* __restrict__ z, long long ldz,
+                                                                const float* __restrict__ b, const float* __restrict__ y,
+                                                                float* __restrict__ rowloss, float* __restrict__ ds,
+                                                                int rows, int d, float inv_rows) {
+  int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  float s = 0.f;
+  for (int c = lane; c < d; c += 32) {
+    const float v = ldf(z + (long long)row * ldz + c);
+    s = fmaf(v, v, s);
+  }
+  s = warp_sum(s) + b[0];
+  if (lane == 0) {
+    float yy = y[row];
+    float e = expf(-fabsf(s));
+    rowloss[row] = fmaxf(s, 0.f) - s * yy + log1pf(e);
+    float sig = s >= 0.f ? 1.f / (1.f + e) : e / (1.f + e);
+    ds[row] = (sig - yy) * inv_rows;
+  }
+}
+cudaError_t goodness_head_fwd(const void* z, long long ldz, const float* b, const float* y, float* rowloss, float* ds,
+                              int rows, int d, float inv_rows, bool bf16, cudaStream_t s) {
+  if (bf16) goodness_head_fwd_kernel<bf16_t><<<cdiv(rows, 8), 256, 0, s>>>((const bf16_t*)z, ldz, b, y, rowloss, ds, rows, d, inv_rows);
+  else goodness_head_fwd_kernel<float><<<cdiv(rows, 8), 256, 0, s>>>((const float*)z, ldz, b, y, rowloss, ds, rows, d, inv_rows);
+  return cudaGetLastError();
+}
+
+// dz = 2 ds z (times act'(src) when z = act(src) closes the block)
+template <typename T>
+__global__ void __launch_bounds__(256) goodness_head_dz_kernel(const float* __restrict__ ds, const T* __restrict__ z,
+                                                               T* __restrict__ dz, int dact, const T* __restrict__ src,
+                                                               long long n, int d) {
+  long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (i >= n) return;
+  float v = 2.f * ds[i / d] * ldf(z + i);
+  if (dact != ACT_NONE) v *= act_deriv(dact, ldf(src + i));
+  stf(dz + i, v);
+}
+cudaError_t goodness_head_dz(const float* ds, const void* z, void* dz, int dact, const void* src, int rows,
+                             int d, bool bf16, cudaStream_t s) {
+  long long n = (long long)rows * d;
+  if (bf16) goodness_head_dz_kernel<bf16_t><<<cdiv(n, 256), 256, 0, s>>>(ds, (const bf16_t*)z, (bf16_t*)dz, dact, (const bf16_t*)src, n, d);
+  else goodness_head_dz_kernel<float><<<cdiv(n, 256), 256, 0, s>>>(ds, (const float*)z, (float*)dz, dact, (const float*)src, n, d);
+  return cudaGetLastError();
+}
+
 // ------------------------------------------------------------------------------------------
 // elementwise
 // ------------------------------------------------------------------------------------------

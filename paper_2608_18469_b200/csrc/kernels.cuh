@@ -138,6 +138,11 @@ cudaError_t bce_head_fwd(const void* z, long long ldz, const float* w, const flo
 // dz[r,c] = ds[r] * w[c]  (times act'(src[r,c]) when dact != ACT_NONE)
 cudaError_t bce_head_dz(const float* ds, const float* w, void* dz, int dact, const void* src, int rows,
                         int d, bool bf16, cudaStream_t s);
+// Goodness head: s[r] = sum_c z[r,c]^2 + b[0]; rowloss and ds as for the BCE head; dz = 2 ds z (* act'(src)).
+cudaError_t goodness_head_fwd(const void* z, long long ldz, const float* b, const float* y, float* rowloss, float* ds,
+                              int rows, int d, float inv_rows, bool bf16, cudaStream_t s);
+cudaError_t goodness_head_dz(const float* ds, const void* z, void* dz, int dact, const void* src, int rows,
+                             int d, bool bf16, cudaStream_t s);
 
 // out = a (.) b, all [n] of T
 cudaError_t ew_mul(const void* a, const void* b, void* out, long long n, bool bf16, cudaStream_t s);

@@ -14,7 +14,7 @@ A *spec* is a plain dict::
      "n_dense", "n_sparse", "table_rows", "emb_dim",   # ctr
      "blocks": [ {"kind": "mlp"|"tower"|"transformer"|"cross"|"dot",
                   "dims": [...], "act": "none"|"relu"|"gelu",
-                  "n_heads": int, "n_cross": int, "head": "bce"|"ce",
+                  "n_heads": int, "n_cross": int, "head": "bce"|"ce"|"goodness",
                   "head_out": int}, ... ],
      "opt": {"kind": "sgd"|"adam"|"adamw", "lr", "beta1", "beta2", "eps", "wd"}}
 
@@ -45,9 +45,9 @@ def _opt(kind, lr, wd=0.0):
 # the five workloads (shapes of the paper's MNIST-MLP, NanoChat and CTR models)
 # ----------------------------------------------------------------------------
 
-def mlp_spec(width, hidden, n_blocks, batch, act, dtype, opt=None):
+def mlp_spec(width, hidden, n_blocks, batch, act, dtype, opt=None, head="bce"):
     blk = {"kind": "mlp", "dims": [width, hidden, width], "act": act,
-           "head": "bce", "head_out": 1}
+           "head": head, "head_out": 1}
     return {"dtype": dtype, "input": "dense", "topo": "chain", "batch": batch,
             "width": width, "blocks": [dict(blk) for _ in range(n_blocks)],
             "opt": opt or _opt("sgd", 1e-2)}
@@ -150,7 +150,8 @@ def tensor_list(spec):
             d_out = dims[-1]
         else:
             raise ValueError(k)
-        out.append((b, "Wh", (blk["head_out"], d_out), True))
+        if blk["head"] != "goodness":                  # the goodness head has no weights, only its threshold bh
+            out.append((b, "Wh", (blk["head_out"], d_out), True))
         out.append((b, "bh", (blk["head_out"],), True))
     return out
 
@@ -178,12 +179,13 @@ def init_params(spec, seed=0, zero_heads=False):
     smaller 1/sqrt(in) bound an 8-deep stack without residuals or norms collapses every sample
     onto the same bias-driven vector, and the gradients become differences of nearly equal sums);
     Linear b ~ U(-1/sqrt(in), 1/sqrt(in)); LayerNorm gain 1, shift 0; CTR tables N(0, (1/8)^2);
-    token embedding N(0, 1); position embedding N(0, 0.1^2).
+    token embedding N(0, 1); position embedding N(0, 0.1^2); the goodness head's threshold bh = minus
+    half the width of z_b (the sum of squares of a unit-variance z_b is about that width).
     Returns a list of float32 arrays aligned with ``tensor_list(spec)``.
     """
     rng = np.random.Generator(np.random.PCG64(seed))
     vals = []
-    fan_in = None
+    fan_in = fan_out = None
     for (b, name, shape, _tr) in tensor_list(spec):
         if name == "tok_emb":
             v = rng.standard_normal(shape)
@@ -196,7 +198,7 @@ def init_params(spec, seed=0, zero_heads=False):
         elif name.endswith("_b") and name.startswith("ln"):
             v = np.zeros(shape)
         elif len(shape) == 2:                       # Linear weight [out, in]
-            fan_in = shape[1]
+            fan_in, fan_out = shape[1], shape[0]
             gain = 2.0 if _followed_by_activation(spec["blocks"][b], name) else 1.0
             bound = math.sqrt(3.0 * gain / fan_in)
             v = rng.uniform(-bound, bound, shape)
@@ -205,6 +207,8 @@ def init_params(spec, seed=0, zero_heads=False):
         else:                                       # Linear bias
             bound = 1.0 / math.sqrt(fan_in)
             v = rng.uniform(-bound, bound, shape)
+            if name == "bh" and b >= 0 and spec["blocks"][b]["head"] == "goodness":
+                v = np.full(shape, -0.5 * fan_out)
             if zero_heads and name == "bh":
                 v = np.zeros(shape)
         vals.append(np.ascontiguousarray(v, dtype=np.float32))

@@ -69,6 +69,11 @@ def _bf16_cases():
     # enough rows (>= 512) for the grouped weight-gradient kernel, with ragged M / N / K tails in every problem
     s["lm_bf16_grouped_ragged"] = synth.lm_spec(2, 192, 3, 328, 100, 6, 777)
     s["mlp_bf16_grouped_ragged"] = synth.mlp_spec(200, 328, 2, 600, "relu", "bf16")
+    # the goodness objective (BCE on sum_j z_j^2) as the local loss, with and without a closing activation
+    s["mlp_bf16_goodness"] = synth.mlp_spec(128, 256, 3, 512, "gelu", "bf16", head="goodness")
+    s["tower_bf16_goodness"] = synth.mlp_spec(128, 256, 2, 512, "relu", "bf16", head="goodness")
+    for blk in s["tower_bf16_goodness"]["blocks"]:
+        blk["kind"] = "tower"
     return s
 
 
@@ -142,13 +147,14 @@ def _bits_equal(a, b):
         assert a[k].tobytes() == b[k].tobytes(), k
 
 
-@pytest.mark.parametrize("name", ["C1", "lm", "ctr", "c5"])
+@pytest.mark.parametrize("name", ["C1", "lm", "ctr", "c5", "goodness"])
 def test_erase_schedule_is_bit_identical_to_serial(name):
     gu = _gu()
     spec = {"C1": synth.config("C1"),
             "lm": synth.lm_spec(3, 128, 2, 256, 64, 4, 512),
             "ctr": synth.ctr_spec(batch=256, table_rows=500, tower=(128, 64, 32)),
-            "c5": synth.config("C5", w=128, batch=512)}[name]
+            "c5": synth.config("C5", w=128, batch=512),
+            "goodness": synth.mlp_spec(128, 256, 3, 512, "gelu", "bf16", head="goodness")}[name]
     flat = synth.init_params(spec, 5)
     batches = [gu.DevBatch(spec, synth.make_batch(spec, 5, index=i)) for i in range(4)]
     serial = gu.run_steps(spec, flat, batches, n_streams=1)

@@ -150,9 +150,30 @@ def test_one_layer_bce_worked_example():
             assert np.allclose(params["blocks"][0]["Wh"][0], stp["w_after"], atol=1e-12, rtol=0)
 
 
+def test_goodness_head_closed_forms():
+    """Section 2.1's goodness objective, pinned by hand: with z = (3, 4) the score is G = 25; with
+    the threshold at 25 (bh = -25) the logit is 0, so a single row costs ln 2, ds = (1/2 - y)/N
+    and dz = 2 ds z; one positive and one negative row with the same z cancel exactly in dbh."""
+    z = np.array([[3.0, 4.0], [3.0, 4.0]])
+    p = {"bh": np.array([-25.0])}
+    y = np.array([1.0, 0.0])
+    loss, dz, g = orc.goodness_head(p, z, y)
+    assert abs(loss - math.log(2.0)) < 1e-15
+    assert np.allclose(dz, [[-1.5, -2.0], [1.5, 2.0]], atol=1e-15)      # 2 * (+-1/4) * z
+    assert abs(g["bh"][0]) < 1e-16 and set(g) == {"bh"}
+    # far above / below the threshold the loss is the margin itself (softplus -> identity / 0)
+    big, _, _ = orc.goodness_head({"bh": np.array([0.0])}, np.array([[30.0, 40.0]]), np.array([0.0]))
+    assert abs(big - 2500.0) < 1e-9
+    small, dz0, _ = orc.goodness_head({"bh": np.array([-5000.0])}, np.array([[30.0, 40.0]]), np.array([0.0]))
+    assert small < 1e-100
+    assert np.all(np.abs(dz0) < 1e-100)
+
+
 @pytest.mark.parametrize("name", list(util.tiny_specs()))
 def test_zero_heads_give_ln2_or_lnV_and_zero_body_gradients(name):
     spec = util.tiny_specs()[name]
+    if any(blk["head"] == "goodness" for blk in spec["blocks"]):
+        pytest.skip("the goodness head has no weights to zero: its closed forms are pinned separately")
     params, batch = _setup(spec, seed=0, zero_heads=True)
     losses, grads = orc.forward_backward(spec, params, batch)
     for b, blk in enumerate(spec["blocks"]):

@@ -70,6 +70,9 @@ def _torch_step(spec, tparams, z0, target, optim):
     for blk, p in zip(spec["blocks"], tparams):
         zin = (z0 if spec["topo"] == "parallel" else z).detach()
         z = _torch_block(spec, blk, p, zin)
+        if blk["head"] == "goodness":       # BCE on the goodness score G = sum_j z_j^2, threshold bh (Section 2.1)
+            losses.append(TF.binary_cross_entropy_with_logits((z * z).sum(dim=1) + p["bh"][0], target))
+            continue
         s = TF.linear(z, p["Wh"], p["bh"])
         if blk["head"] == "bce":
             losses.append(TF.binary_cross_entropy_with_logits(s[:, 0], target))

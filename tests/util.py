@@ -29,6 +29,10 @@ def tiny_specs():
     s["lm"] = synth.lm_spec(2, 4, 2, 6, 3, 2, 5, dtype="f32")
     s["ctr"] = synth.ctr_spec(batch=3, n_dense=2, n_sparse=3, table_rows=7, emb_dim=4,
                               tower=(6, 5, 4), n_cross=2, dtype="f32")
+    s["mlp_goodness"] = synth.mlp_spec(4, 6, 2, 5, "relu", "f32", head="goodness")
+    s["tower_goodness"] = synth.mlp_spec(4, 6, 2, 5, "gelu", "f32", head="goodness")
+    for blk in s["tower_goodness"]["blocks"]:
+        blk["kind"] = "tower"       # the activation also follows the last Linear: z_b = act(u)
     return s
 
 
