@@ -22,14 +22,17 @@ aggregate objective with each z_{b-1} held constant inside block b.
 The paper does not fix f_b, the heads, the losses or the optimizer; the readings
 used here (mean reductions, exact-erf GELU, biased-variance LayerNorm with eps
 1e-5, pre-LN transformer, full-rank DCN-v2 cross layers, strict-lower-triangle
-dot interaction, PyTorch-convention Adam/AdamW) are the ones listed in the
-design notes of this repository.
+dot interaction, PyTorch-convention Adam/AdamW; heads: Linear + mean BCE with
+logits, Linear + mean softmax cross-entropy, or Section 2.1's example itself,
+BCE on the goodness score G_b = sum_j z_bj^2 with a trainable threshold) are the
+ones listed in the design notes of this repository.
 
 Pins (tests/test_oracle_*.py): central finite differences on every parameter of
 every block kind; torch CPU autograd in float64 with .detach() between blocks;
 the stop-gradient invariants; hand-derived closed forms for one-layer logistic
-regression, zero heads (ln 2, ln V), identity cross layers; conservation laws of
-softmax, LayerNorm and attention; Adam's first step.
+regression, zero heads (ln 2, ln V), identity cross layers, the goodness head
+at and far from its threshold; conservation laws of softmax, LayerNorm and
+attention; Adam's first step.
 
 Parameter containers: ``params = {"input": {name: array}, "blocks": [{name: array}, ...]}``.
 """
