@@ -232,13 +232,21 @@ def run_gpu(args, spec, cfg_name):
             per = np.array([evs[i].elapsed_time(evs[i + 1]) for i in range(steps)])
             return max_over_ranks(total_ms), per, model.launch_count() - l0
 
+        def progress(what):   # BENCH_PROGRESS=1: which leg is running, on stderr
+            if os.environ.get("BENCH_PROGRESS"):
+                print(f"[bench] {what}", file=sys.stderr, flush=True)
+
         sampler = ClockSampler(local)
         # serial first (context), then the ERASE schedule under the clock sampler
+        progress("serial leg")
         ser_ms, ser_per, _ = timed(1, flags, args.steps, args.warmup)
         sampler.start()
+        progress("ERASE leg")
         era_ms, era_per, launches = timed(n_streams, eflags, args.steps, args.warmup)
+        progress("ERASE leg, loss on the main stream")
         pap_ms, pap_per, _ = timed(n_streams, flags, args.steps, args.warmup) if eflags != flags else (era_ms, era_per, 0)
         clocks = sampler.stop()
+        progress("end-to-end leg")
 
         # end to end through the C ABI: pinned host batch -> device copy, step, losses back to host
         stage = {k: torch.empty_like(v) for k, v in dev[0].items()}
@@ -263,6 +271,7 @@ def run_gpu(args, spec, cfg_name):
         e2e_ms = max_over_ranks(1e3 * (time.perf_counter() - t0))
 
         # per-kernel attribution: profiled serial steps (events around every operation)
+        progress("profiled steps")
         agg = {}
         nprof = 3
         for i in range(nprof + 1):

@@ -612,7 +612,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 //   tfull[a]   per CTA: accumulator a is complete (delivered to both CTAs)
 //   tempty[a]  leader only: both CTAs' epilogue warps have drained accumulator a (the peer's warps
 //              arrive on it through the cluster's shared-memory window)
-// Tiles are claimed by the leader (dynamic scheduling), in the order of tile_coords.  The output must be
+// Tiles are assigned round-robin to clusters, in the order of tile_coords.  The output must be
 // describable to TMA (it leaves through staged TMA stores); GENERAL as in tc_gemm_kernel.
 constexpr int PAIR_BN = 256;
 constexpr int PAIR_STAGES = 4;
@@ -631,26 +631,6 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {  
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
-}
-// wait on a barrier of this CTA that a thread of the PEER CTA arrives on: acquire at cluster scope
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity) {
-  auto try_wait = [&]() {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-  };
-  if (try_wait()) return true;
-  long long t0 = clock64();
-  while (!try_wait()) {
-    if (clock64() - t0 > WAIT_LIMIT_CYCLES) return false;
-  }
-  return true;
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
@@ -695,17 +675,10 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
-  // tile queue: the leader's producer claims tiles (atomic counter, as in tc_gemm_kernel) and publishes
-  // each one to a 4-entry ring in BOTH CTAs; every role reads its own CTA's ring, and every consumer
-  // of the pair hands the slot back on the LEADER's tq_empty barrier
-  auto tq_full = [&](int i) { return bar_base + 8u * (2 * STAGES + 6 + i); };
-  auto tq_empty = [&](int i) { return bar_base + 8u * (2 * STAGES + 10 + i); };
-  const uint32_t ring_base = bar_base + 8u * (2 * STAGES + 14);
   uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
   volatile uint32_t* tmem_slot_ptr =
       reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * (EPI_STAGE_BYTES + EPI_BIAS_BYTES) + 8u * (2 * STAGES + 4));
   const uint32_t tmem_slot = bar_base + 8u * (2 * STAGES + 4);
-  volatile int* tile_ring = reinterpret_cast<volatile int*>(gen_base + (ring_base - smem_base));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
@@ -730,10 +703,6 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       mbar_init(tfull_bar(a), 1);
       mbar_init(tempty_bar(a), 2 * EPI_WARPS);
     }
-    for (int i = 0; i < 4; i++) {
-      mbar_init(tq_full(i), 1);
-      mbar_init(tq_empty(i), 2 * (1 + EPI_WARPS));   // leader: MMA + epilogue warps; peer: producer + epilogue warps
-    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -751,26 +720,9 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   if (warp == 0) {
     // ------------------------------ TMA producer (both CTAs) ------------------------------
     if (lane == 0) {
-      uint32_t it = 0, slot = 0;
+      uint32_t it = 0;
       bool ok = true;
-      int t = cluster_id < total ? cluster_id : -1;
-      while (ok) {
-        int next = -1;
-        if (leader) {
-          // publish the tile (or the end marker -1) to both CTAs
-          if (!mbar_wait(tq_empty(slot & 3), ((slot >> 2) & 1) ^ 1)) { atomicExch(p.status, 5); ok = false; break; }
-          tile_ring[slot & 3] = t;
-          asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(map_to_cta(ring_base + 4u * (slot & 3), 1)), "r"(t) : "memory");
-          mbar_arrive(tq_full(slot & 3));
-          mbar_arrive_cluster(map_to_cta(tq_full(slot & 3), 1));   // release at cluster scope: the peer sees the tile id
-          if (t >= 0) next = p.sched ? n_clusters + atomicAdd(p.sched, 1) : t + n_clusters;   // latency hides behind this tile's loads
-        } else {
-          if (!mbar_wait_cluster(tq_full(slot & 3), (slot >> 2) & 1)) { atomicExch(p.status, 5); ok = false; break; }
-          t = tile_ring[slot & 3];
-          mbar_arrive_cluster(map_to_cta(tq_empty(slot & 3), 0));
-        }
-        slot++;
-        if (t < 0) break;
+      for (int t = cluster_id; t < total && ok; t += n_clusters) {
         int mt, nt, split;
         tile_coords(t, tiles_m, tiles_n, mt, nt, split);
         const int m0 = mt * 2 * BM + (int)rank * BM;        // this CTA's 128 rows of A
@@ -799,7 +751,6 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             for (int a = 0; a < BN / 128; a++) tma_load_2d_pair(b_dst + a * (BK * 128), &map_b, nb0 + a * 64, k0, lfull);
           }
         }
-        if (leader) t = next < total ? next : -1;
       }
       if (!ok) {  // give copies already in flight time to land before the CTA's shared memory is released
         const long long t0 = clock64();
@@ -813,11 +764,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                              ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
       uint32_t it = 0, lt = 0;
       bool ok = true;
-      for (;; lt++) {
-        if (!mbar_wait(tq_full(lt & 3), (lt >> 2) & 1)) { atomicExch(p.status, 6); break; }
-        const int t = tile_ring[lt & 3];
-        mbar_arrive(tq_empty(lt & 3));
-        if (t < 0 || !ok) break;
+      for (int t = cluster_id; t < total && ok; t += n_clusters, lt++) {
         const int split = t / (tiles_m * tiles_n);
         const int kbeg = split * kchunk, kend = min(p.K, kbeg + kchunk);
         const int num_kb = kend > kbeg ? (kend - kbeg + BK - 1) / BK : 0;
@@ -858,19 +805,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const uint32_t ltempty0 = map_to_cta(tempty_bar(0), 0), ltempty1 = map_to_cta(tempty_bar(1), 0);
     bool store_pending = false;
     uint32_t lt = 0;
-    for (;; lt++) {
-      int t = -1;
-      if (lane == 0) {
-        if (mbar_wait_cluster(tq_full(lt & 3), (lt >> 2) & 1)) {
-          t = tile_ring[lt & 3];
-          if (leader) mbar_arrive(tq_empty(lt & 3));
-          else mbar_arrive_cluster(map_to_cta(tq_empty(lt & 3), 0));
-        } else {
-          atomicExch(p.status, 7);
-        }
-      }
-      t = __shfl_sync(0xffffffffu, t, 0);
-      if (t < 0) break;
+    for (int t = cluster_id; t < total; t += n_clusters, lt++) {
       int mt, nt, split;
       tile_coords(t, tiles_m, tiles_n, mt, nt, split);
       const int m0 = mt * 2 * BM + (int)rank * BM, n0 = nt * BN;
@@ -983,14 +918,6 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
-  }
-  if (p.sched && leader && threadIdx.x == 0) {   // the pair that finishes last leaves the scheduler words at zero
-    __threadfence();
-    if (atomicAdd(p.sched + 1, 1) == n_clusters - 1) {
-      p.sched[0] = 0;
-      p.sched[1] = 0;
-      __threadfence();
-    }
   }
 }
 
@@ -1305,7 +1232,7 @@ cudaError_t launch_pair_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s,
   TcArgs p;
   p.M = g.M; p.N = g.N; p.K = g.K;
   p.C = g.C; p.ldc = g.ldc; p.c_f32 = g.c_f32;
-  p.splits = g.splits; p.ws = g.ws; p.epi = g.epi; p.status = plan.status; p.dbg = plan.dbg; p.sched = plan.sched;
+  p.splits = g.splits; p.ws = g.ws; p.epi = g.epi; p.status = plan.status; p.dbg = plan.dbg; p.sched = nullptr;
   p.tma_c = 1;
   const Epilogue& e = g.epi;
   const bool no_aux = e.alpha == 1.f && e.act == ACT_NONE && !e.pre_out && !e.mul && !e.res && e.dact == ACT_NONE;
@@ -1319,8 +1246,6 @@ cudaError_t launch_pair_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s,
   const long long total = (long long)((g.N + PAIR_BN - 1) / PAIR_BN) * ((g.M + 2 * BM - 1) / (2 * BM)) * g.splits;
   long long cap = ((max_ctas > 1 && max_ctas < num_sms) ? max_ctas : num_sms) / 2;
   dim3 grid(2u * (unsigned)(total < cap ? total : cap));
-  static const int env_static = getenv("ERASE_PAIR_STATIC") ? atoi(getenv("ERASE_PAIR_STATIC")) : 0;
-  if (env_static || total <= (long long)(grid.x / 2)) p.sched = nullptr;   // one tile per pair: nothing to balance
   CUtensorMap ma, mb, mc;
   memcpy(&ma, plan.map_a, sizeof(ma));
   memcpy(&mb, plan.b_mn ? plan.map_b : plan.map_b_half, sizeof(mb));
