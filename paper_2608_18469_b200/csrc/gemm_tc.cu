@@ -13,6 +13,10 @@
 //               tile's main loop
 // Every mbarrier wait is bounded by a clock limit; on expiry the kernel records a status word,
 // skips the rest of its work, still frees its TMEM and returns.
+//
+// Two more kernels further down share these roles and helpers: tc_gemm_pair_kernel (two CTAs of a
+// cluster on one 256 x 256 tile, tcgen05 cta_group::2) for GEMMs with enough tiles to fill the 74
+// CTA pairs, and tc_wgrad_group_kernel (up to four small weight-gradient GEMMs in one launch).
 #include "gemm_tc.cuh"
 
 #include <cuda.h>

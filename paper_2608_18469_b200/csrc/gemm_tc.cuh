@@ -1,9 +1,11 @@
 // Tensor-core GEMM path for bf16 models on sm_100a: operands staged in shared memory by TMA
 // (cp.async.bulk.tensor, 128-byte swizzle), tcgen05.mma issued by one thread with the fp32
 // accumulator in tensor memory (TMEM), epilogue warps reading it back with tcgen05.ld and
-// applying the fused epilogue (bias, activation, residual, DCN-v2 cross, activation derivative).
+// applying the fused epilogue (bias, ReLU, residual, DCN-v2 cross, ReLU derivative; GEMMs that ask
+// for GELU or a pre-activation copy are refused here and use the SIMT kernel).
 // One kernel serves the forward (both operands K-major), the dgrad (B MN-major) and the wgrad
-// (both MN-major), so no operand is ever transposed in memory.
+// (both MN-major), so no operand is ever transposed in memory.  tc_gemm_plan picks the single-CTA
+// kernel (128 x BN tiles) or the CTA-pair kernel (256 x 256 tiles over two SMs, cta_group::2).
 #pragma once
 #include <cuda_runtime.h>
 
