@@ -426,8 +426,68 @@ __global__ void __launch_bounds__(256) layernorm_fwd_kernel(const T* __restrict_
   if (lane == 0) { mean[row] = mu; rstd[row] = r; }
 }
 
+// bf16 rows of d = 256*VPL columns: a lane keeps VPL 16-byte pieces of its row in registers, so the
+// row is read once (the generic kernel above walks over it three times, two bytes per lane and load).
+template <int VPL>
+__global__ void __launch_bounds__(256) layernorm_fwd_vec_kernel(const bf16_t* __restrict__ x, const float* __restrict__ gain,
+                                                                const float* __restrict__ shift, bf16_t* __restrict__ y,
+                                                                float* __restrict__ mean, float* __restrict__ rstd,
+                                                                int rows, int d) {
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  const bf16_t* xr = x + (long long)row * d;
+  float v[VPL][8];
+  float s = 0.f;
+#pragma unroll
+  for (int k = 0; k < VPL; k++) {
+    ld_vec<bf16_t>(xr + (k * 32 + lane) * 8, v[k]);
+#pragma unroll
+    for (int j = 0; j < 8; j++) s += v[k][j];
+  }
+  const float mu = warp_sum(s) / d;
+  float q = 0.f;
+#pragma unroll
+  for (int k = 0; k < VPL; k++)
+#pragma unroll
+    for (int j = 0; j < 8; j++) { const float t = v[k][j] - mu; q = fmaf(t, t, q); }
+  const float r = rsqrtf(warp_sum(q) / d + 1e-5f);
+#pragma unroll
+  for (int k = 0; k < VPL; k++) {
+    const int c = (k * 32 + lane) * 8;
+    const float4 g0 = *reinterpret_cast<const float4*>(gain + c), g1 = *reinterpret_cast<const float4*>(gain + c + 4);
+    const float4 b0 = *reinterpret_cast<const float4*>(shift + c), b1 = *reinterpret_cast<const float4*>(shift + c + 4);
+    const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+    const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+    float o[8];
+#pragma unroll
+    for (int j = 0; j < 8; j++) o[j] = (v[k][j] - mu) * r * gg[j] + bb[j];
+    uint4 w;
+    __nv_bfloat162 h;
+    h = __floats2bfloat162_rn(o[0], o[1]); w.x = *reinterpret_cast<uint32_t*>(&h);
+    h = __floats2bfloat162_rn(o[2], o[3]); w.y = *reinterpret_cast<uint32_t*>(&h);
+    h = __floats2bfloat162_rn(o[4], o[5]); w.z = *reinterpret_cast<uint32_t*>(&h);
+    h = __floats2bfloat162_rn(o[6], o[7]); w.w = *reinterpret_cast<uint32_t*>(&h);
+    *reinterpret_cast<uint4*>(y + (long long)row * d + c) = w;
+  }
+  if (lane == 0) { mean[row] = mu; rstd[row] = r; }
+}
+
 cudaError_t layernorm_fwd(const void* x, const float* gain, const float* shift, void* y, float* mean,
                           float* rstd, int rows, int d, bool bf16, cudaStream_t s) {
+  const bool al = ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y) | reinterpret_cast<uintptr_t>(gain) |
+                    reinterpret_cast<uintptr_t>(shift)) & 15) == 0;
+  if (bf16 && al && d % 256 == 0 && d <= 1024) {
+    const bf16_t* xb = (const bf16_t*)x;
+    bf16_t* yb = (bf16_t*)y;
+    const unsigned grid = cdiv(rows, 8);
+    switch (d / 256) {
+      case 1: layernorm_fwd_vec_kernel<1><<<grid, 256, 0, s>>>(xb, gain, shift, yb, mean, rstd, rows, d); break;
+      case 2: layernorm_fwd_vec_kernel<2><<<grid, 256, 0, s>>>(xb, gain, shift, yb, mean, rstd, rows, d); break;
+      case 3: layernorm_fwd_vec_kernel<3><<<grid, 256, 0, s>>>(xb, gain, shift, yb, mean, rstd, rows, d); break;
+      default: layernorm_fwd_vec_kernel<4><<<grid, 256, 0, s>>>(xb, gain, shift, yb, mean, rstd, rows, d); break;
+    }
+    return cudaGetLastError();
+  }
   if (bf16) layernorm_fwd_kernel<bf16_t><<<cdiv(rows, 8), 256, 0, s>>>((const bf16_t*)x, gain, shift, (bf16_t*)y, mean, rstd, rows, d);
   else layernorm_fwd_kernel<float><<<cdiv(rows, 8), 256, 0, s>>>((const float*)x, gain, shift, (float*)y, mean, rstd, rows, d);
   return cudaGetLastError();
