@@ -521,9 +521,72 @@ __global__ void __launch_bounds__(256) layernorm_bwd_dx_kernel(const T* __restri
   }
 }
 
+// bf16 rows of d = 256*VPL columns: dy and x are read once (16-byte pieces kept in registers)
+template <int VPL>
+__global__ void __launch_bounds__(256) layernorm_bwd_dx_vec_kernel(const bf16_t* __restrict__ dy, const bf16_t* __restrict__ x,
+                                                                   const float* __restrict__ gain,
+                                                                   const float* __restrict__ mean,
+                                                                   const float* __restrict__ rstd, const bf16_t* add,
+                                                                   bf16_t* dx, int rows, int d) {
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  const long long o = (long long)row * d;
+  const float mu = mean[row], r = rstd[row];
+  float g[VPL][8], xh[VPL][8];
+  float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+  for (int k = 0; k < VPL; k++) {
+    const int c = (k * 32 + lane) * 8;
+    ld_vec<bf16_t>(dy + o + c, g[k]);
+    ld_vec<bf16_t>(x + o + c, xh[k]);
+    const float4 g0 = *reinterpret_cast<const float4*>(gain + c), g1 = *reinterpret_cast<const float4*>(gain + c + 4);
+    const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+#pragma unroll
+    for (int j = 0; j < 8; j++) {
+      g[k][j] *= gg[j];
+      xh[k][j] = (xh[k][j] - mu) * r;
+      s1 += g[k][j];
+      s2 += g[k][j] * xh[k][j];
+    }
+  }
+  s1 = warp_sum(s1) / d;
+  s2 = warp_sum(s2) / d;
+#pragma unroll
+  for (int k = 0; k < VPL; k++) {
+    const int c = (k * 32 + lane) * 8;
+    float v[8], a[8];
+    if (add) ld_vec<bf16_t>(add + o + c, a);
+#pragma unroll
+    for (int j = 0; j < 8; j++) {
+      v[j] = r * (g[k][j] - s1 - xh[k][j] * s2);
+      if (add) v[j] += a[j];
+    }
+    uint4 w;
+    __nv_bfloat162 h;
+    h = __floats2bfloat162_rn(v[0], v[1]); w.x = *reinterpret_cast<uint32_t*>(&h);
+    h = __floats2bfloat162_rn(v[2], v[3]); w.y = *reinterpret_cast<uint32_t*>(&h);
+    h = __floats2bfloat162_rn(v[4], v[5]); w.z = *reinterpret_cast<uint32_t*>(&h);
+    h = __floats2bfloat162_rn(v[6], v[7]); w.w = *reinterpret_cast<uint32_t*>(&h);
+    *reinterpret_cast<uint4*>(dx + o + c) = w;
+  }
+}
+
 cudaError_t layernorm_bwd_dx(const void* dy, const void* x, const float* gain, const float* mean,
                              const float* rstd, const void* add, void* dx, int rows, int d, bool bf16,
                              cudaStream_t s) {
+  const bool al = ((reinterpret_cast<uintptr_t>(dy) | reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(gain) |
+                    reinterpret_cast<uintptr_t>(add) | reinterpret_cast<uintptr_t>(dx)) & 15) == 0;
+  if (bf16 && al && d % 256 == 0 && d <= 1024) {
+    const bf16_t* a = (const bf16_t*)dy; const bf16_t* b = (const bf16_t*)x; const bf16_t* c = (const bf16_t*)add; bf16_t* o = (bf16_t*)dx;
+    const unsigned grid = cdiv(rows, 8);
+    switch (d / 256) {
+      case 1: layernorm_bwd_dx_vec_kernel<1><<<grid, 256, 0, s>>>(a, b, gain, mean, rstd, c, o, rows, d); break;
+      case 2: layernorm_bwd_dx_vec_kernel<2><<<grid, 256, 0, s>>>(a, b, gain, mean, rstd, c, o, rows, d); break;
+      case 3: layernorm_bwd_dx_vec_kernel<3><<<grid, 256, 0, s>>>(a, b, gain, mean, rstd, c, o, rows, d); break;
+      default: layernorm_bwd_dx_vec_kernel<4><<<grid, 256, 0, s>>>(a, b, gain, mean, rstd, c, o, rows, d); break;
+    }
+    return cudaGetLastError();
+  }
   if (bf16) layernorm_bwd_dx_kernel<bf16_t><<<cdiv(rows, 8), 256, 0, s>>>((const bf16_t*)dy, (const bf16_t*)x, gain, mean, rstd, (const bf16_t*)add, (bf16_t*)dx, rows, d);
   else layernorm_bwd_dx_kernel<float><<<cdiv(rows, 8), 256, 0, s>>>((const float*)dy, (const float*)x, gain, mean, rstd, (const float*)add, (float*)dx, rows, d);
   return cudaGetLastError();
