@@ -1465,9 +1465,48 @@ __global__ void __launch_bounds__(256) bce_head_dz_kernel(const float* __restric
   stf(dz + i, v);
 }
 
+// one 16-byte piece (8 bf16 / 4 floats of one row) per thread; d a multiple of the piece
+template <typename T>
+__global__ void __launch_bounds__(256) bce_head_dz_vec_kernel(const float* __restrict__ ds, const float* __restrict__ w,
+                                                              T* __restrict__ dz, int dact, const T* __restrict__ src,
+                                                              long long nvec, int dvec) {
+  constexpr int VEC = VecOf<T>::N;
+  const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (i >= nvec) return;
+  const long long row = i / dvec;
+  const int c = (int)(i - row * dvec) * VEC;
+  const float dsr = ds[row];
+  float v[VEC], u[VEC];
+  if (dact != ACT_NONE) ld_vec<T>(src + i * VEC, u);
+#pragma unroll
+  for (int j = 0; j < VEC; j++) {
+    v[j] = dsr * w[c + j];
+    if (dact != ACT_NONE) v[j] *= act_deriv(dact, u[j]);
+  }
+  if (VEC == 8) {
+    uint4 q;
+    __nv_bfloat162 h;
+    h = __floats2bfloat162_rn(v[0], v[1]); q.x = *reinterpret_cast<uint32_t*>(&h);
+    h = __floats2bfloat162_rn(v[2], v[3]); q.y = *reinterpret_cast<uint32_t*>(&h);
+    h = __floats2bfloat162_rn(v[4 % VEC], v[5 % VEC]); q.z = *reinterpret_cast<uint32_t*>(&h);
+    h = __floats2bfloat162_rn(v[6 % VEC], v[7 % VEC]); q.w = *reinterpret_cast<uint32_t*>(&h);
+    *reinterpret_cast<uint4*>(dz + i * VEC) = q;
+  } else {
+    *reinterpret_cast<float4*>(dz + i * VEC) = make_float4(v[0], v[1], v[2], v[3]);
+  }
+}
+
 cudaError_t bce_head_dz(const float* ds, const float* w, void* dz, int dact, const void* src, int rows,
                         int d, bool bf16, cudaStream_t s) {
   long long n = (long long)rows * d;
+  const int vec = bf16 ? 8 : 4;
+  const bool al = ((reinterpret_cast<uintptr_t>(dz) | reinterpret_cast<uintptr_t>(src)) & 15) == 0;
+  if (al && d % vec == 0) {
+    const long long nvec = n / vec;
+    if (bf16) bce_head_dz_vec_kernel<bf16_t><<<cdiv(nvec, 256), 256, 0, s>>>(ds, w, (bf16_t*)dz, dact, (const bf16_t*)src, nvec, d / vec);
+    else bce_head_dz_vec_kernel<float><<<cdiv(nvec, 256), 256, 0, s>>>(ds, w, (float*)dz, dact, (const float*)src, nvec, d / vec);
+    return cudaGetLastError();
+  }
   if (bf16) bce_head_dz_kernel<bf16_t><<<cdiv(n, 256), 256, 0, s>>>(ds, w, (bf16_t*)dz, dact, (const bf16_t*)src, n, d);
   else bce_head_dz_kernel<float><<<cdiv(n, 256), 256, 0, s>>>(ds, w, (float*)dz, dact, (const float*)src, n, d);
   return cudaGetLastError();
