@@ -364,7 +364,8 @@ struct Builder {
     int total = 0;
     for (ReduceJob& j : jobs) {
       int chunks = std::max(1, batch_ctas / std::max(1, all_strips));
-      chunks = std::max(chunks, (j.rows + 1023) / 1024);          // a CTA streams at most about 1024 rows
+      static const int rows_per_cta = getenv("ERASE_REDUCE_ROWS") ? atoi(getenv("ERASE_REDUCE_ROWS")) : 256;
+      chunks = std::max(chunks, (j.rows + rows_per_cta - 1) / rows_per_cta);   // a CTA streams at most about that many rows
       chunks = std::min(chunks, std::max(1, j.rows / 64));
       j.chunks = chunks;
       j.ws = chunks > 1 ? f32_buf((size_t)(j.kind == 1 ? 2 : 1) * chunks * j.cols) : nullptr;
