@@ -80,6 +80,11 @@ def time_oracle(spec, steps, warmup):
     return units_per_step(spec) * steps / dt, 1e3 * dt / steps
 
 
+def metric_name(spec):
+    """One name for both arms: the reference arm times the oracle's step of the same workload."""
+    return f"train {unit_name(spec)}, ERASE early-backward schedule (vs serial schedule of the same kernels)"
+
+
 def run_reference(args, spec, cfg_name):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -89,7 +94,8 @@ def run_reference(args, spec, cfg_name):
     val, ms = time_oracle(spec, steps, warm)
     cores = oracle_threads()
     sample = f"{steps} full oracle step(s) of the workload's batch ({units_per_step(spec)} {unit_name(spec).split('/')[0]}) after {warm} warm-up"
-    line = {"impl": "reference", "metric": f"train {unit_name(spec)} (oracle on host cores)", "value": val,
+    line = {"impl": "reference", "metric": metric_name(spec), "value": val,
+            "note": "the CPU oracle's step of the same workload (its results do not depend on the schedule)",
             "unit": unit_name(spec), "n_gpus": args.gpus, "steps": steps, "warmup": warm, "ms_per_step": ms,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
             "data": "synthetic", "config": {"workload": workload_name(cfg_name, spec)},
@@ -329,7 +335,7 @@ def run_gpu(args, spec, cfg_name):
     qps = lambda per: units / (per * 1e-3)
     arena_mb = binding.arena_bytes(spec) / 2 ** 20
     line = {
-        "metric": f"train {unit_name(spec)}, ERASE early-backward schedule (vs serial schedule of the same kernels)",
+        "metric": metric_name(spec),
         "value": value, "unit": unit_name(spec), "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": era_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": spec["dtype"], "data": "synthetic",
