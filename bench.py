@@ -11,6 +11,7 @@ workload on its own GPU (the path has no exchange step on one node: "replicas on
 is the units all ranks processed divided by the slowest rank's time.
 """
 import argparse
+import atexit
 import json
 import os
 import subprocess
@@ -120,18 +121,25 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
+            atexit.register(self._kill)     # never leave the tool running if the bench dies early
         except Exception:
             self.proc = None
 
+    def _kill(self):
+        if self.proc and self.proc.poll() is None:
+            self.proc.kill()
+
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
 
-    def stop(self):
+    def stop(self, window=None):
+        """Summary of the samples that arrived inside `window` = (t0, t1) of time.time(); the tool
+        needs a moment to start, so it is started well before the timed legs and filtered here."""
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
         self.proc.terminate()
@@ -139,12 +147,16 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm = [float(r[0]) for r in self.rows if len(r) >= 7 and r[0].replace(".", "").isdigit()]
-        mx = [float(r[1]) for r in self.rows if len(r) >= 7 and r[1].replace(".", "").isdigit()]
+        rows = [r for t, r in self.rows if len(r) >= 7 and (window is None or window[0] <= t <= window[1] + 0.1)]
+        scope = "timed legs"
+        if not rows:
+            rows, scope = [r for _, r in self.rows if len(r) >= 7], "whole run (no sample fell into the timed legs)"
+        sm = [float(r[0]) for r in rows if r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in rows if r[1].replace(".", "").isdigit()]
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = [n for i, n in enumerate(names) if any(len(r) >= 7 and r[3 + i] == "Active" for r in self.rows)]
+        reasons = [n for i, n in enumerate(names) if any(r[3 + i] == "Active" for r in rows)]
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": reasons, "samples": len(sm)}
+                "reasons": reasons, "samples": len(sm), "scope": scope}
 
 
 # ------------------------------------------------------------------------------------------------
@@ -191,6 +203,8 @@ def run_gpu(args, spec, cfg_name):
         eflags |= binding.PAR_FWD
     units = units_per_step(spec)
 
+    sampler = ClockSampler(local)
+    sampler.start()
     model = binding.Model(spec)
     model.set_all(synth.init_params(spec, 0))
 
@@ -242,16 +256,16 @@ def run_gpu(args, spec, cfg_name):
             if os.environ.get("BENCH_PROGRESS"):
                 print(f"[bench] {what}", file=sys.stderr, flush=True)
 
-        sampler = ClockSampler(local)
-        # serial first (context), then the ERASE schedule under the clock sampler
+        # serial first (context), then the ERASE schedule; the clock sampler (started before the
+        # model was built) is read over the three timed legs
         progress("serial leg")
+        t_legs = time.time()
         ser_ms, ser_per, _ = timed(1, flags, args.steps, args.warmup)
-        sampler.start()
         progress("ERASE leg")
         era_ms, era_per, launches = timed(n_streams, eflags, args.steps, args.warmup)
         progress("ERASE leg, loss on the main stream")
         pap_ms, pap_per, _ = timed(n_streams, flags, args.steps, args.warmup) if eflags != flags else (era_ms, era_per, 0)
-        clocks = sampler.stop()
+        clocks = sampler.stop((t_legs, time.time()))
         progress("end-to-end leg")
 
         # end to end through the C ABI: pinned host batch -> device copy, step, losses back to host
