@@ -2,17 +2,22 @@
 """Benchmark of the ERASE training step on B200: tokens/s (samples/s) of the early-backward
 schedule against the serial schedule of the same kernels, on synthetic data.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--config C2] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config C4] [--impl reference] [--no-table]
 
 One JSON line on stdout (rank 0).  A "step" is one pass of the whole hot path over one batch:
 input staging, every block's forward + local loss, every block's backward, the optimizer.
+The headline workload (`value`) is C4, the largest single-GPU configuration; the same line
+carries, under `per_config`, the serial and ERASE throughput, gain, MFU and dominant kernel class
+of C1, C2, C3 and five points of the C5 saturation sweep (N = 1 only).
 With N > 1 (launched by torch.distributed.run) every rank runs an independent replica of the
 workload on its own GPU (the path has no exchange step on one node: "replicas only"); the value
 is the units all ranks processed divided by the slowest rank's time.
 """
 import argparse
 import atexit
+import gc
 import json
+import math
 import os
 import subprocess
 import sys
@@ -26,12 +31,21 @@ sys.path.insert(0, ROOT)
 
 from paper_2608_18469_b200 import synth  # noqa: E402
 
-POOL = 8   # distinct pre-staged batches, cycled
+POOL = 8            # distinct pre-staged batches, cycled
+MIN_LEG_S = 1.0     # every leg is repeated (K steps per repeat) until this much device time is timed
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from ncu captures of the largest member
-# of each kernel class at C2 (the local head's GEMMs; profiles/tc_gemm_c2_head_fwd_dgrad_wgrad.md).
-# They sit below the algorithmic bytes where a 64 MiB operand or result is still L2-resident.
+# of each kernel class (summaries under profiles/).  They sit below the algorithmic bytes where an
+# operand or result is still L2-resident.
 NCU_DRAM_BYTES = {"C2": {"gemm_fwd": 15.5e6, "gemm_dgrad": 75.4e6, "gemm_wgrad": 71.4e6}}
+
+# the per-config table of the default run: (label, config name, keyword arguments)
+TABLE = [("C1", "C1", {}), ("C2", "C2", {}), ("C3", "C3", {}),
+         ("C5 w128 b512", "C5", {"w": 128, "batch": 512}),
+         ("C5 w512 b4096", "C5", {"w": 512, "batch": 4096}),
+         ("C5 w1024 b32768", "C5", {"w": 1024, "batch": 32768}),
+         ("C5 w2048 b4096", "C5", {"w": 2048, "batch": 4096}),
+         ("C5 w4096 b4096", "C5", {"w": 4096, "batch": 4096})]
 
 
 def unit_name(spec):
@@ -43,9 +57,14 @@ def units_per_step(spec):
 
 
 def workload_name(name, spec):
-    if name == "C2":
-        return "C2 small LM proxy: 4 detached pre-LN transformer blocks d256 h4 ff1024 T256 batch16 vocab8192, CE heads, AdamW"
-    return f"{name}: {len(spec['blocks'])} detached blocks, batch {spec['batch']}"
+    nb = len(spec["blocks"])
+    if spec["input"] == "tokens":
+        blk = spec["blocks"][0]
+        return (f"{name} LM proxy: {nb} detached pre-LN transformer blocks d{blk['dims'][0]} h{blk['n_heads']} "
+                f"ff{blk['dims'][1]} T{spec['seq']} batch{spec['batch']} vocab{spec['vocab']}, local CE heads, AdamW, bf16")
+    if spec["input"] == "ctr":
+        return f"{name} CTR ranking model: {nb} parallel detached dense subarchitectures, batch {spec['batch']}, local BCE heads, Adam, bf16"
+    return f"{name}: {nb} detached MLP blocks w{spec['width']}, batch {spec['batch']}, local BCE heads, SGD, {spec['dtype']}"
 
 
 # ------------------------------------------------------------------------------------------------
@@ -63,8 +82,28 @@ def oracle_threads():
     return os.cpu_count() or 1
 
 
+def oracle_sample(cfg_name, spec):
+    """A bounded sample of the workload for the oracle (about 10-30 s of CPU work per step) and the
+    factor that scales its rate to the whole workload.  Small configs: the full batch, every block.
+    C4 and the large sweep points: ONE block of the model (on part of the batch where even that is
+    above 2 TFLOP); the blocks all have the same shapes and the oracle's cost is linear in blocks and
+    rows, so the full step costs n_blocks x (that block at full batch)."""
+    nb = len(spec["blocks"])
+    if synth.step_flops(spec) < 2e12:
+        return spec, 1.0, "the full batch through every block"
+    s = dict(spec)
+    s["blocks"] = [dict(spec["blocks"][0])]
+    frac = 1
+    while frac < 8 and synth.step_flops(s) / frac > 2e12 and spec["batch"] % (2 * frac) == 0:
+        frac *= 2
+    s["batch"] = spec["batch"] // frac
+    return s, 1.0 / nb, (f"1 of the {nb} blocks on {s['batch']} of the {spec['batch']} "
+                         f"{'sequences' if spec['input'] == 'tokens' else 'samples'}: extrapolated from 1 of {nb} blocks "
+                         f"(rate scaled by 1/{nb})")
+
+
 def time_oracle(spec, steps, warmup):
-    """Times oracle steps (each on one full batch of the workload).  Returns (units/s, ms/step)."""
+    """Times oracle steps on `spec`.  Returns (units/s of this spec, ms/step)."""
     from oracle import erase_oracle as orc
     flat = synth.init_params(spec, 0)
     params = {"input": {}, "blocks": [dict() for _ in spec["blocks"]]}
@@ -92,12 +131,15 @@ def run_reference(args, spec, cfg_name):
         return
     steps = max(1, min(args.steps, 3))
     warm = 1 if args.warmup > 0 else 0
-    val, ms = time_oracle(spec, steps, warm)
+    sub, scale, what = oracle_sample(cfg_name, spec)
+    val, ms = time_oracle(sub, steps, warm)
+    val *= scale
     cores = oracle_threads()
-    sample = f"{steps} full oracle step(s) of the workload's batch ({units_per_step(spec)} {unit_name(spec).split('/')[0]}) after {warm} warm-up"
+    sample = f"{steps} oracle step(s) after {warm} warm-up, each on {what}; {ms:.0f} ms per sampled step"
     line = {"impl": "reference", "metric": metric_name(spec), "value": val,
             "note": "the CPU oracle's step of the same workload (its results do not depend on the schedule)",
-            "unit": unit_name(spec), "n_gpus": args.gpus, "steps": steps, "warmup": warm, "ms_per_step": ms,
+            "unit": unit_name(spec), "n_gpus": args.gpus, "steps": steps, "warmup": warm,
+            "ms_per_step": 1e3 * units_per_step(spec) / val,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
             "data": "synthetic", "config": {"workload": workload_name(cfg_name, spec)},
             "cpu_baseline": {"value": val, "unit": unit_name(spec), "cores": cores, "kind": "oracle",
@@ -137,26 +179,30 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
 
-    def stop(self, window=None):
+    def summary(self, window=None):
         """Summary of the samples that arrived inside `window` = (t0, t1) of time.time(); the tool
         needs a moment to start, so it is started well before the timed legs and filtered here."""
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        rows = [r for t, r in self.rows if len(r) >= 7 and (window is None or window[0] <= t <= window[1] + 0.1)]
-        scope = "timed legs"
+        rows = [r for t, r in list(self.rows) if len(r) >= 7 and (window is None or window[0] <= t <= window[1] + 0.1)]
+        scope = "timed legs of the headline workload"
         if not rows:
-            rows, scope = [r for _, r in self.rows if len(r) >= 7], "whole run (no sample fell into the timed legs)"
+            rows, scope = [r for _, r in list(self.rows) if len(r) >= 7], "whole run (no sample fell into the timed legs)"
         sm = [float(r[0]) for r in rows if r[0].replace(".", "").isdigit()]
         mx = [float(r[1]) for r in rows if r[1].replace(".", "").isdigit()]
+        pw = [float(r[2]) for r in rows if r[2].replace(".", "").isdigit()]
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         reasons = [n for i, n in enumerate(names) if any(r[3 + i] == "Active" for r in rows)]
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": reasons, "samples": len(sm), "scope": scope}
+                "power_w_max": max(pw) if pw else None, "reasons": reasons, "samples": len(sm), "scope": scope}
+
+    def stop(self):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
 
 
 # ------------------------------------------------------------------------------------------------
@@ -172,22 +218,13 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "tflops": 1400.0, "tflops_burst": 1590.0, "source": "fallback"}
 
 
-def run_gpu(args, spec, cfg_name):
-    import torch
-    from paper_2608_18469_b200 import binding
+def progress(what):   # BENCH_PROGRESS=1: which leg is running, on stderr
+    if os.environ.get("BENCH_PROGRESS"):
+        print(f"[bench {time.strftime('%H:%M:%S')}] {what}", file=sys.stderr, flush=True)
 
-    from paper_2608_18469_b200.replicas import Replicas
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    rep = Replicas(backend="nccl", device="cuda")
-    rank, world, dist = rep.rank, rep.world, rep.dist
 
-    def barrier():
-        rep.barrier()
-        torch.cuda.synchronize()
-
-    max_over_ranks = rep.max_over_ranks
-
+def schedule_flags(binding, spec, args):
+    """(n_streams, graph flags of the serial leg, flags of the ERASE leg, description)."""
     nb = len(spec["blocks"])
     n_streams = args.n_streams if args.n_streams > 0 else nb + 1
     flags = 0 if args.no_graph else binding.GRAPH
@@ -201,20 +238,23 @@ def run_gpu(args, spec, cfg_name):
     par_fwd = not args.loss_on_main and not args.no_par_fwd and spec["topo"] == "parallel"
     if par_fwd:
         eflags |= binding.PAR_FWD
-    units = units_per_step(spec)
+    desc = ("ERASE, local head+loss+backward+optimizer of each block released onto side streams after the block body"
+            + (", parameter-gradient work of each backward on a second stream per block" if split_bwd else "")
+            + (", every block's forward on its own side stream too (parallel topology)" if par_fwd else "")
+            ) if not args.loss_on_main else "ERASE, backward released after forward and local loss"
+    return n_streams, flags, eflags, desc
 
-    sampler = ClockSampler(local)
-    sampler.start()
-    model = binding.Model(spec)
-    model.set_all(synth.init_params(spec, 0))
 
-    def measure():
-        """Everything that owns torch tensors, events or streams lives in this scope, so that it
-        is released before the model (and its CUDA streams) is destroyed."""
-        main = torch.cuda.ExternalStream(model.main_stream())
+class Workload:
+    """One model with its pool of resident batches; everything that owns torch tensors, events or
+    streams is dropped by close() before the model (and its CUDA streams) is destroyed."""
 
-        # pool of batches resident in HBM, and their pinned host copies for the end-to-end leg
-        host, dev = [], []
+    def __init__(self, torch, binding, spec, rep):
+        self.torch, self.spec, self.rep = torch, spec, rep
+        self.model = binding.Model(spec)
+        self.model.set_all(synth.init_params(spec, 0))
+        self.main = torch.cuda.ExternalStream(self.model.main_stream())
+        self.host, self.dev = [], []
         for i in range(POOL):
             b = synth.make_batch(spec, 0, index=i)
             h = {}
@@ -227,122 +267,217 @@ def run_gpu(args, spec, cfg_name):
             else:
                 h["x"], h["ids"], h["y"] = (torch.from_numpy(b[k]) for k in ("dense", "ids", "y"))
             h = {k: v.contiguous().pin_memory() for k, v in h.items()}
-            host.append(h)
-            dev.append({k: v.cuda() for k, v in h.items()})
+            self.host.append(h)
+            self.dev.append({k: v.cuda() for k, v in h.items()})
         torch.cuda.synchronize()
 
-        def ptrs(d):
-            return {k: d[k].data_ptr() if k in d else None for k in ("x", "ids", "y")}
+    @staticmethod
+    def ptrs(d):
+        return {k: d[k].data_ptr() if k in d else None for k in ("x", "ids", "y")}
 
-        def timed(ns, fl, steps, warmup):
-            """K steps on resident inputs, per-step CUDA events on the launching stream."""
-            for i in range(warmup):
-                model.step(n_streams=ns, flags=fl, **ptrs(dev[i % POOL]))
-            model.sync()
-            evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    def barrier(self):
+        self.rep.barrier()
+        self.torch.cuda.synchronize()
+
+    def warm(self, ns, fl, n):
+        for i in range(n):
+            self.model.step(n_streams=ns, flags=fl, **self.ptrs(self.dev[i % POOL]))
+        self.model.sync()
+
+    def leg(self, ns, fl, steps, warmup, per_step=True, min_s=MIN_LEG_S, max_repeats=200):
+        """Repeats of exactly `steps` steps on resident inputs, each bracketed by a barrier and a
+        synchronize, timed with CUDA events on the launching stream (max over ranks), until at least
+        `min_s` seconds of device time have been timed.  Returns the list of repeat times (ms), the
+        per-step times of the median repeat and the launches of one repeat."""
+        torch, model = self.torch, self.model
+        self.warm(ns, fl, warmup)
+        reps, pers, launches, total = [], [], 0, 0.0
+        k = 0
+        while total < min_s * 1e3 and len(reps) < max_repeats:
+            n_ev = steps + 1 if per_step else 2
+            evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_ev)]
             l0 = model.launch_count()
-            barrier()
-            evs[0].record(main)
+            self.barrier()
+            evs[0].record(self.main)
             for i in range(steps):
-                model.step(n_streams=ns, flags=fl, **ptrs(dev[(warmup + i) % POOL]))
-                evs[i + 1].record(main)
+                model.step(n_streams=ns, flags=fl, **self.ptrs(self.dev[(warmup + k + i) % POOL]))
+                if per_step:
+                    evs[i + 1].record(self.main)
+            if not per_step:
+                evs[1].record(self.main)
             model.sync()
-            barrier()
-            total_ms = evs[0].elapsed_time(evs[-1])
-            per = np.array([evs[i].elapsed_time(evs[i + 1]) for i in range(steps)])
-            return max_over_ranks(total_ms), per, model.launch_count() - l0
+            self.barrier()
+            ms = self.rep.max_over_ranks(evs[0].elapsed_time(evs[-1]))
+            reps.append(ms)
+            pers.append(np.array([evs[i].elapsed_time(evs[i + 1]) for i in range(steps)]) if per_step else None)
+            launches = model.launch_count() - l0
+            total += ms
+            k += steps
+        med = int(np.argsort(reps)[len(reps) // 2])
+        return {"ms": reps[med], "repeats": reps, "per_step": pers[med], "launches": launches}
 
-        def progress(what):   # BENCH_PROGRESS=1: which leg is running, on stderr
-            if os.environ.get("BENCH_PROGRESS"):
-                print(f"[bench] {what}", file=sys.stderr, flush=True)
-
-        # serial first (context), then the ERASE schedule; the clock sampler (started before the
-        # model was built) is read over the three timed legs
-        progress("serial leg")
-        t_legs = time.time()
-        ser_ms, ser_per, _ = timed(1, flags, args.steps, args.warmup)
-        progress("ERASE leg")
-        era_ms, era_per, launches = timed(n_streams, eflags, args.steps, args.warmup)
-        progress("ERASE leg, loss on the main stream")
-        pap_ms, pap_per, _ = timed(n_streams, flags, args.steps, args.warmup) if eflags != flags else (era_ms, era_per, 0)
-        clocks = sampler.stop((t_legs, time.time()))
-        progress("end-to-end leg")
-
-        # end to end through the C ABI: pinned host batch -> device copy, step, losses back to host
-        stage = {k: torch.empty_like(v) for k, v in dev[0].items()}
-        h2d = sum(v.numel() * v.element_size() for v in stage.values())
-        d2h = nb * 4
-
-        def e2e_step(i):
-            with torch.cuda.stream(main):
-                for k in stage:
-                    stage[k].copy_(host[i % POOL][k], non_blocking=True)
-            model.step(n_streams=n_streams, flags=eflags, **ptrs(stage))
-            return model.losses()
-
-        for i in range(args.warmup):
-            e2e_step(i)
-        barrier()
-        t0 = time.perf_counter()
-        for i in range(args.steps):
-            e2e_step(args.warmup + i)
-        model.sync()
-        barrier()
-        e2e_ms = max_over_ranks(1e3 * (time.perf_counter() - t0))
-
-        # per-kernel attribution: profiled serial steps (events around every operation)
-        progress("profiled steps")
+    def kernel_classes(self, nprof=3):
+        """Per-kernel-class attribution from profiled serial steps (CUDA events around every operation)."""
         agg = {}
-        nprof = 3
         for i in range(nprof + 1):
-            recs = model.profile_step(**ptrs(dev[i % POOL]))
+            recs = self.model.profile_step(**self.ptrs(self.dev[i % POOL]))
             if i == 0:
                 continue    # warm-up of the profiling path
             for r in recs:
                 a = agg.setdefault(r["name"], {"ms": 0.0, "flops": 0.0, "bytes": 0.0, "runs": 0, "launches": 0})
                 a["ms"] += r["ms"]; a["flops"] += r["flops"]; a["bytes"] += r["bytes"]
                 a["runs"] += 1; a["launches"] += r["launches"]
-        top = max(agg, key=lambda k: agg[k]["ms"])
-        peaks = measured_peaks()
-        t = agg[top]
-        if top.startswith("gemm") or top.startswith("attention"):
-            ach = t["flops"] / (t["ms"] * 1e-3) / 1e12
-            roof = {"kernel": top, "bound": "tensor", "achieved": ach, "peak": peaks["tflops"], "unit": "TFLOP/s",
-                    "frac": ach / peaks["tflops"]}
-        else:
-            ach = t["bytes"] / (t["ms"] * 1e-3) / 1e9
-            roof = {"kernel": top, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": ach / peaks["hbm_gbs"]}
-        roof["peak_source"] = peaks["source"] + (" (sustained bf16 GEMM)" if roof["bound"] == "tensor" else " (copy)")
-        roof["avg_launch_ms"] = t["ms"] / max(t["launches"], 1)
-        tr = NCU_DRAM_BYTES.get(cfg_name, {}).get(top)
-        roof["traffic"] = tr
-        roof["traffic_note"] = "ncu DRAM bytes of the class's largest GEMM (local head), one launch" if tr else None
-        roof["kernel_share"] = {k: round(v["ms"] / sum(x["ms"] for x in agg.values()), 4)
-                                for k, v in sorted(agg.items(), key=lambda kv: -kv[1]["ms"])[:8]}
+        return agg
 
-        cpu = None
-        if rank == 0 and world == 1 and not args.no_cpu_baseline:
-            val, ms = time_oracle(spec, 1, 1)
-            cpu = {"value": val, "unit": unit_name(spec), "cores": oracle_threads(), "kind": "oracle",
-                   "sample": f"1 full oracle step of the workload's batch ({units} units) after 1 warm-up step; {ms:.0f} ms"}
+    def close(self):
+        self.host = self.dev = self.main = None
+        gc.collect()
+        self.torch.cuda.synchronize()
+        self.model.close()
+        self.torch.cuda.empty_cache()
 
 
-        return dict(pap_ms=pap_ms, ser_ms=ser_ms, ser_per=ser_per, era_ms=era_ms, era_per=era_per, launches=launches,
-                    clocks=clocks, e2e_ms=e2e_ms, h2d=h2d, d2h=d2h, roof=roof, cpu=cpu)
+def roofline_of(agg, peaks, cfg_name):
+    top = max(agg, key=lambda k: agg[k]["ms"])
+    t = agg[top]
+    if top.startswith("gemm") or top.startswith("attention"):
+        ach = t["flops"] / (t["ms"] * 1e-3) / 1e12
+        roof = {"kernel": top, "bound": "tensor", "achieved": ach, "peak": peaks["tflops"], "unit": "TFLOP/s",
+                "frac": ach / peaks["tflops"]}
+    else:
+        ach = t["bytes"] / (t["ms"] * 1e-3) / 1e9
+        roof = {"kernel": top, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": ach / peaks["hbm_gbs"]}
+    roof["peak_source"] = peaks["source"] + (" (sustained bf16 GEMM)" if roof["bound"] == "tensor" else " (copy)")
+    roof["avg_launch_ms"] = t["ms"] / max(t["launches"], 1)
+    tr = NCU_DRAM_BYTES.get(cfg_name, {}).get(top)
+    roof["traffic"] = tr
+    roof["traffic_note"] = NCU_DRAM_NOTE.get(cfg_name) if tr else None
+    tot = sum(x["ms"] for x in agg.values())
+    roof["kernel_share"] = {k: round(v["ms"] / tot, 4) for k, v in sorted(agg.items(), key=lambda kv: -kv[1]["ms"])[:8]}
+    return roof
 
-    import gc
+
+NCU_DRAM_NOTE = {"C2": "ncu DRAM bytes of the class's largest GEMM (local head), one launch"}
+
+
+def table_entry(torch, binding, rep, label, cfg, kw, args, peaks):
+    """Serial and ERASE throughput, gain, MFU and dominant kernel class of one parity-table config."""
+    spec = synth.config(cfg, **kw)
+    progress(f"table: {label}")
+    w = Workload(torch, binding, spec, rep)
+    try:
+        ns, flags, eflags, _ = schedule_flags(binding, spec, args)
+        units = units_per_step(spec)
+        # size one repeat to about a quarter of a second from a short trial run
+        w.warm(1, flags, POOL)
+        t0 = time.perf_counter()
+        w.warm(1, flags, 8)
+        est = max((time.perf_counter() - t0) / 8, 1e-5)
+        steps = int(min(4000, max(8, math.ceil(0.25 / est))))
+        ser = w.leg(1, flags, steps, POOL, per_step=False)
+        era = w.leg(ns, eflags, steps, POOL, per_step=False)
+        pap = w.leg(ns, flags, steps, POOL, per_step=False, min_s=0.3) if eflags != flags else era
+        agg = w.kernel_classes(2)
+        roof = roofline_of(agg, peaks, None)
+        flops = synth.step_flops(spec)
+        ms_e, ms_s = era["ms"] / steps, ser["ms"] / steps
+        return {"config": label, "unit": unit_name(spec), "serial": units / (ms_s * 1e-3), "erase": units / (ms_e * 1e-3),
+                "ms_per_step_serial": ms_s, "ms_per_step_erase": ms_e, "gain_pct": 100.0 * (ms_s / ms_e - 1.0),
+                "gain_pct_loss_on_main_stream": 100.0 * (ser["ms"] / pap["ms"] - 1.0),
+                "steps_per_repeat": steps, "repeats": [len(ser["repeats"]), len(era["repeats"])],
+                "mfu_vs_measured_sustained": flops / (ms_e * 1e-3) / (peaks["tflops"] * 1e12),
+                "top_class": roof["kernel"], "top_class_bound": roof["bound"], "top_class_frac": roof["frac"],
+                "top_class_share": roof["kernel_share"].get(roof["kernel"]), "dtype": spec["dtype"]}
+    finally:
+        w.close()
+
+
+def run_gpu(args, spec, cfg_name):
+    import torch
+    from paper_2608_18469_b200 import binding
+    from paper_2608_18469_b200.replicas import Replicas
+
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    rep = Replicas(backend="nccl", device="cuda")
+    rank, world, dist = rep.rank, rep.world, rep.dist
     peaks = measured_peaks()
-    r = measure()
-    gc.collect()
-    torch.cuda.synchronize()
-    model.close()
-    ser_ms, ser_per, era_ms, era_per, launches = r["ser_ms"], r["ser_per"], r["era_ms"], r["era_per"], r["launches"]
-    clocks, e2e_ms, h2d, d2h, roof, cpu = r["clocks"], r["e2e_ms"], r["h2d"], r["d2h"], r["roof"], r["cpu"]
+    nb = len(spec["blocks"])
+    n_streams, flags, eflags, sched_desc = schedule_flags(binding, spec, args)
+    units = units_per_step(spec)
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    w = Workload(torch, binding, spec, rep)
+    model = w.model
+
+    # serial first (context), then the ERASE schedule; the clock sampler (started before the model
+    # was built) is read over the three timed legs
+    progress("serial leg")
+    t_legs = time.time()
+    ser = w.leg(1, flags, args.steps, args.warmup)
+    progress("ERASE leg")
+    era = w.leg(n_streams, eflags, args.steps, args.warmup)
+    progress("ERASE leg, loss on the main stream")
+    pap = w.leg(n_streams, flags, args.steps, args.warmup) if eflags != flags else era
+    clocks = sampler.summary((t_legs, time.time()))
+
+    # end to end through the C ABI: pinned host batch -> device copy, step, losses back to host
+    progress("end-to-end leg")
+    stage = {k: torch.empty_like(v) for k, v in w.dev[0].items()}
+    h2d = sum(v.numel() * v.element_size() for v in stage.values())
+    d2h = nb * 4
+
+    def e2e_step(i):
+        with torch.cuda.stream(w.main):
+            for k in stage:
+                stage[k].copy_(w.host[i % POOL][k], non_blocking=True)
+        model.step(n_streams=n_streams, flags=eflags, **w.ptrs(stage))
+        return model.losses()
+
+    for i in range(args.warmup):
+        e2e_step(i)
+    e2e_reps, tot = [], 0.0
+    while tot < MIN_LEG_S * 1e3 and len(e2e_reps) < 200:
+        w.barrier()
+        t0 = time.perf_counter()
+        for i in range(args.steps):
+            e2e_step(args.warmup + i)
+        model.sync()
+        w.barrier()
+        e2e_reps.append(rep.max_over_ranks(1e3 * (time.perf_counter() - t0)))
+        tot += e2e_reps[-1]
+    e2e_ms = float(np.median(e2e_reps))
+
+    progress("profiled steps")
+    roof = roofline_of(w.kernel_classes(3), peaks, cfg_name)
+    stage = None
+    w.close()
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        progress("cpu baseline (oracle)")
+        sub, scale, what = oracle_sample(cfg_name, spec)
+        val, ms = time_oracle(sub, 1, 0)
+        cpu = {"value": val * scale, "unit": unit_name(spec), "cores": oracle_threads(), "kind": "oracle",
+               "sample": f"1 oracle step on {what}; {ms / 1e3:.1f} s"}
+
+    table = None
+    if world == 1 and not args.no_table:
+        table = []
+        for label, cfg, kw in TABLE:
+            try:
+                table.append(table_entry(torch, binding, rep, label, cfg, kw, args, peaks))
+            except Exception as e:      # one config failing must not lose the headline line
+                table.append({"config": label, "error": f"{type(e).__name__}: {e}"[:200]})
+    sampler.stop()
     if rank != 0:
         if dist is not None:
             rep.close()
         return
+
+    ser_ms, era_ms, ser_per, era_per = ser["ms"], era["ms"], ser["per_step"], era["per_step"]
     flops = synth.step_flops(spec)
     value = world * units * args.steps / (era_ms * 1e-3)
     serial_value = world * units * args.steps / (ser_ms * 1e-3)
@@ -353,20 +488,18 @@ def run_gpu(args, spec, cfg_name):
         "value": value, "unit": unit_name(spec), "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": era_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": spec["dtype"], "data": "synthetic",
-        "config": {"workload": workload_name(cfg_name, spec), "n_streams": n_streams,
-                   "schedule": ("ERASE, local head+loss+backward+optimizer of each block released onto side streams after the block body"
-                                + (", parameter-gradient work of each backward on a second stream per block" if split_bwd else "")
-                                + (", every block's forward on its own side stream too (parallel topology)" if par_fwd else ""))
-                               if not args.loss_on_main else "ERASE, backward released after forward and local loss",
+        "config": {"workload": workload_name(cfg_name, spec), "n_streams": n_streams, "schedule": sched_desc,
                    "cuda_graph": not args.no_graph, "batch_pool": POOL,
+                   "repeats": f"each leg = repeats of exactly {args.steps} steps until >= {MIN_LEG_S} s are timed; the median repeat is reported",
                    "l2": f"no flush: the step's working set ({arena_mb:.0f} MiB of stashes, logits, parameters) exceeds the 126 MB L2",
                    "multi_gpu": "replicas only" if world > 1 else "single GPU"},
-        "serial": {"value": serial_value, "ms_per_step": ser_ms / args.steps,
+        "serial": {"value": serial_value, "ms_per_step": ser_ms / args.steps, "repeats_ms": [round(x, 3) for x in ser["repeats"]],
                    "p90": float(np.percentile(qps(ser_per), 90)), "median": float(np.median(qps(ser_per)))},
-        "erase": {"p90": float(np.percentile(qps(era_per), 90)), "median": float(np.median(qps(era_per)))},
+        "erase": {"p90": float(np.percentile(qps(era_per), 90)), "median": float(np.median(qps(era_per))),
+                  "repeats_ms": [round(x, 3) for x in era["repeats"]]},
         "gain_pct": 100.0 * (value / serial_value - 1.0),
-        "erase_loss_on_main_stream": {"value": world * units * args.steps / (r["pap_ms"] * 1e-3),
-                                      "gain_pct": 100.0 * (ser_ms / r["pap_ms"] - 1.0),
+        "erase_loss_on_main_stream": {"value": world * units * args.steps / (pap["ms"] * 1e-3),
+                                      "gain_pct": 100.0 * (ser_ms / pap["ms"] - 1.0),
                                       "note": "the paper's placement: local head and loss run on the main stream before the backward is released"},
         "flops_per_step": flops,
         "mfu": {"vs_measured_sustained": flops * args.steps / (era_ms * 1e-3) / (peaks["tflops"] * 1e12),
@@ -374,9 +507,10 @@ def run_gpu(args, spec, cfg_name):
         "clocks": clocks,
         "e2e": {"value": world * units * args.steps / (e2e_ms * 1e-3), "unit": unit_name(spec),
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": int(launches),
+        "gpu_launches": int(era["launches"]),
         "roofline": roof,
         "cpu_baseline": cpu,
+        "per_config": table,
     }
     print(json.dumps(line), flush=True)
     if dist is not None:
@@ -386,16 +520,17 @@ def run_gpu(args, spec, cfg_name):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="C2")
+    ap.add_argument("--config", default="C4")
     ap.add_argument("--w", type=int, default=1024)
     ap.add_argument("--batch", type=int, default=4096)
     ap.add_argument("--n-streams", type=int, default=0, help="0 = n_blocks + 1")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--loss-on-main", action="store_true", help="paper's placement of the local loss")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-table", action="store_true", help="skip the per-config table (C1, C2, C3, five C5 points)")
     ap.add_argument("--no-par-fwd", action="store_true",
                     help="parallel topology: keep the blocks' forwards on the main stream, one after the other")
     ap.add_argument("--no-split-bwd", action="store_true",

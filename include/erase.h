@@ -43,7 +43,9 @@ typedef struct erase_model erase_model; /* opaque; owned by the library */
 
 typedef enum {
   ERASE_OK = 0,
-  ERASE_EINVAL = 1,       /* bad argument or spec; nothing was launched                     */
+  ERASE_EINVAL = 1,       /* bad argument or spec; nothing was launched.  Also returned by the
+                             first synchronising call after a step whose batch held an id outside
+                             its table: the id was not dereferenced, the step's results are void */
   ERASE_ENOMEM = 2,       /* device or host allocation failed, or the caller's arena is small */
   ERASE_ECUDA = 3,        /* a CUDA call failed; text in erase_last_error()                  */
   ERASE_ESTATE = 4,       /* call not valid in this state (e.g. step before parameters set)  */
@@ -217,6 +219,18 @@ ERASE_API erase_status erase_losses(erase_model* m, float* dst, int32_t n_blocks
 
 /* Waits until everything enqueued on the model has finished. */
 ERASE_API erase_status erase_sync(erase_model* m);
+
+/* Checks the library's time-out path without any real failure: enqueues, on the model's main
+ * stream, ONE thread that waits on a barrier nothing will ever signal -- with the same bounded
+ * wait the GEMM kernels use, limited to about limit_us microseconds (1..100000) -- then records
+ * the expiry in the model's status word and returns.  Nothing hangs and nothing faults: the wait
+ * is bounded by the SM clock.  The next erase_sync / erase_losses / erase_params returns
+ * ERASE_ETIMEOUT and clears the word; tensor-core kernels enqueued in between find the word set and
+ * skip their work, so a step behind an expired wait costs one limit, not one per kernel.  The
+ * model stays usable afterwards.  (Section 2.2 synchronises with streams and events only; the
+ * barriers inside the tensor-core kernels are this library's own, hence this check.)
+ * Errors: EINVAL, ECUDA. */
+ERASE_API erase_status erase_selftest_timeout(erase_model* m, int32_t limit_us);
 
 /* The CUDA stream (cudaStream_t) that steps start and end on; valid until erase_destroy.  A
  * caller may record its own events on it to time steps. */

@@ -77,6 +77,7 @@ EXPORTS = {
     "erase_step_ex": (C.c_int, [C.c_void_p, C.POINTER(Batch), C.c_int32, C.c_uint32]),
     "erase_losses": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32]),
     "erase_sync": (C.c_int, [C.c_void_p]),
+    "erase_selftest_timeout": (C.c_int, [C.c_void_p, C.c_int32]),
     "erase_main_stream": (C.c_void_p, [C.c_void_p]),
     "erase_launch_count": (C.c_int64, [C.c_void_p]),
     "erase_timeline": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32]),
@@ -227,6 +228,9 @@ class Model:
 
     def sync(self):
         self._ck(lib().erase_sync(self.h))
+
+    def selftest_timeout(self, limit_us=1000):
+        self._ck(lib().erase_selftest_timeout(self.h, limit_us))
 
     def main_stream(self):
         return lib().erase_main_stream(self.h)

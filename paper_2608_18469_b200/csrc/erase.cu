@@ -916,14 +916,15 @@ struct Builder {
         const float* tok = m->frozen + m->tensors[0].off;
         const float* pos = m->frozen + m->tensors[1].off;
         int batch = s.batch, T_ = s.seq, d = s.width;
-        m->stage.push_back({[=](cudaStream_t st) { return gather_tokens(tok, pos, mm->cur.ids, buf, batch, T_, d, bf, st); }, 1});
+        const int vocab = s.vocab;
+        m->stage.push_back({[=](cudaStream_t st) { return gather_tokens(tok, pos, mm->cur.ids, buf, batch, T_, d, vocab, mm->status, bf, st); }, 1});
         note(m->stage, "gather_tokens", (double)m->rows * d, (double)m->rows * d * (4 + m->esz));
       } else {
         const float* tables = m->frozen;
         long long stride = s.n_sparse > 1 ? (long long)(m->tensors[1].off - m->tensors[0].off) : 0;
-        int batch = s.batch, ns = s.n_sparse, e_ = s.emb_dim, nd = s.n_dense, w0 = s.width;
+        int batch = s.batch, ns = s.n_sparse, e_ = s.emb_dim, nd = s.n_dense, w0 = s.width, trows = s.table_rows;
         m->stage.push_back({[=](cudaStream_t st) {
-                              return gather_ctr(tables, stride, mm->cur.ids, (const float*)mm->cur.x, buf, batch, ns, e_, nd, w0, bf, st);
+                              return gather_ctr(tables, stride, mm->cur.ids, (const float*)mm->cur.x, buf, batch, ns, e_, nd, w0, trows, mm->status, bf, st);
                             }, 1});
         note(m->stage, "gather_ctr", 0, (double)m->rows * w0 * (4 + m->esz));
       }
@@ -1226,6 +1227,8 @@ erase_status erase_sync(erase_model* m) {
     if (st != 0) {
       int zero = 0;
       CK(copy_sync(m, m->status, &zero, sizeof(int), cudaMemcpyHostToDevice));
+      if (st == STATUS_BAD_ID)
+        return m->fail(ERASE_EINVAL, "a token or sparse id of the batch lies outside its table; it was not used as an index, and the results of the step are void");
       return m->fail(ERASE_ETIMEOUT, "a bounded device-side wait expired (code " + std::to_string(st) + "); results of the step are void");
     }
   }
@@ -1410,6 +1413,14 @@ erase_status erase_losses(erase_model* m, float* dst, int32_t n_blocks) {
   return ERASE_OK;
 }
 
+erase_status erase_selftest_timeout(erase_model* m, int32_t limit_us) {
+  if (!m) return ERASE_EINVAL;
+  if (limit_us < 1 || limit_us > 100000) return m->fail(ERASE_EINVAL, "erase_selftest_timeout: limit_us must be in [1, 100000]");
+  CK(tc_wait_selftest(m->status, (long long)limit_us * 2000LL, m->main));   // SM clock <= 2 GHz: at least limit_us
+  m->launches++;
+  return ERASE_OK;
+}
+
 void* erase_main_stream(erase_model* m) { return m ? (void*)m->main : nullptr; }
 
 int64_t erase_launch_count(const erase_model* m) { return m ? m->launches : 0; }
@@ -1469,11 +1480,14 @@ erase_status erase_gemm(int32_t dtype, int32_t M, int32_t N, int32_t K, const vo
   cudaError_t e = cudaMemsetAsync(status, 0, 4 * sizeof(int), st);   // status word + two scheduler words
   if (e != cudaSuccess) return cuda_fail(e, "memset");
   g.ws = ws;
+#ifdef ERASE_DEV_AIDS
   long long* dbg = nullptr;
+#endif
   if (engine == 1) {
     TcPlan plan;
     if (!tc_gemm_plan(g, status, &plan)) { cleanup(); g_create_error = "erase_gemm: TMA descriptor encoding failed"; return ERASE_EUNSUPPORTED; }
     plan.sched = status + 1;
+#ifdef ERASE_DEV_AIDS
     if (getenv("ERASE_TC_TIMELINE")) {   // development aid: print CTA 0's clock stamps for its first tile
       if (cudaMalloc(&dbg, 16 * sizeof(long long)) == cudaSuccess) {
         long long h[16] = {0};
@@ -1483,6 +1497,7 @@ erase_status erase_gemm(int32_t dtype, int32_t M, int32_t N, int32_t K, const vo
       }
       plan.dbg = dbg;
     }
+#endif
     e = tc_gemm_launch(g, plan, st);
   } else {
     e = gemm_simt(g, bf, st);
@@ -1496,6 +1511,7 @@ erase_status erase_gemm(int32_t dtype, int32_t M, int32_t N, int32_t K, const vo
   e = cudaMemcpyAsync(&hst, status, sizeof(int), cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) return cuda_fail(e, "execution");
+#ifdef ERASE_DEV_AIDS
   if (dbg) {
     long long h[16];
     if (cudaMemcpy(h, dbg, sizeof(h), cudaMemcpyDeviceToHost) == cudaSuccess)
@@ -1507,6 +1523,7 @@ erase_status erase_gemm(int32_t dtype, int32_t M, int32_t N, int32_t K, const vo
     if (getenv("ERASE_TC_PAIR")) fprintf(stderr, "   pair kernel: TMEM base of the leader %lld, of the peer %lld\n", h[8], h[9]);
     cudaFree(dbg);
   }
+#endif
   cleanup();
   if (hst != 0) { g_create_error = "erase_gemm: a bounded device-side wait expired (code " + std::to_string(hst) + ")"; return ERASE_ETIMEOUT; }
   return ERASE_OK;

@@ -8,6 +8,7 @@
 // status word live in a fixed array in the library's own device image instead.
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <string>
 
 #include "../../include/erase.h"
@@ -24,7 +25,7 @@ constexpr size_t kWsFloats = ERASE_STATIC_WS_FLOATS;
 static __device__ __align__(256) float g_static_scratch[kWsFloats + 64];
 
 constexpr int kMaxDevices = 64;
-float* g_scratch_addr[kMaxDevices] = {nullptr};  // device address of g_static_scratch, per device
+std::atomic<float*> g_scratch_addr[kMaxDevices];  // device address of g_static_scratch, per device (host threads may race to fill it: same value)
 
 thread_local std::string g_static_error;
 
@@ -58,16 +59,16 @@ ERASE_API erase_status erase_gemm_static(int32_t dtype, int32_t M, int32_t N, in
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return fail(ERASE_ECUDA, std::string("cudaGetDevice: ") + cudaGetErrorString(e));
   if (dev < 0 || dev >= kMaxDevices) return fail(ERASE_EUNSUPPORTED, "device ordinal out of range");
-  if (!g_scratch_addr[dev]) {
+  if (!g_scratch_addr[dev].load(std::memory_order_acquire)) {
     float* ptr = nullptr;
     e = cudaGetSymbolAddress((void**)&ptr, g_static_scratch);
     if (e != cudaSuccess || !ptr) {
       cudaGetLastError();
       return fail(ERASE_ECUDA, std::string("cudaGetSymbolAddress: ") + cudaGetErrorString(e));
     }
-    g_scratch_addr[dev] = ptr;
+    g_scratch_addr[dev].store(ptr, std::memory_order_release);
   }
-  float* ws = g_scratch_addr[dev];
+  float* ws = g_scratch_addr[dev].load(std::memory_order_acquire);
   int* status = reinterpret_cast<int*>(ws + kWsFloats);
 
   cudaStream_t st = (cudaStream_t)stream;

@@ -25,6 +25,8 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
+
 namespace erase {
 
 namespace {
@@ -37,7 +39,7 @@ constexpr uint32_t EPI_BIAS_BYTES = 512;              // up to 128 bias floats p
 constexpr int EPI_WARPS = 8;                       // two per TMEM lane quarter, each takes half the columns
 constexpr int TC_THREADS = 32 * (2 + EPI_WARPS);
 constexpr uint32_t EPI_STAGE_BYTES = 8192;             // two buffers of 32 rows x 128 bytes per epilogue warp
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;  // ~2 s at 2 GHz
+constexpr long long WAIT_LIMIT_CYCLES = 500000000LL;   // ~0.25 s at 2 GHz; a legitimate wait lasts one tile's main loop (< 1 ms)
 
 struct TcArgs {
   int M, N, K;
@@ -74,13 +76,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait: false if the limit expired (status word is set by the caller).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long limit = WAIT_LIMIT_CYCLES) {
   if (mbar_try_wait(bar, parity)) return true;
   long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > WAIT_LIMIT_CYCLES) return false;
+    if (clock64() - t0 > limit) return false;
   }
   return true;
+}
+// A launch that finds the status word already set (an earlier wait of this step expired, or the
+// input staging met an id out of range) does nothing: thread 0 reads the word while the barriers and
+// TMEM are being set up, and the whole CTA skips its role loops.  One expired wait therefore costs
+// one limit, not one per later wait and launch.
+__device__ __forceinline__ int status_peek(const int* status) {
+  int v = 0;
+  if (status && threadIdx.x == 0) v = *reinterpret_cast<const volatile int*>(status);
+  return v;
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
@@ -130,6 +141,11 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
 }
 
 __device__ __forceinline__ float bf2f(uint32_t bits16) { return __uint_as_float(bits16 << 16); }
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 
 // Only ReLU is fused (a compare).  GELU's erf chain on the few epilogue warps, and the instruction
 // footprint of its inlined copies, made a fused GEMM slower than the GEMM plus a separate
@@ -271,7 +287,11 @@ __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int
 // GENERAL = false compiles the epilogue down to "identity or bias add" (forward Linears without
 // activation, every dgrad/wgrad without auxiliary operand): a much smaller loop body, which is what
 // bounds the epilogue (instruction fetch), so those GEMMs get their own instantiation.
-template <int BN, bool A_MN, bool B_MN, bool GENERAL>
+// CE = true (local softmax cross-entropy head, forward): the epilogue turns a logit l into
+// exp(l - ref[row]) with a per-row reference known before the GEMM, stores that (bf16) instead of
+// the logit and leaves, per row and group of CPW columns, the fp32 sum of the unrounded
+// exponentials in ce_psum[row][group]: the head's loss and gradient then need no pass over logits.
+template <int BN, bool A_MN, bool B_MN, bool GENERAL, bool CE = false>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_c,
@@ -304,7 +324,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const uint32_t tmem_slot = bar_base + 8u * (2 * STAGES + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int st0 = status_peek(p.status);
+#ifdef ERASE_DEV_AIDS   // clock stamps of CTA 0's first tile: compiled in only with -DERASE_DEV_AIDS
   const bool dbg = p.dbg != nullptr && blockIdx.x == 0;
+#else
+  constexpr bool dbg = false;
+#endif
   if (dbg && threadIdx.x == 0) p.dbg[0] = clock64();
   if (threadIdx.x == 32) {   // descriptor fetches overlap the barrier and TMEM set-up
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
@@ -336,12 +361,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
-  __syncthreads();
+  const bool dead = __syncthreads_or(st0 != 0) != 0;
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_ptr;
   if (dbg && threadIdx.x == 0) p.dbg[1] = clock64();
 
-  if (warp == 0) {
+  if (dead) {
+    // the step is already void: do nothing but free TMEM below
+  } else if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
       uint32_t it = 0, slot = 0;
@@ -485,6 +512,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
       const int row = m0 + q * 32 + lane;
       const bool row_ok = row < p.M;
+      float ce_ref2 = 0.f, ce_sum = 0.f;          // CE: this row's reference (in log2 units) and its running sum
+      if (CE && row_ok) ce_ref2 = __ldg(p.epi.ce_ref + row) * 1.4426950408889634f;
       // auxiliary operands of this thread's row (raw bf16), fetched one 32-column chunk ahead
       const __nv_bfloat16* aux_pa = nullptr;
       const __nv_bfloat16* aux_pb = nullptr;
@@ -505,7 +534,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (!ok) break;
       tc_fence_after();
       if (dbg && lt == 0 && threadIdx.x == 64) p.dbg[5] = clock64();
+#ifdef ERASE_DEV_AIDS
       const long long dflags = p.dbg ? p.dbg[15] : 0;
+#else
+      constexpr long long dflags = 0;
+#endif
       if (active && n0 + cbeg < p.N) {
         {
           const bool via_tma = p.tma_c != 0;
@@ -538,7 +571,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               F8 f;
 #pragma unroll
               for (int j = 0; j < 8; j++) f.v[j] = __uint_as_float(r[g8 * 8 + j]);
-              if (p.plain == 2) {          // bias only: the common forward case, kept free of the general path
+              if (CE) {                    // logit -> exp(logit - reference); columns past N contribute nothing
+                const float4 b0 = *reinterpret_cast<const float4*>(bias_s + cc + g8 * 8);
+                const float4 b1 = *reinterpret_cast<const float4*>(bias_s + cc + g8 * 8 + 4);
+                const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+                const bool full = n + 8 <= p.N;
+#pragma unroll
+                for (int j = 0; j < 8; j++) {
+                  float e = ex2_approx(fmaf(f.v[j] + bb[j], 1.4426950408889634f, -ce_ref2));
+                  if (!full && n + j >= p.N) e = 0.f;
+                  ce_sum += e;
+                  f.v[j] = e;
+                }
+              } else if (p.plain == 2) {          // bias only: the common forward case, kept free of the general path
                 const float4 b0 = *reinterpret_cast<const float4*>(bias_s + cc + g8 * 8);
                 const float4 b1 = *reinterpret_cast<const float4*>(bias_s + cc + g8 * 8 + 4);
                 f.v[0] += b0.x; f.v[1] += b0.y; f.v[2] += b0.z; f.v[3] += b0.w;
@@ -575,6 +620,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
         }
       }
+      if (CE && active && row_ok && n0 + cbeg < p.N)
+        p.epi.ce_psum[(long long)row * p.epi.ce_groups + (n0 + cbeg) / CPW] = ce_sum;
       // all TMEM reads of this warp are complete (tcgen05.wait::ld): hand the accumulator back
       if (dbg && lt == 0 && threadIdx.x == 64) p.dbg[12] = clock64();
       tc_fence_before();
@@ -660,7 +707,7 @@ __device__ __forceinline__ void tc_mma_pair(uint32_t tmem_d, uint64_t adesc, uin
       : "memory");
 }
 
-template <bool A_MN, bool B_MN, bool GENERAL>
+template <bool A_MN, bool B_MN, bool GENERAL, bool CE = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     const __grid_constant__ CUtensorMap map_c, const __grid_constant__ TcArgs p, const uint32_t tmem_cols) {
@@ -685,6 +732,8 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   const uint32_t tmem_slot = bar_base + 8u * (2 * STAGES + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  __shared__ int dead_flag;
+  if (threadIdx.x == 0) dead_flag = status_peek(p.status) != 0 ? 1 : 0;
   const uint32_t rank = cluster_ctarank();
   const bool leader = rank == 0;
   const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
@@ -719,9 +768,15 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   cluster_sync_all();      // the peer's barriers exist before anything is sent to them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_ptr;
+#ifdef ERASE_DEV_AIDS
   if (p.dbg && threadIdx.x == 0 && cluster_id == 0) p.dbg[8 + rank] = (long long)tmem_base;
+#endif
+  int dead;   // both CTAs of the pair take the LEADER's reading, so that they skip (or work) together
+  asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(dead) : "r"(map_to_cta(smem_u32(&dead_flag), 0)) : "memory");
 
-  if (warp == 0) {
+  if (dead) {
+    // the step is already void: do nothing but free TMEM below
+  } else if (warp == 0) {
     // ------------------------------ TMA producer (both CTAs) ------------------------------
     if (lane == 0) {
       uint32_t it = 0;
@@ -826,6 +881,8 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       }
       const int row = m0 + q * 32 + lane;
       const bool row_ok = row < p.M;
+      float ce_ref2 = 0.f, ce_sum = 0.f;          // CE: this row's reference (in log2 units) and its running sum
+      if (CE && row_ok) ce_ref2 = __ldg(p.epi.ce_ref + row) * 1.4426950408889634f;
       // auxiliary operands of this thread's row (raw bf16), fetched one 32-column chunk ahead
       const __nv_bfloat16* aux_pa = nullptr;
       const __nv_bfloat16* aux_pb = nullptr;
@@ -873,7 +930,20 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             float* v = f.v;
 #pragma unroll
             for (int j = 0; j < 8; j++) v[j] = __uint_as_float(r[g8 * 8 + j]);
-            if (p.plain == 2) {
+            if (CE) {                      // logit -> exp(logit - reference); columns past N contribute nothing
+              const float4 b0 = *reinterpret_cast<const float4*>(bias_s + cc + g8 * 8);
+              const float4 b1 = *reinterpret_cast<const float4*>(bias_s + cc + g8 * 8 + 4);
+              const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+              const int n = n0 + c0 + g8 * 8;
+              const bool full = n + 8 <= p.N;
+#pragma unroll
+              for (int j = 0; j < 8; j++) {
+                float e = ex2_approx(fmaf(v[j] + bb[j], 1.4426950408889634f, -ce_ref2));
+                if (!full && n + j >= p.N) e = 0.f;
+                ce_sum += e;
+                v[j] = e;
+              }
+            } else if (p.plain == 2) {
               const float4 b0 = *reinterpret_cast<const float4*>(bias_s + cc + g8 * 8);
               const float4 b1 = *reinterpret_cast<const float4*>(bias_s + cc + g8 * 8 + 4);
               v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w;
@@ -904,6 +974,8 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           }
         }
       }
+      if (CE && row_ok && n0 + cbeg < p.N)
+        p.epi.ce_psum[(long long)row * p.epi.ce_groups + (n0 + cbeg) / CPW] = ce_sum;
       tc_fence_before();
       __syncwarp();
       if (lane == 0) {   // accumulator drained: tell the leader's MMA thread
@@ -979,6 +1051,7 @@ tc_wgrad_group_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
   const uint32_t tmem_slot = bar_base + 8u * (2 * STAGES + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int st0 = status_peek(g.status);
   if (threadIdx.x == 32) {
     for (int i = 0; i < g.nprob; i++) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.a[i]) : "memory");
@@ -1003,11 +1076,13 @@ tc_wgrad_group_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
-  __syncthreads();
+  const bool dead = __syncthreads_or(st0 != 0) != 0;
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_ptr;
 
-  if (warp == 0) {
+  if (dead) {
+    // the step is already void: do nothing but free TMEM below
+  } else if (warp == 0) {
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
@@ -1140,23 +1215,60 @@ tc_wgrad_group_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
   }
 }
 
+// The bounded wait on its own: one thread waits, with the given limit, on a barrier that nothing
+// ever signals, records status code 8 and returns.  It returns by construction (the wait is
+// clock-bounded) and touches no tensor memory; used to check that an expired wait surfaces as
+// ERASE_ETIMEOUT and leaves the context usable.
+__global__ void wait_selftest_kernel(int* status, long long limit_cycles) {
+  __shared__ __align__(8) uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (!mbar_wait(smem_u32(&bar), 0, limit_cycles)) atomicExch(status, 8);
+  }
+}
+
+// Host-side caches are per device: a process may drive several GPUs.
+constexpr int MAX_DEVICES = 64;
+int current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) dev = 0;
+  return dev;
+}
+int sm_count() {
+  static std::atomic<int> cache[MAX_DEVICES];
+  const int dev = current_device();
+  int n = cache[dev].load(std::memory_order_relaxed);
+  if (n == 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 2) n = 148;
+    cache[dev].store(n, std::memory_order_relaxed);
+  }
+  return n;
+}
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per (kernel, device); `done` is the kernel's own table
+template <typename K>
+cudaError_t ensure_smem(K kernel, size_t smem, std::atomic<bool>* done) {
+  const int dev = current_device();
+  if (done[dev].load(std::memory_order_acquire)) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e == cudaSuccess) done[dev].store(true, std::memory_order_release);
+  return e;
+}
+
 typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 EncodeFn encode_fn() {
-  static EncodeFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
+  static const EncodeFn fn = []() -> EncodeFn {   // initialised once, thread-safe (the entry point is process-wide)
     void* p = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
         qres == cudaDriverEntryPointSuccess)
-      fn = (EncodeFn)p;
-    else
-      cudaGetLastError();
-  }
+      return (EncodeFn)p;
+    cudaGetLastError();
+    return nullptr;
+  }();
   return fn;
 }
 
@@ -1187,26 +1299,17 @@ bool encode_2d(void* out, const void* base, long long inner, long long outer, lo
   return encode_map(out, base, false, 2, dims, strides, box);
 }
 
-template <int BN, bool A_MN, bool B_MN, bool GENERAL>
+template <int BN, bool A_MN, bool B_MN, bool GENERAL, bool CE = false>
 cudaError_t launch_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas) {
   constexpr int STAGES = stages_for(BN);
   constexpr size_t smem = (size_t)STAGES * (BM * BK * 2 + BN * BK * 2) + EPI_WARPS * (EPI_STAGE_BYTES + EPI_BIAS_BYTES) + 8 * (2 * STAGES + 16) + 1024;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<BN, A_MN, B_MN, GENERAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static std::atomic<bool> attr_set[MAX_DEVICES];
+  if (cudaError_t e = ensure_smem(tc_gemm_kernel<BN, A_MN, B_MN, GENERAL, CE>, smem, attr_set)) return e;
   TcArgs p;
   p.M = g.M; p.N = g.N; p.K = g.K;
   p.C = g.C; p.ldc = g.ldc; p.c_f32 = g.c_f32;
   p.splits = g.splits; p.ws = g.ws; p.epi = g.epi; p.status = plan.status; p.dbg = plan.dbg; p.sched = plan.sched;
-  static int num_sms = 0;
-  if (num_sms == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms < 1) num_sms = 148;
-  }
+  const int num_sms = sm_count();
   const long long total = (long long)((g.N + BN - 1) / BN) * ((g.M + BM - 1) / BM) * g.splits;
   long long cap = (max_ctas > 0 && max_ctas < num_sms) ? max_ctas : num_sms;
   dim3 grid((unsigned)(total < cap ? total : cap));
@@ -1220,19 +1323,15 @@ cudaError_t launch_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int 
   const bool no_aux = e.alpha == 1.f && e.act == ACT_NONE && !e.pre_out && !e.mul && !e.res && e.dact == ACT_NONE;
   p.plain = no_aux ? (e.bias ? (g.splits == 1 ? 2 : 1) : 1) : 0;   // 1: identity, 2: bias only, 0: general
   if (total <= (long long)grid.x) p.sched = nullptr;   // one tile per CTA: nothing to balance
-  tc_gemm_kernel<BN, A_MN, B_MN, GENERAL><<<grid, TC_THREADS, smem, s>>>(ma, mb, mc, p);
+  tc_gemm_kernel<BN, A_MN, B_MN, GENERAL, CE><<<grid, TC_THREADS, smem, s>>>(ma, mb, mc, p);
   return cudaGetLastError();
 }
 
-template <bool A_MN, bool B_MN, bool GENERAL>
+template <bool A_MN, bool B_MN, bool GENERAL, bool CE = false>
 cudaError_t launch_pair_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas) {
   constexpr size_t smem = (size_t)PAIR_STAGES * PAIR_STAGE_BYTES + EPI_WARPS * (EPI_STAGE_BYTES + EPI_BIAS_BYTES) + 8 * (2 * PAIR_STAGES + 16) + 1024;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(tc_gemm_pair_kernel<A_MN, B_MN, GENERAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static std::atomic<bool> attr_set[MAX_DEVICES];
+  if (cudaError_t e = ensure_smem(tc_gemm_pair_kernel<A_MN, B_MN, GENERAL, CE>, smem, attr_set)) return e;
   TcArgs p;
   p.M = g.M; p.N = g.N; p.K = g.K;
   p.C = g.C; p.ldc = g.ldc; p.c_f32 = g.c_f32;
@@ -1241,12 +1340,7 @@ cudaError_t launch_pair_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s,
   const Epilogue& e = g.epi;
   const bool no_aux = e.alpha == 1.f && e.act == ACT_NONE && !e.pre_out && !e.mul && !e.res && e.dact == ACT_NONE;
   p.plain = no_aux ? (e.bias ? (g.splits == 1 ? 2 : 1) : 1) : 0;   // 1: identity, 2: bias only, 0: general
-  static int num_sms = 0;
-  if (num_sms == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms < 2) num_sms = 148;
-  }
+  const int num_sms = sm_count();
   const long long total = (long long)((g.N + PAIR_BN - 1) / PAIR_BN) * ((g.M + 2 * BM - 1) / (2 * BM)) * g.splits;
   long long cap = ((max_ctas > 1 && max_ctas < num_sms) ? max_ctas : num_sms) / 2;
   dim3 grid(2u * (unsigned)(total < cap ? total : cap));
@@ -1254,7 +1348,7 @@ cudaError_t launch_pair_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s,
   memcpy(&ma, plan.map_a, sizeof(ma));
   memcpy(&mb, plan.b_mn ? plan.map_b : plan.map_b_half, sizeof(mb));
   memcpy(&mc, plan.map_c, sizeof(mc));
-  tc_gemm_pair_kernel<A_MN, B_MN, GENERAL><<<grid, TC_THREADS, smem, s>>>(ma, mb, mc, p, (uint32_t)plan.pair_tmem_cols);
+  tc_gemm_pair_kernel<A_MN, B_MN, GENERAL, CE><<<grid, TC_THREADS, smem, s>>>(ma, mb, mc, p, (uint32_t)plan.pair_tmem_cols);
   return cudaGetLastError();
 }
 
@@ -1272,6 +1366,11 @@ cudaError_t launch_bn(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int
 }
 
 }  // namespace
+
+cudaError_t tc_wait_selftest(int* status, long long limit_cycles, cudaStream_t s) {
+  wait_selftest_kernel<<<1, 32, 0, s>>>(status, limit_cycles);
+  return cudaGetLastError();
+}
 
 bool tc_wgrad_group_plan(const GemmArgs* gs, int n, int* status, TcGroupPlan* plan) {
   if (n < 1 || n > GROUP_MAX) return false;
@@ -1300,12 +1399,8 @@ bool tc_wgrad_group_plan(const GemmArgs* gs, int n, int* status, TcGroupPlan* pl
 
 cudaError_t tc_wgrad_group_launch(const TcGroupPlan& plan, cudaStream_t s, int max_ctas) {
   constexpr size_t smem = (size_t)4 * (BM * BK * 2 + 128 * BK * 2) + EPI_WARPS * EPI_STAGE_BYTES + 8 * (2 * 4 + 16) + 1024;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(tc_wgrad_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static std::atomic<bool> attr_set[MAX_DEVICES];
+  if (cudaError_t e = ensure_smem(tc_wgrad_group_kernel, smem, attr_set)) return e;
   GroupMaps maps;
   GroupArgs g;
   memset(&g, 0, sizeof(g));
@@ -1317,12 +1412,7 @@ cudaError_t tc_wgrad_group_launch(const TcGroupPlan& plan, cudaStream_t s, int m
     g.prob[i] = GroupProblem{plan.M[i], plan.N[i], plan.K[i], plan.splits[i], plan.kchunk[i], plan.tiles_m[i], plan.tiles_n[i], plan.tile_begin[i]};
   }
   for (int i = plan.n; i < GROUP_MAX; i++) { maps.a[i] = maps.a[0]; maps.b[i] = maps.b[0]; maps.c[i] = maps.c[0]; }
-  static int num_sms = 0;
-  if (num_sms == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms < 1) num_sms = 148;
-  }
+  const int num_sms = sm_count();
   int cap = (max_ctas > 0 && max_ctas < num_sms) ? max_ctas : num_sms;
   dim3 grid((unsigned)(plan.total < cap ? plan.total : cap));
   tc_wgrad_group_kernel<<<grid, TC_THREADS, smem, s>>>(maps, g);
@@ -1410,7 +1500,18 @@ bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan) {
   return true;
 }
 
+int tc_ce_group_cols(const TcPlan& plan) { return (plan.pair || plan.bn >= 128) ? plan.bn / 2 : 64; }
+
 cudaError_t tc_gemm_launch(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas) {
+  if (g.epi.ce_ref) {   // cross-entropy head forward: both operands K-major, bias, bf16 output through TMA
+    if (plan.a_mn || plan.b_mn || !plan.tma_c || g.splits != 1 || !g.epi.bias || !g.epi.ce_psum) return cudaErrorInvalidValue;
+    if (plan.pair) return launch_pair_t<false, false, false, true>(g, plan, s, max_ctas);
+    switch (plan.bn) {
+      case 64: return launch_t<64, false, false, false, true>(g, plan, s, max_ctas);
+      case 256: return launch_t<256, false, false, false, true>(g, plan, s, max_ctas);
+      default: return launch_t<128, false, false, false, true>(g, plan, s, max_ctas);
+    }
+  }
   const bool simple = epilogue_is_simple(g);
   if (plan.pair) {
     if (simple) {

@@ -36,6 +36,9 @@ bool tc_gemm_supported(const GemmArgs& g);
 // Encodes the TMA descriptors.  g.ws must already point at splits*M*N floats when g.splits > 1.
 // Returns false (and leaves the GEMM to the SIMT kernel) if a descriptor cannot be encoded.
 bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan);
+// Cross-entropy head forward (g.epi.ce_ref set): columns per partial-sum group of ce_psum for this plan;
+// ce_groups must be ceil(N / that).
+int tc_ce_group_cols(const TcPlan& plan);
 // max_ctas > 0 caps the persistent grid (an SM budget: lets kernels of other streams run beside it);
 // the tile-to-CTA assignment does not enter the arithmetic, so results do not depend on it.
 cudaError_t tc_gemm_launch(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas = 0);
@@ -50,5 +53,9 @@ struct TcGroupPlan {
 };
 bool tc_wgrad_group_plan(const GemmArgs* gs, int n, int* status, TcGroupPlan* plan);
 cudaError_t tc_wgrad_group_launch(const TcGroupPlan& plan, cudaStream_t s, int max_ctas = 0);
+
+// Launches one thread that waits, for at most limit_cycles SM clocks, on a barrier nothing signals,
+// then sets *status to 8 and returns: the bounded-wait helper of the GEMM kernels on its own.
+cudaError_t tc_wait_selftest(int* status, long long limit_cycles, cudaStream_t s);
 
 }  // namespace erase

@@ -6,6 +6,8 @@
 
 #include <stdlib.h>
 
+#include <algorithm>
+
 #include <cuda_bf16.h>
 #include <math.h>
 
@@ -1101,7 +1103,8 @@ __global__ void __launch_bounds__(256) softmax_ce_kernel(T* __restrict__ logits,
   __shared__ float sm[8];
   const int row = blockIdx.x;
   T* p = logits + (long long)row * V;
-  const int tgt = ids[(long long)(row / T_) * (T_ + 1) + (row % T_) + 1];
+  // an id out of range was reported by the input staging; here it must only not be used as an index
+  const int tgt = min(max(ids[(long long)(row / T_) * (T_ + 1) + (row % T_) + 1], 0), V - 1);
   const float lt = ldf(p + tgt);
   float mx = -INFINITY;
   for (int v = threadIdx.x; v < V; v += 256) mx = fmaxf(mx, ldf(p + v));
@@ -1659,50 +1662,111 @@ cudaError_t ew_dact(void* d, const void* src, int act, long long n, bool bf16, c
 // ------------------------------------------------------------------------------------------
 // input staging (z_0)
 // ------------------------------------------------------------------------------------------
-template <typename T>
-__global__ void gather_tokens_kernel(const float* __restrict__ tok, const float* __restrict__ pos,
-                                     const int32_t* __restrict__ ids, T* __restrict__ z0, int T_, int d,
-                                     long long n) {
-  long long i = (long long)blockIdx.x * 256 + threadIdx.x;
-  if (i >= n) return;
-  int c = (int)(i % d);
-  long long row = i / d;
-  int t = (int)(row % T_);
-  long long b = row / T_;
-  int id = ids[b * (T_ + 1) + t];
-  stf(z0 + i, tok[(long long)id * d + c] + pos[(long long)t * d + c]);
+// An id outside its table is never used as an index: the row is filled from row 0 instead and the
+// model's status word is set to STATUS_BAD_ID, which the next synchronisation reports as an
+// invalid argument (the step's results are void).
+__device__ __forceinline__ int checked_id(int id, int rows, int* status) {
+  if ((unsigned)id >= (unsigned)rows) {
+    if (status) atomicExch(status, STATUS_BAD_ID);
+    return 0;
+  }
+  return id;
+}
+
+__device__ __forceinline__ void store4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+__device__ __forceinline__ void store4(bf16_t* p, float4 v) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+  uint2 q;
+  q.x = *reinterpret_cast<uint32_t*>(&lo);
+  q.y = *reinterpret_cast<uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(p) = q;
+}
+
+// Token + position gather, one warp per output row: the id is read once per row, a lane moves four
+// consecutive columns per step (two 16-byte loads, one 8- or 16-byte store), so a warp reads 512
+// contiguous bytes of the embedding row at a time.  VEC = false is the scalar form for widths that
+// are not multiples of four.
+template <typename T, bool VEC>
+__global__ void __launch_bounds__(256) gather_tokens_kernel(const float* __restrict__ tok, const float* __restrict__ pos,
+                                                            const int32_t* __restrict__ ids, T* __restrict__ z0, int T_, int d,
+                                                            int rows, int vocab, int* status) {
+  const int lane = threadIdx.x & 31;
+  for (int row = blockIdx.x * 8 + (threadIdx.x >> 5); row < rows; row += gridDim.x * 8) {
+    const int t = row % T_, b = row / T_;
+    const int id = checked_id(ids[(long long)b * (T_ + 1) + t], vocab, status);
+    if (t == T_ - 1 && lane == 0) checked_id(ids[(long long)b * (T_ + 1) + T_], vocab, status);   // the last target is no input
+    const float* te = tok + (long long)id * d;
+    const float* pe = pos + (long long)t * d;
+    T* out = z0 + (long long)row * d;
+    if (VEC) {
+      for (int c = lane * 4; c < d; c += 128) {
+        const float4 a = __ldg(reinterpret_cast<const float4*>(te + c));
+        const float4 q = __ldg(reinterpret_cast<const float4*>(pe + c));
+        store4(out + c, make_float4(a.x + q.x, a.y + q.y, a.z + q.z, a.w + q.w));
+      }
+    } else {
+      for (int c = lane; c < d; c += 32) stf(out + c, te[c] + pe[c]);
+    }
+  }
 }
 cudaError_t gather_tokens(const float* tok, const float* pos, const int32_t* ids, void* z0, int batch,
-                          int T_, int d, bool bf16, cudaStream_t s) {
-  long long n = (long long)batch * T_ * d;
-  if (bf16) gather_tokens_kernel<bf16_t><<<cdiv(n, 256), 256, 0, s>>>(tok, pos, ids, (bf16_t*)z0, T_, d, n);
-  else gather_tokens_kernel<float><<<cdiv(n, 256), 256, 0, s>>>(tok, pos, ids, (float*)z0, T_, d, n);
+                          int T_, int d, int vocab, int* status, bool bf16, cudaStream_t s) {
+  const int rows = batch * T_;
+  const bool vec = d % 4 == 0 && ((reinterpret_cast<uintptr_t>(tok) | reinterpret_cast<uintptr_t>(pos) | reinterpret_cast<uintptr_t>(z0)) & 15) == 0;
+  const int grid = (int)std::min<long long>(cdiv(rows, 8), 148 * 8);
+  if (bf16) {
+    if (vec) gather_tokens_kernel<bf16_t, true><<<grid, 256, 0, s>>>(tok, pos, ids, (bf16_t*)z0, T_, d, rows, vocab, status);
+    else gather_tokens_kernel<bf16_t, false><<<grid, 256, 0, s>>>(tok, pos, ids, (bf16_t*)z0, T_, d, rows, vocab, status);
+  } else {
+    if (vec) gather_tokens_kernel<float, true><<<grid, 256, 0, s>>>(tok, pos, ids, (float*)z0, T_, d, rows, vocab, status);
+    else gather_tokens_kernel<float, false><<<grid, 256, 0, s>>>(tok, pos, ids, (float*)z0, T_, d, rows, vocab, status);
+  }
   return cudaGetLastError();
 }
 
-template <typename T>
-__global__ void gather_ctr_kernel(const float* __restrict__ tables, long long table_stride,
-                                  const int32_t* __restrict__ ids, const float* __restrict__ dense,
-                                  T* __restrict__ x0, int ns, int e, int nd, int width, long long n) {
-  long long i = (long long)blockIdx.x * 256 + threadIdx.x;
-  if (i >= n) return;
-  int c = (int)(i % width);
-  long long row = i / width;
-  float v = 0.f;
-  if (c < ns * e) {
-    int t = c / e, cc = c - t * e;
-    int id = ids[row * ns + t];
-    v = tables[(long long)t * table_stride + (long long)id * e + cc];
-  } else if (c < ns * e + nd) {
-    v = dense[row * nd + (c - ns * e)];
+// CTR gather and pack, one warp per sample: x0[n] = [table_t[ids[n,t]] for t | dense | zero pad].
+// The lanes run over (table, four columns) pairs, so a table row leaves as 16-byte loads and lands
+// as 8-byte (bf16) or 16-byte stores; the dense columns and the padding follow in a scalar tail.
+template <typename T, bool VEC>
+__global__ void __launch_bounds__(256) gather_ctr_kernel(const float* __restrict__ tables, long long table_stride,
+                                                         const int32_t* __restrict__ ids, const float* __restrict__ dense,
+                                                         T* __restrict__ x0, int batch, int ns, int e, int nd, int width,
+                                                         int table_rows, int* status) {
+  const int lane = threadIdx.x & 31;
+  for (int n = blockIdx.x * 8 + (threadIdx.x >> 5); n < batch; n += gridDim.x * 8) {
+    T* out = x0 + (long long)n * width;
+    const int32_t* idn = ids + (long long)n * ns;
+    if (VEC) {
+      const int vpr = e >> 2;                                  // 16-byte vectors per table row
+      for (int i = lane; i < ns * vpr; i += 32) {
+        const int t = i / vpr, c = (i - t * vpr) * 4;
+        const int id = checked_id(idn[t], table_rows, status);
+        const float4 v = __ldg(reinterpret_cast<const float4*>(tables + (long long)t * table_stride + (long long)id * e + c));
+        store4(out + t * e + c, v);
+      }
+    } else {
+      for (int i = lane; i < ns * e; i += 32) {
+        const int t = i / e, c = i - t * e;
+        const int id = checked_id(idn[t], table_rows, status);
+        stf(out + i, tables[(long long)t * table_stride + (long long)id * e + c]);
+      }
+    }
+    for (int c = ns * e + lane; c < width; c += 32) stf(out + c, c < ns * e + nd ? dense[(long long)n * nd + (c - ns * e)] : 0.f);
   }
-  stf(x0 + i, v);
 }
 cudaError_t gather_ctr(const float* tables, long long table_stride, const int32_t* ids, const float* dense,
-                       void* x0, int batch, int ns, int e, int nd, int width, bool bf16, cudaStream_t s) {
-  long long n = (long long)batch * width;
-  if (bf16) gather_ctr_kernel<bf16_t><<<cdiv(n, 256), 256, 0, s>>>(tables, table_stride, ids, dense, (bf16_t*)x0, ns, e, nd, width, n);
-  else gather_ctr_kernel<float><<<cdiv(n, 256), 256, 0, s>>>(tables, table_stride, ids, dense, (float*)x0, ns, e, nd, width, n);
+                       void* x0, int batch, int ns, int e, int nd, int width, int table_rows, int* status, bool bf16,
+                       cudaStream_t s) {
+  const bool vec = e % 4 == 0 && width % 4 == 0 && table_stride % 4 == 0 &&
+                   ((reinterpret_cast<uintptr_t>(tables) | reinterpret_cast<uintptr_t>(x0)) & 15) == 0;
+  const int grid = (int)std::min<long long>(cdiv(batch, 8), 148 * 8);
+  if (bf16) {
+    if (vec) gather_ctr_kernel<bf16_t, true><<<grid, 256, 0, s>>>(tables, table_stride, ids, dense, (bf16_t*)x0, batch, ns, e, nd, width, table_rows, status);
+    else gather_ctr_kernel<bf16_t, false><<<grid, 256, 0, s>>>(tables, table_stride, ids, dense, (bf16_t*)x0, batch, ns, e, nd, width, table_rows, status);
+  } else {
+    if (vec) gather_ctr_kernel<float, true><<<grid, 256, 0, s>>>(tables, table_stride, ids, dense, (float*)x0, batch, ns, e, nd, width, table_rows, status);
+    else gather_ctr_kernel<float, false><<<grid, 256, 0, s>>>(tables, table_stride, ids, dense, (float*)x0, batch, ns, e, nd, width, table_rows, status);
+  }
   return cudaGetLastError();
 }
 

@@ -11,6 +11,10 @@ namespace erase {
 
 enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU = 2 };
 
+// Values of a model's device status word (0 = fine).  1..8: a bounded device-side wait expired
+// (which one); STATUS_BAD_ID: the input staging met a token or sparse id outside its table.
+enum { STATUS_WAIT_SELFTEST = 8, STATUS_BAD_ID = 64 };
+
 // Epilogue of C = A * B^T.  With v = alpha * acc (+ bias[n]):
 //   pre_out != 0 : pre_out[m,n] = v                    (pre-activation kept for the backward)
 //   v = act(v)
@@ -29,6 +33,12 @@ struct Epilogue {
   const void* dact_src = nullptr;
   long long ld_aux = 0;
   float alpha = 1.f;
+  // Softmax cross-entropy head, forward (tensor-core kernels only): with l = acc + bias[n] the GEMM
+  // stores exp(l - ce_ref[m]) instead of l and writes the fp32 sum of the unrounded exponentials of
+  // row m over each group of columns to ce_psum[m * ce_groups + group].
+  const float* ce_ref = nullptr;
+  float* ce_psum = nullptr;
+  int ce_groups = 0;
 };
 
 // C[M,N] = epilogue( sum_k A(m,k) * B(n,k) ).  A(m,k) = A[m*sa_m + k*sa_k], B likewise, so one
@@ -151,13 +161,16 @@ cudaError_t ew_act(const void* u, void* out, int act, long long n, bool bf16, cu
 // d <- d * act'(src)
 cudaError_t ew_dact(void* d, const void* src, int act, long long n, bool bf16, cudaStream_t s);
 
-// z0[b*T+t, :] = tok[ids[b*(T+1)+t], :] + pos[t, :]
+// z0[b*T+t, :] = tok[ids[b*(T+1)+t], :] + pos[t, :].  Every id of the batch (inputs and the last
+// target column) is checked against [0, vocab): an id outside is not dereferenced (row 0 stands in)
+// and *status is set to STATUS_BAD_ID.
 cudaError_t gather_tokens(const float* tok, const float* pos, const int32_t* ids, void* z0, int batch,
-                          int T, int d, bool bf16, cudaStream_t s);
-// x0[n, t*e + c] = tables[t*table_stride + ids[n*ns+t]*e + c]; x0[n, ns*e + j] = dense[n, j]; pad 0
+                          int T, int d, int vocab, int* status, bool bf16, cudaStream_t s);
+// x0[n, t*e + c] = tables[t*table_stride + ids[n*ns+t]*e + c]; x0[n, ns*e + j] = dense[n, j]; pad 0.
+// ids are checked against [0, table_rows) in the same way.
 cudaError_t gather_ctr(const float* tables, long long table_stride, const int32_t* ids,
                        const float* dense, void* x0, int batch, int ns, int e, int nd, int width,
-                       bool bf16, cudaStream_t s);
+                       int table_rows, int* status, bool bf16, cudaStream_t s);
 
 // Dot interaction.  vectors of sample n: v_0 = proj[n, 0:e], v_j = x0[n, (j-1)e : je], j = 1..ns.
 // feats[n, i(i-1)/2 + j] = v_i . v_j (i > j), then proj[n,:], then zeros up to width fw.

@@ -1,5 +1,8 @@
 """GPU-side test helpers: stage synthetic batches on the device (torch owns the memory) and
 compare the CUDA library with the oracle.  Imported only by tests marked gpu."""
+import json
+import os
+
 import numpy as np
 import torch
 
@@ -7,12 +10,30 @@ from oracle import erase_oracle as orc
 from paper_2608_18469_b200 import binding, synth
 from tests import util
 
-TOL = {"f32": 1e-4, "bf16": 2e-2}     # relative L2 per tensor against the fp64 oracle
-# Optimizer alone (fp64 update rule applied to the library's own gradient vs the fp32 kernel).
-# A tensor that starts at zero (LayerNorm shift) consists of the update only, so its relative
-# error is that of a handful of fp32 operations (m, v, two bias corrections, sqrt, divide):
-# a few 1e-7 each, 2e-6 observed; any formula mistake shows up at 1e-3 or more.
-OPT_TOL = 1e-5
+TOL = {"f32": 1e-4, "bf16": 2e-2}     # relative L2 PER TENSOR against the fp64 oracle
+# Optimizer alone (fp64 update rule applied to the library's own gradient vs the fp32 kernel): a
+# handful of fp32 roundings.  A tensor that starts at zero (LayerNorm shift) consists of the update
+# only, so its relative error is that of the update itself (m, v, two bias corrections, sqrt,
+# divide: a few 1e-7 each, 2e-6 observed); every other tensor is dominated by the parameter.
+OPT_TOL = 2e-6
+OPT_TOL_ZERO_INIT = 1e-5
+
+# bf16 only.  A gradient is a sum over samples; on some instances that sum nearly cancels (a bias
+# gradient on labels drawn independently of the inputs; every gradient of a block right after Adam's
+# first sign step on rare positives), and then no implementation that stores activations in bf16
+# keeps 2e-2 RELATIVE to what is left.  A tensor may exceed 2e-2 only if (a) its (case, step, tensor)
+# is listed in the committed allow-list below, which records the oracle-measured sensitivity of that
+# instance to bf16 storage, and (b) its error stays within a small multiple of the sensitivity
+# measured live, under a fixed cap: biases / LayerNorm shifts 3x and 1e-1, weight matrices 1.5x
+# and 5e-2.  Anything else fails.  The small synthetic cases avoid the list altogether by using
+# seeds on which the instance is well conditioned.
+COND_RULE = {"bias": (3.0, 1e-1), "weight": (1.5, 5e-2)}
+ALLOW_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "bf16_conditioning_allow.json")
+
+
+def _allow_list():
+    with open(ALLOW_PATH) as f:
+        return {(e["case"], e["step"], e["tensor"]): e for e in json.load(f)["entries"]}
 
 
 def oracle_bf16_sensitivity(spec, params, batch):
@@ -68,10 +89,13 @@ def new_model(spec, flat):
     return m
 
 
-def compare_teacher_forced(spec, steps, seed=0, n_streams=2, flags=0, report=None):
+def compare_teacher_forced(spec, steps, seed=0, n_streams=2, flags=0, report=None, case=None):
     """Each step: library and oracle start from the same fp32 parameters and optimizer state;
-    losses and every gradient tensor must agree within TOL; the parameters after the
-    optimizer must match the update rule applied in fp64 to the library's own gradients."""
+    losses and every gradient tensor, each on its own, must agree within TOL; the parameters
+    after the optimizer must match the update rule applied in fp64 to the library's own gradients.
+    `case` names the instance for the bf16 conditioning allow-list (see COND_CAP above); with
+    `report` (a dict) nothing is asserted: worst errors and the list of tensors that would need
+    the allow-list are collected instead."""
     tol = TOL[spec["dtype"]]
     flat = synth.init_params(spec, seed)
     tl = synth.tensor_list(spec)
@@ -79,6 +103,7 @@ def compare_teacher_forced(spec, steps, seed=0, n_streams=2, flags=0, report=Non
     m = new_model(spec, flat)
     params = util.structure(spec, flat)
     state = orc.new_opt_state(params)
+    zero_init = [not np.any(v) for v in flat]      # tensors that consist of optimizer updates only
     worst = {}
     try:
         for it in range(steps):
@@ -114,52 +139,45 @@ def compare_teacher_forced(spec, steps, seed=0, n_streams=2, flags=0, report=Non
                 worst[f"loss{b}"] = max(worst.get(f"loss{b}", 0), err)
                 if report is None:
                     assert err <= tol, (it, "loss", b, got_l[b], want_l[b])
-            # fp32: every tensor on its own.  bf16: every affine map on its own, i.e. a Linear's
-            # weight and bias (or a LayerNorm's gain and shift) are compared as one vector [W | b]:
-            # a bias gradient is a plain sum over samples of the loss gradient and can cancel to
-            # almost nothing on balanced random labels (observed: 6e-4 against a typical 5e-2),
-            # where no bf16 implementation keeps a relative accuracy of its own.
-            groups = {}
             probe = None
             for i in tidx:
                 b, name, _s, _t = tl[i]
                 g = m.grads(i)
                 err = synth.rel_l2(g, want_g[b][name])
-                key = f"grad b{b} {name}"
-                worst[key] = max(worst.get(key, 0), err)
-                if spec["dtype"] == "bf16":
-                    gname = name[:-2] if name.startswith("ln") else name[1:]
-                    gg = groups.setdefault((b, gname), [[], []])
-                    gg[0].append(g.ravel().astype(np.float64))
-                    gg[1].append(want_g[b][name].ravel())
-                elif report is None:
-                    assert err <= tol, (it, key, err)
+                key = f"b{b} {name}"
+                worst[f"grad {key}"] = max(worst.get(f"grad {key}", 0), err)
+                if err > tol:
+                    kind = "weight" if g.ndim == 2 else "bias"
+                    cond, entry = None, None
+                    if spec["dtype"] == "bf16":
+                        if probe is None:
+                            probe = oracle_bf16_sensitivity(spec, util.operand_params(spec, params),
+                                                            util.operand_batch(spec, batch))
+                        cond = synth.rel_l2(probe[b][name], want_g[b][name])
+                        entry = _allow_list().get((case, it, key))
+                    listed = entry is not None and entry["kind"] == kind
+                    mult, cap = COND_RULE[kind]
+                    bound = min(cap, max(tol, mult * cond)) if listed else tol
+                    print(f"[conditioning] case {case} step {it} {key}: err {err:.3e}, oracle bf16 sensitivity "
+                          f"{cond if cond is None else format(cond, '.3e')}, listed {listed}, bound {bound:.3e}")
+                    if report is not None:
+                        report.setdefault("violations", []).append(
+                            {"case": case, "step": it, "tensor": key, "err": float(err),
+                             "sensitivity": None if cond is None else float(cond),
+                             "norm": float(np.linalg.norm(want_g[b][name])), "kind": kind})
+                    else:
+                        assert err <= bound, (case, it, key, err, bound, cond,
+                                              "" if listed else "not in tests/golden/bf16_conditioning_allow.json")
                 # optimizer alone: update rule in fp64 on the library's gradient
                 th, _, _ = orc.optimizer_update(spec["opt"], params["blocks"][b][name], g.astype(np.float64),
                                                 state["m"][b][name], state["v"][b][name], state["t"] + 1)
                 perr = synth.rel_l2(m.params(i), th)
-                key = f"param b{b} {name}"
-                worst[key] = max(worst.get(key, 0), perr)
+                worst[f"param {key}"] = max(worst.get(f"param {key}", 0), perr)
+                ptol = OPT_TOL_ZERO_INIT if zero_init[i] else OPT_TOL
                 if report is None:
-                    assert perr <= OPT_TOL, (it, key, perr)
-            for (b, gname), (got_parts, want_parts) in groups.items():
-                err = synth.rel_l2(np.concatenate(got_parts), np.concatenate(want_parts))
-                key = f"layer b{b} {gname}"
-                worst[key] = max(worst.get(key, 0), err)
-                bound = tol
-                if err > tol:
-                    # ill-conditioned instance?  allow 3x the oracle's own sensitivity to bf16 storage
-                    if probe is None:
-                        probe = oracle_bf16_sensitivity(spec, util.operand_params(spec, params),
-                                                        util.operand_batch(spec, batch))
-                    names = [n for (bb, n, _s2, tr) in tl if tr and bb == b and
-                             (n[:-2] if n.startswith("ln") else n[1:]) == gname]
-                    cond = synth.rel_l2(np.concatenate([probe[b][n].ravel() for n in names]),
-                                        np.concatenate(want_parts))
-                    bound = max(tol, 3.0 * cond)
-                    print(f"[conditioning] step {it} {key}: err {err:.3e}, oracle bf16 sensitivity {cond:.3e}")
-                if report is None:
-                    assert err <= bound, (it, key, err, bound)
+                    assert perr <= ptol, (it, key, perr)
+                else:
+                    worst["param/tol"] = max(worst.get("param/tol", 0), perr / ptol)
             params, state = new_params, new_state
     finally:
         m.close()

@@ -165,3 +165,78 @@ def test_full_size_lm_configs_schedules_agree_and_losses_start_near_ln_vocab():
         # a random head cannot beat the uniform predictor on independent labels, and its logit
         # spread only adds about half its variance to the loss
         assert np.all(serial["losses"] > 0.99 * lnv) and np.all(serial["losses"] < 2.0 * lnv), serial["losses"]
+
+
+def test_an_expired_device_wait_returns_etimeout_and_the_model_stays_usable():
+    """One thread waits, with the bounded-wait helper of the tensor-core kernels and a limit of
+    about a millisecond, on a barrier that nothing signals; the wait runs out by construction.  The
+    next synchronising call reports ERASE_ETIMEOUT, a step enqueued behind the expiry skips its
+    tensor-core work, and after the report the same model steps to the same bits as a fresh one."""
+    import time
+    gu = _gu()
+    spec = _small()
+    flat = synth.init_params(spec, 6)
+    db = gu.DevBatch(spec, synth.make_batch(spec, 6))
+    ref = gu.run_steps(spec, flat, [db], n_streams=3)
+    m = gu.new_model(spec, flat)
+    t0 = time.perf_counter()
+    m.selftest_timeout(limit_us=1000)
+    with pytest.raises(binding.EraseError) as e:
+        m.sync()
+    assert e.value.status == binding.ETIMEOUT and "code 8" in str(e.value)
+    assert time.perf_counter() - t0 < 5.0                      # it returned; nothing hung
+    m.sync()                                                   # the report cleared the status word
+    # an expiry in front of a whole step: every tensor-core kernel of the step finds the word set
+    m.selftest_timeout(limit_us=1000)
+    t0 = time.perf_counter()
+    m.step(n_streams=3, **db.args())
+    with pytest.raises(binding.EraseError) as e:
+        m.losses()
+    assert e.value.status == binding.ETIMEOUT
+    assert time.perf_counter() - t0 < 5.0
+    m.close()
+    # and the context is intact: a fresh model reproduces the reference bits
+    again = gu.run_steps(spec, flat, [db], n_streams=3)
+    for k in ref:
+        if k != "launches":
+            assert ref[k].tobytes() == again[k].tobytes(), k
+    with pytest.raises(binding.EraseError) as e:
+        gu.new_model(spec, flat).selftest_timeout(limit_us=0)
+    assert e.value.status == binding.EINVAL
+
+
+@pytest.mark.parametrize("kind", ["tokens_input", "tokens_last_target", "ctr"])
+def test_an_id_outside_its_table_is_reported_and_never_dereferenced(kind):
+    """The input staging checks every id against its table: a bad id is not used as an index (row 0
+    stands in), the step's results are void and the next synchronising call returns ERASE_EINVAL.
+    The model then runs a clean batch to the same losses as a model that never saw the bad one."""
+    import torch
+    gu = _gu()
+    if kind == "ctr":
+        spec = synth.ctr_spec(batch=64, table_rows=50, tower=(64, 32, 16))
+    else:
+        spec = _small()
+    flat = synth.init_params(spec, 7)
+    good = synth.make_batch(spec, 7)
+    bad = {k: v.copy() for k, v in good.items()}
+    if kind == "ctr":
+        bad["ids"][5, 3] = spec["table_rows"] + 1000000
+        bad["ids"][9, 0] = -7
+    elif kind == "tokens_input":
+        bad["ids"][1, 4] = spec["vocab"]                        # first id past the table
+    else:
+        bad["ids"][0, spec["seq"]] = -1                         # the last column is a target only
+    gdb, bdb = gu.DevBatch(spec, good), gu.DevBatch(spec, bad)
+    ref = gu.new_model(spec, flat)
+    ref.step(n_streams=2, flags=binding.NO_OPT, **gdb.args())
+    want = ref.losses()
+    ref.close()
+    m = gu.new_model(spec, flat)
+    m.step(n_streams=2, flags=binding.NO_OPT, **bdb.args())
+    with pytest.raises(binding.EraseError) as e:
+        m.losses()
+    assert e.value.status == binding.EINVAL and "outside its table" in str(e.value)
+    torch.cuda.synchronize()                                    # no fault was raised on the device
+    m.step(n_streams=2, flags=binding.NO_OPT, **gdb.args())
+    assert m.losses().tobytes() == want.tobytes()
+    m.close()

@@ -114,7 +114,14 @@ def _run(spec, steps, seed=0):
         for b in range(len(tg)):
             for k in tg[b]:
                 assert synth.rel_l2(og[b][k], tg[b][k]) < 1e-10, (it, b, k)
-                assert synth.rel_l2(params["blocks"][b][k], tparams[b][k].detach().numpy()) < 1e-9, (it, b, k)
+                # Parameters agree to 1e-12, plus what the optimizer makes of the (<= 1e-10) difference
+                # between the two gradients: Adam's update lr*m^/(sqrt(v^)+eps) has slope up to lr/eps
+                # where the gradient is mathematically zero and both sides hold rounding noise of
+                # ~1e-17 (the key bias of attention: softmax does not see it); SGD's slope is lr.
+                want = tparams[b][k].detach().numpy()
+                slope = o["lr"] if o["kind"] == "sgd" else o["lr"] / o["eps"]
+                bound = 1e-12 * np.linalg.norm(want) + 2.0 * slope * np.linalg.norm(og[b][k] - tg[b][k])
+                assert np.linalg.norm(params["blocks"][b][k] - want) <= bound, (it, b, k)
 
 
 @pytest.mark.parametrize("name", list(util.tiny_specs()))
