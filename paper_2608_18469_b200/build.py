@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liberase_b200.so")
-SOURCES = ["erase.cu", "kernels.cu", "gemm_tc.cu", "gemm_noalloc.cu", "attention_mma.cu"]
+SOURCES = ["erase.cu", "kernels.cu", "gemm_tc.cu", "gemm_noalloc.cu", "attention_mma.cu", "attention_tc.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 

@@ -464,6 +464,12 @@ __global__ void __launch_bounds__(256) attn_delta_mma(const bf16_t* __restrict__
 
 bool attention_mma_supported(int dh, int d) { return dh == DH && d % 8 == 0; }
 
+cudaError_t attention_delta_bf16(const void* o, const void* dout, float* delta, int batch, int T, int heads, cudaStream_t s) {
+  const long long rows = (long long)batch * T;
+  attn_delta_mma<<<(unsigned)((rows * heads + 7) / 8), 256, 0, s>>>((const bf16_t*)o, (const bf16_t*)dout, delta, rows, T, heads);
+  return cudaGetLastError();
+}
+
 cudaError_t attention_fwd_mma(const void* qkv, void* o, float* lse, int batch, int T, int heads, cudaStream_t s) {
   dim3 grid((T + TS - 1) / TS, heads, batch);
   attn_fwd_mma<<<grid, 128, 0, s>>>((const bf16_t*)qkv, (bf16_t*)o, lse, T, heads, 0.125f);

@@ -642,6 +642,14 @@ struct Builder {
     } else {
       int V = k.head_out, T_ = m->spec.seq;
       void* logits = act_buf((size_t)rows * V);
+      if (head_ce_exp(b, z, d, wh, bh, logits, V, T_, rowloss, loss_out, inv, f, bw, dz)) {
+        if (dact != ACT_NONE) {
+          long long n = (long long)rows * d;
+          bw.push_back({[=](cudaStream_t s) { return ew_dact(dz, dact_src, dact, n, bf, s); }, 1});
+          note(bw, "ew_dact", (double)n, 3.0 * n * m->esz);
+        }
+        return false;
+      }
       lin_fwd(f, z, d, wh, bh, logits, rows, V, d, Epilogue());
       const int ce_fused = getenv("ERASE_CE_FUSED") ? atoi(getenv("ERASE_CE_FUSED")) : 1;   // 0 never, 1 by size, 2 whenever supported
       // worth it when the gradient matrix is far larger than L2 (C4: 1 GB; 346 + 27 us against 322 + 97 us);
@@ -669,6 +677,109 @@ struct Builder {
       }
       return false;
     }
+  }
+
+  // ---- softmax cross-entropy head whose loss and gradient never read the logits back ------------
+  // (bf16 models whose head GEMM runs on the tensor cores; the kernels are described in kernels.cu).
+  // Forward: target logit -> head GEMM with the exp epilogue (P and partial sums) -> finalize ->
+  // exact recomputation of unsafe rows (normally none) -> mean loss.  Backward: dW_h and db_h from
+  // P and the scaled copy of z, the one-hot part added in row order, dz from P W_h.
+  // Returns false (nothing enqueued) when the head does not qualify: the caller then takes the
+  // path with a separate softmax pass.
+  bool head_ce_exp(int /*b*/, const void* z, int d, int wh, int bh, void* logits, int V, int T_, float* rowloss, float* loss_out,
+                   float inv, OpList& f, OpList& bw, void* dz) {
+    const int ce_mode = getenv("ERASE_CE_MODE") ? atoi(getenv("ERASE_CE_MODE")) : 1;   // 0: separate softmax pass
+    erase_model* mm = m;
+    const int rows = m->rows;
+    if (!ce_mode || !m->bf16 || V % 8 || d % 8 || V < 16 || d < 64) return false;
+    GemmArgs g;
+    g.M = rows; g.N = V; g.K = d;
+    g.A = z; g.sa_m = d; g.sa_k = 1;
+    g.B = Wop(wh); g.sb_n = d; g.sb_k = 1;
+    g.C = logits; g.ldc = V;
+    g.epi.bias = Wf(bh);
+    g.epi.ld_aux = V;
+    if (!tc_gemm_supported(g)) return false;
+    // partial sums: one per row and group of columns; the group width (64..128) follows the tile
+    // choice, which is only known with real pointers, so the buffer is sized for the narrowest
+    const int max_groups = (V + 63) / 64;
+    float* psum = f32_buf((size_t)rows * max_groups);
+    float* ref = f32_buf(rows);
+    float* lt = f32_buf(rows);
+    float* rowscale = f32_buf(rows);
+    int* tgt = (int*)dev_alloc(m, (size_t)rows * sizeof(int), &ok);
+    int* bad = (int*)dev_alloc(m, (size_t)(rows + 1) * sizeof(int), &ok);
+    void* zs = act_buf((size_t)rows * d);
+    g.epi.ce_ref = ref;
+    g.epi.ce_psum = psum;
+    TcPlan plan;
+    int* sched = (int*)dev_alloc(m, 2 * sizeof(int), &ok);
+    int groups = max_groups;
+    if (!m->dry) {
+      if (!tc_gemm_plan(g, m->status, &plan)) { ok = false; return true; }
+      plan.sched = sched;
+      if (!plan.tma_c) { ok = false; return true; }
+      const int gc = tc_ce_group_cols(plan);
+      groups = (V + gc - 1) / gc;
+      g.epi.ce_groups = groups;
+    }
+    const void* Wb = Wop(wh);
+    const float* bias = Wf(bh);
+    f.push_back({[=](cudaStream_t s) { return ce_target_logit(z, Wb, bias, mm->cur.ids, T_, rows, d, V, tgt, ref, lt, bad, s); }, 1});
+    note(f, "ce_target_logit", 2.0 * rows * d, 4.0 * rows * d);
+    f.push_back({[g, plan, mm](cudaStream_t s) { return tc_gemm_launch(g, plan, s, mm->sm_budget); }, 1});
+    note(f, "gemm_fwd", 2.0 * rows * V * d, ((double)rows * d + (double)V * d) * 2 + 2.0 * rows * V);
+    f.push_back({[=](cudaStream_t s) { return ce_finalize(psum, groups, ref, lt, z, zs, rowloss, rowscale, bad, rows, d, inv, s); }, 1});
+    note(f, "ce_finalize", (double)rows * groups, 4.0 * rows * groups + 4.0 * rows * d);
+    f.push_back({[=](cudaStream_t s) { return ce_fixup(bad, mm->status, z, Wb, bias, logits, ref, lt, zs, rowloss, rowscale, rows, d, V, inv, s); }, 1});
+    note(f, "ce_fixup", 0, 0);
+    f.push_back({[=](cudaStream_t s) { return reduce_sum(rowloss, rows, inv, loss_out, s); }, 1});
+    note(f, "loss_reduce", rows, 4.0 * rows);
+    // backward: parameter gradients (leaves) ...
+    const size_t before = bw.size();
+    lin_wgrad(bw, logits, zs, d, wh, -1, rows, V, d, true);
+    flush_group(bw);           // a small head's weight gradient may have joined a group: the one-hot part follows it
+    {
+      const int chunks = colsum_chunks(rows, V);
+      float* ws = chunks > 1 ? f32_buf((size_t)chunks * V) : nullptr;
+      float* out = G(bh);
+      int* tk = tickets(V);
+      bw.push_back({[=](cudaStream_t s) { return colsum(logits, true, V, rows, V, rowscale, ws, chunks, tk, out, s); }, 1});
+      note(bw, "colsum", 2.0 * rows * V, 2.0 * rows * V);
+    }
+    float* dW = G(wh);
+    float* db = G(bh);
+    bw.push_back({[=](cudaStream_t s) { return ce_onehot(tgt, z, dW, db, rows, d, V, inv, s); }, 1});
+    note(bw, "ce_onehot", 2.0 * rows * d, 4.0 * rows + 2.0 * rows * d);
+    for (size_t i = before; i < bw.size(); i++) bw[i].leaf = true;
+    // ... and the gradient chain: dz = r (.) (P W_h) - W_h[t]/N from fp32 partials of the GEMM
+    GemmArgs q;
+    q.M = rows; q.N = d; q.K = V;
+    q.A = logits; q.sa_m = V; q.sa_k = 1;
+    q.B = Wop(wh); q.sb_n = 1; q.sb_k = d;
+    q.c_f32 = 1;
+    q.epi.ld_aux = d;
+    int splits = 1;
+    if (rows >= 256 && d >= 256 && V >= 2048) {   // few output tiles, long contraction: split it over the CTA pairs
+      const long long pair_tiles = (long long)((rows + 255) / 256) * ((d + 255) / 256);
+      splits = (int)std::min<long long>(std::min<long long>(74 / pair_tiles, V / 1024), 8);
+      if (splits < 1) splits = 1;
+    }
+    float* part = f32_buf((size_t)splits * rows * d);
+    q.splits = splits;
+    if (splits > 1) { q.ws = part; q.C = part; q.ldc = d; }
+    else { q.C = part; q.ldc = d; }
+    TcPlan qplan;
+    int* qsched = (int*)dev_alloc(m, 2 * sizeof(int), &ok);
+    const bool q_tc = !m->dry && tc_gemm_supported(q) && tc_gemm_plan(q, m->status, &qplan);
+    qplan.sched = qsched;
+    bw.push_back({[=](cudaStream_t s) {
+                    cudaError_t e = q_tc ? tc_gemm_launch(q, qplan, s, mm->sm_budget) : gemm_simt(q, true, s);
+                    if (e != cudaSuccess) return e;
+                    return ce_dz_finish(part, splits, rows, d, rowscale, tgt, Wb, dz, inv, s);
+                  }, 2});
+    note(bw, "gemm_dgrad", 2.0 * rows * V * d, ((double)rows * V + (double)V * d) * 2 + 2.0 * rows * d);
+    return true;
   }
 
   // ---- Linear stack (MLP / TOWER / tower of the DOT block) ---------------------------------
@@ -752,6 +863,7 @@ struct Builder {
     const int d = k.dims[0], ff = k.dims[1], H = k.n_heads, dh = d / H;
     const int rows = m->rows, batch = m->spec.batch, T_ = m->spec.seq;
     const bool bf = m->bf16;
+    erase_model* mm = m;
     enum { LN1G = 0, LN1B, WQKV, BQKV, WPROJ, BPROJ, LN2G, LN2B, W1, B1, W2, B2, WH, BH };
     auto t = [&](int i) { return first + i; };
     // forward
@@ -771,7 +883,7 @@ struct Builder {
       f.push_back({[=](cudaStream_t s) { return layernorm_fwd(z, g1, b1, a, mean1, rstd1, rows, d, bf, s); }, 1});
       note(f, "layernorm_fwd", 8.0 * rows * d, 2.0 * rows * d * m->esz);
       lin_fwd(f, a, d, t(WQKV), t(BQKV), qkv, rows, 3 * d, d, Epilogue());
-      f.push_back({[=](cudaStream_t s) { return attention_fwd(qkv, o, lse, batch, T_, H, dh, bf, s); }, 1});
+      f.push_back({[=](cudaStream_t s) { return attention_fwd(qkv, o, lse, batch, T_, H, dh, bf, s, mm->status); }, 1});
       note(f, "attention_fwd", 4.0 * batch * H * ((double)T_ * (T_ + 1) / 2) * dh, 4.0 * rows * d * m->esz);
       Epilogue e1; e1.res = z;
       lin_fwd(f, o, d, t(WPROJ), t(BPROJ), h, rows, d, d, e1);
@@ -804,7 +916,7 @@ struct Builder {
       mid_flush(bw);   // (off by default) b2, b1, LN2 half-way; the rest (bproj, bqkv, LN1) at the end of B_b
       lin_wgrad(bw, dhb, o, d, t(WPROJ), t(BPROJ), rows, d, d);
       lin_dgrad(bw, dhb, t(WPROJ), dO, rows, d, d, Epilogue());
-      bw.push_back({[=](cudaStream_t s) { return attention_bwd(qkv, o, dO, lse, delta, dqkv, batch, T_, H, dh, bf, s); }, 3});
+      bw.push_back({[=](cudaStream_t s) { return attention_bwd(qkv, o, dO, lse, delta, dqkv, batch, T_, H, dh, bf, s, mm->status); }, 3});
       note(bw, "attention_bwd", 8.0 * batch * H * ((double)T_ * (T_ + 1) / 2) * dh, 8.0 * rows * d * m->esz);
       lin_wgrad(bw, dqkv, a, d, t(WQKV), t(BQKV), rows, 3 * d, d);
       lin_dgrad(bw, dqkv, t(WQKV), da, rows, 3 * d, d, Epilogue());

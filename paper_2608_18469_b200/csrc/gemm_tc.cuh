@@ -54,6 +54,11 @@ struct TcGroupPlan {
 bool tc_wgrad_group_plan(const GemmArgs* gs, int n, int* status, TcGroupPlan* plan);
 cudaError_t tc_wgrad_group_launch(const TcGroupPlan& plan, cudaStream_t s, int max_ctas = 0);
 
+// TMA descriptor (128 bytes, a CUtensorMap) of a row-major bf16 matrix with `inner` contiguous
+// elements per row and `outer` rows `ld` elements apart: tiles of 64 columns x box_rows rows,
+// 128-byte swizzle, zero fill outside.  False if the layout cannot be described (alignment).
+bool tc_encode_rows_bf16(void* map128, const void* base, long long inner, long long outer, long long ld, int box_rows);
+
 // Launches one thread that waits, for at most limit_cycles SM clocks, on a barrier nothing signals,
 // then sets *status to 8 and returns: the bounded-wait helper of the GEMM kernels on its own.
 cudaError_t tc_wait_selftest(int* status, long long limit_cycles, cudaStream_t s);

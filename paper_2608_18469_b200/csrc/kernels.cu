@@ -21,6 +21,15 @@ template <> __device__ __forceinline__ float ldf<bf16_t>(const bf16_t* p) { retu
 template <typename T> __device__ __forceinline__ void stf(T* p, float v);
 template <> __device__ __forceinline__ void stf<float>(float* p, float v) { *p = v; }
 template <> __device__ __forceinline__ void stf<bf16_t>(bf16_t* p, float v) { *p = __float2bfloat16_rn(v); }
+// four consecutive values (p 16-byte aligned for float, 8-byte for bf16)
+__device__ __forceinline__ void store4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+__device__ __forceinline__ void store4(bf16_t* p, float4 v) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+  uint2 q;
+  q.x = *reinterpret_cast<uint32_t*>(&lo);
+  q.y = *reinterpret_cast<uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(p) = q;
+}
 
 __device__ __forceinline__ float act_apply(int act, float v) {
   if (act == ACT_RELU) return v > 0.f ? v : 0.f;
@@ -1047,9 +1056,14 @@ static cudaError_t attention_fwd_t(const T* qkv, T* o, float* lse, int batch, in
   return cudaGetLastError();
 }
 
+// 0: fp32 SIMT / mma.sync kernels only; 1 (default): tcgen05 kernels where they apply
+static int attention_tc_mode() { return getenv("ERASE_ATTN_TC") ? atoi(getenv("ERASE_ATTN_TC")) : 1; }
+
 cudaError_t attention_fwd(const void* qkv, void* o, float* lse, int batch, int T_, int heads, int dh,
-                          bool bf16, cudaStream_t s) {
+                          bool bf16, cudaStream_t s, int* status) {
   if (dh > 32 * ATT_MAXC) return cudaErrorInvalidValue;
+  if (bf16 && attention_tc_mode() && attention_tc_supported(dh, heads * dh, qkv, o))
+    return attention_fwd_tc(qkv, o, lse, batch, T_, heads, status, s);
   if (bf16 && attention_mma_supported(dh, heads * dh)) return attention_fwd_mma(qkv, o, lse, batch, T_, heads, s);
   return bf16 ? attention_fwd_t<bf16_t>((const bf16_t*)qkv, (bf16_t*)o, lse, batch, T_, heads, dh, s)
               : attention_fwd_t<float>((const float*)qkv, (float*)o, lse, batch, T_, heads, dh, s);
@@ -1074,8 +1088,13 @@ static cudaError_t attention_bwd_t(const T* qkv, const T* o, const T* dout, cons
 }
 
 cudaError_t attention_bwd(const void* qkv, const void* o, const void* dout, const float* lse, float* delta,
-                          void* dqkv, int batch, int T_, int heads, int dh, bool bf16, cudaStream_t s) {
+                          void* dqkv, int batch, int T_, int heads, int dh, bool bf16, cudaStream_t s, int* status) {
   if (dh > 32 * ATT_MAXC) return cudaErrorInvalidValue;
+  if (bf16 && attention_tc_mode() && attention_tc_supported(dh, heads * dh, qkv, dout) && (reinterpret_cast<uintptr_t>(dqkv) & 15) == 0) {
+    cudaError_t e = attention_delta_bf16(o, dout, delta, batch, T_, heads, s);
+    if (e != cudaSuccess) return e;
+    return attention_bwd_tc(qkv, dout, lse, delta, dqkv, batch, T_, heads, status, s);
+  }
   if (bf16 && attention_mma_supported(dh, heads * dh)) return attention_bwd_mma(qkv, o, dout, lse, delta, dqkv, batch, T_, heads, s);
   return bf16 ? attention_bwd_t<bf16_t>((const bf16_t*)qkv, (const bf16_t*)o, (const bf16_t*)dout, lse, delta, (bf16_t*)dqkv, batch, T_, heads, dh, s)
               : attention_bwd_t<float>((const float*)qkv, (const float*)o, (const float*)dout, lse, delta, (float*)dqkv, batch, T_, heads, dh, s);
@@ -1442,6 +1461,333 @@ cudaError_t softmax_ce_inplace(void* logits, const int32_t* ids, int T_, float* 
   return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------------------------------
+// Softmax cross-entropy head without a pass over the logits (bf16 models, tensor-core head GEMM).
+//
+// With a per-row reference c_n known BEFORE the head GEMM, the GEMM's epilogue stores
+// P[n,v] = exp(l[n,v] - c_n) (bf16) instead of the logit and leaves fp32 partial sums of the
+// unrounded exponentials.  Then, with S_n = sum_v exp(l[n,v] - c_n):
+//     lse_n = c_n + log S_n,      loss_n = lse_n - l[n,t_n],
+//     dl[n,v] = (softmax - onehot)/N = P[n,v] * r_n - [v = t_n]/N,     r_n = 1 / (S_n N),
+// so the backward GEMMs consume P directly:
+//     dW_h = P^T (r (.) z)  -  (1/N) sum_n onehot(t_n) z_n^T        (rows of z added to rows t_n)
+//     dz_n = r_n (P W_h)_n  -  (1/N) W_h[t_n, :]
+//     db_h = sum_n r_n P[n,:]  -  count(t = v)/N.
+// c_n is the target's own logit (z_n . W_h[t_n] + b_h[t_n], a gather and a dot product): it is at
+// most the row maximum, and it is far enough below it to endanger the exponent range only when the
+// token's loss exceeds ~69 nats.  Such rows (S_n >= 1e30 or not finite) are listed by the finalize
+// kernel and recomputed exactly, with c_n = the true row maximum, by ce_fixup_kernel, which does
+// nothing when the list is empty.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ float dot8_bf16(uint4 a, uint4 b) {
+  const uint32_t x[4] = {a.x, a.y, a.z, a.w}, y[4] = {b.x, b.y, b.z, b.w};
+  float acc = 0.f;
+#pragma unroll
+  for (int j = 0; j < 4; j++) {
+    acc = fmaf(__uint_as_float(x[j] << 16), __uint_as_float(y[j] << 16), acc);
+    acc = fmaf(__uint_as_float(x[j] & 0xffff0000u), __uint_as_float(y[j] & 0xffff0000u), acc);
+  }
+  return acc;
+}
+
+// One warp per row: tgt[n] (clamped into the vocabulary; a bad id was already reported by the
+// input staging), ref[n] = lt[n] = z_n . W[t_n] + b[t_n].  Thread 0 of the launch clears the
+// list of rows to recompute.  d % 8 == 0.
+__global__ void __launch_bounds__(256) ce_target_logit_kernel(const bf16_t* __restrict__ z, const bf16_t* __restrict__ W,
+                                                              const float* __restrict__ bias, const int32_t* __restrict__ ids,
+                                                              int T_, int rows, int d, int V, int* __restrict__ tgt,
+                                                              float* __restrict__ ref, float* __restrict__ lt, int* __restrict__ bad) {
+  if (blockIdx.x == 0 && threadIdx.x == 0) bad[0] = 0;
+  const int lane = threadIdx.x & 31;
+  for (int n = blockIdx.x * 8 + (threadIdx.x >> 5); n < rows; n += gridDim.x * 8) {
+    const int t = min(max(ids[(long long)(n / T_) * (T_ + 1) + (n % T_) + 1], 0), V - 1);
+    const uint4* zr = reinterpret_cast<const uint4*>(z + (long long)n * d);
+    const uint4* wr = reinterpret_cast<const uint4*>(W + (long long)t * d);
+    float acc = 0.f;
+    for (int i = lane; i < (d >> 3); i += 32) acc += dot8_bf16(__ldg(zr + i), __ldg(wr + i));
+    acc = warp_sum(acc);
+    if (lane == 0) {
+      const float l = acc + bias[t];
+      tgt[n] = t;
+      ref[n] = l;
+      lt[n] = l;
+    }
+  }
+}
+
+__device__ __forceinline__ void scale_row_bf16(const bf16_t* __restrict__ z, bf16_t* __restrict__ zs, int d, float r, int lane) {
+  const uint4* src = reinterpret_cast<const uint4*>(z);
+  uint4* dst = reinterpret_cast<uint4*>(zs);
+  for (int i = lane; i < (d >> 3); i += 32) {
+    const uint4 q = src[i];
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+      __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(w[j] << 16) * r, __uint_as_float(w[j] & 0xffff0000u) * r);
+      o[j] = *reinterpret_cast<uint32_t*>(&h);
+    }
+    dst[i] = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
+// One warp per row: S_n from the GEMM's partial sums (lanes stride over the groups, then a fixed
+// shuffle tree), loss_n, r_n, the scaled copy r_n z_n for the weight-gradient GEMM; rows whose sum
+// left the safe range are appended to the list bad[1..] (count in bad[0]).
+__global__ void __launch_bounds__(256) ce_finalize_kernel(const float* __restrict__ psum, int groups, const float* __restrict__ ref,
+                                                          const float* __restrict__ lt, const bf16_t* __restrict__ z,
+                                                          bf16_t* __restrict__ zs, float* __restrict__ rowloss,
+                                                          float* __restrict__ rowscale, int* __restrict__ bad, int rows, int d,
+                                                          float inv_rows) {
+  const int lane = threadIdx.x & 31;
+  for (int n = blockIdx.x * 8 + (threadIdx.x >> 5); n < rows; n += gridDim.x * 8) {
+    const float* ps = psum + (long long)n * groups;
+    float S = 0.f;
+    for (int g = lane; g < groups; g += 32) S += ps[g];
+    S = warp_sum(S);
+    const bool ok = S < 1e30f && S > 0.f;      // false for inf and NaN too
+    const float r = ok ? inv_rows / S : 0.f;
+    if (lane == 0) {
+      rowloss[n] = ok ? ref[n] + logf(S) - lt[n] : 0.f;
+      rowscale[n] = r;
+      if (!ok) bad[1 + atomicAdd(bad, 1)] = n;
+    }
+    scale_row_bf16(z + (long long)n * d, zs + (long long)n * d, d, r, lane);
+  }
+}
+
+// Rows listed by the finalize kernel, one CTA per row at a time: the logits of the row are
+// recomputed from z_n and the head's operands (twice: maximum, then exponentials), P[n,:] is
+// rewritten relative to the true maximum, and loss_n, r_n and the scaled copy of z_n follow.
+// Every quantity of a row depends on that row alone, so the order of the list does not matter.
+__global__ void __launch_bounds__(256) ce_fixup_kernel(const int* __restrict__ bad, const int* __restrict__ status, const bf16_t* __restrict__ z,
+                                                       const bf16_t* __restrict__ W, const float* __restrict__ bias,
+                                                       bf16_t* __restrict__ P, float* __restrict__ ref, const float* __restrict__ lt,
+                                                       bf16_t* __restrict__ zs, float* __restrict__ rowloss,
+                                                       float* __restrict__ rowscale, int d, int V, float inv_rows) {
+  __shared__ float red[8];
+  if (status && *status != 0) return;      // the step is already void (an expired wait, a bad id): its sums mean nothing
+  const int nbad = bad[0];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int i = blockIdx.x; i < nbad; i += gridDim.x) {
+    const int n = bad[1 + i];
+    const uint4* zr = reinterpret_cast<const uint4*>(z + (long long)n * d);
+    auto logit = [&](int v) {
+      const uint4* wr = reinterpret_cast<const uint4*>(W + (long long)v * d);
+      float acc = 0.f;
+      for (int k = lane; k < (d >> 3); k += 32) acc += dot8_bf16(__ldg(zr + k), __ldg(wr + k));
+      return warp_sum(acc) + bias[v];
+    };
+    float mx = -INFINITY;
+    for (int v = warp; v < V; v += 8) mx = fmaxf(mx, logit(v));
+    __syncthreads();
+    if (lane == 0) red[warp] = mx;
+    __syncthreads();
+    mx = red[0];
+#pragma unroll
+    for (int w = 1; w < 8; w++) mx = fmaxf(mx, red[w]);
+    float S = 0.f;
+    for (int v = warp; v < V; v += 8) {
+      const float e = expf(logit(v) - mx);
+      S += e;
+      if (lane == 0) P[(long long)n * V + v] = __float2bfloat16_rn(e);
+    }
+    __syncthreads();
+    if (lane == 0) red[warp] = S;
+    __syncthreads();
+    S = red[0];
+#pragma unroll
+    for (int w = 1; w < 8; w++) S += red[w];
+    const float r = inv_rows / S;
+    if (threadIdx.x == 0) {
+      ref[n] = mx;
+      rowloss[n] = mx + logf(S) - lt[n];
+      rowscale[n] = r;
+    }
+    if (warp == 0) scale_row_bf16(z + (long long)n * d, zs + (long long)n * d, d, r, lane);
+    __syncthreads();
+  }
+}
+
+// dz[n,c] = r_n * sum_s part[s][n,c] - W[t_n,c]/N   (partials in split order; rounded to bf16 once)
+__global__ void __launch_bounds__(256) ce_dz_finish_kernel(const float4* __restrict__ part, int splits, long long mn4, int d4,
+                                                           const float* __restrict__ rowscale, const int* __restrict__ tgt,
+                                                           const bf16_t* __restrict__ W, bf16_t* __restrict__ dz, float inv_rows) {
+  const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (i >= mn4) return;
+  const int n = (int)(i / d4), c = (int)(i - (long long)n * d4) * 4;
+  float4 a = part[i];
+  for (int s = 1; s < splits; s++) {
+    const float4 b = part[(long long)s * mn4 + i];
+    a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+  }
+  const float r = rowscale[n];
+  const uint2 wq = *reinterpret_cast<const uint2*>(W + (long long)tgt[n] * (d4 * 4) + c);
+  const float w0 = __uint_as_float(wq.x << 16), w1 = __uint_as_float(wq.x & 0xffff0000u);
+  const float w2 = __uint_as_float(wq.y << 16), w3 = __uint_as_float(wq.y & 0xffff0000u);
+  store4(dz + (long long)n * (d4 * 4) + c,
+         make_float4(fmaf(a.x, r, -inv_rows * w0), fmaf(a.y, r, -inv_rows * w1), fmaf(a.z, r, -inv_rows * w2), fmaf(a.w, r, -inv_rows * w3)));
+}
+
+// The one-hot part of the head's gradients: dW[t_n,:] -= z_n/N and db[t_n] -= 1/N for every row n.
+// A CTA owns 32 vocabulary rows.  Each of its 8 warps scans one eighth of the targets (in row order,
+// no block-wide synchronisation) and keeps the rows that hit the CTA's range in its own list; the
+// eight lists read one after the other are in row order.  Then each warp takes four of the
+// vocabulary rows and, for each, adds up the listed rows of z in that order in registers (the loads
+// are independent of one another) and updates dW once.  Rows of z that meet in one vocabulary row
+// are therefore always added in the same order: no atomics, the same bits on every run.  If a list
+// overflows (many rows share few targets) the CTA falls back to a block-wide ordered compaction
+// that works its list off whenever it fills up.
+constexpr int CE_SUB = 120;       // entries per warp list (fast path)
+constexpr int CE_LIST = 8 * CE_SUB;
+__global__ void __launch_bounds__(256) ce_onehot_kernel(const int* __restrict__ tgt, const bf16_t* __restrict__ z, float* __restrict__ dW,
+                                                        float* __restrict__ db, int rows, int d, float inv_rows) {
+  __shared__ int list[CE_LIST];     // row index * 32 + (target - v0)
+  __shared__ int wcount[8];
+  __shared__ int fill;
+  const int v0 = blockIdx.x * 32;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  // adds the rows listed in list[w * stride .. w * stride + counts[w]) for w = 0..nl-1 (in that order) to this warp's four vocabulary rows
+  auto work_off = [&](int nl, int stride, const int* counts) {
+    for (int i = 0; i < 4; i++) {
+      const int local = warp * 4 + i, v = v0 + local;
+      int hits = 0;
+      for (int c0 = lane * 8; c0 < d || c0 == lane * 8; c0 += 256) {      // every lane runs once (it counts the hits), d % 8 == 0
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        hits = 0;
+        for (int w = 0; w < nl; w++)
+          for (int k = 0; k < counts[w]; k++) {
+            const int e = list[w * stride + k];
+            if ((e & 31) != local) continue;
+            hits++;
+            if (c0 >= d) continue;
+            const uint4 q = __ldg(reinterpret_cast<const uint4*>(z + (long long)(e >> 5) * d + c0));
+            const uint32_t x[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+            for (int j = 0; j < 4; j++) {
+              acc[2 * j] += __uint_as_float(x[j] << 16);
+              acc[2 * j + 1] += __uint_as_float(x[j] & 0xffff0000u);
+            }
+          }
+        if (hits && c0 < d) {
+          float4* dst = reinterpret_cast<float4*>(dW + (long long)v * d + c0);
+          float4 a = dst[0], b = dst[1];
+          a.x -= inv_rows * acc[0]; a.y -= inv_rows * acc[1]; a.z -= inv_rows * acc[2]; a.w -= inv_rows * acc[3];
+          b.x -= inv_rows * acc[4]; b.y -= inv_rows * acc[5]; b.z -= inv_rows * acc[6]; b.w -= inv_rows * acc[7];
+          dst[0] = a; dst[1] = b;
+        }
+      }
+      if (lane == 0 && hits) db[v] -= inv_rows * (float)hits;
+    }
+  };
+  // fast path: every warp compacts its own eighth of the rows, 128 targets per step (one 16-byte
+  // load per lane, two steps in flight), written to the list in row order (lane-major, then the
+  // four components) through a warp prefix sum of the per-lane hit counts
+  {
+    const int per = ((rows + 7) / 8 + 127) / 128 * 128, lo = warp * per, hi = min(rows, lo + per);
+    const int4* t4 = reinterpret_cast<const int4*>(tgt);
+    int cnt = 0;
+    bool over = false;
+    auto fetch = [&](int base) {
+      const int n0 = base + 4 * lane;
+      return n0 < hi ? __ldg(t4 + (n0 >> 2)) : make_int4(-1, -1, -1, -1);    // tgt is padded to a multiple of 64 entries
+    };
+    auto take = [&](int base, int4 q) {
+      const int n0 = base + 4 * lane;
+      const int t[4] = {q.x, q.y, q.z, q.w};
+      bool hit[4];
+      int mine = 0;
+#pragma unroll
+      for (int j = 0; j < 4; j++) {
+        hit[j] = n0 + j < hi && t[j] >= v0 && t[j] < v0 + 32;
+        mine += hit[j];
+      }
+      int incl = mine;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+      }
+      const int total = __shfl_sync(0xffffffffu, incl, 31);
+      if (cnt + total > CE_SUB) { over = true; return; }
+      int pos = warp * CE_SUB + cnt + incl - mine;
+#pragma unroll
+      for (int j = 0; j < 4; j++)
+        if (hit[j]) list[pos++] = (n0 + j) * 32 + (t[j] - v0);
+      cnt += total;
+    };
+    for (int base = lo; base < hi && !over; base += 256) {
+      const int4 qa = fetch(base), qb = fetch(base + 128);
+      take(base, qa);
+      if (!over && base + 128 < hi) take(base + 128, qb);
+    }
+    if (lane == 0) wcount[warp] = cnt;
+    if (!__syncthreads_or(over)) {
+      work_off(8, CE_SUB, wcount);
+      return;
+    }
+  }
+  // slow path: block-wide ordered compaction, 256 targets at a time, worked off when the list fills up
+  __syncthreads();
+  if (threadIdx.x == 0) fill = 0;
+  __syncthreads();
+  for (int base = 0; base < rows; base += 256) {
+    const int n = base + threadIdx.x;
+    const int t = n < rows ? tgt[n] : -1;
+    const bool hit = t >= v0 && t < v0 + 32;
+    const unsigned m = __ballot_sync(0xffffffffu, hit);
+    if (lane == 0) wcount[warp] = __popc(m);
+    __syncthreads();
+    int off = fill, total = 0;
+#pragma unroll
+    for (int w = 0; w < 8; w++) {
+      if (w < warp) off += wcount[w];
+      total += wcount[w];
+    }
+    if (hit) list[off + __popc(m & ((1u << lane) - 1u))] = n * 32 + (t - v0);
+    __syncthreads();
+    if (threadIdx.x == 0) fill += total;
+    __syncthreads();
+    if (fill > CE_LIST - 256 || base + 256 >= rows) {      // the next 256 targets might not fit, or these were the last
+      work_off(1, 0, &fill);
+      __syncthreads();
+      if (threadIdx.x == 0) fill = 0;
+      __syncthreads();
+    }
+  }
+}
+
+cudaError_t ce_target_logit(const void* z, const void* W, const float* bias, const int32_t* ids, int T_, int rows, int d, int V,
+                            int* tgt, float* ref, float* lt, int* bad, cudaStream_t s) {
+  const int grid = (int)std::min<long long>(cdiv(rows, 8), 148 * 8);
+  ce_target_logit_kernel<<<grid, 256, 0, s>>>((const bf16_t*)z, (const bf16_t*)W, bias, ids, T_, rows, d, V, tgt, ref, lt, bad);
+  return cudaGetLastError();
+}
+cudaError_t ce_finalize(const float* psum, int groups, const float* ref, const float* lt, const void* z, void* zs, float* rowloss,
+                        float* rowscale, int* bad, int rows, int d, float inv_rows, cudaStream_t s) {
+  const int grid = (int)std::min<long long>(cdiv(rows, 8), 148 * 8);
+  ce_finalize_kernel<<<grid, 256, 0, s>>>(psum, groups, ref, lt, (const bf16_t*)z, (bf16_t*)zs, rowloss, rowscale, bad, rows, d, inv_rows);
+  return cudaGetLastError();
+}
+cudaError_t ce_fixup(const int* bad, const int* status, const void* z, const void* W, const float* bias, void* P, float* ref, const float* lt, void* zs,
+                     float* rowloss, float* rowscale, int rows, int d, int V, float inv_rows, cudaStream_t s) {
+  const int grid = rows < 32 ? rows : 32;
+  ce_fixup_kernel<<<grid, 256, 0, s>>>(bad, status, (const bf16_t*)z, (const bf16_t*)W, bias, (bf16_t*)P, ref, lt, (bf16_t*)zs, rowloss, rowscale,
+                                       d, V, inv_rows);
+  return cudaGetLastError();
+}
+cudaError_t ce_dz_finish(const float* part, int splits, int rows, int d, const float* rowscale, const int* tgt, const void* W,
+                         void* dz, float inv_rows, cudaStream_t s) {
+  const long long mn4 = (long long)rows * d / 4;
+  ce_dz_finish_kernel<<<cdiv(mn4, 256), 256, 0, s>>>((const float4*)part, splits, mn4, d / 4, rowscale, tgt, (const bf16_t*)W,
+                                                    (bf16_t*)dz, inv_rows);
+  return cudaGetLastError();
+}
+cudaError_t ce_onehot(const int* tgt, const void* z, float* dW, float* db, int rows, int d, int V, float inv_rows, cudaStream_t s) {
+  ce_onehot_kernel<<<cdiv(V, 32), 256, 0, s>>>(tgt, (const bf16_t*)z, dW, db, rows, d, inv_rows);
+  return cudaGetLastError();
+}
+
 __global__ void __launch_bounds__(1024) reduce_sum_kernel(const float* __restrict__ v, int n, float scale,
                                                           float* __restrict__ out) {
   __shared__ float sm[1024];
@@ -1673,14 +2019,6 @@ __device__ __forceinline__ int checked_id(int id, int rows, int* status) {
   return id;
 }
 
-__device__ __forceinline__ void store4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
-__device__ __forceinline__ void store4(bf16_t* p, float4 v) {
-  __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
-  uint2 q;
-  q.x = *reinterpret_cast<uint32_t*>(&lo);
-  q.y = *reinterpret_cast<uint32_t*>(&hi);
-  *reinterpret_cast<uint2*>(p) = q;
-}
 
 // Token + position gather, one warp per output row: the id is read once per row, a lane moves four
 // consecutive columns per step (two 16-byte loads, one 8- or 16-byte store), so a warp reads 512

@@ -113,11 +113,20 @@ cudaError_t layernorm_param_grad(const void* dy, const void* x, const float* mea
 // Causal self-attention over qkv [batch*T, 3*d] = [Q | K | V], heads are contiguous dh-wide
 // column slices; scale 1/sqrt(dh); o [batch*T, d]; lse [batch*heads*T] (natural log).
 cudaError_t attention_fwd(const void* qkv, void* o, float* lse, int batch, int T, int heads, int dh,
-                          bool bf16, cudaStream_t s);
+                          bool bf16, cudaStream_t s, int* status = nullptr);
 // dqkv [batch*T, 3*d] from do, with delta [batch*heads*T] as scratch.
 cudaError_t attention_bwd(const void* qkv, const void* o, const void* dout, const float* lse,
                           float* delta, void* dqkv, int batch, int T, int heads, int dh, bool bf16,
-                          cudaStream_t s);
+                          cudaStream_t s, int* status = nullptr);
+
+// tcgen05 / TMEM / TMA versions for bf16 with 64-wide heads (attention_tc.cu); same contracts.  status:
+// the model's device status word (bounded waits), may be null.
+bool attention_tc_supported(int dh, int d, const void* qkv, const void* o);
+cudaError_t attention_fwd_tc(const void* qkv, void* o, float* lse, int batch, int T, int heads, int* status, cudaStream_t s);
+// dqkv from dout, lse and delta (delta[b,h,t] = sum_c dout * o over the head's 64 columns, see attention_delta_bf16)
+cudaError_t attention_bwd_tc(const void* qkv, const void* dout, const float* lse, const float* delta, void* dqkv, int batch, int T,
+                             int heads, int* status, cudaStream_t s);
+cudaError_t attention_delta_bf16(const void* o, const void* dout, float* delta, int batch, int T, int heads, cudaStream_t s);
 
 // Tensor-core versions (mma.sync m16n8k16) for bf16 with 64-wide heads; same contracts.
 bool attention_mma_supported(int dh, int d);
@@ -138,6 +147,23 @@ cudaError_t softmax_ce_fused(void* logits, const int32_t* ids, int T, float* row
                              float inv_rows, cudaStream_t s);
 cudaError_t softmax_ce_inplace(void* logits, const int32_t* ids, int T, float* rowloss, int rows, int V,
                                float inv_rows, bool bf16, cudaStream_t s);
+// Softmax cross-entropy head without a pass over the logits (bf16, d % 8 == 0): see kernels.cu.
+//   ce_target_logit  tgt[n] (clamped), ref[n] = lt[n] = z_n . W[t_n] + bias[t_n]; clears bad[0]
+//   (head GEMM with Epilogue::ce_ref = ref writes P = exp(l - ref) and the partial sums psum)
+//   ce_finalize      rowloss, rowscale r_n = 1/(S_n rows), zs = r (.) z; unsafe rows -> bad[1..], bad[0] = count
+//   ce_fixup         recomputes the listed rows exactly (no-op when bad[0] == 0 or *status != 0); bad holds rows+1 ints
+//   ce_dz_finish     dz = r_n * (sum of `splits` fp32 partials of P W) - W[t_n]/rows, rounded once
+//   ce_onehot        dW[t_n,:] -= z_n/rows, db[t_n] -= 1/rows in row order (after the GEMM part of dW, db)
+cudaError_t ce_target_logit(const void* z, const void* W, const float* bias, const int32_t* ids, int T, int rows, int d, int V,
+                            int* tgt, float* ref, float* lt, int* bad, cudaStream_t s);
+cudaError_t ce_finalize(const float* psum, int groups, const float* ref, const float* lt, const void* z, void* zs, float* rowloss,
+                        float* rowscale, int* bad, int rows, int d, float inv_rows, cudaStream_t s);
+cudaError_t ce_fixup(const int* bad, const int* status, const void* z, const void* W, const float* bias, void* P, float* ref, const float* lt, void* zs,
+                     float* rowloss, float* rowscale, int rows, int d, int V, float inv_rows, cudaStream_t s);
+cudaError_t ce_dz_finish(const float* part, int splits, int rows, int d, const float* rowscale, const int* tgt, const void* W,
+                         void* dz, float inv_rows, cudaStream_t s);
+cudaError_t ce_onehot(const int* tgt, const void* z, float* dW, float* db, int rows, int d, int V, float inv_rows, cudaStream_t s);
+
 // out[0] = (sum of v[0..n)) * scale, fixed-order tree in one CTA.
 cudaError_t reduce_sum(const float* v, int n, float scale, float* out, cudaStream_t s);
 

@@ -11,12 +11,15 @@ from paper_2608_18469_b200 import binding, synth
 from tests import util
 
 TOL = {"f32": 1e-4, "bf16": 2e-2}     # relative L2 PER TENSOR against the fp64 oracle
-# Optimizer alone (fp64 update rule applied to the library's own gradient vs the fp32 kernel): a
-# handful of fp32 roundings.  A tensor that starts at zero (LayerNorm shift) consists of the update
-# only, so its relative error is that of the update itself (m, v, two bias corrections, sqrt,
-# divide: a few 1e-7 each, 2e-6 observed); every other tensor is dominated by the parameter.
+# Optimizer alone (fp64 update rule applied to the library's own gradient vs the fp32 kernel).  The
+# new parameter is the old one plus an update; the kernel rounds the parameter to fp32 (relative
+# 6e-8, a few operations: OPT_TOL of its norm) and computes the update with a handful of fp32
+# operations (m, v, two bias corrections, sqrt, divide: a few 1e-7 each, 2e-6 observed:
+# OPT_TOL_UPDATE of the update's norm).  A tensor that starts at zero (LayerNorm shift) or happens
+# to be tiny (a scalar head bias) consists of the update only, every other one is dominated by the
+# parameter; any formula mistake shows up at 1e-3 of the update or more.
 OPT_TOL = 2e-6
-OPT_TOL_ZERO_INIT = 1e-5
+OPT_TOL_UPDATE = 1e-5
 
 # bf16 only.  A gradient is a sum over samples; on some instances that sum nearly cancels (a bias
 # gradient on labels drawn independently of the inputs; every gradient of a block right after Adam's
@@ -89,21 +92,23 @@ def new_model(spec, flat):
     return m
 
 
-def compare_teacher_forced(spec, steps, seed=0, n_streams=2, flags=0, report=None, case=None):
+def compare_teacher_forced(spec, steps, seed=0, n_streams=2, flags=0, report=None, case=None, init_hook=None):
     """Each step: library and oracle start from the same fp32 parameters and optimizer state;
     losses and every gradient tensor, each on its own, must agree within TOL; the parameters
     after the optimizer must match the update rule applied in fp64 to the library's own gradients.
     `case` names the instance for the bf16 conditioning allow-list (see COND_CAP above); with
     `report` (a dict) nothing is asserted: worst errors and the list of tensors that would need
-    the allow-list are collected instead."""
+    the allow-list are collected instead.  `init_hook(values)` may edit the initial parameters in
+    place (a dict keyed by (block, tensor name)) before either side sees them."""
     tol = TOL[spec["dtype"]]
     flat = synth.init_params(spec, seed)
     tl = synth.tensor_list(spec)
+    if init_hook is not None:           # the test's own change to the drawn initial values, by tensor name
+        init_hook({(b, name): v for (b, name, _s, _t), v in zip(tl, flat)})
     tidx = util.trainable_index(spec)
     m = new_model(spec, flat)
     params = util.structure(spec, flat)
     state = orc.new_opt_state(params)
-    zero_init = [not np.any(v) for v in flat]      # tensors that consist of optimizer updates only
     worst = {}
     try:
         for it in range(steps):
@@ -171,13 +176,12 @@ def compare_teacher_forced(spec, steps, seed=0, n_streams=2, flags=0, report=Non
                 # optimizer alone: update rule in fp64 on the library's gradient
                 th, _, _ = orc.optimizer_update(spec["opt"], params["blocks"][b][name], g.astype(np.float64),
                                                 state["m"][b][name], state["v"][b][name], state["t"] + 1)
-                perr = synth.rel_l2(m.params(i), th)
-                worst[f"param {key}"] = max(worst.get(f"param {key}", 0), perr)
-                ptol = OPT_TOL_ZERO_INIT if zero_init[i] else OPT_TOL
+                old = params["blocks"][b][name]
+                pbound = OPT_TOL * np.linalg.norm(old) + OPT_TOL_UPDATE * np.linalg.norm(th - old)
+                perr = float(np.linalg.norm(m.params(i).astype(np.float64) - th)) / max(pbound, 1e-300)
+                worst["param/bound"] = max(worst.get("param/bound", 0), perr)
                 if report is None:
-                    assert perr <= ptol, (it, key, perr)
-                else:
-                    worst["param/tol"] = max(worst.get("param/tol", 0), perr / ptol)
+                    assert perr <= 1.0, (it, key, perr, pbound)
             params, state = new_params, new_state
     finally:
         m.close()

@@ -139,7 +139,7 @@ def test_timeline_profile_and_launch_count():
                 assert tg[b + 1, 0] >= tg[b, 1] - 1e-3        # F_{b+1} follows F_b on the main stream
     recs = m.profile_step(**db.args())
     assert sum(r["launches"] for r in recs) == per_step
-    assert {r["name"] for r in recs} >= {"gemm_fwd", "gemm_dgrad", "gemm_wgrad", "softmax_ce", "opt_update"}
+    assert {r["name"] for r in recs} >= {"gemm_fwd", "gemm_dgrad", "gemm_wgrad", "ce_finalize", "opt_update"}
     assert all(r["ms"] >= 0 for r in recs) and sum(r["flops"] for r in recs) > 0
     m.close()
 

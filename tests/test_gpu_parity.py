@@ -62,6 +62,7 @@ def _bf16_cases():
     s["c5_w512_b512"] = synth.config("C5", w=512, batch=512)
     s["mlp_bf16_ragged"] = synth.mlp_spec(200, 328, 2, 300, "gelu", "bf16")
     s["lm_bf16_small"] = synth.lm_spec(2, 128, 2, 512, 128, 4, 1000)
+    s["lm_bf16_ragged_vocab"] = synth.lm_spec(2, 128, 2, 256, 75, 3, 1016)   # 225 rows, 1016 = 3*256 + 248 logits: ragged in every tile size
     s["lm_bf16_ragged_T"] = synth.lm_spec(2, 192, 3, 384, 100, 3, 777)     # T not a multiple of the 64-tile
     s["lm_bf16_T320"] = synth.lm_spec(1, 64, 1, 128, 320, 2, 300)            # five key tiles per head
     s["lm_bf16_dh32"] = synth.lm_spec(1, 128, 4, 256, 96, 2, 300)            # head width 32: SIMT attention
@@ -97,14 +98,42 @@ def test_bf16_small_with_the_fused_loss_and_bias_gradient_kernel(name, monkeypat
     """The persistent softmax-CE kernel that also produces the head's bias gradient is chosen by
     size (gradient matrices far beyond L2); here it is forced onto small cases, including
     vocabularies whose vector count is not a multiple of the CTA width and fewer rows than CTAs."""
+    monkeypatch.setenv("ERASE_CE_MODE", "0")
     monkeypatch.setenv("ERASE_CE_FUSED", "2")
     _gu().compare_teacher_forced(_bf16_cases()[name], steps=2, seed=3, case=name)
 
 
-def test_large_vocabulary_head_uses_the_fused_loss_kernel_by_size():
-    # 4224 rows x 32000 logits = 270 MB of bf16 gradients: beyond the size threshold; 4000 vectors per row
+@pytest.mark.parametrize("ce_mode", ["1", "0"])
+def test_large_vocabulary_head(ce_mode, monkeypatch):
+    """4224 rows x 32000 logits (270 MB in bf16, 4000 16-byte vectors per row).  Mode 1: the head
+    whose GEMM epilogue leaves exp(logit - reference) and partial sums, so that loss and gradient
+    never read the logits back.  Mode 0: the separate softmax pass, where this size selects the
+    persistent kernel that also produces the bias gradient."""
+    monkeypatch.setenv("ERASE_CE_MODE", ce_mode)
     spec = synth.lm_spec(1, 64, 1, 128, 528, 8, 32000)
     _gu().compare_teacher_forced(spec, steps=1, seed=4, case="lm_vocab32000")
+
+
+@pytest.mark.parametrize("name", ["lm_bf16_small", "lm_bf16_ragged_vocab", "C2"])
+def test_softmax_head_with_the_separate_softmax_pass(name, monkeypatch):
+    """The path that heads which do not qualify for the exp epilogue take (fp32 models,
+    vocabularies or widths that are not multiples of 8), forced onto cases that do qualify."""
+    monkeypatch.setenv("ERASE_CE_MODE", "0")
+    spec = synth.config("C2") if name == "C2" else _bf16_cases()[name]
+    _gu().compare_teacher_forced(spec, steps=2, seed=0 if name == "C2" else 3, case=name)
+
+
+def test_softmax_head_rows_whose_target_logit_is_far_below_the_maximum_are_recomputed():
+    """The exp epilogue measures every logit against the target's own logit.  A head bias that
+    lifts one vocabulary entry by 150 puts the row maximum 150 above that reference for nearly every
+    row: their sums overflow, the finalize kernel lists them, and the fix-up kernel recomputes those
+    rows exactly.  A second entry lifted by 60 stays inside the safe range.  Losses (about 150 nats)
+    and every gradient must still match the oracle."""
+    def lift(values):
+        values[(0, "bh")][7] += 150.0
+        values[(1, "bh")][11] += 60.0
+    spec = synth.lm_spec(2, 128, 2, 256, 96, 3, 1000)
+    _gu().compare_teacher_forced(spec, steps=2, seed=3, case="lm_lifted_bias", init_hook=lift)
 
 
 def test_config2_small_lm_bf16_full_size():
@@ -200,11 +229,9 @@ def test_erase_schedule_is_bit_identical_to_serial(name):
                                      flags=binding.GRAPH | binding.EARLY_HEAD | binding.BLOCK_OPT))
     _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=nb + 1, flags=binding.SPLIT_BWD))
     _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=2,
-                                     flags=binding.GRAPH | binding.EARLY_HEAD | binding.BLOCK_OPT | binding.SPLIT_BWD,
-                                 case="C2_bench"))
+                                     flags=binding.GRAPH | binding.EARLY_HEAD | binding.BLOCK_OPT | binding.SPLIT_BWD))
     _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=nb + 1,
-                                     flags=binding.GRAPH | binding.EARLY_HEAD | binding.BLOCK_OPT | binding.SPLIT_BWD,
-                                 case="C2_bench"))
+                                     flags=binding.GRAPH | binding.EARLY_HEAD | binding.BLOCK_OPT | binding.SPLIT_BWD))
     # parallel topology: every block's forward on its side stream too (ignored on chains)
     P = binding.PAR_FWD
     _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=nb + 1, flags=P))
