@@ -94,7 +94,7 @@ struct AttnArgs {
   float scale_log2;      // scale * log2(e)
   bf16_t* o;             // forward output [rows, d]
   float* lse;            // [batch, H, T], natural log (written by the forward, read by the backward)
-  const float* delta;    // backward: [batch, H, T], sum_c dO * O
+  float* delta;          // backward: [batch, H, T], sum_c dO * O (written by the dQ kernel, read by the dK/dV kernel)
   bf16_t* dqkv;          // backward output [rows, 3 d]
   int* status;
 };
@@ -235,33 +235,46 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
       tc_fence_after();
       const bool diag = j == nt - 1;                  // the only tile with keys beyond some of its queries
       uint32_t r[32];
-      float mx = -INFINITY;
+      // pass 1: row maximum (four independent chains; only the diagonal tile masks keys beyond the query)
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll 1
       for (int c = 0; c < TK / 32; c++) {
         tc_ld32(tm_s + lane_off + c * 32, r);
+        if (diag) {
 #pragma unroll
-        for (int e = 0; e < 32; e++) {
-          const float v = __uint_as_float(r[e]);
-          mx = (diag && c * 32 + e > row) ? mx : fmaxf(mx, v);
+          for (int e = 0; e < 32; e++)
+            if (c * 32 + e > row) r[e] = 0xff800000u;      // -inf
+        }
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) {
+          mx0 = fmaxf(mx0, __uint_as_float(r[e]));
+          mx1 = fmaxf(mx1, __uint_as_float(r[e + 1]));
+          mx2 = fmaxf(mx2, __uint_as_float(r[e + 2]));
+          mx3 = fmaxf(mx3, __uint_as_float(r[e + 3]));
         }
       }
+      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
       const float m_new = fmaxf(m, mx * p.scale_log2);
       const float alpha = ex2f(m - m_new);            // 0 for the first tile (m = -inf)
       if (j > 0 && !take_o(j - 1)) { ok = false; break; }
-      float rowsum = 0.f;
+      // pass 2: exponentials, row sum (four chains), P to shared memory
+      float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll 1
       for (int c = 0; c < TK / 32; c++) {
         tc_ld32(tm_s + lane_off + c * 32, r);
         float pv[32];
 #pragma unroll
-        for (int e = 0; e < 32; e++) {
-          float pe = ex2f(fmaf(__uint_as_float(r[e]), p.scale_log2, -m_new));
-          if (diag && c * 32 + e > row) pe = 0.f;
-          rowsum += pe;
-          pv[e] = pe;
+        for (int e = 0; e < 32; e++) pv[e] = ex2f(fmaf(__uint_as_float(r[e]), p.scale_log2, -m_new));
+        if (diag) {
+#pragma unroll
+          for (int e = 0; e < 32; e++)
+            if (c * 32 + e > row) pv[e] = 0.f;
         }
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) { s0 += pv[e]; s1 += pv[e + 1]; s2 += pv[e + 2]; s3 += pv[e + 3]; }
         store_p32(p_s, row, c * 32, pv);
       }
+      const float rowsum = (s0 + s1) + (s2 + s3);
       l = fmaf(l, alpha, rowsum);
       m = m_new;
       alpha_prev = alpha;
@@ -299,40 +312,66 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
 
 
 // ------------------------------------------------------------------------------------------------
-// backward.  Both kernels: 8 softmax warps (two per TMEM lane quarter, each takes 64 of the 128
-// columns of a tile) and one warp that issues TMA and MMA; TMEM holds the score and dP tiles and
-// the fp32 gradient accumulators, which stay there over the whole walk (no rescaling is needed: the
-// probabilities are recomputed from the final log-sum-exp).
+// backward.  Both kernels: 8 softmax warps (two per TMEM lane quarter, each takes 32 of the 64
+// columns of a sub-tile) and one warp that issues TMA and MMA.  The walk goes over sub-tiles of 64
+// keys (dQ kernel) or 64 queries (dK/dV kernel), so that the score, dP and gradient accumulators
+// take 256 TMEM columns and two CTAs share an SM: one CTA's softmax work hides the other's MMA and
+// barrier latencies.  The gradient accumulators stay in tensor memory over the whole walk (no
+// rescaling is needed: the probabilities are recomputed from the final log-sum-exp).
 // ------------------------------------------------------------------------------------------------
 constexpr int BW_THREADS = 288;
+constexpr int TW = 64;                                   // sub-tile width
+constexpr uint32_t SUB_BYTES = TW * DH * 2;              // a [64, 64] bf16 sub-tile: 8 KB
+constexpr int NST_Q = 3;                                 // K/V sub-tile stages of the dQ kernel
+constexpr int NST_KV = 2;                                // Q/dO sub-tile stages of the dK/dV kernel
 
 __device__ __forceinline__ void softmax_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
-// dQ: one CTA per (query tile, head, sequence), key tiles 0 .. query tile.
+// dot product of one swizzled 128-byte row (64 bf16) of two K-major tiles
+__device__ __forceinline__ float row_dot64(const uint8_t* ta, const uint8_t* tb, int row) {
+  float d0 = 0.f, d1 = 0.f;
+#pragma unroll
+  for (int c = 0; c < 8; c++) {
+    const int off = row * 128 + ((c ^ (row & 7)) << 4);
+    const uint4 qa = *reinterpret_cast<const uint4*>(ta + off), qb = *reinterpret_cast<const uint4*>(tb + off);
+    const uint32_t x[4] = {qa.x, qa.y, qa.z, qa.w}, y[4] = {qb.x, qb.y, qb.z, qb.w};
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+      d0 = fmaf(__uint_as_float(x[j] << 16), __uint_as_float(y[j] << 16), d0);
+      d1 = fmaf(__uint_as_float(x[j] & 0xffff0000u), __uint_as_float(y[j] & 0xffff0000u), d1);
+    }
+  }
+  return d0 + d1;
+}
+
+// dQ (and delta): one CTA per (query tile of 128, head, sequence), key sub-tiles of 64 from 0 up to the tile's last query.
+//   delta[q] = sum_c dO[q,c] O[q,c]  (from the dO and O tiles in shared memory; also written out for the dK/dV kernel)
 //   S = Q K^T, dP = dO V^T (both operands K-major);  dS = P (.) (dP - delta), P = exp(S scale - lse)
 //   dQ += dS K   (A = dS [q, key] K-major from shared memory, B = K [key, dh] MN-major), times scale at the end
-__global__ void __launch_bounds__(BW_THREADS, 1)
-attn_bwd_q_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_constant__ CUtensorMap map_do,
+__global__ void __launch_bounds__(BW_THREADS, 2)
+attn_bwd_q_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kv,
+                     const __grid_constant__ CUtensorMap map_do, const __grid_constant__ CUtensorMap map_o,
                      const __grid_constant__ AttnArgs p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
-  const uint32_t q_s = base, do_s = q_s + TILE_BYTES, k_s = do_s + TILE_BYTES, v_s = k_s + 2 * TILE_BYTES, ds_s = v_s + 2 * TILE_BYTES;
-  const uint32_t bar = ds_s + P_BYTES;
-  const uint32_t q_full = bar, kv_full0 = bar + 8, kv_empty0 = bar + 24, sdp_full = bar + 40, ds_full = bar + 48, ds_free = bar + 56,
-                 acc_full = bar + 64, tmem_slot = bar + 72;
+  const uint32_t q_s = base, do_s = q_s + TILE_BYTES, kv_s = do_s + TILE_BYTES, ds_s = kv_s + NST_Q * 2 * SUB_BYTES;
+  const uint32_t bar = ds_s + TILE_BYTES;
+  const uint32_t q_full = bar, kv_full0 = bar + 8, kv_empty0 = kv_full0 + 8 * NST_Q, sdp_full = kv_empty0 + 8 * NST_Q, ds_full = sdp_full + 8,
+                 ds_free = ds_full + 8, acc_full = ds_free + 8, tmem_slot = acc_full + 8;
   volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - base));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;
   const int h = blockIdx.y, b = blockIdx.z;
   const int d = p.H * DH;
-  const int q0 = qt * TQ, nt = qt + 1;
+  const int q0 = qt * TQ;
+  const int nsub = min(2 * (qt + 1), (p.T + TW - 1) / TW);    // key sub-tiles that hold a key <= the tile's last query
   int st0 = status_peek(p.status);
   if (threadIdx.x == 0 && (base & 1023u)) { set_status(p.status, 10); st0 = 10; }
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
-    for (int s = 0; s < 2; s++) { mbar_init(kv_full0 + 8 * s, 1); mbar_init(kv_empty0 + 8 * s, 1); }
+    for (int s = 0; s < NST_Q; s++) { mbar_init(kv_full0 + 8 * s, 1); mbar_init(kv_empty0 + 8 * s, 1); }
     mbar_init(sdp_full, 1);
     mbar_init(ds_full, 8);
     mbar_init(ds_free, 1);
@@ -342,68 +381,70 @@ attn_bwd_q_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_c
   }
   if (warp == 8) {
     if (lane == 0) {
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_qkv) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_q) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_kv) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&map_do) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_o) : "memory");
     }
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(512u) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(256u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   const bool dead = __syncthreads_or(st0 != 0) != 0;
   tc_fence_after();
   const uint32_t tmem = *tmem_slot_ptr;
-  const uint32_t tm_s = tmem, tm_dp = tmem + 128, tm_dq = tmem + 256;
+  const uint32_t tm_s = tmem, tm_dp = tmem + 64, tm_dq = tmem + 128;
 
   if (dead) {
   } else if (warp == 8) {
     if (lane == 0) {
       const int row0 = b * p.T;
       auto load_kv = [&](int j) {
-        const int s = j & 1;
-        mbar_expect_tx(kv_full0 + 8 * s, 2 * TILE_BYTES);
-        tma_load_2d(k_s + s * TILE_BYTES, &map_qkv, d + h * DH, row0 + j * TK, kv_full0 + 8 * s);
-        tma_load_2d(v_s + s * TILE_BYTES, &map_qkv, 2 * d + h * DH, row0 + j * TK, kv_full0 + 8 * s);
+        const int s = j % NST_Q;
+        const uint32_t full = kv_full0 + 8 * s, dst = kv_s + s * 2 * SUB_BYTES;
+        mbar_expect_tx(full, 2 * SUB_BYTES);
+        tma_load_2d(dst, &map_kv, d + h * DH, row0 + j * TW, full);
+        tma_load_2d(dst + SUB_BYTES, &map_kv, 2 * d + h * DH, row0 + j * TW, full);
       };
-      mbar_expect_tx(q_full, 2 * TILE_BYTES);
-      tma_load_2d(q_s, &map_qkv, h * DH, row0 + q0, q_full);
+      mbar_expect_tx(q_full, 3 * TILE_BYTES);
+      tma_load_2d(q_s, &map_q, h * DH, row0 + q0, q_full);
       tma_load_2d(do_s, &map_do, h * DH, row0 + q0, q_full);
-      load_kv(0);
-      if (nt > 1) load_kv(1);
-      const uint32_t id_s = idesc_of(TK, false, false), id_q = idesc_of(DH, false, true);
+      tma_load_2d(ds_s, &map_o, h * DH, row0 + q0, q_full);      // the O tile: read once for delta, then this buffer holds dS
+      for (int j = 0; j < NST_Q && j < nsub; j++) load_kv(j);
+      const uint32_t id_s = idesc_of(TW, false, false), id_q = idesc_of(DH, false, true);
       bool ok = mbar_wait(q_full, 0);
       if (!ok) set_status(p.status, 21);
       auto issue_dq = [&](int j) {      // dQ += dS_j K_j
-        const int s = j & 1;
+        const uint32_t kj = kv_s + (j % NST_Q) * 2 * SUB_BYTES;
 #pragma unroll
-        for (int kk = 0; kk < TK / 16; kk++)
-          tc_mma(tm_dq, desc_k(ds_s + (kk >> 2) * TILE_BYTES, kk & 3), desc_mn(k_s + s * TILE_BYTES + (kk >> 2) * (TILE_BYTES / 2), kk & 3, TILE_BYTES / 2),
-                 id_q, (j > 0 || kk > 0) ? 1u : 0u);
+        for (int kk = 0; kk < TW / 16; kk++) tc_mma(tm_dq, desc_k(ds_s, kk), desc_mn(kj, kk, SUB_BYTES), id_q, (j > 0 || kk > 0) ? 1u : 0u);
       };
-      for (int j = 0; j < nt && ok; j++) {
-        const int s = j & 1;
-        if (!mbar_wait(kv_full0 + 8 * s, (j >> 1) & 1)) { set_status(p.status, 22); ok = false; break; }
-        if (j > 0 && !mbar_wait(ds_full, (j - 1) & 1)) { set_status(p.status, 23); ok = false; break; }
+      for (int j = 0; j < nsub && ok; j++) {
+        const int s = j % NST_Q;
+        const uint32_t kj = kv_s + s * 2 * SUB_BYTES, vj = kj + SUB_BYTES;
+        if (!mbar_wait(kv_full0 + 8 * s, (j / NST_Q) & 1)) { set_status(p.status, 22); ok = false; break; }
+        if (j > 0 && !mbar_wait(ds_full, (j - 1) & 1)) { set_status(p.status, 23); ok = false; break; }   // S, dP read; dS_{j-1} written
         tc_fence_after();
 #pragma unroll
-        for (int kk = 0; kk < DH / 16; kk++) tc_mma(tm_s, desc_k(q_s, kk), desc_k(k_s + s * TILE_BYTES, kk), id_s, kk > 0 ? 1u : 0u);
+        for (int kk = 0; kk < DH / 16; kk++) tc_mma(tm_s, desc_k(q_s, kk), desc_k(kj, kk), id_s, kk > 0 ? 1u : 0u);
 #pragma unroll
-        for (int kk = 0; kk < DH / 16; kk++) tc_mma(tm_dp, desc_k(do_s, kk), desc_k(v_s + s * TILE_BYTES, kk), id_s, kk > 0 ? 1u : 0u);
+        for (int kk = 0; kk < DH / 16; kk++) tc_mma(tm_dp, desc_k(do_s, kk), desc_k(vj, kk), id_s, kk > 0 ? 1u : 0u);
         tc_commit(sdp_full);
         if (j > 0) {
           issue_dq(j - 1);
           tc_commit(ds_free);
-          tc_commit(kv_empty0 + 8 * ((j - 1) & 1));
-          if (j + 1 < nt) {
-            if (!mbar_wait(kv_empty0 + 8 * ((j - 1) & 1), ((j - 1) >> 1) & 1)) { set_status(p.status, 24); ok = false; break; }
-            load_kv(j + 1);
+          tc_commit(kv_empty0 + 8 * ((j - 1) % NST_Q));
+          if (j - 1 + NST_Q < nsub) {     // the freed stage takes the sub-tile NST_Q further on
+            if (!mbar_wait(kv_empty0 + 8 * ((j - 1) % NST_Q), ((j - 1) / NST_Q) & 1)) { set_status(p.status, 24); ok = false; break; }
+            load_kv(j - 1 + NST_Q);
           }
         }
       }
       if (ok) {
-        if (!mbar_wait(ds_full, (nt - 1) & 1)) { set_status(p.status, 23); ok = false; }
+        if (!mbar_wait(ds_full, (nsub - 1) & 1)) { set_status(p.status, 23); ok = false; }
         if (ok) {
           tc_fence_after();
-          issue_dq(nt - 1);
+          issue_dq(nsub - 1);
         }
       }
       tc_commit(acc_full);        // fires in any case, so that the softmax warps do not wait for their limit
@@ -420,37 +461,51 @@ attn_bwd_q_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_c
     const bool row_ok = t < p.T;
     const long long stat = ((long long)b * p.H + h) * p.T + t;
     const float lse2 = row_ok ? p.lse[stat] * LOG2E : 0.f;
-    const float dl = row_ok ? p.delta[stat] : 0.f;
     bool ok = true;
-    for (int j = 0; j < nt; j++) {
+    float dl = 0.f;
+    {   // delta of this thread's row from the dO and O tiles
+      bool w = mbar_wait(q_full, 0);
+      if (!w) set_status(p.status, 28);
+      w = __all_sync(0xffffffffu, w);
+      if (w) {
+        dl = row_dot64(smem_raw + (do_s - base), smem_raw + (ds_s - base), row);
+        if (half == 0 && row_ok) p.delta[stat] = dl;
+      } else {
+        ok = false;
+      }
+      softmax_bar();              // every row of the O tile has been read: the buffer may now take dS
+    }
+    for (int j = 0; j < nsub && ok; j++) {
       bool w = mbar_wait(sdp_full, j & 1);
       if (!w) set_status(p.status, 25);
       w = __all_sync(0xffffffffu, w);
       if (!w) { ok = false; break; }
       tc_fence_after();
-      const bool diag = j == nt - 1;
-#pragma unroll 1
-      for (int c = 0; c < 2; c++) {
-        const int col0 = half * 64 + c * 32;
-        uint32_t rs[32], rp[32];
-        tc_ld32(tm_s + lane_off + col0, rs);
-        tc_ld32(tm_dp + lane_off + col0, rp);
-        float ds[32];
+      const int col0 = half * 32;
+      const int kcol = j * TW + col0 - q0;                      // key index minus query index = kcol + e - row
+      const bool maskable = j * TW + TW - 1 > q0;              // some key of the sub-tile lies beyond some query
+      uint32_t rs[32], rp[32];
+      tc_ld32_nowait(tm_s + lane_off + col0, rs);
+      tc_ld32_nowait(tm_dp + lane_off + col0, rp);
+      tc_ld_wait();
+      float ds[32];
+      if (maskable) {
 #pragma unroll
         for (int e = 0; e < 32; e++) {
-          float pe = ex2f(fmaf(__uint_as_float(rs[e]), p.scale_log2, -lse2));
-          if (diag && col0 + e > row) pe = 0.f;
+          const float pe = kcol + e > row ? 0.f : ex2f(fmaf(__uint_as_float(rs[e]), p.scale_log2, -lse2));
           ds[e] = pe * (__uint_as_float(rp[e]) - dl);
         }
-        if (c == 0 && j > 0) {        // the previous tile's dQ MMAs must have read dS before it is overwritten
-          bool f = mbar_wait(ds_free, (j - 1) & 1);
-          if (!f) set_status(p.status, 26);
-          f = __all_sync(0xffffffffu, f);
-          if (!f) { ok = false; break; }
-        }
-        store_p32(ds_s, row, col0, ds);
+      } else {
+#pragma unroll
+        for (int e = 0; e < 32; e++) ds[e] = ex2f(fmaf(__uint_as_float(rs[e]), p.scale_log2, -lse2)) * (__uint_as_float(rp[e]) - dl);
       }
-      if (!ok) break;
+      if (j > 0) {                  // the previous sub-tile's dQ MMAs must have read dS before it is overwritten
+        bool f = mbar_wait(ds_free, (j - 1) & 1);
+        if (!f) set_status(p.status, 26);
+        f = __all_sync(0xffffffffu, f);
+        if (!f) { ok = false; break; }
+      }
+      store_p32(ds_s, row, col0, ds);
       tc_fence_before();
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
@@ -484,41 +539,40 @@ attn_bwd_q_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_c
   __syncthreads();
   if (warp == 8) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256u) : "memory");
   }
 }
 
-// dK, dV: one CTA per (key tile, head, sequence), query tiles key tile .. last.  Everything is
-// computed transposed, so that a softmax thread owns a KEY row:
+// dK, dV: one CTA per (key tile of 128, head, sequence), query sub-tiles of 64 from the tile's first key to the end of
+// the sequence.  Everything is computed transposed, so that a softmax thread owns a KEY row:
 //   S^T = K Q^T, dP^T = V dO^T (both operands K-major);  P^T = exp(S^T scale - lse[q]),  dS^T = P^T (.) (dP^T - delta[q])
 //   dV += P^T dO   (A = P^T [key, q] K-major from shared memory, B = dO [q, dh] MN-major)
 //   dK += dS^T Q   (A = dS^T,                                   B = Q  [q, dh] MN-major), times scale at the end
-__global__ void __launch_bounds__(BW_THREADS, 1)
-attn_bwd_kv_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_constant__ CUtensorMap map_do,
-                      const __grid_constant__ AttnArgs p) {
+__global__ void __launch_bounds__(BW_THREADS, 2)
+attn_bwd_kv_tc_kernel(const __grid_constant__ CUtensorMap map_kv, const __grid_constant__ CUtensorMap map_q,
+                      const __grid_constant__ CUtensorMap map_do, const __grid_constant__ AttnArgs p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
-  const uint32_t k_s = base, v_s = k_s + TILE_BYTES, q_s = v_s + TILE_BYTES, do_s = q_s + 2 * TILE_BYTES, pt_s = do_s + 2 * TILE_BYTES,
-                 dst_s = pt_s + P_BYTES;
-  const uint32_t vec_s = dst_s + P_BYTES;                 // lse (log2 units) and delta of the query tile: 2 stages x 2 x 128 floats
-  const uint32_t bar = vec_s + 2048;
-  const uint32_t kv_full = bar, qdo_full0 = bar + 8, qdo_empty0 = bar + 24, sdp_full = bar + 40, pds_full = bar + 48, pds_free = bar + 56,
-                 acc_full = bar + 64, tmem_slot = bar + 72;
+  const uint32_t k_s = base, v_s = k_s + TILE_BYTES, qdo_s = v_s + TILE_BYTES, pt_s = qdo_s + NST_KV * 2 * SUB_BYTES, dst_s = pt_s + TILE_BYTES;
+  const uint32_t vec_s = dst_s + TILE_BYTES;              // lse (log2 units) and delta of the query sub-tile: 2 buffers x 2 x 64 floats
+  const uint32_t bar = vec_s + 1024;
+  const uint32_t kv_full = bar, qdo_full0 = bar + 8, qdo_empty0 = qdo_full0 + 8 * NST_KV, sdp_full = qdo_empty0 + 8 * NST_KV,
+                 pds_full = sdp_full + 8, pds_free = pds_full + 8, acc_full = pds_free + 8, tmem_slot = acc_full + 8;
   volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - base));
   float* vec = reinterpret_cast<float*>(smem_raw + (vec_s - base));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int nq = (p.T + TQ - 1) / TQ;
   const int kt = blockIdx.x;                               // key tile 0 has the longest walk and comes first
   const int h = blockIdx.y, b = blockIdx.z;
   const int d = p.H * DH;
-  const int k0 = kt * TK, n = nq - kt;                     // query tiles kt .. nq-1
+  const int k0 = kt * TK;
+  const int first = 2 * kt, n = (p.T + TW - 1) / TW - first;      // query sub-tiles first .. first+n-1 (n >= 1: k0 < T)
   int st0 = status_peek(p.status);
   if (threadIdx.x == 0 && (base & 1023u)) { set_status(p.status, 10); st0 = 10; }
 
   if (threadIdx.x == 0) {
     mbar_init(kv_full, 1);
-    for (int s = 0; s < 2; s++) { mbar_init(qdo_full0 + 8 * s, 1); mbar_init(qdo_empty0 + 8 * s, 1); }
+    for (int s = 0; s < NST_KV; s++) { mbar_init(qdo_full0 + 8 * s, 1); mbar_init(qdo_empty0 + 8 * s, 1); }
     mbar_init(sdp_full, 1);
     mbar_init(pds_full, 8);
     mbar_init(pds_free, 1);
@@ -528,64 +582,62 @@ attn_bwd_kv_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_
   }
   if (warp == 8) {
     if (lane == 0) {
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_qkv) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_kv) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_q) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&map_do) : "memory");
     }
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(512u) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(256u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   const bool dead = __syncthreads_or(st0 != 0) != 0;
   tc_fence_after();
   const uint32_t tmem = *tmem_slot_ptr;
-  const uint32_t tm_s = tmem, tm_dp = tmem + 128, tm_dv = tmem + 256, tm_dk = tmem + 320;
+  const uint32_t tm_s = tmem, tm_dp = tmem + 64, tm_dv = tmem + 128, tm_dk = tmem + 192;
 
   if (dead) {
   } else if (warp == 8) {
     if (lane == 0) {
       const int row0 = b * p.T;
       auto load_qdo = [&](int ii) {
-        const int s = ii & 1;
-        mbar_expect_tx(qdo_full0 + 8 * s, 2 * TILE_BYTES);
-        tma_load_2d(q_s + s * TILE_BYTES, &map_qkv, h * DH, row0 + (kt + ii) * TQ, qdo_full0 + 8 * s);
-        tma_load_2d(do_s + s * TILE_BYTES, &map_do, h * DH, row0 + (kt + ii) * TQ, qdo_full0 + 8 * s);
+        const int s = ii % NST_KV;
+        const uint32_t full = qdo_full0 + 8 * s, dst = qdo_s + s * 2 * SUB_BYTES;
+        mbar_expect_tx(full, 2 * SUB_BYTES);
+        tma_load_2d(dst, &map_q, h * DH, row0 + (first + ii) * TW, full);
+        tma_load_2d(dst + SUB_BYTES, &map_do, h * DH, row0 + (first + ii) * TW, full);
       };
       mbar_expect_tx(kv_full, 2 * TILE_BYTES);
-      tma_load_2d(k_s, &map_qkv, d + h * DH, row0 + k0, kv_full);
-      tma_load_2d(v_s, &map_qkv, 2 * d + h * DH, row0 + k0, kv_full);
-      load_qdo(0);
-      if (n > 1) load_qdo(1);
-      const uint32_t id_s = idesc_of(TQ, false, false), id_g = idesc_of(DH, false, true);
+      tma_load_2d(k_s, &map_kv, d + h * DH, row0 + k0, kv_full);
+      tma_load_2d(v_s, &map_kv, 2 * d + h * DH, row0 + k0, kv_full);
+      for (int ii = 0; ii < NST_KV && ii < n; ii++) load_qdo(ii);
+      const uint32_t id_s = idesc_of(TW, false, false), id_g = idesc_of(DH, false, true);
       bool ok = mbar_wait(kv_full, 0);
       if (!ok) set_status(p.status, 31);
       auto issue_grads = [&](int ii) {     // dV += P^T dO_i, dK += dS^T Q_i
-        const int s = ii & 1;
+        const uint32_t qi = qdo_s + (ii % NST_KV) * 2 * SUB_BYTES, doi = qi + SUB_BYTES;
 #pragma unroll
-        for (int kk = 0; kk < TQ / 16; kk++)
-          tc_mma(tm_dv, desc_k(pt_s + (kk >> 2) * TILE_BYTES, kk & 3), desc_mn(do_s + s * TILE_BYTES + (kk >> 2) * (TILE_BYTES / 2), kk & 3, TILE_BYTES / 2),
-                 id_g, (ii > 0 || kk > 0) ? 1u : 0u);
+        for (int kk = 0; kk < TW / 16; kk++) tc_mma(tm_dv, desc_k(pt_s, kk), desc_mn(doi, kk, SUB_BYTES), id_g, (ii > 0 || kk > 0) ? 1u : 0u);
 #pragma unroll
-        for (int kk = 0; kk < TQ / 16; kk++)
-          tc_mma(tm_dk, desc_k(dst_s + (kk >> 2) * TILE_BYTES, kk & 3), desc_mn(q_s + s * TILE_BYTES + (kk >> 2) * (TILE_BYTES / 2), kk & 3, TILE_BYTES / 2),
-                 id_g, (ii > 0 || kk > 0) ? 1u : 0u);
+        for (int kk = 0; kk < TW / 16; kk++) tc_mma(tm_dk, desc_k(dst_s, kk), desc_mn(qi, kk, SUB_BYTES), id_g, (ii > 0 || kk > 0) ? 1u : 0u);
       };
       for (int ii = 0; ii < n && ok; ii++) {
-        const int s = ii & 1;
-        if (!mbar_wait(qdo_full0 + 8 * s, (ii >> 1) & 1)) { set_status(p.status, 32); ok = false; break; }
+        const int s = ii % NST_KV;
+        const uint32_t qi = qdo_s + s * 2 * SUB_BYTES, doi = qi + SUB_BYTES;
+        if (!mbar_wait(qdo_full0 + 8 * s, (ii / NST_KV) & 1)) { set_status(p.status, 32); ok = false; break; }
         if (ii > 0 && !mbar_wait(pds_full, (ii - 1) & 1)) { set_status(p.status, 33); ok = false; break; }
         tc_fence_after();
 #pragma unroll
-        for (int kk = 0; kk < DH / 16; kk++) tc_mma(tm_s, desc_k(k_s, kk), desc_k(q_s + s * TILE_BYTES, kk), id_s, kk > 0 ? 1u : 0u);
+        for (int kk = 0; kk < DH / 16; kk++) tc_mma(tm_s, desc_k(k_s, kk), desc_k(qi, kk), id_s, kk > 0 ? 1u : 0u);
 #pragma unroll
-        for (int kk = 0; kk < DH / 16; kk++) tc_mma(tm_dp, desc_k(v_s, kk), desc_k(do_s + s * TILE_BYTES, kk), id_s, kk > 0 ? 1u : 0u);
+        for (int kk = 0; kk < DH / 16; kk++) tc_mma(tm_dp, desc_k(v_s, kk), desc_k(doi, kk), id_s, kk > 0 ? 1u : 0u);
         tc_commit(sdp_full);
         if (ii > 0) {
           issue_grads(ii - 1);
           tc_commit(pds_free);
-          tc_commit(qdo_empty0 + 8 * ((ii - 1) & 1));
-          if (ii + 1 < n) {
-            if (!mbar_wait(qdo_empty0 + 8 * ((ii - 1) & 1), ((ii - 1) >> 1) & 1)) { set_status(p.status, 34); ok = false; break; }
-            load_qdo(ii + 1);
+          tc_commit(qdo_empty0 + 8 * ((ii - 1) % NST_KV));
+          if (ii - 1 + NST_KV < n) {
+            if (!mbar_wait(qdo_empty0 + 8 * ((ii - 1) % NST_KV), ((ii - 1) / NST_KV) & 1)) { set_status(p.status, 34); ok = false; break; }
+            load_qdo(ii - 1 + NST_KV);
           }
         }
       }
@@ -609,15 +661,13 @@ attn_bwd_kv_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_
     const int tid = threadIdx.x;                           // 0..255
     bool ok = true;
     for (int ii = 0; ii < n; ii++) {
-      const int q0 = (kt + ii) * TQ;
-      // this query tile's log-sum-exp (in log2 units) and delta, shared by all key rows; +inf marks a query past the sequence
-      float* vs = vec + (ii & 1) * 256;
+      const int q0 = (first + ii) * TW;
+      // this query sub-tile's log-sum-exp (in log2 units) and delta, shared by all key rows; +inf marks a query past the sequence
+      float* vs = vec + (ii & 1) * 128;
       if (tid < 128) {
-        const int t = q0 + tid;
-        vs[tid] = t < p.T ? p.lse[((long long)b * p.H + h) * p.T + t] * LOG2E : INFINITY;
-      } else {
-        const int t = q0 + tid - 128;
-        vs[tid] = t < p.T ? p.delta[((long long)b * p.H + h) * p.T + t] : 0.f;
+        const int t = q0 + (tid & 63);
+        const long long stat = ((long long)b * p.H + h) * p.T + t;
+        vs[tid] = tid < 64 ? (t < p.T ? p.lse[stat] * LOG2E : INFINITY) : (t < p.T ? p.delta[stat] : 0.f);
       }
       softmax_bar();
       bool w = mbar_wait(sdp_full, ii & 1);
@@ -625,31 +675,40 @@ attn_bwd_kv_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_
       w = __all_sync(0xffffffffu, w);
       if (!w) { ok = false; break; }
       tc_fence_after();
-      const bool diag = ii == 0;                           // query tile == key tile: keys beyond the query are masked
-#pragma unroll 1
-      for (int c = 0; c < 2; c++) {
-        const int col0 = half * 64 + c * 32;
-        uint32_t rs[32], rp[32];
-        tc_ld32(tm_s + lane_off + col0, rs);
-        tc_ld32(tm_dp + lane_off + col0, rp);
-        float pt[32], ds[32];
-#pragma unroll
-        for (int e = 0; e < 32; e++) {
-          float pe = ex2f(fmaf(__uint_as_float(rs[e]), p.scale_log2, -vs[col0 + e]));   // exp2(-inf) = 0 past the sequence
-          if (diag && row > col0 + e) pe = 0.f;
-          pt[e] = pe;
-          ds[e] = pe * (__uint_as_float(rp[e]) - vs[128 + col0 + e]);
-        }
-        if (c == 0 && ii > 0) {       // the previous tile's MMAs must have read P^T and dS^T before they are overwritten
-          bool f = mbar_wait(pds_free, (ii - 1) & 1);
-          if (!f) set_status(p.status, 36);
-          f = __all_sync(0xffffffffu, f);
-          if (!f) { ok = false; break; }
-        }
-        store_p32(pt_s, row, col0, pt);
-        store_p32(dst_s, row, col0, ds);
+      const int col0 = half * 32;
+      const int qcol = q0 + col0 - k0;                      // query index minus key index = qcol + e - row
+      const bool maskable = q0 < k0 + TK - 1;              // some query of the sub-tile lies before some key
+      uint32_t rs[32], rp[32];
+      tc_ld32_nowait(tm_s + lane_off + col0, rs);
+      tc_ld32_nowait(tm_dp + lane_off + col0, rp);
+      if (ii > 0) {                 // the previous sub-tile's MMAs must have read P^T and dS^T before they are overwritten
+        bool f = mbar_wait(pds_free, (ii - 1) & 1);      // (they were issued right behind this sub-tile's score MMAs)
+        if (!f) set_status(p.status, 36);
+        f = __all_sync(0xffffffffu, f);
+        if (!f) { ok = false; break; }
       }
-      if (!ok) break;
+      tc_ld_wait();
+      // eight columns at a time: exponentiate, form dS^T, pack and store both 16-byte pieces
+      const uint32_t prow = pt_s + (uint32_t)row * 128u, drow = dst_s + (uint32_t)row * 128u;
+#pragma unroll
+      for (int g = 0; g < 4; g++) {
+        float l2[8], dl[8], pe[8], de[8];
+        *reinterpret_cast<float4*>(l2) = *reinterpret_cast<const float4*>(vs + col0 + 8 * g);
+        *reinterpret_cast<float4*>(l2 + 4) = *reinterpret_cast<const float4*>(vs + col0 + 8 * g + 4);
+        *reinterpret_cast<float4*>(dl) = *reinterpret_cast<const float4*>(vs + 64 + col0 + 8 * g);
+        *reinterpret_cast<float4*>(dl + 4) = *reinterpret_cast<const float4*>(vs + 64 + col0 + 8 * g + 4);
+#pragma unroll
+        for (int j = 0; j < 8; j++) {
+          const int e = 8 * g + j;
+          float x = ex2f(fmaf(__uint_as_float(rs[e]), p.scale_log2, -l2[j]));      // exp2(-inf) = 0 past the sequence
+          if (maskable && qcol + e < row) x = 0.f;
+          pe[j] = x;
+          de[j] = x * (__uint_as_float(rp[e]) - dl[j]);
+        }
+        const uint32_t piece = (uint32_t)((((col0 >> 3) + g) ^ (row & 7)) << 4);
+        sts_v4(prow + piece, pack_bf(pe[0], pe[1]), pack_bf(pe[2], pe[3]), pack_bf(pe[4], pe[5]), pack_bf(pe[6], pe[7]));
+        sts_v4(drow + piece, pack_bf(de[0], de[1]), pack_bf(de[2], de[3]), pack_bf(de[4], de[5]), pack_bf(de[6], de[7]));
+      }
       tc_fence_before();
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
@@ -663,8 +722,9 @@ attn_bwd_kv_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_
         tc_fence_after();
         const int t = k0 + row;
         uint32_t rv[32], rk[32];
-        tc_ld32(tm_dv + lane_off + half * 32, rv);
-        tc_ld32(tm_dk + lane_off + half * 32, rk);
+        tc_ld32_nowait(tm_dv + lane_off + half * 32, rv);
+        tc_ld32_nowait(tm_dk + lane_off + half * 32, rk);
+        tc_ld_wait();
         if (t < p.T) {
           bf16_t* out = p.dqkv + ((long long)b * p.T + t) * (3 * d) + h * DH + half * 32;
 #pragma unroll
@@ -690,12 +750,12 @@ attn_bwd_kv_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_
   __syncthreads();
   if (warp == 8) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256u) : "memory");
   }
 }
 
-constexpr size_t BWD_Q_SMEM = TILE_BYTES * 6 + P_BYTES + 128;
-constexpr size_t BWD_KV_SMEM = TILE_BYTES * 6 + 2 * P_BYTES + 2048 + 128;
+constexpr size_t BWD_Q_SMEM = TILE_BYTES * 3 + NST_Q * 2 * SUB_BYTES + 128;                 // 96.1 KB: two CTAs per SM
+constexpr size_t BWD_KV_SMEM = TILE_BYTES * 4 + NST_KV * 2 * SUB_BYTES + 1024 + 128;       // 97.1 KB: two CTAs per SM
 
 constexpr size_t FWD_SMEM = TILE_BYTES * 5 + P_BYTES + 128;   // two CTAs per SM: 2 x (112.1 KB + 1 KB reserved) <= 228 KB
 
@@ -728,12 +788,15 @@ cudaError_t attention_fwd_tc(const void* qkv, void* o, float* lse, int batch, in
   return cudaGetLastError();
 }
 
-cudaError_t attention_bwd_tc(const void* qkv, const void* dout, const float* lse, const float* delta, void* dqkv, int batch, int T,
-                             int heads, int* status, cudaStream_t s) {
+cudaError_t attention_bwd_tc(const void* qkv, const void* o, const void* dout, const float* lse, float* delta, void* dqkv, int batch,
+                             int T, int heads, int* status, cudaStream_t s) {
   const int d = heads * DH;
-  CUtensorMap map_qkv, map_do;
-  if (!tc_encode_rows_bf16(&map_qkv, qkv, 3LL * d, (long long)batch * T, 3LL * d, TQ)) return cudaErrorInvalidValue;
-  if (!tc_encode_rows_bf16(&map_do, dout, d, (long long)batch * T, d, TQ)) return cudaErrorInvalidValue;
+  const long long rows = (long long)batch * T;
+  CUtensorMap qkv128, qkv64, do128, do64, o128;        // the same matrices seen as tiles of 128 or 64 rows
+  if (!tc_encode_rows_bf16(&qkv128, qkv, 3LL * d, rows, 3LL * d, 128) || !tc_encode_rows_bf16(&qkv64, qkv, 3LL * d, rows, 3LL * d, TW) ||
+      !tc_encode_rows_bf16(&do128, dout, d, rows, d, 128) || !tc_encode_rows_bf16(&do64, dout, d, rows, d, TW) ||
+      !tc_encode_rows_bf16(&o128, o, d, rows, d, 128))
+    return cudaErrorInvalidValue;
   static std::atomic<bool> attr_set[64];
   int dev = 0;
   cudaGetDevice(&dev);
@@ -751,10 +814,11 @@ cudaError_t attention_bwd_tc(const void* qkv, const void* dout, const float* lse
   a.scale_log2 = 0.125f * LOG2E;
   a.o = nullptr; a.lse = const_cast<float*>(lse); a.delta = delta; a.dqkv = (bf16_t*)dqkv; a.status = status;
   dim3 grid((T + TQ - 1) / TQ, heads, batch);
-  attn_bwd_kv_tc_kernel<<<grid, BW_THREADS, BWD_KV_SMEM, s>>>(map_qkv, map_do, a);
+  // the dQ kernel also produces delta, which the dK/dV kernel reads: it runs first
+  attn_bwd_q_tc_kernel<<<grid, BW_THREADS, BWD_Q_SMEM, s>>>(qkv128, qkv64, do128, o128, a);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  attn_bwd_q_tc_kernel<<<grid, BW_THREADS, BWD_Q_SMEM, s>>>(map_qkv, map_do, a);
+  attn_bwd_kv_tc_kernel<<<grid, BW_THREADS, BWD_KV_SMEM, s>>>(qkv128, qkv64, do64, a);
   return cudaGetLastError();
 }
 

@@ -1090,10 +1090,8 @@ static cudaError_t attention_bwd_t(const T* qkv, const T* o, const T* dout, cons
 cudaError_t attention_bwd(const void* qkv, const void* o, const void* dout, const float* lse, float* delta,
                           void* dqkv, int batch, int T_, int heads, int dh, bool bf16, cudaStream_t s, int* status) {
   if (dh > 32 * ATT_MAXC) return cudaErrorInvalidValue;
-  if (bf16 && attention_tc_mode() && attention_tc_supported(dh, heads * dh, qkv, dout) && (reinterpret_cast<uintptr_t>(dqkv) & 15) == 0) {
-    cudaError_t e = attention_delta_bf16(o, dout, delta, batch, T_, heads, s);
-    if (e != cudaSuccess) return e;
-    return attention_bwd_tc(qkv, dout, lse, delta, dqkv, batch, T_, heads, status, s);
+  if (bf16 && attention_tc_mode() && attention_tc_supported(dh, heads * dh, qkv, dout) && ((reinterpret_cast<uintptr_t>(dqkv) | reinterpret_cast<uintptr_t>(o)) & 15) == 0) {
+    return attention_bwd_tc(qkv, o, dout, lse, delta, dqkv, batch, T_, heads, status, s);
   }
   if (bf16 && attention_mma_supported(dh, heads * dh)) return attention_bwd_mma(qkv, o, dout, lse, delta, dqkv, batch, T_, heads, s);
   return bf16 ? attention_bwd_t<bf16_t>((const bf16_t*)qkv, (const bf16_t*)o, (const bf16_t*)dout, lse, delta, (bf16_t*)dqkv, batch, T_, heads, dh, s)
@@ -1647,37 +1645,66 @@ __global__ void __launch_bounds__(256) ce_onehot_kernel(const int* __restrict__ 
   __shared__ int fill;
   const int v0 = blockIdx.x * 32;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  // adds the rows listed in list[w * stride .. w * stride + counts[w]) for w = 0..nl-1 (in that order) to this warp's four vocabulary rows
+  // Adds the rows listed in list[w * stride .. w * stride + counts[w]) for w = 0..nl-1 (in that order) to
+  // this warp's four vocabulary rows.  Per column chunk the dW loads of all four rows and the z loads
+  // of all listed rows are issued before anything is stored, so a chunk costs one memory round trip
+  // however many rows hit (the slowest warp of the launch sets its duration).
   auto work_off = [&](int nl, int stride, const int* counts) {
-    for (int i = 0; i < 4; i++) {
-      const int local = warp * 4 + i, v = v0 + local;
-      int hits = 0;
-      for (int c0 = lane * 8; c0 < d || c0 == lane * 8; c0 += 256) {      // every lane runs once (it counts the hits), d % 8 == 0
-        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-        hits = 0;
-        for (int w = 0; w < nl; w++)
-          for (int k = 0; k < counts[w]; k++) {
-            const int e = list[w * stride + k];
-            if ((e & 31) != local) continue;
-            hits++;
-            if (c0 >= d) continue;
-            const uint4 q = __ldg(reinterpret_cast<const uint4*>(z + (long long)(e >> 5) * d + c0));
-            const uint32_t x[4] = {q.x, q.y, q.z, q.w};
+    const int first = warp * 4;
+    int hits[4] = {0, 0, 0, 0};
+    for (int w = 0; w < nl; w++)
+      for (int k = 0; k < counts[w]; k++) {
+        const int local = list[w * stride + k] & 31;
 #pragma unroll
-            for (int j = 0; j < 4; j++) {
-              acc[2 * j] += __uint_as_float(x[j] << 16);
-              acc[2 * j + 1] += __uint_as_float(x[j] & 0xffff0000u);
-            }
-          }
-        if (hits && c0 < d) {
-          float4* dst = reinterpret_cast<float4*>(dW + (long long)v * d + c0);
-          float4 a = dst[0], b = dst[1];
-          a.x -= inv_rows * acc[0]; a.y -= inv_rows * acc[1]; a.z -= inv_rows * acc[2]; a.w -= inv_rows * acc[3];
-          b.x -= inv_rows * acc[4]; b.y -= inv_rows * acc[5]; b.z -= inv_rows * acc[6]; b.w -= inv_rows * acc[7];
-          dst[0] = a; dst[1] = b;
-        }
+        for (int i = 0; i < 4; i++) hits[i] += local == first + i;
       }
-      if (lane == 0 && hits) db[v] -= inv_rows * (float)hits;
+    if (!(hits[0] | hits[1] | hits[2] | hits[3])) return;
+    for (int c0 = lane * 8; c0 < d; c0 += 256) {             // d % 8 == 0
+      float4 wa[4], wb[4];
+#pragma unroll
+      for (int i = 0; i < 4; i++)
+        if (hits[i]) {
+          const float4* src = reinterpret_cast<const float4*>(dW + (long long)(v0 + first + i) * d + c0);
+          wa[i] = src[0];
+          wb[i] = src[1];
+        }
+      float acc[4][8];
+#pragma unroll
+      for (int i = 0; i < 4; i++)
+#pragma unroll
+        for (int j = 0; j < 8; j++) acc[i][j] = 0.f;
+      for (int w = 0; w < nl; w++)
+        for (int k = 0; k < counts[w]; k++) {
+          const int e = list[w * stride + k];
+          const int local = e & 31;
+          if (local < first || local >= first + 4) continue;
+          const uint4 q = __ldg(reinterpret_cast<const uint4*>(z + (long long)(e >> 5) * d + c0));
+          const uint32_t x[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+          for (int i = 0; i < 4; i++)
+            if (local == first + i) {
+#pragma unroll
+              for (int j = 0; j < 4; j++) {
+                acc[i][2 * j] += __uint_as_float(x[j] << 16);
+                acc[i][2 * j + 1] += __uint_as_float(x[j] & 0xffff0000u);
+              }
+            }
+        }
+#pragma unroll
+      for (int i = 0; i < 4; i++)
+        if (hits[i]) {
+          float4 a = wa[i], b = wb[i];
+          a.x -= inv_rows * acc[i][0]; a.y -= inv_rows * acc[i][1]; a.z -= inv_rows * acc[i][2]; a.w -= inv_rows * acc[i][3];
+          b.x -= inv_rows * acc[i][4]; b.y -= inv_rows * acc[i][5]; b.z -= inv_rows * acc[i][6]; b.w -= inv_rows * acc[i][7];
+          float4* dst = reinterpret_cast<float4*>(dW + (long long)(v0 + first + i) * d + c0);
+          dst[0] = a;
+          dst[1] = b;
+        }
+    }
+    if (lane == 0) {
+#pragma unroll
+      for (int i = 0; i < 4; i++)
+        if (hits[i]) db[v0 + first + i] -= inv_rows * (float)hits[i];
     }
   };
   // fast path: every warp compacts its own eighth of the rows, 128 targets per step (one 16-byte

@@ -123,9 +123,9 @@ cudaError_t attention_bwd(const void* qkv, const void* o, const void* dout, cons
 // the model's device status word (bounded waits), may be null.
 bool attention_tc_supported(int dh, int d, const void* qkv, const void* o);
 cudaError_t attention_fwd_tc(const void* qkv, void* o, float* lse, int batch, int T, int heads, int* status, cudaStream_t s);
-// dqkv from dout, lse and delta (delta[b,h,t] = sum_c dout * o over the head's 64 columns, see attention_delta_bf16)
-cudaError_t attention_bwd_tc(const void* qkv, const void* dout, const float* lse, const float* delta, void* dqkv, int batch, int T,
-                             int heads, int* status, cudaStream_t s);
+// dqkv from dout, o and lse; delta [batch*heads*T] is scratch (delta[b,h,t] = sum_c dout * o over the head's 64 columns)
+cudaError_t attention_bwd_tc(const void* qkv, const void* o, const void* dout, const float* lse, float* delta, void* dqkv, int batch,
+                             int T, int heads, int* status, cudaStream_t s);
 cudaError_t attention_delta_bf16(const void* o, const void* dout, float* delta, int batch, int T, int heads, cudaStream_t s);
 
 // Tensor-core versions (mma.sync m16n8k16) for bf16 with 64-wide heads; same contracts.
