@@ -681,9 +681,10 @@ struct Builder {
 
   // ---- softmax cross-entropy head whose loss and gradient never read the logits back ------------
   // (bf16 models whose head GEMM runs on the tensor cores; the kernels are described in kernels.cu).
-  // Forward: target logit -> head GEMM with the exp epilogue (P and partial sums) -> finalize ->
-  // exact recomputation of unsafe rows (normally none) -> mean loss.  Backward: dW_h and db_h from
-  // P and the scaled copy of z, the one-hot part added in row order, dz from P W_h.
+  // Forward: target logit -> head GEMM with the exp epilogue (P and partial sums) -> finalize (loss,
+  // row scales, one patched element of P per row) -> exact recomputation of unsafe rows (normally
+  // none) -> mean loss.  Backward: the gradient of the logits is (row scale) (.) P, so dW_h comes from P
+  // and the scaled copy of z, db_h from a weighted column sum of P, dz from P W_h.
   // Returns false (nothing enqueued) when the head does not qualify: the caller then takes the
   // path with a separate softmax pass.
   bool head_ce_exp(int /*b*/, const void* z, int d, int wh, int bh, void* logits, int V, int T_, float* rowloss, float* loss_out,
@@ -729,16 +730,15 @@ struct Builder {
     note(f, "ce_target_logit", 2.0 * rows * d, 4.0 * rows * d);
     f.push_back({[g, plan, mm](cudaStream_t s) { return tc_gemm_launch(g, plan, s, mm->sm_budget); }, 1});
     note(f, "gemm_fwd", 2.0 * rows * V * d, ((double)rows * d + (double)V * d) * 2 + 2.0 * rows * V);
-    f.push_back({[=](cudaStream_t s) { return ce_finalize(psum, groups, ref, lt, z, zs, rowloss, rowscale, bad, rows, d, inv, s); }, 1});
+    f.push_back({[=](cudaStream_t s) { return ce_finalize(psum, groups, ref, lt, tgt, logits, V, z, zs, rowloss, rowscale, bad, rows, d, inv, s); }, 1});
     note(f, "ce_finalize", (double)rows * groups, 4.0 * rows * groups + 4.0 * rows * d);
-    f.push_back({[=](cudaStream_t s) { return ce_fixup(bad, mm->status, z, Wb, bias, logits, ref, lt, zs, rowloss, rowscale, rows, d, V, inv, s); }, 1});
+    f.push_back({[=](cudaStream_t s) { return ce_fixup(bad, mm->status, tgt, z, Wb, bias, logits, ref, lt, zs, rowloss, rowscale, rows, d, V, inv, s); }, 1});
     note(f, "ce_fixup", 0, 0);
     f.push_back({[=](cudaStream_t s) { return reduce_sum(rowloss, rows, inv, loss_out, s); }, 1});
     note(f, "loss_reduce", rows, 4.0 * rows);
     // backward: parameter gradients (leaves) ...
     const size_t before = bw.size();
     lin_wgrad(bw, logits, zs, d, wh, -1, rows, V, d, true);
-    flush_group(bw);           // a small head's weight gradient may have joined a group: the one-hot part follows it
     {
       const int chunks = colsum_chunks(rows, V);
       float* ws = chunks > 1 ? f32_buf((size_t)chunks * V) : nullptr;
@@ -747,12 +747,8 @@ struct Builder {
       bw.push_back({[=](cudaStream_t s) { return colsum(logits, true, V, rows, V, rowscale, ws, chunks, tk, out, s); }, 1});
       note(bw, "colsum", 2.0 * rows * V, 2.0 * rows * V);
     }
-    float* dW = G(wh);
-    float* db = G(bh);
-    bw.push_back({[=](cudaStream_t s) { return ce_onehot(tgt, z, dW, db, rows, d, V, inv, s); }, 1});
-    note(bw, "ce_onehot", 2.0 * rows * d, 4.0 * rows + 2.0 * rows * d);
     for (size_t i = before; i < bw.size(); i++) bw[i].leaf = true;
-    // ... and the gradient chain: dz = r (.) (P W_h) - W_h[t]/N from fp32 partials of the GEMM
+    // ... and the gradient chain: dz = r (.) (P W_h) from fp32 partials of the GEMM
     GemmArgs q;
     q.M = rows; q.N = d; q.K = V;
     q.A = logits; q.sa_m = V; q.sa_k = 1;
@@ -776,7 +772,7 @@ struct Builder {
     bw.push_back({[=](cudaStream_t s) {
                     cudaError_t e = q_tc ? tc_gemm_launch(q, qplan, s, mm->sm_budget) : gemm_simt(q, true, s);
                     if (e != cudaSuccess) return e;
-                    return ce_dz_finish(part, splits, rows, d, rowscale, tgt, Wb, dz, inv, s);
+                    return ce_dz_finish(part, splits, rows, d, rowscale, dz, s);
                   }, 2});
     note(bw, "gemm_dgrad", 2.0 * rows * V * d, ((double)rows * V + (double)V * d) * 2 + 2.0 * rows * d);
     return true;

@@ -1466,11 +1466,10 @@ cudaError_t softmax_ce_inplace(void* logits, const int32_t* ids, int T_, float* 
 // P[n,v] = exp(l[n,v] - c_n) (bf16) instead of the logit and leaves fp32 partial sums of the
 // unrounded exponentials.  Then, with S_n = sum_v exp(l[n,v] - c_n):
 //     lse_n = c_n + log S_n,      loss_n = lse_n - l[n,t_n],
-//     dl[n,v] = (softmax - onehot)/N = P[n,v] * r_n - [v = t_n]/N,     r_n = 1 / (S_n N),
-// so the backward GEMMs consume P directly:
-//     dW_h = P^T (r (.) z)  -  (1/N) sum_n onehot(t_n) z_n^T        (rows of z added to rows t_n)
-//     dz_n = r_n (P W_h)_n  -  (1/N) W_h[t_n, :]
-//     db_h = sum_n r_n P[n,:]  -  count(t = v)/N.
+//     dl[n,v] = (softmax - onehot)/N = r_n * (P[n,v] - S_n [v = t_n]),     r_n = 1 / (S_n N).
+// The finalize kernel therefore patches ONE element per row, P[n,t_n] <- P[n,t_n] - S_n, and from
+// then on the gradient of the logits is r (.) P: the backward GEMMs consume P directly,
+//     dW_h = P^T (r (.) z),     dz_n = r_n (P W_h)_n,     db_h = sum_n r_n P[n,:].
 // c_n is the target's own logit (z_n . W_h[t_n] + b_h[t_n], a gather and a dot product): it is at
 // most the row maximum, and it is far enough below it to endanger the exponent range only when the
 // token's loss exceeds ~69 nats.  Such rows (S_n >= 1e30 or not finite) are listed by the finalize
@@ -1530,10 +1529,12 @@ __device__ __forceinline__ void scale_row_bf16(const bf16_t* __restrict__ z, bf1
 }
 
 // One warp per row: S_n from the GEMM's partial sums (lanes stride over the groups, then a fixed
-// shuffle tree), loss_n, r_n, the scaled copy r_n z_n for the weight-gradient GEMM; rows whose sum
-// left the safe range are appended to the list bad[1..] (count in bad[0]).
+// shuffle tree), loss_n, r_n, the patch P[n,t_n] -= S_n, the scaled copy r_n z_n for the
+// weight-gradient GEMM; rows whose sum left the safe range are appended to the list bad[1..]
+// (count in bad[0]).
 __global__ void __launch_bounds__(256) ce_finalize_kernel(const float* __restrict__ psum, int groups, const float* __restrict__ ref,
-                                                          const float* __restrict__ lt, const bf16_t* __restrict__ z,
+                                                          const float* __restrict__ lt, const int* __restrict__ tgt,
+                                                          bf16_t* __restrict__ P, int V, const bf16_t* __restrict__ z,
                                                           bf16_t* __restrict__ zs, float* __restrict__ rowloss,
                                                           float* __restrict__ rowscale, int* __restrict__ bad, int rows, int d,
                                                           float inv_rows) {
@@ -1548,7 +1549,8 @@ __global__ void __launch_bounds__(256) ce_finalize_kernel(const float* __restric
     if (lane == 0) {
       rowloss[n] = ok ? ref[n] + logf(S) - lt[n] : 0.f;
       rowscale[n] = r;
-      if (!ok) bad[1 + atomicAdd(bad, 1)] = n;
+      if (ok) P[(long long)n * V + tgt[n]] = __float2bfloat16_rn(expf(lt[n] - ref[n]) - S);   // the one-hot part of the gradient
+      else bad[1 + atomicAdd(bad, 1)] = n;
     }
     scale_row_bf16(z + (long long)n * d, zs + (long long)n * d, d, r, lane);
   }
@@ -1558,8 +1560,8 @@ __global__ void __launch_bounds__(256) ce_finalize_kernel(const float* __restric
 // recomputed from z_n and the head's operands (twice: maximum, then exponentials), P[n,:] is
 // rewritten relative to the true maximum, and loss_n, r_n and the scaled copy of z_n follow.
 // Every quantity of a row depends on that row alone, so the order of the list does not matter.
-__global__ void __launch_bounds__(256) ce_fixup_kernel(const int* __restrict__ bad, const int* __restrict__ status, const bf16_t* __restrict__ z,
-                                                       const bf16_t* __restrict__ W, const float* __restrict__ bias,
+__global__ void __launch_bounds__(256) ce_fixup_kernel(const int* __restrict__ bad, const int* __restrict__ status, const int* __restrict__ tgt,
+                                                       const bf16_t* __restrict__ z, const bf16_t* __restrict__ W, const float* __restrict__ bias,
                                                        bf16_t* __restrict__ P, float* __restrict__ ref, const float* __restrict__ lt,
                                                        bf16_t* __restrict__ zs, float* __restrict__ rowloss,
                                                        float* __restrict__ rowscale, int d, int V, float inv_rows) {
@@ -1597,191 +1599,30 @@ __global__ void __launch_bounds__(256) ce_fixup_kernel(const int* __restrict__ b
 #pragma unroll
     for (int w = 1; w < 8; w++) S += red[w];
     const float r = inv_rows / S;
-    if (threadIdx.x == 0) {
+    if (threadIdx.x == 0) {      // (the barrier above ordered every warp's writes of P before this patch)
       ref[n] = mx;
       rowloss[n] = mx + logf(S) - lt[n];
       rowscale[n] = r;
+      P[(long long)n * V + tgt[n]] = __float2bfloat16_rn(expf(lt[n] - mx) - S);
     }
     if (warp == 0) scale_row_bf16(z + (long long)n * d, zs + (long long)n * d, d, r, lane);
     __syncthreads();
   }
 }
 
-// dz[n,c] = r_n * sum_s part[s][n,c] - W[t_n,c]/N   (partials in split order; rounded to bf16 once)
+// dz[n,c] = r_n * sum_s part[s][n,c]   (partials of P W_h in split order; rounded to bf16 once)
 __global__ void __launch_bounds__(256) ce_dz_finish_kernel(const float4* __restrict__ part, int splits, long long mn4, int d4,
-                                                           const float* __restrict__ rowscale, const int* __restrict__ tgt,
-                                                           const bf16_t* __restrict__ W, bf16_t* __restrict__ dz, float inv_rows) {
+                                                           const float* __restrict__ rowscale, bf16_t* __restrict__ dz) {
   const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
   if (i >= mn4) return;
-  const int n = (int)(i / d4), c = (int)(i - (long long)n * d4) * 4;
+  const int n = (int)(i / d4);
   float4 a = part[i];
   for (int s = 1; s < splits; s++) {
     const float4 b = part[(long long)s * mn4 + i];
     a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
   }
   const float r = rowscale[n];
-  const uint2 wq = *reinterpret_cast<const uint2*>(W + (long long)tgt[n] * (d4 * 4) + c);
-  const float w0 = __uint_as_float(wq.x << 16), w1 = __uint_as_float(wq.x & 0xffff0000u);
-  const float w2 = __uint_as_float(wq.y << 16), w3 = __uint_as_float(wq.y & 0xffff0000u);
-  store4(dz + (long long)n * (d4 * 4) + c,
-         make_float4(fmaf(a.x, r, -inv_rows * w0), fmaf(a.y, r, -inv_rows * w1), fmaf(a.z, r, -inv_rows * w2), fmaf(a.w, r, -inv_rows * w3)));
-}
-
-// The one-hot part of the head's gradients: dW[t_n,:] -= z_n/N and db[t_n] -= 1/N for every row n.
-// A CTA owns 32 vocabulary rows.  Each of its 8 warps scans one eighth of the targets (in row order,
-// no block-wide synchronisation) and keeps the rows that hit the CTA's range in its own list; the
-// eight lists read one after the other are in row order.  Then each warp takes four of the
-// vocabulary rows and, for each, adds up the listed rows of z in that order in registers (the loads
-// are independent of one another) and updates dW once.  Rows of z that meet in one vocabulary row
-// are therefore always added in the same order: no atomics, the same bits on every run.  If a list
-// overflows (many rows share few targets) the CTA falls back to a block-wide ordered compaction
-// that works its list off whenever it fills up.
-constexpr int CE_SUB = 120;       // entries per warp list (fast path)
-constexpr int CE_LIST = 8 * CE_SUB;
-__global__ void __launch_bounds__(256) ce_onehot_kernel(const int* __restrict__ tgt, const bf16_t* __restrict__ z, float* __restrict__ dW,
-                                                        float* __restrict__ db, int rows, int d, float inv_rows) {
-  __shared__ int list[CE_LIST];     // row index * 32 + (target - v0)
-  __shared__ int wcount[8];
-  __shared__ int fill;
-  const int v0 = blockIdx.x * 32;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  // Adds the rows listed in list[w * stride .. w * stride + counts[w]) for w = 0..nl-1 (in that order) to
-  // this warp's four vocabulary rows.  Per column chunk the dW loads of all four rows and the z loads
-  // of all listed rows are issued before anything is stored, so a chunk costs one memory round trip
-  // however many rows hit (the slowest warp of the launch sets its duration).
-  auto work_off = [&](int nl, int stride, const int* counts) {
-    const int first = warp * 4;
-    int hits[4] = {0, 0, 0, 0};
-    for (int w = 0; w < nl; w++)
-      for (int k = 0; k < counts[w]; k++) {
-        const int local = list[w * stride + k] & 31;
-#pragma unroll
-        for (int i = 0; i < 4; i++) hits[i] += local == first + i;
-      }
-    if (!(hits[0] | hits[1] | hits[2] | hits[3])) return;
-    for (int c0 = lane * 8; c0 < d; c0 += 256) {             // d % 8 == 0
-      float4 wa[4], wb[4];
-#pragma unroll
-      for (int i = 0; i < 4; i++)
-        if (hits[i]) {
-          const float4* src = reinterpret_cast<const float4*>(dW + (long long)(v0 + first + i) * d + c0);
-          wa[i] = src[0];
-          wb[i] = src[1];
-        }
-      float acc[4][8];
-#pragma unroll
-      for (int i = 0; i < 4; i++)
-#pragma unroll
-        for (int j = 0; j < 8; j++) acc[i][j] = 0.f;
-      for (int w = 0; w < nl; w++)
-        for (int k = 0; k < counts[w]; k++) {
-          const int e = list[w * stride + k];
-          const int local = e & 31;
-          if (local < first || local >= first + 4) continue;
-          const uint4 q = __ldg(reinterpret_cast<const uint4*>(z + (long long)(e >> 5) * d + c0));
-          const uint32_t x[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-          for (int i = 0; i < 4; i++)
-            if (local == first + i) {
-#pragma unroll
-              for (int j = 0; j < 4; j++) {
-                acc[i][2 * j] += __uint_as_float(x[j] << 16);
-                acc[i][2 * j + 1] += __uint_as_float(x[j] & 0xffff0000u);
-              }
-            }
-        }
-#pragma unroll
-      for (int i = 0; i < 4; i++)
-        if (hits[i]) {
-          float4 a = wa[i], b = wb[i];
-          a.x -= inv_rows * acc[i][0]; a.y -= inv_rows * acc[i][1]; a.z -= inv_rows * acc[i][2]; a.w -= inv_rows * acc[i][3];
-          b.x -= inv_rows * acc[i][4]; b.y -= inv_rows * acc[i][5]; b.z -= inv_rows * acc[i][6]; b.w -= inv_rows * acc[i][7];
-          float4* dst = reinterpret_cast<float4*>(dW + (long long)(v0 + first + i) * d + c0);
-          dst[0] = a;
-          dst[1] = b;
-        }
-    }
-    if (lane == 0) {
-#pragma unroll
-      for (int i = 0; i < 4; i++)
-        if (hits[i]) db[v0 + first + i] -= inv_rows * (float)hits[i];
-    }
-  };
-  // fast path: every warp compacts its own eighth of the rows, 128 targets per step (one 16-byte
-  // load per lane, two steps in flight), written to the list in row order (lane-major, then the
-  // four components) through a warp prefix sum of the per-lane hit counts
-  {
-    const int per = ((rows + 7) / 8 + 127) / 128 * 128, lo = warp * per, hi = min(rows, lo + per);
-    const int4* t4 = reinterpret_cast<const int4*>(tgt);
-    int cnt = 0;
-    bool over = false;
-    auto fetch = [&](int base) {
-      const int n0 = base + 4 * lane;
-      return n0 < hi ? __ldg(t4 + (n0 >> 2)) : make_int4(-1, -1, -1, -1);    // tgt is padded to a multiple of 64 entries
-    };
-    auto take = [&](int base, int4 q) {
-      const int n0 = base + 4 * lane;
-      const int t[4] = {q.x, q.y, q.z, q.w};
-      bool hit[4];
-      int mine = 0;
-#pragma unroll
-      for (int j = 0; j < 4; j++) {
-        hit[j] = n0 + j < hi && t[j] >= v0 && t[j] < v0 + 32;
-        mine += hit[j];
-      }
-      int incl = mine;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int up = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += up;
-      }
-      const int total = __shfl_sync(0xffffffffu, incl, 31);
-      if (cnt + total > CE_SUB) { over = true; return; }
-      int pos = warp * CE_SUB + cnt + incl - mine;
-#pragma unroll
-      for (int j = 0; j < 4; j++)
-        if (hit[j]) list[pos++] = (n0 + j) * 32 + (t[j] - v0);
-      cnt += total;
-    };
-    for (int base = lo; base < hi && !over; base += 256) {
-      const int4 qa = fetch(base), qb = fetch(base + 128);
-      take(base, qa);
-      if (!over && base + 128 < hi) take(base + 128, qb);
-    }
-    if (lane == 0) wcount[warp] = cnt;
-    if (!__syncthreads_or(over)) {
-      work_off(8, CE_SUB, wcount);
-      return;
-    }
-  }
-  // slow path: block-wide ordered compaction, 256 targets at a time, worked off when the list fills up
-  __syncthreads();
-  if (threadIdx.x == 0) fill = 0;
-  __syncthreads();
-  for (int base = 0; base < rows; base += 256) {
-    const int n = base + threadIdx.x;
-    const int t = n < rows ? tgt[n] : -1;
-    const bool hit = t >= v0 && t < v0 + 32;
-    const unsigned m = __ballot_sync(0xffffffffu, hit);
-    if (lane == 0) wcount[warp] = __popc(m);
-    __syncthreads();
-    int off = fill, total = 0;
-#pragma unroll
-    for (int w = 0; w < 8; w++) {
-      if (w < warp) off += wcount[w];
-      total += wcount[w];
-    }
-    if (hit) list[off + __popc(m & ((1u << lane) - 1u))] = n * 32 + (t - v0);
-    __syncthreads();
-    if (threadIdx.x == 0) fill += total;
-    __syncthreads();
-    if (fill > CE_LIST - 256 || base + 256 >= rows) {      // the next 256 targets might not fit, or these were the last
-      work_off(1, 0, &fill);
-      __syncthreads();
-      if (threadIdx.x == 0) fill = 0;
-      __syncthreads();
-    }
-  }
+  store4(dz + i * 4, make_float4(a.x * r, a.y * r, a.z * r, a.w * r));
 }
 
 cudaError_t ce_target_logit(const void* z, const void* W, const float* bias, const int32_t* ids, int T_, int rows, int d, int V,
@@ -1790,28 +1631,23 @@ cudaError_t ce_target_logit(const void* z, const void* W, const float* bias, con
   ce_target_logit_kernel<<<grid, 256, 0, s>>>((const bf16_t*)z, (const bf16_t*)W, bias, ids, T_, rows, d, V, tgt, ref, lt, bad);
   return cudaGetLastError();
 }
-cudaError_t ce_finalize(const float* psum, int groups, const float* ref, const float* lt, const void* z, void* zs, float* rowloss,
-                        float* rowscale, int* bad, int rows, int d, float inv_rows, cudaStream_t s) {
+cudaError_t ce_finalize(const float* psum, int groups, const float* ref, const float* lt, const int* tgt, void* P, int V, const void* z,
+                        void* zs, float* rowloss, float* rowscale, int* bad, int rows, int d, float inv_rows, cudaStream_t s) {
   const int grid = (int)std::min<long long>(cdiv(rows, 8), 148 * 8);
-  ce_finalize_kernel<<<grid, 256, 0, s>>>(psum, groups, ref, lt, (const bf16_t*)z, (bf16_t*)zs, rowloss, rowscale, bad, rows, d, inv_rows);
+  ce_finalize_kernel<<<grid, 256, 0, s>>>(psum, groups, ref, lt, tgt, (bf16_t*)P, V, (const bf16_t*)z, (bf16_t*)zs, rowloss, rowscale, bad,
+                                          rows, d, inv_rows);
   return cudaGetLastError();
 }
-cudaError_t ce_fixup(const int* bad, const int* status, const void* z, const void* W, const float* bias, void* P, float* ref, const float* lt, void* zs,
-                     float* rowloss, float* rowscale, int rows, int d, int V, float inv_rows, cudaStream_t s) {
+cudaError_t ce_fixup(const int* bad, const int* status, const int* tgt, const void* z, const void* W, const float* bias, void* P, float* ref,
+                     const float* lt, void* zs, float* rowloss, float* rowscale, int rows, int d, int V, float inv_rows, cudaStream_t s) {
   const int grid = rows < 32 ? rows : 32;
-  ce_fixup_kernel<<<grid, 256, 0, s>>>(bad, status, (const bf16_t*)z, (const bf16_t*)W, bias, (bf16_t*)P, ref, lt, (bf16_t*)zs, rowloss, rowscale,
-                                       d, V, inv_rows);
+  ce_fixup_kernel<<<grid, 256, 0, s>>>(bad, status, tgt, (const bf16_t*)z, (const bf16_t*)W, bias, (bf16_t*)P, ref, lt, (bf16_t*)zs, rowloss,
+                                       rowscale, d, V, inv_rows);
   return cudaGetLastError();
 }
-cudaError_t ce_dz_finish(const float* part, int splits, int rows, int d, const float* rowscale, const int* tgt, const void* W,
-                         void* dz, float inv_rows, cudaStream_t s) {
+cudaError_t ce_dz_finish(const float* part, int splits, int rows, int d, const float* rowscale, void* dz, cudaStream_t s) {
   const long long mn4 = (long long)rows * d / 4;
-  ce_dz_finish_kernel<<<cdiv(mn4, 256), 256, 0, s>>>((const float4*)part, splits, mn4, d / 4, rowscale, tgt, (const bf16_t*)W,
-                                                    (bf16_t*)dz, inv_rows);
-  return cudaGetLastError();
-}
-cudaError_t ce_onehot(const int* tgt, const void* z, float* dW, float* db, int rows, int d, int V, float inv_rows, cudaStream_t s) {
-  ce_onehot_kernel<<<cdiv(V, 32), 256, 0, s>>>(tgt, (const bf16_t*)z, dW, db, rows, d, inv_rows);
+  ce_dz_finish_kernel<<<cdiv(mn4, 256), 256, 0, s>>>((const float4*)part, splits, mn4, d / 4, rowscale, (bf16_t*)dz);
   return cudaGetLastError();
 }
 

@@ -150,19 +150,17 @@ cudaError_t softmax_ce_inplace(void* logits, const int32_t* ids, int T, float* r
 // Softmax cross-entropy head without a pass over the logits (bf16, d % 8 == 0): see kernels.cu.
 //   ce_target_logit  tgt[n] (clamped), ref[n] = lt[n] = z_n . W[t_n] + bias[t_n]; clears bad[0]
 //   (head GEMM with Epilogue::ce_ref = ref writes P = exp(l - ref) and the partial sums psum)
-//   ce_finalize      rowloss, rowscale r_n = 1/(S_n rows), zs = r (.) z; unsafe rows -> bad[1..], bad[0] = count
+//   ce_finalize      rowloss, rowscale r_n = 1/(S_n rows), P[n,t_n] -= S_n, zs = r (.) z; unsafe rows -> bad[1..], bad[0] = count
 //   ce_fixup         recomputes the listed rows exactly (no-op when bad[0] == 0 or *status != 0); bad holds rows+1 ints
-//   ce_dz_finish     dz = r_n * (sum of `splits` fp32 partials of P W) - W[t_n]/rows, rounded once
-//   ce_onehot        dW[t_n,:] -= z_n/rows, db[t_n] -= 1/rows in row order (after the GEMM part of dW, db)
+//   ce_dz_finish     dz = r_n * (sum of `splits` fp32 partials of P W), rounded once
+// after which the gradient of the logits is r (.) P: dW = P^T zs, db = column sums of P weighted by r.
 cudaError_t ce_target_logit(const void* z, const void* W, const float* bias, const int32_t* ids, int T, int rows, int d, int V,
                             int* tgt, float* ref, float* lt, int* bad, cudaStream_t s);
-cudaError_t ce_finalize(const float* psum, int groups, const float* ref, const float* lt, const void* z, void* zs, float* rowloss,
-                        float* rowscale, int* bad, int rows, int d, float inv_rows, cudaStream_t s);
-cudaError_t ce_fixup(const int* bad, const int* status, const void* z, const void* W, const float* bias, void* P, float* ref, const float* lt, void* zs,
-                     float* rowloss, float* rowscale, int rows, int d, int V, float inv_rows, cudaStream_t s);
-cudaError_t ce_dz_finish(const float* part, int splits, int rows, int d, const float* rowscale, const int* tgt, const void* W,
-                         void* dz, float inv_rows, cudaStream_t s);
-cudaError_t ce_onehot(const int* tgt, const void* z, float* dW, float* db, int rows, int d, int V, float inv_rows, cudaStream_t s);
+cudaError_t ce_finalize(const float* psum, int groups, const float* ref, const float* lt, const int* tgt, void* P, int V, const void* z,
+                        void* zs, float* rowloss, float* rowscale, int* bad, int rows, int d, float inv_rows, cudaStream_t s);
+cudaError_t ce_fixup(const int* bad, const int* status, const int* tgt, const void* z, const void* W, const float* bias, void* P, float* ref,
+                     const float* lt, void* zs, float* rowloss, float* rowscale, int rows, int d, int V, float inv_rows, cudaStream_t s);
+cudaError_t ce_dz_finish(const float* part, int splits, int rows, int d, const float* rowscale, void* dz, cudaStream_t s);
 
 // out[0] = (sum of v[0..n)) * scale, fixed-order tree in one CTA.
 cudaError_t reduce_sum(const float* v, int n, float scale, float* out, cudaStream_t s);
