@@ -170,6 +170,18 @@ typedef struct {
                             staging: up to n_streams-1 blocks train side by side.  Wider than the
                             paper's overlap of B_b with F_{b+1} (Section 2.2); same kernels, same bits. */
 
+#define ERASE_PERSISTENT 128u /* co-schedule F_{b+1} and B_b inside ONE persistent kernel on a partition of the SMs
+                            (Section 2.2: B_b overlaps F_{b+1}; Sections 1 and 3.1: small GEMMs leave SMs idle and
+                            can share the device).  The step runs on the main stream alone, n_streams is
+                            ignored: stage s launches one dual-list kernel whose first share of the CTAs works
+                            through the GEMMs and GELU passes of F_s and the rest through those of B_{s-1}, each
+                            list in order with device-side completion counters between dependent problems; the
+                            heads, losses, reductions and the optimizer stay ordinary launches between stages.
+                            Same tile arithmetic in the same order: same bits as the serial schedule.  Available
+                            for bf16 chains of MLP / tower blocks (the saturation-sweep models); other models get
+                            ERASE_EUNSUPPORTED with the reason in erase_last_error().  May be combined with
+                            ERASE_GRAPH and ERASE_NO_OPT; the stream-placement flags are ignored.          */
+
 /* Device bytes erase_create needs for this spec when given an arena; 0 if the spec is invalid. */
 ERASE_API size_t erase_arena_bytes(const erase_model_spec* spec);
 

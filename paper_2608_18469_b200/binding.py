@@ -16,7 +16,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "liberase_b200.so")
 
 OK, EINVAL, ENOMEM, ECUDA, ESTATE, ETIMEOUT, EUNSUPPORTED = range(7)
-GRAPH, NO_OPT, EARLY_HEAD, BLOCK_OPT, SPLIT_BWD, STAMPS, PAR_FWD = 1, 2, 4, 8, 16, 32, 64
+GRAPH, NO_OPT, EARLY_HEAD, BLOCK_OPT, SPLIT_BWD, STAMPS, PAR_FWD, PERSISTENT = 1, 2, 4, 8, 16, 32, 64, 128
 MAX_DIMS = 8
 
 _DTYPE = {"f32": 0, "bf16": 1}

@@ -32,6 +32,14 @@ struct Op {
   double flops = 0;         // algorithmic floating-point operations of one run
   double bytes = 0;         // algorithmic bytes (each operand read once, each result written once)
   bool leaf = false;        // backward op that only produces parameter gradients: nothing in B_b reads its output
+  // What the persistent schedule needs to run this operation inside the dual-list kernel instead:
+  std::vector<GemmArgs> pg;                              // the tensor-core GEMMs it consists of ...
+  std::function<cudaError_t(cudaStream_t)> post;         // ... and what follows them (split-K reduction), if anything
+  int post_launches = 0;
+  int pew = 0;                                           // 1: ew_dst = gelu(ew_src), 2: ew_dst *= gelu'(ew_src)  (bf16)
+  const void* ew_src = nullptr;
+  void* ew_dst = nullptr;
+  long long ew_n = 0;
 };
 typedef std::vector<Op> OpList;
 
@@ -103,6 +111,18 @@ struct erase_model {
   std::vector<OpList> fwd, hfwd, bwd;  // per block: body forward, local head + loss, backward
   erase_batch cur = {nullptr, nullptr, nullptr};
   std::map<GraphKey, std::pair<cudaGraphExec_t, int64_t>> graphs;   // executable graph and the kernels it launches
+
+  // Persistent schedule (ERASE_PERSISTENT): stage s runs F_s and B_{s-1} in one dual-list kernel.
+  struct PStage {
+    std::vector<Op*> pre;        // operations of B_{s-1} in front of its first tensor-core GEMM (head dz, its reductions)
+    TcDualPlan* plan = nullptr;
+    std::vector<Op*> covered;    // operations whose GEMMs / elementwise passes run inside the kernel (their `post` follows it)
+    std::vector<Op*> after;      // parameter-gradient leaves of B_{s-1} that stay ordinary launches
+  };
+  std::vector<PStage> pstage;
+  int* pdone = nullptr;          // device counters of the dual-list kernels, tc_dual_max() per stage
+  bool persistent_ok = false;
+  std::string persistent_why;
 
   int sm_budget = 0;   // CTA cap for persistent GEMMs enqueued next (0 = all SMs); set per stream by the scheduler
   int64_t launches = 0;
@@ -401,14 +421,18 @@ struct Builder {
     const bool use_tc = tc_ok && !m->dry && tc_gemm_plan(g, m->status, &plan);
     plan.sched = sched;
     if (use_tc) {
-      if (g.splits > 1)
+      if (g.splits > 1) {
         ops.push_back({[g, plan, out, ldo, out_bf, mm = m](cudaStream_t s) {
                          cudaError_t e = tc_gemm_launch(g, plan, s, mm->sm_budget);
                          if (e != cudaSuccess) return e;
                          return splitk_reduce(g.ws, g.splits, (long long)g.M * g.N, g.N, out, ldo, s, out_bf);
                        }, 2});
-      else
+        ops.back().post = [g, out, ldo, out_bf](cudaStream_t s) { return splitk_reduce(g.ws, g.splits, (long long)g.M * g.N, g.N, out, ldo, s, out_bf); };
+        ops.back().post_launches = 1;
+      } else {
         ops.push_back({[g, plan, mm = m](cudaStream_t s) { return tc_gemm_launch(g, plan, s, mm->sm_budget); }, 1});
+      }
+      ops.back().pg = {g};
       return;
     }
     if (g.splits > 1) {
@@ -429,11 +453,13 @@ struct Builder {
     bool bf = m->bf16;
     ops.push_back({[=](cudaStream_t s) { return ew_act(u, y, act, n, bf, s); }, 1});
     note(ops, "ew_act", 10.0 * n, 2.0 * n * m->esz);
+    if (bf && act == ACT_GELU) { ops.back().pew = 1; ops.back().ew_src = u; ops.back().ew_dst = y; ops.back().ew_n = n; }
   }
   void dact_op(OpList& ops, void* d, const void* src, int act, long long n) {
     bool bf = m->bf16;
     ops.push_back({[=](cudaStream_t s) { return ew_dact(d, src, act, n, bf, s); }, 1});
     note(ops, "ew_dact", 10.0 * n, 3.0 * n * m->esz);
+    if (bf && act == ACT_GELU) { ops.back().pew = 2; ops.back().ew_src = src; ops.back().ew_dst = d; ops.back().ew_n = n; }
   }
 
   // Y[M,N] = epi(X[M,K] W[N,K]^T)
@@ -574,6 +600,11 @@ struct Builder {
                      }, n + 1});
     note(ops, "gemm_wgrad", flops, bytes);
     ops.back().leaf = true;
+    if (planned) {
+      ops.back().pg = gs;
+      ops.back().post = [dev, n, total](cudaStream_t s) { return reduce_batch(dev, n, total, s); };
+      ops.back().post_launches = 1;
+    }
     group.clear();
   }
 
@@ -1009,6 +1040,7 @@ struct Builder {
     m->status = (int*)dev_alloc(m, sizeof(int), &ok);
     m->losses = f32_buf(m->B);
     m->stamps = (unsigned long long*)dev_alloc(m, (size_t)(2 * (2 * m->B + 1) + 1) * sizeof(unsigned long long), &ok);
+    m->pdone = (int*)dev_alloc(m, (size_t)(m->B + 1) * tc_dual_max() * sizeof(int), &ok);
     // z_0
     // z_0: dense batches are copied into a model-owned buffer (so every block reads memory whose
     // address is fixed at build time); token and CTR batches are gathered from the frozen tables.
@@ -1126,6 +1158,74 @@ cudaError_t run_ops(erase_model* m, OpList& ops, cudaStream_t s) {
     m->launches += op.launches;
   }
   return cudaSuccess;
+}
+
+// Persistent schedule: which operations of F_s and B_{s-1} go into stage s's dual-list kernel.
+// Qualifies: bf16 chains whose block bodies consist of tensor-core GEMMs and GELU passes (MLP and
+// tower blocks); anything else leaves persistent_ok false with the reason in persistent_why.
+void plan_persistent(erase_model* m) {
+  m->persistent_ok = false;
+  if (!m->bf16) { m->persistent_why = "the persistent schedule needs a bf16 model"; return; }
+  if (m->spec.topo != ERASE_TOPO_CHAIN) { m->persistent_why = "the persistent schedule needs a chain of blocks"; return; }
+  const int B = m->B;
+  m->pstage.assign(B + 1, erase_model::PStage());
+  auto capable = [](const Op& op) { return !op.pg.empty() || op.pew != 0; };
+  for (int s = 0; s <= B; s++) {
+    erase_model::PStage& st = m->pstage[s];
+    std::vector<DualItem> items;
+    auto add = [&](Op& op, int list) {
+      if (op.pew) {
+        DualItem it;
+        it.kind = op.pew; it.ew_src = op.ew_src; it.ew_dst = op.ew_dst; it.ew_n = op.ew_n; it.list = list; it.leaf = op.leaf ? 1 : 0;
+        items.push_back(it);
+      } else {
+        for (const GemmArgs& g : op.pg) {
+          DualItem it;
+          it.kind = 0; it.g = g; it.list = list; it.leaf = op.leaf ? 1 : 0;
+          items.push_back(it);
+        }
+      }
+      st.covered.push_back(&op);
+    };
+    if (s < B)
+      for (Op& op : m->fwd[s]) {
+        if (!capable(op)) { m->persistent_why = std::string("block forward holds an operation the dual-list kernel does not cover: ") + op.name; return; }
+        add(op, 0);
+      }
+    if (s >= 1) {
+      bool started = false;
+      for (Op& op : m->bwd[s - 1]) {
+        if (capable(op)) { started = true; add(op, 1); }
+        else if (!started) st.pre.push_back(&op);
+        else if (op.leaf) st.after.push_back(&op);
+        else { m->persistent_why = std::string("block backward holds an operation the dual-list kernel does not cover: ") + op.name; return; }
+      }
+    }
+    if (items.empty()) continue;
+    if ((int)items.size() > tc_dual_max()) { m->persistent_why = "a stage has more problems than the dual-list kernel takes"; return; }
+    st.plan = tc_dual_plan(items.data(), (int)items.size(), m->pdone + (size_t)s * tc_dual_max(), m->status);
+    if (!st.plan) { m->persistent_why = "a GEMM of the model does not fit the dual-list kernel (shape, alignment or epilogue)"; return; }
+  }
+  m->persistent_ok = true;
+}
+
+// One step in the persistent schedule, all on the main stream: stage s = [front of B_{s-1}] ->
+// dual-list kernel {F_s || B_{s-1}} -> split-K reductions and parameter-gradient leaves -> local head of block s.
+erase_status enqueue_persistent(erase_model* m, unsigned flags) {
+  const int B = m->B;
+  cudaStream_t st = m->main;
+  CK(run_ops(m, m->stage, st));
+  for (int s = 0; s <= B; s++) {
+    erase_model::PStage& ps = m->pstage[s];
+    for (Op* op : ps.pre) { CK(op->fn(st)); m->launches += op->launches; }
+    if (ps.plan) { CK(tc_dual_launch(ps.plan, st)); m->launches += 1; }
+    for (Op* op : ps.covered)
+      if (op->post) { CK(op->post(st)); m->launches += op->post_launches; }
+    for (Op* op : ps.after) { CK(op->fn(st)); m->launches += op->launches; }
+    if (s < B) CK(run_ops(m, m->hfwd[s], st));
+  }
+  if (!(flags & ERASE_NO_OPT)) CK(run_ops(m, m->opt, st));
+  return ERASE_OK;
 }
 
 // timed: 0 no timeline, 1 CUDA events (never while capturing), 2 device clock stamps written by
@@ -1286,6 +1386,7 @@ erase_status erase_create(const erase_model_spec* spec, erase_model** out) {
   m->ev_time.assign(2 * (2 * m->B + 1) + 1, nullptr);
   for (auto& e : m->ev_time)
     if (!mk(&e, cudaEventDefault)) return bail(ERASE_ECUDA, "event creation failed");
+  plan_persistent(m);
   if (cudaDeviceSynchronize() != cudaSuccess) return bail(ERASE_ECUDA, "device error after model set-up");
   *out = m;
   return ERASE_OK;
@@ -1306,6 +1407,7 @@ void erase_destroy(erase_model* m) {
   for (auto s : m->side) if (s) cudaStreamDestroy(s);
   for (auto s : m->leaf) if (s) cudaStreamDestroy(s);
   if (m->main) cudaStreamDestroy(m->main);
+  for (auto& ps : m->pstage) if (ps.plan) tc_dual_free(ps.plan);
   for (void* p : m->owned) cudaFree(p);
   cudaGetLastError();
   delete m;
@@ -1413,7 +1515,14 @@ static erase_status check_step_args(erase_model* m, const erase_batch* batch);
 erase_status erase_step_ex(erase_model* m, const erase_batch* batch, int32_t n_streams, uint32_t flags) {
   if (!m) return ERASE_EINVAL;
   if (n_streams < 1) return m->fail(ERASE_EINVAL, "erase_step: n_streams must be >= 1");
-  if (flags & ~(ERASE_GRAPH | ERASE_NO_OPT | ERASE_EARLY_HEAD | ERASE_BLOCK_OPT | ERASE_SPLIT_BWD | ERASE_STAMPS | ERASE_PAR_FWD)) return m->fail(ERASE_EINVAL, "erase_step: unknown flag");
+  if (flags & ~(ERASE_GRAPH | ERASE_NO_OPT | ERASE_EARLY_HEAD | ERASE_BLOCK_OPT | ERASE_SPLIT_BWD | ERASE_STAMPS | ERASE_PAR_FWD | ERASE_PERSISTENT))
+    return m->fail(ERASE_EINVAL, "erase_step: unknown flag");
+  const bool persistent = (flags & ERASE_PERSISTENT) != 0;
+  if (persistent) {
+    if (!m->persistent_ok) return m->fail(ERASE_EUNSUPPORTED, "erase_step: ERASE_PERSISTENT: " + m->persistent_why);
+    if (flags & ERASE_STAMPS) return m->fail(ERASE_EINVAL, "erase_step: ERASE_PERSISTENT records no timeline");
+    flags &= ~(ERASE_EARLY_HEAD | ERASE_BLOCK_OPT | ERASE_SPLIT_BWD | ERASE_PAR_FWD);   // stream placements: meaningless on one stream
+  }
   const int stamp_mode = (flags & ERASE_STAMPS) ? 2 : 0;
   erase_status cst = check_step_args(m, batch);
   if (cst != ERASE_OK) return cst;
@@ -1425,7 +1534,7 @@ erase_status erase_step_ex(erase_model* m, const erase_batch* batch, int32_t n_s
     if (it == m->graphs.end()) {
       int64_t before = m->launches;
       CK(cudaStreamBeginCapture(m->main, cudaStreamCaptureModeThreadLocal));
-      erase_status st = enqueue_step(m, n_streams, flags, stamp_mode);
+      erase_status st = persistent ? enqueue_persistent(m, flags) : enqueue_step(m, n_streams, flags, stamp_mode);
       cudaGraph_t graph = nullptr;
       cudaError_t e = cudaStreamEndCapture(m->main, &graph);
       const int64_t captured = m->launches - before;
@@ -1443,9 +1552,9 @@ erase_status erase_step_ex(erase_model* m, const erase_batch* batch, int32_t n_s
     m->timeline_valid = stamp_mode != 0;
     m->timeline_stamps = true;
   } else {
-    erase_status st = enqueue_step(m, n_streams, flags, stamp_mode ? 2 : 1);
+    erase_status st = persistent ? enqueue_persistent(m, flags) : enqueue_step(m, n_streams, flags, stamp_mode ? 2 : 1);
     if (st != ERASE_OK) return st;
-    m->timeline_valid = true;
+    m->timeline_valid = !persistent;
     m->timeline_stamps = stamp_mode != 0;
   }
   m->stepped = true;

@@ -19,6 +19,7 @@
 // CTA pairs, and tc_wgrad_group_kernel (up to four small weight-gradient GEMMs in one launch).
 #include "gemm_tc.cuh"
 #include "tc_ptx.cuh"
+#include "ew_math.cuh"
 
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -1128,6 +1129,376 @@ tc_wgrad_group_kernel(const __grid_constant__ GroupMaps maps, const __grid_const
   }
 }
 
+// =================================================================================================
+// Dual-list persistent kernel: the forward of block b+1 and the backward of block b in ONE launch,
+// each on its own share of the SMs (paper Section 2.2: B_b overlaps F_{b+1}; Sections 1 and 3.1:
+// small GEMMs leave SMs idle and can share the device).  A launch carries up to DUAL_MAX problems
+// in two ordered lists.  CTAs [0, split) work through list 0, the others through list 1; inside a
+// list the tiles of all problems form one sequence that the list's CTAs take round-robin.  A problem
+// may name an earlier problem of its list whose output it reads: before a CTA touches such a tile
+// it waits (bounded) until a device counter says every tile of that problem has been stored.
+// Every CTA walks its list in order and never waits for a later problem, all CTAs of the launch
+// are resident (grid <= SMs, one CTA per SM), so the waits always resolve.
+//   kind 0: GEMM tile (128 x 128), roles and pipeline as in tc_wgrad_group_kernel, operand majors
+//           chosen per problem; epilogue: bias, ReLU, ReLU derivative; bf16 or fp32 output or
+//           fp32 split-K partials, all through TMA stores
+//   kind 1: y = gelu(u), kind 2: g = g * gelu'(u) on 32 Ki-element chunks of bf16 data, done by the
+//           eight epilogue warps with the same functions as the stand-alone elementwise kernel
+// The arithmetic of a tile does not depend on which CTA computes it or when: the results are the
+// bits of the same operations launched one by one.
+constexpr int DUAL_MAX = 8;
+constexpr int DUAL_EW_CHUNK = 32768;
+constexpr long long DUAL_WAIT_CYCLES = 500000000LL;
+struct DualProblem {
+  int kind;                       // 0 GEMM, 1 gelu, 2 gelu derivative
+  int M, N, K, splits, kchunk, tiles_m, tiles_n;
+  int a_mn, b_mn;
+  int out_mode;                   // 0: bf16 [M, N]; 1: fp32 [M, N]; 2: fp32 split-K partials [splits, M, N]
+  int relu, dact_relu;
+  int dep;                        // problem whose completion this one waits for, or -1
+  int signal;                     // a later problem waits for this one: count finished tiles
+  int ntiles, tile_begin;         // tiles of this problem; index of its first tile in its list's sequence
+  const float* bias;
+  const __nv_bfloat16* dact_src;
+  long long ld_aux;
+  const __nv_bfloat16* ew_src;
+  __nv_bfloat16* ew_dst;
+  long long ew_n;
+};
+struct DualArgs {
+  int nprob, split;
+  int first[2], count[2], total[2];   // per list: first problem, number of problems, tiles
+  int* done;                          // [DUAL_MAX] finished epilogue-warp tiles per problem, zero at launch
+  int* status;
+  DualProblem prob[DUAL_MAX];
+};
+struct DualMaps {
+  CUtensorMap a[DUAL_MAX], b[DUAL_MAX], c[DUAL_MAX];
+};
+
+__device__ __forceinline__ int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+// waits until problem `dep` has stored all its tiles (8 epilogue warps each); false on expiry
+__device__ __forceinline__ bool dual_wait_dep(const DualArgs& g, int dep) {
+  if (dep < 0) return true;
+  const int need = g.prob[dep].ntiles * EPI_WARPS;
+  if (ld_acquire(g.done + dep) >= need) return true;
+  const long long t0 = clock64();
+  while (ld_acquire(g.done + dep) < need) {
+    if (clock64() - t0 > DUAL_WAIT_CYCLES) return false;
+    __nanosleep(64);
+  }
+  return true;
+}
+__device__ __forceinline__ int dual_find(const DualArgs& g, int list, int t) {
+  int pi = g.first[list];
+  const int end = g.first[list] + g.count[list];
+  while (pi + 1 < end && t >= g.prob[pi + 1].tile_begin) pi++;
+  return pi;
+}
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+tc_dual_kernel(const __grid_constant__ DualMaps maps, const __grid_constant__ DualArgs g) {
+  extern __shared__ uint8_t smem_raw[];
+  constexpr int BN = 128;
+  constexpr uint32_t A_BYTES = BM * BK * 2;
+  constexpr uint32_t B_BYTES = BN * BK * 2;
+  constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr uint32_t TMEM_COLS = 2 * BN;
+  constexpr int STAGES = 4;
+  constexpr int CPW = BN / 2;
+
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t epi_base = smem_base + STAGES * STAGE_BYTES;
+  const uint32_t bias_base = epi_base + EPI_WARPS * EPI_STAGE_BYTES;
+  const uint32_t bar_base = bias_base + EPI_WARPS * EPI_BIAS_BYTES;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+  uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
+  volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(gen_base + (bar_base - smem_base) + 8u * (2 * STAGES + 4));
+  const uint32_t tmem_slot = bar_base + 8u * (2 * STAGES + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int list = (int)blockIdx.x < g.split ? 0 : 1;
+  const int rank = list == 0 ? (int)blockIdx.x : (int)blockIdx.x - g.split;
+  const int nrank = list == 0 ? g.split : (int)gridDim.x - g.split;
+  const int total = g.total[list];
+  const int st0 = status_peek(g.status);
+  if (threadIdx.x == 32) {
+    for (int i = 0; i < g.nprob; i++) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.a[i]) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.b[i]) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.c[i]) : "memory");
+    }
+  }
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; s++) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; a++) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), EPI_WARPS);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  const bool dead = __syncthreads_or(st0 != 0) != 0;
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot_ptr;
+
+  if (dead) {
+    // the step is already void: do nothing but free TMEM below
+  } else if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int t = rank; t < total && ok; t += nrank) {
+        const int pi = dual_find(g, list, t);
+        const DualProblem& q = g.prob[pi];
+        if (q.kind != 0) continue;                      // elementwise chunks need no staging
+        if (!dual_wait_dep(g, q.dep)) { atomicExch(g.status, 41); ok = false; break; }
+        asm volatile("fence.proxy.async;" ::: "memory");   // the other CTAs' stores are ordered before this CTA's TMA reads
+        const int local = t - q.tile_begin, per = q.tiles_m * q.tiles_n;
+        const int split = local / per, r = local - split * per;
+        const int mt = r / q.tiles_n, nt = r - mt * q.tiles_n;
+        const int m0 = mt * BM, n0 = nt * BN;
+        const int kbeg = split * q.kchunk, kend = min(q.K, kbeg + q.kchunk);
+        const int num_kb = kend > kbeg ? (kend - kbeg + BK - 1) / BK : 0;
+        for (int kb = 0; kb < num_kb; kb++, it++) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!mbar_wait(empty_bar(s), ph ^ 1)) { atomicExch(g.status, 1); ok = false; break; }
+          mbar_expect_tx(full_bar(s), STAGE_BYTES);
+          const uint32_t a_dst = smem_base + s * STAGE_BYTES;
+          const uint32_t b_dst = a_dst + A_BYTES;
+          const int k0 = kbeg + kb * BK;
+          if (!q.a_mn) {
+            tma_load_2d(a_dst, &maps.a[pi], k0, m0, full_bar(s));
+          } else {
+#pragma unroll
+            for (int a = 0; a < BM / 64; a++) tma_load_2d(a_dst + a * (BK * 128), &maps.a[pi], m0 + a * 64, k0, full_bar(s));
+          }
+          if (!q.b_mn) {
+            tma_load_2d(b_dst, &maps.b[pi], k0, n0, full_bar(s));
+          } else {
+#pragma unroll
+            for (int a = 0; a < BN / 64; a++) tma_load_2d(b_dst + a * (BK * 128), &maps.b[pi], n0 + a * 64, k0, full_bar(s));
+          }
+        }
+      }
+      if (!ok) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) {}
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer ------------------------------
+    if (lane == 0) {
+      uint32_t it = 0, lt = 0;
+      bool ok = true;
+      for (int t = rank; t < total && ok; t += nrank) {
+        const int pi = dual_find(g, list, t);
+        const DualProblem& q = g.prob[pi];
+        if (q.kind != 0) continue;
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((q.a_mn ? 1u : 0u) << 15) | ((q.b_mn ? 1u : 0u) << 16) |
+                               ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+        const int local = t - q.tile_begin, split = local / (q.tiles_m * q.tiles_n);
+        const int kbeg = split * q.kchunk, kend = min(q.K, kbeg + q.kchunk);
+        const int num_kb = kend > kbeg ? (kend - kbeg + BK - 1) / BK : 0;
+        const uint32_t ab = lt & 1, aph = (lt >> 1) & 1;
+        if (!mbar_wait(tempty_bar(ab), aph ^ 1)) { atomicExch(g.status, 4); ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + ab * BN;
+        for (int kb = 0; kb < num_kb; kb++, it++) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!mbar_wait(full_bar(s), ph)) { atomicExch(g.status, 2); ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_src = smem_base + s * STAGE_BYTES;
+          const uint32_t b_src = a_src + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; k++) {
+            const uint64_t ad = q.a_mn ? smem_desc(a_src + k * (UMMA_K * 128), BK * 128, 1024) : smem_desc(a_src + k * (UMMA_K * 2), 16, 1024);
+            const uint64_t bd = q.b_mn ? smem_desc(b_src + k * (UMMA_K * 128), BK * 128, 1024) : smem_desc(b_src + k * (UMMA_K * 2), 16, 1024);
+            tc_mma(tmem_d, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          }
+          tc_commit(empty_bar(s));
+        }
+        tc_commit(tfull_bar(ab));
+        lt++;
+      }
+    }
+  } else {
+    // ------------------------------ epilogue / elementwise warps ------------------------------
+    const int ew = warp - 2;
+    const int q4 = warp & 3;
+    const int cbeg = (ew / 4) * CPW;
+    const uint32_t stage0 = epi_base + ew * EPI_STAGE_BYTES;
+    float* bias_s = reinterpret_cast<float*>(gen_base + (bias_base - smem_base) + ew * EPI_BIAS_BYTES);
+    uint32_t sbuf = 0;
+    bool store_pending = false;
+    uint32_t lt = 0;
+    for (int t = rank; t < total; t += nrank) {
+      const int pi = dual_find(g, list, t);
+      const DualProblem& q = g.prob[pi];
+      if (q.kind != 0) {
+        // ---- elementwise chunk: the 256 threads of these warps, 16 bytes per access ----
+        bool ok = true;
+        if (lane == 0) ok = dual_wait_dep(g, q.dep);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) { if (lane == 0) atomicExch(g.status, 42); break; }
+        asm volatile("fence.proxy.async;" ::: "memory");
+        const long long beg = (long long)(t - q.tile_begin) * DUAL_EW_CHUNK;
+        const long long end = beg + DUAL_EW_CHUNK < q.ew_n ? beg + DUAL_EW_CHUNK : q.ew_n;
+        for (long long i = beg + (long long)(ew * 32 + lane) * 8; i < end; i += 256 * 8) {     // ew_n % 8 == 0
+          const uint4 u = *reinterpret_cast<const uint4*>(q.ew_src + i);
+          float x[8], y[8];
+          unpack8_bf16(u, x);
+          if (q.kind == 1) {
+#pragma unroll
+            for (int j = 0; j < 8; j++) y[j] = gelu_bf16_value(x[j]);
+          } else {
+            unpack8_bf16(*reinterpret_cast<const uint4*>(q.ew_dst + i), y);
+#pragma unroll
+            for (int j = 0; j < 8; j++) y[j] = y[j] * gelu_bf16_deriv(x[j]);
+          }
+          uint4 o;
+          o.x = pack2(y[0], y[1]); o.y = pack2(y[2], y[3]); o.z = pack2(y[4], y[5]); o.w = pack2(y[6], y[7]);
+          *reinterpret_cast<uint4*>(q.ew_dst + i) = o;
+        }
+        if (q.signal) {
+          __threadfence();
+          __syncwarp();
+          if (lane == 0) atomicAdd(g.done + pi, 1);
+        }
+        continue;
+      }
+      const int local = t - q.tile_begin, per = q.tiles_m * q.tiles_n;
+      const int split = local / per, r = local - split * per;
+      const int mt = r / q.tiles_n, nt = r - mt * q.tiles_n;
+      const int m0 = mt * BM, n0 = nt * BN;
+      const int kbeg = split * q.kchunk, kend = min(q.K, kbeg + q.kchunk);
+      const bool empty_k = kend <= kbeg;
+      const uint32_t ab = lt & 1, aph = (lt >> 1) & 1;
+      lt++;
+      if (q.bias) {
+        __syncwarp();
+        for (int j = lane; j < CPW; j += 32) {
+          const int n = n0 + cbeg + j;
+          bias_s[j] = n < q.N ? __ldg(q.bias + n) : 0.f;
+        }
+        __syncwarp();
+      }
+      const int row = m0 + q4 * 32 + lane;
+      const bool row_ok = row < q.M;
+      bool ok = mbar_wait(tfull_bar(ab), aph);
+      if (!ok) atomicExch(g.status, 3);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const bool rows_in = m0 + q4 * 32 < q.M;
+      const bool f32 = q.out_mode != 0;
+      if (n0 + cbeg < q.N) {
+#pragma unroll 1
+        for (int cc = 0; cc < CPW; cc += 32) {
+          const int c0 = cbeg + cc;
+          if (n0 + c0 >= q.N) break;
+          uint32_t rr[32];
+          if (!empty_k) {
+            tc_ld32(tmem_base + ab * BN + ((uint32_t)(q4 * 32) << 16) + (uint32_t)c0, rr);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; j++) rr[j] = 0u;
+          }
+          if (f32 || (cc & 63) == 0) {
+            sbuf ^= 1;
+            if (lane == 0 && store_pending) tma_store_wait_read1();
+            __syncwarp();
+          }
+          const uint32_t stage = stage0 + sbuf * 4096;
+          const uint32_t my_row = stage + lane * 128;
+#pragma unroll
+          for (int g8 = 0; g8 < 4; g8++) {
+            float v[8];
+#pragma unroll
+            for (int j = 0; j < 8; j++) v[j] = __uint_as_float(rr[g8 * 8 + j]);
+            const int n = n0 + c0 + g8 * 8;
+            if (q.bias) {
+              const float4 b0 = *reinterpret_cast<const float4*>(bias_s + cc + g8 * 8);
+              const float4 b1 = *reinterpret_cast<const float4*>(bias_s + cc + g8 * 8 + 4);
+              v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w;
+              v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+            }
+            if (q.relu) {
+#pragma unroll
+              for (int j = 0; j < 8; j++) v[j] = fmaxf(v[j], 0.f);
+            }
+            if (q.dact_relu && row_ok && n < q.N) {       // N % 8 == 0 whenever an auxiliary operand is present
+              float tsrc[8];
+              unpack8_bf16(*reinterpret_cast<const uint4*>(q.dact_src + (long long)row * q.ld_aux + n), tsrc);
+#pragma unroll
+              for (int j = 0; j < 8; j++) v[j] = tsrc[j] > 0.f ? v[j] : 0.f;
+            }
+            if (f32) {
+              const uint32_t s0 = my_row + (((2 * g8) ^ (lane & 7)) << 4), s1 = my_row + (((2 * g8 + 1) ^ (lane & 7)) << 4);
+              st_shared_v4(s0, __float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]));
+              st_shared_v4(s1, __float_as_uint(v[4]), __float_as_uint(v[5]), __float_as_uint(v[6]), __float_as_uint(v[7]));
+            } else {
+              const uint32_t s0 = my_row + (((((cc & 63) >> 3) + g8) ^ (lane & 7)) << 4);
+              st_shared_v4(s0, pack2(v[0], v[1]), pack2(v[2], v[3]), pack2(v[4], v[5]), pack2(v[6], v[7]));
+            }
+          }
+          const bool last_chunk = (cc & 63) == 32 || n0 + c0 + 32 >= q.N;
+          if (f32 || last_chunk) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0 && rows_in) {
+              const int x = f32 ? n0 + c0 : n0 + cbeg + (cc & ~63), y = m0 + q4 * 32;
+              if (q.out_mode == 2) tma_store_3d(&maps.c[pi], stage, x, y, split);
+              else tma_store_2d(&maps.c[pi], stage, x, y);
+              tma_store_commit();
+              store_pending = true;
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(ab));
+      if (q.signal) {     // a later problem reads this output: report the tile once its stores have landed
+        if (lane == 0) {
+          if (store_pending) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+          store_pending = false;
+          asm volatile("fence.proxy.async;" ::: "memory");
+          __threadfence();
+          atomicAdd(g.done + pi, 1);
+        }
+        __syncwarp();
+      }
+    }
+    if (lane == 0 && store_pending) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
 // The bounded wait on its own: one thread waits, with the given limit, on a barrier that nothing
 // ever signals, records status code 8 and returns.  It returns by construction (the wait is
 // clock-bounded) and touches no tensor memory; used to check that an expired wait surfaces as
@@ -1279,6 +1650,125 @@ cudaError_t launch_bn(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int
 }
 
 }  // namespace
+
+// ---- dual-list persistent kernel: host side ---------------------------------------------------
+struct TcDualPlan {
+  DualArgs args;
+  DualMaps maps;
+  int grid;
+};
+
+int tc_dual_max() { return DUAL_MAX; }
+
+TcDualPlan* tc_dual_plan(const DualItem* items_in, int n, int* done_dev, int* status) {
+  if (n < 1 || n > DUAL_MAX || !done_dev) return nullptr;
+  // list 0 first, then list 1, each in the given order
+  DualItem items[DUAL_MAX];
+  int cnt = 0, first1 = 0;
+  for (int l = 0; l < 2; l++) {
+    if (l == 1) first1 = cnt;
+    for (int i = 0; i < n; i++)
+      if (items_in[i].list == l) items[cnt++] = items_in[i];
+  }
+  if (cnt != n) return nullptr;
+  TcDualPlan* plan = new TcDualPlan();
+  DualArgs& a = plan->args;
+  memset(&a, 0, sizeof(a));
+  a.nprob = n;
+  a.done = done_dev;
+  a.status = status;
+  a.first[0] = 0; a.count[0] = first1;
+  a.first[1] = first1; a.count[1] = n - first1;
+  double work[2] = {0, 0};
+  auto fail = [&]() { delete plan; return (TcDualPlan*)nullptr; };
+  for (int l = 0; l < 2; l++) {
+    int tiles = 0, last_chain = -1;
+    for (int i = a.first[l]; i < a.first[l] + a.count[l]; i++) {
+      const DualItem& it = items[i];
+      DualProblem& q = a.prob[i];
+      q.kind = it.kind;
+      q.dep = last_chain;
+      q.tile_begin = tiles;
+      if (it.kind == 0) {
+        const GemmArgs& g = it.g;
+        const Epilogue& e = g.epi;
+        if (!tc_gemm_supported(g) || e.alpha != 1.f || e.mul || e.res || e.pre_out || e.ce_ref || (e.act != ACT_NONE && e.act != ACT_RELU) ||
+            (e.dact != ACT_NONE && e.dact != ACT_RELU) || (g.splits > 1 && (!g.ws || e.bias || e.act != ACT_NONE || e.dact != ACT_NONE)))
+          return fail();
+        q.M = g.M; q.N = g.N; q.K = g.K; q.splits = g.splits;
+        q.kchunk = (((g.K + g.splits - 1) / g.splits) + BK - 1) / BK * BK;
+        q.tiles_m = (g.M + BM - 1) / BM;
+        q.tiles_n = (g.N + 127) / 128;
+        q.a_mn = g.sa_k != 1; q.b_mn = g.sb_k != 1;
+        q.relu = e.act == ACT_RELU; q.dact_relu = e.dact == ACT_RELU;
+        q.bias = e.bias;
+        q.dact_src = (const __nv_bfloat16*)e.dact_src;
+        q.ld_aux = e.ld_aux ? e.ld_aux : g.N;
+        q.ntiles = q.tiles_m * q.tiles_n * g.splits;
+        bool ok = q.a_mn ? encode_2d(&plan->maps.a[i], g.A, g.M, g.K, g.sa_k, BK) : encode_2d(&plan->maps.a[i], g.A, g.K, g.M, g.sa_m, BM);
+        ok = ok && (q.b_mn ? encode_2d(&plan->maps.b[i], g.B, g.N, g.K, g.sb_k, BK) : encode_2d(&plan->maps.b[i], g.B, g.K, g.N, g.sb_n, 128));
+        if (!ok) return fail();
+        if (g.splits > 1) {
+          q.out_mode = 2;
+          cuuint64_t dims[3] = {(cuuint64_t)g.N, (cuuint64_t)g.M, (cuuint64_t)g.splits};
+          cuuint64_t str[2] = {(cuuint64_t)g.N * 4, (cuuint64_t)g.M * g.N * 4};
+          cuuint32_t box[3] = {32u, 32u, 1u};
+          ok = encode_map(&plan->maps.c[i], g.ws, true, 3, dims, str, box);
+        } else if (g.c_f32) {
+          q.out_mode = 1;
+          cuuint64_t dims[2] = {(cuuint64_t)g.N, (cuuint64_t)g.M};
+          cuuint64_t str[1] = {(cuuint64_t)g.ldc * 4};
+          cuuint32_t box[2] = {32u, 32u};
+          ok = encode_map(&plan->maps.c[i], g.C, true, 2, dims, str, box);
+        } else {
+          q.out_mode = 0;
+          cuuint64_t dims[2] = {(cuuint64_t)g.N, (cuuint64_t)g.M};
+          cuuint64_t str[1] = {(cuuint64_t)g.ldc * 2};
+          cuuint32_t box[2] = {64u, 32u};
+          ok = encode_map(&plan->maps.c[i], g.C, false, 2, dims, str, box);
+        }
+        if (!ok) return fail();
+        work[l] += (double)q.ntiles * ((q.kchunk + BK - 1) / BK + 6);
+      } else {
+        if (it.ew_n < 8 || it.ew_n % 8 || ((reinterpret_cast<uintptr_t>(it.ew_src) | reinterpret_cast<uintptr_t>(it.ew_dst)) & 15)) return fail();
+        q.ew_src = (const __nv_bfloat16*)it.ew_src;
+        q.ew_dst = (__nv_bfloat16*)it.ew_dst;
+        q.ew_n = it.ew_n;
+        q.ntiles = (int)((it.ew_n + DUAL_EW_CHUNK - 1) / DUAL_EW_CHUNK);
+        plan->maps.a[i] = plan->maps.a[0]; plan->maps.b[i] = plan->maps.b[0]; plan->maps.c[i] = plan->maps.c[0];
+        work[l] += (double)q.ntiles * 8;
+      }
+      tiles += q.ntiles;
+      if (!it.leaf) last_chain = i;
+    }
+    a.total[l] = tiles;
+  }
+  for (int i = 0; i < n; i++)
+    for (int j = i + 1; j < n; j++)
+      if (a.prob[j].dep == i) a.prob[i].signal = 1;
+  for (int i = n; i < DUAL_MAX; i++) { plan->maps.a[i] = plan->maps.a[0]; plan->maps.b[i] = plan->maps.b[0]; plan->maps.c[i] = plan->maps.c[0]; }
+  const int sms = sm_count();
+  plan->grid = sms;
+  if (a.total[0] == 0) a.split = 0;
+  else if (a.total[1] == 0) a.split = sms;
+  else {
+    int sp = (int)(sms * work[0] / (work[0] + work[1]) + 0.5);
+    a.split = sp < 1 ? 1 : (sp > sms - 1 ? sms - 1 : sp);
+  }
+  return plan;
+}
+
+void tc_dual_free(TcDualPlan* plan) { delete plan; }
+
+cudaError_t tc_dual_launch(const TcDualPlan* plan, cudaStream_t s) {
+  constexpr size_t smem = (size_t)4 * (BM * BK * 2 + 128 * BK * 2) + EPI_WARPS * (EPI_STAGE_BYTES + EPI_BIAS_BYTES) + 8 * (2 * 4 + 16) + 1024;
+  static std::atomic<bool> attr_set[MAX_DEVICES];
+  if (cudaError_t e = ensure_smem(tc_dual_kernel, smem, attr_set)) return e;
+  cudaError_t e = cudaMemsetAsync(plan->args.done, 0, DUAL_MAX * sizeof(int), s);
+  if (e != cudaSuccess) return e;
+  tc_dual_kernel<<<plan->grid, TC_THREADS, smem, s>>>(plan->maps, plan->args);
+  return cudaGetLastError();
+}
 
 bool tc_encode_rows_bf16(void* map128, const void* base, long long inner, long long outer, long long ld, int box_rows) {
   return encode_2d(map128, base, inner, outer, ld, box_rows);

@@ -54,6 +54,29 @@ struct TcGroupPlan {
 bool tc_wgrad_group_plan(const GemmArgs* gs, int n, int* status, TcGroupPlan* plan);
 cudaError_t tc_wgrad_group_launch(const TcGroupPlan& plan, cudaStream_t s, int max_ctas = 0);
 
+// Dual-list persistent kernel: up to tc_dual_max() problems in two ordered lists (list 0: the forward of
+// one block, list 1: the backward of another), each list on its own share of the SMs, in ONE launch.
+//   kind 0: GEMM g (bf16, tensor-core shapes; epilogue: bias, ReLU, ReLU derivative; split-K writes its
+//           fp32 partials to g.ws, which the caller reduces afterwards as for tc_gemm_launch)
+//   kind 1: ew_dst = gelu(ew_src); kind 2: ew_dst *= gelu'(ew_src)   (bf16, ew_n % 8 == 0)
+// A problem that is not a leaf is waited for by the problems behind it in its list (they read its
+// output); a leaf (a weight gradient) is read by nothing inside the launch.  done_dev: tc_dual_max() ints of
+// device memory owned by the caller (cleared by every launch).  Returns null if a problem does not fit.
+struct DualItem {
+  int kind = 0;
+  GemmArgs g;
+  const void* ew_src = nullptr;
+  void* ew_dst = nullptr;
+  long long ew_n = 0;
+  int list = 0;
+  int leaf = 0;
+};
+struct TcDualPlan;
+int tc_dual_max();
+TcDualPlan* tc_dual_plan(const DualItem* items, int n, int* done_dev, int* status);
+void tc_dual_free(TcDualPlan* plan);
+cudaError_t tc_dual_launch(const TcDualPlan* plan, cudaStream_t s);
+
 // TMA descriptor (128 bytes, a CUtensorMap) of a row-major bf16 matrix with `inner` contiguous
 // elements per row and `outer` rows `ld` elements apart: tiles of 64 columns x box_rows rows,
 // 128-byte swizzle, zero fill outside.  False if the layout cannot be described (alignment).

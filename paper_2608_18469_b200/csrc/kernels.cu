@@ -3,6 +3,7 @@
 // of the step (LayerNorm, causal attention, losses, gathers, dot interaction, optimizer).
 // Reductions are fixed-partition / fixed-order: no floating-point atomics anywhere.
 #include "kernels.cuh"
+#include "ew_math.cuh"
 
 #include <stdlib.h>
 
@@ -48,36 +49,12 @@ __device__ __forceinline__ float act_deriv(int act, float u) {
   return 1.f;
 }
 
-// Phi(u) and phi(u) of the standard normal for the exact-erf GELU on bf16 data: erf from the
-// Abramowitz-Stegun 7.1.26 rational form (|error| <= 1.5e-7, far below bf16 resolution) -- one
-// reciprocal, one exponential and a 5-term polynomial shared by the value and the derivative,
-// about half the instructions of erff + expf, which is what bounded the GELU passes (3.3 TB/s).
-__device__ __forceinline__ void normal_cdf_pdf_fast(float u, float& cdf, float& pdf) {
-  const float x = fabsf(u) * 0.70710678118654752f;
-  const float t = __fdividef(1.f, fmaf(0.3275911f, x, 1.f));
-  const float e = __expf(-0.5f * u * u);
-  float q = fmaf(1.061405429f, t, -1.453152027f);
-  q = fmaf(q, t, 1.421413741f);
-  q = fmaf(q, t, -0.284496736f);
-  q = fmaf(q, t, 0.254829592f);
-  q = 0.5f * q * t * e;                 // (1 - erf(x)) / 2
-  cdf = u >= 0.f ? 1.f - q : q;
-  pdf = 0.39894228040143268f * e;
-}
 template <typename T> __device__ __forceinline__ float gelu_ew(float u);
 template <> __device__ __forceinline__ float gelu_ew<float>(float u) { return act_apply(ACT_GELU, u); }
-template <> __device__ __forceinline__ float gelu_ew<bf16_t>(float u) {
-  float c, p;
-  normal_cdf_pdf_fast(u, c, p);
-  return u * c;
-}
+template <> __device__ __forceinline__ float gelu_ew<bf16_t>(float u) { return gelu_bf16_value(u); }
 template <typename T> __device__ __forceinline__ float dgelu_ew(float u);
 template <> __device__ __forceinline__ float dgelu_ew<float>(float u) { return act_deriv(ACT_GELU, u); }
-template <> __device__ __forceinline__ float dgelu_ew<bf16_t>(float u) {
-  float c, p;
-  normal_cdf_pdf_fast(u, c, p);
-  return fmaf(u, p, c);
-}
+template <> __device__ __forceinline__ float dgelu_ew<bf16_t>(float u) { return gelu_bf16_deriv(u); }
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

@@ -239,3 +239,35 @@ def test_erase_schedule_is_bit_identical_to_serial(name):
     _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=nb + 1,
                                      flags=binding.GRAPH | binding.EARLY_HEAD | binding.BLOCK_OPT | P))
     assert serial["launches"] > 0
+    # F_{b+1} and B_b inside one persistent kernel on a partition of the SMs: bf16 chains of MLP blocks
+    if name in ("c5", "goodness"):
+        _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=1, flags=binding.PERSISTENT))
+        _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=nb + 1, flags=binding.PERSISTENT | binding.GRAPH))
+    else:
+        with pytest.raises(binding.EraseError) as e:
+            gu.run_steps(spec, flat, batches[:1], n_streams=1, flags=binding.PERSISTENT)
+        assert e.value.status == binding.EUNSUPPORTED
+
+
+@pytest.mark.parametrize("name", ["relu_ragged", "gelu_w1024", "tower_relu", "wide_split"])
+def test_persistent_co_scheduled_kernel_is_bit_identical_to_serial(name):
+    """ERASE_PERSISTENT on shapes that reach every part of the dual-list kernel: ragged M / N / K tails,
+    fused ReLU and ReLU-derivative epilogues, GELU passes as elementwise problems, grouped and
+    stand-alone weight gradients with split-K partials, several tiles per CTA.  The losses, gradients,
+    parameters and optimizer state must be the bits of the serial schedule, which launches the same
+    GEMMs one by one (partly on 256 x 256 CTA-pair tiles)."""
+    from paper_2608_18469_b200 import binding
+    gu = _gu()
+    spec = {"relu_ragged": synth.mlp_spec(200, 328, 3, 600, "relu", "bf16"),
+            "gelu_w1024": synth.mlp_spec(1024, 4096, 3, 4096, "gelu", "bf16"),
+            "tower_relu": synth.mlp_spec(256, 512, 3, 1024, "relu", "bf16"),
+            "wide_split": synth.mlp_spec(2048, 8192, 2, 512, "gelu", "bf16")}[name]
+    if name == "tower_relu":
+        for blk in spec["blocks"]:
+            blk["kind"] = "tower"
+    flat = synth.init_params(spec, 6)
+    batches = [gu.DevBatch(spec, synth.make_batch(spec, 6, index=i)) for i in range(3)]
+    serial = gu.run_steps(spec, flat, batches, n_streams=1)
+    _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=1, flags=binding.PERSISTENT))
+    _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=1, flags=binding.PERSISTENT | binding.GRAPH))
+    assert np.isfinite(serial["losses"]).all()
