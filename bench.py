@@ -378,6 +378,13 @@ def table_entry(torch, binding, rep, label, cfg, kw, args, peaks):
         ser = w.leg(1, flags, steps, POOL, per_step=False)
         era = w.leg(ns, eflags, steps, POOL, per_step=False)
         pap = w.leg(ns, flags, steps, POOL, per_step=False, min_s=0.3) if eflags != flags else era
+        # F_{b+1} and B_b inside one persistent kernel on a partition of the SMs, where the model qualifies
+        per = None
+        try:
+            per = w.leg(1, flags | binding.PERSISTENT, steps, POOL, per_step=False, min_s=0.5)
+        except binding.EraseError as e:
+            if e.status != binding.EUNSUPPORTED:
+                raise
         agg = w.kernel_classes(2)
         roof = roofline_of(agg, peaks, None)
         flops = synth.step_flops(spec)
@@ -385,6 +392,8 @@ def table_entry(torch, binding, rep, label, cfg, kw, args, peaks):
         return {"config": label, "unit": unit_name(spec), "serial": units / (ms_s * 1e-3), "erase": units / (ms_e * 1e-3),
                 "ms_per_step_serial": ms_s, "ms_per_step_erase": ms_e, "gain_pct": 100.0 * (ms_s / ms_e - 1.0),
                 "gain_pct_loss_on_main_stream": 100.0 * (ser["ms"] / pap["ms"] - 1.0),
+                "persistent": None if per is None else units / (per["ms"] / steps * 1e-3),
+                "gain_pct_persistent": None if per is None else 100.0 * (ser["ms"] / per["ms"] - 1.0),
                 "steps_per_repeat": steps, "repeats": [len(ser["repeats"]), len(era["repeats"])],
                 "mfu_vs_measured_sustained": flops / (ms_e * 1e-3) / (peaks["tflops"] * 1e12),
                 "top_class": roof["kernel"], "top_class_bound": roof["bound"], "top_class_frac": roof["frac"],

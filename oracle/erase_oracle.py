@@ -14,6 +14,17 @@ What it computes (paper Section 2.1, Eq. 1, and Section 2.2, Eq. 2):
                                               so nothing reaches z_{b-1} or other blocks)
   theta_b <- optimizer(theta_b, g_b)
 
+Optionally the model ends with the UNDETACHED REMAINDER of Section 2.2 (Eq. 2): a main network
+(block kind "main", always last) that reads u = [z_0 | sg[z_1] | ... | sg[z_B]] (z_0 only with
+"reads_input"), a tower Linear-act-...-Linear-act with its own head, whose loss is L_main.  Its
+backward is the usual one: it trains the main network's own parameters and, through the
+undetached z_0 columns of u, the producer of z_0 -- the embedding tables (spec["train_input"]):
+d L_main / d table_t[r] is the sum of the z_0-gradient slices of every sample whose id in
+column t is r (a scatter-add; repeated ids add up).  The sg[z_b] columns pass nothing back, and
+the detached blocks still see z_0 through sg (Eq. 1), so the tables receive gradient from L_main
+alone.  Tables are updated on the rows the batch touched only (untouched rows keep their values
+and moments; the bias correction uses the global step count).
+
 ERASE itself is only a schedule of this computation (early backward per block on
 side streams), so it has no separate oracle: every schedule must reproduce these
 numbers.  With all lambda_i = 1 and no L_main, g is also the gradient of Eq. 2's
@@ -344,22 +355,69 @@ def head_loss(blk, p, z, target):
 # the step
 # ----------------------------------------------------------------------------
 
-def forward_backward(spec, params, batch):
-    """Losses l_1..l_B and gradients g_1..g_B (a dict per block) for one batch."""
+def main_input(blk, z0, outs):
+    """u = [z_0 | sg[z_1] | ... | sg[z_B]]: the value only; which columns pass a gradient back is
+    decided in the backward (the z_0 columns, and only with reads_input)."""
+    return np.concatenate(([z0] if blk.get("reads_input") else []) + outs, axis=1)
+
+
+def input_gradients(spec, batch, dz0):
+    """Gradient of the producer of z_0 from dz0 = d L_main / d z_0 [rows, width].
+    ctr   : table_t[r] receives the sum over the samples n with ids[n, t] = r of dz0[n, t*e:(t+1)*e]
+    tokens: tok_emb[r] receives the rows of dz0 whose input token is r; pos_emb[t] the sum over sequences
+    dense : z_0 is data, nothing to train."""
+    kind = spec["input"]
+    if kind == "ctr":
+        ids = np.asarray(batch["ids"])
+        e = spec["emb_dim"]
+        out = {}
+        for t in range(spec["n_sparse"]):
+            g = np.zeros((spec["table_rows"], e), F)
+            for n in range(ids.shape[0]):                    # the scatter-add, written out
+                g[ids[n, t]] += dz0[n, t * e:(t + 1) * e]
+            out[f"table{t}"] = g
+        return out
+    if kind == "tokens":
+        ids = np.asarray(batch["ids"])[:, :-1]
+        bt, t = ids.shape
+        d3 = dz0.reshape(bt, t, -1)
+        gt = np.zeros((spec["vocab"], d3.shape[-1]), F)
+        for b in range(bt):
+            for i in range(t):
+                gt[ids[b, i]] += d3[b, i]
+        return {"tok_emb": gt, "pos_emb": d3.sum(axis=0)}
+    return {}
+
+
+def forward_backward(spec, params, batch, want_input=False):
+    """Losses l_1..l_B (then L_main) and gradients (a dict per block) for one batch.
+    With want_input a third value: {name: gradient} of the trainable input tables (from L_main)."""
     inp = params.get("input", {})
     z0, target = stage_input(spec, inp, batch)
-    losses, grads = [], []
+    losses, grads, outs = [], [], []
+    ginput = {}
     z = z0
     for blk, p64 in zip(spec["blocks"], params["blocks"]):
         p = {k: np.asarray(v, F) for k, v in p64.items()}
+        if blk["kind"] == "main":                               # the undetached remainder: usual backward
+            u = main_input(blk, z0, outs)
+            zout, cache = _mlp_fwd(blk, p, u, act_last=True)
+            loss, dz, g = head_loss(blk, p, zout, target)
+            du = _mlp_bwd(blk, p, cache, dz, g, need_dx=True)
+            if blk.get("reads_input") and spec.get("train_input"):
+                ginput = input_gradients(spec, batch, du[:, :z0.shape[1]])   # the sg[z_b] columns pass nothing back
+            losses.append(float(loss))
+            grads.append(g)
+            continue
         zin = z0 if spec["topo"] == "parallel" else z       # value of sg[z_{b-1}]
         zout, cache = block_forward(spec, blk, p, zin)
         loss, dz, g = head_loss(blk, p, zout, target)
         block_backward(spec, blk, p, zin, cache, dz, g)
         losses.append(float(loss))
         grads.append(g)
+        outs.append(zout)
         z = zout                                            # passed on detached
-    return losses, grads
+    return (losses, grads, ginput) if want_input else (losses, grads)
 
 
 def forward_only(spec, params, batch):
@@ -368,10 +426,17 @@ def forward_only(spec, params, batch):
     z0, target = stage_input(spec, inp, batch)
     out = []
     z = z0
+    outs = []
     for blk, p64 in zip(spec["blocks"], params["blocks"]):
         p = {k: np.asarray(v, F) for k, v in p64.items()}
+        if blk["kind"] == "main":
+            zm, _ = _mlp_fwd(blk, p, main_input(blk, z0, outs), act_last=True)
+            s = linear_fwd(zm, p["Wh"], p["bh"])
+            out.append(float(bce_with_logits(s[:, 0], target)[0] if blk["head"] == "bce" else softmax_ce(s, target)[0]))
+            continue
         zin = z0 if spec["topo"] == "parallel" else z
         z, _ = block_forward(spec, blk, p, zin)
+        outs.append(z)
         if blk["head"] == "goodness":
             out.append(float(goodness_head(p, z, target)[0]))
             continue
@@ -386,7 +451,32 @@ def forward_only(spec, params, batch):
 def new_opt_state(params):
     return {"t": 0,
             "m": [{k: np.zeros_like(np.asarray(v, F)) for k, v in p.items()} for p in params["blocks"]],
-            "v": [{k: np.zeros_like(np.asarray(v, F)) for k, v in p.items()} for p in params["blocks"]]}
+            "v": [{k: np.zeros_like(np.asarray(v, F)) for k, v in p.items()} for p in params["blocks"]],
+            "m_in": {k: np.zeros_like(np.asarray(v, F)) for k, v in params.get("input", {}).items()},
+            "v_in": {k: np.zeros_like(np.asarray(v, F)) for k, v in params.get("input", {}).items()}}
+
+
+def optimizer_update_rows(opt, theta, g, touched, m, v, t):
+    """The same update on the rows `touched` (boolean mask) only: untouched rows keep their
+    values and moments.  t is the global step count."""
+    th2, m2, v2 = optimizer_update(opt, theta[touched], g[touched], m[touched], v[touched], t)
+    theta, m, v = theta.copy(), m.copy(), v.copy()
+    theta[touched], m[touched], v[touched] = th2, m2, v2
+    return theta, m, v
+
+
+def touched_rows(spec, batch, name):
+    """Rows of input table `name` that the batch reads."""
+    ids = np.asarray(batch["ids"])
+    if spec["input"] == "ctr":
+        mask = np.zeros(spec["table_rows"], bool)
+        mask[ids[:, int(name[5:])]] = True
+        return mask
+    if name == "tok_emb":
+        mask = np.zeros(spec["vocab"], bool)
+        mask[ids[:, :-1].ravel()] = True
+        return mask
+    return np.ones(spec["seq"], bool)
 
 
 def optimizer_update(opt, theta, g, m, v, t):
@@ -414,10 +504,14 @@ def optimizer_update(opt, theta, g, m, v, t):
 
 def step(spec, params, state, batch):
     """One training step.  Returns (losses, grads, new_params, new_state); inputs untouched."""
-    losses, grads = forward_backward(spec, params, batch)
+    losses, grads, ginput = forward_backward(spec, params, batch, want_input=True)
     t = state["t"] + 1
-    new_p = {"input": params.get("input", {}), "blocks": []}
-    new_s = {"t": t, "m": [], "v": []}
+    new_p = {"input": dict(params.get("input", {})), "blocks": []}
+    new_s = {"t": t, "m": [], "v": [], "m_in": dict(state.get("m_in", {})), "v_in": dict(state.get("v_in", {}))}
+    for k, g in ginput.items():                                 # trainable input tables: the rows this batch touched
+        th, m1, v1 = optimizer_update_rows(spec["opt"], np.asarray(params["input"][k], F), g, touched_rows(spec, batch, k),
+                                           np.asarray(state["m_in"][k], F), np.asarray(state["v_in"][k], F), t)
+        new_p["input"][k], new_s["m_in"][k], new_s["v_in"][k] = th, m1, v1
     for b, p in enumerate(params["blocks"]):
         np_, nm, nv = {}, {}, {}
         for k in p:

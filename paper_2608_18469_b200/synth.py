@@ -12,7 +12,8 @@ A *spec* is a plain dict::
      "width": int,                      # dense: input width
      "seq": int, "vocab": int,          # tokens
      "n_dense", "n_sparse", "table_rows", "emb_dim",   # ctr
-     "blocks": [ {"kind": "mlp"|"tower"|"transformer"|"cross"|"dot",
+     "train_input": bool,               # ctr with a main block: the tables are trained (by L_main)
+     "blocks": [ {"kind": "mlp"|"tower"|"transformer"|"cross"|"dot"|"main",
                   "dims": [...], "act": "none"|"relu"|"gelu",
                   "n_heads": int, "n_cross": int, "head": "bce"|"ce"|"goodness",
                   "head_out": int}, ... ],
@@ -25,6 +26,8 @@ Block kinds (detached blocks of Eq. 1; the local head is part of the block):
   cross        n_cross DCN-v2 layers of width dims[0]
   dot          Linear(16->emb_dim) on the padded dense features, pairwise dots of
                the 27 vectors, then a tower over dims (dims[0] = padded feature count)
+  main         (last block only) the undetached remainder of Eq. 2: a tower over
+               [z_0 | sg[z_1] | .. | sg[z_B]] (z_0 with "reads_input") with loss L_main
 """
 from __future__ import annotations
 
@@ -85,6 +88,24 @@ def ctr_spec(batch=4096, n_dense=13, n_sparse=26, table_rows=100000, emb_dim=64,
             "opt": opt or _opt("adam", 1e-3)}
 
 
+def block_out_width(blk):
+    return blk["dims"][0] if blk["kind"] in ("cross", "transformer") else blk["dims"][-1]
+
+
+def with_main(spec, tower=(256, 128), reads_input=True, train_input=True, act="relu"):
+    """The same model followed by the undetached remainder of Eq. 2: a main tower (activation after
+    every Linear) over u = [z_0 | sg[z_1] | ... | sg[z_B]] with its own BCE head, loss L_main and the
+    usual end-of-step backward; with train_input its gradient reaches the input tables through the
+    z_0 columns of u.  Dense and CTR inputs (the head needs labels)."""
+    s = dict(spec)
+    width = (spec["width"] if reads_input else 0) + sum(block_out_width(b) for b in spec["blocks"])
+    main = {"kind": "main", "dims": [width, *tower], "act": act, "head": "bce", "head_out": 1,
+            "reads_input": bool(reads_input)}
+    s["blocks"] = [dict(b) for b in spec["blocks"]] + [main]
+    s["train_input"] = bool(train_input and reads_input and spec["input"] == "ctr")
+    return s
+
+
 def config(name, **kw):
     """The named workloads C1..C5 (C5 takes w= and batch=)."""
     if name == "C1":
@@ -112,15 +133,16 @@ C5_BATCHES = (512, 4096, 32768)
 
 def tensor_list(spec):
     out = []
+    tin = bool(spec.get("train_input"))     # the main network's backward reaches the input tables
     if spec["input"] == "tokens":
         out.append((-1, "tok_emb", (spec["vocab"], spec["width"]), False))
         out.append((-1, "pos_emb", (spec["seq"], spec["width"]), False))
     elif spec["input"] == "ctr":
         for t in range(spec["n_sparse"]):
-            out.append((-1, f"table{t}", (spec["table_rows"], spec["emb_dim"]), False))
+            out.append((-1, f"table{t}", (spec["table_rows"], spec["emb_dim"]), tin))
     for b, blk in enumerate(spec["blocks"]):
         k, dims = blk["kind"], blk["dims"]
-        if k in ("mlp", "tower"):
+        if k in ("mlp", "tower", "main"):
             for i, (a, o) in enumerate(zip(dims, dims[1:])):
                 out.append((b, f"W{i}", (o, a), True))
                 out.append((b, f"b{i}", (o,), True))
@@ -164,7 +186,7 @@ def _followed_by_activation(blk, name):
     i = int(name[1:])
     if k == "mlp":
         return blk["act"] != "none" and i < len(blk["dims"]) - 2
-    if k in ("tower", "dot"):
+    if k in ("tower", "dot", "main"):
         return blk["act"] != "none"
     if k == "transformer":
         return name == "W1"
@@ -294,7 +316,10 @@ def step_flops(spec):
     total = 0
     for blk in spec["blocks"]:
         k, dims = blk["kind"], blk["dims"]
-        if k in ("mlp", "tower"):
+        if k == "main":                      # the usual backward: the first layer's dgrad is needed too
+            f = sum(lin(a, o) for a, o in zip(dims, dims[1:])) + lin(dims[-1], blk["head_out"])
+            total += 3 * f
+        elif k in ("mlp", "tower"):
             f = sum(lin(a, o) for a, o in zip(dims, dims[1:])) + lin(dims[-1], blk["head_out"])
             total += f + 2 * f - lin(dims[0], dims[1])
         elif k == "transformer":
