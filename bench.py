@@ -37,7 +37,8 @@ MIN_LEG_S = 1.0     # every leg is repeated (K steps per repeat) until this much
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from ncu captures of the largest member
 # of each kernel class (summaries under profiles/).  They sit below the algorithmic bytes where an
 # operand or result is still L2-resident.
-NCU_DRAM_BYTES = {"C2": {"gemm_fwd": 15.5e6, "gemm_dgrad": 75.4e6, "gemm_wgrad": 71.4e6}}
+NCU_DRAM_BYTES = {"C2": {"gemm_fwd": 15.5e6, "gemm_dgrad": 75.4e6, "gemm_wgrad": 71.4e6},
+                  "C4": {"gemm_fwd": 567.5e6, "gemm_dgrad": 678.0e6, "gemm_wgrad": 706.2e6}}
 
 # the per-config table of the default run: (label, config name, keyword arguments)
 TABLE = [("C1", "C1", {}), ("C2", "C2", {}), ("C3", "C3", {}),
@@ -358,7 +359,9 @@ def roofline_of(agg, peaks, cfg_name):
     return roof
 
 
-NCU_DRAM_NOTE = {"C2": "ncu DRAM bytes of the class's largest GEMM (local head), one launch"}
+NCU_DRAM_NOTE = {"C2": "ncu DRAM bytes of the class's largest GEMM (local head), one launch",
+                 "C4": "ncu dram__bytes_read.sum + dram__bytes_write.sum of the class's largest GEMM (the local head's, 8192 x 32768 x 768), "
+                       "one full-size launch: profiles/tc_gemm_c4_head_ce_fwd_wgrad_dgrad.md"}
 
 
 def table_entry(torch, binding, rep, label, cfg, kw, args, peaks):

@@ -60,8 +60,16 @@ typedef enum { ERASE_BLK_MLP = 0,         /* Linear act Linear ... (no activatio
                ERASE_BLK_TOWER = 1,       /* Linear act after every Linear                        */
                ERASE_BLK_TRANSFORMER = 2, /* pre-LN causal transformer block, dims = {d, d_ff}    */
                ERASE_BLK_CROSS = 3,       /* n_cross DCN-v2 layers x_{l+1} = x0 * (W x_l + b) + x_l */
-               ERASE_BLK_DOT = 4          /* dense projection, pairwise dots, then a tower        */
+               ERASE_BLK_DOT = 4,         /* dense projection, pairwise dots, then a tower        */
+               ERASE_BLK_MAIN = 5         /* last block only: the UNDETACHED remainder of Section 2.2, Eq. 2.  A tower
+                                             (activation after every Linear) over u = [z_0 | sg z_1 | .. | sg z_B]
+                                             (z_0 only with ERASE_MAIN_READS_INPUT), BCE head, loss L_main.  Its
+                                             backward is the usual one: it runs behind the last forward, trains the
+                                             tower and -- with train_input -- the input tables through the z_0
+                                             columns of u; the sg z_b columns pass nothing back.  dims[0] must be
+                                             the width of u.  Dense or CTR input.                              */
 } erase_block_kind;
+#define ERASE_MAIN_READS_INPUT 1   /* erase_block_spec.flags of a MAIN block: u starts with the undetached z_0 */
 typedef enum { ERASE_ACT_NONE = 0, ERASE_ACT_RELU = 1, ERASE_ACT_GELU = 2 } erase_act;
 typedef enum { ERASE_HEAD_BCE = 0,        /* Linear(d->1) + mean binary cross-entropy with logits */
                ERASE_HEAD_SOFTMAX_CE = 1, /* Linear(d->head_out) + mean softmax cross-entropy     */
@@ -90,6 +98,7 @@ typedef struct {
   int32_t n_cross;              /* CROSS: number of cross layers                                 */
   int32_t head;                 /* erase_head_kind                                               */
   int32_t head_out;             /* 1 for BCE; vocabulary size for softmax cross-entropy          */
+  int32_t flags;                /* MAIN: ERASE_MAIN_READS_INPUT; 0 otherwise                     */
 } erase_block_spec;
 
 /* The whole model.  Trainable tensors are Linear weights W [out, in] row-major, biases, and
@@ -112,6 +121,12 @@ typedef struct {
   int32_t opt;        /* erase_opt_kind                                                          */
   float lr, beta1, beta2, eps, weight_decay; /* Adam: m,v with bias correction, update
                          lr*mhat/(sqrt(vhat)+eps); AdamW first shrinks theta by (1 - lr*wd)      */
+  int32_t train_input; /* CTR with a MAIN block that reads z_0: the embedding tables are trained by L_main
+                         (gradient = scatter-add of dL_main/dz_0 by id, summed in sample order; the
+                         optimizer touches only the rows the batch read; untouched rows keep their
+                         values and moments).  Tables then count as trainable tensors: erase_grads
+                         returns their dense gradient of the last step, erase_opt_state their moments.
+                         batch <= 16384.                                                           */
   void* arena;        /* DEVICE, optional: caller-owned memory the model lives in (256-byte
                          aligned); NULL = the library allocates with cudaMalloc                  */
   size_t arena_bytes; /* size of arena; at least erase_arena_bytes(spec)                         */
@@ -226,7 +241,8 @@ ERASE_API erase_status erase_set_opt_state(erase_model* m, int32_t idx, const fl
 ERASE_API erase_status erase_step(erase_model* m, const erase_batch* batch, int32_t n_streams);
 ERASE_API erase_status erase_step_ex(erase_model* m, const erase_batch* batch, int32_t n_streams, uint32_t flags);
 
-/* Waits for the last step and copies the local losses l_1..l_B (n_blocks floats) to dst. */
+/* Waits for the last step and copies the local losses l_1..l_B (n_blocks floats; a MAIN block is the
+ * last of them and its entry is L_main) to dst. */
 ERASE_API erase_status erase_losses(erase_model* m, float* dst, int32_t n_blocks);
 
 /* Waits until everything enqueued on the model has finished. */

@@ -21,7 +21,7 @@ MAX_DIMS = 8
 
 _DTYPE = {"f32": 0, "bf16": 1}
 _INPUT = {"dense": 0, "tokens": 1, "ctr": 2}
-_KIND = {"mlp": 0, "tower": 1, "transformer": 2, "cross": 3, "dot": 4}
+_KIND = {"mlp": 0, "tower": 1, "transformer": 2, "cross": 3, "dot": 4, "main": 5}
 _ACT = {"none": 0, "relu": 1, "gelu": 2}
 _HEAD = {"bce": 0, "ce": 1, "goodness": 2}
 _OPT = {"sgd": 0, "adam": 1, "adamw": 2}
@@ -31,7 +31,7 @@ _TOPO = {"chain": 0, "parallel": 1}
 class BlockSpec(C.Structure):
     _fields_ = [("kind", C.c_int32), ("n_dims", C.c_int32), ("dims", C.c_int32 * MAX_DIMS),
                 ("act", C.c_int32), ("n_heads", C.c_int32), ("n_cross", C.c_int32),
-                ("head", C.c_int32), ("head_out", C.c_int32)]
+                ("head", C.c_int32), ("head_out", C.c_int32), ("flags", C.c_int32)]
 
 
 class ModelSpec(C.Structure):
@@ -40,7 +40,8 @@ class ModelSpec(C.Structure):
                 ("n_sparse", C.c_int32), ("table_rows", C.c_int32), ("emb_dim", C.c_int32),
                 ("n_blocks", C.c_int32), ("blocks", C.POINTER(BlockSpec)), ("opt", C.c_int32),
                 ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
-                ("weight_decay", C.c_float), ("arena", C.c_void_p), ("arena_bytes", C.c_size_t)]
+                ("weight_decay", C.c_float), ("train_input", C.c_int32), ("arena", C.c_void_p),
+                ("arena_bytes", C.c_size_t)]
 
 
 class Batch(C.Structure):
@@ -120,6 +121,7 @@ def make_spec(spec, arena=None, arena_bytes=0):
         b.n_cross = blk.get("n_cross", 0)
         b.head = _HEAD[blk["head"]]
         b.head_out = blk["head_out"]
+        b.flags = 1 if blk.get("reads_input") else 0
     o = spec["opt"]
     ms = ModelSpec(dtype=_DTYPE[spec["dtype"]], input=_INPUT[spec["input"]], topo=_TOPO[spec["topo"]],
                    batch=spec["batch"], width=spec["width"], seq=spec.get("seq", 0),
@@ -128,7 +130,8 @@ def make_spec(spec, arena=None, arena_bytes=0):
                    emb_dim=spec.get("emb_dim", 0), n_blocks=len(blocks),
                    blocks=C.cast(blocks, C.POINTER(BlockSpec)), opt=_OPT[o["kind"]], lr=o["lr"],
                    beta1=o.get("beta1", 0.9), beta2=o.get("beta2", 0.999), eps=o.get("eps", 1e-8),
-                   weight_decay=o.get("wd", 0.0), arena=arena, arena_bytes=arena_bytes)
+                   weight_decay=o.get("wd", 0.0), train_input=1 if spec.get("train_input") else 0,
+                   arena=arena, arena_bytes=arena_bytes)
     return ms, blocks
 
 

@@ -52,6 +52,7 @@ struct Tensor {
   size_t n;    // elements
   size_t off;  // element offset inside the frozen or the trainable arena
   bool set;
+  int table = -1;   // index of the CTR input table this tensor is (trained by the main network with train_input), else -1
 };
 
 struct GraphKey {
@@ -107,10 +108,18 @@ struct erase_model {
 
   OpList stage, opt;
   OpList opt_tick_op;            // advances the Adam step counter (per-block optimizer mode)
+  OpList opt_tables;             // the input tables' sparse update (per-block optimizer mode: behind the main block's backward)
   std::vector<OpList> opt_blk;   // the optimizer restricted to block b's slice of the parameter arena
   std::vector<OpList> fwd, hfwd, bwd;  // per block: body forward, local head + loss, backward
   erase_batch cur = {nullptr, nullptr, nullptr};
   std::map<GraphKey, std::pair<cudaGraphExec_t, int64_t>> graphs;   // executable graph and the kernels it launches
+
+  // The main network's gradient into the input tables (train_input): sparse result of the last step.
+  bool train_input = false;
+  int* emb_sorted = nullptr; int* emb_seg = nullptr; int* emb_uniq = nullptr; int* emb_nuniq = nullptr;
+  float* emb_grow = nullptr;
+  float* mom1_in = nullptr; float* mom2_in = nullptr;   // Adam moments of the tables (frozen-arena offsets)
+  long long table_stride = 0;
 
   // Persistent schedule (ERASE_PERSISTENT): stage s runs F_s and B_{s-1} in one dual-list kernel.
   struct PStage {
@@ -239,10 +248,34 @@ bool validate(const erase_model_spec* s, std::string* why) {
         out = k.dims[k.n_dims - 1];
         break;
       }
+      case ERASE_BLK_MAIN: {
+        if (b != s->n_blocks - 1 || s->n_blocks < 2) return bad("a MAIN block must be the last of at least two blocks");
+        if (s->input == ERASE_IN_TOKENS || k.head != ERASE_HEAD_BCE) return bad("MAIN block needs labels (dense or CTR input) and a BCE head");
+        if (k.n_dims < 2) return bad("MAIN block needs a tower");
+        long long w = (k.flags & ERASE_MAIN_READS_INPUT) ? s->width : 0;
+        int pw = s->width;
+        for (int i = 0; i < b; i++) {
+          const erase_block_spec& q = s->blocks[i];
+          const int o = (q.kind == ERASE_BLK_CROSS || q.kind == ERASE_BLK_TRANSFORMER) ? q.dims[0] : q.dims[q.n_dims - 1];
+          w += o;
+          pw = o;
+        }
+        (void)pw;
+        if (k.dims[0] != w) return bad("MAIN dims[0] must be the width of [z_0 | z_1 | .. | z_B]");
+        if (b + 1 > CONCAT_MAX) return bad("too many blocks in front of a MAIN block");
+        out = k.dims[k.n_dims - 1];
+        break;
+      }
       default:
         return bad("block kind");
     }
     prev = out;
+  }
+  if (s->train_input) {
+    const erase_block_spec& last = s->blocks[s->n_blocks - 1];
+    if (s->input != ERASE_IN_CTR || last.kind != ERASE_BLK_MAIN || !(last.flags & ERASE_MAIN_READS_INPUT))
+      return bad("train_input needs CTR input and a MAIN block that reads z_0");
+    if (s->batch > embed_max_batch()) return bad("train_input: batch too large for the embedding backward");
   }
   return true;
 }
@@ -270,7 +303,10 @@ void build_tensor_table(erase_model* m) {
     add_tensor(m, -1, "tok_emb", s.vocab, s.width, false);
     add_tensor(m, -1, "pos_emb", s.seq, s.width, false);
   } else if (s.input == ERASE_IN_CTR) {
-    for (int t = 0; t < s.n_sparse; t++) add_tensor(m, -1, "table" + std::to_string(t), s.table_rows, s.emb_dim, false);
+    for (int t = 0; t < s.n_sparse; t++) {
+      add_tensor(m, -1, "table" + std::to_string(t), s.table_rows, s.emb_dim, false);
+      if (s.train_input) m->tensors.back().table = t;
+    }
   }
   for (int b = 0; b < m->B; b++) {
     const erase_block_spec& k = m->blocks[b];
@@ -285,6 +321,7 @@ void build_tensor_table(erase_model* m) {
     switch (k.kind) {
       case ERASE_BLK_MLP:
       case ERASE_BLK_TOWER:
+      case ERASE_BLK_MAIN:
         linears(0);
         break;
       case ERASE_BLK_TRANSFORMER: {
@@ -1026,6 +1063,49 @@ struct Builder {
     return st.out;
   }
 
+  // ---- the undetached remainder (Eq. 2): main network over u = [z_0 | sg z_1 | .. | sg z_B] --------------
+  std::vector<const void*> outs;      // z_1 .. z_B as the blocks are built
+  std::vector<int> out_w;
+  void* block_main(int b, const erase_block_spec& k, const void* z0, int first, OpList& f, OpList& bw) {
+    erase_model* mm = m;
+    const erase_model_spec& s = m->spec;
+    const int rows = m->rows, win = k.dims[0];
+    const bool bf = m->bf16, reads = (k.flags & ERASE_MAIN_READS_INPUT) != 0;
+    void* u = act_buf((size_t)rows * win);
+    ConcatArgs ca;
+    int off = 0;
+    auto src = [&](const void* p, int w) {
+      ca.src[ca.n] = p; ca.width[ca.n] = w; ca.offset[ca.n] = off; ca.ld[ca.n] = w;
+      ca.n++; off += w;
+    };
+    if (reads) src(z0, s.width);
+    for (size_t i = 0; i < outs.size(); i++) src(outs[i], out_w[i]);
+    ca.total = win;
+    f.push_back({[=](cudaStream_t st) { return concat_cols(ca, u, rows, bf, st); }, 1});
+    note(f, "concat", 0, 2.0 * rows * win * m->esz);
+    const int L = k.n_dims - 1;
+    Stack st = stack_fwd(f, k, u, win, true, first);
+    const int dout = k.dims[L];
+    void* dz = act_buf((size_t)rows * dout);
+    bool lb = head(b, k, st.out, dout, first + 2 * L, first + 2 * L + 1, f, bw, dz, st.act[L - 1], st.src[L - 1], first + 2 * (L - 1) + 1);
+    const bool need_du = reads && s.train_input;
+    void* du = stack_bwd(bw, k, st, win, dz, first, need_du, lb);
+    if (need_du) {
+      // only the z_0 columns of du carry on: the sg z_b columns pass nothing back (Eq. 1)
+      const int ns = s.n_sparse, e_ = s.emb_dim, trows = s.table_rows, batch = s.batch;
+      m->emb_sorted = (int*)dev_alloc(m, (size_t)ns * batch * sizeof(int), &ok);
+      m->emb_seg = (int*)dev_alloc(m, (size_t)ns * (batch + 1) * sizeof(int), &ok);
+      m->emb_uniq = (int*)dev_alloc(m, (size_t)ns * batch * sizeof(int), &ok);
+      m->emb_nuniq = (int*)dev_alloc(m, (size_t)ns * sizeof(int), &ok);
+      m->emb_grow = f32_buf((size_t)ns * batch * e_);
+      int* so = m->emb_sorted; int* sg_ = m->emb_seg; int* un = m->emb_uniq; int* nu = m->emb_nuniq;
+      float* gr = m->emb_grow;
+      bw.push_back({[=](cudaStream_t s2) { return embed_backward(du, win, mm->cur.ids, batch, ns, e_, trows, so, sg_, un, nu, gr, bf, s2); }, 2});
+      note(bw, "embed_backward", (double)batch * ns * e_, (double)batch * ns * e_ * (m->esz + 4));
+    }
+    return st.out;
+  }
+
   bool build() {
     erase_model* mm = m;
     const erase_model_spec& s = m->spec;
@@ -1036,6 +1116,9 @@ struct Builder {
     m->grad = f32_buf(m->train_n);
     if (s.opt != ERASE_OPT_SGD) { m->mom1 = f32_buf(m->train_n); m->mom2 = f32_buf(m->train_n); }
     if (bf) m->shadow = dev_alloc(m, m->train_n * 2, &ok);
+    m->train_input = s.train_input != 0;
+    if (m->train_input && s.opt != ERASE_OPT_SGD) { m->mom1_in = f32_buf(m->frozen_n); m->mom2_in = f32_buf(m->frozen_n); }
+    m->table_stride = s.input == ERASE_IN_CTR && s.n_sparse > 1 ? (long long)(m->tensors[1].off - m->tensors[0].off) : 0;
     m->tick = (double*)dev_alloc(m, 3 * sizeof(double), &ok);
     m->status = (int*)dev_alloc(m, sizeof(int), &ok);
     m->losses = f32_buf(m->B);
@@ -1085,7 +1168,10 @@ struct Builder {
         case ERASE_BLK_TRANSFORMER: zout = block_transformer(b, k, zin, first, m->fwd[b], m->bwd[b]); break;
         case ERASE_BLK_CROSS: zout = block_cross(b, k, zin, first, m->fwd[b], m->bwd[b]); break;
         case ERASE_BLK_DOT: zout = block_dot(b, k, zin, first, m->fwd[b], m->bwd[b]); break;
+        case ERASE_BLK_MAIN: zout = block_main(b, k, z0, first, m->fwd[b], m->bwd[b]); break;
       }
+      outs.push_back(zout);
+      out_w.push_back((k.kind == ERASE_BLK_CROSS || k.kind == ERASE_BLK_TRANSFORMER) ? k.dims[0] : k.dims[k.n_dims - 1]);
       flush_group(m->bwd[b]);
       flush_jobs(m->bwd[b]);
       z = zout;
@@ -1102,6 +1188,17 @@ struct Builder {
       note(m->opt, "opt_tick");
       m->opt.push_back({[=](cudaStream_t st) { return opt_update(th, gr, m1, m2, sh, n, kind, lr, b1, b2, eps, wd, tick, st); }, 1});
       note(m->opt, "opt_update", 10.0 * n, (double)n * (kind == ERASE_OPT_SGD ? 12 : 28) + (sh ? 2.0 * n : 0));
+      if (m->train_input) {      // the input tables: only the rows this batch read (follows the embedding backward of the main block)
+        float* tb = m->frozen; float* mi = m->mom1_in; float* vi = m->mom2_in;
+        const long long tstride = m->table_stride;
+        const int batch = s.batch, ns = s.n_sparse, e_ = s.emb_dim;
+        int* un = m->emb_uniq; int* nu = m->emb_nuniq; float* gr = m->emb_grow;
+        Op top{[=](cudaStream_t st) { return embed_update(tb, tstride, mi, vi, batch, ns, e_, un, nu, gr, kind, lr, b1, b2, eps, wd, tick, st); }, 1};
+        top.name = "embed_update";
+        top.bytes = (double)batch * ns * e_ * (kind == ERASE_OPT_SGD ? 12 : 28);
+        m->opt.push_back(top);
+        m->opt_tables.push_back(top);
+      }
       // per-block variant: the same update on block b's contiguous slice, runnable as soon as B_b is done
       m->opt_tick_op.push_back({[=](cudaStream_t st) { return opt_tick(tick, b1, b2, st); }, 1});
       note(m->opt_tick_op, "opt_tick");
@@ -1267,7 +1364,8 @@ erase_status enqueue_step(erase_model* m, int n_streams, unsigned flags, int tim
     // Parallel topology (every block reads z_0): the forwards are independent of one another too, so
     // with ERASE_PAR_FWD block b's whole chain F_b, l_b, B_b (and its optimizer) runs on its side
     // stream, released by ONE event behind the input staging.
-    const bool par_fwd = (flags & ERASE_PAR_FWD) != 0 && m->spec.topo == ERASE_TOPO_PARALLEL;
+    // (a main network reads every block's output: its forward stays behind all the others on the main stream)
+    const bool par_fwd = (flags & ERASE_PAR_FWD) != 0 && m->spec.topo == ERASE_TOPO_PARALLEL && m->blocks[B - 1].kind != ERASE_BLK_MAIN;
     if (par_fwd) CK(cudaEventRecord(m->ev_opt, m->main));
     for (int b = 0; b < B; b++) {
       cudaStream_t sd = m->side[b % ns];
@@ -1316,6 +1414,7 @@ erase_status enqueue_step(erase_model* m, int n_streams, unsigned flags, int tim
       }
       CK(mark(2 * (B + b) + 1, sd));
       if (block_opt) CK(run_ops(m, m->opt_blk[b], sd));
+      if (block_opt && b == B - 1) CK(run_ops(m, m->opt_tables, sd));
       CK(cudaEventRecord(m->ev_b[b], sd));
     }
     for (int b = 0; b < B; b++) CK(cudaStreamWaitEvent(m->main, m->ev_b[b], 0));  // join
@@ -1423,7 +1522,7 @@ erase_status erase_tensor_info(const erase_model* m, int32_t idx, int32_t* block
   if (name) { std::strncpy(name, t.name.c_str(), 31); name[31] = 0; }
   if (rank) *rank = t.rank;
   if (shape) { shape[0] = t.shape[0]; shape[1] = t.rank > 1 ? t.shape[1] : 0; shape[2] = shape[3] = 0; }
-  if (trainable) *trainable = t.trainable ? 1 : 0;
+  if (trainable) *trainable = (t.trainable || t.table >= 0) ? 1 : 0;
   return ERASE_OK;
 }
 
@@ -1478,15 +1577,40 @@ erase_status erase_params(erase_model* m, int32_t idx, float* dst, size_t n) {
   return copy_out(m, idx, dst, n, m ? m->theta : nullptr, m ? m->frozen : nullptr, "erase_params");
 }
 erase_status erase_grads(erase_model* m, int32_t idx, float* dst, size_t n) {
+  if (m && dst && tensor_check(m, idx, n) && m->tensors[idx].table >= 0) {
+    // an input table trained by the main network: the step left its gradient as (distinct row, summed slice)
+    // pairs; the dense gradient is assembled here on the host (rows nobody read are exactly zero)
+    if (!m->stepped) return m->fail(ERASE_ESTATE, "erase_grads: no step has run");
+    erase_status st = erase_sync(m);
+    if (st != ERASE_OK) return st;
+    const int t = m->tensors[idx].table, batch = m->spec.batch, e = m->spec.emb_dim;
+    int nu = 0;
+    CK(copy_sync(m, &nu, m->emb_nuniq + t, sizeof(int), cudaMemcpyDeviceToHost));
+    if (nu < 0 || nu > batch) return m->fail(ERASE_ESTATE, "erase_grads: no table gradient has been computed");
+    std::vector<int> rows((size_t)nu);
+    std::vector<float> vals((size_t)nu * e);
+    if (nu) {
+      CK(copy_sync(m, rows.data(), m->emb_uniq + (size_t)t * batch, (size_t)nu * sizeof(int), cudaMemcpyDeviceToHost));
+      CK(copy_sync(m, vals.data(), m->emb_grow + (size_t)t * batch * e, (size_t)nu * e * sizeof(float), cudaMemcpyDeviceToHost));
+    }
+    std::memset(dst, 0, n * sizeof(float));
+    for (int i = 0; i < nu; i++) std::memcpy(dst + (size_t)rows[i] * e, vals.data() + (size_t)i * e, (size_t)e * sizeof(float));
+    return ERASE_OK;
+  }
   return copy_out(m, idx, dst, n, m ? m->grad : nullptr, nullptr, "erase_grads");
 }
 
 erase_status erase_opt_state(erase_model* m, int32_t idx, float* mom1, float* mom2, size_t n, int64_t* t) {
   if (!m) return ERASE_EINVAL;
-  if (!tensor_check(m, idx, n) || !m->tensors[idx].trainable) return m->fail(ERASE_EINVAL, "erase_opt_state: bad index or size");
+  if (!tensor_check(m, idx, n) || !(m->tensors[idx].trainable || m->tensors[idx].table >= 0)) return m->fail(ERASE_EINVAL, "erase_opt_state: bad index or size");
   erase_status st = erase_sync(m);
   if (st != ERASE_OK) return st;
   const Tensor& tt = m->tensors[idx];
+  if (tt.table >= 0) {      // an input table: its moments live beside the frozen arena
+    if (mom1) { if (m->mom1_in) CK(copy_sync(m, mom1, m->mom1_in + tt.off, n * 4, cudaMemcpyDeviceToHost)); else std::memset(mom1, 0, n * 4); }
+    if (mom2) { if (m->mom2_in) CK(copy_sync(m, mom2, m->mom2_in + tt.off, n * 4, cudaMemcpyDeviceToHost)); else std::memset(mom2, 0, n * 4); }
+    mom1 = mom2 = nullptr;
+  }
   if (mom1) { if (m->mom1) CK(copy_sync(m, mom1, m->mom1 + tt.off, n * 4, cudaMemcpyDeviceToHost)); else std::memset(mom1, 0, n * 4); }
   if (mom2) { if (m->mom2) CK(copy_sync(m, mom2, m->mom2 + tt.off, n * 4, cudaMemcpyDeviceToHost)); else std::memset(mom2, 0, n * 4); }
   if (t) {
@@ -1499,10 +1623,15 @@ erase_status erase_opt_state(erase_model* m, int32_t idx, float* mom1, float* mo
 
 erase_status erase_set_opt_state(erase_model* m, int32_t idx, const float* mom1, const float* mom2, size_t n, int64_t t) {
   if (!m) return ERASE_EINVAL;
-  if (!tensor_check(m, idx, n) || !m->tensors[idx].trainable || t < 0) return m->fail(ERASE_EINVAL, "erase_set_opt_state: bad index, size or t");
+  if (!tensor_check(m, idx, n) || !(m->tensors[idx].trainable || m->tensors[idx].table >= 0) || t < 0) return m->fail(ERASE_EINVAL, "erase_set_opt_state: bad index, size or t");
   erase_status st = erase_sync(m);
   if (st != ERASE_OK) return st;
   const Tensor& tt = m->tensors[idx];
+  if (tt.table >= 0) {
+    if (mom1 && m->mom1_in) CK(copy_sync(m, m->mom1_in + tt.off, mom1, n * 4, cudaMemcpyHostToDevice));
+    if (mom2 && m->mom2_in) CK(copy_sync(m, m->mom2_in + tt.off, mom2, n * 4, cudaMemcpyHostToDevice));
+    mom1 = mom2 = nullptr;
+  }
   if (mom1 && m->mom1) CK(copy_sync(m, m->mom1 + tt.off, mom1, n * 4, cudaMemcpyHostToDevice));
   if (mom2 && m->mom2) CK(copy_sync(m, m->mom2 + tt.off, mom2, n * 4, cudaMemcpyHostToDevice));
   double tk[3] = {(double)t, 1.0 - std::pow((double)m->spec.beta1, (double)t), 1.0 - std::pow((double)m->spec.beta2, (double)t)};

@@ -8,6 +8,7 @@
 #include <stdlib.h>
 
 #include <algorithm>
+#include <atomic>
 
 #include <cuda_bf16.h>
 #include <math.h>
@@ -2081,6 +2082,163 @@ cudaError_t opt_update(float* theta, const float* grad, float* m, float* v, void
   auto al = [](const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; };
   const int vec = al(theta, 16) && al(grad, 16) && (!m || al(m, 16)) && (!v || al(v, 16)) && (!shadow || al(shadow, 8));
   opt_update_kernel<<<cdiv((n + 3) / 4, 256), 256, 0, s>>>(theta, grad, m, v, (bf16_t*)shadow, n, kind, lr, beta1, beta2, eps, wd, tick, vec);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// The undetached remainder (Section 2.2, Eq. 2): input of the main network and the embedding backward
+// ------------------------------------------------------------------------------------------
+// u[n, off_s .. off_s + w_s) = src_s[n, 0 .. w_s) for up to CONCAT_MAX sources: u = [z_0 | z_1 | ... | z_B]
+template <typename T>
+__global__ void __launch_bounds__(256) concat_kernel(ConcatArgs a, T* __restrict__ u, int rows) {
+  const int src = blockIdx.y;
+  const T* p = (const T*)a.src[src];
+  const int w = a.width[src], off = a.offset[src];
+  const long long n = (long long)rows * w;
+  for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n; i += (long long)gridDim.x * 256) {
+    const long long r = i / w;
+    const int c = (int)(i - r * w);
+    u[r * a.total + off + c] = p[r * a.ld[src] + c];
+  }
+}
+cudaError_t concat_cols(const ConcatArgs& a, void* u, int rows, bool bf16, cudaStream_t s) {
+  int wmax = 1;
+  for (int i = 0; i < a.n; i++) wmax = std::max(wmax, a.width[i]);
+  dim3 grid((unsigned)std::min<long long>(cdiv((long long)rows * wmax, 256), 148 * 4), a.n);
+  if (bf16) concat_kernel<bf16_t><<<grid, 256, 0, s>>>(a, (bf16_t*)u, rows);
+  else concat_kernel<float><<<grid, 256, 0, s>>>(a, (float*)u, rows);
+  return cudaGetLastError();
+}
+
+// Embedding backward, step 1: one CTA per table sorts (id, sample) pairs (bitonic, in shared memory),
+// so that the samples that read one table row are contiguous and in sample order, and numbers the
+// distinct rows: sorted_n[t][pos] = sample at sorted position pos, seg_start[t][s] = first position of
+// the s-th distinct row (seg_start[t][n_uniq] = batch), uniq_id[t][s] = that row, n_uniq[t].
+__global__ void __launch_bounds__(1024) embed_sort_kernel(const int32_t* __restrict__ ids, int batch, int ns, int table_rows, int npow2,
+                                                          int* __restrict__ sorted_n, int* __restrict__ seg_start,
+                                                          int* __restrict__ uniq_id, int* __restrict__ n_uniq) {
+  extern __shared__ unsigned long long keys[];
+  __shared__ int scan[1024];
+  const int t = blockIdx.x;
+  for (int i = threadIdx.x; i < npow2; i += 1024) {
+    unsigned long long k = ~0ull;                            // padding sorts to the end
+    if (i < batch) {
+      int id = ids[(long long)i * ns + t];
+      id = min(max(id, 0), table_rows - 1);                  // a bad id was reported by the input staging
+      k = ((unsigned long long)(unsigned)id << 32) | (unsigned)i;
+    }
+    keys[i] = k;
+  }
+  __syncthreads();
+  for (int size = 2; size <= npow2; size <<= 1)
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int i = threadIdx.x; i < npow2 / 2; i += 1024) {
+        const int lo = (i / stride) * stride * 2 + (i % stride), hi = lo + stride;
+        const bool up = (lo & size) == 0;
+        const unsigned long long a = keys[lo], b = keys[hi];
+        if ((a > b) == up) { keys[lo] = b; keys[hi] = a; }
+      }
+      __syncthreads();
+    }
+  // segment starts and their numbering: every thread owns a contiguous run of positions
+  const int per = (batch + 1023) / 1024, lo = threadIdx.x * per, hi = min(batch, lo + per);
+  int cnt = 0;
+  for (int i = lo; i < hi; i++) cnt += (i == 0 || (keys[i] >> 32) != (keys[i - 1] >> 32));
+  scan[threadIdx.x] = cnt;
+  __syncthreads();
+  for (int o = 1; o < 1024; o <<= 1) {                       // inclusive scan over the 1024 counts
+    const int v = threadIdx.x >= o ? scan[threadIdx.x - o] : 0;
+    __syncthreads();
+    scan[threadIdx.x] += v;
+    __syncthreads();
+  }
+  int seg = scan[threadIdx.x] - cnt;
+  int* sn = sorted_n + (long long)t * batch;
+  int* ss = seg_start + (long long)t * (batch + 1);
+  int* ui = uniq_id + (long long)t * batch;
+  for (int i = lo; i < hi; i++) {
+    sn[i] = (int)(keys[i] & 0xffffffffu);
+    if (i == 0 || (keys[i] >> 32) != (keys[i - 1] >> 32)) {
+      ss[seg] = i;
+      ui[seg] = (int)(keys[i] >> 32);
+      seg++;
+    }
+  }
+  if (threadIdx.x == 1023) {
+    n_uniq[t] = scan[1023];
+    ss[scan[1023]] = batch;
+  }
+}
+
+// Step 2: one warp per distinct row: grow[t][s][:] = sum over the samples of segment s, in sample order,
+// of dz0[n, t*e : (t+1)*e] -- the scatter-add without atomics (one writer, fixed order).
+template <typename T>
+__global__ void __launch_bounds__(256) embed_rows_kernel(const T* __restrict__ dz0, long long ld, int batch, int e,
+                                                         const int* __restrict__ sorted_n, const int* __restrict__ seg_start,
+                                                         const int* __restrict__ n_uniq, float* __restrict__ grow) {
+  const int t = blockIdx.y, seg = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (seg >= n_uniq[t]) return;
+  const int* sn = sorted_n + (long long)t * batch;
+  const int* ss = seg_start + (long long)t * (batch + 1);
+  const int beg = ss[seg], end = ss[seg + 1];
+  for (int c = lane; c < e; c += 32) {
+    float acc = 0.f;
+    for (int pos = beg; pos < end; pos++) acc += ldf(dz0 + (long long)sn[pos] * ld + t * e + c);
+    grow[((long long)t * batch + seg) * e + c] = acc;
+  }
+}
+
+// Step 3: the optimizer on the touched rows only (untouched rows keep values and moments; the bias
+// correction is the global one in tick[]); the same element update as the dense optimizer.
+__global__ void __launch_bounds__(256) embed_update_kernel(float* __restrict__ tables, long long table_stride, float* __restrict__ m,
+                                                           float* __restrict__ v, int batch, int e, const int* __restrict__ uniq_id,
+                                                           const int* __restrict__ n_uniq, const float* __restrict__ grow, int kind,
+                                                           float lr, float b1, float b2, float eps, float wd,
+                                                           const double* __restrict__ tick) {
+  const int t = blockIdx.y, seg = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (seg >= n_uniq[t]) return;
+  float bc1 = 1.f, bc2 = 1.f;
+  if (kind != 0) { bc1 = (float)tick[1]; bc2 = (float)tick[2]; }
+  const long long base = (long long)t * table_stride + (long long)uniq_id[(long long)t * batch + seg] * e;
+  for (int c = lane; c < e; c += 32) {
+    float th = tables[base + c], mm = 0.f, vv = 0.f;
+    if (kind != 0) { mm = m[base + c]; vv = v[base + c]; }
+    opt_element(th, grow[((long long)t * batch + seg) * e + c], mm, vv, kind, lr, b1, b2, eps, wd, bc1, bc2);
+    if (kind != 0) { m[base + c] = mm; v[base + c] = vv; }
+    tables[base + c] = th;
+  }
+}
+
+int embed_max_batch() { return 16384; }
+
+cudaError_t embed_backward(const void* dz0, long long ld, const int32_t* ids, int batch, int ns, int e, int table_rows, int* sorted_n,
+                           int* seg_start, int* uniq_id, int* n_uniq, float* grow, bool bf16, cudaStream_t s) {
+  int npow2 = 1;
+  while (npow2 < batch) npow2 <<= 1;
+  const size_t smem = (size_t)npow2 * sizeof(unsigned long long);
+  static std::atomic<size_t> attr[64];
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev < 0 || dev >= 64) dev = 0;
+  if (smem > 48 * 1024 && smem > attr[dev].load()) {
+    cudaError_t e2 = cudaFuncSetAttribute(embed_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e2 != cudaSuccess) return e2;
+    attr[dev].store(smem);
+  }
+  embed_sort_kernel<<<ns, 1024, smem, s>>>(ids, batch, ns, table_rows, npow2, sorted_n, seg_start, uniq_id, n_uniq);
+  cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess) return err;
+  dim3 grid(cdiv(batch, 8), ns);
+  if (bf16) embed_rows_kernel<bf16_t><<<grid, 256, 0, s>>>((const bf16_t*)dz0, ld, batch, e, sorted_n, seg_start, n_uniq, grow);
+  else embed_rows_kernel<float><<<grid, 256, 0, s>>>((const float*)dz0, ld, batch, e, sorted_n, seg_start, n_uniq, grow);
+  return cudaGetLastError();
+}
+
+cudaError_t embed_update(float* tables, long long table_stride, float* m, float* v, int batch, int ns, int e, const int* uniq_id,
+                         const int* n_uniq, const float* grow, int kind, float lr, float beta1, float beta2, float eps, float wd,
+                         const double* tick, cudaStream_t s) {
+  dim3 grid(cdiv(batch, 8), ns);
+  embed_update_kernel<<<grid, 256, 0, s>>>(tables, table_stride, m, v, batch, e, uniq_id, n_uniq, grow, kind, lr, beta1, beta2, eps, wd, tick);
   return cudaGetLastError();
 }
 

@@ -204,6 +204,28 @@ cudaError_t dot_fwd(const void* proj, const void* x0, long long ldx0, void* feat
 cudaError_t dot_bwd(const void* dfeat, const void* x0, long long ldx0, void* dproj, int batch, int ns,
                     int e, int fw, bool bf16, cudaStream_t s);
 
+// u = [src_0 | src_1 | ...] column-wise (the input of the main network, Eq. 2): u[r, offset_i + c] = src_i[r * ld_i + c]
+constexpr int CONCAT_MAX = 32;
+struct ConcatArgs {
+  int n = 0, total = 0;
+  const void* src[CONCAT_MAX];
+  int width[CONCAT_MAX], offset[CONCAT_MAX];
+  long long ld[CONCAT_MAX];
+};
+cudaError_t concat_cols(const ConcatArgs& a, void* u, int rows, bool bf16, cudaStream_t s);
+
+// Embedding backward (the main network's gradient into the input tables), deterministic scatter-add:
+// per table the (id, sample) pairs are sorted, distinct rows numbered, and one warp per distinct row
+// adds the samples' slices dz0[n, t*e:(t+1)*e] in sample order into grow[t][s][:]; uniq_id[t][s] names
+// the row, n_uniq[t] counts them.  sorted_n, uniq_id: ns*batch ints; seg_start: ns*(batch+1); grow: ns*batch*e floats.
+// batch <= embed_max_batch().  embed_update applies the optimizer to those rows only.
+int embed_max_batch();
+cudaError_t embed_backward(const void* dz0, long long ld, const int32_t* ids, int batch, int ns, int e, int table_rows, int* sorted_n,
+                           int* seg_start, int* uniq_id, int* n_uniq, float* grow, bool bf16, cudaStream_t s);
+cudaError_t embed_update(float* tables, long long table_stride, float* m, float* v, int batch, int ns, int e, const int* uniq_id,
+                         const int* n_uniq, const float* grow, int kind, float lr, float beta1, float beta2, float eps, float wd,
+                         const double* tick, cudaStream_t s);
+
 // Optimizer over a flat range.  kind 0 SGD, 1 Adam, 2 AdamW.  tick[0] = step count t (as float
 // bits of an int64 are avoided: tick is {t, 1-beta1^t, 1-beta2^t} kept on the device so that a
 // replayed CUDA graph advances it).  shadow (bf16 copy of theta) may be null.

@@ -92,6 +92,13 @@ def new_model(spec, flat):
     return m
 
 
+def _slots(params, state, b):
+    """Parameter and moment containers of block b, or of the trained input tables for b < 0."""
+    if b < 0:
+        return params["input"], state["m_in"], state["v_in"]
+    return params["blocks"][b], state["m"][b], state["v"][b]
+
+
 def compare_teacher_forced(spec, steps, seed=0, n_streams=2, flags=0, report=None, case=None, init_hook=None):
     """Each step: library and oracle start from the same fp32 parameters and optimizer state;
     losses and every gradient tensor, each on its own, must agree within TOL; the parameters
@@ -118,19 +125,25 @@ def compare_teacher_forced(spec, steps, seed=0, n_streams=2, flags=0, report=Non
             if it > 0:
                 for i in tidx:
                     b, name, _s, _t = tl[i]
-                    p32 = params["blocks"][b][name].astype(np.float32)
-                    params["blocks"][b][name] = p32.astype(np.float64)
-                    m32 = state["m"][b][name].astype(np.float32)
-                    v32 = state["v"][b][name].astype(np.float32)
-                    state["m"][b][name], state["v"][b][name] = m32.astype(np.float64), v32.astype(np.float64)
+                    pd, md, vd = _slots(params, state, b)
+                    p32 = pd[name].astype(np.float32)
+                    pd[name] = p32.astype(np.float64)
+                    m32 = md[name].astype(np.float32)
+                    v32 = vd[name].astype(np.float32)
+                    md[name], vd[name] = m32.astype(np.float64), v32.astype(np.float64)
                     m.set_params(i, p32)
                     m.set_opt_state(i, m32, v32, state["t"])
             m.step(n_streams=n_streams, flags=flags, **db.args())
             got_l = m.losses()
             # oracle: forward/backward at the operand values, optimizer on the fp32 masters
-            want_l, want_g = orc.forward_backward(spec, util.operand_params(spec, params), util.operand_batch(spec, batch))
-            new_params = {"input": params["input"], "blocks": []}
-            new_state = {"t": state["t"] + 1, "m": [], "v": []}
+            want_l, want_g, want_gin = orc.forward_backward(spec, util.operand_params(spec, params), util.operand_batch(spec, batch),
+                                                            want_input=True)
+            new_params = {"input": dict(params["input"]), "blocks": []}
+            new_state = {"t": state["t"] + 1, "m": [], "v": [], "m_in": dict(state["m_in"]), "v_in": dict(state["v_in"])}
+            touched = {k: orc.touched_rows(spec, batch, k) for k in want_gin}
+            for k, g in want_gin.items():       # trained input tables: the rows this batch read
+                new_params["input"][k], new_state["m_in"][k], new_state["v_in"][k] = orc.optimizer_update_rows(
+                    spec["opt"], params["input"][k], g, touched[k], state["m_in"][k], state["v_in"][k], state["t"] + 1)
             for b, p in enumerate(params["blocks"]):
                 np_, nm, nv = {}, {}, {}
                 for k in p:
@@ -148,8 +161,9 @@ def compare_teacher_forced(spec, steps, seed=0, n_streams=2, flags=0, report=Non
             for i in tidx:
                 b, name, _s, _t = tl[i]
                 g = m.grads(i)
-                err = synth.rel_l2(g, want_g[b][name])
-                key = f"b{b} {name}"
+                want = want_gin[name] if b < 0 else want_g[b][name]
+                err = synth.rel_l2(g, want)
+                key = f"b{b} {name}" if b >= 0 else f"input {name}"
                 worst[f"grad {key}"] = max(worst.get(f"grad {key}", 0), err)
                 if err > tol:
                     kind = "weight" if g.ndim == 2 else "bias"
@@ -158,25 +172,29 @@ def compare_teacher_forced(spec, steps, seed=0, n_streams=2, flags=0, report=Non
                         if probe is None:
                             probe = oracle_bf16_sensitivity(spec, util.operand_params(spec, params),
                                                             util.operand_batch(spec, batch))
-                        cond = synth.rel_l2(probe[b][name], want_g[b][name])
-                        entry = _allow_list().get((case, it, key))
+                        cond = synth.rel_l2(probe[b][name], want) if b >= 0 else None
+                        entry = _allow_list().get((case, it, key)) if b >= 0 else None
                     listed = entry is not None and entry["kind"] == kind
                     mult, cap = COND_RULE[kind]
-                    bound = min(cap, max(tol, mult * cond)) if listed else tol
+                    bound = min(cap, max(tol, mult * cond)) if listed and cond is not None else tol
                     print(f"[conditioning] case {case} step {it} {key}: err {err:.3e}, oracle bf16 sensitivity "
                           f"{cond if cond is None else format(cond, '.3e')}, listed {listed}, bound {bound:.3e}")
                     if report is not None:
                         report.setdefault("violations", []).append(
                             {"case": case, "step": it, "tensor": key, "err": float(err),
                              "sensitivity": None if cond is None else float(cond),
-                             "norm": float(np.linalg.norm(want_g[b][name])), "kind": kind})
+                             "norm": float(np.linalg.norm(want)), "kind": kind})
                     else:
                         assert err <= bound, (case, it, key, err, bound, cond,
                                               "" if listed else "not in tests/golden/bf16_conditioning_allow.json")
                 # optimizer alone: update rule in fp64 on the library's gradient
-                th, _, _ = orc.optimizer_update(spec["opt"], params["blocks"][b][name], g.astype(np.float64),
-                                                state["m"][b][name], state["v"][b][name], state["t"] + 1)
-                old = params["blocks"][b][name]
+                pd, md, vd = _slots(params, state, b)
+                if b < 0:
+                    th, _, _ = orc.optimizer_update_rows(spec["opt"], pd[name], g.astype(np.float64), touched[name],
+                                                         md[name], vd[name], state["t"] + 1)
+                else:
+                    th, _, _ = orc.optimizer_update(spec["opt"], pd[name], g.astype(np.float64), md[name], vd[name], state["t"] + 1)
+                old = pd[name]
                 pbound = OPT_TOL * np.linalg.norm(old) + OPT_TOL_UPDATE * np.linalg.norm(th - old)
                 perr = float(np.linalg.norm(m.params(i).astype(np.float64) - th)) / max(pbound, 1e-300)
                 worst["param/bound"] = max(worst.get("param/bound", 0), perr)

@@ -179,6 +179,38 @@ def test_config5_upper_sweep_two_blocks(w):
     _gu().compare_teacher_forced(spec, steps=1, seed=0, case=f"C5_w{w}_b512_two_blocks")
 
 
+@pytest.mark.parametrize("name", ["ctr_main_f32", "ctr_main_bf16", "ctr_main_frozen_tables", "mlp_main_bf16"])
+def test_main_network_and_embedding_backward(name):
+    """The undetached remainder of Eq. 2: a main network over [z_0 | sg z_1 | .. | sg z_B] with L_main,
+    its usual backward, and (CTR) the gradient into the embedding tables: scatter-add by id with many
+    repeated ids (Zipf draws on small tables), optimizer on the touched rows only.  Losses, every
+    gradient (tables included, dense) and the updated tables are compared with the oracle."""
+    adam = {"kind": "adam", "lr": 1e-3, "wd": 0.0, "beta1": 0.9, "beta2": 0.999, "eps": 1e-8}
+    if name == "ctr_main_f32":
+        spec = synth.with_main(synth.ctr_spec(batch=150, n_dense=13, n_sparse=5, table_rows=50, emb_dim=8, tower=(72, 40, 24),
+                                              n_cross=3, dtype="f32", opt=adam), tower=(64, 32))
+    elif name == "ctr_main_bf16":        # 2048 samples: a table row's gradient sums few samples, its bf16 noise falls with 1/sqrt(batch)
+        spec = synth.with_main(synth.ctr_spec(batch=2048, table_rows=1000, tower=(256, 128, 64)), tower=(256, 128))
+    elif name == "ctr_main_frozen_tables":
+        spec = synth.with_main(synth.ctr_spec(batch=256, table_rows=300, tower=(128, 64, 32)), tower=(128, 64), train_input=False)
+    else:                                # the first three blocks of the w128/b512 sweep point, on its well-conditioned seed
+        spec = synth.with_main(synth.mlp_spec(128, 512, 3, 512, "gelu", "bf16"), tower=(256, 64))
+    _gu().compare_teacher_forced(spec, steps=3 if name != "mlp_main_bf16" else 2, seed=5 if name != "mlp_main_bf16" else 4, case=name)
+
+
+def test_main_network_schedules_are_bit_identical():
+    from paper_2608_18469_b200 import binding
+    gu = _gu()
+    spec = synth.with_main(synth.ctr_spec(batch=256, table_rows=200, tower=(128, 64, 32)), tower=(128, 64))
+    flat = synth.init_params(spec, 7)
+    batches = [gu.DevBatch(spec, synth.make_batch(spec, 7, index=i)) for i in range(3)]
+    nb = len(spec["blocks"])
+    serial = gu.run_steps(spec, flat, batches, n_streams=1)
+    for ns, fl in ((nb + 1, 0), (3, binding.GRAPH), (nb + 1, binding.GRAPH | binding.EARLY_HEAD | binding.BLOCK_OPT | binding.SPLIT_BWD),
+                   (nb + 1, binding.PAR_FWD | binding.EARLY_HEAD)):
+        _bits_equal(serial, gu.run_steps(spec, flat, batches, n_streams=ns, flags=fl))
+
+
 def _edge_cases():
     s = {}
     s["mlp_bf16_batch1"] = synth.mlp_spec(64, 128, 2, 1, "gelu", "bf16")                 # a single row
