@@ -99,14 +99,15 @@ def _slots(params, state, b):
     return params["blocks"][b], state["m"][b], state["v"][b]
 
 
-def compare_teacher_forced(spec, steps, seed=0, n_streams=2, flags=0, report=None, case=None, init_hook=None):
+def compare_teacher_forced(spec, steps, seed=0, n_streams=2, flags=0, report=None, case=None, init_hook=None, label_p=None):
     """Each step: library and oracle start from the same fp32 parameters and optimizer state;
     losses and every gradient tensor, each on its own, must agree within TOL; the parameters
     after the optimizer must match the update rule applied in fp64 to the library's own gradients.
     `case` names the instance for the bf16 conditioning allow-list (see COND_CAP above); with
     `report` (a dict) nothing is asserted: worst errors and the list of tensors that would need
     the allow-list are collected instead.  `init_hook(values)` may edit the initial parameters in
-    place (a dict keyed by (block, tensor name)) before either side sees them."""
+    place (a dict keyed by (block, tensor name)) before either side sees them; `label_p` overrides the
+    probability of a positive label of the synthetic batches."""
     tol = TOL[spec["dtype"]]
     flat = synth.init_params(spec, seed)
     tl = synth.tensor_list(spec)
@@ -119,7 +120,7 @@ def compare_teacher_forced(spec, steps, seed=0, n_streams=2, flags=0, report=Non
     worst = {}
     try:
         for it in range(steps):
-            batch = synth.make_batch(spec, seed, index=it)
+            batch = synth.make_batch(spec, seed, index=it, label_p=label_p)
             db = DevBatch(spec, batch)
             # teacher forcing: library <- oracle state (rounded to fp32, oracle continues from the same)
             if it > 0:

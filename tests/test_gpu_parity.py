@@ -193,9 +193,14 @@ def test_main_network_and_embedding_backward(name):
         spec = synth.with_main(synth.ctr_spec(batch=2048, table_rows=1000, tower=(256, 128, 64)), tower=(256, 128))
     elif name == "ctr_main_frozen_tables":
         spec = synth.with_main(synth.ctr_spec(batch=256, table_rows=300, tower=(128, 64, 32)), tower=(128, 64), train_input=False)
-    else:                                # the first three blocks of the w128/b512 sweep point, on its well-conditioned seed
-        spec = synth.with_main(synth.mlp_spec(128, 512, 3, 512, "gelu", "bf16"), tower=(256, 64))
-    _gu().compare_teacher_forced(spec, steps=3 if name != "mlp_main_bf16" else 2, seed=5 if name != "mlp_main_bf16" else 4, case=name)
+    else:
+        # Dense input, nothing but the main network and the blocks to train.  With BALANCED labels this
+        # chain is ill-conditioned on almost every draw (the features of all samples are nearly the same
+        # vector, so every gradient is that vector times sum_n (sigmoid(s_n) - y_n), which cancels: the
+        # oracle's own bf16-storage sensitivity is 3e-2 .. 7e-2 on 9 of 11 seeds); 20 % positives keep the
+        # sum away from zero and the instance well conditioned.
+        spec = synth.with_main(synth.mlp_spec(128, 512, 3, 2048, "gelu", "bf16"), tower=(256, 64))
+    _gu().compare_teacher_forced(spec, steps=3, seed=5, case=name, label_p=0.2 if name == "mlp_main_bf16" else None)
 
 
 def test_main_network_schedules_are_bit_identical():
