@@ -499,6 +499,21 @@ struct Builder {
     if (bf && act == ACT_GELU) { ops.back().pew = 2; ops.back().ew_src = src; ops.back().ew_dst = d; ops.back().ew_n = n; }
   }
 
+  // Split count for a GEMM of `tiles` 256 x 256 CTA-pair tiles over a contraction of length `kdim`, written
+  // as fp32 partials: few tiles -> fill one wave of the 74 pairs; a little more than a whole number of
+  // waves (96 tiles: two waves, the second 30 % full) -> the split that fills its last wave best, as long
+  // as every split keeps at least 4096 of the contraction (C4's head dgrad, K = 32768: 393 -> 296 us).
+  static int pair_wave_splits(long long tiles, int kdim) {
+    const int smax = std::min(8, kdim / 1024);
+    if (smax < 2 || tiles < 1) return 1;
+    if (tiles <= 37) return (int)std::min<long long>(74 / tiles, smax);
+    auto eff = [&](int s) { const long long t = tiles * s; return (double)t / (74.0 * ((t + 73) / 74)); };
+    int best = 1;
+    for (int s = 2; s <= smax && kdim / s >= 4096; s++)     // (a split of a 3072-long contraction cost more in partials than it won: 47 -> 56 us)
+      if (eff(s) > eff(best) + 0.04) best = s;
+    return eff(best) >= eff(1) + 0.15 ? best : 1;
+  }
+
   // Y[M,N] = epi(X[M,K] W[N,K]^T)
   void lin_fwd(OpList& ops, const void* X, long long ldx, int widx, int bidx, void* Y, int M, int N, int K, Epilogue e) {
     GemmArgs g;
@@ -526,10 +541,7 @@ struct Builder {
     // (fp32 partials, summed in a fixed order and rounded once).
     const bool plain = !e.bias && e.act == ACT_NONE && !e.mul && !e.res && e.dact == ACT_NONE && !e.pre_out && e.alpha == 1.f;
     if (m->bf16 && plain && M >= 256 && K >= 256 && N >= 2048) {
-      const long long pair_tiles = (long long)((M + 255) / 256) * ((K + 255) / 256);
-      int splits = (int)(74 / pair_tiles);
-      if (splits > N / 1024) splits = N / 1024;
-      if (splits > 8) splits = 8;
+      const int splits = pair_wave_splits((long long)((M + 255) / 256) * ((K + 255) / 256), N);
       if (splits > 1) g.splits = splits;
     }
     gemm_tag = "gemm_dgrad";
@@ -824,11 +836,8 @@ struct Builder {
     q.c_f32 = 1;
     q.epi.ld_aux = d;
     int splits = 1;
-    if (rows >= 256 && d >= 256 && V >= 2048) {   // few output tiles, long contraction: split it over the CTA pairs
-      const long long pair_tiles = (long long)((rows + 255) / 256) * ((d + 255) / 256);
-      splits = (int)std::min<long long>(std::min<long long>(74 / pair_tiles, V / 1024), 8);
-      if (splits < 1) splits = 1;
-    }
+    if (rows >= 256 && d >= 256 && V >= 2048)     // few output tiles (or a badly filled last wave), long contraction: split it over the CTA pairs
+      splits = pair_wave_splits((long long)((rows + 255) / 256) * ((d + 255) / 256), V);
     float* part = f32_buf((size_t)splits * rows * d);
     q.splits = splits;
     if (splits > 1) { q.ws = part; q.C = part; q.ldc = d; }

@@ -1862,6 +1862,8 @@ bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan) {
   // CTA-pair kernel (256 x 256 tiles over two SMs) when its tiles keep most of the 74 pairs busy
   static const int env_pair = getenv("ERASE_TC_PAIR") ? atoi(getenv("ERASE_TC_PAIR")) : 1;
   const long long pair_tiles = (long long)((g.M + 2 * BM - 1) / (2 * BM)) * ((g.N + PAIR_BN - 1) / PAIR_BN) * g.splits;
+  // (GEMMs with a little more than one wave of pair tiles, e.g. C4's 96-tile N = 768 ones, were also tried as
+  // 128 x 256 single-CTA tiles, which fill two waves of 148 evenly: 3-14 % slower, so the pair kernel keeps them.)
   const bool want_pair = env_pair && (epilogue_is_simple(g) || !plan->a_mn) && g.M >= 256 && g.N > 128 && pair_tiles >= 56;
   if (want_pair) plan->bn = 256;
   if (getenv("ERASE_TC_BN")) { int f = atoi(getenv("ERASE_TC_BN")); if ((f == 64 || f == 128 || f == 256) && f <= (g.N + 63) / 64 * 64) plan->bn = f; }
