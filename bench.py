@@ -252,7 +252,7 @@ def pick_schedule(w, binding, spec, args, n_streams, gflags):
         w.warm(n_streams, gflags | f, POOL)
         r = w.leg(n_streams, gflags | f, max(4, min(args.steps, 10)), 2, per_step=False, min_s=0.0, max_repeats=2)
         trials.append((min(r["repeats"]), f, d))
-    best = min(trials)
+    best = w.rep.agree_on(min(trials))     # data-parallel ranks must all step with one schedule: rank 0's pick
     return gflags | best[1], best[2], {d.split(",")[0] + ("" if f == 0 else f" [flags {f}]"): round(t, 3) for t, f, d in trials}
 
 
@@ -282,14 +282,16 @@ class Workload:
     """One model with its pool of resident batches; everything that owns torch tensors, events or
     streams is dropped by close() before the model (and its CUDA streams) is destroyed."""
 
-    def __init__(self, torch, binding, spec, rep):
+    def __init__(self, torch, binding, spec, rep, data_parallel=False):
         self.torch, self.spec, self.rep = torch, spec, rep
         self.model = binding.Model(spec)
         self.model.set_all(synth.init_params(spec, 0))
+        if data_parallel:       # one model over all ranks: same parameters everywhere, each rank its own batches
+            rep.attach(self.model, binding.comm_unique_id)
         self.main = torch.cuda.ExternalStream(self.model.main_stream())
         self.host, self.dev = [], []
         for i in range(POOL):
-            b = synth.make_batch(spec, 0, index=i)
+            b = synth.make_batch(spec, 0, index=i + (POOL * rep.rank if data_parallel else 0))
             h = {}
             if spec["input"] == "dense":
                 x = torch.from_numpy(b["x"])
@@ -449,12 +451,14 @@ def run_gpu(args, spec, cfg_name):
     rank, world, dist = rep.rank, rep.world, rep.dist
     peaks = measured_peaks()
     nb = len(spec["blocks"])
+    if args.data_parallel:
+        spec = dict(spec, replicas=world)      # every loss is the mean over the global batch = world x batch
     n_streams, flags, eflags, sched_desc = schedule_flags(binding, spec, args)
     units = units_per_step(spec)
 
     sampler = ClockSampler(local)
     sampler.start()
-    w = Workload(torch, binding, spec, rep)
+    w = Workload(torch, binding, spec, rep, data_parallel=args.data_parallel)
     model = w.model
 
     # serial first (context), then the ERASE schedule; the clock sampler (started before the model
@@ -541,7 +545,9 @@ def run_gpu(args, spec, cfg_name):
                    "cuda_graph": not args.no_graph, "batch_pool": POOL,
                    "repeats": f"each leg = repeats of exactly {args.steps} steps until >= {MIN_LEG_S} s are timed; the median repeat is reported",
                    "l2": f"no flush: the step's working set ({arena_mb:.0f} MiB of stashes, logits, parameters) exceeds the 126 MB L2",
-                   "multi_gpu": "replicas only" if world > 1 else "single GPU"},
+                   "multi_gpu": (f"data parallel: one model on {world} shards of a global batch of {world} x {spec['batch']}, each block's "
+                                 "gradients summed over the ranks by one NCCL all-reduce right behind that block's backward, on its stream"
+                                 if args.data_parallel else "replicas only" if world > 1 else "single GPU")},
         "serial": {"value": serial_value, "ms_per_step": ser_ms / args.steps, "repeats_ms": [round(x, 3) for x in ser["repeats"]],
                    "p90": float(np.percentile(qps(ser_per), 90)), "median": float(np.median(qps(ser_per)))},
         "erase": {"p90": float(np.percentile(qps(era_per), 90)), "median": float(np.median(qps(era_per))),
@@ -561,9 +567,29 @@ def run_gpu(args, spec, cfg_name):
         "cpu_baseline": cpu,
         "per_config": table,
     }
-    print(json.dumps(line), flush=True)
+    emit(json.dumps(line))
     if dist is not None:
         rep.close()
+
+
+_STDOUT_FD = None
+
+
+def quiet_stdout():
+    """Libraries loaded during the run (NCCL prints its version banner) write to file descriptor 1: send it to
+    stderr for the duration, so that the JSON line stays the only thing on stdout."""
+    global _STDOUT_FD
+    sys.stdout.flush()
+    _STDOUT_FD = os.dup(1)
+    os.dup2(2, 1)
+
+
+def emit(text):
+    sys.stdout.flush()
+    if _STDOUT_FD is None:
+        print(text, flush=True)
+    else:
+        os.write(_STDOUT_FD, (text + "\n").encode())
 
 
 def main():
@@ -584,7 +610,12 @@ def main():
                     help="parallel topology: keep the blocks' forwards on the main stream, one after the other")
     ap.add_argument("--no-split-bwd", action="store_true",
                     help="keep the parameter-gradient work of each B_b on the block's own side stream")
+    ap.add_argument("--data-parallel", action="store_true",
+                    help="N ranks train ONE model (per-block gradient all-reduce inside the step) instead of N independent "
+                         "replicas; runs without graph replay")
     args = ap.parse_args()
+    if args.data_parallel:
+        args.no_graph = True       # the library offers no graph replay around the exchange
     if args.impl == "ours":
         # at least 3 warm-up steps; with graph replay at least one per pooled batch, so that every
         # (batch pointers, schedule) graph is captured and instantiated before the timed region
@@ -593,6 +624,7 @@ def main():
     if args.impl == "reference":
         run_reference(args, spec, args.config)
     else:
+        quiet_stdout()
         run_gpu(args, spec, args.config)
 
 

@@ -50,7 +50,8 @@ typedef enum {
   ERASE_ECUDA = 3,        /* a CUDA call failed; text in erase_last_error()                  */
   ERASE_ESTATE = 4,       /* call not valid in this state (e.g. step before parameters set)  */
   ERASE_ETIMEOUT = 5,     /* a bounded device-side wait expired; the step's results are void */
-  ERASE_EUNSUPPORTED = 6  /* valid request that this build does not implement                */
+  ERASE_EUNSUPPORTED = 6, /* valid request that this build does not implement                */
+  ERASE_ECOMM = 7         /* NCCL could not be loaded, or one of its calls failed            */
 } erase_status;
 
 typedef enum { ERASE_F32 = 0, ERASE_BF16 = 1 } erase_dtype;      /* operand/activation precision;
@@ -127,6 +128,10 @@ typedef struct {
                          values and moments).  Tables then count as trainable tensors: erase_grads
                          returns their dense gradient of the last step, erase_opt_state their moments.
                          batch <= 16384.                                                           */
+  int32_t replicas;   /* data-parallel replicas that train this model together (0 and 1: this model alone).
+                         Each replica steps on its own `batch` samples; every local loss is the mean over
+                         all replicas * batch samples, so a replica's own losses and gradients are its
+                         share of the sums (see erase_comm_init).                                 */
   void* arena;        /* DEVICE, optional: caller-owned memory the model lives in (256-byte
                          aligned); NULL = the library allocates with cudaMalloc                  */
   size_t arena_bytes; /* size of arena; at least erase_arena_bytes(spec)                         */
@@ -197,6 +202,13 @@ typedef struct {
                             ERASE_EUNSUPPORTED with the reason in erase_last_error().  May be combined with
                             ERASE_GRAPH and ERASE_NO_OPT; the stream-placement flags are ignored.          */
 
+#define ERASE_LOCAL_GRADS 256u /* step without the exchange between replicas: losses and gradients stay this
+                            replica's share of the global sums (they add up, over the replicas, to the
+                            losses and gradients of one model on the union of the batches).  For callers
+                            that exchange gradients themselves, usually with ERASE_NO_OPT, and for
+                            accumulating a large batch in pieces.  The only way to step a model built
+                            with replicas > 1 that has no communicator.                               */
+
 /* Device bytes erase_create needs for this spec when given an arena; 0 if the spec is invalid. */
 ERASE_API size_t erase_arena_bytes(const erase_model_spec* spec);
 
@@ -259,6 +271,37 @@ ERASE_API erase_status erase_sync(erase_model* m);
  * barriers inside the tensor-core kernels are this library's own, hence this check.)
  * Errors: EINVAL, ECUDA. */
 ERASE_API erase_status erase_selftest_timeout(erase_model* m, int32_t limit_us);
+
+/* Data-parallel replicas (Section 3: the CTR model is trained on eight GPUs with gradient
+ * synchronisation between them; Sections 2.2 and 4: once backward passes leave the main stream, every
+ * rank must still issue its collectives in one and the same order, or ranks wait on one another).
+ * One process per GPU holds one replica built from the
+ * same spec (replicas = world) and the same parameters.  A step then is: every replica runs F_b, l_b and
+ * B_b on its own batch; right behind B_b, on the stream B_b ran on, block b's slice of the fp32
+ * gradient arena is summed over the replicas in place (one NCCL all-reduce per block, so the exchange of
+ * block b overlaps F_{b+1..} exactly as B_b does); the B local losses are summed the same way at the
+ * join; the optimizer (of the block, with ERASE_BLOCK_OPT; else the sweep) follows the exchange, so every
+ * replica applies the same update to the same values and the replicas stay bit-identical to one
+ * another.  The order of the exchanges depends only on (n_streams, flags): pass the same to every replica.
+ *
+ * erase_comm_unique_id: fills 128 HOST bytes with a fresh NCCL id; call on one replica and carry the
+ *   bytes to the others by any means (a file, a socket, torch.distributed).
+ * erase_comm_init: collective over the replicas (blocks until all have called it, as
+ *   ncclCommInitRank does); the current CUDA device must be the model's.  world must equal the
+ *   spec's replicas (1 is allowed: a communicator of one, the exchange then changes nothing).  The
+ *   communicator lives until erase_destroy.
+ * erase_comm_order: the block index of every exchange the last step enqueued, in enqueue order
+ *   (-1 stands for the losses), at most cap entries; *n_out = their number.  Serial schedule:
+ *   B-1, .., 0, -1; ERASE: 0, .., B-1, -1.
+ * NCCL is loaded when first needed ("libnccl.so.2", or the file the environment variable
+ * ERASE_NCCL_LIB names).  A replica that stops stepping leaves the others waiting inside NCCL: the
+ * library adds no watchdog of its own.  Not offered with a communicator attached: ERASE_GRAPH, and
+ * train_input with world > 1 (sparse table gradients are not exchanged).
+ * Errors: EINVAL, ESTATE (a communicator is attached already), EUNSUPPORTED, ECOMM, ECUDA. */
+#define ERASE_COMM_ID_BYTES 128
+ERASE_API erase_status erase_comm_unique_id(void* id_out);
+ERASE_API erase_status erase_comm_init(erase_model* m, int32_t rank, int32_t world, const void* id);
+ERASE_API erase_status erase_comm_order(erase_model* m, int32_t* blocks_out, int32_t cap, int32_t* n_out);
 
 /* The CUDA stream (cudaStream_t) that steps start and end on; valid until erase_destroy.  A
  * caller may record its own events on it to time steps. */

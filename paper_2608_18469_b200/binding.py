@@ -15,8 +15,10 @@ import numpy as np
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "liberase_b200.so")
 
-OK, EINVAL, ENOMEM, ECUDA, ESTATE, ETIMEOUT, EUNSUPPORTED = range(7)
+OK, EINVAL, ENOMEM, ECUDA, ESTATE, ETIMEOUT, EUNSUPPORTED, ECOMM = range(8)
 GRAPH, NO_OPT, EARLY_HEAD, BLOCK_OPT, SPLIT_BWD, STAMPS, PAR_FWD, PERSISTENT = 1, 2, 4, 8, 16, 32, 64, 128
+LOCAL_GRADS = 256
+COMM_ID_BYTES = 128
 MAX_DIMS = 8
 
 _DTYPE = {"f32": 0, "bf16": 1}
@@ -40,7 +42,8 @@ class ModelSpec(C.Structure):
                 ("n_sparse", C.c_int32), ("table_rows", C.c_int32), ("emb_dim", C.c_int32),
                 ("n_blocks", C.c_int32), ("blocks", C.POINTER(BlockSpec)), ("opt", C.c_int32),
                 ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
-                ("weight_decay", C.c_float), ("train_input", C.c_int32), ("arena", C.c_void_p),
+                ("weight_decay", C.c_float), ("train_input", C.c_int32), ("replicas", C.c_int32),
+                ("arena", C.c_void_p),
                 ("arena_bytes", C.c_size_t)]
 
 
@@ -79,6 +82,9 @@ EXPORTS = {
     "erase_losses": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32]),
     "erase_sync": (C.c_int, [C.c_void_p]),
     "erase_selftest_timeout": (C.c_int, [C.c_void_p, C.c_int32]),
+    "erase_comm_unique_id": (C.c_int, [C.c_void_p]),
+    "erase_comm_init": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
+    "erase_comm_order": (C.c_int, [C.c_void_p, C.POINTER(C.c_int32), C.c_int32, C.POINTER(C.c_int32)]),
     "erase_main_stream": (C.c_void_p, [C.c_void_p]),
     "erase_launch_count": (C.c_int64, [C.c_void_p]),
     "erase_timeline": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32]),
@@ -131,8 +137,17 @@ def make_spec(spec, arena=None, arena_bytes=0):
                    blocks=C.cast(blocks, C.POINTER(BlockSpec)), opt=_OPT[o["kind"]], lr=o["lr"],
                    beta1=o.get("beta1", 0.9), beta2=o.get("beta2", 0.999), eps=o.get("eps", 1e-8),
                    weight_decay=o.get("wd", 0.0), train_input=1 if spec.get("train_input") else 0,
-                   arena=arena, arena_bytes=arena_bytes)
+                   replicas=spec.get("replicas", 0), arena=arena, arena_bytes=arena_bytes)
     return ms, blocks
+
+
+def comm_unique_id():
+    """A fresh NCCL id (128 bytes) for erase_comm_init; make it on one replica and send it to the others."""
+    buf = C.create_string_buffer(COMM_ID_BYTES)
+    st = lib().erase_comm_unique_id(buf)
+    if st != OK:
+        raise EraseError(st, lib().erase_last_error(None).decode())
+    return buf.raw
 
 
 def _fptr(a):
@@ -234,6 +249,19 @@ class Model:
 
     def selftest_timeout(self, limit_us=1000):
         self._ck(lib().erase_selftest_timeout(self.h, limit_us))
+
+    def comm_init(self, rank, world, unique_id):
+        """Collective over the replicas: attach an NCCL communicator made from ``unique_id`` (128 bytes)."""
+        buf = C.create_string_buffer(bytes(unique_id), COMM_ID_BYTES)
+        self._ck(lib().erase_comm_init(self.h, rank, world, buf))
+
+    def comm_order(self):
+        """Block index of every exchange the last step enqueued, in order (-1: the losses)."""
+        cap = self.n_blocks + 1
+        out = (C.c_int32 * cap)()
+        n = C.c_int32()
+        self._ck(lib().erase_comm_order(self.h, out, cap, C.byref(n)))
+        return [out[i] for i in range(min(n.value, cap))]
 
     def main_stream(self):
         return lib().erase_main_stream(self.h)

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liberase_b200.so")
-SOURCES = ["erase.cu", "kernels.cu", "gemm_tc.cu", "gemm_noalloc.cu", "attention_mma.cu", "attention_tc.cu"]
+SOURCES = ["erase.cu", "kernels.cu", "gemm_tc.cu", "gemm_noalloc.cu", "attention_mma.cu", "attention_tc.cu", "nccl_dyn.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 
@@ -42,7 +42,7 @@ def build(force=False, verbose=False):
             sys.stderr.write(out)
         if p.returncode:
             raise RuntimeError(f"nvcc failed on {src}")
-    subprocess.check_call([nvcc, "-shared", "-o", LIB, *objs, "-lcudart"])
+    subprocess.check_call([nvcc, "-shared", "-o", LIB, *objs, "-lcudart", "-ldl"])
     return LIB
 
 

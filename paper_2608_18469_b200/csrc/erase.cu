@@ -17,6 +17,7 @@
 #include <vector>
 
 #include "gemm_tc.cuh"
+#include "nccl_dyn.cuh"
 #include "kernels.cuh"
 
 using namespace erase;
@@ -132,6 +133,15 @@ struct erase_model {
   int* pdone = nullptr;          // device counters of the dual-list kernels, tc_dual_max() per stage
   bool persistent_ok = false;
   std::string persistent_why;
+
+  // Data-parallel replicas: every replica steps on its own rows; block b's slice of the gradient arena is
+  // summed over the replicas right behind B_b, on the stream B_b ran on.
+  int replicas = 1;                                  // the losses are means over replicas * rows rows
+  NcclComm comm = nullptr;
+  int comm_rank = 0, comm_world = 1;
+  bool exchange_on = false;                          // this step sums gradients and losses over the replicas
+  std::vector<std::pair<size_t, size_t>> blk_seg;    // per block: offset and length of its slice of the trainable arena
+  std::vector<int> exch_order;                       // block index of every exchange the last step enqueued, in order (-1: the losses)
 
   int sm_budget = 0;   // CTA cap for persistent GEMMs enqueued next (0 = all SMs); set per stream by the scheduler
   int64_t launches = 0;
@@ -271,6 +281,7 @@ bool validate(const erase_model_spec* s, std::string* why) {
     }
     prev = out;
   }
+  if (s->replicas < 0 || s->replicas > 65536) return bad("replicas out of range");
   if (s->train_input) {
     const erase_block_spec& last = s->blocks[s->n_blocks - 1];
     if (s->input != ERASE_IN_CTR || last.kind != ERASE_BLK_MAIN || !(last.flags & ERASE_MAIN_READS_INPUT))
@@ -681,7 +692,7 @@ struct Builder {
     int rows = m->rows;
     float* rowloss = f32_buf(rows);
     float* loss_out = m->losses + b;
-    float inv = 1.f / (float)rows;
+    float inv = 1.f / ((float)rows * (float)m->replicas);   // mean over every replica's rows: the replicas' gradients then simply add
     if (k.head == ERASE_HEAD_GOODNESS) {
       // Section 2.1: BCE on the goodness score G = sum_j z_j^2 with the logit G + bh.  The head has
       // no weight tensor, so its threshold sits where Wh would (index wh).
@@ -1212,6 +1223,7 @@ struct Builder {
       m->opt_tick_op.push_back({[=](cudaStream_t st) { return opt_tick(tick, b1, b2, st); }, 1});
       note(m->opt_tick_op, "opt_tick");
       m->opt_blk.resize(m->B);
+      m->blk_seg.assign(m->B, std::make_pair((size_t)0, (size_t)0));
       for (int b = 0; b < m->B; b++) {
         size_t lo = (size_t)-1, hi = 0;
         for (const Tensor& t : m->tensors)
@@ -1222,6 +1234,7 @@ struct Builder {
           }
         if (hi <= lo) continue;
         long long nb = (long long)(hi - lo);
+        m->blk_seg[b] = std::make_pair(lo, hi - lo);
         float* thb = th + lo; float* grb = gr + lo;
         float* m1b = m1 ? m1 + lo : nullptr; float* m2b = m2 ? m2 + lo : nullptr;
         void* shb = sh ? (void*)((__nv_bfloat16*)sh + lo) : nullptr;
@@ -1241,6 +1254,7 @@ erase_status init_model(erase_model* m, const erase_model_spec* spec, bool dry) 
   m->bf16 = spec->dtype == ERASE_BF16;
   m->esz = m->bf16 ? 2 : 4;
   m->rows = spec->batch * (spec->input == ERASE_IN_TOKENS ? spec->seq : 1);
+  m->replicas = spec->replicas > 1 ? spec->replicas : 1;
   m->dry = dry;
   if (!dry && spec->arena) {
     m->arena = (char*)spec->arena;
@@ -1265,6 +1279,28 @@ cudaError_t run_ops(erase_model* m, OpList& ops, cudaStream_t s) {
   }
   return cudaSuccess;
 }
+
+// Data-parallel exchange of block b (b = -1: the B local losses): an in-place sum over the replicas,
+// enqueued on the stream that just produced the values.  Every replica enqueues its exchanges in the
+// same order because the order is a function of (n_streams, flags) alone and the host enqueues in program order.
+erase_status exchange(erase_model* m, int b, cudaStream_t st) {
+  if (!m->exchange_on) return ERASE_OK;
+  float* buf = b < 0 ? m->losses : m->grad + m->blk_seg[b].first;
+  const size_t n = b < 0 ? (size_t)m->B : m->blk_seg[b].second;
+  m->exch_order.push_back(b);
+  if (n == 0) return ERASE_OK;
+  std::string why;
+  const NcclApi* api = nccl_api(&why);
+  if (!api) return m->fail(ERASE_ECOMM, why);
+  const int r = api->all_reduce(buf, buf, n, NCCL_FLOAT32, NCCL_SUM, m->comm, st);
+  if (r != 0) return m->fail(ERASE_ECOMM, std::string("ncclAllReduce: ") + api->error_string(r));
+  return ERASE_OK;
+}
+#define CKX(call)                          \
+  do {                                     \
+    erase_status x_ = (call);              \
+    if (x_ != ERASE_OK) return x_;         \
+  } while (0)
 
 // Persistent schedule: which operations of F_s and B_{s-1} go into stage s's dual-list kernel.
 // Qualifies: bf16 chains whose block bodies consist of tensor-core GEMMs and GELU passes (MLP and
@@ -1328,8 +1364,10 @@ erase_status enqueue_persistent(erase_model* m, unsigned flags) {
     for (Op* op : ps.covered)
       if (op->post) { CK(op->post(st)); m->launches += op->post_launches; }
     for (Op* op : ps.after) { CK(op->fn(st)); m->launches += op->launches; }
+    if (s >= 1) CKX(exchange(m, s - 1, st));                 // B_{s-1} is complete
     if (s < B) CK(run_ops(m, m->hfwd[s], st));
   }
+  CKX(exchange(m, -1, st));
   if (!(flags & ERASE_NO_OPT)) CK(run_ops(m, m->opt, st));
   return ERASE_OK;
 }
@@ -1362,6 +1400,7 @@ erase_status enqueue_step(erase_model* m, int n_streams, unsigned flags, int tim
       CK(mark(2 * (B + b), m->main));
       CK(run_ops(m, m->bwd[b], m->main));
       CK(mark(2 * (B + b) + 1, m->main));
+      CKX(exchange(m, b, m->main));
     }
   } else {
     const int ns = n_streams - 1;
@@ -1422,6 +1461,7 @@ erase_status enqueue_step(erase_model* m, int n_streams, unsigned flags, int tim
         CK(cudaStreamWaitEvent(sd, e, 0));
       }
       CK(mark(2 * (B + b) + 1, sd));
+      CKX(exchange(m, b, sd));     // overlaps the later blocks' forwards like B_b itself; the optimizer waits for it
       if (block_opt) CK(run_ops(m, m->opt_blk[b], sd));
       if (block_opt && b == B - 1) CK(run_ops(m, m->opt_tables, sd));
       CK(cudaEventRecord(m->ev_b[b], sd));
@@ -1429,6 +1469,7 @@ erase_status enqueue_step(erase_model* m, int n_streams, unsigned flags, int tim
     for (int b = 0; b < B; b++) CK(cudaStreamWaitEvent(m->main, m->ev_b[b], 0));  // join
     m->sm_budget = 0;
   }
+  CKX(exchange(m, -1, m->main));
   CK(mark(4 * B, m->main));
   if (do_opt && !block_opt) CK(run_ops(m, m->opt, m->main));
   CK(mark(4 * B + 1, m->main));
@@ -1505,6 +1546,10 @@ void erase_destroy(erase_model* m) {
   if (m->main) cudaStreamSynchronize(m->main);
   for (auto s : m->side) if (s) cudaStreamSynchronize(s);
   for (auto s : m->leaf) if (s) cudaStreamSynchronize(s);
+  if (m->comm) {
+    if (const NcclApi* api = nccl_api(nullptr)) api->comm_destroy(m->comm);
+    m->comm = nullptr;
+  }
   for (auto& kv : m->graphs) cudaGraphExecDestroy(kv.second.first);
   for (auto e : m->ev_f) if (e) cudaEventDestroy(e);
   for (auto e : m->ev_b) if (e) cudaEventDestroy(e);
@@ -1653,8 +1698,15 @@ static erase_status check_step_args(erase_model* m, const erase_batch* batch);
 erase_status erase_step_ex(erase_model* m, const erase_batch* batch, int32_t n_streams, uint32_t flags) {
   if (!m) return ERASE_EINVAL;
   if (n_streams < 1) return m->fail(ERASE_EINVAL, "erase_step: n_streams must be >= 1");
-  if (flags & ~(ERASE_GRAPH | ERASE_NO_OPT | ERASE_EARLY_HEAD | ERASE_BLOCK_OPT | ERASE_SPLIT_BWD | ERASE_STAMPS | ERASE_PAR_FWD | ERASE_PERSISTENT))
+  if (flags & ~(ERASE_GRAPH | ERASE_NO_OPT | ERASE_EARLY_HEAD | ERASE_BLOCK_OPT | ERASE_SPLIT_BWD | ERASE_STAMPS | ERASE_PAR_FWD | ERASE_PERSISTENT |
+                ERASE_LOCAL_GRADS))
     return m->fail(ERASE_EINVAL, "erase_step: unknown flag");
+  m->exchange_on = m->comm != nullptr && !(flags & ERASE_LOCAL_GRADS);
+  if (m->replicas > 1 && !m->comm && !(flags & ERASE_LOCAL_GRADS))
+    return m->fail(ERASE_ESTATE, "erase_step: the model was built for several replicas: attach a communicator (erase_comm_init) or pass ERASE_LOCAL_GRADS");
+  if (m->exchange_on && (flags & ERASE_GRAPH))
+    return m->fail(ERASE_EUNSUPPORTED, "erase_step: ERASE_GRAPH is not offered while a communicator is attached (pass ERASE_LOCAL_GRADS to step without the exchange)");
+  flags &= ~ERASE_LOCAL_GRADS;   // not a property of the enqueued work: keeps graph keys and schedules as they were
   const bool persistent = (flags & ERASE_PERSISTENT) != 0;
   if (persistent) {
     if (!m->persistent_ok) return m->fail(ERASE_EUNSUPPORTED, "erase_step: ERASE_PERSISTENT: " + m->persistent_why);
@@ -1666,6 +1718,7 @@ erase_status erase_step_ex(erase_model* m, const erase_batch* batch, int32_t n_s
   if (cst != ERASE_OK) return cst;
   if (n_streams > m->B + 1) n_streams = m->B + 1;
   m->cur = *batch;
+  m->exch_order.clear();
   if (flags & ERASE_GRAPH) {
     GraphKey key{batch->x, batch->ids, batch->y, n_streams, flags};
     auto it = m->graphs.find(key);
@@ -1881,6 +1934,49 @@ erase_status erase_gemm(int32_t dtype, int32_t M, int32_t N, int32_t K, const vo
 #endif
   cleanup();
   if (hst != 0) { g_create_error = "erase_gemm: a bounded device-side wait expired (code " + std::to_string(hst) + ")"; return ERASE_ETIMEOUT; }
+  return ERASE_OK;
+}
+
+erase_status erase_comm_unique_id(void* id_out) {
+  if (!id_out) { g_create_error = "erase_comm_unique_id: id_out is NULL"; return ERASE_EINVAL; }
+  std::string why;
+  const NcclApi* api = nccl_api(&why);
+  if (!api) { g_create_error = "erase_comm_unique_id: " + why; return ERASE_ECOMM; }
+  NcclId id;
+  const int r = api->get_unique_id(&id);
+  if (r != 0) { g_create_error = std::string("ncclGetUniqueId: ") + api->error_string(r); return ERASE_ECOMM; }
+  std::memcpy(id_out, id.bytes, NCCL_ID_BYTES);
+  return ERASE_OK;
+}
+
+erase_status erase_comm_init(erase_model* m, int32_t rank, int32_t world, const void* id) {
+  if (!m) return ERASE_EINVAL;
+  if (!id || world < 1 || rank < 0 || rank >= world) return m->fail(ERASE_EINVAL, "erase_comm_init: id is NULL or rank/world out of range");
+  if (world != m->replicas) return m->fail(ERASE_EINVAL, "erase_comm_init: world differs from the spec's replicas");
+  if (m->comm) return m->fail(ERASE_ESTATE, "erase_comm_init: a communicator is already attached");
+  if (world > 1 && m->train_input)
+    return m->fail(ERASE_EUNSUPPORTED, "erase_comm_init: the sparse table gradients of train_input are not exchanged between replicas");
+  std::string why;
+  const NcclApi* api = nccl_api(&why);
+  if (!api) return m->fail(ERASE_ECOMM, "erase_comm_init: " + why);
+  erase_status st = erase_sync(m);
+  if (st != ERASE_OK) return st;
+  NcclId nid;
+  std::memcpy(nid.bytes, id, NCCL_ID_BYTES);
+  NcclComm c = nullptr;
+  const int r = api->comm_init_rank(&c, world, nid, rank);
+  if (r != 0) return m->fail(ERASE_ECOMM, std::string("ncclCommInitRank: ") + api->error_string(r));
+  m->comm = c;
+  m->comm_rank = rank;
+  m->comm_world = world;
+  return ERASE_OK;
+}
+
+erase_status erase_comm_order(erase_model* m, int32_t* blocks_out, int32_t cap, int32_t* n_out) {
+  if (!m) return ERASE_EINVAL;
+  if (!n_out || cap < 0 || (cap > 0 && !blocks_out)) return m->fail(ERASE_EINVAL, "erase_comm_order: bad argument");
+  *n_out = (int32_t)m->exch_order.size();
+  for (int32_t i = 0; i < cap && i < *n_out; i++) blocks_out[i] = m->exch_order[i];
   return ERASE_OK;
 }
 

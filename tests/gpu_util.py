@@ -209,14 +209,19 @@ def compare_teacher_forced(spec, steps, seed=0, n_streams=2, flags=0, report=Non
     return worst
 
 
-def run_steps(spec, flat, batches, n_streams, flags=0):
-    """Free-running steps; returns per-step losses and the final raw state for bit comparison."""
+def run_steps(spec, flat, batches, n_streams, flags=0, attach=None, orders=None):
+    """Free-running steps; returns per-step losses and the final raw state for bit comparison.
+    attach(model) runs once before the first step; orders (a list) receives every step's exchange order."""
     m = new_model(spec, flat)
     try:
+        if attach is not None:
+            attach(m)
         losses = []
         for db in batches:
             m.step(n_streams=n_streams, flags=flags, **db.args())
             losses.append(m.losses().copy())
+            if orders is not None:
+                orders.append(m.comm_order())
         tidx = util.trainable_index(spec)
         final = {"losses": np.array(losses)}
         for i in tidx:
