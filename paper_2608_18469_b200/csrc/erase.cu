@@ -1929,6 +1929,10 @@ erase_status erase_gemm(int32_t dtype, int32_t M, int32_t N, int32_t K, const vo
     fprintf(stderr, "   epilogue detail: staged %lld | store issued %lld | loop done %lld | fenced %lld | arrived %lld\n",
             h[10] - h[0], h[11] - h[0], h[12] - h[0], h[13] - h[0], h[6] - h[0]);
     if (getenv("ERASE_TC_PAIR")) fprintf(stderr, "   pair kernel: TMEM base of the leader %lld, of the peer %lld\n", h[8], h[9]);
+    if (getenv("ERASE_TC_WAITS"))
+      fprintf(stderr, "   pair kernel, CTA 0 (cycles): MMA thread first tile -> last operand wait %lld over %lld tiles | waiting for a drained accumulator %lld | "
+              "for operands %lld || epilogue warp 0: waiting for an accumulator %lld | draining %lld || producer waiting for a free stage %lld\n",
+              h[3] - h[0], h[10], h[1], h[2], h[4], h[5], h[7]);
     cudaFree(dbg);
   }
 #endif

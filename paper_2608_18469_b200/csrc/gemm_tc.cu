@@ -111,6 +111,9 @@ __device__ __forceinline__ void store8_bf16(__nv_bfloat16* p, int valid, bool ve
 // aux_a: 8 residual values, aux_b: 8 multiplier or derivative-source values (raw bf16).
 struct F8 { float v[8]; };
 
+// BIAS_REGS = false: bias8 points at this warp's slice of the bias in shared memory (two 16-byte loads);
+// true: at eight values the caller already holds in registers.
+template <bool BIAS_REGS = false>
 __device__ __forceinline__ F8 epilogue_values8(const TcArgs& p, F8 in, const float* bias8, uint4 aux_a, uint4 aux_b) {
   float* v = in.v;
   const Epilogue& e = p.epi;
@@ -119,11 +122,16 @@ __device__ __forceinline__ F8 epilogue_values8(const TcArgs& p, F8 in, const flo
 #pragma unroll
     for (int j = 0; j < 8; j++) v[j] *= e.alpha;
   }
-  if (e.bias) {   // this warp's slice of the bias was copied to shared memory while the tile was being multiplied
-    const float4 b0 = *reinterpret_cast<const float4*>(bias8);
-    const float4 b1 = *reinterpret_cast<const float4*>(bias8 + 4);
-    v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w;
-    v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+  if (e.bias) {
+    if (BIAS_REGS) {
+#pragma unroll
+      for (int j = 0; j < 8; j++) v[j] += bias8[j];
+    } else {
+      const float4 b0 = *reinterpret_cast<const float4*>(bias8);
+      const float4 b1 = *reinterpret_cast<const float4*>(bias8 + 4);
+      v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w;
+      v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+    }
   }
   if (e.act == ACT_RELU) {
 #pragma unroll
@@ -580,7 +588,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // Tiles are assigned round-robin to clusters, in the order of tile_coords.  The output must be
 // describable to TMA (it leaves through staged TMA stores); GENERAL as in tc_gemm_kernel.
 constexpr int PAIR_BN = 256;
-constexpr int PAIR_STAGES = 4;
+#ifndef PAIR_STAGES_N
+#define PAIR_STAGES_N 5
+#endif
+#ifndef PAIR_EPI_BUFS_N
+#define PAIR_EPI_BUFS_N 2
+#endif
+constexpr int PAIR_STAGES = PAIR_STAGES_N;
+constexpr int PAIR_EPI_BUFS = PAIR_EPI_BUFS_N;                      // 4 KB output staging buffers per epilogue warp
+constexpr uint32_t PAIR_EPI_BYTES = 4096u * PAIR_EPI_BUFS;
+constexpr uint32_t PAIR_BIAS_BYTES = 2u * 2u * (PAIR_BN / 2) * 4u;   // two column halves x two tile parities x 128 floats
 constexpr uint32_t PAIR_STAGE_BYTES = 2u * BM * BK * 2u;   // 128 x 64 of A + 128 x 64 of B, bf16
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -625,29 +642,34 @@ template <bool A_MN, bool B_MN, bool GENERAL, bool CE = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     const __grid_constant__ CUtensorMap map_c, const __grid_constant__ TcArgs p, const uint32_t tmem_cols) {
-  extern __shared__ uint8_t smem_raw[];
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
   constexpr int BN = PAIR_BN;
   constexpr int STAGES = PAIR_STAGES;
   constexpr uint32_t A_BYTES = BM * BK * 2;
   constexpr uint32_t STAGE_BYTES = PAIR_STAGE_BYTES;
   constexpr int CPW = BN / 2;
 
-  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  // The operand stages need a 1024-byte aligned base (128-byte swizzle); the kernel has no static shared
+  // memory, so the dynamic array starts the CTA's window.  Should it ever not, the kernel reports it and works on nothing.
+  const uint32_t smem_base = smem_u32(smem_raw);
   const uint32_t epi_base = smem_base + STAGES * STAGE_BYTES;
-  const uint32_t bias_base = epi_base + EPI_WARPS * EPI_STAGE_BYTES;
-  const uint32_t bar_base = bias_base + EPI_WARPS * EPI_BIAS_BYTES;
+  const uint32_t bar_base = epi_base + EPI_WARPS * PAIR_EPI_BYTES + PAIR_BIAS_BYTES;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
   uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
   volatile uint32_t* tmem_slot_ptr =
-      reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * (EPI_STAGE_BYTES + EPI_BIAS_BYTES) + 8u * (2 * STAGES + 4));
+      reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * PAIR_EPI_BYTES + PAIR_BIAS_BYTES + 8u * (2 * STAGES + 4));
   const uint32_t tmem_slot = bar_base + 8u * (2 * STAGES + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  __shared__ int dead_flag;
-  if (threadIdx.x == 0) dead_flag = status_peek(p.status) != 0 ? 1 : 0;
+  volatile int* dead_flag_ptr = reinterpret_cast<volatile int*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * PAIR_EPI_BYTES + PAIR_BIAS_BYTES + 8u * (2 * STAGES + 6));
+  if (threadIdx.x == 0) {
+    const bool misaligned = (smem_base & 1023u) != 0;
+    if (misaligned) atomicExch(p.status, 9);
+    *dead_flag_ptr = (misaligned || status_peek(p.status) != 0) ? 1 : 0;
+  }
   const uint32_t rank = cluster_ctarank();
   const bool leader = rank == 0;
   const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
@@ -686,7 +708,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   if (p.dbg && threadIdx.x == 0 && cluster_id == 0) p.dbg[8 + rank] = (long long)tmem_base;
 #endif
   int dead;   // both CTAs of the pair take the LEADER's reading, so that they skip (or work) together
-  asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(dead) : "r"(map_to_cta(smem_u32(&dead_flag), 0)) : "memory");
+  asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(dead) : "r"(map_to_cta(bar_base + 8u * (2 * STAGES + 6), 0)) : "memory");
 
   if (dead) {
     // the step is already void: do nothing but free TMEM below
@@ -705,7 +727,13 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         for (int kb = 0; kb < num_kb; kb++, it++) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
+#ifdef ERASE_DEV_AIDS
+          const long long w0 = clock64();
+#endif
           if (!mbar_wait(empty_bar(s), ph ^ 1)) { atomicExch(p.status, 1); ok = false; break; }
+#ifdef ERASE_DEV_AIDS
+          if (p.dbg && blockIdx.x == 0) p.dbg[7] += clock64() - w0;      // producer: waiting for a free stage
+#endif
           if (leader) mbar_expect_tx(full_bar(s), 2 * STAGE_BYTES);   // this CTA's bytes and the peer's
           const uint32_t lfull = map_to_cta(full_bar(s), 0);
           const uint32_t a_dst = smem_base + s * STAGE_BYTES;
@@ -742,13 +770,27 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         const int kbeg = split * kchunk, kend = min(p.K, kbeg + kchunk);
         const int num_kb = kend > kbeg ? (kend - kbeg + BK - 1) / BK : 0;
         const uint32_t ab = naccum == 2 ? (lt & 1) : 0u, aph = naccum == 2 ? ((lt >> 1) & 1) : (lt & 1);
+#ifdef ERASE_DEV_AIDS
+        const bool acct = p.dbg && blockIdx.x == 0;
+        long long w0 = acct ? clock64() : 0;
+        if (acct && lt == 0) p.dbg[0] = w0;
+#endif
         if (!mbar_wait(tempty_bar(ab), aph ^ 1)) { atomicExch(p.status, 4); ok = false; break; }
+#ifdef ERASE_DEV_AIDS
+        if (acct) { p.dbg[1] += clock64() - w0; p.dbg[10] += 1; }       // MMA thread: waiting for a drained accumulator
+#endif
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + ab * BN;
         for (int kb = 0; kb < num_kb; kb++, it++) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
+#ifdef ERASE_DEV_AIDS
+          w0 = acct ? clock64() : 0;
+#endif
           if (!mbar_wait(full_bar(s), ph)) { atomicExch(p.status, 2); ok = false; break; }
+#ifdef ERASE_DEV_AIDS
+          if (acct) { const long long w1 = clock64(); p.dbg[2] += w1 - w0; p.dbg[3] = w1; }   // MMA thread: waiting for operands
+#endif
           tc_fence_after();
           const uint32_t a_src = smem_base + s * STAGE_BYTES;
           const uint32_t b_src = a_src + A_BYTES;
@@ -771,9 +813,8 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const int ew = warp - 2;
     const int q = warp & 3;
     const int cbeg = (ew / 4) * CPW;
-    const uint32_t stage0 = epi_base + ew * EPI_STAGE_BYTES;
+    const uint32_t stage0 = epi_base + ew * PAIR_EPI_BYTES;
     uint32_t sbuf = 0;
-    float* bias_s = reinterpret_cast<float*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * EPI_STAGE_BYTES + ew * EPI_BIAS_BYTES);
     const bool f32 = p.splits > 1 || p.c_f32;
     const uint32_t ltempty0 = map_to_cta(tempty_bar(0), 0), ltempty1 = map_to_cta(tempty_bar(1), 0);
     bool store_pending = false;
@@ -785,13 +826,24 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       const int kbeg = split * kchunk, kend = min(p.K, kbeg + kchunk);
       const bool empty_k = kend <= kbeg;
       const uint32_t ab = naccum == 2 ? (lt & 1) : 0u, aph = naccum == 2 ? ((lt >> 1) & 1) : (lt & 1);
-      if (p.epi.bias && p.splits == 1) {
-        __syncwarp();
-        for (int j = lane; j < CPW; j += 32) {
-          const int n = n0 + cbeg + j;
-          bias_s[j] = n < p.N ? __ldg(p.epi.bias + n) : 0.f;
+      // Bias: the four warps that share a column half share one 128-float slice per tile parity.  Each warp
+      // fetches the slice into registers now (the latency hides behind the MMAs) and writes it -- every warp
+      // the same values -- once the tile's accumulator is complete: by then every warp of the pair has drained
+      // the tile before the previous one, the last reader of this parity's slice.  A warp reads only behind
+      // its own writes, so no barrier between the warps is needed.
+      const bool need_bias = p.epi.bias != nullptr && p.splits == 1;
+      float* bias_s = reinterpret_cast<float*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * PAIR_EPI_BYTES) + ((ew / 4) * 2 + (lt & 1)) * CPW;
+      float4 bias_pre = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (need_bias) {
+        const int n = n0 + cbeg + lane * 4;
+        const float* bp = p.epi.bias + n;
+        if (n + 4 <= p.N) {
+          bias_pre = __ldg(reinterpret_cast<const float4*>(bp));
+        } else {
+          if (n < p.N) bias_pre.x = __ldg(bp);
+          if (n + 1 < p.N) bias_pre.y = __ldg(bp + 1);
+          if (n + 2 < p.N) bias_pre.z = __ldg(bp + 2);
         }
-        __syncwarp();
       }
       const int row = m0 + q * 32 + lane;
       const bool row_ok = row < p.M;
@@ -809,12 +861,29 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         if (n0 + cbeg < p.N && (aux_pa || aux_pb)) aux_issue(aux_pa, aux_pb, row_ok, n0 + cbeg, p.N, aux_nxt);
       }
       const bool use_aux = GENERAL && (aux_pa || aux_pb);
+#ifdef ERASE_DEV_AIDS
+      const bool acct = p.dbg && blockIdx.x == 0 && threadIdx.x == 64;
+      const long long e0 = acct ? clock64() : 0;
+#endif
       bool ok = mbar_wait(tfull_bar(ab), aph);
       if (!ok) atomicExch(p.status, 3);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
+#ifdef ERASE_DEV_AIDS
+      const long long e1 = acct ? clock64() : 0;
+      if (acct) p.dbg[4] += e1 - e0;                                   // epilogue warp 0: waiting for a finished accumulator
+#endif
+      if (need_bias) {
+        *reinterpret_cast<float4*>(bias_s + lane * 4) = bias_pre;
+        __syncwarp();
+      }
       const bool rows_in = m0 + q * 32 < p.M;      // warp-uniform: any of this warp's 32 rows inside the matrix
+#ifdef ERASE_DEV_AIDS
+      const long long dflags = p.dbg ? p.dbg[15] : 0;   // 1: no TMA stores, 2: no TMEM loads, 4: no staging writes
+#else
+      constexpr long long dflags = 0;
+#endif
       if (n0 + cbeg < p.N) {
 #pragma unroll 1
         for (int cc = 0; cc < CPW; cc += 32) {
@@ -825,15 +894,21 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             if (cc + 32 < CPW && n0 + c0 + 32 < p.N) aux_issue(aux_pa, aux_pb, row_ok, n0 + c0 + 32, p.N, aux_nxt);
           }
           uint32_t r[32];
-          if (!empty_k) {
-            tc_ld32(tmem_base + ab * BN + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+          const bool from_tmem = !empty_k && !(dflags & 2);
+          if (from_tmem) tc_ld32_issue(tmem_base + ab * BN + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+          if (from_tmem) {
+            tc_ld_wait(r);
           } else {
 #pragma unroll
             for (int j = 0; j < 32; j++) r[j] = 0u;
           }
           if (f32 || (cc & 63) == 0) {
-            sbuf ^= 1;
-            if (lane == 0 && store_pending) tma_store_wait_read1();
+            if (PAIR_EPI_BUFS == 2) {
+              sbuf ^= 1;
+              if (lane == 0 && store_pending) tma_store_wait_read1();
+            } else if (lane == 0 && store_pending) {
+              asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            }
             __syncwarp();
           }
           const uint32_t stage = stage0 + sbuf * 4096;
@@ -865,7 +940,9 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             } else if (GENERAL && !p.plain && p.splits == 1 && row_ok && n0 + c0 + g8 * 8 < p.N) {
               f = epilogue_values8(p, f, bias_s + cc + g8 * 8, aux_cur.a[g8], aux_cur.b[g8]);
             }
-            if (f32) {
+            if (dflags & 4) {
+              if (v[0] == 123.456f) st_shared_v4(my_row, 0u, 0u, 0u, 0u);     // keeps the values alive without the writes
+            } else if (f32) {
               const uint32_t s0 = my_row + (((2 * g8) ^ (lane & 7)) << 4), s1 = my_row + (((2 * g8 + 1) ^ (lane & 7)) << 4);
               st_shared_v4(s0, __float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]));
               st_shared_v4(s1, __float_as_uint(v[4]), __float_as_uint(v[5]), __float_as_uint(v[6]), __float_as_uint(v[7]));
@@ -878,7 +955,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           if (f32 || last_chunk) {
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
-            if (lane == 0 && rows_in) {
+            if (lane == 0 && rows_in && !(dflags & 1)) {
               const int x = f32 ? n0 + c0 : n0 + cbeg + (cc & ~63), y = m0 + q * 32;
               if (p.splits > 1) tma_store_3d(&map_c, stage, x, y, split);
               else tma_store_2d(&map_c, stage, x, y);
@@ -892,6 +969,9 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         p.epi.ce_psum[(long long)row * p.epi.ce_groups + (n0 + cbeg) / CPW] = ce_sum;
       tc_fence_before();
       __syncwarp();
+#ifdef ERASE_DEV_AIDS
+      if (acct) p.dbg[5] += clock64() - e1;                            // epilogue warp 0: draining one accumulator
+#endif
       if (lane == 0) {   // accumulator drained: tell the leader's MMA thread
         if (leader) mbar_arrive(tempty_bar(ab));
         else mbar_arrive_cluster(ab ? ltempty1 : ltempty0);
@@ -1613,7 +1693,8 @@ cudaError_t launch_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int 
 
 template <bool A_MN, bool B_MN, bool GENERAL, bool CE = false>
 cudaError_t launch_pair_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas) {
-  constexpr size_t smem = (size_t)PAIR_STAGES * PAIR_STAGE_BYTES + EPI_WARPS * (EPI_STAGE_BYTES + EPI_BIAS_BYTES) + 8 * (2 * PAIR_STAGES + 16) + 1024;
+  constexpr size_t smem = (size_t)PAIR_STAGES * PAIR_STAGE_BYTES + EPI_WARPS * PAIR_EPI_BYTES + PAIR_BIAS_BYTES + 8 * (2 * PAIR_STAGES + 16);
+  static_assert(smem <= 232448, "pair kernel: shared memory over the per-CTA limit");
   static std::atomic<bool> attr_set[MAX_DEVICES];
   if (cudaError_t e = ensure_smem(tc_gemm_pair_kernel<A_MN, B_MN, GENERAL, CE>, smem, attr_set)) return e;
   TcArgs p;
