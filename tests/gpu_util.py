@@ -1,8 +1,5 @@
 """GPU-side test helpers: stage synthetic batches on the device (torch owns the memory) and
 compare the CUDA library with the oracle.  Imported only by tests marked gpu."""
-import json
-import os
-
 import numpy as np
 import torch
 
@@ -21,22 +18,13 @@ TOL = {"f32": 1e-4, "bf16": 2e-2}     # relative L2 PER TENSOR against the fp64 
 OPT_TOL = 2e-6
 OPT_TOL_UPDATE = 1e-5
 
-# bf16 only.  A gradient is a sum over samples; on some instances that sum nearly cancels (a bias
-# gradient on labels drawn independently of the inputs; every gradient of a block right after Adam's
-# first sign step on rare positives), and then no implementation that stores activations in bf16
-# keeps 2e-2 RELATIVE to what is left.  A tensor may exceed 2e-2 only if (a) its (case, step, tensor)
-# is listed in the committed allow-list below, which records the oracle-measured sensitivity of that
-# instance to bf16 storage, and (b) its error stays within a small multiple of the sensitivity
-# measured live, under a fixed cap: biases / LayerNorm shifts 3x and 1e-1, weight matrices 1.5x
-# and 5e-2.  Anything else fails.  The small synthetic cases avoid the list altogether by using
-# seeds on which the instance is well conditioned.
-COND_RULE = {"bias": (3.0, 1e-1), "weight": (1.5, 5e-2)}
-ALLOW_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "bf16_conditioning_allow.json")
-
-
-def _allow_list():
-    with open(ALLOW_PATH) as f:
-        return {(e["case"], e["step"], e["tensor"]): e for e in json.load(f)["entries"]}
+# bf16: a hard 2e-2 per tensor, no exceptions.  A gradient is a sum over samples; on some instances that
+# sum nearly cancels (a bias gradient on labels drawn independently of the inputs; every gradient of a
+# block right after Adam's first sign step on rare positives), and then no implementation that stores
+# activations in bf16 keeps 2e-2 RELATIVE to what is left.  The parity cases therefore run on seeds whose
+# instances are well conditioned (chosen by scanning seeds; the scan results are in the design notes);
+# when a tensor does fail, the message carries the oracle-measured sensitivity of that instance to bf16
+# storage (below), so that a conditioning problem can be told from a kernel bug at a glance.
 
 
 def oracle_bf16_sensitivity(spec, params, batch):
@@ -103,9 +91,8 @@ def compare_teacher_forced(spec, steps, seed=0, n_streams=2, flags=0, report=Non
     """Each step: library and oracle start from the same fp32 parameters and optimizer state;
     losses and every gradient tensor, each on its own, must agree within TOL; the parameters
     after the optimizer must match the update rule applied in fp64 to the library's own gradients.
-    `case` names the instance for the bf16 conditioning allow-list (see COND_CAP above); with
-    `report` (a dict) nothing is asserted: worst errors and the list of tensors that would need
-    the allow-list are collected instead.  `init_hook(values)` may edit the initial parameters in
+    `case` names the instance in messages; with `report` (a dict) nothing is asserted: worst errors and
+    the list of tensors over the tolerance are collected instead.  `init_hook(values)` may edit the initial parameters in
     place (a dict keyed by (block, tensor name)) before either side sees them; `label_p` overrides the
     probability of a positive label of the synthetic batches."""
     tol = TOL[spec["dtype"]]
@@ -167,27 +154,21 @@ def compare_teacher_forced(spec, steps, seed=0, n_streams=2, flags=0, report=Non
                 key = f"b{b} {name}" if b >= 0 else f"input {name}"
                 worst[f"grad {key}"] = max(worst.get(f"grad {key}", 0), err)
                 if err > tol:
-                    kind = "weight" if g.ndim == 2 else "bias"
-                    cond, entry = None, None
-                    if spec["dtype"] == "bf16":
+                    cond = None
+                    if spec["dtype"] == "bf16" and b >= 0:      # diagnostic only: how ill-conditioned is this instance?
                         if probe is None:
                             probe = oracle_bf16_sensitivity(spec, util.operand_params(spec, params),
                                                             util.operand_batch(spec, batch))
-                        cond = synth.rel_l2(probe[b][name], want) if b >= 0 else None
-                        entry = _allow_list().get((case, it, key)) if b >= 0 else None
-                    listed = entry is not None and entry["kind"] == kind
-                    mult, cap = COND_RULE[kind]
-                    bound = min(cap, max(tol, mult * cond)) if listed and cond is not None else tol
-                    print(f"[conditioning] case {case} step {it} {key}: err {err:.3e}, oracle bf16 sensitivity "
-                          f"{cond if cond is None else format(cond, '.3e')}, listed {listed}, bound {bound:.3e}")
+                        cond = synth.rel_l2(probe[b][name], want)
+                    print(f"[parity] case {case} step {it} {key}: err {err:.3e} > {tol:.0e}; oracle bf16 sensitivity of this "
+                          f"instance {cond if cond is None else format(cond, '.3e')}")
                     if report is not None:
                         report.setdefault("violations", []).append(
                             {"case": case, "step": it, "tensor": key, "err": float(err),
                              "sensitivity": None if cond is None else float(cond),
-                             "norm": float(np.linalg.norm(want)), "kind": kind})
+                             "norm": float(np.linalg.norm(want))})
                     else:
-                        assert err <= bound, (case, it, key, err, bound, cond,
-                                              "" if listed else "not in tests/golden/bf16_conditioning_allow.json")
+                        assert err <= tol, (case, it, key, err, tol, "oracle bf16 sensitivity", cond)
                 # optimizer alone: update rule in fp64 on the library's gradient
                 pd, md, vd = _slots(params, state, b)
                 if b < 0:
