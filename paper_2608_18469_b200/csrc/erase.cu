@@ -450,14 +450,15 @@ struct Builder {
     jobs_flops = jobs_bytes = 0;
   }
 
-  void gemm(OpList& ops, GemmArgs g) {
+  void gemm(OpList& ops, GemmArgs g, bool* xcol_used = nullptr) {
     size_t before = ops.size();
-    gemm_inner(ops, g);
+    gemm_inner(ops, g, xcol_used);
     double fl = 2.0 * g.M * g.N * g.K;
     double by = ((double)g.M * g.K + (double)g.N * g.K) * m->esz + (double)g.M * g.N * (g.c_f32 ? 4 : m->esz);
     if (ops.size() > before) note(ops, gemm_tag, fl, by);
   }
-  void gemm_inner(OpList& ops, GemmArgs g) {
+  void gemm_inner(OpList& ops, GemmArgs g, bool* xcol_used = nullptr) {
+    if (xcol_used) *xcol_used = false;
     const bool bf = m->bf16;
     const bool tc_ok = bf && tc_gemm_supported(g);
     void* out = g.C;
@@ -468,6 +469,7 @@ struct Builder {
     int* sched = tc_ok ? (int*)dev_alloc(m, 2 * sizeof(int), &ok) : nullptr;   // dynamic tile scheduler words (zeroed)
     const bool use_tc = tc_ok && !m->dry && tc_gemm_plan(g, m->status, &plan);
     plan.sched = sched;
+    if (use_tc && xcol_used) *xcol_used = plan.xcol != 0;
     if (use_tc) {
       if (g.splits > 1) {
         ops.push_back({[g, plan, out, ldo, out_bf, mm = m](cudaStream_t s) {
@@ -559,14 +561,19 @@ struct Builder {
     gemm(ops, g);
   }
   // dW[N,K] = dY[M,N]^T X[M,K]  (fp32, deterministic split over M), db[N] = column sums of dY
+  // xcol_out (with xcol_used): X has 16 more columns behind its K; ask the GEMM for dY^T times the first of them as
+  // well (GemmArgs::xcol_out).  *xcol_used says whether the plan took it; if not, the caller forms that product itself.
   void lin_wgrad(OpList& ops, const void* dY, const void* X, long long ldx, int widx, int bidx, int M, int N, int K,
-                 bool skip_bias = false, bool bias_now = false) {
+                 bool skip_bias = false, bool bias_now = false, float* xcol_out = nullptr, bool* xcol_used = nullptr) {
     GemmArgs g;
     g.M = N; g.N = K; g.K = M;
     g.A = dY; g.sa_m = 1; g.sa_k = N;
     g.B = X; g.sb_n = 1; g.sb_k = ldx;
     g.C = G(widx); g.ldc = K; g.c_f32 = 1;
+    g.xcol_out = xcol_out;
+    if (xcol_used) *xcol_used = false;
     if (groupable(g)) {   // a small weight gradient: runs with the block's other small ones in one launch
+      g.xcol_out = nullptr;
       group.push_back(g);
       if (bidx >= 0 && !skip_bias) {
         if (bias_now || (double)M * N * m->esz > 16.0e6) { bias_grad(ops, dY, N, M, N, bidx); ops.back().leaf = true; }
@@ -590,7 +597,8 @@ struct Builder {
     g.splits = splits < 1 ? 1 : splits;
     gemm_tag = "gemm_wgrad";
     const size_t before = ops.size();
-    gemm(ops, g);
+    if (g.splits > 1) g.xcol_out = nullptr;
+    gemm(ops, g, xcol_used);
     if (bidx >= 0 && !skip_bias) {
       // a large dY (the logits) is summed right behind its wgrad, while it is still in L2
       if (bias_now || (double)M * N * m->esz > 16.0e6) bias_grad(ops, dY, N, M, N, bidx);
@@ -801,7 +809,10 @@ struct Builder {
     float* rowscale = f32_buf(rows);
     int* tgt = (int*)dev_alloc(m, (size_t)rows * sizeof(int), &ok);
     int* bad = (int*)dev_alloc(m, (size_t)(rows + 1) * sizeof(int), &ok);
-    void* zs = act_buf((size_t)rows * d);
+    // r (.) z for the weight-gradient GEMM, each row followed by [r_n, 0 x 15]: with those the same GEMM also
+    // forms the bias gradient sum_n r_n P[n,:] (GemmArgs::xcol_out) where its plan allows
+    const int ldzs = d + 16;
+    void* zs = act_buf((size_t)rows * ldzs);
     g.epi.ce_ref = ref;
     g.epi.ce_psum = psum;
     TcPlan plan;
@@ -821,22 +832,27 @@ struct Builder {
     note(f, "ce_target_logit", 2.0 * rows * d, 4.0 * rows * d);
     f.push_back({[g, plan, mm](cudaStream_t s) { return tc_gemm_launch(g, plan, s, mm->sm_budget); }, 1});
     note(f, "gemm_fwd", 2.0 * rows * V * d, ((double)rows * d + (double)V * d) * 2 + 2.0 * rows * V);
-    f.push_back({[=](cudaStream_t s) { return ce_finalize(psum, groups, ref, lt, tgt, logits, V, z, zs, rowloss, rowscale, bad, rows, d, inv, s); }, 1});
+    f.push_back({[=](cudaStream_t s) { return ce_finalize(psum, groups, ref, lt, tgt, logits, V, z, zs, ldzs, rowloss, rowscale, bad, rows, d, inv, s); }, 1});
     note(f, "ce_finalize", (double)rows * groups, 4.0 * rows * groups + 4.0 * rows * d);
-    f.push_back({[=](cudaStream_t s) { return ce_fixup(bad, mm->status, tgt, z, Wb, bias, logits, ref, lt, zs, rowloss, rowscale, rows, d, V, inv, s); }, 1});
+    f.push_back({[=](cudaStream_t s) { return ce_fixup(bad, mm->status, tgt, z, Wb, bias, logits, ref, lt, zs, ldzs, rowloss, rowscale, rows, d, V, inv, s); }, 1});
     note(f, "ce_fixup", 0, 0);
     f.push_back({[=](cudaStream_t s) { return reduce_sum(rowloss, rows, inv, loss_out, s); }, 1});
     note(f, "loss_reduce", rows, 4.0 * rows);
     // backward: parameter gradients (leaves) ...
     const size_t before = bw.size();
-    lin_wgrad(bw, logits, zs, d, wh, -1, rows, V, d, true);
+    const int env_xcol = getenv("ERASE_HEAD_XCOL") ? atoi(getenv("ERASE_HEAD_XCOL")) : 1;   // 0: separate weighted column sum of P
+    bool db_in_wgrad = false;
+    lin_wgrad(bw, logits, zs, ldzs, wh, -1, rows, V, d, true, false, env_xcol ? G(bh) : nullptr, &db_in_wgrad);
     {
+      // (the scratch of the separate pass is laid out either way: the sizing pass cannot know the GEMM's plan)
       const int chunks = colsum_chunks(rows, V);
       float* ws = chunks > 1 ? f32_buf((size_t)chunks * V) : nullptr;
       float* out = G(bh);
       int* tk = tickets(V);
-      bw.push_back({[=](cudaStream_t s) { return colsum(logits, true, V, rows, V, rowscale, ws, chunks, tk, out, s); }, 1});
-      note(bw, "colsum", 2.0 * rows * V, 2.0 * rows * V);
+      if (!db_in_wgrad) {
+        bw.push_back({[=](cudaStream_t s) { return colsum(logits, true, V, rows, V, rowscale, ws, chunks, tk, out, s); }, 1});
+        note(bw, "colsum", 2.0 * rows * V, 2.0 * rows * V);
+      }
     }
     for (size_t i = before; i < bw.size(); i++) bw[i].leaf = true;
     // ... and the gradient chain: dz = r (.) (P W_h) from fp32 partials of the GEMM

@@ -55,6 +55,7 @@ struct TcArgs {
   int tma_c;       // C (or the split-K partials) leaves through shared memory + TMA store
   int plain;       // 1: the epilogue is the identity; 2: bias add only; 0: general
   int* sched;      // {next tile counter, finished CTAs}, zero between launches; null = static round-robin
+  float* xcol_out; // CTA-pair kernel: one more, 16-wide column tile at n = N whose first column goes here (GemmArgs::xcol_out)
 };
 
 __device__ __forceinline__ float bf2f(uint32_t bits16) { return __uint_as_float(bits16 << 16); }
@@ -679,7 +680,11 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_c) : "memory");
   }
-  const int tiles_m = (p.M + 2 * BM - 1) / (2 * BM), tiles_n = (p.N + BN - 1) / BN;
+  // xcol: behind the column tiles of C comes one narrow tile per row tile, at n = N (a multiple of BN), 16 wide
+  const bool xcol = p.xcol_out != nullptr;
+  const int tiles_n_main = (p.N + BN - 1) / BN;
+  const int tiles_m = (p.M + 2 * BM - 1) / (2 * BM), tiles_n = tiles_n_main + (xcol ? 1 : 0);
+  constexpr int XCOL_N = 16;
   const int total = tiles_m * tiles_n * p.splits;
   const int kchunk = (((p.K + p.splits - 1) / p.splits) + BK - 1) / BK * BK;
 
@@ -721,7 +726,8 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         int mt, nt, split;
         tile_coords(t, tiles_m, tiles_n, mt, nt, split);
         const int m0 = mt * 2 * BM + (int)rank * BM;        // this CTA's 128 rows of A
-        const int nb0 = nt * BN + (int)rank * (BN / 2);     // this CTA's 128 columns of B
+        const bool narrow = xcol && nt == tiles_n_main;
+        const int nb0 = narrow ? p.N + (int)rank * (XCOL_N / 2) : nt * BN + (int)rank * (BN / 2);     // this CTA's half of the tile's B columns
         const int kbeg = split * kchunk, kend = min(p.K, kbeg + kchunk);
         const int num_kb = kend > kbeg ? (kend - kbeg + BK - 1) / BK : 0;
         for (int kb = 0; kb < num_kb; kb++, it++) {
@@ -734,7 +740,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 #ifdef ERASE_DEV_AIDS
           if (p.dbg && blockIdx.x == 0) p.dbg[7] += clock64() - w0;      // producer: waiting for a free stage
 #endif
-          if (leader) mbar_expect_tx(full_bar(s), 2 * STAGE_BYTES);   // this CTA's bytes and the peer's
+          if (leader) mbar_expect_tx(full_bar(s), narrow ? 2 * (A_BYTES + BK * 128) : 2 * STAGE_BYTES);   // this CTA's bytes and the peer's
           const uint32_t lfull = map_to_cta(full_bar(s), 0);
           const uint32_t a_dst = smem_base + s * STAGE_BYTES;
           const uint32_t b_dst = a_dst + A_BYTES;
@@ -749,7 +755,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             tma_load_2d_pair(b_dst, &map_b, k0, nb0, lfull);
           } else {
 #pragma unroll
-            for (int a = 0; a < BN / 128; a++) tma_load_2d_pair(b_dst + a * (BK * 128), &map_b, nb0 + a * 64, k0, lfull);
+            for (int a = 0; a < (narrow ? 1 : BN / 128); a++) tma_load_2d_pair(b_dst + a * (BK * 128), &map_b, nb0 + a * 64, k0, lfull);
           }
         }
       }
@@ -766,7 +772,10 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       uint32_t it = 0, lt = 0;
       bool ok = true;
       for (int t = cluster_id; t < total && ok; t += n_clusters, lt++) {
-        const int split = t / (tiles_m * tiles_n);
+        int mt_, nt_, split;
+        tile_coords(t, tiles_m, tiles_n, mt_, nt_, split);
+        const bool narrow = xcol && nt_ == tiles_n_main;
+        const uint32_t idesc_t = narrow ? ((idesc & ~(0x3Fu << 17)) | ((uint32_t)(XCOL_N >> 3) << 17)) : idesc;
         const int kbeg = split * kchunk, kend = min(p.K, kbeg + kchunk);
         const int num_kb = kend > kbeg ? (kend - kbeg + BK - 1) / BK : 0;
         const uint32_t ab = naccum == 2 ? (lt & 1) : 0u, aph = naccum == 2 ? ((lt >> 1) & 1) : (lt & 1);
@@ -801,7 +810,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                                      : smem_desc(a_src + k * (UMMA_K * 2), 16, 1024);
             const uint64_t bd = B_MN ? smem_desc(b_src + k * (UMMA_K * 128), BK * 128, 1024)
                                      : smem_desc(b_src + k * (UMMA_K * 2), 16, 1024);
-            tc_mma_pair(tmem_d, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+            tc_mma_pair(tmem_d, ad, bd, idesc_t, (kb > 0 || k > 0) ? 1u : 0u);
           }
           tc_commit_pair(empty_bar(s));
         }
@@ -884,7 +893,18 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 #else
       constexpr long long dflags = 0;
 #endif
-      if (n0 + cbeg < p.N) {
+      if (xcol && nt == tiles_n_main) {            // the narrow tile: its first column is the extra product
+        if (cbeg == 0 && rows_in) {
+          uint32_t r[32];
+          if (!empty_k) {
+            tc_ld32(tmem_base + ab * BN + ((uint32_t)(q * 32) << 16), r);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; j++) r[j] = 0u;
+          }
+          if (row_ok) p.xcol_out[row] = __uint_as_float(r[0]);
+        }
+      } else if (n0 + cbeg < p.N) {
 #pragma unroll 1
         for (int cc = 0; cc < CPW; cc += 32) {
           const int c0 = cbeg + cc;
@@ -1673,6 +1693,7 @@ cudaError_t launch_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int 
   p.M = g.M; p.N = g.N; p.K = g.K;
   p.C = g.C; p.ldc = g.ldc; p.c_f32 = g.c_f32;
   p.splits = g.splits; p.ws = g.ws; p.epi = g.epi; p.status = plan.status; p.dbg = plan.dbg; p.sched = plan.sched;
+  p.xcol_out = nullptr;
   const int num_sms = sm_count();
   const long long total = (long long)((g.N + BN - 1) / BN) * ((g.M + BM - 1) / BM) * g.splits;
   long long cap = (max_ctas > 0 && max_ctas < num_sms) ? max_ctas : num_sms;
@@ -1701,12 +1722,13 @@ cudaError_t launch_pair_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s,
   p.M = g.M; p.N = g.N; p.K = g.K;
   p.C = g.C; p.ldc = g.ldc; p.c_f32 = g.c_f32;
   p.splits = g.splits; p.ws = g.ws; p.epi = g.epi; p.status = plan.status; p.dbg = plan.dbg; p.sched = nullptr;
+  p.xcol_out = plan.xcol ? g.xcol_out : nullptr;
   p.tma_c = 1;
   const Epilogue& e = g.epi;
   const bool no_aux = e.alpha == 1.f && e.act == ACT_NONE && !e.pre_out && !e.mul && !e.res && e.dact == ACT_NONE;
   p.plain = no_aux ? (e.bias ? (g.splits == 1 ? 2 : 1) : 1) : 0;   // 1: identity, 2: bias only, 0: general
   const int num_sms = sm_count();
-  const long long total = (long long)((g.N + PAIR_BN - 1) / PAIR_BN) * ((g.M + 2 * BM - 1) / (2 * BM)) * g.splits;
+  const long long total = (long long)((g.N + PAIR_BN - 1) / PAIR_BN + (plan.xcol ? 1 : 0)) * ((g.M + 2 * BM - 1) / (2 * BM)) * g.splits;
   long long cap = ((max_ctas > 1 && max_ctas < num_sms) ? max_ctas : num_sms) / 2;
   dim3 grid(2u * (unsigned)(total < cap ? total : cap));
   CUtensorMap ma, mb, mc;
@@ -1752,6 +1774,8 @@ TcDualPlan* tc_dual_plan(const DualItem* items_in, int n, int* done_dev, int* st
       if (items_in[i].list == l) items[cnt++] = items_in[i];
   }
   if (cnt != n) return nullptr;
+  for (int i = 0; i < n; i++)
+    if (items[i].kind == 0 && items[i].g.xcol_out) return nullptr;   // the extra-column product exists in the pair kernel only
   TcDualPlan* plan = new TcDualPlan();
   DualArgs& a = plan->args;
   memset(&a, 0, sizeof(a));
@@ -1954,8 +1978,11 @@ bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan) {
   if (!plan->a_mn) ok = encode_2d(plan->map_a, g.A, g.K, g.M, g.sa_m, BM);
   else ok = encode_2d(plan->map_a, g.A, g.M, g.K, g.sa_k, BK);
   if (!ok) return false;
+  // extra-column product: weight-gradient layout on the pair kernel, no split, N a multiple of the tile width
+  const bool want_xcol = g.xcol_out != nullptr && want_pair && plan->a_mn && plan->b_mn && g.splits == 1 && g.N % PAIR_BN == 0 &&
+                         plan->bn == 256;
   if (!plan->b_mn) ok = encode_2d(plan->map_b, g.B, g.K, g.N, g.sb_n, plan->bn);
-  else ok = encode_2d(plan->map_b, g.B, g.N, g.K, g.sb_k, BK);
+  else ok = encode_2d(plan->map_b, g.B, g.N + (want_xcol ? 16 : 0), g.K, g.sb_k, BK);
   if (!ok) return false;
   // outputs through TMA stores where their layout allows it (else the kernel stores directly)
   memset(plan->map_c, 0, sizeof(plan->map_c));
@@ -1987,6 +2014,9 @@ bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan) {
       plan->pair = okp ? 1 : 0;
     }
   }
+  plan->xcol = (want_xcol && plan->pair) ? 1 : 0;
+  if (want_xcol && !plan->xcol)     // the map was encoded 16 columns too wide for a kernel that will not read them: encode it again
+    if (!encode_2d(plan->map_b, g.B, g.N, g.K, g.sb_k, BK)) return false;
   return true;
 }
 

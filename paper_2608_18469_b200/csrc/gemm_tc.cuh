@@ -28,6 +28,7 @@ struct TcPlan {
   int* status = nullptr;  // device word set non-zero when a bounded wait expired
   int* sched = nullptr;   // two zero-initialised device ints for dynamic tile scheduling (null: static order)
   long long* dbg = nullptr;  // optional device buffer (16 slots) for clock64 stamps of CTA 0, development aid
+  int xcol = 0;              // the launch also forms GemmArgs::xcol_out (extra-column product)
 };
 
 // True if the tensor-core kernel can take this GEMM: bf16 operands, 16-byte aligned bases,

@@ -1506,6 +1506,16 @@ __device__ __forceinline__ void scale_row_bf16(const bf16_t* __restrict__ z, bf1
   }
 }
 
+// The 16 columns behind a scaled row (row stride d + 16): the row scale itself, then zeros.  The weight-gradient
+// GEMM multiplies P^T with them too, which makes the head's bias gradient sum_n r_n P[n,:] its 769th column.
+__device__ __forceinline__ void scale_row_tail(bf16_t* __restrict__ zs_row, int d, int ldzs, float r, int lane) {
+  if (ldzs >= d + 16 && lane < 2) {
+    const __nv_bfloat16 rb = __float2bfloat16_rn(r);
+    const uint32_t first = lane == 0 ? (uint32_t)(*reinterpret_cast<const unsigned short*>(&rb)) : 0u;
+    reinterpret_cast<uint4*>(zs_row + d)[lane] = make_uint4(first, 0u, 0u, 0u);
+  }
+}
+
 // One warp per row: S_n from the GEMM's partial sums (lanes stride over the groups, then a fixed
 // shuffle tree), loss_n, r_n, the patch P[n,t_n] -= S_n, the scaled copy r_n z_n for the
 // weight-gradient GEMM; rows whose sum left the safe range are appended to the list bad[1..]
@@ -1515,7 +1525,7 @@ __global__ void __launch_bounds__(256) ce_finalize_kernel(const float* __restric
                                                           bf16_t* __restrict__ P, int V, const bf16_t* __restrict__ z,
                                                           bf16_t* __restrict__ zs, float* __restrict__ rowloss,
                                                           float* __restrict__ rowscale, int* __restrict__ bad, int rows, int d,
-                                                          float inv_rows) {
+                                                          int ldzs, float inv_rows) {
   const int lane = threadIdx.x & 31;
   for (int n = blockIdx.x * 8 + (threadIdx.x >> 5); n < rows; n += gridDim.x * 8) {
     const float* ps = psum + (long long)n * groups;
@@ -1530,7 +1540,8 @@ __global__ void __launch_bounds__(256) ce_finalize_kernel(const float* __restric
       if (ok) P[(long long)n * V + tgt[n]] = __float2bfloat16_rn(expf(lt[n] - ref[n]) - S);   // the one-hot part of the gradient
       else bad[1 + atomicAdd(bad, 1)] = n;
     }
-    scale_row_bf16(z + (long long)n * d, zs + (long long)n * d, d, r, lane);
+    scale_row_bf16(z + (long long)n * d, zs + (long long)n * ldzs, d, r, lane);
+    scale_row_tail(zs + (long long)n * ldzs, d, ldzs, r, lane);
   }
 }
 
@@ -1542,7 +1553,7 @@ __global__ void __launch_bounds__(256) ce_fixup_kernel(const int* __restrict__ b
                                                        const bf16_t* __restrict__ z, const bf16_t* __restrict__ W, const float* __restrict__ bias,
                                                        bf16_t* __restrict__ P, float* __restrict__ ref, const float* __restrict__ lt,
                                                        bf16_t* __restrict__ zs, float* __restrict__ rowloss,
-                                                       float* __restrict__ rowscale, int d, int V, float inv_rows) {
+                                                       float* __restrict__ rowscale, int d, int ldzs, int V, float inv_rows) {
   __shared__ float red[8];
   if (status && *status != 0) return;      // the step is already void (an expired wait, a bad id): its sums mean nothing
   const int nbad = bad[0];
@@ -1583,7 +1594,10 @@ __global__ void __launch_bounds__(256) ce_fixup_kernel(const int* __restrict__ b
       rowscale[n] = r;
       P[(long long)n * V + tgt[n]] = __float2bfloat16_rn(expf(lt[n] - mx) - S);
     }
-    if (warp == 0) scale_row_bf16(z + (long long)n * d, zs + (long long)n * d, d, r, lane);
+    if (warp == 0) {
+      scale_row_bf16(z + (long long)n * d, zs + (long long)n * ldzs, d, r, lane);
+      scale_row_tail(zs + (long long)n * ldzs, d, ldzs, r, lane);
+    }
     __syncthreads();
   }
 }
@@ -1610,17 +1624,17 @@ cudaError_t ce_target_logit(const void* z, const void* W, const float* bias, con
   return cudaGetLastError();
 }
 cudaError_t ce_finalize(const float* psum, int groups, const float* ref, const float* lt, const int* tgt, void* P, int V, const void* z,
-                        void* zs, float* rowloss, float* rowscale, int* bad, int rows, int d, float inv_rows, cudaStream_t s) {
+                        void* zs, int ldzs, float* rowloss, float* rowscale, int* bad, int rows, int d, float inv_rows, cudaStream_t s) {
   const int grid = (int)std::min<long long>(cdiv(rows, 8), 148 * 8);
   ce_finalize_kernel<<<grid, 256, 0, s>>>(psum, groups, ref, lt, tgt, (bf16_t*)P, V, (const bf16_t*)z, (bf16_t*)zs, rowloss, rowscale, bad,
-                                          rows, d, inv_rows);
+                                          rows, d, ldzs, inv_rows);
   return cudaGetLastError();
 }
 cudaError_t ce_fixup(const int* bad, const int* status, const int* tgt, const void* z, const void* W, const float* bias, void* P, float* ref,
-                     const float* lt, void* zs, float* rowloss, float* rowscale, int rows, int d, int V, float inv_rows, cudaStream_t s) {
+                     const float* lt, void* zs, int ldzs, float* rowloss, float* rowscale, int rows, int d, int V, float inv_rows, cudaStream_t s) {
   const int grid = rows < 32 ? rows : 32;
   ce_fixup_kernel<<<grid, 256, 0, s>>>(bad, status, tgt, (const bf16_t*)z, (const bf16_t*)W, bias, (bf16_t*)P, ref, lt, (bf16_t*)zs, rowloss,
-                                       rowscale, d, V, inv_rows);
+                                       rowscale, d, ldzs, V, inv_rows);
   return cudaGetLastError();
 }
 cudaError_t ce_dz_finish(const float* part, int splits, int rows, int d, const float* rowscale, void* dz, cudaStream_t s) {

@@ -55,6 +55,13 @@ struct GemmArgs {
   int splits = 1;
   float* ws = nullptr;
   Epilogue epi;
+  // Weight-gradient layout on the CTA-pair tensor-core kernel only (A and B both strided over k, no split,
+  // N a multiple of 256): B carries 16 more columns behind its N (B(n, k) is valid for n < N + 16), and
+  // xcol_out[m] = sum_k A(m, k) B(N, k), the product with the first of them, fp32, M values.  With the local
+  // softmax head this is its bias gradient: A = P, column N of B = the row scales.  The extra columns cost one
+  // narrow tile per row tile (a 16-wide MMA on the A tiles the neighbouring column tiles are reading anyway)
+  // instead of a second pass over A.  tc_gemm_plan says whether a plan takes it (TcPlan::xcol).
+  float* xcol_out = nullptr;
 };
 
 cudaError_t gemm_simt(const GemmArgs& g, bool bf16, cudaStream_t s);
@@ -151,15 +158,16 @@ cudaError_t softmax_ce_inplace(void* logits, const int32_t* ids, int T, float* r
 //   ce_target_logit  tgt[n] (clamped), ref[n] = lt[n] = z_n . W[t_n] + bias[t_n]; clears bad[0]
 //   (head GEMM with Epilogue::ce_ref = ref writes P = exp(l - ref) and the partial sums psum)
 //   ce_finalize      rowloss, rowscale r_n = 1/(S_n rows), P[n,t_n] -= S_n, zs = r (.) z; unsafe rows -> bad[1..], bad[0] = count
+//                    (zs has row stride ldzs; with ldzs >= d + 16 each row ends in [r_n, 0 x 15]: GemmArgs::xcol_out)
 //   ce_fixup         recomputes the listed rows exactly (no-op when bad[0] == 0 or *status != 0); bad holds rows+1 ints
 //   ce_dz_finish     dz = r_n * (sum of `splits` fp32 partials of P W), rounded once
 // after which the gradient of the logits is r (.) P: dW = P^T zs, db = column sums of P weighted by r.
 cudaError_t ce_target_logit(const void* z, const void* W, const float* bias, const int32_t* ids, int T, int rows, int d, int V,
                             int* tgt, float* ref, float* lt, int* bad, cudaStream_t s);
 cudaError_t ce_finalize(const float* psum, int groups, const float* ref, const float* lt, const int* tgt, void* P, int V, const void* z,
-                        void* zs, float* rowloss, float* rowscale, int* bad, int rows, int d, float inv_rows, cudaStream_t s);
+                        void* zs, int ldzs, float* rowloss, float* rowscale, int* bad, int rows, int d, float inv_rows, cudaStream_t s);
 cudaError_t ce_fixup(const int* bad, const int* status, const int* tgt, const void* z, const void* W, const float* bias, void* P, float* ref,
-                     const float* lt, void* zs, float* rowloss, float* rowscale, int rows, int d, int V, float inv_rows, cudaStream_t s);
+                     const float* lt, void* zs, int ldzs, float* rowloss, float* rowscale, int rows, int d, int V, float inv_rows, cudaStream_t s);
 cudaError_t ce_dz_finish(const float* part, int splits, int rows, int d, const float* rowscale, void* dz, cudaStream_t s);
 
 // out[0] = (sum of v[0..n)) * scale, fixed-order tree in one CTA.

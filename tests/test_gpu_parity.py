@@ -114,6 +114,30 @@ def test_large_vocabulary_head(ce_mode, monkeypatch):
     _gu().compare_teacher_forced(spec, steps=1, seed=4, case="lm_vocab32000")
 
 
+@pytest.mark.parametrize("in_wgrad", ["1", "0"])
+def test_softmax_head_bias_gradient_inside_the_weight_gradient_gemm(in_wgrad, monkeypatch):
+    """d = 256, V = 16384: wide enough for the CTA-pair kernel (64 pair tiles), so the head's weight-gradient
+    GEMM takes the 16 extra columns behind r (.) z and its narrow tiles leave db_h = sum_n r_n P[n,:]; with the
+    switch off the same gradient comes from the separate weighted column sum over P.  Both against the oracle,
+    and the fix-up path (rows recomputed with the true maximum rewrite r_n and the extra column) with the first."""
+    monkeypatch.setenv("ERASE_HEAD_XCOL", in_wgrad)
+    gu = _gu()
+    spec = synth.lm_spec(1, 256, 4, 512, 64, 8, 16384)
+    m = gu.new_model(spec, synth.init_params(spec, 4))
+    try:
+        db = gu.DevBatch(spec, synth.make_batch(spec, 4))
+        names = [r["name"] for r in m.profile_step(**db.args())]
+        # the block's own bias gradients are batched reductions: the only plain column sum is the head's
+        assert ("colsum" in names) == (in_wgrad == "0"), names
+    finally:
+        m.close()
+    gu.compare_teacher_forced(spec, steps=2, seed=4, case="lm_head_bias_in_wgrad")
+    if in_wgrad == "1":
+        def lift(values):
+            values[(0, "bh")][7] += 150.0
+        gu.compare_teacher_forced(spec, steps=1, seed=4, case="lm_head_bias_in_wgrad_fixup", init_hook=lift)
+
+
 @pytest.mark.parametrize("name", ["lm_bf16_small", "lm_bf16_ragged_vocab", "C2"])
 def test_softmax_head_with_the_separate_softmax_pass(name, monkeypatch):
     """The path that heads which do not qualify for the exp epilogue take (fp32 models,
