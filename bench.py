@@ -38,7 +38,7 @@ MIN_LEG_S = 1.0     # every leg is repeated (K steps per repeat) until this much
 # of each kernel class (summaries under profiles/).  They sit below the algorithmic bytes where an
 # operand or result is still L2-resident.
 NCU_DRAM_BYTES = {"C2": {"gemm_fwd": 15.5e6, "gemm_dgrad": 75.4e6, "gemm_wgrad": 71.4e6},
-                  "C4": {"gemm_fwd": 567.5e6, "gemm_dgrad": 678.0e6, "gemm_wgrad": 706.2e6}}
+                  "C4": {"gemm_fwd": 567.6e6, "gemm_dgrad": 712.0e6, "gemm_wgrad": 736.8e6}}
 
 # the per-config table of the default run: (label, config name, keyword arguments)
 TABLE = [("C1", "C1", {}), ("C2", "C2", {}), ("C3", "C3", {}),
@@ -359,9 +359,11 @@ class Workload:
             if i == 0:
                 continue    # warm-up of the profiling path
             for r in recs:
-                a = agg.setdefault(r["name"], {"ms": 0.0, "flops": 0.0, "bytes": 0.0, "runs": 0, "launches": 0})
+                a = agg.setdefault(r["name"], {"ms": 0.0, "flops": 0.0, "bytes": 0.0, "runs": 0, "launches": 0, "big": {}})
                 a["ms"] += r["ms"]; a["flops"] += r["flops"]; a["bytes"] += r["bytes"]
                 a["runs"] += 1; a["launches"] += r["launches"]
+                b = a["big"].setdefault(r["flops"], {"ms": 0.0, "runs": 0})     # the class's members by size
+                b["ms"] += r["ms"]; b["runs"] += 1
         return agg
 
     def close(self):
@@ -390,6 +392,16 @@ def roofline_of(agg, peaks, cfg_name):
     roof["traffic_note"] = NCU_DRAM_NOTE.get(cfg_name) if tr else None
     tot = sum(x["ms"] for x in agg.values())
     roof["kernel_share"] = {k: round(v["ms"] / tot, 4) for k, v in sorted(agg.items(), key=lambda kv: -kv[1]["ms"])[:8]}
+    # the same figure for every tensor-bound class, and for the largest member of each (one launch kind: the local head's GEMM)
+    by = {}
+    for k, v in agg.items():
+        if not k.startswith("gemm") or v["flops"] <= 0:
+            continue
+        fl, b = max(v["big"].items(), key=lambda kv: kv[0])
+        by[k] = {"frac": round(v["flops"] / (v["ms"] * 1e-3) / 1e12 / peaks["tflops"], 4), "share": round(v["ms"] / tot, 4),
+                 "largest_launch": {"gflop": round(fl / 1e9, 2), "avg_launch_ms": round(b["ms"] / b["runs"], 4),
+                                    "frac": round(fl / (b["ms"] / b["runs"] * 1e-3) / 1e12 / peaks["tflops"], 4)}}
+    roof["tensor_classes"] = by
     return roof
 
 

@@ -1966,7 +1966,9 @@ bool tc_gemm_plan(const GemmArgs& g, int* status, TcPlan* plan) {
   plan->bn = g.N <= 64 ? 64 : (g.N >= 256 && tiles256 >= 148 ? 256 : 128);
   // CTA-pair kernel (256 x 256 tiles over two SMs) when its tiles keep most of the 74 pairs busy
   static const int env_pair = getenv("ERASE_TC_PAIR") ? atoi(getenv("ERASE_TC_PAIR")) : 1;
-  const long long pair_tiles = (long long)((g.M + 2 * BM - 1) / (2 * BM)) * ((g.N + PAIR_BN - 1) / PAIR_BN) * g.splits;
+  // (a request for the extra-column product brings one narrow tile per row tile: they count)
+  const bool xcol_shape = g.xcol_out != nullptr && g.sa_k != 1 && g.sb_k != 1 && g.splits == 1 && g.N % PAIR_BN == 0;
+  const long long pair_tiles = (long long)((g.M + 2 * BM - 1) / (2 * BM)) * ((g.N + PAIR_BN - 1) / PAIR_BN + (xcol_shape ? 1 : 0)) * g.splits;
   // (GEMMs with a little more than one wave of pair tiles, e.g. C4's 96-tile N = 768 ones, were also tried as
   // 128 x 256 single-CTA tiles, which fill two waves of 148 evenly: 3-14 % slower, so the pair kernel keeps them.)
   const bool want_pair = env_pair && (epilogue_is_simple(g) || !plan->a_mn) && g.M >= 256 && g.N > 128 && pair_tiles >= 56;
