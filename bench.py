@@ -233,6 +233,10 @@ def candidate_schedules(binding, spec, args):
     if chain and not args.no_split_bwd:
         out.append((binding.SPLIT_BWD, "ERASE, backward released after forward and local loss, parameter-gradient work of each "
                                        "backward on a second stream per block"))
+    if chain and not args.no_split_bwd:
+        out.append((binding.EARLY_HEAD | binding.SPLIT_BWD,
+                    "ERASE, local head+loss+backward of each block released onto side streams after the block body, parameter-gradient "
+                    "work of each backward on a second stream per block, one optimizer sweep after the join"))
     f = binding.EARLY_HEAD | binding.BLOCK_OPT
     d = "ERASE, local head+loss+backward+optimizer of each block released onto side streams after the block body"
     if chain and not args.no_split_bwd:
