@@ -41,6 +41,13 @@ constexpr uint32_t EPI_BIAS_BYTES = 512;              // up to 128 bias floats p
 constexpr int EPI_WARPS = 8;                       // two per TMEM lane quarter, each takes half the columns
 constexpr int TC_THREADS = 32 * (2 + EPI_WARPS);
 constexpr uint32_t EPI_STAGE_BYTES = 8192;             // two buffers of 32 rows x 128 bytes per epilogue warp
+// (one buffer instead of two, as in the CTA-pair kernel, was measured here as well: C3 2 % faster under the
+// overlapped schedule, the 512-wide MLP point 3 % slower, C1, C2 and the 128-wide point unchanged: two stay)
+#ifndef SINGLE_EPI_BUFS_N
+#define SINGLE_EPI_BUFS_N 2
+#endif
+constexpr int SINGLE_EPI_BUFS = SINGLE_EPI_BUFS_N;     // the single-CTA GEMM kernel's staging buffers per epilogue warp
+constexpr uint32_t SINGLE_EPI_BYTES = 4096u * SINGLE_EPI_BUFS;
 
 struct TcArgs {
   int M, N, K;
@@ -229,7 +236,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t epi_base = smem_base + STAGES * STAGE_BYTES;          // EPI_WARPS x 4 KB output staging
-  const uint32_t bias_base = epi_base + EPI_WARPS * EPI_STAGE_BYTES;    // EPI_WARPS x CPW floats of bias
+  const uint32_t bias_base = epi_base + EPI_WARPS * SINGLE_EPI_BYTES;    // EPI_WARPS x CPW floats of bias
   const uint32_t bar_base = bias_base + EPI_WARPS * EPI_BIAS_BYTES;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
@@ -241,9 +248,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   auto tq_empty = [&](int i) { return bar_base + 8u * (2 * STAGES + 10 + i); };
   uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
   volatile uint32_t* tmem_slot_ptr =
-      reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * (EPI_STAGE_BYTES + EPI_BIAS_BYTES) + 8u * (2 * STAGES + 4));
+      reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * (SINGLE_EPI_BYTES + EPI_BIAS_BYTES) + 8u * (2 * STAGES + 4));
   volatile int* tile_ring =
-      reinterpret_cast<volatile int*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * (EPI_STAGE_BYTES + EPI_BIAS_BYTES) + 8u * (2 * STAGES + 14));
+      reinterpret_cast<volatile int*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * (SINGLE_EPI_BYTES + EPI_BIAS_BYTES) + 8u * (2 * STAGES + 14));
   const uint32_t tmem_slot = bar_base + 8u * (2 * STAGES + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -401,9 +408,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int q = warp & 3;                       // TMEM lane quarter this warp may read
     const int cbeg = (ew / 4) * CPW;              // first tile column of this warp
     const bool active = cbeg < BN;                // BN = 64: only one warp per quarter has columns
-    const uint32_t stage0 = epi_base + ew * EPI_STAGE_BYTES;   // two 4 KB buffers, used alternately
+    const uint32_t stage0 = epi_base + ew * SINGLE_EPI_BYTES;   // two 4 KB buffers, used alternately
     uint32_t sbuf = 0;
-    float* bias_s = reinterpret_cast<float*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * EPI_STAGE_BYTES + ew * EPI_BIAS_BYTES);
+    float* bias_s = reinterpret_cast<float*>(gen_base + STAGES * STAGE_BYTES + EPI_WARPS * SINGLE_EPI_BYTES + ew * EPI_BIAS_BYTES);
     const bool out_f32 = p.splits > 1 || p.c_f32;
     bool store_pending = false;                   // lane 0: TMA stores may still be reading the staging buffers
     uint32_t lt = 0;
@@ -482,8 +489,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               for (int j = 0; j < 32; j++) r[j] = 0u;
             }
             if (via_tma && (f32 || (cc & 63) == 0)) { // next staging buffer: its previous store (two stores ago) must have read it
-              sbuf ^= 1;
-              if (lane == 0 && store_pending) tma_store_wait_read1();
+              if (SINGLE_EPI_BUFS == 2) {
+                sbuf ^= 1;
+                if (lane == 0 && store_pending) tma_store_wait_read1();
+              } else if (lane == 0 && store_pending) {
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+              }
               __syncwarp();
             }
             const uint32_t stage = stage0 + sbuf * 4096;
@@ -1690,7 +1701,7 @@ bool encode_2d(void* out, const void* base, long long inner, long long outer, lo
 template <int BN, bool A_MN, bool B_MN, bool GENERAL, bool CE = false>
 cudaError_t launch_t(const GemmArgs& g, const TcPlan& plan, cudaStream_t s, int max_ctas) {
   constexpr int STAGES = stages_for(BN);
-  constexpr size_t smem = (size_t)STAGES * (BM * BK * 2 + BN * BK * 2) + EPI_WARPS * (EPI_STAGE_BYTES + EPI_BIAS_BYTES) + 8 * (2 * STAGES + 16) + 1024;
+  constexpr size_t smem = (size_t)STAGES * (BM * BK * 2 + BN * BK * 2) + EPI_WARPS * (SINGLE_EPI_BYTES + EPI_BIAS_BYTES) + 8 * (2 * STAGES + 16) + 1024;
   static std::atomic<bool> attr_set[MAX_DEVICES];
   if (cudaError_t e = ensure_smem(tc_gemm_kernel<BN, A_MN, B_MN, GENERAL, CE>, smem, attr_set)) return e;
   TcArgs p;
