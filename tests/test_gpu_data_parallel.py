@@ -25,17 +25,19 @@ def _shard(spec, batch, r, world):
     return {k: v[r * per:(r + 1) * per] for k, v in batch.items()}
 
 
-@pytest.mark.parametrize("name", ["mlp_f32", "ctr_f32", "lm_f32"])
+@pytest.mark.parametrize("name", ["mlp_f32", "ctr_f32", "lm_f32", "lm_bf16"])
 def test_shares_of_two_shards_add_up_to_the_oracle_on_the_union_batch(name):
     gu = _gu()
     full = {"mlp_f32": synth.mlp_spec(64, 128, 3, 96, "gelu", "f32"),
             "ctr_f32": synth.ctr_spec(batch=64, table_rows=50, tower=(64, 32, 16), dtype="f32"),
-            "lm_f32": synth.lm_spec(2, 64, 2, 128, 24, 4, 96, dtype="f32")}[name]
+            "lm_f32": synth.lm_spec(2, 64, 2, 128, 24, 4, 96, dtype="f32"),
+            "lm_bf16": synth.lm_spec(2, 128, 2, 256, 64, 8, 512)}[name]      # the softmax head fused into its GEMM
+    tol = gu.TOL[full["dtype"]]
     world = 2
     local = dict(full, batch=full["batch"] // world, replicas=world)
     flat = synth.init_params(full, 3)
     batch = synth.make_batch(full, 3)
-    want_l, want_g = orc.forward_backward(full, util.structure(full, flat), batch)
+    want_l, want_g = orc.forward_backward(full, util.operand_params(full, util.structure(full, flat)), util.operand_batch(full, batch))
     tl = synth.tensor_list(full)
     tidx = util.trainable_index(full)
     m = gu.new_model(local, flat)
@@ -53,10 +55,10 @@ def test_shares_of_two_shards_add_up_to_the_oracle_on_the_union_batch(name):
             for i in tidx:
                 grads[i] = grads[i] + m.grads(i).astype(np.float64)
             assert m.comm_order() == []                       # nothing was exchanged
-        np.testing.assert_allclose(loss, want_l, rtol=1e-4)
+        np.testing.assert_allclose(loss, want_l, rtol=tol)
         for i in tidx:
             b, tname, _s, _t = tl[i]
-            assert synth.rel_l2(grads[i], want_g[b][tname]) <= 1e-4, (b, tname)
+            assert synth.rel_l2(grads[i], want_g[b][tname]) <= tol, (b, tname)
     finally:
         m.close()
 
