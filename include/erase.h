@@ -286,12 +286,12 @@ ERASE_API erase_status erase_selftest_timeout(erase_model* m, int32_t limit_us);
  *
  * erase_comm_unique_id: fills 128 HOST bytes with a fresh NCCL id; call on one replica and carry the
  *   bytes to the others by any means (a file, a socket, torch.distributed).
- * erase_comm_init: collective over the replicas (blocks until all have called it, as
- *   ncclCommInitRank does); the current CUDA device must be the model's.  world must equal the
+ * erase_comm_init: id = those 128 bytes (HOST).  Collective over the replicas (blocks until all have called
+ *   it, as ncclCommInitRank does); the current CUDA device must be the model's.  world must equal the
  *   spec's replicas (1 is allowed: a communicator of one, the exchange then changes nothing).  The
  *   communicator lives until erase_destroy.
  * erase_comm_order: the block index of every exchange the last step enqueued, in enqueue order
- *   (-1 stands for the losses), at most cap entries; *n_out = their number.  Serial schedule:
+ *   (-1 stands for the losses), at most cap entries into blocks_out (HOST); *n_out = their number.  Serial schedule:
  *   B-1, .., 0, -1; ERASE: 0, .., B-1, -1.
  * NCCL is loaded when first needed ("libnccl.so.2", or the file the environment variable
  * ERASE_NCCL_LIB names).  A replica that stops stepping leaves the others waiting inside NCCL: the
