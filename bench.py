@@ -38,7 +38,7 @@ MIN_LEG_S = 1.0     # every leg is repeated (K steps per repeat) until this much
 # of each kernel class (summaries under profiles/).  They sit below the algorithmic bytes where an
 # operand or result is still L2-resident.
 NCU_DRAM_BYTES = {"C2": {"gemm_fwd": 15.5e6, "gemm_dgrad": 75.4e6, "gemm_wgrad": 71.4e6},
-                  "C4": {"gemm_fwd": 567.6e6, "gemm_dgrad": 712.0e6, "gemm_wgrad": 736.8e6}}
+                  "C4": {"gemm_fwd": 565.4e6, "gemm_dgrad": 710.9e6, "gemm_wgrad": 736.5e6}}
 
 # the per-config table of the default run: (label, config name, keyword arguments)
 TABLE = [("C1", "C1", {}), ("C2", "C2", {}), ("C3", "C3", {}),
