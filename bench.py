@@ -414,6 +414,11 @@ NCU_DRAM_NOTE = {"C2": "ncu DRAM bytes of the class's largest GEMM (local head),
                        "one full-size launch: profiles/tc_gemm_c4_head_ce_fwd_wgrad_dgrad.md"}
 
 
+# --sweep: the whole saturation sweep (C5: five widths x three batch sizes) instead of the default table's five points
+SWEEP = [("C1", "C1", {}), ("C2", "C2", {}), ("C3", "C3", {})] + [
+    (f"C5 w{w} b{b}", "C5", {"w": w, "batch": b}) for w in (128, 512, 1024, 2048, 4096) for b in (512, 4096, 32768)]
+
+
 def table_entry(torch, binding, rep, label, cfg, kw, args, peaks):
     """Serial and ERASE throughput, gain, MFU and dominant kernel class of one parity-table config."""
     spec = synth.config(cfg, **kw)
@@ -533,7 +538,7 @@ def run_gpu(args, spec, cfg_name):
     table = None
     if world == 1 and not args.no_table:
         table = []
-        for label, cfg, kw in TABLE:
+        for label, cfg, kw in (SWEEP if args.sweep else TABLE):
             try:
                 table.append(table_entry(torch, binding, rep, label, cfg, kw, args, peaks))
             except Exception as e:      # one config failing must not lose the headline line
@@ -622,6 +627,8 @@ def main():
     ap.add_argument("--loss-on-main", action="store_true", help="paper's placement of the local loss")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-table", action="store_true", help="skip the per-config table (C1, C2, C3, five C5 points)")
+    ap.add_argument("--sweep", action="store_true",
+                    help="per-config table over the whole C5 sweep (15 points, several minutes) instead of five of its points")
     ap.add_argument("--no-par-fwd", action="store_true",
                     help="parallel topology: keep the blocks' forwards on the main stream, one after the other")
     ap.add_argument("--no-split-bwd", action="store_true",
