@@ -18,14 +18,20 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// One try_wait may keep the thread suspended for up to this long before it reports "not yet" (it returns at
+// once when the phase completes).  Without the hint the hardware's own, much shorter limit applies and the
+// ~300 waiting threads of a GEMM CTA wake up and poll again far more often; on a power-capped step that
+// polling costs clock: C4 23.6 -> 23.35 ms per step with the hint, both schedules.  The bounded waits check
+// their clock between two try_waits, so a limit is overrun by at most this much.
+constexpr uint32_t TRY_WAIT_SUSPEND_NS = 100000u;
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(TRY_WAIT_SUSPEND_NS)
       : "memory");
   return ok != 0;
 }
